@@ -1,0 +1,287 @@
+"""Plan oracle: exhaustive parenthesization of a Linnea Mul chain.  TEST INFRASTRUCTURE ONLY.
+
+This file is the slow, plainly-correct statement of what the planner must return.  It shares no
+code with the CUDA library and must never be imported by the product path; only tests, the smoke
+check and the benchmark's CPU-baseline leg use it.
+
+What it follows (paper Section 2):
+  * "Types": a Matrix is (property, static [rows, cols], element type); Identity is a square matrix
+    with ones on the diagonal, there so that A*I = A and I*I = I can be expressed.
+  * "Transformations": identity simplification (A*I -> A), matrix-chain reordering that "minimizes
+    the number of scalar multiplications", generalised to account for matrix properties, and
+    property propagation that turns the equation's Term into a concrete Matrix type.
+
+The chain-reordering transformation is a dynamic program that reaches the minimum-cost binary tree;
+the plain definition of that result is "the cheapest of ALL binary trees", so the oracle enumerates
+every tree (Catalan many) and keeps the cheapest.
+
+Readings taken where the paper is silent (each also listed in the design notes):
+  * cost of one product = number of scalar multiplications a_il * b_lj in which BOTH factors are
+    structurally non-zero (non-strict triangles: the diagonal is an ordinary entry);
+  * Identity operands are removed before the enumeration and never appear in the result string;
+  * ties: the tree whose pre-order list of split positions is lexicographically smallest;
+  * property of a product = join in  Identity < {lowerTri, upperTri} < general;
+  * reported mul_flops = 2 * multiplications; add_flops = structural non-zeros of the Add terms.
+    (The factor 2 and the add_flops convention are bookkeeping of this project: parity unpinned by
+    the paper, which only speaks of scalar multiplications.)
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass
+from typing import List, Optional, Sequence, Tuple
+
+GENERAL, LOWER_TRI, UPPER_TRI, IDENTITY = 0, 1, 2, 3
+
+
+class OracleError(ValueError):
+    """Raised with a short reason code: 'invalid_arg', 'property', 'shape_mismatch'."""
+
+    def __init__(self, code: str, msg: str = ""):
+        super().__init__(f"{code}: {msg}" if msg else code)
+        self.code = code
+
+
+@dataclass(frozen=True)
+class Desc:
+    rows: int
+    cols: int
+    prop: int
+
+
+@dataclass(frozen=True)
+class Step:
+    lhs: int          # ids: 0..n-1 original chain operands, n.. intermediates in emission order
+    rhs: int
+    out: int
+    m: int
+    n: int
+    k: int
+    lhs_prop: int
+    rhs_prop: int
+    out_prop: int
+    mults: int
+
+
+@dataclass(frozen=True)
+class Plan:
+    paren: str
+    mults: int
+    mul_flops: int
+    add_flops: int
+    steps: Tuple[Step, ...]
+    product_desc: Desc     # the Mul chain's value before the Add terms
+    result_desc: Desc      # the equation's Term made concrete
+    kept: Tuple[int, ...]  # original indices that survive identity simplification
+
+
+# ----------------------------------------------------------------------------------------------
+# structure and cost of one product
+# ----------------------------------------------------------------------------------------------
+
+def in_structure(prop: int, i: int, j: int) -> bool:
+    """Is entry (i, j) a structural non-zero of a matrix with this property?"""
+    if prop == GENERAL:
+        return True
+    if prop == LOWER_TRI:
+        return i >= j
+    if prop == UPPER_TRI:
+        return i <= j
+    if prop == IDENTITY:
+        return i == j
+    raise OracleError("property", f"unknown property {prop}")
+
+
+def brute_force_nonzeros(d: Desc) -> int:
+    """Structural non-zeros by counting (tiny shapes; used to check `structural_nonzeros`)."""
+    return sum(1 for i in range(d.rows) for j in range(d.cols) if in_structure(d.prop, i, j))
+
+
+def structural_nonzeros(d: Desc) -> int:
+    if d.prop == GENERAL:
+        return d.rows * d.cols
+    if d.prop in (LOWER_TRI, UPPER_TRI):
+        return d.rows * (d.rows + 1) // 2
+    return d.rows
+
+
+def brute_force_mults(a: Desc, b: Desc) -> int:
+    """#{(i, l, j): (i, l) in S(A) and (l, j) in S(B)} by counting, for tiny shapes."""
+    assert a.cols == b.rows
+    count = 0
+    for i in range(a.rows):
+        for l in range(a.cols):
+            if not in_structure(a.prop, i, l):
+                continue
+            for j in range(b.cols):
+                if in_structure(b.prop, l, j):
+                    count += 1
+    return count
+
+
+def product_mults(a: Desc, b: Desc) -> int:
+    """Useful scalar multiplications of A*B in closed form (both operands non-Identity)."""
+    assert a.cols == b.rows
+    ta = a.prop in (LOWER_TRI, UPPER_TRI)
+    tb = b.prop in (LOWER_TRI, UPPER_TRI)
+    if a.prop == IDENTITY or b.prop == IDENTITY:
+        return 0
+    if not ta and not tb:
+        return a.rows * a.cols * b.cols
+    if ta and not tb:
+        n = a.rows
+        return b.cols * n * (n + 1) // 2
+    if tb and not ta:
+        n = b.rows
+        return a.rows * n * (n + 1) // 2
+    n = a.rows
+    if a.prop == b.prop:           # L*L or U*U: sum over l of (#rows below l) * (#cols left of l) ...
+        return n * (n + 1) * (n + 2) // 6
+    return n * (n + 1) * (2 * n + 1) // 6   # L*U, U*L: sum of squares
+
+
+def join(p: int, q: int) -> int:
+    """Property of a product: least upper bound in Identity < {lowerTri, upperTri} < general."""
+    if p == IDENTITY:
+        return q
+    if q == IDENTITY:
+        return p
+    if p == q:
+        return p
+    return GENERAL
+
+
+def sum_property(product_prop: int, add_props: Sequence[int]) -> int:
+    """Property of (chain value) + T1 + ... + Tk.  With no terms it is the product's own property.
+
+    A sum with at least one term is never typed Identity (I + I = 2I): an Identity summand counts
+    through its footprint, which fits either triangle.  All-Identity sums are reported lowerTri.
+    """
+    if not add_props:
+        return product_prop
+    props = [product_prop] + list(add_props)
+    concrete = [p for p in props if p != IDENTITY]
+    if not concrete:
+        return LOWER_TRI
+    out = concrete[0]
+    for p in concrete[1:]:
+        out = p if p == out else GENERAL
+    return out
+
+
+# ----------------------------------------------------------------------------------------------
+# validation and identity simplification
+# ----------------------------------------------------------------------------------------------
+
+def _validate(chain: Sequence[Desc], add: Sequence[Desc]) -> None:
+    if len(chain) < 1:
+        raise OracleError("invalid_arg", "empty chain")
+    for d in list(chain) + list(add):
+        if d.rows < 1 or d.cols < 1:
+            raise OracleError("invalid_arg", "non-positive dimension")
+        if d.prop not in (GENERAL, LOWER_TRI, UPPER_TRI, IDENTITY):
+            raise OracleError("property", "unknown property")
+        if d.prop != GENERAL and d.rows != d.cols:
+            raise OracleError("property", "triangular / Identity matrices are square")
+    for a, b in zip(chain[:-1], chain[1:]):
+        if a.cols != b.rows:
+            raise OracleError("shape_mismatch", "inner dimensions differ")
+    rows, cols = chain[0].rows, chain[-1].cols
+    for t in add:
+        if (t.rows, t.cols) != (rows, cols):
+            raise OracleError("shape_mismatch", "Add term shape differs from the chain's")
+
+
+# ----------------------------------------------------------------------------------------------
+# exhaustive enumeration
+# ----------------------------------------------------------------------------------------------
+
+# A tree over reduced positions lo..hi is either the int `lo` (a leaf, lo == hi) or (split, left, right)
+# where left covers lo..split and right covers split+1..hi.
+
+def all_trees(lo: int, hi: int):
+    if lo == hi:
+        yield lo
+        return
+    for split in range(lo, hi):
+        for left in all_trees(lo, split):
+            for right in all_trees(split + 1, hi):
+                yield (split, left, right)
+
+
+def _tree_desc_cost(tree, descs: Sequence[Desc]) -> Tuple[Desc, int]:
+    if isinstance(tree, int):
+        return descs[tree], 0
+    _, left, right = tree
+    dl, cl = _tree_desc_cost(left, descs)
+    dr, cr = _tree_desc_cost(right, descs)
+    node = Desc(dl.rows, dr.cols, join(dl.prop, dr.prop))
+    return node, cl + cr + product_mults(dl, dr)
+
+
+def _preorder_splits(tree) -> List[int]:
+    if isinstance(tree, int):
+        return []
+    split, left, right = tree
+    return [split] + _preorder_splits(left) + _preorder_splits(right)
+
+
+def _paren(tree, kept: Sequence[int]) -> str:
+    if isinstance(tree, int):
+        return str(kept[tree])
+    _, left, right = tree
+    return "(" + _paren(left, kept) + "*" + _paren(right, kept) + ")"
+
+
+def plan(chain: Sequence[Tuple[int, int, int]], add: Sequence[Tuple[int, int, int]] = ()) -> Plan:
+    """Plan `X = prod(chain) + sum(add)`; operands are (rows, cols, property) triples."""
+    cdescs = [Desc(*c) for c in chain]
+    adescs = [Desc(*a) for a in add]
+    _validate(cdescs, adescs)
+    n = len(cdescs)
+    rows, cols = cdescs[0].rows, cdescs[-1].cols
+
+    kept = tuple(i for i, d in enumerate(cdescs) if d.prop != IDENTITY)
+    add_flops = sum(structural_nonzeros(t) for t in adescs)
+
+    if not kept:     # I*I*...*I = I
+        product = Desc(rows, cols, IDENTITY)
+        return Plan("I", 0, 0, add_flops, (), product,
+                    Desc(rows, cols, sum_property(IDENTITY, [t.prop for t in adescs])), kept)
+
+    reduced = [cdescs[i] for i in kept]
+    best = None
+    for tree in all_trees(0, len(reduced) - 1):
+        _, cost = _tree_desc_cost(tree, reduced)
+        key = (cost, _preorder_splits(tree))
+        if best is None or key < best[0]:
+            best = (key, tree)
+    (cost, _), tree = best
+
+    steps: List[Step] = []
+    next_id = [n]
+
+    def emit(t) -> Tuple[int, Desc]:
+        if isinstance(t, int):
+            return kept[t], reduced[t]
+        _, left, right = t
+        lid, ld = emit(left)
+        rid, rd = emit(right)
+        out = Desc(ld.rows, rd.cols, join(ld.prop, rd.prop))
+        oid = next_id[0]
+        next_id[0] += 1
+        steps.append(Step(lid, rid, oid, ld.rows, rd.cols, ld.cols, ld.prop, rd.prop, out.prop,
+                          product_mults(ld, rd)))
+        return oid, out
+
+    _, product = emit(tree)
+    assert sum(s.mults for s in steps) == cost
+    result = Desc(rows, cols, sum_property(product.prop, [t.prop for t in adescs]))
+    return Plan(_paren(tree, kept), cost, 2 * cost, add_flops, tuple(steps), product, result, kept)
+
+
+def catalan(r: int) -> int:
+    """Number of binary trees over r leaves (r >= 1)."""
+    c = 1
+    for i in range(r - 1):
+        c = c * 2 * (2 * i + 1) // (i + 2)
+    return c

@@ -1,0 +1,205 @@
+"""Seeded synthetic Linnea equations: shapes, properties and random entries.
+
+This module is shared by the CPU oracle's tests, the GPU parity tests and the
+benchmark.  It only *describes* equations and draws their entries; it holds no
+planning and no product arithmetic, so neither implementation can inherit the
+other's mistakes through it.
+
+An equation is ``X = M1 * M2 * ... * Mn + T1 + ... + Tk`` (paper Section 2,
+"Operations": variadic Mul and Add inside an Equation).  Every matrix carries
+one compile-time property (paper Section 2, "Matrix Attribute" and "Types").
+
+Storage convention for generated data (paper Section 2: the property dictates
+how the dense buffer is filled): dense row-major float32; entries outside a
+triangular operand's structure are ``+0.0``; Identity operands are never
+materialised (``None``).
+
+Random stream: NumPy's Philox counter-based generator keyed by
+``(seed, operand index)``; operand indices count the chain first, then the
+Add terms.  The same key always yields the same matrix.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass, field, replace
+from typing import List, Optional, Sequence
+
+import numpy as np
+
+GENERAL, LOWER_TRI, UPPER_TRI, IDENTITY = 0, 1, 2, 3
+PROPERTY_NAMES = {GENERAL: "general", LOWER_TRI: "lowerTri", UPPER_TRI: "upperTri", IDENTITY: "Identity"}
+
+
+@dataclass(frozen=True)
+class Operand:
+    """One matrix of an equation: static shape, property and entry distribution.
+
+    dist: "uniform"  -> U(-1, 1)
+          "normal"   -> N(0, sigma^2)
+          "ones"     -> every structural entry 1 (the paper's Listing 2 fill)
+    Triangular operands always use: strict part from `dist`, diagonal 1 + U(0, 1)
+    (except dist == "ones"), other half exactly zero.
+    """
+    rows: int
+    cols: int
+    prop: int = GENERAL
+    dist: str = "uniform"
+    sigma: float = 1.0
+
+
+@dataclass(frozen=True)
+class Equation:
+    name: str
+    seed: int
+    chain: Sequence[Operand]
+    add: Sequence[Operand] = field(default_factory=tuple)
+    batch: int = 1  # > 1: `batch` independent instances sharing one plan
+
+    def descs(self):
+        return [(o.rows, o.cols, o.prop) for o in self.chain]
+
+    def add_descs(self):
+        return [(o.rows, o.cols, o.prop) for o in self.add]
+
+
+def _draw(rng: np.random.Generator, shape, dist: str, sigma: float) -> np.ndarray:
+    if dist == "uniform":
+        return (rng.random(shape, dtype=np.float32) * np.float32(2.0) - np.float32(1.0)).astype(np.float32)
+    if dist == "normal":
+        return (rng.standard_normal(shape, dtype=np.float32) * np.float32(sigma)).astype(np.float32)
+    if dist == "ones":
+        return np.ones(shape, dtype=np.float32)
+    raise ValueError(f"unknown distribution {dist!r}")
+
+
+def generate_operand(op: Operand, seed: int, index: int, batch: int = 1) -> Optional[np.ndarray]:
+    """Dense float32 array for one operand; shape (rows, cols), or (batch, rows, cols) if batch > 1.
+
+    Returns None for Identity (it is a type, not data).
+    """
+    if op.prop == IDENTITY:
+        return None
+    rng = np.random.Generator(np.random.Philox(key=[int(seed), int(index)]))
+    shape = (batch, op.rows, op.cols) if batch > 1 else (op.rows, op.cols)
+    m = _draw(rng, shape, op.dist, op.sigma)
+    if op.prop in (LOWER_TRI, UPPER_TRI):
+        if op.rows != op.cols:
+            raise ValueError("triangular operands are square")
+        n = op.rows
+        if op.dist != "ones":
+            diag = np.float32(1.0) + rng.random(shape[:-1], dtype=np.float32)
+            idx = np.arange(n)
+            m[..., idx, idx] = diag
+        keep = np.tril(np.ones((n, n), dtype=bool)) if op.prop == LOWER_TRI else np.triu(np.ones((n, n), dtype=bool))
+        m = np.where(keep, m, np.float32(0.0)).astype(np.float32)
+    return np.ascontiguousarray(m, dtype=np.float32)
+
+
+def generate(eq: Equation):
+    """(chain arrays, add-term arrays); Identity entries are None."""
+    chain = [generate_operand(o, eq.seed, i, eq.batch) for i, o in enumerate(eq.chain)]
+    add = [generate_operand(o, eq.seed, len(eq.chain) + i, eq.batch) for i, o in enumerate(eq.add)]
+    return chain, add
+
+
+# --------------------------------------------------------------------------
+# The benchmark's configurations (shapes, properties, distributions, seeds).
+# --------------------------------------------------------------------------
+
+def config_tiny(seed: int = 0) -> Equation:
+    """X = L*A*B: L 64x64 lowerTri, A 64x32, B 32x48, U(-1,1)."""
+    return Equation("tiny_LAB", seed, (
+        Operand(64, 64, LOWER_TRI), Operand(64, 32), Operand(32, 48)))
+
+
+def config_tiny_identity_left(seed: int = 0) -> Equation:
+    """X = I*L (the product must vanish from the plan)."""
+    return Equation("tiny_IL", seed, (Operand(64, 64, IDENTITY), Operand(64, 64, LOWER_TRI)))
+
+
+def config_tiny_identity_right(seed: int = 0) -> Equation:
+    """X = L*I."""
+    return Equation("tiny_LI", seed, (Operand(64, 64, LOWER_TRI), Operand(64, 64, IDENTITY)))
+
+
+def config_five_general(seed: int = 1) -> Equation:
+    """Five general matrices whose parenthesization dominates the cost; N(0,1)."""
+    dims = [1024, 256, 2048, 64, 1024, 512]
+    return Equation("five_general", seed, tuple(
+        Operand(dims[i], dims[i + 1], GENERAL, "normal") for i in range(5)))
+
+
+def config_property_heavy(n: int = 4096, seed: int = 2) -> Equation:
+    """X = L*U*I*B + C, all n x n; the Identity between U and B is to be eliminated."""
+    return Equation(f"LUIB_plus_C_{n}", seed, (
+        Operand(n, n, LOWER_TRI), Operand(n, n, UPPER_TRI), Operand(n, n, IDENTITY),
+        Operand(n, n, GENERAL, "normal")), (Operand(n, n, GENERAL, "normal"),))
+
+
+def config_large_square(n: int = 8192, seed: int = 3) -> Equation:
+    """X = L*A*U*B, all n x n; A, B ~ N(0, 1/n) so that magnitudes stay O(1)."""
+    s = float(n) ** -0.5
+    return Equation(f"LAUB_{n}", seed, (
+        Operand(n, n, LOWER_TRI), Operand(n, n, GENERAL, "normal", s),
+        Operand(n, n, UPPER_TRI), Operand(n, n, GENERAL, "normal", s)))
+
+
+def config_batched(batch: int = 4096, seed: int = 4) -> Equation:
+    """`batch` instances of X_i = L_i*A_i*B_i + C_i (64x64, 64x64, 64x16, 64x16), U(-1,1)."""
+    return Equation(f"batched_LAB_plus_C_x{batch}", seed, (
+        Operand(64, 64, LOWER_TRI), Operand(64, 64), Operand(64, 16)), (Operand(64, 16),), batch=batch)
+
+
+def config_paper_chain(seed: int = 5) -> Equation:
+    """The chain of the paper's Section 4: 800x1100, 1100x900, 900x1200, 1200x100; N(0,1)."""
+    dims = [800, 1100, 900, 1200, 100]
+    return Equation("paper_section4_chain", seed, tuple(
+        Operand(dims[i], dims[i + 1], GENERAL, "normal") for i in range(4)))
+
+
+def config_listing2() -> Equation:
+    """Listing 2 of the paper: two 5x5 lowerTri matrices filled with the constant 1."""
+    return Equation("listing2_LL_5", 0, (
+        Operand(5, 5, LOWER_TRI, "ones"), Operand(5, 5, LOWER_TRI, "ones")))
+
+
+def random_equation(seed: int, max_len: int = 6, max_dim: int = 96, allow_add: bool = True,
+                    dim_multiple: int = 1) -> Equation:
+    """A random well-formed equation (for property tests): random length, dims, properties.
+
+    Triangular / Identity operands are only placed where the neighbouring dimensions are equal,
+    which the generator arranges by repeating a dimension.
+    """
+    rng = np.random.Generator(np.random.Philox(key=[int(seed), 0xC0FFEE]))
+    n = int(rng.integers(1, max_len + 1))
+    chain: List[Operand] = []
+    cur = int(rng.integers(1, max_dim // dim_multiple + 1)) * dim_multiple
+    for _ in range(n):
+        kind = int(rng.integers(0, 6))
+        if kind == 0:
+            chain.append(Operand(cur, cur, LOWER_TRI))
+        elif kind == 1:
+            chain.append(Operand(cur, cur, UPPER_TRI))
+        elif kind == 2:
+            chain.append(Operand(cur, cur, IDENTITY))
+        else:
+            nxt = int(rng.integers(1, max_dim // dim_multiple + 1)) * dim_multiple
+            chain.append(Operand(cur, nxt, GENERAL, "normal" if kind == 3 else "uniform"))
+            cur = nxt
+    rows, cols = chain[0].rows, chain[-1].cols
+    add: List[Operand] = []
+    if allow_add:
+        for _ in range(int(rng.integers(0, 3))):
+            kind = int(rng.integers(0, 5))
+            if rows == cols and kind == 0:
+                add.append(Operand(rows, cols, LOWER_TRI))
+            elif rows == cols and kind == 1:
+                add.append(Operand(rows, cols, UPPER_TRI))
+            elif rows == cols and kind == 2:
+                add.append(Operand(rows, cols, IDENTITY))
+            else:
+                add.append(Operand(rows, cols, GENERAL))
+    return Equation(f"random_{seed}", seed, tuple(chain), tuple(add))
+
+
+def with_batch(eq: Equation, batch: int) -> Equation:
+    return replace(eq, batch=batch, name=f"{eq.name}_x{batch}")
