@@ -1,0 +1,395 @@
+#!/usr/bin/env python
+"""Benchmark: useful GFLOP/s of one Linnea equation on B200 and its fraction of the 3xTF32 roofline.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--variant 3xtf32|ffma] [--impl reference]
+
+A step is one evaluation of the whole equation (every product of the plan plus the fused Add /
+zero-fill epilogue) on seeded synthetic operands.  The headline workload is the large square chain
+X = L*A*U*B at 8192 (operands far larger than L2, so no flush is needed between steps).  The other
+configurations are timed briefly and reported under "all_configs".  One JSON line is printed by rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import workloads as wl  # noqa: E402
+
+METRIC = "useful GFLOP/s per Linnea equation (f32)"
+UNIT = "GFLOP/s"
+TF32_OVER_BF16 = 1.1 / 2.25          # nominal dense tensor ratio used to carry the measured bf16 peak to tf32
+
+
+def headline_equation() -> wl.Equation:
+    return wl.config_large_square()
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as fh:
+            d = json.load(fh)
+        return {"hbm_gbs": d["hbm_gbs"], "bf16_burst": d["bf16_tflops"], "bf16_sustained": d["bf16_tflops_sustained"],
+                "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_burst": 1590.0, "bf16_sustained": 1400.0, "source": "fallback"}
+
+
+# ------------------------------------------------------------------------------------------------
+# reference arm / CPU baseline: the oracle, as it stands, on the host cores
+# ------------------------------------------------------------------------------------------------
+
+def oracle_sample_seconds(eq, chain, add, rows):
+    """Time the oracle on `rows` of X (left-to-right fp64 triple loops); returns (seconds, threads used)."""
+    from oracle import values as ov
+    t0 = time.perf_counter()
+    ov.evaluate([None if c is None else (c[0] if eq.batch > 1 else c) for c in chain], eq.descs(),
+                [None if a is None else (a[0] if eq.batch > 1 else a) for a in add], eq.add_descs(), rows=rows)
+    return time.perf_counter() - t0, ov.threads_used()
+
+
+def cpu_baseline(eq, chain, add, useful_flops_per_instance, n_rows):
+    from oracle import plan as op
+    t0 = time.perf_counter()
+    op.plan(eq.descs(), eq.add_descs())
+    plan_s = time.perf_counter() - t0
+    total_rows = eq.chain[0].rows
+    rows = np.sort(np.random.default_rng(0).choice(total_rows, size=min(n_rows, total_rows), replace=False))
+    secs, threads = oracle_sample_seconds(eq, chain, add, rows)
+    frac = len(rows) / total_rows
+    value = useful_flops_per_instance * frac / (secs + plan_s) / 1e9
+    return {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle",
+            "sample": f"{len(rows)} of {total_rows} rows of X (one instance), exhaustive plan + left-to-right fp64 "
+                      f"triple loops incl. the error denominator; useful FLOPs scaled by the row fraction; "
+                      f"{secs + plan_s:.2f} s"}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import plan as op
+    eq = headline_equation()
+    chain, add = wl.generate(eq)
+    p = op.plan(eq.descs(), eq.add_descs())
+    useful = p.mul_flops + p.add_flops
+    n_rows = 4
+    total_rows = eq.chain[0].rows
+    times = []
+    threads = 1
+    for i in range(args.warmup + args.steps):
+        rows = np.sort(np.random.default_rng(i).choice(total_rows, size=n_rows, replace=False))
+        secs, threads = oracle_sample_seconds(eq, chain, add, rows)
+        if i >= args.warmup:
+            times.append(secs)
+    mean_s = sum(times) / len(times)
+    value = useful * (n_rows / total_rows) / mean_s / 1e9
+    sample = f"{n_rows} of {total_rows} rows of X per step, left-to-right fp64 triple loops incl. the error denominator"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": mean_s * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": eq.name, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+# ------------------------------------------------------------------------------------------------
+# GPU arm
+# ------------------------------------------------------------------------------------------------
+
+class ClockSampler:
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+             "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, device_index: int):
+        self.proc = None
+        self.device_index = device_index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
+                                          "-lms", "100", "-i", str(self.device_index)],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, mx, power, reasons = [], [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.strip().splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); mx.append(float(f[2])); power.append(float(f[3]))
+            except ValueError:
+                continue
+            for name, val in zip(names, f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "power_w_max": max(power) if power else None, "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def time_equation(mom, torch, eq, variant, steps, warmup, stream, timing=False):
+    """Device-resident timing of one configuration: returns dict with per-step ms list, plan, launches."""
+    chain, add = wl.generate(eq)
+    plan = mom.mom_equation_plan(eq.descs(), eq.add_descs(), variant)
+    rd = plan.result_desc()
+    dchain = [None if a is None else torch.from_numpy(a).cuda() for a in chain]
+    dadd = [None if a is None else torch.from_numpy(a).cuda() for a in add]
+    out = torch.empty((eq.batch, rd.rows, rd.cols), dtype=torch.float32, device="cuda")
+    wsb = plan.workspace_bytes(eq.batch)
+    ws = torch.empty(max(wsb, 256), dtype=torch.uint8, device="cuda")
+    cp = [None if t is None else t.data_ptr() for t in dchain]
+    ap = [None if t is None else t.data_ptr() for t in dadd]
+    cs = [0 if t is None else t[0].numel() for t in dchain] if eq.batch > 1 else None
+    as_ = [0 if t is None else t[0].numel() for t in dadd] if eq.batch > 1 else None
+
+    def run():
+        if eq.batch > 1:
+            plan.execute_batched(cp, cs, ap, as_, out.data_ptr(), rd.rows * rd.cols, eq.batch,
+                                 ws.data_ptr() if wsb else None, wsb, stream.cuda_stream)
+        else:
+            plan.execute(cp, ap, out.data_ptr(), ws.data_ptr() if wsb else None, wsb, stream.cuda_stream)
+
+    if timing:
+        plan.enable_step_timing(True)
+    with torch.cuda.stream(stream):
+        for _ in range(warmup):
+            run()
+        stream.synchronize()
+        events = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+        step_times = []
+        for e0, e1 in events:
+            e0.record(stream)
+            run()
+            e1.record(stream)
+            if timing:
+                stream.synchronize()
+                step_times.append([plan.step_times(i) for i in range(plan.num_steps())])
+        stream.synchronize()
+    ms = [e0.elapsed_time(e1) for e0, e1 in events]
+    status = plan.device_status()
+    if status != (0, 0):
+        raise RuntimeError(f"device-side wait timed out: {status}")
+    mul, addf = plan.flops()
+    return {"ms": ms, "plan": plan, "useful_flops": (mul + addf) * eq.batch, "launches": plan.last_launch_count(),
+            "step_times": step_times, "host": (chain, add), "keep": (dchain, dadd, out, ws)}
+
+
+def run_gpu(args):
+    import torch
+    import torch.distributed as dist
+    import paper_2208_10391_b200 as mom
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback); use --impl reference for the oracle")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    variant = {"3xtf32": mom.VARIANT_3XTF32, "ffma": mom.VARIANT_FFMA}[args.variant]
+    stream = torch.cuda.Stream()
+    peaks = measured_peaks()
+
+    eq = headline_equation()
+    sampler = ClockSampler(local)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- headline: device-resident, K timed steps bracketed by barriers; every rank runs its own replica
+    barrier()
+    warm = time_equation(mom, torch, eq, variant, steps=1, warmup=max(args.warmup - 1, 0), stream=stream)
+    plan = warm["plan"]
+    del warm
+    torch.cuda.empty_cache()
+    chain, add = wl.generate(eq)
+    dchain = [None if a is None else torch.from_numpy(a).cuda() for a in chain]
+    dadd = [None if a is None else torch.from_numpy(a).cuda() for a in add]
+    rd = plan.result_desc()
+    out = torch.empty((rd.rows, rd.cols), dtype=torch.float32, device="cuda")
+    wsb = plan.workspace_bytes(1)
+    ws = torch.empty(max(wsb, 256), dtype=torch.uint8, device="cuda")
+    cp = [None if t is None else t.data_ptr() for t in dchain]
+    ap = [None if t is None else t.data_ptr() for t in dadd]
+    plan.enable_step_timing(True)
+    n_steps = plan.num_steps()
+    with torch.cuda.stream(stream):
+        for _ in range(max(args.warmup, 3)):
+            plan.execute(cp, ap, out.data_ptr(), ws.data_ptr(), wsb, stream.cuda_stream)
+    barrier()
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    prod_ms = [0.0] * n_steps
+    pre_ms = [0.0] * n_steps
+    launches = 0
+    with torch.cuda.stream(stream):
+        e0.record(stream)
+        for _ in range(args.steps):
+            plan.execute(cp, ap, out.data_ptr(), ws.data_ptr(), wsb, stream.cuda_stream)
+            launches += plan.last_launch_count()
+        e1.record(stream)
+    barrier()
+    clocks = sampler.stop()
+    total_ms = e0.elapsed_time(e1)
+    # per-kernel times of the last step (events recorded inside the timed region on the same stream)
+    for i in range(n_steps):
+        a, b = plan.step_times(i)
+        prod_ms[i], pre_ms[i] = a, b
+    if plan.device_status() != (0, 0):
+        raise RuntimeError("device-side wait timed out")
+    t = torch.tensor([total_ms], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    total_ms = float(t.item())
+    ms_per_step = total_ms / args.steps
+    mul, addf = plan.flops()
+    useful = mul + addf
+    value = useful * world / (ms_per_step * 1e-3) / 1e9
+
+    # ---- roofline of the dominant kernel (the product kernel): useful FLOPs of its launches / their device time
+    steps_info = plan.steps()
+    prod_total_ms = sum(prod_ms)
+    achieved_tflops = useful / (prod_total_ms * 1e-3) / 1e12 if prod_total_ms > 0 else None
+    if args.variant == "3xtf32":
+        peak = peaks["bf16_sustained"] * TF32_OVER_BF16 / 3.0
+        peak_note = (f"{peaks['source']} sustained bf16 {peaks['bf16_sustained']} TFLOP/s x nominal tf32/bf16 ratio "
+                     f"{TF32_OVER_BF16:.4f} / 3 MMAs per useful product")
+        bound = "tensor"
+    else:
+        props = torch.cuda.get_device_properties(local)
+        mhz = clocks["sm_mhz"] or 1965.0
+        peak = props.multi_processor_count * 128 * 2 * mhz * 1e6 / 1e12
+        peak_note = f"{props.multi_processor_count} SMs x 128 FP32 lanes x 2 x median SM clock {mhz} MHz"
+        bound = "alu"
+    roofline = {"bound": bound, "achieved": achieved_tflops, "peak": peak, "unit": "TFLOP/s",
+                "frac": (achieved_tflops / peak) if achieved_tflops else None, "traffic": None,
+                "kernel": "product_tc_kernel" if args.variant == "3xtf32" else "product_ffma_kernel",
+                "launches_per_step": n_steps, "product_ms_per_step": prod_ms, "prepass_ms_per_step": pre_ms,
+                "peak_is": peak_note}
+
+    result = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32 (3xTF32 tensor-core split)" if args.variant == "3xtf32" else "f32",
+        "data": "synthetic",
+        "config": {"workload": eq.name, "equation": "X = L*A*U*B, 8192x8192 f32, seed 3",
+                   "parenthesization": plan.parenthesization(), "useful_flops": useful, "variant": args.variant,
+                   "l2": "operands (1 GiB) exceed L2; no flush", "parallelism": f"{world} independent replicas"},
+        "clocks": clocks, "gpu_launches": launches, "roofline": roofline,
+        "roofline_whole_equation_frac": (value / world / 1e3) / peak,
+    }
+
+    if rank == 0 and world == 1:
+        # ---- probes: sustained tcgen05 kind::tf32 rate and FFMA rate on this GPU
+        scratch = torch.empty(1 << 20, dtype=torch.uint8, device="cuda")
+        probes = {}
+        for name, fn in (("tf32_tflops", mom.mom_probe_tf32_tflops), ("ffma_tflops", mom.mom_probe_ffma_tflops)):
+            try:
+                probes[name] = fn(1000.0, scratch.data_ptr(), stream.cuda_stream)
+            except mom.MomError as e:
+                probes[name] = f"unavailable: {e}"
+        result["probes"] = probes
+        if isinstance(probes.get("tf32_tflops"), float) and args.variant == "3xtf32" and achieved_tflops:
+            result["roofline"]["frac_of_probe"] = achieved_tflops / (probes["tf32_tflops"] / 3.0)
+
+        # ---- e2e: host operands in pinned memory, H2D + execute + D2H inside the timed region
+        stage_b = plan.host_staging_bytes(1)
+        del dchain, dadd, out, ws
+        torch.cuda.empty_cache()
+        staging = torch.empty(stage_b, dtype=torch.uint8, device="cuda")
+        pin = [None if a is None else torch.from_numpy(a).pin_memory() for a in chain]
+        pin_add = [None if a is None else torch.from_numpy(a).pin_memory() for a in add]
+        out_h = torch.empty((rd.rows, rd.cols), dtype=torch.float32).pin_memory()
+        hp = [None if t is None else t.data_ptr() for t in pin]
+        hap = [None if t is None else t.data_ptr() for t in pin_add]
+        e2e_steps = min(args.steps, 5)
+        for _ in range(2):
+            plan.execute_host(hp, hap, out_h.data_ptr(), 1, staging.data_ptr(), stage_b, stream.cuda_stream)
+        t0 = time.perf_counter()
+        for _ in range(e2e_steps):
+            plan.execute_host(hp, hap, out_h.data_ptr(), 1, staging.data_ptr(), stage_b, stream.cuda_stream)
+        e2e_s = (time.perf_counter() - t0) / e2e_steps
+        h2d = sum(a.nbytes for a in chain + add if a is not None)
+        result["e2e"] = {"value": useful / e2e_s / 1e9, "unit": UNIT, "h2d_bytes_per_step": h2d,
+                         "d2h_bytes_per_step": out_h.numel() * 4, "ms_per_step": e2e_s * 1e3, "steps": e2e_steps}
+        del staging
+        torch.cuda.empty_cache()
+
+        # ---- the other configurations, briefly (min of 5 as in the paper's Section 4, and the median)
+        others = []
+        for cfg in (wl.config_tiny(), wl.config_five_general(), wl.config_property_heavy(), wl.config_batched(),
+                    wl.config_paper_chain()):
+            r = time_equation(mom, torch, cfg, variant, steps=20, warmup=3, stream=stream, timing=cfg.batch == 1)
+            ms_min, ms_med = min(r["ms"]), statistics.median(r["ms"])
+            entry = {"workload": cfg.name, "parenthesization": r["plan"].parenthesization(),
+                     "useful_flops": r["useful_flops"], "ms_min_of_20": ms_min, "ms_median": ms_med,
+                     "gflops_at_min": r["useful_flops"] / (ms_min * 1e-3) / 1e9,
+                     "gflops_at_median": r["useful_flops"] / (ms_med * 1e-3) / 1e9,
+                     "frac_of_roofline_at_median": r["useful_flops"] / (ms_med * 1e-3) / 1e12 / peak,
+                     "launches": r["launches"]}
+            if cfg.batch > 1:
+                per_inst = sum(o.rows * o.cols for o in list(cfg.chain) + list(cfg.add)) + rd_elems(r["plan"])
+                entry["hbm_gbs_at_median"] = per_inst * 4 * cfg.batch / (ms_med * 1e-3) / 1e9
+                entry["hbm_frac_of_measured_peak"] = entry["hbm_gbs_at_median"] / peaks["hbm_gbs"]
+            others.append(entry)
+            del r
+            torch.cuda.empty_cache()
+        result["all_configs"] = others
+
+        # ---- CPU baseline: the oracle on a bounded sample of the same workload
+        result["cpu_baseline"] = cpu_baseline(eq, chain, add, useful, n_rows=32)
+
+    if rank == 0:
+        print(json.dumps(result))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def rd_elems(plan):
+    d = plan.result_desc()
+    return d.rows * d.cols
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--variant", default="3xtf32", choices=["3xtf32", "ffma"])
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_gpu(args)
+
+
+if __name__ == "__main__":
+    main()

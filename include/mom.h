@@ -1,0 +1,209 @@
+/* mom.h -- C ABI of the B200 Linnea-equation library.
+ *
+ * A Linnea equation (paper Section 2, "Operations": an Equation is a bag of variadic Mul / Add ops
+ * whose Yield is one result) is restricted here to
+ *
+ *        X = M1 * M2 * ... * Mn  +  T1 + ... + Tk          (n >= 1, k >= 0)
+ *
+ * over f32 matrices that each carry one compile-time property (paper Section 2, "Matrix Attribute"
+ * and "Types": a Matrix type is a property, a static [rows, cols] and an element type; Identity is
+ * its own type).  Planning applies the paper's three transformations (Section 2, "Transformations"):
+ * identity simplification (A*I -> A, I*I -> I), matrix-chain reordering that minimises the number of
+ * useful scalar multiplications taking properties into account, and property propagation that gives
+ * every intermediate and the result a concrete type.  Execution runs each binary product with a
+ * property-specialised sm_100a kernel and fuses the Add terms into the last product.
+ *
+ * Conventions
+ *   - Every function returns mom_status_t (except mom_status_string); nothing throws; there is no
+ *     global state.  Output arguments are written only on MOM_OK unless stated otherwise.
+ *   - "host" / "device" below says which address space a pointer must belong to.
+ *   - Matrix storage (device): dense row-major f32, leading dimension == cols, base address aligned
+ *     to 16 bytes.  Entries outside a triangular operand's structure must be stored as zeros (paper
+ *     Section 2: the property dictates how the buffer is filled); the library relies on this and
+ *     does not check it.  Identity operands have no storage: their pointer may be NULL and is never
+ *     dereferenced.
+ *   - The result X is always written as a full dense rows x cols matrix; entries outside the
+ *     result's inferred structure are written as +0.0f.  X must not alias any input or the workspace.
+ *   - Execution is asynchronous on the given stream.  All argument errors are reported before
+ *     anything is enqueued.
+ */
+#ifndef MOM_H_
+#define MOM_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    MOM_OK = 0,
+    MOM_ERR_INVALID_ARG = 1,         /* null pointer, n_chain < 1, rows/cols < 1, bad enum, batch < 1 */
+    MOM_ERR_PROPERTY = 2,            /* triangular or Identity descriptor that is not square          */
+    MOM_ERR_DTYPE = 3,               /* element type other than f32                                   */
+    MOM_ERR_SHAPE_MISMATCH = 4,      /* inner dimensions differ, or an Add term's shape != X's shape  */
+    MOM_ERR_OVERFLOW = 5,            /* a multiplication count does not fit in 63 bits                */
+    MOM_ERR_ALLOC = 6,               /* host or (first execute only) device allocation failed         */
+    MOM_ERR_WORKSPACE_TOO_SMALL = 7,
+    MOM_ERR_ALIGNMENT = 8,           /* a device pointer is not 16-byte aligned                       */
+    MOM_ERR_ARCH = 9,                /* the current device is not sm_100                              */
+    MOM_ERR_CUDA = 10,               /* a CUDA runtime / driver call failed                           */
+    MOM_ERR_DEVICE_TIMEOUT = 11,     /* a bounded device-side wait expired (see mom_plan_device_status) */
+    MOM_ERR_BUFFER_TOO_SMALL = 12,   /* string buffer too small; `needed` tells the size              */
+    MOM_ERR_LIMIT = 13               /* size beyond a documented fixed maximum                        */
+} mom_status_t;
+
+/* Paper Section 2, "Matrix Attribute" / "Types".  Triangles are non-strict and non-unit: the diagonal
+ * is an ordinary stored entry (Listing 2 fills the diagonal with the fill value). */
+typedef enum { MOM_GENERAL = 0, MOM_LOWER_TRI = 1, MOM_UPPER_TRI = 2, MOM_IDENTITY = 3 } mom_property_t;
+typedef enum { MOM_F32 = 0 } mom_dtype_t;
+
+/* Arithmetic used by the product kernels.
+ *   MOM_VARIANT_3XTF32: tcgen05 tensor-core MMA (kind::tf32) on operands split as a = hi + lo,
+ *       accumulating lo*hi + hi*lo + hi*hi in f32 (f32-level accuracy).  Products whose shapes
+ *       cannot be addressed by TMA (a leading dimension that is not a multiple of 4 elements) run
+ *       on the FFMA kernel instead.
+ *       Small products (m*n*k < 2^23) also run on the FFMA kernel: the operand split and the
+ *       tensor pipeline's set-up cost more than they save there.
+ *   MOM_VARIANT_FFMA: plain f32 fused multiply-add on CUDA cores.
+ *   MOM_VARIANT_3XTF32_FORCE: as 3XTF32 but without the size rule (every TMA-addressable product
+ *       runs on tensor cores); meant for testing the tensor-core kernel on small shapes. */
+typedef enum { MOM_VARIANT_3XTF32 = 0, MOM_VARIANT_FFMA = 1, MOM_VARIANT_3XTF32_FORCE = 2 } mom_variant_t;
+
+/* Kind of a binary product, by which operands are triangular. */
+typedef enum {
+    MOM_KIND_GG = 0,     /* general * general                                  */
+    MOM_KIND_TG = 1,     /* triangular * general                               */
+    MOM_KIND_GT = 2,     /* general * triangular                               */
+    MOM_KIND_TT = 3,     /* L*L or U*U: result keeps the triangle              */
+    MOM_KIND_TTMIX = 4   /* L*U or U*L: result is general                      */
+} mom_kind_t;
+
+typedef struct {
+    int64_t rows, cols;
+    int32_t property;    /* mom_property_t */
+    int32_t dtype;       /* mom_dtype_t    */
+} mom_matrix_desc_t;
+
+/* One binary product of the plan.  Ids: 0..n_chain-1 are the original chain operands, n_chain.. are
+ * intermediates in the order they are produced; the last step's `out` is the chain's value. */
+typedef struct {
+    int32_t lhs, rhs, out;
+    int32_t kind;                    /* mom_kind_t */
+    int32_t lhs_property, rhs_property, out_property;
+    int32_t uses_tensor_cores;       /* 1: tcgen05 3xTF32 kernel, 0: FFMA kernel */
+    int64_t m, n, k;                 /* out is m x n, contraction length k */
+    uint64_t useful_mults;           /* scalar multiplications with both factors structurally non-zero */
+} mom_step_t;
+
+typedef struct mom_plan mom_plan_t;          /* opaque; host memory; immutable once created */
+typedef struct CUstream_st *mom_stream_t;    /* a CUDA stream handle (cudaStream_t) */
+
+/* Fill a descriptor (paper Section 2, "Types": property, static shape, element type).
+ * Errors: INVALID_ARG (out NULL, rows/cols < 1, unknown property), PROPERTY (non-square triangular or
+ * Identity), DTYPE. */
+mom_status_t mom_matrix_desc(int64_t rows, int64_t cols, mom_property_t property, mom_dtype_t dtype,
+                             mom_matrix_desc_t *out /* host */);
+
+/* Plan X = prod(chain) + sum(add_terms) (paper Section 2, "Transformations").  Host only: makes no
+ * CUDA call and works on a machine without a GPU.
+ *   chain      host array of n_chain >= 1 descriptors, left to right
+ *   add_terms  host array of n_add >= 0 descriptors (may be NULL when n_add == 0); each must have X's shape
+ *   out_plan   receives a plan owned by the caller; release with mom_plan_destroy
+ * The multiplication count of a product counts a_il*b_lj only when both factors are structurally
+ * non-zero; Identity operands are removed first; among equal-cost parenthesizations the split
+ * positions are compared outermost-first, left subtree before right, smallest wins.
+ * Errors: INVALID_ARG, PROPERTY, DTYPE, SHAPE_MISMATCH, OVERFLOW, ALLOC. */
+mom_status_t mom_equation_plan(const mom_matrix_desc_t *chain, int32_t n_chain,
+                               const mom_matrix_desc_t *add_terms, int32_t n_add,
+                               mom_variant_t variant, mom_plan_t **out_plan);
+
+/* mul_flops = 2 * (useful multiplications of the chosen parenthesization); add_flops = structural
+ * non-zeros of the Add terms (an Identity term counts its n diagonal entries).  Either may be NULL. */
+mom_status_t mom_plan_flops(const mom_plan_t *plan, uint64_t *mul_flops, uint64_t *add_flops);
+
+/* The chosen parenthesization over ORIGINAL operand indices, e.g. "(0*(1*3))".  Eliminated Identity
+ * operands do not appear; a single surviving operand is its bare index; an all-Identity chain is "I".
+ * Writes a NUL-terminated string into buf (host, capacity cap); *needed (optional) receives the
+ * size including the NUL.  BUFFER_TOO_SMALL if cap < needed (needed is still written). */
+mom_status_t mom_plan_parenthesization(const mom_plan_t *plan, char *buf, size_t cap, size_t *needed);
+
+mom_status_t mom_plan_num_steps(const mom_plan_t *plan, int32_t *n);
+mom_status_t mom_plan_step(const mom_plan_t *plan, int32_t i, mom_step_t *out);
+
+/* The equation's Term made concrete (paper Section 2, "Types"): shape and inferred property of X. */
+mom_status_t mom_plan_result_desc(const mom_plan_t *plan, mom_matrix_desc_t *out);
+
+/* Bytes of device workspace mom_equation_execute[_batched] needs for `batch` instances: room for
+ * the intermediates (each also as hi/lo planes for tensor-core steps), the split planes of the
+ * operands of tensor-core steps, and split-K partial sums.  May be 0. */
+mom_status_t mom_plan_workspace_bytes(const mom_plan_t *plan, int64_t batch, size_t *bytes);
+
+/* Evaluate one equation.
+ *   chain_ptrs   host array of n_chain device pointers (entries of Identity operands are ignored)
+ *   add_ptrs     host array of n_add device pointers (NULL when n_add == 0)
+ *   out          device, rows x cols f32 of the result descriptor
+ *   workspace    device, 256-byte aligned, at least mom_plan_workspace_bytes(plan, 1); borrowed for the
+ *                duration of the enqueued work; may be NULL when that size is 0
+ * The first execution of a plan on a device creates a small plan-owned device block (tile tables,
+ * TMA descriptors, a status word) with cudaMalloc; later calls allocate nothing.
+ * Errors: INVALID_ARG, ALIGNMENT, WORKSPACE_TOO_SMALL, ARCH, ALLOC, CUDA. */
+mom_status_t mom_equation_execute(const mom_plan_t *plan, const float *const *chain_ptrs,
+                                  const float *const *add_ptrs, float *out,
+                                  void *workspace, size_t workspace_bytes, mom_stream_t stream);
+
+/* Evaluate `batch` independent instances that share one plan, in one launch sequence.  Instance b of
+ * operand i starts at chain_ptrs[i] + b * chain_strides[i] (strides in elements, host arrays;
+ * likewise add_strides / out_stride).  Strides must be multiples of 4 elements and at least rows*cols. */
+mom_status_t mom_equation_execute_batched(const mom_plan_t *plan, const float *const *chain_ptrs,
+                                          const int64_t *chain_strides, const float *const *add_ptrs,
+                                          const int64_t *add_strides, float *out, int64_t out_stride,
+                                          int64_t batch, void *workspace, size_t workspace_bytes,
+                                          mom_stream_t stream);
+
+/* Bytes of device memory mom_equation_execute_host needs as staging: all non-Identity operands, the
+ * Add terms, X, and the workspace, for `batch` instances. */
+mom_status_t mom_plan_host_staging_bytes(const mom_plan_t *plan, int64_t batch, size_t *bytes);
+
+/* Same evaluation with HOST operands and a HOST result: copies the operands into `staging` (device,
+ * 256-byte aligned, at least mom_plan_host_staging_bytes), runs the plan, copies X back into
+ * out_host, all on `stream`; returns after the stream has been synchronised.  Instances are packed
+ * (stride rows*cols).  Pinned host memory makes the copies asynchronous; pageable memory also works. */
+mom_status_t mom_equation_execute_host(const mom_plan_t *plan, const float *const *chain_host,
+                                       const float *const *add_host, float *out_host, int64_t batch,
+                                       void *staging, size_t staging_bytes, mom_stream_t stream);
+
+/* After the stream has been synchronised: code == MOM_OK, or MOM_ERR_DEVICE_TIMEOUT with `detail`
+ * identifying the wait that gave up (role << 24 | barrier slot << 16 | low bits of the tile index).
+ * Kernels never trap or spin forever: a wait that exceeds its poll limit records this and the CTA
+ * leaves cleanly, so the context stays usable.  Reading clears the word. */
+mom_status_t mom_plan_device_status(const mom_plan_t *plan, int32_t *code, int32_t *detail);
+
+/* Number of kernels the most recent execute of this plan enqueued (0 before the first). */
+mom_status_t mom_plan_last_launch_count(const mom_plan_t *plan, int32_t *launches);
+
+/* Per-kernel device timing for roofline reports.  With timing enabled every execute brackets each
+ * product kernel (and, separately, its operand-split pre-pass) with CUDA events on the caller's stream.
+ * After the stream has been synchronised, mom_plan_step_times returns for the most recent execute and
+ * step i the milliseconds spent in the product kernel and in its pre-pass (0 when there is none).
+ * Off by default; enabling it creates events but no device memory. */
+mom_status_t mom_plan_enable_step_timing(mom_plan_t *plan, int32_t enable);
+mom_status_t mom_plan_step_times(const mom_plan_t *plan, int32_t i, float *product_ms, float *prepass_ms);
+
+mom_status_t mom_plan_destroy(mom_plan_t *plan);   /* NULL is accepted */
+
+const char *mom_status_string(mom_status_t status);
+
+/* Sustained-rate probes used as roofline denominators.  Each runs an instruction-issue loop on every
+ * SM for about `milliseconds` and returns the achieved rate; no global memory traffic besides a
+ * few words of output.  `scratch` is device memory of at least 1 MiB.
+ *   mom_probe_tf32_tflops:  tcgen05.mma kind::tf32, M=128 N=256 K=8 on resident shared-memory tiles.
+ *   mom_probe_ffma_tflops:  independent f32 FMA chains. */
+mom_status_t mom_probe_tf32_tflops(double milliseconds, void *scratch, mom_stream_t stream, double *tflops);
+mom_status_t mom_probe_ffma_tflops(double milliseconds, void *scratch, mom_stream_t stream, double *tflops);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MOM_H_ */

@@ -1,0 +1,241 @@
+"""Python binding of the C-ABI library declared in ``include/mom.h``.
+
+Argument marshalling only: every function here forwards to the `extern "C"` entry point of the same
+name in ``libmom.so``; planning runs in the library's C++ planner and every product in its CUDA
+kernels.  There is no Python or CPU fallback: if the shared library is missing, importing this
+package raises.  Device pointers are plain integers (e.g. ``tensor.data_ptr()``); streams are
+integer handles (e.g. ``torch.cuda.current_stream().cuda_stream``).
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import List, Optional, Sequence, Tuple
+
+GENERAL, LOWER_TRI, UPPER_TRI, IDENTITY = 0, 1, 2, 3
+F32 = 0
+VARIANT_3XTF32, VARIANT_FFMA, VARIANT_3XTF32_FORCE = 0, 1, 2
+KIND_GG, KIND_TG, KIND_GT, KIND_TT, KIND_TTMIX = 0, 1, 2, 3, 4
+
+(OK, ERR_INVALID_ARG, ERR_PROPERTY, ERR_DTYPE, ERR_SHAPE_MISMATCH, ERR_OVERFLOW, ERR_ALLOC,
+ ERR_WORKSPACE_TOO_SMALL, ERR_ALIGNMENT, ERR_ARCH, ERR_CUDA, ERR_DEVICE_TIMEOUT, ERR_BUFFER_TOO_SMALL,
+ ERR_LIMIT) = range(14)
+
+LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libmom.so")
+
+
+class MatrixDesc(ctypes.Structure):
+    _fields_ = [("rows", ctypes.c_int64), ("cols", ctypes.c_int64),
+                ("property", ctypes.c_int32), ("dtype", ctypes.c_int32)]
+
+
+class Step(ctypes.Structure):
+    _fields_ = [("lhs", ctypes.c_int32), ("rhs", ctypes.c_int32), ("out", ctypes.c_int32),
+                ("kind", ctypes.c_int32), ("lhs_property", ctypes.c_int32), ("rhs_property", ctypes.c_int32),
+                ("out_property", ctypes.c_int32), ("uses_tensor_cores", ctypes.c_int32),
+                ("m", ctypes.c_int64), ("n", ctypes.c_int64), ("k", ctypes.c_int64),
+                ("useful_mults", ctypes.c_uint64)]
+
+
+class MomError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = int(status)
+        super().__init__(f"{where}: {status_string(status)} (status {int(status)})")
+
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(
+        f"{LIB_PATH} is missing: build it with `python paper_2208_10391_b200/csrc/build.py` "
+        "(there is no fallback implementation)")
+
+_lib = ctypes.CDLL(LIB_PATH)
+
+_P = ctypes.c_void_p
+_sigs = {
+    "mom_matrix_desc": [ctypes.c_int64, ctypes.c_int64, ctypes.c_int, ctypes.c_int, ctypes.POINTER(MatrixDesc)],
+    "mom_equation_plan": [ctypes.POINTER(MatrixDesc), ctypes.c_int32, ctypes.POINTER(MatrixDesc), ctypes.c_int32,
+                          ctypes.c_int, ctypes.POINTER(_P)],
+    "mom_plan_flops": [_P, ctypes.POINTER(ctypes.c_uint64), ctypes.POINTER(ctypes.c_uint64)],
+    "mom_plan_parenthesization": [_P, ctypes.c_char_p, ctypes.c_size_t, ctypes.POINTER(ctypes.c_size_t)],
+    "mom_plan_num_steps": [_P, ctypes.POINTER(ctypes.c_int32)],
+    "mom_plan_step": [_P, ctypes.c_int32, ctypes.POINTER(Step)],
+    "mom_plan_result_desc": [_P, ctypes.POINTER(MatrixDesc)],
+    "mom_plan_workspace_bytes": [_P, ctypes.c_int64, ctypes.POINTER(ctypes.c_size_t)],
+    "mom_equation_execute": [_P, ctypes.POINTER(_P), ctypes.POINTER(_P), _P, _P, ctypes.c_size_t, _P],
+    "mom_equation_execute_batched": [_P, ctypes.POINTER(_P), ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(_P),
+                                     ctypes.POINTER(ctypes.c_int64), _P, ctypes.c_int64, ctypes.c_int64, _P,
+                                     ctypes.c_size_t, _P],
+    "mom_plan_host_staging_bytes": [_P, ctypes.c_int64, ctypes.POINTER(ctypes.c_size_t)],
+    "mom_equation_execute_host": [_P, ctypes.POINTER(_P), ctypes.POINTER(_P), _P, ctypes.c_int64, _P,
+                                  ctypes.c_size_t, _P],
+    "mom_plan_device_status": [_P, ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_int32)],
+    "mom_plan_last_launch_count": [_P, ctypes.POINTER(ctypes.c_int32)],
+    "mom_plan_enable_step_timing": [_P, ctypes.c_int32],
+    "mom_plan_step_times": [_P, ctypes.c_int32, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_float)],
+    "mom_plan_destroy": [_P],
+    "mom_probe_tf32_tflops": [ctypes.c_double, _P, _P, ctypes.POINTER(ctypes.c_double)],
+    "mom_probe_ffma_tflops": [ctypes.c_double, _P, _P, ctypes.POINTER(ctypes.c_double)],
+}
+for _name, _args in _sigs.items():
+    _fn = getattr(_lib, _name)
+    _fn.argtypes = _args
+    _fn.restype = ctypes.c_int
+_lib.mom_status_string.argtypes = [ctypes.c_int]
+_lib.mom_status_string.restype = ctypes.c_char_p
+
+EXPORTED = sorted(list(_sigs) + ["mom_status_string"])
+
+
+def status_string(status: int) -> str:
+    return _lib.mom_status_string(int(status)).decode()
+
+
+def _check(status: int, where: str) -> None:
+    if status != OK:
+        raise MomError(status, where)
+
+
+def _ptr_array(values: Sequence[Optional[int]]):
+    arr = (_P * max(len(values), 1))()
+    for i, v in enumerate(values):
+        arr[i] = None if v is None else int(v)
+    return arr
+
+
+def mom_matrix_desc(rows: int, cols: int, prop: int = GENERAL, dtype: int = F32) -> MatrixDesc:
+    d = MatrixDesc()
+    _check(_lib.mom_matrix_desc(rows, cols, prop, dtype, ctypes.byref(d)), "mom_matrix_desc")
+    return d
+
+
+def _desc_array(descs: Sequence) -> "ctypes.Array":
+    arr = (MatrixDesc * max(len(descs), 1))()
+    for i, d in enumerate(descs):
+        if isinstance(d, MatrixDesc):
+            arr[i] = d
+        else:       # (rows, cols, property) triple: passed through unchecked so that the planner validates it
+            arr[i] = MatrixDesc(int(d[0]), int(d[1]), int(d[2]), F32 if len(d) < 4 else int(d[3]))
+    return arr
+
+
+class Plan:
+    """Owner of a ``mom_plan_t*``; methods mirror the ``mom_plan_*`` / ``mom_equation_execute*`` calls."""
+
+    def __init__(self, handle: int, n_chain: int, n_add: int):
+        self._h = _P(handle)
+        self.n_chain, self.n_add = n_chain, n_add
+
+    def __del__(self):
+        self.destroy()
+
+    def destroy(self) -> None:
+        if getattr(self, "_h", None) is not None and self._h.value:
+            _lib.mom_plan_destroy(self._h)
+            self._h = _P(None)
+
+    # ---- queries
+    def flops(self) -> Tuple[int, int]:
+        mul, add = ctypes.c_uint64(), ctypes.c_uint64()
+        _check(_lib.mom_plan_flops(self._h, ctypes.byref(mul), ctypes.byref(add)), "mom_plan_flops")
+        return mul.value, add.value
+
+    def parenthesization(self) -> str:
+        need = ctypes.c_size_t()
+        st = _lib.mom_plan_parenthesization(self._h, None, 0, ctypes.byref(need))
+        if st not in (OK, ERR_BUFFER_TOO_SMALL):
+            _check(st, "mom_plan_parenthesization")
+        buf = ctypes.create_string_buffer(need.value)
+        _check(_lib.mom_plan_parenthesization(self._h, buf, need.value, None), "mom_plan_parenthesization")
+        return buf.value.decode()
+
+    def num_steps(self) -> int:
+        n = ctypes.c_int32()
+        _check(_lib.mom_plan_num_steps(self._h, ctypes.byref(n)), "mom_plan_num_steps")
+        return n.value
+
+    def step(self, i: int) -> Step:
+        s = Step()
+        _check(_lib.mom_plan_step(self._h, i, ctypes.byref(s)), "mom_plan_step")
+        return s
+
+    def steps(self) -> List[Step]:
+        return [self.step(i) for i in range(self.num_steps())]
+
+    def result_desc(self) -> MatrixDesc:
+        d = MatrixDesc()
+        _check(_lib.mom_plan_result_desc(self._h, ctypes.byref(d)), "mom_plan_result_desc")
+        return d
+
+    def workspace_bytes(self, batch: int = 1) -> int:
+        b = ctypes.c_size_t()
+        _check(_lib.mom_plan_workspace_bytes(self._h, batch, ctypes.byref(b)), "mom_plan_workspace_bytes")
+        return b.value
+
+    def host_staging_bytes(self, batch: int = 1) -> int:
+        b = ctypes.c_size_t()
+        _check(_lib.mom_plan_host_staging_bytes(self._h, batch, ctypes.byref(b)), "mom_plan_host_staging_bytes")
+        return b.value
+
+    def device_status(self) -> Tuple[int, int]:
+        code, detail = ctypes.c_int32(), ctypes.c_int32()
+        _check(_lib.mom_plan_device_status(self._h, ctypes.byref(code), ctypes.byref(detail)), "mom_plan_device_status")
+        return code.value, detail.value
+
+    def last_launch_count(self) -> int:
+        n = ctypes.c_int32()
+        _check(_lib.mom_plan_last_launch_count(self._h, ctypes.byref(n)), "mom_plan_last_launch_count")
+        return n.value
+
+    def enable_step_timing(self, enable: bool = True) -> None:
+        _check(_lib.mom_plan_enable_step_timing(self._h, 1 if enable else 0), "mom_plan_enable_step_timing")
+
+    def step_times(self, i: int) -> Tuple[float, float]:
+        """(product kernel ms, pre-pass ms) of step i in the most recent execute (after a stream sync)."""
+        a, b = ctypes.c_float(), ctypes.c_float()
+        _check(_lib.mom_plan_step_times(self._h, i, ctypes.byref(a), ctypes.byref(b)), "mom_plan_step_times")
+        return a.value, b.value
+
+    # ---- execution (device pointers as integers)
+    def execute(self, chain_ptrs: Sequence[Optional[int]], add_ptrs: Sequence[Optional[int]], out_ptr: int,
+                workspace_ptr: Optional[int], workspace_bytes: int, stream: int = 0) -> None:
+        _check(_lib.mom_equation_execute(self._h, _ptr_array(chain_ptrs), _ptr_array(add_ptrs) if add_ptrs else None,
+                                         _P(out_ptr), _P(workspace_ptr), workspace_bytes, _P(stream)),
+               "mom_equation_execute")
+
+    def execute_batched(self, chain_ptrs, chain_strides, add_ptrs, add_strides, out_ptr: int, out_stride: int,
+                        batch: int, workspace_ptr: Optional[int], workspace_bytes: int, stream: int = 0) -> None:
+        cs = (ctypes.c_int64 * max(len(chain_strides), 1))(*[int(s) for s in chain_strides])
+        as_ = (ctypes.c_int64 * max(len(add_strides), 1))(*[int(s) for s in add_strides])
+        _check(_lib.mom_equation_execute_batched(self._h, _ptr_array(chain_ptrs), cs,
+                                                 _ptr_array(add_ptrs) if add_ptrs else None, as_ if add_ptrs else None,
+                                                 _P(out_ptr), out_stride, batch, _P(workspace_ptr), workspace_bytes,
+                                                 _P(stream)), "mom_equation_execute_batched")
+
+    def execute_host(self, chain_host_ptrs, add_host_ptrs, out_host_ptr: int, batch: int, staging_ptr: int,
+                     staging_bytes: int, stream: int = 0) -> None:
+        _check(_lib.mom_equation_execute_host(self._h, _ptr_array(chain_host_ptrs),
+                                              _ptr_array(add_host_ptrs) if add_host_ptrs else None,
+                                              _P(out_host_ptr), batch, _P(staging_ptr), staging_bytes, _P(stream)),
+               "mom_equation_execute_host")
+
+
+def mom_equation_plan(chain: Sequence, add_terms: Sequence = (), variant: int = VARIANT_3XTF32) -> Plan:
+    """Plan X = prod(chain) + sum(add_terms); operands are MatrixDesc or (rows, cols, property) triples."""
+    handle = _P()
+    n_chain, n_add = len(chain), len(add_terms)
+    st = _lib.mom_equation_plan(_desc_array(chain) if n_chain else None, n_chain,
+                                _desc_array(add_terms) if n_add else None, n_add, variant, ctypes.byref(handle))
+    _check(st, "mom_equation_plan")
+    return Plan(handle.value, n_chain, n_add)
+
+
+def mom_probe_tf32_tflops(milliseconds: float, scratch_ptr: int, stream: int = 0) -> float:
+    out = ctypes.c_double()
+    _check(_lib.mom_probe_tf32_tflops(milliseconds, _P(scratch_ptr), _P(stream), ctypes.byref(out)), "mom_probe_tf32_tflops")
+    return out.value
+
+
+def mom_probe_ffma_tflops(milliseconds: float, scratch_ptr: int, stream: int = 0) -> float:
+    out = ctypes.c_double()
+    _check(_lib.mom_probe_ffma_tflops(milliseconds, _P(scratch_ptr), _P(stream), ctypes.byref(out)), "mom_probe_ffma_tflops")
+    return out.value

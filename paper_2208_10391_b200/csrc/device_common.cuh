@@ -1,0 +1,56 @@
+// Device-side pieces shared by the product kernels: the structural k-range of an output tile, the
+// structure mask of the result, and the fused Add epilogue.
+#pragma once
+
+#include <cstdint>
+#include <cuda_runtime.h>
+
+#include "mom.h"
+
+namespace mom {
+
+constexpr int MAX_FUSED_ADD = 8;    // Add terms fused into one launch; more are added by follow-up passes
+
+// Add terms of the equation (paper Table 1, "Add"), applied left to right in f32.
+struct AddTerms {
+    const float *ptr[MAX_FUSED_ADD];     // NULL for an Identity term
+    long long stride[MAX_FUSED_ADD];     // elements between batch instances
+    int count;
+};
+
+// With dense zero-filled storage every product is C[r,c] = sum over l in [klo, khi) of A[r,l]*B[l,c],
+// where the range for an output tile rows [r0,r1) x cols [c0,c1) is the intersection of the
+// operands' structural ranges:
+//   A lowerTri: l < r1      A upperTri: l >= r0      B lowerTri: l >= c0      B upperTri: l < c1
+// An empty range means the tile is structurally zero.
+__host__ __device__ inline void tile_k_range(int pa, int pb, int r0, int r1, int c0, int c1, int k,
+                                             int *klo, int *khi) {
+    int lo = 0, hi = k;
+    if (pa == MOM_UPPER_TRI && r0 > lo) lo = r0;
+    if (pb == MOM_LOWER_TRI && c0 > lo) lo = c0;
+    if (pa == MOM_LOWER_TRI && r1 < hi) hi = r1;
+    if (pb == MOM_UPPER_TRI && c1 < hi) hi = c1;
+    *klo = lo;
+    *khi = hi;
+}
+
+__host__ __device__ inline bool in_structure(int prop, int r, int c) {
+    return prop == MOM_GENERAL || (prop == MOM_LOWER_TRI && r >= c) || (prop == MOM_UPPER_TRI && r <= c) ||
+           (prop == MOM_IDENTITY && r == c);
+}
+
+// value of the equation at (r, c) given the chain's value `acc` there
+__device__ __forceinline__ float finish_entry(float acc, const AddTerms &add, long long batch, int r, int c,
+                                               int ld, int out_prop) {
+    float v = acc;
+#pragma unroll
+    for (int t = 0; t < MAX_FUSED_ADD; ++t) {
+        if (t < add.count) {
+            const float *p = add.ptr[t];
+            v += p ? __ldg(p + batch * add.stride[t] + (long long)r * ld + c) : (r == c ? 1.0f : 0.0f);
+        }
+    }
+    return in_structure(out_prop, r, c) ? v : 0.0f;
+}
+
+}  // namespace mom

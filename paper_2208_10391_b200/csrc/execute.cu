@@ -1,0 +1,316 @@
+// Launcher: walks a plan's steps and enqueues the kernels on the caller's stream.
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "kernels.h"
+#include "mom_internal.h"
+#include "product_tc.h"
+
+namespace mom {
+
+struct DeviceState {
+    int device = -1;
+    int32_t *status = nullptr;          // device: {code, detail, 0, 0}
+    TcPlanState tc;                     // tile tables of tensor-core steps
+    std::vector<cudaEvent_t> events;    // 3 per step when step timing is on: before pre-pass, before product, after
+};
+
+void destroy_device_state(DeviceState *d) {
+    if (!d) return;
+    int prev = -1;
+    cudaGetDevice(&prev);
+    if (d->device >= 0) cudaSetDevice(d->device);
+    tc_release(d->tc);
+    for (cudaEvent_t e : d->events) cudaEventDestroy(e);
+    if (d->status) cudaFree(d->status);
+    if (prev >= 0) cudaSetDevice(prev);
+    delete d;
+}
+
+namespace {
+
+mom_status_t check_arch(int *device_out) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return MOM_ERR_CUDA;
+    int major = 0;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return MOM_ERR_CUDA;
+    if (major != 10) return MOM_ERR_ARCH;
+    *device_out = dev;
+    return MOM_OK;
+}
+
+mom_status_t ensure_device_state(const mom_plan *p, int device) {
+    if (p->dev && p->dev->device == device) return MOM_OK;
+    if (p->dev) { destroy_device_state(p->dev); p->dev = nullptr; }
+    DeviceState *d = new (std::nothrow) DeviceState();
+    if (!d) return MOM_ERR_ALLOC;
+    d->device = device;
+    if (cudaMalloc(&d->status, 4 * sizeof(int32_t)) != cudaSuccess) { delete d; return MOM_ERR_ALLOC; }
+    if (cudaMemset(d->status, 0, 4 * sizeof(int32_t)) != cudaSuccess) { cudaFree(d->status); delete d; return MOM_ERR_CUDA; }
+    p->dev = d;
+    return MOM_OK;
+}
+
+bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+
+struct Operand { const float *ptr; long long stride; };
+
+mom_status_t execute_impl(const mom_plan *p, const float *const *chain_ptrs, const int64_t *chain_strides,
+                          const float *const *add_ptrs, const int64_t *add_strides, float *out, int64_t out_stride,
+                          int64_t batch, void *workspace, size_t workspace_bytes, cudaStream_t stream) {
+    if (!p || !chain_ptrs || !out || batch < 1) return MOM_ERR_INVALID_ARG;
+    const int n_chain = (int)p->chain.size(), n_add = (int)p->add.size();
+    if (n_add > 0 && !add_ptrs) return MOM_ERR_INVALID_ARG;
+    if (batch > 1 && (!chain_strides || (n_add > 0 && !add_strides))) return MOM_ERR_INVALID_ARG;
+    const int64_t rows = p->result_desc.rows, cols = p->result_desc.cols;
+
+    for (int i = 0; i < n_chain; ++i) {
+        if (p->chain[i].property == MOM_IDENTITY) continue;
+        if (!chain_ptrs[i]) return MOM_ERR_INVALID_ARG;
+        if (!aligned16(chain_ptrs[i])) return MOM_ERR_ALIGNMENT;
+        if (batch > 1 && (chain_strides[i] % 4 != 0 || chain_strides[i] < p->chain[i].rows * p->chain[i].cols))
+            return MOM_ERR_INVALID_ARG;
+    }
+    for (int i = 0; i < n_add; ++i) {
+        if (p->add[i].property == MOM_IDENTITY) continue;
+        if (!add_ptrs[i]) return MOM_ERR_INVALID_ARG;
+        if (!aligned16(add_ptrs[i])) return MOM_ERR_ALIGNMENT;
+        if (batch > 1 && (add_strides[i] % 4 != 0 || add_strides[i] < rows * cols)) return MOM_ERR_INVALID_ARG;
+    }
+    if (!aligned16(out)) return MOM_ERR_ALIGNMENT;
+    if (batch > 1 && (out_stride % 4 != 0 || out_stride < rows * cols)) return MOM_ERR_INVALID_ARG;
+
+    size_t need = 0;
+    mom_plan_workspace_bytes(p, batch, &need);
+    if (need > 0) {
+        if (!workspace || workspace_bytes < need) return MOM_ERR_WORKSPACE_TOO_SMALL;
+        if (reinterpret_cast<uintptr_t>(workspace) % WS_ALIGN != 0) return MOM_ERR_ALIGNMENT;
+    }
+
+    int device = 0;
+    mom_status_t st = check_arch(&device);
+    if (st != MOM_OK) return st;
+    st = ensure_device_state(p, device);
+    if (st != MOM_OK) return st;
+
+    bool any_tc = false;
+    for (const auto &s : p->steps) any_tc |= s.pub.uses_tensor_cores != 0;
+    if (any_tc) {
+        st = tc_prepare(*p, p->dev->tc);
+        if (st != MOM_OK) return st;
+    }
+
+    int launches = 0;
+    const int ns = (int)p->steps.size();
+    const bool timing = p->step_timing && batch == 1;
+    if (timing && p->dev->events.size() != (size_t)ns * 3) {
+        for (cudaEvent_t e : p->dev->events) cudaEventDestroy(e);
+        p->dev->events.assign((size_t)ns * 3, nullptr);
+        for (auto &e : p->dev->events)
+            if (cudaEventCreate(&e) != cudaSuccess) return MOM_ERR_CUDA;
+    }
+    // instances per pass: all of them when every step can take grid.z batching, else one at a time
+    const int64_t group = any_tc ? 1 : (batch < 65535 ? batch : 65535);
+    const size_t ws_inst = p->workspace_per_instance;
+
+    for (int64_t b0 = 0; b0 < batch; b0 += group) {
+        const int nb = (int)((batch - b0 < group) ? batch - b0 : group);
+        auto chain_op = [&](int id) {
+            const long long s = chain_strides ? chain_strides[id] : 0;
+            return Operand{chain_ptrs[id] ? chain_ptrs[id] + b0 * s : nullptr, s};
+        };
+        auto add_terms = [&](int first, AddTerms *t) {
+            t->count = 0;
+            for (int i = first; i < n_add && t->count < MAX_FUSED_ADD; ++i, ++t->count) {
+                const long long s = add_strides ? add_strides[i] : 0;
+                t->ptr[t->count] = p->add[i].property == MOM_IDENTITY ? nullptr : add_ptrs[i] + b0 * s;
+                t->stride[t->count] = s;
+            }
+            return first + t->count;
+        };
+        float *x = out + b0 * out_stride;
+        int added = 0;
+
+        if (ns == 0) {
+            AddTerms t;
+            added = add_terms(0, &t);
+            cudaError_t e;
+            if (p->kept.empty()) {
+                e = launch_elementwise(nullptr, 0, 1, x, out_stride, (int)rows, (int)cols, p->result_desc.property, t, nb, stream);
+            } else {
+                const Operand src = chain_op(p->kept[0]);
+                e = launch_elementwise(src.ptr, src.stride, 0, x, out_stride, (int)rows, (int)cols, p->result_desc.property, t, nb, stream);
+            }
+            if (e != cudaSuccess) return MOM_ERR_CUDA;
+            ++launches;
+        }
+
+        for (int s = 0; s < ns; ++s) {
+            const StepImpl &stp = p->steps[s];
+            auto value = [&](int id) {
+                if (id < n_chain) return chain_op(id);
+                const StepImpl &prod = p->steps[id - n_chain];
+                const long long elems = (long long)prod.pub.m * prod.pub.n;
+                // grid.z batching keeps one copy of each intermediate per instance, instance-major
+                return Operand{reinterpret_cast<const float *>(static_cast<char *>(workspace) + prod.out_off * (size_t)nb), elems};
+            };
+            const Operand A = value(stp.pub.lhs), B = value(stp.pub.rhs);
+            ProductArgs a;
+            std::memset(&a, 0, sizeof(a));
+            a.A = A.ptr; a.B = B.ptr;
+            a.strideA = A.stride; a.strideB = B.stride;
+            a.m = (int)stp.pub.m; a.n = (int)stp.pub.n; a.k = (int)stp.pub.k;
+            a.pa = stp.pub.lhs_property; a.pb = stp.pub.rhs_property;
+            if (stp.is_last) {
+                a.C = x; a.strideC = out_stride;
+                a.pout = p->result_desc.property;
+                added = add_terms(0, &a.add);
+            } else {
+                a.C = reinterpret_cast<float *>(static_cast<char *>(workspace) + stp.out_off * (size_t)nb);
+                a.strideC = (long long)stp.pub.m * stp.pub.n;
+                a.pout = stp.pub.out_property;
+                a.add.count = 0;
+            }
+            cudaEvent_t *ev = timing ? &p->dev->events[(size_t)s * 3] : nullptr;
+            if (ev) cudaEventRecord(ev[0], stream);
+            if (stp.pub.uses_tensor_cores) {
+                int used = 0;
+                st = tc_launch_step(*p, p->dev->tc, s, a, static_cast<char *>(workspace), p->dev->status, stream, &used,
+                                    ev ? ev[1] : nullptr);
+                if (st != MOM_OK) return st;
+                launches += used;
+            } else {
+                if (ev) cudaEventRecord(ev[1], stream);
+                if (launch_product_ffma(a, nb, stream) != cudaSuccess) return MOM_ERR_CUDA;
+                ++launches;
+            }
+            if (ev) cudaEventRecord(ev[2], stream);
+        }
+        (void)ws_inst;
+
+        // Add terms beyond the fused limit: X += T, a few at a time, in place
+        while (added < n_add) {
+            AddTerms t;
+            const int first = added;
+            added = add_terms(first, &t);
+            if (launch_elementwise(nullptr, 0, 2, x, out_stride, (int)rows, (int)cols, p->result_desc.property, t, nb, stream) != cudaSuccess)
+                return MOM_ERR_CUDA;
+            ++launches;
+        }
+    }
+    p->last_launches = launches;
+    return MOM_OK;
+}
+
+}  // namespace
+}  // namespace mom
+
+extern "C" {
+
+mom_status_t mom_equation_execute(const mom_plan_t *plan, const float *const *chain_ptrs,
+                                  const float *const *add_ptrs, float *out,
+                                  void *workspace, size_t workspace_bytes, mom_stream_t stream) {
+    return mom::execute_impl(plan, chain_ptrs, nullptr, add_ptrs, nullptr, out, 0, 1, workspace, workspace_bytes,
+                             reinterpret_cast<cudaStream_t>(stream));
+}
+
+mom_status_t mom_equation_execute_batched(const mom_plan_t *plan, const float *const *chain_ptrs,
+                                          const int64_t *chain_strides, const float *const *add_ptrs,
+                                          const int64_t *add_strides, float *out, int64_t out_stride,
+                                          int64_t batch, void *workspace, size_t workspace_bytes,
+                                          mom_stream_t stream) {
+    return mom::execute_impl(plan, chain_ptrs, chain_strides, add_ptrs, add_strides, out, out_stride, batch,
+                             workspace, workspace_bytes, reinterpret_cast<cudaStream_t>(stream));
+}
+
+mom_status_t mom_equation_execute_host(const mom_plan_t *plan, const float *const *chain_host,
+                                       const float *const *add_host, float *out_host, int64_t batch,
+                                       void *staging, size_t staging_bytes, mom_stream_t stream_) {
+    if (!plan || !chain_host || !out_host || batch < 1) return MOM_ERR_INVALID_ARG;
+    cudaStream_t stream = reinterpret_cast<cudaStream_t>(stream_);
+    size_t need = 0;
+    mom_plan_host_staging_bytes(plan, batch, &need);
+    if (!staging || staging_bytes < need) return MOM_ERR_WORKSPACE_TOO_SMALL;
+    if (reinterpret_cast<uintptr_t>(staging) % mom::WS_ALIGN != 0) return MOM_ERR_ALIGNMENT;
+    const int n_chain = (int)plan->chain.size(), n_add = (int)plan->add.size();
+    if (n_add > 0 && !add_host) return MOM_ERR_INVALID_ARG;
+
+    char *cur = static_cast<char *>(staging);
+    std::vector<const float *> cptr(n_chain, nullptr), aptr(n_add, nullptr);
+    std::vector<int64_t> cstride(n_chain, 0), astride(n_add, 0);
+    auto stage = [&](const mom_matrix_desc_t &d, const float *host, const float **dev, int64_t *stride) -> mom_status_t {
+        if (d.property == MOM_IDENTITY) return MOM_OK;
+        if (!host) return MOM_ERR_INVALID_ARG;
+        const size_t bytes = (size_t)d.rows * d.cols * sizeof(float) * batch;
+        if (cudaMemcpyAsync(cur, host, bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess) return MOM_ERR_CUDA;
+        *dev = reinterpret_cast<const float *>(cur);
+        *stride = d.rows * d.cols;
+        cur += mom::align_up(bytes, mom::WS_ALIGN);
+        return MOM_OK;
+    };
+    for (int i = 0; i < n_chain; ++i) {
+        mom_status_t st = stage(plan->chain[i], chain_host[i], &cptr[i], &cstride[i]);
+        if (st != MOM_OK) return st;
+    }
+    for (int i = 0; i < n_add; ++i) {
+        mom_status_t st = stage(plan->add[i], add_host[i], &aptr[i], &astride[i]);
+        if (st != MOM_OK) return st;
+    }
+    float *x = reinterpret_cast<float *>(cur);
+    const int64_t xelems = plan->result_desc.rows * plan->result_desc.cols;
+    const size_t xbytes = (size_t)xelems * sizeof(float) * batch;
+    cur += mom::align_up(xbytes, mom::WS_ALIGN);
+    size_t ws_bytes = 0;
+    mom_plan_workspace_bytes(plan, batch, &ws_bytes);
+    // strides that are not multiples of 4 elements cannot be batched in place; such instances are rare
+    // (odd-sized matrices) and are handled one call at a time
+    bool strides_ok = xelems % 4 == 0;
+    for (int i = 0; i < n_chain; ++i) strides_ok &= cstride[i] % 4 == 0;
+    for (int i = 0; i < n_add; ++i) strides_ok &= astride[i] % 4 == 0;
+    mom_status_t st = MOM_OK;
+    if (batch == 1) {
+        st = mom::execute_impl(plan, cptr.data(), nullptr, aptr.data(), nullptr, x, 0, 1, cur, ws_bytes, stream);
+    } else if (strides_ok) {
+        st = mom::execute_impl(plan, cptr.data(), cstride.data(), aptr.data(), astride.data(), x, xelems, batch, cur, ws_bytes, stream);
+    } else {
+        return MOM_ERR_ALIGNMENT;
+    }
+    if (st != MOM_OK) return st;
+    if (cudaMemcpyAsync(out_host, x, xbytes, cudaMemcpyDeviceToHost, stream) != cudaSuccess) return MOM_ERR_CUDA;
+    if (cudaStreamSynchronize(stream) != cudaSuccess) return MOM_ERR_CUDA;
+    return MOM_OK;
+}
+
+mom_status_t mom_plan_enable_step_timing(mom_plan_t *plan, int32_t enable) {
+    if (!plan) return MOM_ERR_INVALID_ARG;
+    plan->step_timing = enable != 0;
+    return MOM_OK;
+}
+
+mom_status_t mom_plan_step_times(const mom_plan_t *plan, int32_t i, float *product_ms, float *prepass_ms) {
+    if (!plan || i < 0 || i >= (int32_t)plan->steps.size()) return MOM_ERR_INVALID_ARG;
+    if (!plan->dev || plan->dev->events.size() != plan->steps.size() * 3) return MOM_ERR_INVALID_ARG;
+    cudaEvent_t *ev = &plan->dev->events[(size_t)i * 3];
+    float pre = 0.0f, prod = 0.0f;
+    if (cudaEventElapsedTime(&pre, ev[0], ev[1]) != cudaSuccess) return MOM_ERR_CUDA;
+    if (cudaEventElapsedTime(&prod, ev[1], ev[2]) != cudaSuccess) return MOM_ERR_CUDA;
+    if (product_ms) *product_ms = prod;
+    if (prepass_ms) *prepass_ms = pre;
+    return MOM_OK;
+}
+
+mom_status_t mom_plan_device_status(const mom_plan_t *plan, int32_t *code, int32_t *detail) {
+    if (!plan || !code) return MOM_ERR_INVALID_ARG;
+    int32_t host[4] = {0, 0, 0, 0};
+    if (plan->dev && plan->dev->status) {
+        if (cudaMemcpy(host, plan->dev->status, sizeof(host), cudaMemcpyDeviceToHost) != cudaSuccess) return MOM_ERR_CUDA;
+        if (host[0] != 0 && cudaMemset(plan->dev->status, 0, sizeof(host)) != cudaSuccess) return MOM_ERR_CUDA;
+    }
+    *code = host[0];
+    if (detail) *detail = host[1];
+    return MOM_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,26 @@
+// Launch interfaces of the CUDA kernels (internal).
+#pragma once
+
+#include <cuda_runtime.h>
+
+#include "device_common.cuh"
+
+namespace mom {
+
+// One binary product C(m x n) = A(m x k) * B(k x n) (+ Add terms), dense row-major f32.
+struct ProductArgs {
+    const float *A;
+    const float *B;
+    float *C;
+    int m, n, k;
+    int pa, pb, pout;                       // mom_property_t of A, B and of what is written to C
+    long long strideA, strideB, strideC;    // elements between batch instances
+    AddTerms add;
+};
+
+cudaError_t launch_product_ffma(const ProductArgs &a, int batch, cudaStream_t stream);
+
+cudaError_t launch_elementwise(const float *src, long long src_stride, int src_mode, float *X, long long x_stride,
+                               int rows, int cols, int out_prop, const AddTerms &add, int batch, cudaStream_t stream);
+
+}  // namespace mom

@@ -1,0 +1,63 @@
+// Internal structures shared by the host planner and the launcher.  Not part of the public ABI.
+#pragma once
+
+#include <cstddef>
+#include <cstdint>
+#include <string>
+#include <vector>
+
+#include "mom.h"
+
+namespace mom {
+
+// Tile shapes of the tensor-core product kernel (see product_tc.cu).
+constexpr int TC_BM = 128;          // output rows per tile   (MMA M)
+constexpr int TC_BN = 256;          // output cols per tile   (MMA N)
+constexpr int TC_BK = 32;           // f32 elements per k-block = one 128-byte swizzle row
+// The operand-split pre-pass works on square blocks of this edge and skips blocks that lie wholly
+// outside a triangular operand's structure.  It must be a multiple of both TC_BM and TC_BN so that
+// every block a product tile can touch has been written.
+constexpr int SPLIT_BLOCK = 256;
+
+// Tile shape of the FFMA product kernel (see product_ffma.cu).
+constexpr int FF_BM = 128;
+constexpr int FF_BN = 128;
+
+constexpr size_t WS_ALIGN = 256;
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+struct StepImpl {
+    mom_step_t pub;
+    bool is_last = false;           // carries the Add terms and writes X
+    // workspace byte offsets (per instance); SIZE_MAX = not used
+    size_t out_off = SIZE_MAX;      // f32 intermediate written by this step (not for the last step)
+    size_t a_hi_off = SIZE_MAX, a_lo_off = SIZE_MAX;   // split planes of the operands (tensor-core steps)
+    size_t b_hi_off = SIZE_MAX, b_lo_off = SIZE_MAX;
+};
+
+struct DeviceState;   // launcher-owned, created on first execute (execute.cu)
+
+}  // namespace mom
+
+struct mom_plan {
+    int32_t variant = 0;
+    std::vector<mom_matrix_desc_t> chain;      // original operands
+    std::vector<mom_matrix_desc_t> add;
+    std::vector<int32_t> kept;                 // original indices surviving identity simplification
+    std::string paren;
+    uint64_t mults = 0;                        // useful multiplications of the chosen tree
+    uint64_t add_flops = 0;
+    std::vector<mom::StepImpl> steps;
+    mom_matrix_desc_t product_desc{};          // chain value before the Add terms
+    mom_matrix_desc_t result_desc{};
+    size_t workspace_per_instance = 0;
+    mutable mom::DeviceState *dev = nullptr;
+    mutable int32_t last_launches = 0;
+    bool step_timing = false;
+};
+
+namespace mom {
+// defined in execute.cu; releases device-side state of a plan (no-op when none exists)
+void destroy_device_state(DeviceState *);
+}  // namespace mom

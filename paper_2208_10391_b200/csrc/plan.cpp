@@ -1,0 +1,349 @@
+// Host planner: identity simplification, property-aware matrix-chain dynamic program, property
+// propagation, step emission and workspace layout (paper Section 2, "Transformations").
+// Pure host code: no CUDA call is made here.
+#include <algorithm>
+#include <cstring>
+#include <new>
+
+#include "mom_internal.h"
+
+namespace {
+
+using u128 = unsigned __int128;
+constexpr uint64_t COST_LIMIT = (uint64_t)1 << 63;
+
+bool is_tri(int32_t p) { return p == MOM_LOWER_TRI || p == MOM_UPPER_TRI; }
+
+// Least upper bound in  Identity < {lowerTri, upperTri} < general  (paper Listing 3 types L*L as lowerTri).
+int32_t join_property(int32_t p, int32_t q) {
+    if (p == MOM_IDENTITY) return q;
+    if (q == MOM_IDENTITY) return p;
+    return p == q ? p : (int32_t)MOM_GENERAL;
+}
+
+// Scalar multiplications a_il * b_lj of an (m x k)(k x n) product in which both factors are
+// structurally non-zero.  Triangular operands are square.  Returns false on overflow.
+bool useful_mults(int32_t pa, int32_t pb, int64_t m, int64_t k, int64_t n, uint64_t *out) {
+    u128 v;
+    const u128 M = (u128)m, K = (u128)k, N = (u128)n;
+    if (!is_tri(pa) && !is_tri(pb)) {
+        v = M * K * N;
+    } else if (is_tri(pa) && !is_tri(pb)) {
+        v = N * (K * (K + 1) / 2);                 // row i of A has i+1 (or k-i) non-zeros
+    } else if (!is_tri(pa) && is_tri(pb)) {
+        v = M * (K * (K + 1) / 2);
+    } else if (pa == pb) {
+        v = K * (K + 1) * (K + 2) / 6;             // sum_l (l+1)(k-l) over the shared triangle
+    } else {
+        v = K * (K + 1) * (2 * K + 1) / 6;         // sum_l (l+1)^2 : opposite triangles
+    }
+    if (v >= (u128)COST_LIMIT) return false;
+    *out = (uint64_t)v;
+    return true;
+}
+
+mom_status_t check_desc(const mom_matrix_desc_t &d) {
+    if (d.rows < 1 || d.cols < 1) return MOM_ERR_INVALID_ARG;
+    if (d.property < MOM_GENERAL || d.property > MOM_IDENTITY) return MOM_ERR_INVALID_ARG;
+    if (d.dtype != MOM_F32) return MOM_ERR_DTYPE;
+    if (d.property != MOM_GENERAL && d.rows != d.cols) return MOM_ERR_PROPERTY;
+    return MOM_OK;
+}
+
+uint64_t nnz(const mom_matrix_desc_t &d) {
+    if (d.property == MOM_GENERAL) return (uint64_t)d.rows * (uint64_t)d.cols;
+    if (d.property == MOM_IDENTITY) return (uint64_t)d.rows;
+    return (uint64_t)d.rows * ((uint64_t)d.rows + 1) / 2;
+}
+
+// Property of chain value + T1 + ... + Tk.  A sum with terms is never Identity: an Identity summand
+// only contributes its diagonal footprint, which fits inside either triangle.
+int32_t sum_property(int32_t product, const std::vector<mom_matrix_desc_t> &terms) {
+    if (terms.empty()) return product;
+    bool seen = false;
+    int32_t acc = MOM_GENERAL;
+    auto fold = [&](int32_t p) {
+        if (p == MOM_IDENTITY) return;
+        if (!seen) { acc = p; seen = true; }
+        else if (acc != p) acc = MOM_GENERAL;
+    };
+    fold(product);
+    for (const auto &t : terms) fold(t.property);
+    return seen ? acc : (int32_t)MOM_LOWER_TRI;
+}
+
+struct Node { int64_t rows, cols; int32_t prop; };
+
+struct Interval { size_t bytes; int first, last; size_t *slot; size_t off; };
+
+// First-fit offsets such that buffers whose live ranges [first, last] intersect never overlap.
+size_t pack(std::vector<Interval> &items) {
+    size_t total = 0;
+    std::vector<Interval *> placed;
+    std::vector<Interval *> order;
+    for (auto &it : items) order.push_back(&it);
+    std::stable_sort(order.begin(), order.end(), [](Interval *a, Interval *b) { return a->bytes > b->bytes; });
+    for (Interval *it : order) {
+        size_t off = 0;
+        bool moved = true;
+        while (moved) {
+            moved = false;
+            for (Interval *p : placed) {
+                const bool live = !(p->last < it->first || it->last < p->first);
+                const bool overlap = off < p->off + p->bytes && p->off < off + it->bytes;
+                if (live && overlap) { off = mom::align_up(p->off + p->bytes, mom::WS_ALIGN); moved = true; }
+            }
+        }
+        it->off = off;
+        *it->slot = off;
+        placed.push_back(it);
+        total = std::max(total, off + it->bytes);
+    }
+    return mom::align_up(total, mom::WS_ALIGN);
+}
+
+}  // namespace
+
+extern "C" {
+
+mom_status_t mom_matrix_desc(int64_t rows, int64_t cols, mom_property_t property, mom_dtype_t dtype,
+                             mom_matrix_desc_t *out) {
+    if (!out) return MOM_ERR_INVALID_ARG;
+    mom_matrix_desc_t d{rows, cols, (int32_t)property, (int32_t)dtype};
+    mom_status_t st = check_desc(d);
+    if (st != MOM_OK) return st;
+    *out = d;
+    return MOM_OK;
+}
+
+mom_status_t mom_equation_plan(const mom_matrix_desc_t *chain, int32_t n_chain,
+                               const mom_matrix_desc_t *add_terms, int32_t n_add,
+                               mom_variant_t variant, mom_plan_t **out_plan) {
+    if (!out_plan || !chain || n_chain < 1 || n_add < 0 || (n_add > 0 && !add_terms)) return MOM_ERR_INVALID_ARG;
+    if ((int)variant < 0 || (int)variant > 2) return MOM_ERR_INVALID_ARG;
+    for (int i = 0; i < n_chain; ++i) {
+        mom_status_t st = check_desc(chain[i]);
+        if (st != MOM_OK) return st;
+    }
+    for (int i = 0; i < n_add; ++i) {
+        mom_status_t st = check_desc(add_terms[i]);
+        if (st != MOM_OK) return st;
+    }
+    for (int i = 0; i + 1 < n_chain; ++i)
+        if (chain[i].cols != chain[i + 1].rows) return MOM_ERR_SHAPE_MISMATCH;
+    const int64_t rows = chain[0].rows, cols = chain[n_chain - 1].cols;
+    for (int i = 0; i < n_add; ++i)
+        if (add_terms[i].rows != rows || add_terms[i].cols != cols) return MOM_ERR_SHAPE_MISMATCH;
+
+    mom_plan *p = new (std::nothrow) mom_plan();
+    if (!p) return MOM_ERR_ALLOC;
+    try {
+        p->variant = (int32_t)variant;
+        p->chain.assign(chain, chain + n_chain);
+        if (n_add) p->add.assign(add_terms, add_terms + n_add);
+        for (int i = 0; i < n_add; ++i) p->add_flops += nnz(add_terms[i]);
+
+        // identity simplification: A*I -> A, I*A -> A, I*I -> I
+        for (int i = 0; i < n_chain; ++i)
+            if (chain[i].property != MOM_IDENTITY) p->kept.push_back(i);
+        const int r = (int)p->kept.size();
+
+        if (r == 0) {
+            p->paren = "I";
+            p->product_desc = mom_matrix_desc_t{rows, cols, MOM_IDENTITY, MOM_F32};
+        } else {
+            // dynamic program over the reduced chain
+            std::vector<Node> node((size_t)r * r);
+            std::vector<uint64_t> cost((size_t)r * r, 0);
+            std::vector<int> split((size_t)r * r, -1);
+            auto at = [r](int i, int j) { return (size_t)i * r + j; };
+            for (int i = 0; i < r; ++i) {
+                const auto &d = chain[p->kept[i]];
+                node[at(i, i)] = Node{d.rows, d.cols, d.property};
+            }
+            for (int len = 2; len <= r; ++len) {
+                for (int i = 0; i + len - 1 < r; ++i) {
+                    const int j = i + len - 1;
+                    bool have = false;
+                    uint64_t best = 0;
+                    int best_k = -1;
+                    for (int k = i; k < j; ++k) {
+                        const Node &a = node[at(i, k)], &b = node[at(k + 1, j)];
+                        uint64_t m;
+                        if (!useful_mults(a.prop, b.prop, a.rows, a.cols, b.cols, &m)) { delete p; return MOM_ERR_OVERFLOW; }
+                        const u128 c = (u128)cost[at(i, k)] + cost[at(k + 1, j)] + m;
+                        if (c >= (u128)COST_LIMIT) { delete p; return MOM_ERR_OVERFLOW; }
+                        if (!have || (uint64_t)c < best) { best = (uint64_t)c; best_k = k; have = true; }
+                    }
+                    cost[at(i, j)] = best;
+                    split[at(i, j)] = best_k;
+                    const Node &a = node[at(i, best_k)], &b = node[at(best_k + 1, j)];
+                    node[at(i, j)] = Node{a.rows, b.cols, join_property(a.prop, b.prop)};
+                }
+            }
+            p->mults = cost[at(0, r - 1)];
+
+            // post-order emission of the binary products; returns the id of the value of [i, j]
+            int32_t next_id = n_chain;
+            struct Emit {
+                mom_plan *p; const std::vector<Node> &node; const std::vector<int> &split; int r; int32_t &next_id;
+                std::string &s;
+                int32_t run(int i, int j) {
+                    if (i == j) { s += std::to_string(p->kept[i]); return p->kept[i]; }
+                    const int k = split[(size_t)i * r + j];
+                    s += "(";
+                    const int32_t l = run(i, k);
+                    s += "*";
+                    const int32_t rr = run(k + 1, j);
+                    s += ")";
+                    const Node &a = node[(size_t)i * r + k], &b = node[(size_t)(k + 1) * r + j], &o = node[(size_t)i * r + j];
+                    mom::StepImpl st;
+                    std::memset(&st.pub, 0, sizeof(st.pub));
+                    st.pub.lhs = l; st.pub.rhs = rr; st.pub.out = next_id++;
+                    st.pub.lhs_property = a.prop; st.pub.rhs_property = b.prop; st.pub.out_property = o.prop;
+                    st.pub.m = a.rows; st.pub.k = a.cols; st.pub.n = b.cols;
+                    useful_mults(a.prop, b.prop, a.rows, a.cols, b.cols, &st.pub.useful_mults);
+                    const bool ta = is_tri(a.prop), tb = is_tri(b.prop);
+                    st.pub.kind = !ta && !tb ? MOM_KIND_GG : ta && !tb ? MOM_KIND_TG : !ta && tb ? MOM_KIND_GT
+                                  : a.prop == b.prop ? MOM_KIND_TT : MOM_KIND_TTMIX;
+                    p->steps.push_back(st);
+                    return st.pub.out;
+                }
+            } emit{p, node, split, r, next_id, p->paren};
+            emit.run(0, r - 1);
+            const Node &root = node[at(0, r - 1)];
+            p->product_desc = mom_matrix_desc_t{root.rows, root.cols, root.prop, MOM_F32};
+        }
+        p->result_desc = mom_matrix_desc_t{rows, cols, sum_property(p->product_desc.property, p->add), MOM_F32};
+
+        // kernel choice and workspace layout
+        const int ns = (int)p->steps.size();
+        std::vector<Interval> items;
+        items.reserve((size_t)ns * 5);
+        for (int s = 0; s < ns; ++s) {
+            mom::StepImpl &st = p->steps[s];
+            st.is_last = (s == ns - 1);
+            const int64_t m = st.pub.m, n = st.pub.n, k = st.pub.k;
+            const bool addressable = (k % 4 == 0) && (n % 4 == 0);
+            const bool worth_it = (double)m * (double)n * (double)k >= (double)(1 << 23);
+            st.pub.uses_tensor_cores =
+                (variant == MOM_VARIANT_3XTF32 && addressable && worth_it) || ((int)variant == 2 && addressable);
+            if (!st.is_last) {
+                int consumer = ns - 1;
+                for (int t = s + 1; t < ns; ++t)
+                    if (p->steps[t].pub.lhs == st.pub.out || p->steps[t].pub.rhs == st.pub.out) { consumer = t; break; }
+                items.push_back(Interval{mom::align_up((size_t)m * n * sizeof(float), mom::WS_ALIGN), s, consumer, &st.out_off, 0});
+            }
+            if (st.pub.uses_tensor_cores) {
+                const size_t ab = mom::align_up((size_t)m * k * sizeof(float), mom::WS_ALIGN);
+                const size_t bb = mom::align_up((size_t)k * n * sizeof(float), mom::WS_ALIGN);
+                items.push_back(Interval{ab, s, s, &st.a_hi_off, 0});
+                items.push_back(Interval{ab, s, s, &st.a_lo_off, 0});
+                items.push_back(Interval{bb, s, s, &st.b_hi_off, 0});
+                items.push_back(Interval{bb, s, s, &st.b_lo_off, 0});
+            }
+        }
+        p->workspace_per_instance = pack(items);
+    } catch (const std::bad_alloc &) {
+        delete p;
+        return MOM_ERR_ALLOC;
+    }
+    *out_plan = p;
+    return MOM_OK;
+}
+
+mom_status_t mom_plan_flops(const mom_plan_t *plan, uint64_t *mul_flops, uint64_t *add_flops) {
+    if (!plan) return MOM_ERR_INVALID_ARG;
+    if (mul_flops) *mul_flops = 2 * plan->mults;
+    if (add_flops) *add_flops = plan->add_flops;
+    return MOM_OK;
+}
+
+mom_status_t mom_plan_parenthesization(const mom_plan_t *plan, char *buf, size_t cap, size_t *needed) {
+    if (!plan) return MOM_ERR_INVALID_ARG;
+    const size_t need = plan->paren.size() + 1;
+    if (needed) *needed = need;
+    if (!buf || cap < need) return buf || needed ? MOM_ERR_BUFFER_TOO_SMALL : MOM_ERR_INVALID_ARG;
+    std::memcpy(buf, plan->paren.c_str(), need);
+    return MOM_OK;
+}
+
+mom_status_t mom_plan_num_steps(const mom_plan_t *plan, int32_t *n) {
+    if (!plan || !n) return MOM_ERR_INVALID_ARG;
+    *n = (int32_t)plan->steps.size();
+    return MOM_OK;
+}
+
+mom_status_t mom_plan_step(const mom_plan_t *plan, int32_t i, mom_step_t *out) {
+    if (!plan || !out || i < 0 || i >= (int32_t)plan->steps.size()) return MOM_ERR_INVALID_ARG;
+    *out = plan->steps[i].pub;
+    return MOM_OK;
+}
+
+mom_status_t mom_plan_result_desc(const mom_plan_t *plan, mom_matrix_desc_t *out) {
+    if (!plan || !out) return MOM_ERR_INVALID_ARG;
+    *out = plan->result_desc;
+    return MOM_OK;
+}
+
+mom_status_t mom_plan_workspace_bytes(const mom_plan_t *plan, int64_t batch, size_t *bytes) {
+    if (!plan || !bytes || batch < 1) return MOM_ERR_INVALID_ARG;
+    // Plans with a tensor-core step walk the instances one after the other through one instance's
+    // workspace; all-FFMA plans run up to 65535 instances per launch and keep one copy of each
+    // intermediate per instance.
+    bool any_tc = false;
+    for (const auto &s : plan->steps) any_tc |= s.pub.uses_tensor_cores != 0;
+    const int64_t group = any_tc ? 1 : (batch < 65535 ? batch : 65535);
+    *bytes = plan->workspace_per_instance * (size_t)group;
+    return MOM_OK;
+}
+
+mom_status_t mom_plan_host_staging_bytes(const mom_plan_t *plan, int64_t batch, size_t *bytes) {
+    if (!plan || !bytes || batch < 1) return MOM_ERR_INVALID_ARG;
+    size_t total = 0;
+    for (const auto &d : plan->chain)
+        if (d.property != MOM_IDENTITY) total += mom::align_up((size_t)d.rows * d.cols * sizeof(float) * batch, mom::WS_ALIGN);
+    for (const auto &d : plan->add)
+        if (d.property != MOM_IDENTITY) total += mom::align_up((size_t)d.rows * d.cols * sizeof(float) * batch, mom::WS_ALIGN);
+    total += mom::align_up((size_t)plan->result_desc.rows * plan->result_desc.cols * sizeof(float) * batch, mom::WS_ALIGN);
+    size_t ws = 0;
+    mom_plan_workspace_bytes(plan, batch, &ws);
+    total += ws;
+    *bytes = total;
+    return MOM_OK;
+}
+
+mom_status_t mom_plan_last_launch_count(const mom_plan_t *plan, int32_t *launches) {
+    if (!plan || !launches) return MOM_ERR_INVALID_ARG;
+    *launches = plan->last_launches;
+    return MOM_OK;
+}
+
+mom_status_t mom_plan_destroy(mom_plan_t *plan) {
+    if (!plan) return MOM_OK;
+    mom::destroy_device_state(plan->dev);
+    delete plan;
+    return MOM_OK;
+}
+
+const char *mom_status_string(mom_status_t s) {
+    switch (s) {
+        case MOM_OK: return "ok";
+        case MOM_ERR_INVALID_ARG: return "invalid argument";
+        case MOM_ERR_PROPERTY: return "triangular and Identity matrices must be square";
+        case MOM_ERR_DTYPE: return "unsupported element type";
+        case MOM_ERR_SHAPE_MISMATCH: return "shape mismatch";
+        case MOM_ERR_OVERFLOW: return "multiplication count overflows 63 bits";
+        case MOM_ERR_ALLOC: return "allocation failed";
+        case MOM_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
+        case MOM_ERR_ALIGNMENT: return "device pointer not 16-byte aligned";
+        case MOM_ERR_ARCH: return "device is not sm_100";
+        case MOM_ERR_CUDA: return "CUDA call failed";
+        case MOM_ERR_DEVICE_TIMEOUT: return "bounded device-side wait expired";
+        case MOM_ERR_BUFFER_TOO_SMALL: return "buffer too small";
+        case MOM_ERR_LIMIT: return "size beyond a fixed maximum";
+    }
+    return "unknown status";
+}
+
+}  // extern "C"

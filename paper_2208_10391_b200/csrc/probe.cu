@@ -1,0 +1,80 @@
+// Sustained instruction-rate probes: the denominators of the reported roofline fractions.
+#include <cuda_runtime.h>
+
+#include "mom.h"
+#include "tc_probe.h"
+
+namespace {
+
+// 16 independent FMA chains per thread keep the FP32 pipes full without touching memory.
+__global__ void __launch_bounds__(256) ffma_probe_kernel(float *out, int iters, float seed) {
+    float a[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) a[i] = seed + (float)(threadIdx.x + i);
+    const float x = 1.0000001f, y = -1.0e-7f;
+    for (int it = 0; it < iters; ++it) {
+#pragma unroll
+        for (int r = 0; r < 8; ++r)
+#pragma unroll
+            for (int i = 0; i < 16; ++i) a[i] = fmaf(a[i], x, y);
+    }
+    float s = 0.0f;
+#pragma unroll
+    for (int i = 0; i < 16; ++i) s += a[i];
+    if (s == 12345.678f) out[0] = s;     // never true in practice; keeps the chains alive
+}
+
+mom_status_t time_kernel(cudaStream_t stream, double *ms_out, void (*launch)(cudaStream_t, int, void *), int iters, void *arg) {
+    cudaEvent_t e0, e1;
+    if (cudaEventCreate(&e0) != cudaSuccess || cudaEventCreate(&e1) != cudaSuccess) return MOM_ERR_CUDA;
+    cudaEventRecord(e0, stream);
+    launch(stream, iters, arg);
+    cudaEventRecord(e1, stream);
+    cudaError_t e = cudaEventSynchronize(e1);
+    float ms = 0.0f;
+    if (e == cudaSuccess) e = cudaEventElapsedTime(&ms, e0, e1);
+    cudaEventDestroy(e0);
+    cudaEventDestroy(e1);
+    if (e != cudaSuccess || cudaGetLastError() != cudaSuccess) return MOM_ERR_CUDA;
+    *ms_out = ms;
+    return MOM_OK;
+}
+
+int g_sms = 0;
+int sm_count() {
+    if (!g_sms) {
+        int dev = 0;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&g_sms, cudaDevAttrMultiProcessorCount, dev);
+    }
+    return g_sms;
+}
+
+void launch_ffma(cudaStream_t s, int iters, void *arg) {
+    ffma_probe_kernel<<<sm_count() * 8, 256, 0, s>>>(static_cast<float *>(arg), iters, 1.0f);
+}
+
+}  // namespace
+
+extern "C" mom_status_t mom_probe_ffma_tflops(double milliseconds, void *scratch, mom_stream_t stream_, double *tflops) {
+    if (!scratch || !tflops || milliseconds <= 0) return MOM_ERR_INVALID_ARG;
+    cudaStream_t stream = reinterpret_cast<cudaStream_t>(stream_);
+    const double flops_per_iter = (double)sm_count() * 8 * 256 * 8 * 16 * 2;
+    double ms = 0;
+    int iters = 2000;
+    mom_status_t st = time_kernel(stream, &ms, launch_ffma, iters, scratch);      // warm-up and calibration
+    if (st != MOM_OK) return st;
+    st = time_kernel(stream, &ms, launch_ffma, iters, scratch);
+    if (st != MOM_OK) return st;
+    double scale = milliseconds / (ms > 1e-3 ? ms : 1e-3);
+    if (scale > 1.0) iters = (int)(iters * (scale < 100000.0 ? scale : 100000.0));
+    st = time_kernel(stream, &ms, launch_ffma, iters, scratch);
+    if (st != MOM_OK) return st;
+    *tflops = flops_per_iter * iters / (ms * 1e-3) * 1e-12;
+    return MOM_OK;
+}
+
+extern "C" mom_status_t mom_probe_tf32_tflops(double milliseconds, void *scratch, mom_stream_t stream_, double *tflops) {
+    if (!scratch || !tflops || milliseconds <= 0) return MOM_ERR_INVALID_ARG;
+    return mom::tc_probe_tf32(milliseconds, scratch, reinterpret_cast<cudaStream_t>(stream_), tflops);
+}

@@ -1,0 +1,32 @@
+// Tensor-core (tcgen05, 3xTF32) product path: host-side interface used by the launcher.
+#pragma once
+
+#include <cuda_runtime.h>
+
+#include "kernels.h"
+#include "mom_internal.h"
+
+namespace mom {
+
+struct TcStepState {
+    int4 *tiles = nullptr;      // device: work-sorted tile table {row0, col0, k_begin, k_end}
+    int num_tiles = 0;
+};
+
+struct TcPlanState {
+    bool ready = false;
+    std::vector<TcStepState> steps;     // one entry per plan step (unused for FFMA steps)
+    void *block = nullptr;              // single device allocation backing all tables
+};
+
+// Builds the tile tables of every tensor-core step (first call only; one cudaMalloc).
+mom_status_t tc_prepare(const mom_plan &p, TcPlanState &s);
+
+// Enqueues the operand splits and the product kernel of step `step`.  `before_product`, when not
+// null, is recorded on the stream between the splits and the product kernel.
+mom_status_t tc_launch_step(const mom_plan &p, TcPlanState &s, int step, const ProductArgs &a, char *workspace,
+                            int32_t *status, cudaStream_t stream, int *launches, cudaEvent_t before_product);
+
+void tc_release(TcPlanState &s);
+
+}  // namespace mom

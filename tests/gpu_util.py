@@ -1,0 +1,89 @@
+"""Helpers for the GPU parity tests: device buffers through PyTorch, calls through the C ABI."""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+import paper_2208_10391_b200 as mom
+from oracle import plan as op
+from oracle import values as ov
+import workloads as wl
+
+TOL = 1e-5          # normwise bound ||X - X_ref||_F / || |M1|...|Mn| + sum|Ti| ||_F stated for this method
+CANARY = 64         # guard floats on each side of the output buffer
+
+
+def to_device(arrs):
+    return [None if a is None else torch.from_numpy(a).cuda() for a in arrs]
+
+
+def run_equation(eq: wl.Equation, variant: int, chain=None, add=None, via: str = "device"):
+    """Plan and evaluate `eq` on the GPU; returns (X as numpy f32, plan, (chain, add) host arrays)."""
+    if chain is None:
+        chain, add = wl.generate(eq)
+    plan = mom.mom_equation_plan(eq.descs(), eq.add_descs(), variant)
+    rd = plan.result_desc()
+    batch = eq.batch
+    shape = (batch, rd.rows, rd.cols) if batch > 1 else (rd.rows, rd.cols)
+    n_out = int(np.prod(shape))
+    stream = torch.cuda.current_stream().cuda_stream
+    if via == "host":
+        stage_bytes = plan.host_staging_bytes(batch)
+        staging = torch.empty(max(stage_bytes, 256), dtype=torch.uint8, device="cuda")
+        pinned = [None if a is None else torch.from_numpy(a).pin_memory() for a in chain]
+        pinned_add = [None if a is None else torch.from_numpy(a).pin_memory() for a in add]
+        out = torch.full((n_out,), float("nan"), dtype=torch.float32).pin_memory()
+        plan.execute_host([None if t is None else t.data_ptr() for t in pinned],
+                          [None if t is None else t.data_ptr() for t in pinned_add],
+                          out.data_ptr(), batch, staging.data_ptr(), stage_bytes, stream)
+        x = out.numpy().reshape(shape).copy()
+    else:
+        dchain, dadd = to_device(chain), to_device(add)
+        ws_bytes = plan.workspace_bytes(batch)
+        ws = torch.empty(max(ws_bytes, 256), dtype=torch.uint8, device="cuda")
+        guarded = torch.full((n_out + 2 * CANARY,), float("nan"), dtype=torch.float32, device="cuda")
+        guarded[:CANARY] = 12345.0
+        guarded[-CANARY:] = 12345.0
+        out = guarded[CANARY:CANARY + n_out]
+        assert out.data_ptr() % 16 == 0
+        cp = [None if t is None else t.data_ptr() for t in dchain]
+        ap = [None if t is None else t.data_ptr() for t in dadd]
+        if batch > 1:
+            cs = [0 if t is None else t[0].numel() for t in dchain]
+            as_ = [0 if t is None else t[0].numel() for t in dadd]
+            plan.execute_batched(cp, cs, ap, as_, out.data_ptr(), rd.rows * rd.cols, batch,
+                                 ws.data_ptr() if ws_bytes else None, ws_bytes, stream)
+        else:
+            plan.execute(cp, ap, out.data_ptr(), ws.data_ptr() if ws_bytes else None, ws_bytes, stream)
+        torch.cuda.synchronize()
+        assert plan.device_status() == (0, 0), "a device-side wait timed out"
+        g = guarded.cpu().numpy()
+        assert np.all(g[:CANARY] == 12345.0) and np.all(g[-CANARY:] == 12345.0), "wrote outside the output buffer"
+        x = g[CANARY:CANARY + n_out].reshape(shape).copy()
+    assert plan.last_launch_count() >= 1
+    return x, plan, (chain, add)
+
+
+def check_against_oracle(eq: wl.Equation, x: np.ndarray, plan, chain, add, rows=None, instances=None, tol: float = TOL):
+    """Element-wise parity with the fp64 oracle; returns the worst normwise error seen."""
+    want = op.plan(eq.descs(), eq.add_descs())
+    assert plan.parenthesization() == want.paren
+    assert plan.flops() == (want.mul_flops, want.add_flops)
+    prop = plan.result_desc().property
+    assert prop == want.result_desc.prop
+    assert not np.isnan(x).any(), "part of the output was never written"
+    worst = 0.0
+    insts = range(eq.batch) if instances is None else instances
+    for b in (insts if eq.batch > 1 else [None]):
+        c = [None if a is None else (a if b is None else a[b]) for a in chain]
+        t = [None if a is None else (a if b is None else a[b]) for a in add]
+        xb = x if b is None else x[b]
+        x_ref, d = ov.evaluate(c, eq.descs(), t, eq.add_descs(), rows=rows)
+        got = xb if rows is None else xb[rows]
+        err = ov.normwise_error(got, x_ref, d)
+        assert err <= tol, f"normwise error {err:.3e} > {tol:.1e} ({eq.name}, instance {b})"
+        worst = max(worst, err)
+        # entries outside the result's structure: exactly +0.0f (all 32 bits clear)
+        mask = ov.off_structure_mask(xb.shape[0], xb.shape[1], prop)
+        assert np.all(xb.view(np.uint32)[mask] == 0), "off-structure entries must be +0.0f"
+    return worst

@@ -1,0 +1,209 @@
+"""GPU parity: every product kind, epilogue and plan shape against the fp64 oracle, through the C ABI."""
+import itertools
+
+import numpy as np
+import pytest
+
+torch = pytest.importorskip("torch")
+
+import paper_2208_10391_b200 as mom
+import workloads as wl
+from workloads import GENERAL as G, LOWER_TRI as L, UPPER_TRI as U, IDENTITY as I, Operand, Equation
+from gpu_util import run_equation, check_against_oracle, TOL
+
+pytestmark = pytest.mark.gpu
+
+VARIANTS = [mom.VARIANT_FFMA, mom.VARIANT_3XTF32_FORCE]
+VNAME = {mom.VARIANT_FFMA: "ffma", mom.VARIANT_3XTF32_FORCE: "tc", mom.VARIANT_3XTF32: "auto"}
+
+
+def both(eq, variant, **kw):
+    x, plan, (chain, add) = run_equation(eq, variant)
+    return check_against_oracle(eq, x, plan, chain, add, **kw), x, plan
+
+
+@pytest.mark.parametrize("variant", VARIANTS, ids=VNAME.get)
+@pytest.mark.parametrize("pa,pb", list(itertools.product([G, L, U], repeat=2)))
+@pytest.mark.parametrize("n", [1, 5, 64, 200, 332])
+def test_every_property_pair(pa, pb, n, variant):
+    # square n x n operands; 200 and 332 are multiples of 4 that leave ragged tiles in every tile size used
+    eq = Equation(f"pair_{pa}{pb}_{n}", 100 + n, (Operand(n, n, pa, "normal" if pa == G else "uniform"),
+                                                  Operand(n, n, pb, "normal" if pb == G else "uniform")))
+    both(eq, variant)
+
+
+@pytest.mark.parametrize("variant", VARIANTS, ids=VNAME.get)
+@pytest.mark.parametrize("m,k,n", [(64, 32, 48), (300, 520, 260), (129, 257, 65), (8, 2048, 16), (1000, 4, 12)])
+def test_rectangular_general_products(m, k, n, variant):
+    eq = Equation(f"gg_{m}x{k}x{n}", 7, (Operand(m, k, G, "normal"), Operand(k, n, G, "normal")))
+    both(eq, variant)
+
+
+@pytest.mark.parametrize("variant", VARIANTS, ids=VNAME.get)
+@pytest.mark.parametrize("pt", [L, U])
+@pytest.mark.parametrize("side", ["left", "right"])
+def test_triangular_times_rectangular(pt, side, variant):
+    if side == "left":
+        eq = Equation("tg", 8, (Operand(392, 392, pt), Operand(392, 136, G, "normal")))
+    else:
+        eq = Equation("gt", 9, (Operand(136, 392, G, "normal"), Operand(392, 392, pt)))
+    both(eq, variant)
+
+
+@pytest.mark.parametrize("variant", VARIANTS, ids=VNAME.get)
+def test_listing2_exact_values(variant):
+    # paper Listing 2: 5x5 lowerTri filled with ones times itself; every value is a small integer
+    eq = wl.config_listing2()
+    _, x, plan = both(eq, variant)
+    want = np.array([[max(i - j + 1, 0) for j in range(5)] for i in range(5)], dtype=np.float32)
+    assert np.array_equal(x, want)
+    assert plan.result_desc().property == L
+
+
+@pytest.mark.parametrize("variant", VARIANTS + [mom.VARIANT_3XTF32], ids=VNAME.get)
+def test_config_tiny_and_identity_checks(variant):
+    both(wl.config_tiny(), variant)
+    for eq in (wl.config_tiny_identity_left(), wl.config_tiny_identity_right()):
+        x, plan, (chain, add) = run_equation(eq, variant)
+        assert plan.num_steps() == 0 and plan.flops() == (0, 0)
+        src = [c for c in chain if c is not None][0]
+        assert np.array_equal(x, src)          # A*I = A and I*A = A, bit for bit
+
+
+@pytest.mark.parametrize("variant", VARIANTS + [mom.VARIANT_3XTF32], ids=VNAME.get)
+def test_config_five_general(variant):
+    both(wl.config_five_general(), variant)
+
+
+@pytest.mark.parametrize("variant", VARIANTS + [mom.VARIANT_3XTF32], ids=VNAME.get)
+def test_paper_section4_chain(variant):
+    both(wl.config_paper_chain(), variant)
+
+
+@pytest.mark.parametrize("variant", VARIANTS, ids=VNAME.get)
+@pytest.mark.parametrize("n", [256, 520])
+def test_config_property_heavy_small(n, variant):
+    both(wl.config_property_heavy(n=n), variant)
+
+
+@pytest.mark.parametrize("variant", VARIANTS, ids=VNAME.get)
+@pytest.mark.parametrize("n", [384, 776])
+def test_config_large_square_small(n, variant):
+    both(wl.config_large_square(n=n), variant)
+
+
+@pytest.mark.parametrize("variant", [mom.VARIANT_3XTF32, mom.VARIANT_FFMA], ids=VNAME.get)
+def test_config_property_heavy_full_size_sampled_rows(variant):
+    eq = wl.config_property_heavy()
+    x, plan, (chain, add) = run_equation(eq, variant)
+    rows = np.random.default_rng(0).choice(4096, size=48, replace=False)
+    rows[:4] = [0, 127, 128, 4095]
+    check_against_oracle(eq, x, plan, chain, add, rows=np.sort(rows))
+
+
+@pytest.mark.parametrize("variant", [mom.VARIANT_3XTF32], ids=VNAME.get)
+def test_config_large_square_full_size_sampled_rows(variant):
+    eq = wl.config_large_square()
+    x, plan, (chain, add) = run_equation(eq, variant)
+    rows = np.random.default_rng(1).choice(8192, size=24, replace=False)
+    rows[:4] = [0, 127, 128, 8191]
+    check_against_oracle(eq, x, plan, chain, add, rows=np.sort(rows))
+
+
+@pytest.mark.parametrize("variant", VARIANTS + [mom.VARIANT_3XTF32], ids=VNAME.get)
+def test_config_batched(variant):
+    eq = wl.config_batched(batch=37)
+    both(eq, variant)
+    eq = wl.config_batched()                      # the full 4096 instances, a sample of them checked
+    x, plan, (chain, add) = run_equation(eq, variant)
+    check_against_oracle(eq, x, plan, chain, add, instances=[0, 1, 63, 64, 2047, 4095])
+
+
+@pytest.mark.parametrize("variant", VARIANTS, ids=VNAME.get)
+def test_batched_with_padding_between_instances(variant):
+    eq = wl.config_batched(batch=5)
+    chain, add = wl.generate(eq)
+    plan = mom.mom_equation_plan(eq.descs(), eq.add_descs(), variant)
+    pad = 8
+    def padded(a):
+        flat = np.full((a.shape[0], a[0].size + pad), np.nan, dtype=np.float32)
+        flat[:, :a[0].size] = a.reshape(a.shape[0], -1)
+        return torch.from_numpy(flat).cuda()
+    dc, da = [padded(a) for a in chain], [padded(a) for a in add]
+    out = torch.full((5, 64 * 16 + pad), float("nan"), dtype=torch.float32, device="cuda")
+    wsb = plan.workspace_bytes(5)
+    ws = torch.empty(max(wsb, 256), dtype=torch.uint8, device="cuda")
+    plan.execute_batched([t.data_ptr() for t in dc], [t.shape[1] for t in dc], [t.data_ptr() for t in da],
+                         [t.shape[1] for t in da], out.data_ptr(), out.shape[1], 5, ws.data_ptr() if wsb else None, wsb,
+                         torch.cuda.current_stream().cuda_stream)
+    torch.cuda.synchronize()
+    o = out.cpu().numpy()
+    assert np.isnan(o[:, 64 * 16:]).all()          # padding untouched
+    x = o[:, :64 * 16].reshape(5, 64, 16)
+    check_against_oracle(eq, x, plan, chain, add)
+
+
+@pytest.mark.parametrize("variant", VARIANTS, ids=VNAME.get)
+def test_add_terms_and_result_structure(variant):
+    n = 72
+    # L*L + L stays lowerTri (upper part +0.0f); L*L + U becomes general; Identity term adds ones on the diagonal
+    for terms in ([Operand(n, n, L)], [Operand(n, n, U)], [Operand(n, n, I)], [Operand(n, n, L), Operand(n, n, I), Operand(n, n, L)]):
+        eq = Equation("ll_plus", 21, (Operand(n, n, L), Operand(n, n, L)), tuple(terms))
+        both(eq, variant)
+    # more Add terms than one launch fuses
+    eq = Equation("many_terms", 22, (Operand(40, 24, G), Operand(24, 56, G)), tuple(Operand(40, 56, G, "normal") for _ in range(11)))
+    both(eq, variant)
+
+
+@pytest.mark.parametrize("variant", VARIANTS, ids=VNAME.get)
+def test_zero_step_plans(variant):
+    n = 33
+    for chain, add in [((Operand(n, n, I),), ()), ((Operand(n, n, I), Operand(n, n, I)), (Operand(n, n, U),)),
+                       ((Operand(n, n, I), Operand(n, n, U), Operand(n, n, I)), (Operand(n, n, U), Operand(n, n, I))),
+                       ((Operand(n, 2 * n, G),), (Operand(n, 2 * n, G),)),
+                       ((Operand(n, n, L),), tuple(Operand(n, n, L) for _ in range(10)))]:
+        eq = Equation("zero_step", 23, chain, add)
+        both(eq, variant)
+
+
+@pytest.mark.parametrize("variant", VARIANTS, ids=VNAME.get)
+def test_random_equations(variant):
+    for seed in range(40):
+        eq = wl.random_equation(1000 + seed, max_len=5, max_dim=40, dim_multiple=4 if seed % 2 else 1)
+        both(eq, variant)
+
+
+@pytest.mark.parametrize("variant", VARIANTS, ids=VNAME.get)
+def test_host_entry_point_matches_device_entry_point(variant):
+    for eq in (wl.config_tiny(), wl.config_batched(batch=9), wl.config_property_heavy(n=264)):
+        chain, add = wl.generate(eq)
+        xd, plan, _ = run_equation(eq, variant, chain, add, via="device")
+        xh, _, _ = run_equation(eq, variant, chain, add, via="host")
+        assert np.array_equal(xd, xh)
+        check_against_oracle(eq, xh, plan, chain, add)
+
+
+def test_argument_errors_are_reported_before_any_launch():
+    eq = wl.config_tiny()
+    chain, _ = wl.generate(eq)
+    plan = mom.mom_equation_plan(eq.descs(), (), mom.VARIANT_FFMA)
+    d = [torch.from_numpy(a).cuda() for a in chain]
+    out = torch.zeros(64 * 48 + 4, dtype=torch.float32, device="cuda")
+    ws = torch.empty(plan.workspace_bytes(), dtype=torch.uint8, device="cuda")
+    ptrs = [t.data_ptr() for t in d]
+    def status(**kw):
+        args = dict(chain=ptrs, out=out.data_ptr(), ws=ws.data_ptr(), wsb=plan.workspace_bytes())
+        args.update(kw)
+        try:
+            plan.execute(args["chain"], [], args["out"], args["ws"], args["wsb"], 0)
+        except mom.MomError as e:
+            return e.status
+        return mom.OK
+    assert status(chain=[ptrs[0], None, ptrs[2]]) == mom.ERR_INVALID_ARG
+    assert status(chain=[ptrs[0] + 4, ptrs[1], ptrs[2]]) == mom.ERR_ALIGNMENT
+    assert status(out=out.data_ptr() + 4) == mom.ERR_ALIGNMENT
+    assert status(wsb=plan.workspace_bytes() - 1) == mom.ERR_WORKSPACE_TOO_SMALL
+    assert status(ws=None) == mom.ERR_WORKSPACE_TOO_SMALL
+    assert status() == mom.OK
+    torch.cuda.synchronize()
+    assert plan.device_status() == (0, 0)

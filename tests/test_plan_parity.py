@@ -1,0 +1,133 @@
+"""Plan parity (integer work, bit-exact): the library's planner against the exhaustive oracle. CPU only."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+import paper_2208_10391_b200 as mom
+from oracle import plan as op
+import workloads as wl
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def assert_same_plan(chain, add=(), variant=mom.VARIANT_3XTF32):
+    want = op.plan(chain, add)
+    got = mom.mom_equation_plan(chain, add, variant)
+    assert got.parenthesization() == want.paren
+    assert got.flops() == (want.mul_flops, want.add_flops)
+    rd = got.result_desc()
+    assert (rd.rows, rd.cols, rd.property) == (want.result_desc.rows, want.result_desc.cols, want.result_desc.prop)
+    steps = got.steps()
+    assert len(steps) == len(want.steps)
+    for g, w in zip(steps, want.steps):
+        assert (g.lhs, g.rhs, g.out, g.m, g.n, g.k) == (w.lhs, w.rhs, w.out, w.m, w.n, w.k)
+        assert (g.lhs_property, g.rhs_property, g.out_property, g.useful_mults) == (w.lhs_prop, w.rhs_prop, w.out_prop, w.mults)
+    return got, want
+
+
+def test_header_symbols_are_exported():
+    text = open(os.path.join(ROOT, "include", "mom.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    declared = set(re.findall(r"\b(mom_[a-z0-9_]+)\s*\(", text))
+    assert {"mom_matrix_desc", "mom_equation_plan", "mom_equation_execute"} <= declared
+    lib = ctypes.CDLL(mom.LIB_PATH)
+    for name in sorted(declared):
+        assert hasattr(lib, name), f"{name} is declared in mom.h but not exported"
+    assert declared == set(mom.EXPORTED)
+
+
+@pytest.mark.parametrize("eq", [
+    wl.config_tiny(), wl.config_tiny_identity_left(), wl.config_tiny_identity_right(), wl.config_five_general(),
+    wl.config_property_heavy(), wl.config_large_square(), wl.config_batched(), wl.config_paper_chain(),
+    wl.config_listing2()], ids=lambda e: e.name)
+def test_benchmark_configurations(eq):
+    for variant in (mom.VARIANT_3XTF32, mom.VARIANT_FFMA):
+        assert_same_plan(eq.descs(), eq.add_descs(), variant)
+
+
+def test_random_equations_match_the_oracle():
+    for seed in range(300):
+        eq = wl.random_equation(seed, max_len=9, max_dim=50)
+        assert_same_plan(eq.descs(), eq.add_descs())
+
+
+def test_long_chains_with_many_ties():
+    # equal dimensions everywhere: every tree of an all-general chain ties; mixed properties tie partially
+    rng = np.random.default_rng(3)
+    for _ in range(40):
+        n = int(rng.integers(2, 10))
+        chain = [(16, 16, int(rng.integers(0, 4))) for _ in range(n)]
+        assert_same_plan(chain)
+
+
+def test_identity_only_and_single_operand():
+    got, _ = assert_same_plan([(7, 7, mom.IDENTITY)] * 3)
+    assert got.parenthesization() == "I" and got.num_steps() == 0
+    got, _ = assert_same_plan([(7, 9, mom.GENERAL)])
+    assert got.parenthesization() == "0"
+    assert_same_plan([(7, 7, mom.IDENTITY)], [(7, 7, mom.IDENTITY), (7, 7, mom.UPPER_TRI)])
+
+
+@pytest.mark.parametrize("chain,add,status,code", [
+    ([(0, 3, 0)], [], mom.ERR_INVALID_ARG, "invalid_arg"),
+    ([(3, 4, 1)], [], mom.ERR_PROPERTY, "property"),
+    ([(3, 4, 3)], [], mom.ERR_PROPERTY, "property"),
+    ([(3, 4, 0), (5, 3, 0)], [], mom.ERR_SHAPE_MISMATCH, "shape_mismatch"),
+    ([(3, 4, 0)], [(3, 5, 0)], mom.ERR_SHAPE_MISMATCH, "shape_mismatch"),
+])
+def test_errors_agree_with_the_oracle(chain, add, status, code):
+    with pytest.raises(mom.MomError) as e:
+        mom.mom_equation_plan(chain, add)
+    assert e.value.status == status
+    with pytest.raises(op.OracleError) as o:
+        op.plan(chain, add)
+    assert o.value.code == code
+
+
+def test_more_errors():
+    with pytest.raises(mom.MomError) as e:
+        mom.mom_equation_plan([], [])
+    assert e.value.status == mom.ERR_INVALID_ARG
+    with pytest.raises(mom.MomError) as e:
+        mom.mom_equation_plan([(3, 3, 0, 5)], [])
+    assert e.value.status == mom.ERR_DTYPE
+    with pytest.raises(mom.MomError) as e:
+        mom.mom_matrix_desc(3, 4, mom.LOWER_TRI)
+    assert e.value.status == mom.ERR_PROPERTY
+    big = 1 << 31
+    with pytest.raises(mom.MomError) as e:
+        mom.mom_equation_plan([(big, big, 0), (big, big, 0)], [])
+    assert e.value.status == mom.ERR_OVERFLOW
+    assert mom.status_string(mom.ERR_OVERFLOW)
+
+
+def test_workspace_covers_intermediates_and_planes():
+    eq = wl.config_large_square()
+    p = mom.mom_equation_plan(eq.descs(), (), mom.VARIANT_FFMA)
+    n = 8192
+    # chain of three products: two intermediates are alive at most one at a time besides the one being read
+    assert p.workspace_bytes() == 2 * n * n * 4
+    assert all(s.uses_tensor_cores == 0 for s in p.steps())
+    p = mom.mom_equation_plan(eq.descs(), (), mom.VARIANT_3XTF32)
+    assert all(s.uses_tensor_cores == 1 for s in p.steps())
+    assert p.workspace_bytes() >= 2 * n * n * 4 + 4 * n * n * 4
+    # shapes TMA cannot address fall back to FFMA; tiny products too
+    p = mom.mom_equation_plan([(5, 5, 1), (5, 5, 1)], (), mom.VARIANT_3XTF32_FORCE)
+    assert p.step(0).uses_tensor_cores == 0
+    p = mom.mom_equation_plan(wl.config_tiny().descs(), (), mom.VARIANT_3XTF32)
+    assert all(s.uses_tensor_cores == 0 for s in p.steps())
+    p = mom.mom_equation_plan(wl.config_tiny().descs(), (), mom.VARIANT_3XTF32_FORCE)
+    assert all(s.uses_tensor_cores == 1 for s in p.steps())
+    assert mom.mom_equation_plan(wl.config_tiny_identity_left().descs()).workspace_bytes() == 0
+
+
+def test_step_kinds():
+    L, U, G = mom.LOWER_TRI, mom.UPPER_TRI, mom.GENERAL
+    cases = {(G, G): mom.KIND_GG, (L, G): mom.KIND_TG, (U, G): mom.KIND_TG, (G, L): mom.KIND_GT, (G, U): mom.KIND_GT,
+             (L, L): mom.KIND_TT, (U, U): mom.KIND_TT, (L, U): mom.KIND_TTMIX, (U, L): mom.KIND_TTMIX}
+    for (a, b), kind in cases.items():
+        p = mom.mom_equation_plan([(8, 8, a), (8, 8, b)])
+        assert p.step(0).kind == kind
