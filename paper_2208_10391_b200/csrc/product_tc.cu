@@ -1,9 +1,578 @@
-// placeholder until the tensor-core kernel lands
+// Tensor-core product kernel: C = A*B (+ Add terms) with f32-level accuracy from three tcgen05
+// kind::tf32 MMAs per k-step (3xTF32): with a = a_hi + a_lo and b = b_hi + b_lo (both halves exactly
+// representable in tf32), C accumulates a_lo*b_hi + a_hi*b_lo + a_hi*b_hi in f32 in tensor memory.
+//
+// Data flow of one product step
+//   1. split_planes_kernel writes the hi and lo planes of A (m x k, as stored) and of B TRANSPOSED
+//      (n x k), so that both MMA operands are K-major.  Blocks that lie wholly outside a triangular
+//      operand's structure are skipped: no tile ever reads them.
+//   2. product_tc_kernel, persistent, one CTA per SM, walks a work-sorted tile table.  Per tile:
+//        warp 0   TMA producer: per k-block loads A_hi, A_lo (128 rows x 16 k) and Bt_hi, Bt_lo
+//                 (256 rows x 16 k), 64-byte rows with the 64B swizzle, into a 4-stage ring;
+//        warp 1   MMA issuer: 2 k-steps x 3 MMAs (M128 N256 K8) per stage into one of two 256-column
+//                 accumulators in tensor memory; tcgen05.commit releases the stage / publishes the tile;
+//        warps 2-5 epilogue: tcgen05.ld 32 columns at a time, Add terms, structure mask, swizzled
+//                 staging in shared memory, TMA store (coalesced, clipped at the matrix edge).
+//      The k-range of a tile is the intersection of the operands' structural ranges, so all-zero
+//      blocks of triangular operands are never loaded or multiplied, and structurally-zero output
+//      tiles are only zero-filled.
+// Every wait is bounded: after a time limit the CTA records MOM_ERR_DEVICE_TIMEOUT and leaves.
+#include <algorithm>
+#include <cstring>
+#include <vector>
+
+#include <cuda.h>
+
 #include "product_tc.h"
-namespace mom {
-mom_status_t tc_prepare(const mom_plan &, TcPlanState &) { return MOM_ERR_CUDA; }
-mom_status_t tc_launch_step(const mom_plan &, TcPlanState &, int, const ProductArgs &, char *, int32_t *, cudaStream_t, int *, cudaEvent_t) { return MOM_ERR_CUDA; }
-void tc_release(TcPlanState &) {}
-}
 #include "tc_probe.h"
-namespace mom { mom_status_t tc_probe_tf32(double, void *, cudaStream_t, double *) { return MOM_ERR_CUDA; } }
+#include "tc_ptx.cuh"
+
+namespace mom {
+
+namespace {
+
+constexpr int BM = TC_BM, BN = TC_BN;
+constexpr int BK = 16;                       // f32 elements per pipeline stage (two K=8 MMA steps)
+constexpr int STAGES = 4;
+constexpr int A_PLANE_BYTES = BM * BK * 4;   // 8 KiB
+constexpr int B_PLANE_BYTES = BN * BK * 4;   // 16 KiB
+constexpr int STAGE_BYTES = 2 * A_PLANE_BYTES + 2 * B_PLANE_BYTES;   // 48 KiB
+constexpr int EPI_BOX_BYTES = 32 * 32 * 4;   // 32 rows x 32 columns staged per TMA store
+constexpr int EPI_BYTES = 4 * 2 * EPI_BOX_BYTES;                     // 4 warps x 2 buffers
+constexpr int NUM_BARRIERS = 2 * STAGES + 4 + 1;
+constexpr int SMEM_BYTES = 1024 + STAGES * STAGE_BYTES + EPI_BYTES + 256;
+constexpr int THREADS = 192;
+constexpr uint32_t TMEM_COLS = 512;          // two accumulators of BN columns
+constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;   // 2 s: far beyond any legitimate wait
+
+static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
+static_assert(SPLIT_BLOCK % BM == 0 && SPLIT_BLOCK % BN == 0, "split blocks must cover whole tiles");
+
+struct Shared {
+    uint32_t stage[STAGES];      // shared-space byte address of each stage
+    uint32_t epi;                // staging buffers
+    uint32_t full[STAGES], empty[STAGES], tmem_full[2], tmem_empty[2], drain;
+    uint32_t tmem_slot;
+    volatile int *abort_flag;
+};
+
+__device__ __forceinline__ unsigned long long global_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+
+// Bounded wait: false when the limit was reached (records the failure) or another role gave up.
+__device__ __forceinline__ bool wait_barrier(uint32_t bar, uint32_t parity, volatile int *abort_flag, int32_t *status, int detail) {
+    unsigned long long start = 0;
+    for (uint32_t i = 0;; ++i) {
+        if (ptx::mbar_try_wait(bar, parity)) return true;
+        if ((i & 63) == 63) {
+            if (*abort_flag) return false;
+            const unsigned long long now = global_ns();
+            if (start == 0) start = now;
+            else if (now - start > WAIT_LIMIT_NS) break;
+        }
+    }
+    if (atomicCAS(status, 0, (int)MOM_ERR_DEVICE_TIMEOUT) == 0) status[1] = detail;
+    *abort_flag = 1;
+    __threadfence_block();
+    return false;
+}
+
+struct TcParams {
+    const int4 *tiles;
+    int num_tiles;
+    int m, n;
+    int pout;
+    AddTerms add;
+    int32_t *status;
+};
+
+// K-major operand tile with 64-byte rows under the 64B swizzle: 8-row groups are 512 bytes apart; a
+// K=8 step is 32 bytes along the row.
+__device__ __forceinline__ uint64_t kmajor_desc(uint32_t tile, int kstep) {
+    return ptx::smem_desc(tile + kstep * 32, 16, 512, ptx::SWIZZLE_64B);
+}
+
+__global__ void __launch_bounds__(THREADS, 1)
+product_tc_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_constant__ CUtensorMap map_a_lo,
+                  const __grid_constant__ CUtensorMap map_b_hi, const __grid_constant__ CUtensorMap map_b_lo,
+                  const __grid_constant__ CUtensorMap map_c, const TcParams prm) {
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ int abort_word;
+    const uint32_t base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t bars = base + STAGES * STAGE_BYTES + EPI_BYTES;
+    Shared sh;
+#pragma unroll
+    for (int s = 0; s < STAGES; ++s) {
+        sh.stage[s] = base + s * STAGE_BYTES;
+        sh.full[s] = bars + 8 * s;
+        sh.empty[s] = bars + 8 * (STAGES + s);
+    }
+    sh.epi = base + STAGES * STAGE_BYTES;
+    sh.tmem_full[0] = bars + 8 * (2 * STAGES);
+    sh.tmem_full[1] = bars + 8 * (2 * STAGES + 1);
+    sh.tmem_empty[0] = bars + 8 * (2 * STAGES + 2);
+    sh.tmem_empty[1] = bars + 8 * (2 * STAGES + 3);
+    sh.drain = bars + 8 * (2 * STAGES + 4);
+    sh.tmem_slot = bars + 8 * NUM_BARRIERS;
+    sh.abort_flag = &abort_word;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    if (threadIdx.x == 0) {
+        abort_word = 0;
+#pragma unroll
+        for (int s = 0; s < STAGES; ++s) { ptx::mbar_init(sh.full[s], 1); ptx::mbar_init(sh.empty[s], 1); }
+        ptx::mbar_init(sh.tmem_full[0], 1);
+        ptx::mbar_init(sh.tmem_full[1], 1);
+        ptx::mbar_init(sh.tmem_empty[0], 4);
+        ptx::mbar_init(sh.tmem_empty[1], 4);
+        ptx::mbar_init(sh.drain, 1);
+        ptx::fence_barrier_init();
+    }
+    if (warp == 1) {
+        ptx::tmem_alloc(sh.tmem_slot, TMEM_COLS);
+        ptx::tmem_relinquish();
+    }
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    ptx::tc_fence_after_sync();
+    uint32_t tmem_base;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(tmem_base) : "r"(sh.tmem_slot));
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer
+        uint32_t it = 0;
+        bool ok = true;
+        for (int t = blockIdx.x; t < prm.num_tiles && ok; t += gridDim.x) {
+            const int4 tile = prm.tiles[t];
+            for (int kb = tile.z; kb < tile.w; kb += BK, ++it) {
+                const int s = it % STAGES;
+                const uint32_t parity = ((it / STAGES) & 1) ^ 1;
+                if (lane == 0) ok = wait_barrier(sh.empty[s], parity, sh.abort_flag, prm.status, (1 << 24) | (s << 16) | (t & 0xFFFF));
+                ok = __shfl_sync(0xffffffffu, ok, 0);
+                if (!ok) break;
+                if (lane == 0) ptx::mbar_arrive_expect_tx(sh.full[s], STAGE_BYTES);
+                __syncwarp();
+                if (lane == 0) ptx::tma_load_2d(sh.stage[s], &map_a_hi, kb, tile.x, sh.full[s]);
+                else if (lane == 1) ptx::tma_load_2d(sh.stage[s] + A_PLANE_BYTES, &map_a_lo, kb, tile.x, sh.full[s]);
+                else if (lane == 2) ptx::tma_load_2d(sh.stage[s] + 2 * A_PLANE_BYTES, &map_b_hi, kb, tile.y, sh.full[s]);
+                else if (lane == 3) ptx::tma_load_2d(sh.stage[s] + 2 * A_PLANE_BYTES + B_PLANE_BYTES, &map_b_lo, kb, tile.y, sh.full[s]);
+            }
+        }
+        // On the failure path, let loads that are still in flight land before the CTA exits.
+        if (*sh.abort_flag && lane == 0) {
+            for (uint32_t back = 1; back <= (uint32_t)STAGES && back <= it; ++back) {
+                const uint32_t j = it - back;
+                for (uint32_t i = 0; i < (1u << 20); ++i)
+                    if (ptx::mbar_try_wait(sh.full[j % STAGES], (j / STAGES) & 1)) break;
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer (one thread)
+        if (lane == 0) {
+            constexpr uint32_t idesc = ptx::instr_desc_tf32(BM, BN, 0, 0);
+            uint32_t it = 0, acc_it = 0;
+            bool ok = true;
+            for (int t = blockIdx.x; t < prm.num_tiles && ok; t += gridDim.x) {
+                const int4 tile = prm.tiles[t];
+                if (tile.z >= tile.w) continue;                  // structurally zero: nothing to multiply
+                const uint32_t acc = acc_it & 1;
+                ok = wait_barrier(sh.tmem_empty[acc], ((acc_it >> 1) & 1) ^ 1, sh.abort_flag, prm.status, (2 << 24) | (acc << 16) | (t & 0xFFFF));
+                if (!ok) break;
+                ptx::tc_fence_after_sync();
+                const uint32_t d = tmem_base + acc * BN;
+                uint32_t accumulate = 0;
+                for (int kb = tile.z; kb < tile.w; kb += BK, ++it) {
+                    const int s = it % STAGES;
+                    ok = wait_barrier(sh.full[s], (it / STAGES) & 1, sh.abort_flag, prm.status, (3 << 24) | (s << 16) | (t & 0xFFFF));
+                    if (!ok) break;
+                    ptx::tc_fence_after_sync();
+                    const uint32_t a_hi = sh.stage[s], a_lo = a_hi + A_PLANE_BYTES;
+                    const uint32_t b_hi = a_hi + 2 * A_PLANE_BYTES, b_lo = b_hi + B_PLANE_BYTES;
+#pragma unroll
+                    for (int ks = 0; ks < BK / 8; ++ks) {
+                        const uint64_t da_hi = kmajor_desc(a_hi, ks), da_lo = kmajor_desc(a_lo, ks);
+                        const uint64_t db_hi = kmajor_desc(b_hi, ks), db_lo = kmajor_desc(b_lo, ks);
+                        ptx::mma_tf32(d, da_lo, db_hi, idesc, accumulate);      // small terms first
+                        ptx::mma_tf32(d, da_hi, db_lo, idesc, 1);
+                        ptx::mma_tf32(d, da_hi, db_hi, idesc, 1);
+                        accumulate = 1;
+                    }
+                    ptx::mma_commit(sh.empty[s]);                 // stage reusable once these MMAs have read it
+                }
+                if (!ok) break;
+                ptx::mma_commit(sh.tmem_full[acc]);               // accumulator complete
+                ++acc_it;
+            }
+            if (*sh.abort_flag) {                                 // failure path: let issued MMAs finish before TMEM is freed
+                ptx::mma_commit(sh.drain);
+                for (uint32_t i = 0; i < (1u << 20); ++i)
+                    if (ptx::mbar_try_wait(sh.drain, 0)) break;
+            }
+        }
+        __syncwarp();
+    } else {
+        // ------------------------------------------------------------------ epilogue (warps 2..5)
+        const int q = warp & 3;                                   // TMEM lane quarter this warp may read
+        const uint32_t stage_buf = sh.epi + (warp - 2) * 2 * EPI_BOX_BYTES;
+        uint32_t acc_it = 0, store_it = 0;
+        bool ok = true;
+        for (int t = blockIdx.x; t < prm.num_tiles && ok; t += gridDim.x) {
+            const int4 tile = prm.tiles[t];
+            const bool zero_tile = tile.z >= tile.w;
+            const uint32_t acc = acc_it & 1;
+            if (!zero_tile) {
+                ok = wait_barrier(sh.tmem_full[acc], (acc_it >> 1) & 1, sh.abort_flag, prm.status, (4 << 24) | (acc << 16) | (t & 0xFFFF));
+                if (!ok) break;
+                ptx::tc_fence_after_sync();
+            }
+            const int r = tile.x + q * 32 + lane;                 // this thread's output row
+            const int rows_left = prm.m - (tile.x + q * 32);      // rows of this warp's slab inside the matrix
+#pragma unroll 1
+            for (int c = 0; c < BN / 32; ++c) {
+                const int col0 = tile.y + c * 32;
+                if (col0 >= prm.n) break;
+                float v[32];
+                if (!zero_tile) {
+                    ptx::tmem_ld_32cols(tmem_base + acc * BN + c * 32 + ((uint32_t)(q * 32) << 16), v);
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) v[j] = 0.0f;
+                }
+                if (rows_left > 0) {
+                    const bool row_ok = r < prm.m;
+                    // Add terms, left to right
+                    for (int a = 0; a < prm.add.count; ++a) {
+                        const float *p = prm.add.ptr[a];
+                        if (p) {
+                            if (row_ok) {
+                                const float4 *src = reinterpret_cast<const float4 *>(p + (long long)r * prm.n + col0);
+#pragma unroll
+                                for (int j = 0; j < 8; ++j) {
+                                    if (col0 + 4 * j < prm.n) {
+                                        const float4 x = __ldg(src + j);
+                                        v[4 * j] += x.x; v[4 * j + 1] += x.y; v[4 * j + 2] += x.z; v[4 * j + 3] += x.w;
+                                    }
+                                }
+                            }
+                        } else {                                   // Identity term
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) v[j] += (col0 + j == r) ? 1.0f : 0.0f;
+                        }
+                    }
+                    if (prm.pout != MOM_GENERAL) {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) v[j] = in_structure(prm.pout, r, col0 + j) ? v[j] : 0.0f;
+                    }
+                    // staging buffer: 32 rows of 128 bytes, 16-byte chunk j of row i stored at chunk j ^ (i & 7)
+                    const uint32_t buf = stage_buf + (store_it & 1) * EPI_BOX_BYTES;
+                    if (lane == 0) ptx::tma_store_wait_read<1>();  // the store that last read this buffer is done
+                    __syncwarp();
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        const uint32_t dst = buf + lane * 128 + ((j ^ (lane & 7)) << 4);
+                        asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "f"(v[4 * j]), "f"(v[4 * j + 1]),
+                                     "f"(v[4 * j + 2]), "f"(v[4 * j + 3]) : "memory");
+                    }
+                    ptx::fence_proxy_async_smem();
+                    __syncwarp();
+                    if (lane == 0) {
+                        ptx::tma_store_2d(&map_c, col0, tile.x + q * 32, buf);
+                        ptx::tma_store_commit();
+                    }
+                    ++store_it;
+                }
+            }
+            if (!zero_tile) {
+                ptx::tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(sh.tmem_empty[acc]);
+                ++acc_it;
+            }
+        }
+        if (lane == 0) ptx::tma_store_wait_all();
+    }
+
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    ptx::tc_fence_after_sync();
+    if (warp == 1) ptx::tmem_dealloc(tmem_base, TMEM_COLS);
+}
+
+// hi = rna_tf32(a), lo = rna_tf32(a - hi) for every block of SPLIT_BLOCK x SPLIT_BLOCK entries that
+// intersects the operand's structure.  The planes keep the operand's layout (rows x cols) or, with
+// TRANSPOSE, hold the transposed operand (cols x rows).  rows and cols are multiples of 4 where a
+// vector access needs it: the plain path requires cols % 4 == 0.
+template <bool TRANSPOSE>
+__global__ void __launch_bounds__(256)
+split_planes_kernel(const float *__restrict__ src, float *__restrict__ hi, float *__restrict__ lo, int rows, int cols, int prop) {
+    const int br = blockIdx.y * SPLIT_BLOCK, bc = blockIdx.x * SPLIT_BLOCK;
+    if (prop == MOM_LOWER_TRI && bc > br + SPLIT_BLOCK - 1) return;     // block wholly above the diagonal
+    if (prop == MOM_UPPER_TRI && br > bc + SPLIT_BLOCK - 1) return;     // wholly below
+    const int r1 = min(br + SPLIT_BLOCK, rows), c1 = min(bc + SPLIT_BLOCK, cols);
+    if (!TRANSPOSE) {
+        const int vec_per_row = (c1 - bc) >> 2;
+        const int total = (r1 - br) * vec_per_row;
+        for (int e = threadIdx.x; e < total; e += blockDim.x) {
+            const int r = br + e / vec_per_row, c = bc + ((e % vec_per_row) << 2);
+            const size_t off = (size_t)r * cols + c;
+            const float4 a = __ldg(reinterpret_cast<const float4 *>(src + off));
+            float4 h, l;
+            h.x = ptx::to_tf32(a.x); h.y = ptx::to_tf32(a.y); h.z = ptx::to_tf32(a.z); h.w = ptx::to_tf32(a.w);
+            l.x = ptx::to_tf32(a.x - h.x); l.y = ptx::to_tf32(a.y - h.y); l.z = ptx::to_tf32(a.z - h.z); l.w = ptx::to_tf32(a.w - h.w);
+            *reinterpret_cast<float4 *>(hi + off) = h;
+            *reinterpret_cast<float4 *>(lo + off) = l;
+        }
+    } else {
+        __shared__ float tile[32][33];
+        const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;           // 32 x 8 threads
+        for (int sr = br; sr < r1; sr += 32) {
+            for (int sc = bc; sc < c1; sc += 32) {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int r = sr + ty + 8 * i, c = sc + tx;
+                    tile[ty + 8 * i][tx] = (r < rows && c < cols) ? __ldg(src + (size_t)r * cols + c) : 0.0f;
+                }
+                __syncthreads();
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int c = sc + ty + 8 * i, r = sr + tx;               // plane entry (c, r), r contiguous
+                    if (c < cols && r < rows) {
+                        const float a = tile[tx][ty + 8 * i];
+                        const float h = ptx::to_tf32(a);
+                        hi[(size_t)c * rows + r] = h;
+                        lo[(size_t)c * rows + r] = ptx::to_tf32(a - h);
+                    }
+                }
+                __syncthreads();
+            }
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// host side
+// ---------------------------------------------------------------------------------------------
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
+                                  const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+// 2-D f32 row-major matrix (rows x cols), box of box_rows x box_cols elements
+bool make_map(CUtensorMap *map, const void *ptr, int rows, int cols, int box_rows, int box_cols, CUtensorMapSwizzle swz) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)cols * sizeof(float)};
+    const cuuint32_t box[2] = {(cuuint32_t)box_cols, (cuuint32_t)box_rows};
+    const cuuint32_t elem[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void *>(ptr), dims, strides, box, elem,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+int g_sm_count = 0;
+bool g_attr_set = false;
+
+}  // namespace
+
+mom_status_t tc_prepare(const mom_plan &p, TcPlanState &s) {
+    if (s.ready) return MOM_OK;
+    const int ns = (int)p.steps.size();
+    s.steps.assign(ns, TcStepState{});
+    std::vector<std::vector<int4>> tables(ns);
+    size_t total = 0;
+    for (int i = 0; i < ns; ++i) {
+        const mom_step_t &st = p.steps[i].pub;
+        if (!st.uses_tensor_cores) continue;
+        const int m = (int)st.m, n = (int)st.n, k = (int)st.k;
+        std::vector<int4> &tab = tables[i];
+        for (int r0 = 0; r0 < m; r0 += BM)
+            for (int c0 = 0; c0 < n; c0 += BN) {
+                int klo, khi;
+                tile_k_range(st.lhs_property, st.rhs_property, r0, std::min(r0 + BM, m), c0, std::min(c0 + BN, n), k, &klo, &khi);
+                if (klo >= khi) { klo = 0; khi = 0; }
+                klo = klo / BK * BK;                      // leading extra elements are stored zeros
+                tab.push_back(make_int4(r0, c0, klo, khi));
+            }
+        // heaviest tiles first so that the persistent CTAs finish together; zero tiles last
+        std::stable_sort(tab.begin(), tab.end(), [](const int4 &a, const int4 &b) { return (a.w - a.z) > (b.w - b.z); });
+        total += tab.size();
+    }
+    if (total == 0) { s.ready = true; return MOM_OK; }
+    if (cudaMalloc(&s.block, total * sizeof(int4)) != cudaSuccess) return MOM_ERR_ALLOC;
+    int4 *cur = static_cast<int4 *>(s.block);
+    for (int i = 0; i < ns; ++i) {
+        if (tables[i].empty()) continue;
+        if (cudaMemcpy(cur, tables[i].data(), tables[i].size() * sizeof(int4), cudaMemcpyHostToDevice) != cudaSuccess) {
+            cudaFree(s.block);
+            s.block = nullptr;
+            return MOM_ERR_CUDA;
+        }
+        s.steps[i].tiles = cur;
+        s.steps[i].num_tiles = (int)tables[i].size();
+        cur += tables[i].size();
+    }
+    s.ready = true;
+    return MOM_OK;
+}
+
+void tc_release(TcPlanState &s) {
+    if (s.block) cudaFree(s.block);
+    s.block = nullptr;
+    s.steps.clear();
+    s.ready = false;
+}
+
+mom_status_t tc_launch_step(const mom_plan &p, TcPlanState &s, int step, const ProductArgs &a, char *workspace,
+                            int32_t *status, cudaStream_t stream, int *launches, cudaEvent_t before_product) {
+    const StepImpl &st = p.steps[step];
+    if (!s.ready || step >= (int)s.steps.size() || !s.steps[step].tiles) return MOM_ERR_INVALID_ARG;
+    if (!g_sm_count) {
+        int dev = 0;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&g_sm_count, cudaDevAttrMultiProcessorCount, dev);
+    }
+    if (!g_attr_set) {
+        if (cudaFuncSetAttribute(product_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess)
+            return MOM_ERR_CUDA;
+        g_attr_set = true;
+    }
+    float *a_hi = reinterpret_cast<float *>(workspace + st.a_hi_off), *a_lo = reinterpret_cast<float *>(workspace + st.a_lo_off);
+    float *b_hi = reinterpret_cast<float *>(workspace + st.b_hi_off), *b_lo = reinterpret_cast<float *>(workspace + st.b_lo_off);
+
+    auto blocks = [](int x) { return (x + SPLIT_BLOCK - 1) / SPLIT_BLOCK; };
+    split_planes_kernel<false><<<dim3(blocks(a.k), blocks(a.m)), 256, 0, stream>>>(a.A, a_hi, a_lo, a.m, a.k, a.pa);
+    split_planes_kernel<true><<<dim3(blocks(a.n), blocks(a.k)), 256, 0, stream>>>(a.B, b_hi, b_lo, a.k, a.n, a.pb);
+    if (cudaGetLastError() != cudaSuccess) return MOM_ERR_CUDA;
+    if (before_product) cudaEventRecord(before_product, stream);
+
+    // A planes are m x k, B planes are n x k (transposed): both K-major with 16-element (64-byte) box rows
+    CUtensorMap ma_hi, ma_lo, mb_hi, mb_lo, mc;
+    bool ok = make_map(&ma_hi, a_hi, a.m, a.k, BM, BK, CU_TENSOR_MAP_SWIZZLE_64B) &&
+              make_map(&ma_lo, a_lo, a.m, a.k, BM, BK, CU_TENSOR_MAP_SWIZZLE_64B) &&
+              make_map(&mb_hi, b_hi, a.n, a.k, BN, BK, CU_TENSOR_MAP_SWIZZLE_64B) &&
+              make_map(&mb_lo, b_lo, a.n, a.k, BN, BK, CU_TENSOR_MAP_SWIZZLE_64B) &&
+              make_map(&mc, a.C, a.m, a.n, 32, 32, CU_TENSOR_MAP_SWIZZLE_128B);
+    if (!ok) return MOM_ERR_CUDA;
+
+    TcParams prm;
+    prm.tiles = s.steps[step].tiles;
+    prm.num_tiles = s.steps[step].num_tiles;
+    prm.m = a.m;
+    prm.n = a.n;
+    prm.pout = a.pout;
+    prm.add = a.add;
+    prm.status = status;
+    const int grid = std::min(prm.num_tiles, g_sm_count);
+    product_tc_kernel<<<grid, THREADS, SMEM_BYTES, stream>>>(ma_hi, ma_lo, mb_hi, mb_lo, mc, prm);
+    if (cudaGetLastError() != cudaSuccess) return MOM_ERR_CUDA;
+    *launches = 3;
+    return MOM_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// TF32 rate probe: every SM issues M128 N256 K8 kind::tf32 MMAs on resident shared-memory tiles.
+// ---------------------------------------------------------------------------------------------
+namespace {
+
+constexpr int PROBE_BATCH = 64;                 // MMAs between commits
+constexpr int PROBE_SMEM = 1024 + 8192 + 16384 + 64;
+
+__global__ void __launch_bounds__(128, 1) tf32_probe_kernel(int batches, int32_t *status) {
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ int abort_word;
+    const uint32_t base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t a_tile = base, b_tile = base + 8192, bar0 = base + 8192 + 16384, bar1 = bar0 + 8, slot = bar0 + 16;
+    // finite, tf32-representable operand values
+    for (int i = threadIdx.x; i < (8192 + 16384) / 4; i += blockDim.x) {
+        const float v = (float)((i * 37 + blockIdx.x) % 61 - 30) * 0.03125f;
+        asm volatile("st.shared.f32 [%0], %1;" ::"r"(base + 4 * i), "f"(v) : "memory");
+    }
+    if (threadIdx.x == 0) {
+        abort_word = 0;
+        ptx::mbar_init(bar0, 1);
+        ptx::mbar_init(bar1, 1);
+        ptx::fence_barrier_init();
+    }
+    ptx::fence_proxy_async_smem();
+    if (threadIdx.x < 32) {
+        ptx::tmem_alloc(slot, 256);
+        ptx::tmem_relinquish();
+    }
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    ptx::tc_fence_after_sync();
+    uint32_t tmem_base;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(tmem_base) : "r"(slot));
+    if (threadIdx.x == 0) {
+        constexpr uint32_t idesc = ptx::instr_desc_tf32(128, 256, 0, 0);
+        const uint64_t da = kmajor_desc(a_tile, 0), db = kmajor_desc(b_tile, 0);
+        bool ok = true;
+        for (int b = 0; b < batches && ok; ++b) {
+            for (int i = 0; i < PROBE_BATCH; ++i) ptx::mma_tf32(tmem_base, da, db, idesc, (b | i) ? 1u : 0u);
+            ptx::mma_commit((b & 1) ? bar1 : bar0);
+            if (b >= 1) ok = wait_barrier(((b - 1) & 1) ? bar1 : bar0, ((b - 1) >> 1) & 1, &abort_word, status, (5 << 24) | (b & 0xFFFF));
+        }
+        if (ok && batches > 0) wait_barrier(((batches - 1) & 1) ? bar1 : bar0, ((batches - 1) >> 1) & 1, &abort_word, status, (6 << 24));
+    }
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    ptx::tc_fence_after_sync();
+    if (threadIdx.x < 32) ptx::tmem_dealloc(tmem_base, 256);
+}
+
+}  // namespace
+
+mom_status_t tc_probe_tf32(double milliseconds, void *scratch, cudaStream_t stream, double *tflops) {
+    int dev = 0, sms = 0, major = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return MOM_ERR_CUDA;
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+    if (major != 10) return MOM_ERR_ARCH;
+    if (cudaFuncSetAttribute(tf32_probe_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, PROBE_SMEM) != cudaSuccess) return MOM_ERR_CUDA;
+    int32_t *status = static_cast<int32_t *>(scratch);
+    if (cudaMemsetAsync(status, 0, 16, stream) != cudaSuccess) return MOM_ERR_CUDA;
+    cudaEvent_t e0, e1;
+    if (cudaEventCreate(&e0) != cudaSuccess || cudaEventCreate(&e1) != cudaSuccess) return MOM_ERR_CUDA;
+    auto run = [&](int batches, float *ms) -> bool {
+        cudaEventRecord(e0, stream);
+        tf32_probe_kernel<<<sms, 128, PROBE_SMEM, stream>>>(batches, status);
+        cudaEventRecord(e1, stream);
+        return cudaEventSynchronize(e1) == cudaSuccess && cudaGetLastError() == cudaSuccess &&
+               cudaEventElapsedTime(ms, e0, e1) == cudaSuccess;
+    };
+    float ms = 0.0f;
+    int batches = 256;
+    bool ok = run(batches, &ms) && run(batches, &ms);
+    if (ok) {
+        double scale = milliseconds / (ms > 1e-3f ? ms : 1e-3f);
+        if (scale > 1.0) batches = (int)(batches * (scale < 50000.0 ? scale : 50000.0));
+        ok = run(batches, &ms);
+    }
+    int32_t host[2] = {0, 0};
+    if (ok) ok = cudaMemcpy(host, status, sizeof(host), cudaMemcpyDeviceToHost) == cudaSuccess;
+    cudaEventDestroy(e0);
+    cudaEventDestroy(e1);
+    if (!ok) return MOM_ERR_CUDA;
+    if (host[0] != 0) return MOM_ERR_DEVICE_TIMEOUT;
+    *tflops = (double)sms * batches * PROBE_BATCH * 2.0 * 128 * 256 * 8 / (ms * 1e-3) * 1e-12;
+    return MOM_OK;
+}
+
+}  // namespace mom
