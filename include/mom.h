@@ -195,6 +195,38 @@ mom_status_t mom_plan_destroy(mom_plan_t *plan);   /* NULL is accepted */
 
 const char *mom_status_string(mom_status_t status);
 
+/* One product C = A * B on the tensor-core (3xTF32) kernel without any allocation.  (The paper has no
+ * counterpart: this entry point exists for callers of this library, not for the method.)
+ *
+ * Who needs it: code that may not call cudaMalloc at the point where it needs a product -- for
+ * example a plug-in running inside a host application that owns and budgets all device memory, or
+ * a latency-critical loop where an allocation (which may synchronise the device) is not acceptable,
+ * and that has no spare buffer to lend as workspace.  mom_equation_execute needs a caller workspace
+ * and creates a small plan-owned block on first use; this call needs neither.  Its scratch (the hi
+ * and lo planes of both operands, the tile table, a status word) is a fixed array of 16 MiB + 33 KiB
+ * built into the library; every GPU that loads the library holds that much memory until the process
+ * exits.
+ *
+ *   A (m x k), B (k x n), C (m x n): device, dense row-major f32, 16-byte aligned; k and n multiples of 4.
+ *   pa, pb: MOM_GENERAL, MOM_LOWER_TRI or MOM_UPPER_TRI (triangular operands square, zeros stored
+ *           outside the triangle); C gets the product's structure (L*L lower, U*U upper, else general)
+ *           with +0.0f outside it.
+ *   device_status: optional device pointer to 4 ints that the caller has zeroed; receives
+ *           {MOM_ERR_DEVICE_TIMEOUT, detail} if a bounded device-side wait expires.  NULL: an internal
+ *           word is used (cleared by each call) and the outcome cannot be read back.
+ * Limits: 2*(m*k + k*n)*4 bytes (each plane rounded up to 256 bytes) must fit in 16 MiB -- e.g.
+ * 1024 x 1024 times 1024 x 1024 -- and the output may have at most 2048 tiles of 128 x 256; beyond that
+ * MOM_ERR_LIMIT is returned and nothing is enqueued.  Other errors: INVALID_ARG, PROPERTY, ALIGNMENT,
+ * ARCH, CUDA.
+ * The first call on each device looks up the array's device address (with that device current); make
+ * that first call before any stream capture.  No cudaMalloc, cudaFree or other allocating routine is
+ * called.  Asynchronous on `stream`.  All calls on a device share the one array, which keeps the last
+ * call's contents (each call rewrites what it reads and clears its status word): two calls that may
+ * overlap on the GPU -- different streams without ordering -- race and give wrong results. */
+mom_status_t mom_product_3xtf32_noalloc(int64_t m, int64_t n, int64_t k, mom_property_t pa, mom_property_t pb,
+                                        const float *A, const float *B, float *C, int32_t *device_status,
+                                        mom_stream_t stream);
+
 /* Sustained-rate probes used as roofline denominators.  Each runs an instruction-issue loop on every
  * SM for about `milliseconds` and returns the achieved rate; no global memory traffic besides a
  * few words of output.  `scratch` is device memory of at least 1 MiB.

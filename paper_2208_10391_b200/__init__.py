@@ -73,6 +73,8 @@ _sigs = {
     "mom_plan_enable_step_timing": [_P, ctypes.c_int32],
     "mom_plan_step_times": [_P, ctypes.c_int32, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_float)],
     "mom_plan_destroy": [_P],
+    "mom_product_3xtf32_noalloc": [ctypes.c_int64, ctypes.c_int64, ctypes.c_int64, ctypes.c_int, ctypes.c_int, _P, _P, _P,
+                                   _P, _P],
     "mom_probe_tf32_tflops": [ctypes.c_double, _P, _P, ctypes.POINTER(ctypes.c_double)],
     "mom_probe_ffma_tflops": [ctypes.c_double, _P, _P, ctypes.POINTER(ctypes.c_double)],
 }
@@ -227,6 +229,19 @@ def mom_equation_plan(chain: Sequence, add_terms: Sequence = (), variant: int = 
                                 _desc_array(add_terms) if n_add else None, n_add, variant, ctypes.byref(handle))
     _check(st, "mom_equation_plan")
     return Plan(handle.value, n_chain, n_add)
+
+
+def mom_product_3xtf32_noalloc(m: int, n: int, k: int, pa: int, pb: int, a_ptr: int, b_ptr: int, c_ptr: int,
+                               device_status_ptr: Optional[int] = None, stream: int = 0) -> None:
+    """C = A*B on the tensor-core kernel using only the library's built-in scratch array (no allocation).
+
+    For callers that cannot allocate device memory where they need the product (a plug-in inside an
+    application that owns all device memory, a loop that must not hit an allocator).  Sizes beyond the
+    array (2*(m*k + k*n) floats over 16 MiB) raise MomError(ERR_LIMIT).  Calls share one array per device:
+    do not let two of them overlap on the GPU.
+    """
+    _check(_lib.mom_product_3xtf32_noalloc(m, n, k, pa, pb, _P(a_ptr), _P(b_ptr), _P(c_ptr), _P(device_status_ptr),
+                                           _P(stream)), "mom_product_3xtf32_noalloc")
 
 
 def mom_probe_tf32_tflops(milliseconds: float, scratch_ptr: int, stream: int = 0) -> float:

@@ -576,3 +576,106 @@ mom_status_t tc_probe_tf32(double milliseconds, void *scratch, cudaStream_t stre
 }
 
 }  // namespace mom
+
+// ---------------------------------------------------------------------------------------------
+// Allocation-free single product (mom_product_3xtf32_noalloc).  The hi/lo planes, the tile table
+// and a status word live in one fixed array that is part of the loaded module, so the call needs
+// neither a caller workspace nor any allocation.
+// ---------------------------------------------------------------------------------------------
+namespace mom {
+namespace {
+
+constexpr size_t NOALLOC_PLANES_BYTES = (size_t)16 << 20;            // A_hi, A_lo, Bt_hi, Bt_lo together
+constexpr int NOALLOC_MAX_TILES = 2048;
+constexpr size_t NOALLOC_TABLE_OFFSET = NOALLOC_PLANES_BYTES;
+constexpr size_t NOALLOC_STATUS_OFFSET = NOALLOC_TABLE_OFFSET + (size_t)NOALLOC_MAX_TILES * sizeof(int4);
+constexpr size_t NOALLOC_TOTAL_BYTES = NOALLOC_STATUS_OFFSET + 256;
+constexpr int NOALLOC_MAX_DEVICES = 64;
+
+// Held by every GPU that loads the library until the process exits.  In host code this name is only a
+// handle for cudaGetSymbolAddress; the device address is looked up once per device below.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[NOALLOC_TOTAL_BYTES];
+
+unsigned char *g_noalloc_device_ptr[NOALLOC_MAX_DEVICES] = {};
+
+// one thread per output tile, row-major tile order
+__global__ void noalloc_build_tiles_kernel(int4 *tiles, int m, int n, int k, int pa, int pb) {
+    const int cols = (n + BN - 1) / BN, total = ((m + BM - 1) / BM) * cols;
+    const int t = blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= total) return;
+    const int r0 = (t / cols) * BM, c0 = (t % cols) * BN;
+    int klo, khi;
+    tile_k_range(pa, pb, r0, min(r0 + BM, m), c0, min(c0 + BN, n), k, &klo, &khi);
+    if (klo >= khi) { klo = 0; khi = 0; }
+    tiles[t] = make_int4(r0, c0, klo / BK * BK, khi);
+}
+
+}  // namespace
+}  // namespace mom
+
+extern "C" mom_status_t mom_product_3xtf32_noalloc(int64_t m64, int64_t n64, int64_t k64, mom_property_t pa,
+                                                   mom_property_t pb, const float *A, const float *B, float *C,
+                                                   int32_t *device_status, mom_stream_t stream_) {
+    using namespace mom;
+    if (!A || !B || !C || m64 < 1 || n64 < 1 || k64 < 1) return MOM_ERR_INVALID_ARG;
+    if (pa < MOM_GENERAL || pa > MOM_UPPER_TRI || pb < MOM_GENERAL || pb > MOM_UPPER_TRI) return MOM_ERR_INVALID_ARG;
+    if ((pa != MOM_GENERAL && m64 != k64) || (pb != MOM_GENERAL && k64 != n64)) return MOM_ERR_PROPERTY;
+    if (k64 % 4 != 0 || n64 % 4 != 0) return MOM_ERR_INVALID_ARG;      // leading dimensions TMA can address
+    if ((reinterpret_cast<uintptr_t>(A) | reinterpret_cast<uintptr_t>(B) | reinterpret_cast<uintptr_t>(C)) & 15) return MOM_ERR_ALIGNMENT;
+    if (m64 > (1 << 20) || n64 > (1 << 20) || k64 > (1 << 20)) return MOM_ERR_LIMIT;
+    const int m = (int)m64, n = (int)n64, k = (int)k64;
+    const size_t a_bytes = align_up((size_t)m * k * sizeof(float), WS_ALIGN);
+    const size_t b_bytes = align_up((size_t)k * n * sizeof(float), WS_ALIGN);
+    const long long tiles = (long long)((m + BM - 1) / BM) * ((n + BN - 1) / BN);
+    if (2 * a_bytes + 2 * b_bytes > NOALLOC_PLANES_BYTES || tiles > NOALLOC_MAX_TILES) return MOM_ERR_LIMIT;
+
+    int dev = 0, major = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return MOM_ERR_CUDA;
+    if (dev < 0 || dev >= NOALLOC_MAX_DEVICES) return MOM_ERR_LIMIT;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return MOM_ERR_CUDA;
+    if (major != 10) return MOM_ERR_ARCH;
+    if (!g_noalloc_device_ptr[dev]) {          // once per device, with that device current
+        void *p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_noalloc_scratch) != cudaSuccess || !p) return MOM_ERR_CUDA;
+        g_noalloc_device_ptr[dev] = static_cast<unsigned char *>(p);
+    }
+    if (!g_sm_count) cudaDeviceGetAttribute(&g_sm_count, cudaDevAttrMultiProcessorCount, dev);
+    if (!g_attr_set) {
+        if (cudaFuncSetAttribute(product_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess)
+            return MOM_ERR_CUDA;
+        g_attr_set = true;
+    }
+    cudaStream_t stream = reinterpret_cast<cudaStream_t>(stream_);
+    unsigned char *base = g_noalloc_device_ptr[dev];
+    float *a_hi = reinterpret_cast<float *>(base), *a_lo = reinterpret_cast<float *>(base + a_bytes);
+    float *b_hi = reinterpret_cast<float *>(base + 2 * a_bytes), *b_lo = reinterpret_cast<float *>(base + 2 * a_bytes + b_bytes);
+    int4 *table = reinterpret_cast<int4 *>(base + NOALLOC_TABLE_OFFSET);
+    int32_t *status = device_status ? device_status : reinterpret_cast<int32_t *>(base + NOALLOC_STATUS_OFFSET);
+    // the array keeps whatever the previous call left: the status word must start at zero, the tile
+    // table and every plane block a tile can read are rewritten below
+    if (!device_status && cudaMemsetAsync(status, 0, 4 * sizeof(int32_t), stream) != cudaSuccess) return MOM_ERR_CUDA;
+
+    auto blocks = [](int x) { return (x + SPLIT_BLOCK - 1) / SPLIT_BLOCK; };
+    noalloc_build_tiles_kernel<<<(unsigned)((tiles + 127) / 128), 128, 0, stream>>>(table, m, n, k, (int)pa, (int)pb);
+    split_planes_kernel<false><<<dim3(blocks(k), blocks(m)), 256, 0, stream>>>(A, a_hi, a_lo, m, k, (int)pa);
+    split_planes_kernel<true><<<dim3(blocks(n), blocks(k)), 256, 0, stream>>>(B, b_hi, b_lo, k, n, (int)pb);
+    if (cudaGetLastError() != cudaSuccess) return MOM_ERR_CUDA;
+
+    CUtensorMap ma_hi, ma_lo, mb_hi, mb_lo, mc;
+    const bool ok = make_map(&ma_hi, a_hi, m, k, BM, BK, CU_TENSOR_MAP_SWIZZLE_64B) &&
+                    make_map(&ma_lo, a_lo, m, k, BM, BK, CU_TENSOR_MAP_SWIZZLE_64B) &&
+                    make_map(&mb_hi, b_hi, n, k, BN, BK, CU_TENSOR_MAP_SWIZZLE_64B) &&
+                    make_map(&mb_lo, b_lo, n, k, BN, BK, CU_TENSOR_MAP_SWIZZLE_64B) &&
+                    make_map(&mc, C, m, n, 32, 32, CU_TENSOR_MAP_SWIZZLE_128B);
+    if (!ok) return MOM_ERR_CUDA;
+    TcParams prm;
+    prm.tiles = table;
+    prm.num_tiles = (int)tiles;
+    prm.m = m;
+    prm.n = n;
+    prm.pout = pa == MOM_GENERAL || pb == MOM_GENERAL || pa != pb ? (int)MOM_GENERAL : (int)pa;
+    prm.add.count = 0;
+    prm.status = status;
+    product_tc_kernel<<<std::min(prm.num_tiles, g_sm_count), THREADS, SMEM_BYTES, stream>>>(ma_hi, ma_lo, mb_hi, mb_lo, mc, prm);
+    return cudaGetLastError() == cudaSuccess ? MOM_OK : MOM_ERR_CUDA;
+}
