@@ -218,6 +218,16 @@ def run_gpu(args):
     eq = headline_equation()
     sampler = ClockSampler(local)
 
+    if args.only:
+        # one named configuration, nothing else: the small case for profiler captures
+        cfgs = {c.name: c for c in (wl.config_tiny(), wl.config_five_general(), wl.config_property_heavy(),
+                                    wl.config_large_square(), wl.config_batched(), wl.config_paper_chain())}
+        cfg = cfgs[args.only]
+        r = time_equation(mom, torch, cfg, variant, steps=args.steps, warmup=args.warmup, stream=stream, timing=cfg.batch == 1)
+        print(json.dumps({"workload": cfg.name, "variant": args.variant, "ms": r["ms"], "useful_flops": r["useful_flops"],
+                          "launches": r["launches"], "step_times_ms": r["step_times"][-1:] }))
+        return
+
     def barrier():
         if world > 1:
             dist.barrier()
@@ -238,12 +248,12 @@ def run_gpu(args):
     ws = torch.empty(max(wsb, 256), dtype=torch.uint8, device="cuda")
     cp = [None if t is None else t.data_ptr() for t in dchain]
     ap = [None if t is None else t.data_ptr() for t in dadd]
-    plan.enable_step_timing(True)
     n_steps = plan.num_steps()
     with torch.cuda.stream(stream):
         for _ in range(max(args.warmup, 3)):
             plan.execute(cp, ap, out.data_ptr(), ws.data_ptr(), wsb, stream.cuda_stream)
     barrier()
+    plan.enable_step_timing(True)      # per-kernel events, averaged over the timed executes
     sampler.start()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     prod_ms = [0.0] * n_steps
@@ -258,7 +268,7 @@ def run_gpu(args):
     barrier()
     clocks = sampler.stop()
     total_ms = e0.elapsed_time(e1)
-    # per-kernel times of the last step (events recorded inside the timed region on the same stream)
+    # per-kernel mean times over the timed region (events recorded inside it, on the same stream)
     for i in range(n_steps):
         a, b = plan.step_times(i)
         prod_ms[i], pre_ms[i] = a, b
@@ -364,7 +374,7 @@ def run_gpu(args):
         result["all_configs"] = others
 
         # ---- CPU baseline: the oracle on a bounded sample of the same workload
-        result["cpu_baseline"] = cpu_baseline(eq, chain, add, useful, n_rows=32)
+        result["cpu_baseline"] = cpu_baseline(eq, chain, add, useful, n_rows=256)
 
     if rank == 0:
         print(json.dumps(result))
@@ -384,6 +394,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--variant", default="3xtf32", choices=["3xtf32", "ffma"])
+    ap.add_argument("--only", default=None, help="time just this workload (by name) and print a short JSON line")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

@@ -185,8 +185,9 @@ mom_status_t mom_plan_last_launch_count(const mom_plan_t *plan, int32_t *launche
 
 /* Per-kernel device timing for roofline reports.  With timing enabled every execute brackets each
  * product kernel (and, separately, its operand-split pre-pass) with CUDA events on the caller's stream.
- * After the stream has been synchronised, mom_plan_step_times returns for the most recent execute and
- * step i the milliseconds spent in the product kernel and in its pre-pass (0 when there is none).
+ * After the stream has been synchronised, mom_plan_step_times returns for step i the milliseconds spent
+ * in the product kernel and in its pre-pass (0 when there is none), averaged over the executes made since
+ * timing was enabled (at most the 32 most recent).
  * Off by default; enabling it creates events but no device memory. */
 mom_status_t mom_plan_enable_step_timing(mom_plan_t *plan, int32_t enable);
 mom_status_t mom_plan_step_times(const mom_plan_t *plan, int32_t i, float *product_ms, float *prepass_ms);

@@ -14,8 +14,12 @@ struct DeviceState {
     int device = -1;
     int32_t *status = nullptr;          // device: {code, detail, 0, 0}
     TcPlanState tc;                     // tile tables of tensor-core steps
-    std::vector<cudaEvent_t> events;    // 3 per step when step timing is on: before pre-pass, before product, after
+    // step timing: a ring of TIMING_SLOTS executes, 3 events per step (before pre-pass, before product, after)
+    std::vector<cudaEvent_t> events;
+    long long timed_executes = 0;       // executes recorded since timing was enabled
 };
+
+constexpr int TIMING_SLOTS = 32;
 
 void destroy_device_state(DeviceState *d) {
     if (!d) return;
@@ -105,9 +109,10 @@ mom_status_t execute_impl(const mom_plan *p, const float *const *chain_ptrs, con
     int launches = 0;
     const int ns = (int)p->steps.size();
     const bool timing = p->step_timing && batch == 1;
-    if (timing && p->dev->events.size() != (size_t)ns * 3) {
+    if (timing && p->dev->events.size() != (size_t)ns * 3 * TIMING_SLOTS) {
         for (cudaEvent_t e : p->dev->events) cudaEventDestroy(e);
-        p->dev->events.assign((size_t)ns * 3, nullptr);
+        p->dev->timed_executes = 0;
+        p->dev->events.assign((size_t)ns * 3 * TIMING_SLOTS, nullptr);
         for (auto &e : p->dev->events)
             if (cudaEventCreate(&e) != cudaSuccess) return MOM_ERR_CUDA;
     }
@@ -173,7 +178,7 @@ mom_status_t execute_impl(const mom_plan *p, const float *const *chain_ptrs, con
                 a.pout = stp.pub.out_property;
                 a.add.count = 0;
             }
-            cudaEvent_t *ev = timing ? &p->dev->events[(size_t)s * 3] : nullptr;
+            cudaEvent_t *ev = timing ? &p->dev->events[((size_t)(p->dev->timed_executes % TIMING_SLOTS) * ns + s) * 3] : nullptr;
             if (ev) cudaEventRecord(ev[0], stream);
             if (stp.pub.uses_tensor_cores) {
                 int used = 0;
@@ -200,6 +205,7 @@ mom_status_t execute_impl(const mom_plan *p, const float *const *chain_ptrs, con
             ++launches;
         }
     }
+    if (timing) ++p->dev->timed_executes;
     p->last_launches = launches;
     return MOM_OK;
 }
@@ -286,16 +292,26 @@ mom_status_t mom_equation_execute_host(const mom_plan_t *plan, const float *cons
 mom_status_t mom_plan_enable_step_timing(mom_plan_t *plan, int32_t enable) {
     if (!plan) return MOM_ERR_INVALID_ARG;
     plan->step_timing = enable != 0;
+    if (plan->dev) plan->dev->timed_executes = 0;
     return MOM_OK;
 }
 
 mom_status_t mom_plan_step_times(const mom_plan_t *plan, int32_t i, float *product_ms, float *prepass_ms) {
     if (!plan || i < 0 || i >= (int32_t)plan->steps.size()) return MOM_ERR_INVALID_ARG;
-    if (!plan->dev || plan->dev->events.size() != plan->steps.size() * 3) return MOM_ERR_INVALID_ARG;
-    cudaEvent_t *ev = &plan->dev->events[(size_t)i * 3];
+    const size_t ns = plan->steps.size();
+    if (!plan->dev || plan->dev->events.size() != ns * 3 * mom::TIMING_SLOTS || plan->dev->timed_executes < 1) return MOM_ERR_INVALID_ARG;
+    const long long have = plan->dev->timed_executes < mom::TIMING_SLOTS ? plan->dev->timed_executes : mom::TIMING_SLOTS;
     float pre = 0.0f, prod = 0.0f;
-    if (cudaEventElapsedTime(&pre, ev[0], ev[1]) != cudaSuccess) return MOM_ERR_CUDA;
-    if (cudaEventElapsedTime(&prod, ev[1], ev[2]) != cudaSuccess) return MOM_ERR_CUDA;
+    for (long long slot = 0; slot < have; ++slot) {        // mean over the recorded executes (the most recent ring-full)
+        cudaEvent_t *ev = &plan->dev->events[((size_t)slot * ns + i) * 3];
+        float a = 0.0f, b = 0.0f;
+        if (cudaEventElapsedTime(&a, ev[0], ev[1]) != cudaSuccess) return MOM_ERR_CUDA;
+        if (cudaEventElapsedTime(&b, ev[1], ev[2]) != cudaSuccess) return MOM_ERR_CUDA;
+        pre += a;
+        prod += b;
+    }
+    pre /= (float)have;
+    prod /= (float)have;
     if (product_ms) *product_ms = prod;
     if (prepass_ms) *prepass_ms = pre;
     return MOM_OK;

@@ -7,9 +7,10 @@
 //      (n x k), so that both MMA operands are K-major.  Blocks that lie wholly outside a triangular
 //      operand's structure are skipped: no tile ever reads them.
 //   2. product_tc_kernel, persistent, one CTA per SM, walks a work-sorted tile table.  Per tile:
-//        warp 0   TMA producer: per k-block loads A_hi, A_lo (128 rows x 16 k) and Bt_hi, Bt_lo
-//                 (256 rows x 16 k), 64-byte rows with the 64B swizzle, into a 4-stage ring;
-//        warp 1   MMA issuer: 2 k-steps x 3 MMAs (M128 N256 K8) per stage into one of two 256-column
+//        warp 0   TMA producer: per k-block loads A_hi, A_lo (128 rows x 32 k) and Bt_hi, Bt_lo
+//                 (256 rows x 32 k), 128-byte rows with the 128B swizzle, into a 2-stage ring of
+//                 96 KiB stages (64-byte rows cost twice the TMA requests per byte and ran 30 % slower);
+//        warp 1   MMA issuer: 4 k-steps x 3 MMAs (M128 N256 K8) per stage into one of two 256-column
 //                 accumulators in tensor memory; tcgen05.commit releases the stage / publishes the tile;
 //        warps 2-5 epilogue: tcgen05.ld 32 columns at a time, Add terms, structure mask, swizzled
 //                 staging in shared memory, TMA store (coalesced, clipped at the matrix edge).
@@ -32,11 +33,13 @@ namespace mom {
 namespace {
 
 constexpr int BM = TC_BM, BN = TC_BN;
-constexpr int BK = 16;                       // f32 elements per pipeline stage (two K=8 MMA steps)
-constexpr int STAGES = 4;
-constexpr int A_PLANE_BYTES = BM * BK * 4;   // 8 KiB
-constexpr int B_PLANE_BYTES = BN * BK * 4;   // 16 KiB
-constexpr int STAGE_BYTES = 2 * A_PLANE_BYTES + 2 * B_PLANE_BYTES;   // 48 KiB
+constexpr int BK = 32;                       // f32 elements per pipeline stage: one 128-byte swizzle row, four K=8 MMA steps
+constexpr int STAGES = 2;
+constexpr int ROW_BYTES = BK * 4;
+constexpr CUtensorMapSwizzle OPERAND_TMA_SWIZZLE = BK == 32 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B;
+constexpr int A_PLANE_BYTES = BM * BK * 4;   // 16 KiB
+constexpr int B_PLANE_BYTES = BN * BK * 4;   // 32 KiB
+constexpr int STAGE_BYTES = 2 * A_PLANE_BYTES + 2 * B_PLANE_BYTES;   // 96 KiB
 constexpr int EPI_BOX_BYTES = 32 * 32 * 4;   // 32 rows x 32 columns staged per TMA store
 constexpr int EPI_BYTES = 4 * 2 * EPI_BOX_BYTES;                     // 4 warps x 2 buffers
 constexpr int NUM_BARRIERS = 2 * STAGES + 4 + 1;
@@ -89,10 +92,14 @@ struct TcParams {
     int32_t *status;
 };
 
-// K-major operand tile with 64-byte rows under the 64B swizzle: 8-row groups are 512 bytes apart; a
-// K=8 step is 32 bytes along the row.
+// K-major operand tile whose rows are one swizzle span long (128 bytes under the 128B swizzle, or 64
+// under the 64B one): 8-row groups are 8 rows apart; a K=8 step is 32 bytes along the row.
 __device__ __forceinline__ uint64_t kmajor_desc(uint32_t tile, int kstep) {
-    return ptx::smem_desc(tile + kstep * 32, 16, 512, ptx::SWIZZLE_64B);
+    return ptx::smem_desc(tile + kstep * 32, 16, 8 * ROW_BYTES, BK == 32 ? ptx::SWIZZLE_128B : ptx::SWIZZLE_64B);
+}
+// the rate probe's resident tiles: 64-byte rows, 64B swizzle
+__device__ __forceinline__ uint64_t kmajor_desc_64(uint32_t tile) {
+    return ptx::smem_desc(tile, 16, 512, ptx::SWIZZLE_64B);
 }
 
 __global__ void __launch_bounds__(THREADS, 1)
@@ -302,52 +309,56 @@ product_tc_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_con
     if (warp == 1) ptx::tmem_dealloc(tmem_base, TMEM_COLS);
 }
 
-// hi = rna_tf32(a), lo = rna_tf32(a - hi) for every block of SPLIT_BLOCK x SPLIT_BLOCK entries that
-// intersects the operand's structure.  The planes keep the operand's layout (rows x cols) or, with
-// TRANSPOSE, hold the transposed operand (cols x rows).  rows and cols are multiples of 4 where a
-// vector access needs it: the plain path requires cols % 4 == 0.
+// hi = rna_tf32(a), lo = rna_tf32(a - hi).  The planes keep the operand's layout (rows x cols) or, with
+// TRANSPOSE, hold the transposed operand (cols x rows).  One CTA handles a 64 x 64 piece; pieces whose
+// enclosing SPLIT_BLOCK x SPLIT_BLOCK block lies wholly outside a triangular operand's structure are
+// skipped (no product tile reads them).  rows and cols are multiples of 4 wherever a vector access
+// needs it: the plain path needs cols % 4 == 0, the transposing path rows % 4 == 0.
+constexpr int SPLIT_PIECE = 64;
+
 template <bool TRANSPOSE>
 __global__ void __launch_bounds__(256)
 split_planes_kernel(const float *__restrict__ src, float *__restrict__ hi, float *__restrict__ lo, int rows, int cols, int prop) {
-    const int br = blockIdx.y * SPLIT_BLOCK, bc = blockIdx.x * SPLIT_BLOCK;
+    const int pr = blockIdx.y * SPLIT_PIECE, pc = blockIdx.x * SPLIT_PIECE;
+    const int br = pr / SPLIT_BLOCK * SPLIT_BLOCK, bc = pc / SPLIT_BLOCK * SPLIT_BLOCK;
     if (prop == MOM_LOWER_TRI && bc > br + SPLIT_BLOCK - 1) return;     // block wholly above the diagonal
     if (prop == MOM_UPPER_TRI && br > bc + SPLIT_BLOCK - 1) return;     // wholly below
-    const int r1 = min(br + SPLIT_BLOCK, rows), c1 = min(bc + SPLIT_BLOCK, cols);
     if (!TRANSPOSE) {
-        const int vec_per_row = (c1 - bc) >> 2;
-        const int total = (r1 - br) * vec_per_row;
-        for (int e = threadIdx.x; e < total; e += blockDim.x) {
-            const int r = br + e / vec_per_row, c = bc + ((e % vec_per_row) << 2);
-            const size_t off = (size_t)r * cols + c;
-            const float4 a = __ldg(reinterpret_cast<const float4 *>(src + off));
-            float4 h, l;
-            h.x = ptx::to_tf32(a.x); h.y = ptx::to_tf32(a.y); h.z = ptx::to_tf32(a.z); h.w = ptx::to_tf32(a.w);
-            l.x = ptx::to_tf32(a.x - h.x); l.y = ptx::to_tf32(a.y - h.y); l.z = ptx::to_tf32(a.z - h.z); l.w = ptx::to_tf32(a.w - h.w);
-            *reinterpret_cast<float4 *>(hi + off) = h;
-            *reinterpret_cast<float4 *>(lo + off) = l;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int e = threadIdx.x + 256 * i;                         // 64 rows x 16 float4
+            const int r = pr + (e >> 4), c = pc + ((e & 15) << 2);
+            if (r < rows && c < cols) {
+                const size_t off = (size_t)r * cols + c;
+                const float4 a = __ldg(reinterpret_cast<const float4 *>(src + off));
+                float4 h, l;
+                h.x = ptx::to_tf32(a.x); h.y = ptx::to_tf32(a.y); h.z = ptx::to_tf32(a.z); h.w = ptx::to_tf32(a.w);
+                l.x = ptx::to_tf32(a.x - h.x); l.y = ptx::to_tf32(a.y - h.y); l.z = ptx::to_tf32(a.z - h.z); l.w = ptx::to_tf32(a.w - h.w);
+                *reinterpret_cast<float4 *>(hi + off) = h;
+                *reinterpret_cast<float4 *>(lo + off) = l;
+            }
         }
     } else {
-        __shared__ float tile[32][33];
-        const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;           // 32 x 8 threads
-        for (int sr = br; sr < r1; sr += 32) {
-            for (int sc = bc; sc < c1; sc += 32) {
+        __shared__ float tile[SPLIT_PIECE][SPLIT_PIECE + 1];
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const int r = sr + ty + 8 * i, c = sc + tx;
-                    tile[ty + 8 * i][tx] = (r < rows && c < cols) ? __ldg(src + (size_t)r * cols + c) : 0.0f;
-                }
-                __syncthreads();
+        for (int i = 0; i < 16; ++i) {
+            const int e = threadIdx.x + 256 * i;                         // 64 x 64 scalars, row-contiguous reads
+            const int r = e >> 6, c = e & 63;
+            tile[r][c] = (pr + r < rows && pc + c < cols) ? __ldg(src + (size_t)(pr + r) * cols + pc + c) : 0.0f;
+        }
+        __syncthreads();
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const int c = sc + ty + 8 * i, r = sr + tx;               // plane entry (c, r), r contiguous
-                    if (c < cols && r < rows) {
-                        const float a = tile[tx][ty + 8 * i];
-                        const float h = ptx::to_tf32(a);
-                        hi[(size_t)c * rows + r] = h;
-                        lo[(size_t)c * rows + r] = ptx::to_tf32(a - h);
-                    }
-                }
-                __syncthreads();
+        for (int i = 0; i < 4; ++i) {
+            const int e = threadIdx.x + 256 * i;                         // 64 plane rows x 16 float4
+            const int c = e >> 4, r = (e & 15) << 2;                     // plane entry (pc + c, pr + r .. +3)
+            if (pc + c < cols && pr + r < rows) {
+                float4 h, l;
+                const float a0 = tile[r][c], a1 = tile[r + 1][c], a2 = tile[r + 2][c], a3 = tile[r + 3][c];
+                h.x = ptx::to_tf32(a0); h.y = ptx::to_tf32(a1); h.z = ptx::to_tf32(a2); h.w = ptx::to_tf32(a3);
+                l.x = ptx::to_tf32(a0 - h.x); l.y = ptx::to_tf32(a1 - h.y); l.z = ptx::to_tf32(a2 - h.z); l.w = ptx::to_tf32(a3 - h.w);
+                const size_t off = (size_t)(pc + c) * rows + pr + r;
+                *reinterpret_cast<float4 *>(hi + off) = h;
+                *reinterpret_cast<float4 *>(lo + off) = l;
             }
         }
     }
@@ -456,7 +467,7 @@ mom_status_t tc_launch_step(const mom_plan &p, TcPlanState &s, int step, const P
     float *a_hi = reinterpret_cast<float *>(workspace + st.a_hi_off), *a_lo = reinterpret_cast<float *>(workspace + st.a_lo_off);
     float *b_hi = reinterpret_cast<float *>(workspace + st.b_hi_off), *b_lo = reinterpret_cast<float *>(workspace + st.b_lo_off);
 
-    auto blocks = [](int x) { return (x + SPLIT_BLOCK - 1) / SPLIT_BLOCK; };
+    auto blocks = [](int x) { return (x + SPLIT_PIECE - 1) / SPLIT_PIECE; };
     split_planes_kernel<false><<<dim3(blocks(a.k), blocks(a.m)), 256, 0, stream>>>(a.A, a_hi, a_lo, a.m, a.k, a.pa);
     split_planes_kernel<true><<<dim3(blocks(a.n), blocks(a.k)), 256, 0, stream>>>(a.B, b_hi, b_lo, a.k, a.n, a.pb);
     if (cudaGetLastError() != cudaSuccess) return MOM_ERR_CUDA;
@@ -464,10 +475,10 @@ mom_status_t tc_launch_step(const mom_plan &p, TcPlanState &s, int step, const P
 
     // A planes are m x k, B planes are n x k (transposed): both K-major with 16-element (64-byte) box rows
     CUtensorMap ma_hi, ma_lo, mb_hi, mb_lo, mc;
-    bool ok = make_map(&ma_hi, a_hi, a.m, a.k, BM, BK, CU_TENSOR_MAP_SWIZZLE_64B) &&
-              make_map(&ma_lo, a_lo, a.m, a.k, BM, BK, CU_TENSOR_MAP_SWIZZLE_64B) &&
-              make_map(&mb_hi, b_hi, a.n, a.k, BN, BK, CU_TENSOR_MAP_SWIZZLE_64B) &&
-              make_map(&mb_lo, b_lo, a.n, a.k, BN, BK, CU_TENSOR_MAP_SWIZZLE_64B) &&
+    bool ok = make_map(&ma_hi, a_hi, a.m, a.k, BM, BK, OPERAND_TMA_SWIZZLE) &&
+              make_map(&ma_lo, a_lo, a.m, a.k, BM, BK, OPERAND_TMA_SWIZZLE) &&
+              make_map(&mb_hi, b_hi, a.n, a.k, BN, BK, OPERAND_TMA_SWIZZLE) &&
+              make_map(&mb_lo, b_lo, a.n, a.k, BN, BK, OPERAND_TMA_SWIZZLE) &&
               make_map(&mc, a.C, a.m, a.n, 32, 32, CU_TENSOR_MAP_SWIZZLE_128B);
     if (!ok) return MOM_ERR_CUDA;
 
@@ -522,7 +533,7 @@ __global__ void __launch_bounds__(128, 1) tf32_probe_kernel(int batches, int32_t
     asm volatile("ld.shared.u32 %0, [%1];" : "=r"(tmem_base) : "r"(slot));
     if (threadIdx.x == 0) {
         constexpr uint32_t idesc = ptx::instr_desc_tf32(128, 256, 0, 0);
-        const uint64_t da = kmajor_desc(a_tile, 0), db = kmajor_desc(b_tile, 0);
+        const uint64_t da = kmajor_desc_64(a_tile), db = kmajor_desc_64(b_tile);
         bool ok = true;
         for (int b = 0; b < batches && ok; ++b) {
             for (int i = 0; i < PROBE_BATCH; ++i) ptx::mma_tf32(tmem_base, da, db, idesc, (b | i) ? 1u : 0u);
@@ -655,17 +666,17 @@ extern "C" mom_status_t mom_product_3xtf32_noalloc(int64_t m64, int64_t n64, int
     // table and every plane block a tile can read are rewritten below
     if (!device_status && cudaMemsetAsync(status, 0, 4 * sizeof(int32_t), stream) != cudaSuccess) return MOM_ERR_CUDA;
 
-    auto blocks = [](int x) { return (x + SPLIT_BLOCK - 1) / SPLIT_BLOCK; };
+    auto blocks = [](int x) { return (x + SPLIT_PIECE - 1) / SPLIT_PIECE; };
     noalloc_build_tiles_kernel<<<(unsigned)((tiles + 127) / 128), 128, 0, stream>>>(table, m, n, k, (int)pa, (int)pb);
     split_planes_kernel<false><<<dim3(blocks(k), blocks(m)), 256, 0, stream>>>(A, a_hi, a_lo, m, k, (int)pa);
     split_planes_kernel<true><<<dim3(blocks(n), blocks(k)), 256, 0, stream>>>(B, b_hi, b_lo, k, n, (int)pb);
     if (cudaGetLastError() != cudaSuccess) return MOM_ERR_CUDA;
 
     CUtensorMap ma_hi, ma_lo, mb_hi, mb_lo, mc;
-    const bool ok = make_map(&ma_hi, a_hi, m, k, BM, BK, CU_TENSOR_MAP_SWIZZLE_64B) &&
-                    make_map(&ma_lo, a_lo, m, k, BM, BK, CU_TENSOR_MAP_SWIZZLE_64B) &&
-                    make_map(&mb_hi, b_hi, n, k, BN, BK, CU_TENSOR_MAP_SWIZZLE_64B) &&
-                    make_map(&mb_lo, b_lo, n, k, BN, BK, CU_TENSOR_MAP_SWIZZLE_64B) &&
+    const bool ok = make_map(&ma_hi, a_hi, m, k, BM, BK, OPERAND_TMA_SWIZZLE) &&
+                    make_map(&ma_lo, a_lo, m, k, BM, BK, OPERAND_TMA_SWIZZLE) &&
+                    make_map(&mb_hi, b_hi, n, k, BN, BK, OPERAND_TMA_SWIZZLE) &&
+                    make_map(&mb_lo, b_lo, n, k, BN, BK, OPERAND_TMA_SWIZZLE) &&
                     make_map(&mc, C, m, n, 32, 32, CU_TENSOR_MAP_SWIZZLE_128B);
     if (!ok) return MOM_ERR_CUDA;
     TcParams prm;
