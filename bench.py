@@ -187,7 +187,10 @@ def time_equation(mom, torch, eq, variant, steps, warmup, stream, timing=False):
             e1.record(stream)
             if timing:
                 stream.synchronize()
-                step_times.append([plan.step_times(i) for i in range(plan.num_steps())])
+                try:
+                    step_times.append([plan.step_times(i) for i in range(plan.num_steps())])
+                except mom.MomError:        # fused single-kernel plans have no per-step events
+                    step_times.append([])
         stream.synchronize()
     ms = [e0.elapsed_time(e1) for e0, e1 in events]
     status = plan.device_status()

@@ -4,6 +4,7 @@
 #include <new>
 #include <vector>
 
+#include "fused_small.h"
 #include "kernels.h"
 #include "mom_internal.h"
 #include "product_tc.h"
@@ -104,6 +105,39 @@ mom_status_t execute_impl(const mom_plan *p, const float *const *chain_ptrs, con
     if (any_tc) {
         st = tc_prepare(*p, p->dev->tc);
         if (st != MOM_OK) return st;
+    }
+
+    if (p->fused_ok) {
+        FusedPlan fp;
+        std::memset(&fp, 0, sizeof(fp));
+        fp.n_ops = (int)p->kept.size();
+        for (int i = 0; i < fp.n_ops; ++i) {
+            const int id = p->kept[i];
+            fp.ops[i] = FusedOperand{chain_ptrs[id], chain_strides ? chain_strides[id] : 0, (int)p->chain[id].rows,
+                                     (int)p->chain[id].cols, p->chain[id].property, p->fused_value_off[id], p->fused_value_ld[id]};
+        }
+        fp.n_steps = (int)p->steps.size();
+        for (int s = 0; s < fp.n_steps; ++s) {
+            const StepImpl &stp = p->steps[s];
+            fp.steps[s] = FusedStep{p->fused_value_off[stp.pub.lhs], p->fused_value_off[stp.pub.rhs],
+                                    stp.is_last ? -1 : p->fused_value_off[stp.pub.out], (int)stp.pub.m, (int)stp.pub.n,
+                                    (int)stp.pub.k, stp.pub.lhs_property, stp.pub.rhs_property,
+                                    stp.is_last ? p->result_desc.property : stp.pub.out_property,
+                                    p->fused_value_ld[stp.pub.lhs], p->fused_value_ld[stp.pub.rhs],
+                                    stp.is_last ? 0 : p->fused_value_ld[stp.pub.out]};
+        }
+        fp.add.count = n_add;
+        for (int i = 0; i < n_add; ++i) {
+            fp.add.ptr[i] = p->add[i].property == MOM_IDENTITY ? nullptr : add_ptrs[i];
+            fp.add.stride[i] = add_strides ? add_strides[i] : 0;
+        }
+        fp.out = out;
+        fp.out_stride = out_stride;
+        fp.batch = batch;
+        fp.use_mma = p->variant != MOM_VARIANT_FFMA;
+        if (launch_fused_small(fp, p->fused_smem_bytes, stream) != cudaSuccess) return MOM_ERR_CUDA;
+        p->last_launches = 1;
+        return MOM_OK;
     }
 
     int launches = 0;

@@ -1,0 +1,275 @@
+// Fused small-equation kernel: a whole plan (every product, the Add terms, the structure mask) for
+// one instance per CTA, with the operands and all intermediates resident in shared memory.  Batched
+// small equations are bound by HBM traffic, so each operand is read exactly once (only the
+// structural part of triangular operands), nothing intermediate touches global memory, and several
+// CTAs per SM overlap one instance's loads with another's arithmetic.
+//
+// Two arithmetic variants of the products:
+//   MMA   warp-level mma.sync m16n8k8 tf32 with the 3xTF32 split done in registers on the
+//         fragments (a = hi + lo; lo*hi + hi*lo + hi*hi accumulated in f32).  The problem per CTA
+//         is far too small for a tcgen05/TMEM pipeline, and the bound here is HBM, not the tensor pipe.
+//   FFMA  plain f32 FMA on cells of 2 rows x 4 columns.
+#include <cstring>
+
+#include "fused_small.h"
+
+namespace mom {
+
+namespace {
+
+constexpr int THREADS = 256;
+constexpr int WARPS = THREADS / 32;
+
+// Copy one operand (rows x cols, row-major, leading dimension cols) into shared memory with leading
+// dimension ld.  Only the part inside the structure is read; the rest is zero-filled.  16-byte
+// asynchronous copies (cp.async) keep every load of every operand in flight at once; a copy with
+// source size 0 writes zeros.  The caller waits with cp_async_wait_all() + __syncthreads().
+__device__ void load_operand(float *__restrict__ dst, const float *__restrict__ src, int rows, int cols, int ld, int prop) {
+    const int vec_per_row = (cols + 3) >> 2;
+    const bool vec_ok = (cols & 3) == 0 && (reinterpret_cast<uintptr_t>(src) & 15) == 0;
+    // thread -> (row, float4 column); when the row length divides the block the column stays fixed and
+    // the row advances by a constant, which avoids a division per copy
+    const bool regular = (THREADS % vec_per_row) == 0;
+    int r = threadIdx.x / vec_per_row, c = (threadIdx.x - r * vec_per_row) << 2;
+    const int r_step = THREADS / vec_per_row;
+    for (int e = threadIdx.x; e < rows * vec_per_row; e += THREADS, r += r_step) {
+        if (!regular) { r = e / vec_per_row; c = (e - r * vec_per_row) << 2; }
+        // columns [c, c+4) intersect the structure of row r?
+        const bool needed = prop == MOM_GENERAL || (prop == MOM_LOWER_TRI && c <= r) || (prop == MOM_UPPER_TRI && c + 3 >= r);
+        float *d = dst + r * ld + c;
+        const float *p = src + (size_t)r * cols + c;
+        if (vec_ok) {
+            const uint32_t daddr = static_cast<uint32_t>(__cvta_generic_to_shared(d));
+            asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(daddr), "l"(p), "r"(needed ? 16 : 0) : "memory");
+        } else {
+            float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (needed) {
+                if (c < cols) v.x = __ldg(p);
+                if (c + 1 < cols) v.y = __ldg(p + 1);
+                if (c + 2 < cols) v.z = __ldg(p + 2);
+                if (c + 3 < cols) v.w = __ldg(p + 3);
+            }
+            *reinterpret_cast<float4 *>(d) = v;
+        }
+    }
+}
+
+__device__ __forceinline__ void cp_async_wait_all() {
+    asm volatile("cp.async.commit_group;\n\tcp.async.wait_group 0;" ::: "memory");
+}
+
+// a = hi + lo with both halves representable in tf32.  Rounding to tf32 (10 mantissa bits, ties away
+// from zero) is done on the bit pattern with full-rate integer instructions: add half a unit of the
+// last kept place to the magnitude, clear the 13 dropped bits.  (The cvt.rna.tf32.f32 instruction gives
+// the same result but issues at conversion-pipe rate, which made it the bottleneck of this kernel.)
+__device__ __forceinline__ uint32_t round_tf32_bits(float a) { return (__float_as_uint(a) + 0x1000u) & 0xFFFFE000u; }
+__device__ __forceinline__ void split_tf32(float a, uint32_t &hi, uint32_t &lo) {
+    hi = round_tf32_bits(a);
+    lo = round_tf32_bits(a - __uint_as_float(hi));
+}
+
+__device__ __forceinline__ void mma_tf32(float (&d)[4], const uint32_t (&a)[4], const uint32_t (&b)[2]) {
+    asm volatile("mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b[0]), "r"(b[1]));
+}
+
+// store one output entry pair (r, c), (r, c+1) of a step: into shared memory for an intermediate
+// (masked to its structure, padded columns zero) or, on the last step, into X with the Add terms
+__device__ __forceinline__ void store_pair(const FusedPlan &fp, const FusedStep &st, float *smem, long long inst, int r, int c,
+                                           float v0, float v1) {
+    if (r >= st.m) return;
+    if (st.out_off >= 0) {
+        if (c >= st.ldc) return;
+        float *C = smem + st.out_off + r * st.ldc + c;
+        C[0] = (c < st.n && in_structure(st.pout, r, c)) ? v0 : 0.f;
+        if (c + 1 < st.ldc) C[1] = (c + 1 < st.n && in_structure(st.pout, r, c + 1)) ? v1 : 0.f;
+    } else {
+        if (c >= st.n) return;
+        float *X = fp.out + inst * fp.out_stride + (size_t)r * st.n + c;
+        const float x0 = finish_entry(v0, fp.add, inst, r, c, st.n, st.pout);
+        if (c + 1 < st.n) {
+            const float x1 = finish_entry(v1, fp.add, inst, r, c + 1, st.n, st.pout);
+            if ((reinterpret_cast<uintptr_t>(X) & 7) == 0) *reinterpret_cast<float2 *>(X) = make_float2(x0, x1);
+            else { X[0] = x0; X[1] = x1; }
+        } else {
+            X[0] = x0;
+        }
+    }
+}
+
+// Whole-tile tensor-core product (m, n multiples of 16 resp. 8*NTW, k a multiple of 8): output tiles of
+// 16 x (8*NTW) dealt round-robin to the warps; no clamping, pointers advance by constants.  The small
+// terms (lo*hi, hi*lo) and the main term (hi*hi) go to separate accumulators: two independent MMA
+// chains per 8-column tile instead of one three times as long.
+template <int NTW>
+__device__ void product_mma_whole(const FusedPlan &fp, const FusedStep &st, float *smem, long long inst) {
+    const float *__restrict__ A = smem + st.a_off;
+    const float *__restrict__ B = smem + st.b_off;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
+    constexpr int TW = 8 * NTW;
+    const int tiles_n = st.n / TW, tiles = (st.m >> 4) * tiles_n;
+    for (int tile = warp; tile < tiles; tile += WARPS) {
+        const int r0 = (tile / tiles_n) << 4, c0 = (tile % tiles_n) * TW;
+        int klo, khi;
+        tile_k_range(st.pa, st.pb, r0, r0 + 16, c0, c0 + TW, st.k, &klo, &khi);
+        klo &= ~7;
+        float main_acc[NTW][4], small_acc[NTW][4];
+#pragma unroll
+        for (int j = 0; j < NTW; ++j)
+#pragma unroll
+            for (int q = 0; q < 4; ++q) main_acc[j][q] = small_acc[j][q] = 0.f;
+        const float *a0p = A + (r0 + g) * st.lda + klo + t, *a1p = a0p + 8 * st.lda;
+        const float *bp = B + (klo + t) * st.ldb + c0 + g;
+        const int b4 = 4 * st.ldb, b8 = 8 * st.ldb;
+#pragma unroll 2
+        for (int l = klo; l < khi; l += 8, a0p += 8, a1p += 8, bp += b8) {
+            uint32_t a_hi[4], a_lo[4];
+            split_tf32(a0p[0], a_hi[0], a_lo[0]);
+            split_tf32(a1p[0], a_hi[1], a_lo[1]);
+            split_tf32(a0p[4], a_hi[2], a_lo[2]);
+            split_tf32(a1p[4], a_hi[3], a_lo[3]);
+#pragma unroll
+            for (int j = 0; j < NTW; ++j) {
+                uint32_t b_hi[2], b_lo[2];
+                split_tf32(bp[8 * j], b_hi[0], b_lo[0]);
+                split_tf32(bp[b4 + 8 * j], b_hi[1], b_lo[1]);
+                mma_tf32(small_acc[j], a_lo, b_hi);
+                mma_tf32(main_acc[j], a_hi, b_hi);
+                mma_tf32(small_acc[j], a_hi, b_lo);
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < NTW; ++j) {
+            store_pair(fp, st, smem, inst, r0 + g, c0 + 8 * j + 2 * t, main_acc[j][0] + small_acc[j][0], main_acc[j][1] + small_acc[j][1]);
+            store_pair(fp, st, smem, inst, r0 + g + 8, c0 + 8 * j + 2 * t, main_acc[j][2] + small_acc[j][2], main_acc[j][3] + small_acc[j][3]);
+        }
+    }
+}
+
+// One product on tensor cores: 16 x 16 output tiles dealt round-robin to the warps.
+__device__ void product_mma(const FusedPlan &fp, const FusedStep &st, float *smem, long long inst) {
+    if (((st.m | st.n) & 15) == 0 && (st.k & 7) == 0) {
+        // with few 16 x 16 tiles, 16 x 8 tiles give every warp of the CTA something to do
+        if ((st.m >> 4) * (st.n >> 4) < WARPS) product_mma_whole<1>(fp, st, smem, inst);
+        else product_mma_whole<2>(fp, st, smem, inst);
+        return;
+    }
+    const float *__restrict__ A = smem + st.a_off;
+    const float *__restrict__ B = smem + st.b_off;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
+    const int tiles_n = (st.n + 15) >> 4, tiles = ((st.m + 15) >> 4) * tiles_n;
+    for (int tile = warp; tile < tiles; tile += WARPS) {
+        const int r0 = (tile / tiles_n) << 4, c0 = (tile % tiles_n) << 4;
+        int klo, khi;
+        tile_k_range(st.pa, st.pb, r0, min(r0 + 16, st.m), c0, min(c0 + 16, st.n), st.k, &klo, &khi);
+        klo &= ~7;
+        float acc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+        // rows / columns outside the matrix are clamped for the address and zeroed by the flag
+        const int ra = min(r0 + g, st.m - 1), rb = min(r0 + g + 8, st.m - 1);
+        const float fa = r0 + g < st.m ? 1.f : 0.f, fb = r0 + g + 8 < st.m ? 1.f : 0.f;
+        const int n0 = min(c0 + g, st.n - 1), n1 = min(c0 + 8 + g, st.n - 1);
+        const float f0 = c0 + g < st.n ? 1.f : 0.f, f1 = c0 + 8 + g < st.n ? 1.f : 0.f;
+        for (int l = klo; l < khi; l += 8) {
+            const int k0 = min(l + t, st.k - 1), k1 = min(l + t + 4, st.k - 1);
+            const float e0 = l + t < st.k ? 1.f : 0.f, e1 = l + t + 4 < st.k ? 1.f : 0.f;
+            uint32_t a_hi[4], a_lo[4], b_hi[2], b_lo[2];
+            split_tf32(A[ra * st.lda + k0] * (fa * e0), a_hi[0], a_lo[0]);
+            split_tf32(A[rb * st.lda + k0] * (fb * e0), a_hi[1], a_lo[1]);
+            split_tf32(A[ra * st.lda + k1] * (fa * e1), a_hi[2], a_lo[2]);
+            split_tf32(A[rb * st.lda + k1] * (fb * e1), a_hi[3], a_lo[3]);
+            split_tf32(B[k0 * st.ldb + n0] * (f0 * e0), b_hi[0], b_lo[0]);
+            split_tf32(B[k1 * st.ldb + n0] * (f0 * e1), b_hi[1], b_lo[1]);
+            mma_tf32(acc[0], a_lo, b_hi);
+            mma_tf32(acc[0], a_hi, b_lo);
+            mma_tf32(acc[0], a_hi, b_hi);
+            split_tf32(B[k0 * st.ldb + n1] * (f1 * e0), b_hi[0], b_lo[0]);
+            split_tf32(B[k1 * st.ldb + n1] * (f1 * e1), b_hi[1], b_lo[1]);
+            mma_tf32(acc[1], a_lo, b_hi);
+            mma_tf32(acc[1], a_hi, b_lo);
+            mma_tf32(acc[1], a_hi, b_hi);
+        }
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            store_pair(fp, st, smem, inst, r0 + g, c0 + 8 * h + 2 * t, acc[h][0], acc[h][1]);
+            store_pair(fp, st, smem, inst, r0 + g + 8, c0 + 8 * h + 2 * t, acc[h][2], acc[h][3]);
+        }
+    }
+}
+
+// One product with plain FMA: cells of 2 rows x 4 columns dealt round-robin to the threads.
+__device__ void product_ffma(const FusedPlan &fp, const FusedStep &st, float *smem, long long inst) {
+    const float *__restrict__ A = smem + st.a_off;
+    const float *__restrict__ B = smem + st.b_off;
+    const int cells_per_row = (st.n + 3) >> 2, row_pairs = (st.m + 1) >> 1;
+    for (int cell = threadIdx.x; cell < row_pairs * cells_per_row; cell += THREADS) {
+        const int r = (cell / cells_per_row) << 1, c = (cell % cells_per_row) << 2;
+        const bool two = r + 1 < st.m;
+        int klo, khi;
+        tile_k_range(st.pa, st.pb, r, two ? r + 2 : r + 1, c, min(c + 4, st.n), st.k, &klo, &khi);
+        float a0[4] = {0.f, 0.f, 0.f, 0.f}, a1[4] = {0.f, 0.f, 0.f, 0.f};
+        const float *ar0 = A + r * st.lda, *ar1 = A + (two ? r + 1 : r) * st.lda;
+        for (int l = klo; l < khi; ++l) {
+            const float4 b = *reinterpret_cast<const float4 *>(B + l * st.ldb + c);   // padded columns hold zeros
+            const float x0 = ar0[l], x1 = ar1[l];
+            a0[0] = fmaf(x0, b.x, a0[0]); a0[1] = fmaf(x0, b.y, a0[1]); a0[2] = fmaf(x0, b.z, a0[2]); a0[3] = fmaf(x0, b.w, a0[3]);
+            a1[0] = fmaf(x1, b.x, a1[0]); a1[1] = fmaf(x1, b.y, a1[1]); a1[2] = fmaf(x1, b.z, a1[2]); a1[3] = fmaf(x1, b.w, a1[3]);
+        }
+        store_pair(fp, st, smem, inst, r, c, a0[0], a0[1]);
+        store_pair(fp, st, smem, inst, r, c + 2, a0[2], a0[3]);
+        if (two) {
+            store_pair(fp, st, smem, inst, r + 1, c, a1[0], a1[1]);
+            store_pair(fp, st, smem, inst, r + 1, c + 2, a1[2], a1[3]);
+        }
+    }
+}
+
+template <bool MMA>
+__global__ void __launch_bounds__(THREADS)
+fused_small_kernel(const FusedPlan fp) {
+    extern __shared__ __align__(16) float smem[];
+    for (long long inst = blockIdx.x; inst < fp.batch; inst += gridDim.x) {
+        for (int i = 0; i < fp.n_ops; ++i) {
+            const FusedOperand &op = fp.ops[i];
+            load_operand(smem + op.smem_off, op.ptr + inst * op.stride, op.rows, op.cols, op.ld, op.prop);
+        }
+        cp_async_wait_all();
+        __syncthreads();
+        for (int s = 0; s < fp.n_steps; ++s) {
+            if (MMA) product_mma(fp, fp.steps[s], smem, inst);
+            else product_ffma(fp, fp.steps[s], smem, inst);
+            __syncthreads();
+        }
+    }
+}
+
+int g_sm_count = 0;
+int g_max_smem[2] = {0, 0};
+
+}  // namespace
+
+cudaError_t launch_fused_small(const FusedPlan &fp, size_t smem_bytes, cudaStream_t stream) {
+    if (!g_sm_count) {
+        int dev = 0;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&g_sm_count, cudaDevAttrMultiProcessorCount, dev);
+    }
+    const int v = fp.use_mma ? 1 : 0;
+    if ((int)smem_bytes > g_max_smem[v]) {
+        cudaError_t e = v ? cudaFuncSetAttribute(fused_small_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes)
+                          : cudaFuncSetAttribute(fused_small_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
+        if (e != cudaSuccess) return e;
+        g_max_smem[v] = (int)smem_bytes;
+    }
+    // enough CTAs to fill every SM several times over; each walks instances with a grid stride
+    long long per_sm = smem_bytes ? (long long)(220 * 1024) / (long long)smem_bytes : 8;
+    if (per_sm > 8) per_sm = 8;
+    if (per_sm < 1) per_sm = 1;
+    long long grid = (long long)g_sm_count * per_sm;
+    if (grid > fp.batch) grid = fp.batch;
+    if (v) fused_small_kernel<true><<<(unsigned)grid, THREADS, smem_bytes, stream>>>(fp);
+    else fused_small_kernel<false><<<(unsigned)grid, THREADS, smem_bytes, stream>>>(fp);
+    return cudaGetLastError();
+}
+
+}  // namespace mom

@@ -52,6 +52,11 @@ struct mom_plan {
     mom_matrix_desc_t product_desc{};          // chain value before the Add terms
     mom_matrix_desc_t result_desc{};
     size_t workspace_per_instance = 0;
+    // fused small-equation kernel: whole plan in shared memory, one instance per CTA (no workspace)
+    bool fused_ok = false;
+    size_t fused_smem_bytes = 0;
+    std::vector<int> fused_value_off;          // shared-memory offset (floats) per value id; -1 = not resident
+    std::vector<int> fused_value_ld;           // shared-memory leading dimension (floats) per value id
     mutable mom::DeviceState *dev = nullptr;
     mutable int32_t last_launches = 0;
     bool step_timing = false;

@@ -5,6 +5,7 @@
 #include <cstring>
 #include <new>
 
+#include "fused_small.h"
 #include "mom_internal.h"
 
 namespace {
@@ -244,6 +245,41 @@ mom_status_t mom_equation_plan(const mom_matrix_desc_t *chain, int32_t n_chain,
             }
         }
         p->workspace_per_instance = pack(items);
+
+        // Small equations run as one fused kernel with every operand and intermediate in shared memory.
+        {
+            bool any_tc = false;
+            for (const auto &st : p->steps) any_tc |= st.pub.uses_tensor_cores != 0;
+            const int values = n_chain + ns;
+            p->fused_value_off.assign(values, -1);
+            size_t floats = 0;
+            bool ok = ns >= 1 && ns <= mom::FUSED_MAX_STEPS && (int)p->kept.size() <= mom::FUSED_MAX_OPERANDS &&
+                      n_add <= mom::MAX_FUSED_ADD && !any_tc;
+            // every value feeds exactly one product: remember on which side
+            std::vector<char> is_rhs(values, 0);
+            for (const auto &st : p->steps) is_rhs[st.pub.rhs] = 1;
+            p->fused_value_ld.assign(values, 0);
+            if (ok) {
+                for (int id : p->kept) {
+                    p->fused_value_off[id] = (int)floats;
+                    p->fused_value_ld[id] = mom::fused_ld((int)chain[id].cols, is_rhs[id] != 0);
+                    floats += (size_t)chain[id].rows * p->fused_value_ld[id];
+                    if (floats * sizeof(float) > mom::FUSED_MAX_SMEM) { ok = false; break; }
+                }
+            }
+            if (ok) {
+                for (int s = 0; s + 1 < ns; ++s) {
+                    const int id = n_chain + s;
+                    p->fused_value_off[id] = (int)floats;
+                    p->fused_value_ld[id] = mom::fused_ld((int)p->steps[s].pub.n, is_rhs[id] != 0);
+                    floats += (size_t)p->steps[s].pub.m * p->fused_value_ld[id];
+                    if (floats * sizeof(float) > mom::FUSED_MAX_SMEM) { ok = false; break; }
+                }
+            }
+            p->fused_ok = ok;
+            p->fused_smem_bytes = ok ? floats * sizeof(float) : 0;
+            if (ok) p->workspace_per_instance = 0;
+        }
     } catch (const std::bad_alloc &) {
         delete p;
         return MOM_ERR_ALLOC;

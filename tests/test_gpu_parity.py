@@ -119,6 +119,22 @@ def test_config_batched(variant):
     check_against_oracle(eq, x, plan, chain, add, instances=[0, 1, 63, 64, 2047, 4095])
 
 
+@pytest.mark.parametrize("variant", [mom.VARIANT_FFMA, mom.VARIANT_3XTF32], ids=VNAME.get)
+@pytest.mark.parametrize("n", [1, 5, 8, 12, 16, 24, 27, 32])
+def test_batched_small_chains(n, variant):
+    # plans of the form M1*(M2*(M3*B)) with a narrow B, batched: the fused shared-memory kernel
+    for chain, add in [
+        ((Operand(64, 64, L), Operand(64, 64, G), Operand(64, n, G)), (Operand(64, n, G),)),
+        ((Operand(40, 72, G, "normal"), Operand(72, 72, U), Operand(72, 52, G), Operand(52, n, G)), ()),
+        ((Operand(36, 36, U), Operand(36, n, G)), (Operand(36, n, G), Operand(36, n, G))),
+        ((Operand(100, 20, G), Operand(20, n, G)), ()),
+        ((Operand(28, 26, G), Operand(26, 26, L), Operand(26, 4 * ((n + 3) // 4), G)), ()),      # k = 26: not a multiple of 4
+    ]:
+        eq = Equation(f"narrow_n{n}", 40 + n, chain, add, batch=45)
+        plan = mom.mom_equation_plan(eq.descs(), eq.add_descs(), variant)
+        both(eq, variant)
+
+
 @pytest.mark.parametrize("variant", VARIANTS, ids=VNAME.get)
 def test_batched_with_padding_between_instances(variant):
     eq = wl.config_batched(batch=5)
@@ -184,11 +200,13 @@ def test_host_entry_point_matches_device_entry_point(variant):
 
 
 def test_argument_errors_are_reported_before_any_launch():
-    eq = wl.config_tiny()
+    # large enough not to run as one fused shared-memory kernel, so that it needs a workspace
+    eq = Equation("errors", 5, (Operand(200, 200, L), Operand(200, 200, G), Operand(200, 48, G)))
     chain, _ = wl.generate(eq)
     plan = mom.mom_equation_plan(eq.descs(), (), mom.VARIANT_FFMA)
+    assert plan.workspace_bytes() > 0
     d = [torch.from_numpy(a).cuda() for a in chain]
-    out = torch.zeros(64 * 48 + 4, dtype=torch.float32, device="cuda")
+    out = torch.zeros(200 * 48 + 4, dtype=torch.float32, device="cuda")
     ws = torch.empty(plan.workspace_bytes(), dtype=torch.uint8, device="cuda")
     ptrs = [t.data_ptr() for t in d]
     def status(**kw):
