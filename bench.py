@@ -30,6 +30,22 @@ UNIT = "GFLOP/s"
 TF32_OVER_BF16 = 1.1 / 2.25          # nominal dense tensor ratio used to carry the measured bf16 peak to tf32
 
 
+def max_over_ranks(value_ms: float, world: int, device="cpu") -> float:
+    """Slowest rank's time (every rank gets it); a no-op for one rank."""
+    if world <= 1:
+        return float(value_ms)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([value_ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_gflops(useful_flops_per_replica: int, world: int, ms_per_step: float) -> float:
+    """Replicas are independent: the job's throughput is every rank's work over the slowest rank's time."""
+    return useful_flops_per_replica * world / (ms_per_step * 1e-3) / 1e9
+
+
 def headline_equation() -> wl.Equation:
     return wl.config_large_square()
 
@@ -109,6 +125,7 @@ def run_reference(args):
 # ------------------------------------------------------------------------------------------------
 
 class ClockSampler:
+    """nvidia-smi polled in the background; only samples taken inside [begin(), end()] are reported."""
     QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
              "clocks_event_reasons.sw_power_cap")
@@ -116,27 +133,53 @@ class ClockSampler:
     def __init__(self, device_index: int):
         self.proc = None
         self.device_index = device_index
+        self.lines = []          # (host time, text)
+        self.t0 = self.t1 = None
+        self.thread = None
 
     def start(self):
+        import threading
         try:
             self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
-                                          "-lms", "100", "-i", str(self.device_index)],
+                                          "-lms", "50", "-i", str(self.device_index)],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except OSError:
             self.proc = None
+            return
+
+        def reader():
+            for line in self.proc.stdout:
+                self.lines.append((time.time(), line))
+        self.thread = threading.Thread(target=reader, daemon=True)
+        self.thread.start()
+
+    def wait_for_first_sample(self, timeout: float = 10.0):
+        t = time.time()
+        while self.proc is not None and not self.lines and time.time() - t < timeout:
+            time.sleep(0.05)
+
+    def begin(self):
+        self.t0 = time.time()
+
+    def end(self):
+        self.t1 = time.time()
 
     def stop(self):
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.06)
         self.proc.terminate()
         try:
-            out, _ = self.proc.communicate(timeout=5)
+            self.proc.wait(timeout=5)
         except subprocess.TimeoutExpired:
             self.proc.kill()
-            out, _ = self.proc.communicate()
+        if self.thread is not None:
+            self.thread.join(timeout=2)
         sm, mx, power, reasons = [], [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for line in out.strip().splitlines():
+        for stamp, line in list(self.lines):
+            if self.t0 is not None and not (self.t0 <= stamp <= (self.t1 or stamp) + 0.05):
+                continue
             f = [x.strip() for x in line.split(",")]
             if len(f) < 9:
                 continue
@@ -220,6 +263,8 @@ def run_gpu(args):
 
     eq = headline_equation()
     sampler = ClockSampler(local)
+    if not args.only:
+        sampler.start()
 
     if args.only:
         # one named configuration, nothing else: the small case for profiler captures
@@ -257,7 +302,8 @@ def run_gpu(args):
             plan.execute(cp, ap, out.data_ptr(), ws.data_ptr(), wsb, stream.cuda_stream)
     barrier()
     plan.enable_step_timing(True)      # per-kernel events, averaged over the timed executes
-    sampler.start()
+    sampler.wait_for_first_sample()
+    sampler.begin()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     prod_ms = [0.0] * n_steps
     pre_ms = [0.0] * n_steps
@@ -269,6 +315,7 @@ def run_gpu(args):
             launches += plan.last_launch_count()
         e1.record(stream)
     barrier()
+    sampler.end()
     clocks = sampler.stop()
     total_ms = e0.elapsed_time(e1)
     # per-kernel mean times over the timed region (events recorded inside it, on the same stream)
@@ -277,14 +324,11 @@ def run_gpu(args):
         prod_ms[i], pre_ms[i] = a, b
     if plan.device_status() != (0, 0):
         raise RuntimeError("device-side wait timed out")
-    t = torch.tensor([total_ms], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    total_ms = float(t.item())
+    total_ms = max_over_ranks(total_ms, world, "cuda")
     ms_per_step = total_ms / args.steps
     mul, addf = plan.flops()
     useful = mul + addf
-    value = useful * world / (ms_per_step * 1e-3) / 1e9
+    value = whole_job_gflops(useful, world, ms_per_step)
 
     # ---- roofline of the dominant kernel (the product kernel): useful FLOPs of its launches / their device time
     steps_info = plan.steps()
@@ -393,7 +437,7 @@ def rd_elems(plan):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--variant", default="3xtf32", choices=["3xtf32", "ffma"])

@@ -309,6 +309,247 @@ product_tc_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_con
     if (warp == 1) ptx::tmem_dealloc(tmem_base, TMEM_COLS);
 }
 
+// ---------------------------------------------------------------------------------------------
+// CTA-pair variant (cta_group::2): two CTAs of a cluster share one 256 x 256 output tile.  Each CTA
+// loads its own 128 rows of A and only its own half (128 columns) of B -- the tensor cores of the pair
+// exchange the B halves -- so a stage is 64 KiB instead of 96 (three stages fit) and the L2 / shared
+// memory traffic per flop drops by a third.  The leader CTA (cluster rank 0) issues every MMA; each CTA
+// counts its own loads on its own "full" barrier and the peer relays completion to the leader with one
+// remote arrive per stage; tcgen05.commit with a CTA mask releases the stage in both CTAs and publishes
+// the accumulator to both epilogues; the peer's epilogue warps tell the leader over the cluster when an
+// accumulator may be overwritten.
+// ---------------------------------------------------------------------------------------------
+constexpr int P_BM = 2 * BM;                  // rows of a pair tile
+constexpr int P_STAGES = 3;
+constexpr int P_A_PLANE_BYTES = BM * BK * 4;          // 16 KiB: this CTA's 128 rows
+constexpr int P_B_PLANE_BYTES = (BN / 2) * BK * 4;    // 16 KiB: this CTA's 128 columns of B
+constexpr int P_STAGE_BYTES = 2 * P_A_PLANE_BYTES + 2 * P_B_PLANE_BYTES;   // 64 KiB
+constexpr int P_NUM_BARRIERS = 3 * P_STAGES + 4 + 1;
+constexpr int P_SMEM_BYTES = 1024 + P_STAGES * P_STAGE_BYTES + EPI_BYTES + 256;
+static_assert(P_SMEM_BYTES <= 227 * 1024, "shared memory budget");
+
+__global__ void __launch_bounds__(THREADS, 1)
+product_tc_pair_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_constant__ CUtensorMap map_a_lo,
+                       const __grid_constant__ CUtensorMap map_b_hi, const __grid_constant__ CUtensorMap map_b_lo,
+                       const __grid_constant__ CUtensorMap map_c, const TcParams prm) {
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ int abort_word;
+    const uint32_t base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t epi = base + P_STAGES * P_STAGE_BYTES;
+    const uint32_t bars = epi + EPI_BYTES;
+    auto stage_addr = [&](int s) { return base + s * P_STAGE_BYTES; };
+    auto full_bar = [&](int s) { return bars + 8 * s; };
+    auto empty_bar = [&](int s) { return bars + 8 * (P_STAGES + s); };
+    auto tmem_full_bar = [&](int a) { return bars + 8 * (2 * P_STAGES + a); };
+    auto tmem_empty_bar = [&](int a) { return bars + 8 * (2 * P_STAGES + 2 + a); };
+    const uint32_t drain_bar = bars + 8 * (2 * P_STAGES + 4);
+    auto peer_ready_bar = [&](int s) { return bars + 8 * (2 * P_STAGES + 5 + s); };   // leader: the peer's stage has landed
+    const uint32_t tmem_slot = bars + 8 * P_NUM_BARRIERS;
+    volatile int *abort_flag = &abort_word;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = ptx::cluster_cta_rank();           // 0 = leader
+    const int pair = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
+
+    if (threadIdx.x == 0) {
+        abort_word = 0;
+        for (int s = 0; s < P_STAGES; ++s) {
+            ptx::mbar_init(full_bar(s), 1);
+            ptx::mbar_init(empty_bar(s), 1);
+            ptx::mbar_init(peer_ready_bar(s), 1);
+        }
+        ptx::mbar_init(tmem_full_bar(0), 1);
+        ptx::mbar_init(tmem_full_bar(1), 1);
+        ptx::mbar_init(tmem_empty_bar(0), 8);               // four epilogue warps in each CTA
+        ptx::mbar_init(tmem_empty_bar(1), 8);
+        ptx::mbar_init(drain_bar, 1);
+        ptx::fence_barrier_init();
+    }
+    if (warp == 1) {
+        ptx::tmem_alloc_pair(tmem_slot, TMEM_COLS);
+        ptx::tmem_relinquish_pair();
+    }
+    ptx::tc_fence_before_sync();
+    ptx::cluster_sync();                                     // the peer's barriers exist before anything signals them
+    ptx::tc_fence_after_sync();
+    uint32_t tmem_base;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(tmem_base) : "r"(tmem_slot));
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer (both CTAs)
+        uint32_t it = 0;
+        bool ok = true;
+        for (int t = pair; t < prm.num_tiles && ok; t += num_pairs) {
+            const int4 tile = prm.tiles[t];
+            for (int kb = tile.z; kb < tile.w; kb += BK, ++it) {
+                const int s = it % P_STAGES;
+                const uint32_t parity = ((it / P_STAGES) & 1) ^ 1;
+                if (lane == 0) ok = wait_barrier(empty_bar(s), parity, abort_flag, prm.status, (1 << 24) | (s << 16) | (t & 0xFFFF));
+                ok = __shfl_sync(0xffffffffu, ok, 0);
+                if (!ok) break;
+                // each CTA counts its own loads on its own barrier (per-transaction updates of a barrier in the
+                // other SM were several times slower); the peer's MMA warp relays "landed" to the leader
+                if (lane == 0) ptx::mbar_arrive_expect_tx(full_bar(s), P_STAGE_BYTES);
+                __syncwarp();
+                const uint32_t st = stage_addr(s);
+                const int a_row = tile.x + (int)rank * BM, b_row = tile.y + (int)rank * (BN / 2);
+                if (lane == 0) ptx::tma_load_2d(st, &map_a_hi, kb, a_row, full_bar(s));
+                else if (lane == 1) ptx::tma_load_2d(st + P_A_PLANE_BYTES, &map_a_lo, kb, a_row, full_bar(s));
+                else if (lane == 2) ptx::tma_load_2d(st + 2 * P_A_PLANE_BYTES, &map_b_hi, kb, b_row, full_bar(s));
+                else if (lane == 3) ptx::tma_load_2d(st + 2 * P_A_PLANE_BYTES + P_B_PLANE_BYTES, &map_b_lo, kb, b_row, full_bar(s));
+            }
+        }
+        // failure path: give loads that are still in flight time to land before this CTA's memory goes away
+        if (*abort_flag && lane == 0) {
+            const unsigned long long t0 = global_ns();
+            while (global_ns() - t0 < 200000ull) { }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ peer CTA: relay "stage landed" to the leader
+        if (lane == 0 && rank != 0) {
+            uint32_t it = 0;
+            bool ok = true;
+            for (int t = pair; t < prm.num_tiles && ok; t += num_pairs) {
+                const int4 tile = prm.tiles[t];
+                for (int kb = tile.z; kb < tile.w; kb += BK, ++it) {
+                    const int s = it % P_STAGES;
+                    ok = wait_barrier(full_bar(s), (it / P_STAGES) & 1, abort_flag, prm.status, (7 << 24) | (s << 16) | (t & 0xFFFF));
+                    if (!ok) break;
+                    ptx::mbar_arrive_cluster(ptx::map_to_cta(peer_ready_bar(s), 0));
+                }
+            }
+        }
+        // ------------------------------------------------------------------ MMA issuer (leader CTA, one thread)
+        if (lane == 0 && rank == 0) {
+            constexpr uint32_t idesc = ptx::instr_desc_tf32(P_BM, BN, 0, 0);
+            uint32_t it = 0, acc_it = 0;
+            bool ok = true;
+            for (int t = pair; t < prm.num_tiles && ok; t += num_pairs) {
+                const int4 tile = prm.tiles[t];
+                if (tile.z >= tile.w) continue;
+                const uint32_t acc = acc_it & 1;
+                ok = wait_barrier(tmem_empty_bar(acc), ((acc_it >> 1) & 1) ^ 1, abort_flag, prm.status, (2 << 24) | (acc << 16) | (t & 0xFFFF));
+                if (!ok) break;
+                ptx::tc_fence_after_sync();
+                const uint32_t d = tmem_base + acc * BN;
+                uint32_t accumulate = 0;
+                for (int kb = tile.z; kb < tile.w; kb += BK, ++it) {
+                    const int s = it % P_STAGES;
+                    ok = wait_barrier(full_bar(s), (it / P_STAGES) & 1, abort_flag, prm.status, (3 << 24) | (s << 16) | (t & 0xFFFF)) &&
+                         wait_barrier(peer_ready_bar(s), (it / P_STAGES) & 1, abort_flag, prm.status, (8 << 24) | (s << 16) | (t & 0xFFFF));
+                    if (!ok) break;
+                    ptx::tc_fence_after_sync();
+                    const uint32_t a_hi = stage_addr(s), a_lo = a_hi + P_A_PLANE_BYTES;
+                    const uint32_t b_hi = a_hi + 2 * P_A_PLANE_BYTES, b_lo = b_hi + P_B_PLANE_BYTES;
+#pragma unroll
+                    for (int ks = 0; ks < BK / 8; ++ks) {
+                        const uint64_t da_hi = kmajor_desc(a_hi, ks), da_lo = kmajor_desc(a_lo, ks);
+                        const uint64_t db_hi = kmajor_desc(b_hi, ks), db_lo = kmajor_desc(b_lo, ks);
+                        ptx::mma_tf32_pair(d, da_lo, db_hi, idesc, accumulate);
+                        ptx::mma_tf32_pair(d, da_hi, db_lo, idesc, 1);
+                        ptx::mma_tf32_pair(d, da_hi, db_hi, idesc, 1);
+                        accumulate = 1;
+                    }
+                    ptx::mma_commit_pair(empty_bar(s), 3);           // both CTAs may refill this stage
+                }
+                if (!ok) break;
+                ptx::mma_commit_pair(tmem_full_bar(acc), 3);          // both epilogues may read
+                ++acc_it;
+            }
+            if (*abort_flag) {
+                ptx::mma_commit_pair(drain_bar, 1);
+                for (uint32_t i = 0; i < (1u << 20); ++i)
+                    if (ptx::mbar_try_wait(drain_bar, 0)) break;
+            }
+        }
+        __syncwarp();
+    } else {
+        // ------------------------------------------------------------------ epilogue (warps 2..5, both CTAs)
+        const int q = warp & 3;
+        const uint32_t stage_buf = epi + (warp - 2) * 2 * EPI_BOX_BYTES;
+        uint32_t acc_it = 0, store_it = 0;
+        bool ok = true;
+        for (int t = pair; t < prm.num_tiles && ok; t += num_pairs) {
+            const int4 tile = prm.tiles[t];
+            const bool zero_tile = tile.z >= tile.w;
+            const uint32_t acc = acc_it & 1;
+            if (!zero_tile) {
+                ok = wait_barrier(tmem_full_bar(acc), (acc_it >> 1) & 1, abort_flag, prm.status, (4 << 24) | (acc << 16) | (t & 0xFFFF));
+                if (!ok) break;
+                ptx::tc_fence_after_sync();
+            }
+            const int row0 = tile.x + (int)rank * BM + q * 32;   // first row of this warp's slab
+            const int r = row0 + lane;
+            const int rows_left = prm.m - row0;
+#pragma unroll 1
+            for (int c = 0; c < BN / 32; ++c) {
+                const int col0 = tile.y + c * 32;
+                if (col0 >= prm.n) break;
+                float v[32];
+                if (!zero_tile) {
+                    ptx::tmem_ld_32cols(tmem_base + acc * BN + c * 32 + ((uint32_t)(q * 32) << 16), v);
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) v[j] = 0.0f;
+                }
+                if (rows_left > 0) {
+                    const bool row_ok = r < prm.m;
+                    for (int a = 0; a < prm.add.count; ++a) {
+                        const float *p = prm.add.ptr[a];
+                        if (p) {
+                            if (row_ok) {
+                                const float4 *src = reinterpret_cast<const float4 *>(p + (long long)r * prm.n + col0);
+#pragma unroll
+                                for (int j = 0; j < 8; ++j) {
+                                    if (col0 + 4 * j < prm.n) {
+                                        const float4 x = __ldg(src + j);
+                                        v[4 * j] += x.x; v[4 * j + 1] += x.y; v[4 * j + 2] += x.z; v[4 * j + 3] += x.w;
+                                    }
+                                }
+                            }
+                        } else {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) v[j] += (col0 + j == r) ? 1.0f : 0.0f;
+                        }
+                    }
+                    if (prm.pout != MOM_GENERAL) {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) v[j] = in_structure(prm.pout, r, col0 + j) ? v[j] : 0.0f;
+                    }
+                    const uint32_t buf = stage_buf + (store_it & 1) * EPI_BOX_BYTES;
+                    if (lane == 0) ptx::tma_store_wait_read<1>();
+                    __syncwarp();
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        const uint32_t dst = buf + lane * 128 + ((j ^ (lane & 7)) << 4);
+                        asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "f"(v[4 * j]), "f"(v[4 * j + 1]),
+                                     "f"(v[4 * j + 2]), "f"(v[4 * j + 3]) : "memory");
+                    }
+                    ptx::fence_proxy_async_smem();
+                    __syncwarp();
+                    if (lane == 0) {
+                        ptx::tma_store_2d(&map_c, col0, row0, buf);
+                        ptx::tma_store_commit();
+                    }
+                    ++store_it;
+                }
+            }
+            if (!zero_tile) {
+                ptx::tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive_cluster(ptx::map_to_cta(tmem_empty_bar(acc), 0));
+                ++acc_it;
+            }
+        }
+        if (lane == 0) ptx::tma_store_wait_all();
+    }
+
+    ptx::tc_fence_before_sync();
+    ptx::cluster_sync();                                     // nobody leaves while the peer may still signal it
+    ptx::tc_fence_after_sync();
+    if (warp == 1) ptx::tmem_dealloc_pair(tmem_base, TMEM_COLS);
+}
+
 // hi = rna_tf32(a), lo = rna_tf32(a - hi).  The planes keep the operand's layout (rows x cols) or, with
 // TRANSPOSE, hold the transposed operand (cols x rows).  One CTA handles a 64 x 64 piece; pieces whose
 // enclosing SPLIT_BLOCK x SPLIT_BLOCK block lies wholly outside a triangular operand's structure are
@@ -413,16 +654,41 @@ mom_status_t tc_prepare(const mom_plan &p, TcPlanState &s) {
         if (!st.uses_tensor_cores) continue;
         const int m = (int)st.m, n = (int)st.n, k = (int)st.k;
         std::vector<int4> &tab = tables[i];
-        for (int r0 = 0; r0 < m; r0 += BM)
+        // CTA pairs (256-row tiles) once there are enough of them to occupy most of the GPU's 74 pairs
+        const long long pair_tiles = (long long)((m + P_BM - 1) / P_BM) * ((n + BN - 1) / BN);
+        s.steps[i].pair = m >= P_BM && pair_tiles >= 48;
+        const int tile_rows = s.steps[i].pair ? P_BM : BM;
+        for (int r0 = 0; r0 < m; r0 += tile_rows)
             for (int c0 = 0; c0 < n; c0 += BN) {
                 int klo, khi;
-                tile_k_range(st.lhs_property, st.rhs_property, r0, std::min(r0 + BM, m), c0, std::min(c0 + BN, n), k, &klo, &khi);
+                tile_k_range(st.lhs_property, st.rhs_property, r0, std::min(r0 + tile_rows, m), c0, std::min(c0 + BN, n), k, &klo, &khi);
                 if (klo >= khi) { klo = 0; khi = 0; }
                 klo = klo / BK * BK;                      // leading extra elements are stored zeros
                 tab.push_back(make_int4(r0, c0, klo, khi));
             }
-        // heaviest tiles first so that the persistent CTAs finish together; zero tiles last
-        std::stable_sort(tab.begin(), tab.end(), [](const int4 &a, const int4 &b) { return (a.w - a.z) > (b.w - b.z); });
+        // Order.  Unequal tiles (triangular operands): heaviest first, so that the persistent CTAs, which
+        // take tiles round-robin, finish together; structurally zero tiles last.  Equal tiles (general
+        // operands): tiles that run at the same time should share operand panels in L2, so they are
+        // grouped into super-tiles of SUPER_ROWS x SUPER_COLS tiles (about one wave of CTAs, equal bytes
+        // of A and B panels).  (Super-tiles for unequal tiles cost more in imbalance than they saved.)
+        bool uniform = true;
+        for (const int4 &t : tab) uniform &= (t.w - t.z) == (tab[0].w - tab[0].z);
+        if (!uniform) {
+            std::stable_sort(tab.begin(), tab.end(), [](const int4 &a, const int4 &b) { return (a.w - a.z) > (b.w - b.z); });
+        } else {
+            constexpr int SUPER_ROWS = 16, SUPER_COLS = 8;
+            const int super_cols = ((n + BN - 1) / BN + SUPER_COLS - 1) / SUPER_COLS;
+            auto super_of = [&](const int4 &t) { return (t.x / BM / SUPER_ROWS) * super_cols + (t.y / BN / SUPER_COLS); };
+            std::vector<long long> super_work((size_t)(((m + BM - 1) / BM + SUPER_ROWS - 1) / SUPER_ROWS + 1) * super_cols, 0);
+            for (const int4 &t : tab) super_work[super_of(t)] += t.w - t.z;
+            std::stable_sort(tab.begin(), tab.end(), [&](const int4 &a, const int4 &b) {
+                const bool za = a.w <= a.z, zb = b.w <= b.z;
+                if (za != zb) return zb;
+                const int sa = super_of(a), sb = super_of(b);
+                if (sa != sb) return super_work[sa] != super_work[sb] ? super_work[sa] > super_work[sb] : sa < sb;
+                return (a.w - a.z) > (b.w - b.z);
+            });
+        }
         total += tab.size();
     }
     if (total == 0) { s.ready = true; return MOM_OK; }
@@ -477,8 +743,8 @@ mom_status_t tc_launch_step(const mom_plan &p, TcPlanState &s, int step, const P
     CUtensorMap ma_hi, ma_lo, mb_hi, mb_lo, mc;
     bool ok = make_map(&ma_hi, a_hi, a.m, a.k, BM, BK, OPERAND_TMA_SWIZZLE) &&
               make_map(&ma_lo, a_lo, a.m, a.k, BM, BK, OPERAND_TMA_SWIZZLE) &&
-              make_map(&mb_hi, b_hi, a.n, a.k, BN, BK, OPERAND_TMA_SWIZZLE) &&
-              make_map(&mb_lo, b_lo, a.n, a.k, BN, BK, OPERAND_TMA_SWIZZLE) &&
+              make_map(&mb_hi, b_hi, a.n, a.k, s.steps[step].pair ? BN / 2 : BN, BK, OPERAND_TMA_SWIZZLE) &&
+              make_map(&mb_lo, b_lo, a.n, a.k, s.steps[step].pair ? BN / 2 : BN, BK, OPERAND_TMA_SWIZZLE) &&
               make_map(&mc, a.C, a.m, a.n, 32, 32, CU_TENSOR_MAP_SWIZZLE_128B);
     if (!ok) return MOM_ERR_CUDA;
 
@@ -490,8 +756,40 @@ mom_status_t tc_launch_step(const mom_plan &p, TcPlanState &s, int step, const P
     prm.pout = a.pout;
     prm.add = a.add;
     prm.status = status;
-    const int grid = std::min(prm.num_tiles, g_sm_count);
-    product_tc_kernel<<<grid, THREADS, SMEM_BYTES, stream>>>(ma_hi, ma_lo, mb_hi, mb_lo, mc, prm);
+    if (s.steps[step].pair) {
+        static bool pair_attr_set = false;
+        if (!pair_attr_set) {
+            if (cudaFuncSetAttribute(product_tc_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, P_SMEM_BYTES) != cudaSuccess)
+                return MOM_ERR_CUDA;
+            pair_attr_set = true;
+        }
+        cudaLaunchConfig_t cfg;
+        std::memset(&cfg, 0, sizeof(cfg));
+        cfg.gridDim = dim3(g_sm_count / 2 * 2);
+        cfg.blockDim = dim3(THREADS);
+        cfg.dynamicSmemBytes = P_SMEM_BYTES;
+        cfg.stream = stream;
+        cudaLaunchAttribute attr;
+        attr.id = cudaLaunchAttributeClusterDimension;
+        attr.val.clusterDim.x = 2;
+        attr.val.clusterDim.y = 1;
+        attr.val.clusterDim.z = 1;
+        cfg.attrs = &attr;
+        cfg.numAttrs = 1;
+        // A persistent grid must not exceed what is co-resident: not every SM can host half of a CTA pair
+        // (the pair must sit on one TPC), so ask how many clusters fit instead of assuming SMs / 2.
+        static int max_pairs = 0;
+        if (!max_pairs) {
+            int n = 0;
+            if (cudaOccupancyMaxActiveClusters(&n, product_tc_pair_kernel, &cfg) != cudaSuccess || n < 1) return MOM_ERR_CUDA;
+            max_pairs = n;
+        }
+        cfg.gridDim = dim3(2 * std::min(prm.num_tiles, max_pairs));
+        if (cudaLaunchKernelEx(&cfg, product_tc_pair_kernel, ma_hi, ma_lo, mb_hi, mb_lo, mc, prm) != cudaSuccess) return MOM_ERR_CUDA;
+    } else {
+        const int grid = std::min(prm.num_tiles, g_sm_count);
+        product_tc_kernel<<<grid, THREADS, SMEM_BYTES, stream>>>(ma_hi, ma_lo, mb_hi, mb_lo, mc, prm);
+    }
     if (cudaGetLastError() != cudaSuccess) return MOM_ERR_CUDA;
     *launches = 3;
     return MOM_OK;

@@ -1,0 +1,47 @@
+"""The benchmark's multi-rank bookkeeping (replicas only: barrier, slowest rank's time, summed work) on CPU with gloo."""
+import os
+import sys
+
+import pytest
+
+torch = pytest.importorskip("torch")
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _worker(rank, world, port, out):
+    sys.path.insert(0, ROOT)
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    import bench
+    dist.barrier()
+    ms = bench.max_over_ranks(10.0 + 5.0 * rank, world)          # rank 1 is the slow one
+    value = bench.whole_job_gflops(2_000_000_000, world, ms)
+    out.put((rank, ms, value))
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_two_ranks_report_the_slowest_time_and_the_summed_work():
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    port = 29500 + os.getpid() % 2000
+    procs = [ctx.Process(target=_worker, args=(r, 2, port, q)) for r in range(2)]
+    for p in procs:
+        p.start()
+    results = sorted(q.get(timeout=120) for _ in procs)
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    for rank, ms, value in results:
+        assert ms == 15.0                                            # max over ranks, seen by both
+        assert value == pytest.approx(2 * 2e9 / 15e-3 / 1e9)        # two replicas' work over that time
+
+
+def test_single_rank_is_a_no_op():
+    sys.path.insert(0, ROOT)
+    import bench
+    assert bench.max_over_ranks(7.5, 1) == 7.5
+    assert bench.whole_job_gflops(10**9, 1, 1.0) == pytest.approx(1000.0)
