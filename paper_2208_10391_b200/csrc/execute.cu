@@ -193,6 +193,8 @@ mom_status_t execute_impl(const mom_plan *p, const float *const *chain_ptrs, con
                 const StepImpl &prod = p->steps[id - n_chain];
                 const long long elems = (long long)prod.pub.m * prod.pub.n;
                 // grid.z batching keeps one copy of each intermediate per instance, instance-major
+                // (a tensor-core step that feeds another one leaves no f32 intermediate: its consumer reads planes)
+                if (prod.out_off == SIZE_MAX) return Operand{nullptr, elems};
                 return Operand{reinterpret_cast<const float *>(static_cast<char *>(workspace) + prod.out_off * (size_t)nb), elems};
             };
             const Operand A = value(stp.pub.lhs), B = value(stp.pub.rhs);
@@ -207,7 +209,8 @@ mom_status_t execute_impl(const mom_plan *p, const float *const *chain_ptrs, con
                 a.pout = p->result_desc.property;
                 added = add_terms(0, &a.add);
             } else {
-                a.C = reinterpret_cast<float *>(static_cast<char *>(workspace) + stp.out_off * (size_t)nb);
+                a.C = stp.out_off == SIZE_MAX ? nullptr
+                                              : reinterpret_cast<float *>(static_cast<char *>(workspace) + stp.out_off * (size_t)nb);
                 a.strideC = (long long)stp.pub.m * stp.pub.n;
                 a.pout = stp.pub.out_property;
                 a.add.count = 0;

@@ -34,6 +34,11 @@ struct StepImpl {
     size_t out_off = SIZE_MAX;      // f32 intermediate written by this step (not for the last step)
     size_t a_hi_off = SIZE_MAX, a_lo_off = SIZE_MAX;   // split planes of the operands (tensor-core steps)
     size_t b_hi_off = SIZE_MAX, b_lo_off = SIZE_MAX;
+    // When this tensor-core step feeds another tensor-core step, its epilogue writes the consumer's hi/lo
+    // planes directly (transposed if the consumer takes it as right operand) and no f32 intermediate exists.
+    int planes_out = 0;             // 0: f32 output; 1: planes as stored (consumer's left operand); 2: transposed planes
+    size_t planes_hi_off = SIZE_MAX, planes_lo_off = SIZE_MAX;
+    bool a_planes_ready = false, b_planes_ready = false;   // this step's operand planes come from the producing step
 };
 
 struct DeviceState;   // launcher-owned, created on first execute (execute.cu)

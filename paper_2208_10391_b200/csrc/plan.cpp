@@ -229,22 +229,47 @@ mom_status_t mom_equation_plan(const mom_matrix_desc_t *chain, int32_t n_chain,
             const bool worth_it = (double)m * (double)n * (double)k >= (double)(1 << 23);
             st.pub.uses_tensor_cores =
                 (variant == MOM_VARIANT_3XTF32 && addressable && worth_it) || ((int)variant == 2 && addressable);
-            if (!st.is_last) {
-                int consumer = ns - 1;
-                for (int t = s + 1; t < ns; ++t)
-                    if (p->steps[t].pub.lhs == st.pub.out || p->steps[t].pub.rhs == st.pub.out) { consumer = t; break; }
-                items.push_back(Interval{mom::align_up((size_t)m * n * sizeof(float), mom::WS_ALIGN), s, consumer, &st.out_off, 0});
+        }
+        for (int s = 0; s < ns; ++s) {
+            mom::StepImpl &st = p->steps[s];
+            const int64_t m = st.pub.m, n = st.pub.n, k = st.pub.k;
+            int consumer = -1;
+            for (int t = s + 1; t < ns; ++t)
+                if (p->steps[t].pub.lhs == st.pub.out || p->steps[t].pub.rhs == st.pub.out) { consumer = t; break; }
+            // a tensor-core producer writes a tensor-core consumer's operand planes itself
+            const bool fused_planes = consumer >= 0 && st.pub.uses_tensor_cores && p->steps[consumer].pub.uses_tensor_cores;
+            if (fused_planes) {
+                mom::StepImpl &c = p->steps[consumer];
+                if (c.pub.lhs == st.pub.out) { st.planes_out = 1; c.a_planes_ready = true; }
+                else { st.planes_out = 2; c.b_planes_ready = true; }
+            } else if (!st.is_last) {
+                items.push_back(Interval{mom::align_up((size_t)m * n * sizeof(float), mom::WS_ALIGN), s, consumer < 0 ? ns - 1 : consumer, &st.out_off, 0});
             }
             if (st.pub.uses_tensor_cores) {
                 const size_t ab = mom::align_up((size_t)m * k * sizeof(float), mom::WS_ALIGN);
                 const size_t bb = mom::align_up((size_t)k * n * sizeof(float), mom::WS_ALIGN);
-                items.push_back(Interval{ab, s, s, &st.a_hi_off, 0});
-                items.push_back(Interval{ab, s, s, &st.a_lo_off, 0});
-                items.push_back(Interval{bb, s, s, &st.b_hi_off, 0});
-                items.push_back(Interval{bb, s, s, &st.b_lo_off, 0});
+                // planes written by an earlier step live from that step on
+                int a_from = s, b_from = s;
+                for (int t = 0; t < s; ++t) {
+                    if (p->steps[t].pub.out == st.pub.lhs && st.a_planes_ready) a_from = t;
+                    if (p->steps[t].pub.out == st.pub.rhs && st.b_planes_ready) b_from = t;
+                }
+                items.push_back(Interval{ab, a_from, s, &st.a_hi_off, 0});
+                items.push_back(Interval{ab, a_from, s, &st.a_lo_off, 0});
+                items.push_back(Interval{bb, b_from, s, &st.b_hi_off, 0});
+                items.push_back(Interval{bb, b_from, s, &st.b_lo_off, 0});
             }
         }
         p->workspace_per_instance = pack(items);
+        for (int s = 0; s < ns; ++s) {                  // a producer's plane targets are its consumer's operand planes
+            mom::StepImpl &st = p->steps[s];
+            if (!st.planes_out) continue;
+            for (int t = s + 1; t < ns; ++t) {
+                const mom::StepImpl &c = p->steps[t];
+                if (st.planes_out == 1 && c.pub.lhs == st.pub.out) { st.planes_hi_off = c.a_hi_off; st.planes_lo_off = c.a_lo_off; }
+                if (st.planes_out == 2 && c.pub.rhs == st.pub.out) { st.planes_hi_off = c.b_hi_off; st.planes_lo_off = c.b_lo_off; }
+            }
+        }
 
         // Small equations run as one fused kernel with every operand and intermediate in shared memory.
         {

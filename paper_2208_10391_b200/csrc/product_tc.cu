@@ -88,6 +88,7 @@ struct TcParams {
     int num_tiles;
     int m, n;
     int pout;
+    int out_mode;            // 0: f32 result through map_c; 1: hi/lo planes (map_c, map_c2); 2: transposed hi/lo planes
     AddTerms add;
     int32_t *status;
 };
@@ -102,10 +103,88 @@ __device__ __forceinline__ uint64_t kmajor_desc_64(uint32_t tile) {
     return ptx::smem_desc(tile, 16, 512, ptx::SWIZZLE_64B);
 }
 
+// Epilogue of one 32-row x 32-column chunk held as one row per thread: Add terms, structure mask, then
+// one of three outputs, each staged in shared memory under the 128B swizzle and written by TMA (coalesced,
+// clipped at the matrix edge):
+//   out_mode 0  the f32 values (the equation's result, or an intermediate read by an FFMA step);
+//   out_mode 1  the hi and lo planes of the values, for a tensor-core step that takes them as left operand;
+//   out_mode 2  the same planes transposed, for a tensor-core step that takes them as right operand.
+// Writing the planes here saves the consumer's split pass and the f32 round trip through HBM.
+__device__ __forceinline__ uint32_t round_tf32_bits(float a) { return (__float_as_uint(a) + 0x1000u) & 0xFFFFE000u; }
+
+__device__ __forceinline__ void epilogue_chunk(const TcParams &prm, const CUtensorMap *map_c, const CUtensorMap *map_c2,
+                                               float (&v)[32], int r, int row0, int col0, int lane, uint32_t stage_buf,
+                                               uint32_t &store_it) {
+    const bool row_ok = r < prm.m;
+    for (int a = 0; a < prm.add.count; ++a) {                   // Add terms, left to right
+        const float *p = prm.add.ptr[a];
+        if (p) {
+            if (row_ok) {
+                const float4 *src = reinterpret_cast<const float4 *>(p + (long long)r * prm.n + col0);
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    if (col0 + 4 * j < prm.n) {
+                        const float4 x = __ldg(src + j);
+                        v[4 * j] += x.x; v[4 * j + 1] += x.y; v[4 * j + 2] += x.z; v[4 * j + 3] += x.w;
+                    }
+                }
+            }
+        } else {                                                 // Identity term
+#pragma unroll
+            for (int j = 0; j < 32; ++j) v[j] += (col0 + j == r) ? 1.0f : 0.0f;
+        }
+    }
+    if (prm.pout != MOM_GENERAL) {
+#pragma unroll
+        for (int j = 0; j < 32; ++j) v[j] = in_structure(prm.pout, r, col0 + j) ? v[j] : 0.0f;
+    }
+    const int passes = prm.out_mode == 0 ? 1 : 2;                // f32, or hi then lo
+#pragma unroll 1
+    for (int pass = 0; pass < passes; ++pass) {
+        const uint32_t buf = stage_buf + (store_it & 1) * EPI_BOX_BYTES;
+        if (lane == 0) ptx::tma_store_wait_read<1>();            // the store that last read this buffer is done
+        __syncwarp();
+        if (prm.out_mode != 2) {
+            // 32 rows of 128 bytes: 16-byte chunk j of row i stored at chunk j ^ (i & 7)
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                float w[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const float x = v[4 * j + e];
+                    const float hi = __uint_as_float(round_tf32_bits(x));
+                    w[e] = prm.out_mode == 0 ? x : pass == 0 ? hi : __uint_as_float(round_tf32_bits(x - hi));
+                }
+                const uint32_t dst = buf + lane * 128 + ((j ^ (lane & 7)) << 4);
+                asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "f"(w[0]), "f"(w[1]), "f"(w[2]), "f"(w[3]) : "memory");
+            }
+        } else {
+            // transposed box: row j of the box is output column col0 + j, position lane is output row row0 + lane
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+                const float x = v[j];
+                const float hi = __uint_as_float(round_tf32_bits(x));
+                const float w = pass == 0 ? hi : __uint_as_float(round_tf32_bits(x - hi));
+                const uint32_t dst = buf + j * 128 + ((((uint32_t)lane >> 2) ^ (j & 7)) << 4) + ((lane & 3) << 2);
+                asm volatile("st.shared.f32 [%0], %1;" ::"r"(dst), "f"(w) : "memory");
+            }
+        }
+        ptx::fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) {
+            const CUtensorMap *map = pass == 0 ? map_c : map_c2;
+            if (prm.out_mode != 2) ptx::tma_store_2d(map, col0, row0, buf);
+            else ptx::tma_store_2d(map, row0, col0, buf);
+            ptx::tma_store_commit();
+        }
+        ++store_it;
+    }
+}
+
 __global__ void __launch_bounds__(THREADS, 1)
 product_tc_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_constant__ CUtensorMap map_a_lo,
                   const __grid_constant__ CUtensorMap map_b_hi, const __grid_constant__ CUtensorMap map_b_lo,
-                  const __grid_constant__ CUtensorMap map_c, const TcParams prm) {
+                  const __grid_constant__ CUtensorMap map_c, const __grid_constant__ CUtensorMap map_c2, const TcParams prm) {
     extern __shared__ uint8_t smem_raw[];
     __shared__ int abort_word;
     const uint32_t base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -249,49 +328,7 @@ product_tc_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_con
 #pragma unroll
                     for (int j = 0; j < 32; ++j) v[j] = 0.0f;
                 }
-                if (rows_left > 0) {
-                    const bool row_ok = r < prm.m;
-                    // Add terms, left to right
-                    for (int a = 0; a < prm.add.count; ++a) {
-                        const float *p = prm.add.ptr[a];
-                        if (p) {
-                            if (row_ok) {
-                                const float4 *src = reinterpret_cast<const float4 *>(p + (long long)r * prm.n + col0);
-#pragma unroll
-                                for (int j = 0; j < 8; ++j) {
-                                    if (col0 + 4 * j < prm.n) {
-                                        const float4 x = __ldg(src + j);
-                                        v[4 * j] += x.x; v[4 * j + 1] += x.y; v[4 * j + 2] += x.z; v[4 * j + 3] += x.w;
-                                    }
-                                }
-                            }
-                        } else {                                   // Identity term
-#pragma unroll
-                            for (int j = 0; j < 32; ++j) v[j] += (col0 + j == r) ? 1.0f : 0.0f;
-                        }
-                    }
-                    if (prm.pout != MOM_GENERAL) {
-#pragma unroll
-                        for (int j = 0; j < 32; ++j) v[j] = in_structure(prm.pout, r, col0 + j) ? v[j] : 0.0f;
-                    }
-                    // staging buffer: 32 rows of 128 bytes, 16-byte chunk j of row i stored at chunk j ^ (i & 7)
-                    const uint32_t buf = stage_buf + (store_it & 1) * EPI_BOX_BYTES;
-                    if (lane == 0) ptx::tma_store_wait_read<1>();  // the store that last read this buffer is done
-                    __syncwarp();
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) {
-                        const uint32_t dst = buf + lane * 128 + ((j ^ (lane & 7)) << 4);
-                        asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "f"(v[4 * j]), "f"(v[4 * j + 1]),
-                                     "f"(v[4 * j + 2]), "f"(v[4 * j + 3]) : "memory");
-                    }
-                    ptx::fence_proxy_async_smem();
-                    __syncwarp();
-                    if (lane == 0) {
-                        ptx::tma_store_2d(&map_c, col0, tile.x + q * 32, buf);
-                        ptx::tma_store_commit();
-                    }
-                    ++store_it;
-                }
+                if (rows_left > 0) epilogue_chunk(prm, &map_c, &map_c2, v, r, tile.x + q * 32, col0, lane, stage_buf, store_it);
             }
             if (!zero_tile) {
                 ptx::tc_fence_before_sync();
@@ -331,7 +368,7 @@ static_assert(P_SMEM_BYTES <= 227 * 1024, "shared memory budget");
 __global__ void __launch_bounds__(THREADS, 1)
 product_tc_pair_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_constant__ CUtensorMap map_a_lo,
                        const __grid_constant__ CUtensorMap map_b_hi, const __grid_constant__ CUtensorMap map_b_lo,
-                       const __grid_constant__ CUtensorMap map_c, const TcParams prm) {
+                       const __grid_constant__ CUtensorMap map_c, const __grid_constant__ CUtensorMap map_c2, const TcParams prm) {
     extern __shared__ uint8_t smem_raw[];
     __shared__ int abort_word;
     const uint32_t base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -492,47 +529,7 @@ product_tc_pair_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __gri
 #pragma unroll
                     for (int j = 0; j < 32; ++j) v[j] = 0.0f;
                 }
-                if (rows_left > 0) {
-                    const bool row_ok = r < prm.m;
-                    for (int a = 0; a < prm.add.count; ++a) {
-                        const float *p = prm.add.ptr[a];
-                        if (p) {
-                            if (row_ok) {
-                                const float4 *src = reinterpret_cast<const float4 *>(p + (long long)r * prm.n + col0);
-#pragma unroll
-                                for (int j = 0; j < 8; ++j) {
-                                    if (col0 + 4 * j < prm.n) {
-                                        const float4 x = __ldg(src + j);
-                                        v[4 * j] += x.x; v[4 * j + 1] += x.y; v[4 * j + 2] += x.z; v[4 * j + 3] += x.w;
-                                    }
-                                }
-                            }
-                        } else {
-#pragma unroll
-                            for (int j = 0; j < 32; ++j) v[j] += (col0 + j == r) ? 1.0f : 0.0f;
-                        }
-                    }
-                    if (prm.pout != MOM_GENERAL) {
-#pragma unroll
-                        for (int j = 0; j < 32; ++j) v[j] = in_structure(prm.pout, r, col0 + j) ? v[j] : 0.0f;
-                    }
-                    const uint32_t buf = stage_buf + (store_it & 1) * EPI_BOX_BYTES;
-                    if (lane == 0) ptx::tma_store_wait_read<1>();
-                    __syncwarp();
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) {
-                        const uint32_t dst = buf + lane * 128 + ((j ^ (lane & 7)) << 4);
-                        asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "f"(v[4 * j]), "f"(v[4 * j + 1]),
-                                     "f"(v[4 * j + 2]), "f"(v[4 * j + 3]) : "memory");
-                    }
-                    ptx::fence_proxy_async_smem();
-                    __syncwarp();
-                    if (lane == 0) {
-                        ptx::tma_store_2d(&map_c, col0, row0, buf);
-                        ptx::tma_store_commit();
-                    }
-                    ++store_it;
-                }
+                if (rows_left > 0) epilogue_chunk(prm, &map_c, &map_c2, v, r, row0, col0, lane, stage_buf, store_it);
             }
             if (!zero_tile) {
                 ptx::tc_fence_before_sync();
@@ -733,19 +730,36 @@ mom_status_t tc_launch_step(const mom_plan &p, TcPlanState &s, int step, const P
     float *a_hi = reinterpret_cast<float *>(workspace + st.a_hi_off), *a_lo = reinterpret_cast<float *>(workspace + st.a_lo_off);
     float *b_hi = reinterpret_cast<float *>(workspace + st.b_hi_off), *b_lo = reinterpret_cast<float *>(workspace + st.b_lo_off);
 
+    // operand planes: written by the producing step's epilogue, or split here from the f32 operand
     auto blocks = [](int x) { return (x + SPLIT_PIECE - 1) / SPLIT_PIECE; };
-    split_planes_kernel<false><<<dim3(blocks(a.k), blocks(a.m)), 256, 0, stream>>>(a.A, a_hi, a_lo, a.m, a.k, a.pa);
-    split_planes_kernel<true><<<dim3(blocks(a.n), blocks(a.k)), 256, 0, stream>>>(a.B, b_hi, b_lo, a.k, a.n, a.pb);
+    int split_launches = 0;
+    if (!st.a_planes_ready) {
+        split_planes_kernel<false><<<dim3(blocks(a.k), blocks(a.m)), 256, 0, stream>>>(a.A, a_hi, a_lo, a.m, a.k, a.pa);
+        ++split_launches;
+    }
+    if (!st.b_planes_ready) {
+        split_planes_kernel<true><<<dim3(blocks(a.n), blocks(a.k)), 256, 0, stream>>>(a.B, b_hi, b_lo, a.k, a.n, a.pb);
+        ++split_launches;
+    }
     if (cudaGetLastError() != cudaSuccess) return MOM_ERR_CUDA;
     if (before_product) cudaEventRecord(before_product, stream);
 
-    // A planes are m x k, B planes are n x k (transposed): both K-major with 16-element (64-byte) box rows
-    CUtensorMap ma_hi, ma_lo, mb_hi, mb_lo, mc;
+    // A planes are m x k, B planes are n x k (transposed): both K-major with 32-element (128-byte) box rows.
+    // Output: the f32 matrix, or the consumer's planes (m x n as stored, or n x m transposed).
+    CUtensorMap ma_hi, ma_lo, mb_hi, mb_lo, mc, mc2;
     bool ok = make_map(&ma_hi, a_hi, a.m, a.k, BM, BK, OPERAND_TMA_SWIZZLE) &&
               make_map(&ma_lo, a_lo, a.m, a.k, BM, BK, OPERAND_TMA_SWIZZLE) &&
               make_map(&mb_hi, b_hi, a.n, a.k, s.steps[step].pair ? BN / 2 : BN, BK, OPERAND_TMA_SWIZZLE) &&
-              make_map(&mb_lo, b_lo, a.n, a.k, s.steps[step].pair ? BN / 2 : BN, BK, OPERAND_TMA_SWIZZLE) &&
-              make_map(&mc, a.C, a.m, a.n, 32, 32, CU_TENSOR_MAP_SWIZZLE_128B);
+              make_map(&mb_lo, b_lo, a.n, a.k, s.steps[step].pair ? BN / 2 : BN, BK, OPERAND_TMA_SWIZZLE);
+    if (st.planes_out == 0) {
+        ok = ok && make_map(&mc, a.C, a.m, a.n, 32, 32, CU_TENSOR_MAP_SWIZZLE_128B);
+        mc2 = mc;
+    } else {
+        float *p_hi = reinterpret_cast<float *>(workspace + st.planes_hi_off), *p_lo = reinterpret_cast<float *>(workspace + st.planes_lo_off);
+        const int rows = st.planes_out == 1 ? a.m : a.n, cols = st.planes_out == 1 ? a.n : a.m;
+        ok = ok && make_map(&mc, p_hi, rows, cols, 32, 32, CU_TENSOR_MAP_SWIZZLE_128B) &&
+             make_map(&mc2, p_lo, rows, cols, 32, 32, CU_TENSOR_MAP_SWIZZLE_128B);
+    }
     if (!ok) return MOM_ERR_CUDA;
 
     TcParams prm;
@@ -754,6 +768,7 @@ mom_status_t tc_launch_step(const mom_plan &p, TcPlanState &s, int step, const P
     prm.m = a.m;
     prm.n = a.n;
     prm.pout = a.pout;
+    prm.out_mode = st.planes_out;
     prm.add = a.add;
     prm.status = status;
     if (s.steps[step].pair) {
@@ -785,13 +800,13 @@ mom_status_t tc_launch_step(const mom_plan &p, TcPlanState &s, int step, const P
             max_pairs = n;
         }
         cfg.gridDim = dim3(2 * std::min(prm.num_tiles, max_pairs));
-        if (cudaLaunchKernelEx(&cfg, product_tc_pair_kernel, ma_hi, ma_lo, mb_hi, mb_lo, mc, prm) != cudaSuccess) return MOM_ERR_CUDA;
+        if (cudaLaunchKernelEx(&cfg, product_tc_pair_kernel, ma_hi, ma_lo, mb_hi, mb_lo, mc, mc2, prm) != cudaSuccess) return MOM_ERR_CUDA;
     } else {
         const int grid = std::min(prm.num_tiles, g_sm_count);
-        product_tc_kernel<<<grid, THREADS, SMEM_BYTES, stream>>>(ma_hi, ma_lo, mb_hi, mb_lo, mc, prm);
+        product_tc_kernel<<<grid, THREADS, SMEM_BYTES, stream>>>(ma_hi, ma_lo, mb_hi, mb_lo, mc, mc2, prm);
     }
     if (cudaGetLastError() != cudaSuccess) return MOM_ERR_CUDA;
-    *launches = 3;
+    *launches = 1 + split_launches;
     return MOM_OK;
 }
 
@@ -983,8 +998,9 @@ extern "C" mom_status_t mom_product_3xtf32_noalloc(int64_t m64, int64_t n64, int
     prm.m = m;
     prm.n = n;
     prm.pout = pa == MOM_GENERAL || pb == MOM_GENERAL || pa != pb ? (int)MOM_GENERAL : (int)pa;
+    prm.out_mode = 0;
     prm.add.count = 0;
     prm.status = status;
-    product_tc_kernel<<<std::min(prm.num_tiles, g_sm_count), THREADS, SMEM_BYTES, stream>>>(ma_hi, ma_lo, mb_hi, mb_lo, mc, prm);
+    product_tc_kernel<<<std::min(prm.num_tiles, g_sm_count), THREADS, SMEM_BYTES, stream>>>(ma_hi, ma_lo, mb_hi, mb_lo, mc, mc, prm);
     return cudaGetLastError() == cudaSuccess ? MOM_OK : MOM_ERR_CUDA;
 }
