@@ -39,6 +39,10 @@ struct StepImpl {
     int planes_out = 0;             // 0: f32 output; 1: planes as stored (consumer's left operand); 2: transposed planes
     size_t planes_hi_off = SIZE_MAX, planes_lo_off = SIZE_MAX;
     bool a_planes_ready = false, b_planes_ready = false;   // this step's operand planes come from the producing step
+    // Split-K: products with few output tiles and a long contraction run `split_k` k-slices per tile on
+    // different CTAs; the slices' partial sums go to scratch and a small kernel adds them up.
+    int split_k = 1;
+    size_t partial_off = SIZE_MAX;
 };
 
 struct DeviceState;   // launcher-owned, created on first execute (execute.cu)

@@ -220,7 +220,7 @@ mom_status_t mom_equation_plan(const mom_matrix_desc_t *chain, int32_t n_chain,
         // kernel choice and workspace layout
         const int ns = (int)p->steps.size();
         std::vector<Interval> items;
-        items.reserve((size_t)ns * 5);
+        items.reserve((size_t)ns * 6);
         for (int s = 0; s < ns; ++s) {
             mom::StepImpl &st = p->steps[s];
             st.is_last = (s == ns - 1);
@@ -229,6 +229,14 @@ mom_status_t mom_equation_plan(const mom_matrix_desc_t *chain, int32_t n_chain,
             const bool worth_it = (double)m * (double)n * (double)k >= (double)(1 << 23);
             st.pub.uses_tensor_cores =
                 (variant == MOM_VARIANT_3XTF32 && addressable && worth_it) || ((int)variant == 2 && addressable);
+            if (st.pub.uses_tensor_cores) {
+                // few output tiles, long contraction: split k over otherwise idle SMs
+                const int64_t tiles = ((m + mom::TC_BM - 1) / mom::TC_BM) * ((n + mom::TC_BN - 1) / mom::TC_BN);
+                if (tiles <= 37 && k >= 512) {
+                    int64_t split = std::min<int64_t>(std::min<int64_t>(148 / tiles, k / 128), 32);
+                    if (split >= 2) st.split_k = (int)split;
+                }
+            }
         }
         for (int s = 0; s < ns; ++s) {
             mom::StepImpl &st = p->steps[s];
@@ -237,7 +245,8 @@ mom_status_t mom_equation_plan(const mom_matrix_desc_t *chain, int32_t n_chain,
             for (int t = s + 1; t < ns; ++t)
                 if (p->steps[t].pub.lhs == st.pub.out || p->steps[t].pub.rhs == st.pub.out) { consumer = t; break; }
             // a tensor-core producer writes a tensor-core consumer's operand planes itself
-            const bool fused_planes = consumer >= 0 && st.pub.uses_tensor_cores && p->steps[consumer].pub.uses_tensor_cores;
+            const bool fused_planes = consumer >= 0 && st.pub.uses_tensor_cores && p->steps[consumer].pub.uses_tensor_cores &&
+                                      st.split_k == 1;
             if (fused_planes) {
                 mom::StepImpl &c = p->steps[consumer];
                 if (c.pub.lhs == st.pub.out) { st.planes_out = 1; c.a_planes_ready = true; }
@@ -258,6 +267,10 @@ mom_status_t mom_equation_plan(const mom_matrix_desc_t *chain, int32_t n_chain,
                 items.push_back(Interval{ab, a_from, s, &st.a_lo_off, 0});
                 items.push_back(Interval{bb, b_from, s, &st.b_hi_off, 0});
                 items.push_back(Interval{bb, b_from, s, &st.b_lo_off, 0});
+                if (st.split_k > 1) {
+                    const size_t slab_rows = (size_t)((m + mom::TC_BM - 1) / mom::TC_BM * mom::TC_BM);
+                    items.push_back(Interval{mom::align_up((size_t)st.split_k * slab_rows * n * sizeof(float), mom::WS_ALIGN), s, s, &st.partial_off, 0});
+                }
             }
         }
         p->workspace_per_instance = pack(items);

@@ -83,12 +83,17 @@ __device__ __forceinline__ bool wait_barrier(uint32_t bar, uint32_t parity, vola
     return false;
 }
 
+// tile table entry: x = first row | k-slice << 24, y = first column, z..w = k-range
+constexpr int TILE_SLICE_SHIFT = 24;
+constexpr int TILE_ROW_MASK = (1 << TILE_SLICE_SHIFT) - 1;
+
 struct TcParams {
     const int4 *tiles;
     int num_tiles;
     int m, n;
     int pout;
     int out_mode;            // 0: f32 result through map_c; 1: hi/lo planes (map_c, map_c2); 2: transposed hi/lo planes
+    int slice_rows;          // split-K: rows between the partial-sum slabs of consecutive k-slices (0: no split)
     AddTerms add;
     int32_t *status;
 };
@@ -242,8 +247,9 @@ product_tc_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_con
                 if (!ok) break;
                 if (lane == 0) ptx::mbar_arrive_expect_tx(sh.full[s], STAGE_BYTES);
                 __syncwarp();
-                if (lane == 0) ptx::tma_load_2d(sh.stage[s], &map_a_hi, kb, tile.x, sh.full[s]);
-                else if (lane == 1) ptx::tma_load_2d(sh.stage[s] + A_PLANE_BYTES, &map_a_lo, kb, tile.x, sh.full[s]);
+                const int a_row = tile.x & TILE_ROW_MASK;            // (the k-slice index rides in the top bits)
+                if (lane == 0) ptx::tma_load_2d(sh.stage[s], &map_a_hi, kb, a_row, sh.full[s]);
+                else if (lane == 1) ptx::tma_load_2d(sh.stage[s] + A_PLANE_BYTES, &map_a_lo, kb, a_row, sh.full[s]);
                 else if (lane == 2) ptx::tma_load_2d(sh.stage[s] + 2 * A_PLANE_BYTES, &map_b_hi, kb, tile.y, sh.full[s]);
                 else if (lane == 3) ptx::tma_load_2d(sh.stage[s] + 2 * A_PLANE_BYTES + B_PLANE_BYTES, &map_b_lo, kb, tile.y, sh.full[s]);
             }
@@ -315,8 +321,11 @@ product_tc_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_con
                 if (!ok) break;
                 ptx::tc_fence_after_sync();
             }
-            const int r = tile.x + q * 32 + lane;                 // this thread's output row
-            const int rows_left = prm.m - (tile.x + q * 32);      // rows of this warp's slab inside the matrix
+            const int slab_row = (tile.x & TILE_ROW_MASK) + q * 32;   // first row of this warp's slab
+            const int r = slab_row + lane;                        // this thread's output row
+            const int rows_left = prm.m - slab_row;               // rows of the slab inside the matrix
+            // split-K: slice i of a tile stores its partial sums into slab i of the scratch matrix
+            const int store_row = slab_row + (int)((unsigned)tile.x >> TILE_SLICE_SHIFT) * prm.slice_rows;
 #pragma unroll 1
             for (int c = 0; c < BN / 32; ++c) {
                 const int col0 = tile.y + c * 32;
@@ -328,7 +337,7 @@ product_tc_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_con
 #pragma unroll
                     for (int j = 0; j < 32; ++j) v[j] = 0.0f;
                 }
-                if (rows_left > 0) epilogue_chunk(prm, &map_c, &map_c2, v, r, tile.x + q * 32, col0, lane, stage_buf, store_it);
+                if (rows_left > 0) epilogue_chunk(prm, &map_c, &map_c2, v, r, store_row, col0, lane, stage_buf, store_it);
             }
             if (!zero_tile) {
                 ptx::tc_fence_before_sync();
@@ -602,6 +611,29 @@ split_planes_kernel(const float *__restrict__ src, float *__restrict__ hi, float
     }
 }
 
+// Split-K: sum the k-slices' partial results, then the usual finish (Add terms, structure mask).
+// partial is (slices x slice_rows) x n; n is a multiple of 4.
+__global__ void __launch_bounds__(256)
+splitk_reduce_kernel(const float *__restrict__ partial, int slices, int slice_rows, float *__restrict__ C, int m, int n,
+                     int pout, AddTerms add) {
+    const int vec_per_row = n >> 2;
+    const long long total = (long long)m * vec_per_row;
+    for (long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (long long)gridDim.x * blockDim.x) {
+        const int r = (int)(e / vec_per_row), c = (int)(e % vec_per_row) << 2;
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int s = 0; s < slices; ++s) {
+            const float4 v = __ldg(reinterpret_cast<const float4 *>(partial + ((size_t)s * slice_rows + r) * n + c));
+            acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+        }
+        float4 o;
+        o.x = finish_entry(acc.x, add, 0, r, c, n, pout);
+        o.y = finish_entry(acc.y, add, 0, r, c + 1, n, pout);
+        o.z = finish_entry(acc.z, add, 0, r, c + 2, n, pout);
+        o.w = finish_entry(acc.w, add, 0, r, c + 3, n, pout);
+        *reinterpret_cast<float4 *>(C + (size_t)r * n + c) = o;
+    }
+}
+
 // ---------------------------------------------------------------------------------------------
 // host side
 // ---------------------------------------------------------------------------------------------
@@ -654,6 +686,8 @@ mom_status_t tc_prepare(const mom_plan &p, TcPlanState &s) {
         // CTA pairs (256-row tiles) once there are enough of them to occupy most of the GPU's 74 pairs
         const long long pair_tiles = (long long)((m + P_BM - 1) / P_BM) * ((n + BN - 1) / BN);
         s.steps[i].pair = m >= P_BM && pair_tiles >= 48;
+        const int split = p.steps[i].split_k;
+        if (split > 1) s.steps[i].pair = false;
         const int tile_rows = s.steps[i].pair ? P_BM : BM;
         for (int r0 = 0; r0 < m; r0 += tile_rows)
             for (int c0 = 0; c0 < n; c0 += BN) {
@@ -661,7 +695,17 @@ mom_status_t tc_prepare(const mom_plan &p, TcPlanState &s) {
                 tile_k_range(st.lhs_property, st.rhs_property, r0, std::min(r0 + tile_rows, m), c0, std::min(c0 + BN, n), k, &klo, &khi);
                 if (klo >= khi) { klo = 0; khi = 0; }
                 klo = klo / BK * BK;                      // leading extra elements are stored zeros
-                tab.push_back(make_int4(r0, c0, klo, khi));
+                if (split <= 1) {
+                    tab.push_back(make_int4(r0, c0, klo, khi));
+                } else {
+                    // every slice of every tile gets an entry (an empty one only zero-fills its slab), so the
+                    // reduction may read all slabs
+                    const int len = ((khi - klo + split - 1) / split + BK - 1) / BK * BK;
+                    for (int i2 = 0; i2 < split; ++i2) {
+                        const int lo = std::min(klo + i2 * len, khi), hi = std::min(lo + len, khi);
+                        tab.push_back(make_int4(r0 | (i2 << TILE_SLICE_SHIFT), c0, lo < hi ? lo : 0, lo < hi ? hi : 0));
+                    }
+                }
             }
         // Order.  Unequal tiles (triangular operands): heaviest first, so that the persistent CTAs, which
         // take tiles round-robin, finish together; structurally zero tiles last.  Equal tiles (general
@@ -675,7 +719,7 @@ mom_status_t tc_prepare(const mom_plan &p, TcPlanState &s) {
         } else {
             constexpr int SUPER_ROWS = 16, SUPER_COLS = 8;
             const int super_cols = ((n + BN - 1) / BN + SUPER_COLS - 1) / SUPER_COLS;
-            auto super_of = [&](const int4 &t) { return (t.x / BM / SUPER_ROWS) * super_cols + (t.y / BN / SUPER_COLS); };
+            auto super_of = [&](const int4 &t) { return ((t.x & TILE_ROW_MASK) / BM / SUPER_ROWS) * super_cols + (t.y / BN / SUPER_COLS); };
             std::vector<long long> super_work((size_t)(((m + BM - 1) / BM + SUPER_ROWS - 1) / SUPER_ROWS + 1) * super_cols, 0);
             for (const int4 &t : tab) super_work[super_of(t)] += t.w - t.z;
             std::stable_sort(tab.begin(), tab.end(), [&](const int4 &a, const int4 &b) {
@@ -751,7 +795,12 @@ mom_status_t tc_launch_step(const mom_plan &p, TcPlanState &s, int step, const P
               make_map(&ma_lo, a_lo, a.m, a.k, BM, BK, OPERAND_TMA_SWIZZLE) &&
               make_map(&mb_hi, b_hi, a.n, a.k, s.steps[step].pair ? BN / 2 : BN, BK, OPERAND_TMA_SWIZZLE) &&
               make_map(&mb_lo, b_lo, a.n, a.k, s.steps[step].pair ? BN / 2 : BN, BK, OPERAND_TMA_SWIZZLE);
-    if (st.planes_out == 0) {
+    const int slice_rows = st.split_k > 1 ? (a.m + BM - 1) / BM * BM : 0;
+    float *partial = st.split_k > 1 ? reinterpret_cast<float *>(workspace + st.partial_off) : nullptr;
+    if (st.split_k > 1) {
+        ok = ok && make_map(&mc, partial, st.split_k * slice_rows, a.n, 32, 32, CU_TENSOR_MAP_SWIZZLE_128B);
+        mc2 = mc;
+    } else if (st.planes_out == 0) {
         ok = ok && make_map(&mc, a.C, a.m, a.n, 32, 32, CU_TENSOR_MAP_SWIZZLE_128B);
         mc2 = mc;
     } else {
@@ -767,9 +816,11 @@ mom_status_t tc_launch_step(const mom_plan &p, TcPlanState &s, int step, const P
     prm.num_tiles = s.steps[step].num_tiles;
     prm.m = a.m;
     prm.n = a.n;
-    prm.pout = a.pout;
+    prm.pout = st.split_k > 1 ? (int)MOM_GENERAL : a.pout;      // split-K: mask and Add terms are applied by the reduction
     prm.out_mode = st.planes_out;
+    prm.slice_rows = slice_rows;
     prm.add = a.add;
+    if (st.split_k > 1) prm.add.count = 0;
     prm.status = status;
     if (s.steps[step].pair) {
         static bool pair_attr_set = false;
@@ -807,6 +858,13 @@ mom_status_t tc_launch_step(const mom_plan &p, TcPlanState &s, int step, const P
     }
     if (cudaGetLastError() != cudaSuccess) return MOM_ERR_CUDA;
     *launches = 1 + split_launches;
+    if (st.split_k > 1) {
+        const long long vecs = (long long)a.m * (a.n / 4);
+        const int blocks_r = (int)std::min<long long>((vecs + 255) / 256, (long long)g_sm_count * 8);
+        splitk_reduce_kernel<<<blocks_r, 256, 0, stream>>>(partial, st.split_k, slice_rows, a.C, a.m, a.n, a.pout, a.add);
+        if (cudaGetLastError() != cudaSuccess) return MOM_ERR_CUDA;
+        ++*launches;
+    }
     return MOM_OK;
 }
 
@@ -999,6 +1057,7 @@ extern "C" mom_status_t mom_product_3xtf32_noalloc(int64_t m64, int64_t n64, int
     prm.n = n;
     prm.pout = pa == MOM_GENERAL || pb == MOM_GENERAL || pa != pb ? (int)MOM_GENERAL : (int)pa;
     prm.out_mode = 0;
+    prm.slice_rows = 0;
     prm.add.count = 0;
     prm.status = status;
     product_tc_kernel<<<std::min(prm.num_tiles, g_sm_count), THREADS, SMEM_BYTES, stream>>>(ma_hi, ma_lo, mb_hi, mb_lo, mc, mc, prm);

@@ -50,6 +50,24 @@ def test_triangular_times_rectangular(pt, side, variant):
     both(eq, variant)
 
 
+@pytest.mark.parametrize("pa,pb", [(G, G), (L, G), (U, G), (G, L), (G, U), (L, L), (U, L)])
+def test_split_k_products(pa, pb):
+    # few output tiles and a long contraction: the tensor-core kernel runs k-slices on different CTAs and a
+    # small kernel adds the partial sums (and applies the Add terms and the structure mask)
+    n = 640
+    shapes = {(G, G): ((256, 2048), (2048, 64)), (L, G): ((n, n), (n, 136)), (U, G): ((n, n), (n, 136)),
+              (G, L): ((72, n), (n, n)), (G, U): ((72, n), (n, n)), (L, L): ((n, n), (n, n)), (U, L): ((n, n), (n, n))}
+    (am, ak), (bk, bn) = shapes[(pa, pb)]
+    add = (Operand(am, bn, G, "normal"), Operand(am, bn, I)) if am == bn else (Operand(am, bn, G, "normal"),)
+    eq = Equation(f"splitk_{pa}{pb}", 60, (Operand(am, ak, pa, "normal" if pa == G else "uniform"),
+                                           Operand(bk, bn, pb, "normal" if pb == G else "uniform")), add)
+    both(eq, mom.VARIANT_3XTF32_FORCE)
+    # the same product as the inner step of a chain whose next step is a tensor-core step too
+    eq = Equation(f"splitk_chain_{pa}{pb}", 61, (Operand(200, am, G, "normal"), Operand(am, ak, pa, "normal" if pa == G else "uniform"),
+                                                 Operand(bk, bn, pb, "normal" if pb == G else "uniform")))
+    both(eq, mom.VARIANT_3XTF32_FORCE)
+
+
 @pytest.mark.parametrize("variant", VARIANTS, ids=VNAME.get)
 def test_listing2_exact_values(variant):
     # paper Listing 2: 5x5 lowerTri filled with ones times itself; every value is a small integer
