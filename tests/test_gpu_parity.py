@@ -110,6 +110,23 @@ def test_config_large_square_small(n, variant):
     both(wl.config_large_square(n=n), variant)
 
 
+@pytest.mark.parametrize("case", ["LG", "GU_plus_C", "chain"])
+def test_pair_kernel_ragged_shapes(case):
+    # big enough for the CTA-pair tensor-core kernel (256-row tiles), with edges that are not multiples of the tile
+    m, k, n = 3336, 3064, 3592
+    if case == "LG":
+        eq = Equation("pair_LG", 70, (Operand(m, m, L), Operand(m, n, G, "normal", 0.02)))
+    elif case == "GU_plus_C":
+        eq = Equation("pair_GU", 71, (Operand(m, n, G, "normal", 0.02), Operand(n, n, U)), (Operand(m, n, G, "normal"),))
+    else:
+        eq = Equation("pair_chain", 72, (Operand(m, m, U), Operand(m, k, G, "normal", 0.02), Operand(k, k, L), Operand(k, n, G, "normal", 0.02)))
+    x, plan, (chain, add) = run_equation(eq, mom.VARIANT_3XTF32)
+    assert all(s.uses_tensor_cores for s in plan.steps())
+    rows = np.sort(np.random.default_rng(3).choice(m, size=40, replace=False))
+    rows[:6] = [0, 127, 128, 255, 256, m - 1]
+    check_against_oracle(eq, x, plan, chain, add, rows=np.sort(rows))
+
+
 @pytest.mark.parametrize("variant", [mom.VARIANT_3XTF32, mom.VARIANT_FFMA], ids=VNAME.get)
 def test_config_property_heavy_full_size_sampled_rows(variant):
     eq = wl.config_property_heavy()
