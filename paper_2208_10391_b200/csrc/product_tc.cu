@@ -714,8 +714,35 @@ mom_status_t tc_prepare(const mom_plan &p, TcPlanState &s) {
         // of A and B panels).  (Super-tiles for unequal tiles cost more in imbalance than they saved.)
         bool uniform = true;
         for (const int4 &t : tab) uniform &= (t.w - t.z) == (tab[0].w - tab[0].z);
+        int sms = 0;
+        {
+            int dev = 0;
+            cudaGetDevice(&dev);
+            cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        }
+        const int units = std::max(1, std::min((int)tab.size(), s.steps[i].pair ? sms / 2 : sms));   // CTAs, or CTA pairs
+        s.steps[i].units = units;
         if (!uniform) {
+            // Longest-processing-time list scheduling on the host: tiles by decreasing cost, each to the unit
+            // with the least work so far.  Unit u then owns table entries u, u + units, u + 2*units, ...; rounds
+            // a unit has no tile for hold a dummy entry that lies outside the matrix (nothing loaded or stored).
             std::stable_sort(tab.begin(), tab.end(), [](const int4 &a, const int4 &b) { return (a.w - a.z) > (b.w - b.z); });
+            constexpr long long TILE_OVERHEAD = 3 * BK;         // epilogue and pipeline fill, in k units
+            std::vector<std::vector<int4>> mine(units);
+            std::vector<long long> load(units, 0);
+            for (const int4 &t : tab) {
+                int best = 0;
+                for (int u = 1; u < units; ++u)
+                    if (load[u] < load[best]) best = u;
+                mine[best].push_back(t);
+                load[best] += (t.w - t.z) + TILE_OVERHEAD;
+            }
+            size_t rounds = 0;
+            for (const auto &v : mine) rounds = std::max(rounds, v.size());
+            const int4 dummy = make_int4(TILE_ROW_MASK & ~(P_BM - 1), n + BN, 0, 0);
+            tab.assign(rounds * units, dummy);
+            for (int u = 0; u < units; ++u)
+                for (size_t r = 0; r < mine[u].size(); ++r) tab[r * units + u] = mine[u][r];
         } else {
             constexpr int SUPER_ROWS = 16, SUPER_COLS = 8;
             const int super_cols = ((n + BN - 1) / BN + SUPER_COLS - 1) / SUPER_COLS;
@@ -850,10 +877,11 @@ mom_status_t tc_launch_step(const mom_plan &p, TcPlanState &s, int step, const P
             if (cudaOccupancyMaxActiveClusters(&n, product_tc_pair_kernel, &cfg) != cudaSuccess || n < 1) return MOM_ERR_CUDA;
             max_pairs = n;
         }
-        cfg.gridDim = dim3(2 * std::min(prm.num_tiles, max_pairs));
+        if (max_pairs < s.steps[step].units) return MOM_ERR_CUDA;   // the table was laid out for co-resident pairs
+        cfg.gridDim = dim3(2 * s.steps[step].units);
         if (cudaLaunchKernelEx(&cfg, product_tc_pair_kernel, ma_hi, ma_lo, mb_hi, mb_lo, mc, mc2, prm) != cudaSuccess) return MOM_ERR_CUDA;
     } else {
-        const int grid = std::min(prm.num_tiles, g_sm_count);
+        const int grid = std::min(s.steps[step].units, g_sm_count);
         product_tc_kernel<<<grid, THREADS, SMEM_BYTES, stream>>>(ma_hi, ma_lo, mb_hi, mb_lo, mc, mc2, prm);
     }
     if (cudaGetLastError() != cudaSuccess) return MOM_ERR_CUDA;
