@@ -21,6 +21,8 @@ Readings taken where the paper is silent (each also listed in the design notes):
   * Identity operands are removed before the enumeration and never appear in the result string;
   * ties: the tree whose pre-order list of split positions is lexicographically smallest;
   * property of a product = join in  Identity < {lowerTri, upperTri} < general;
+  * a transposed operand (paper Table 1, "Transpose") takes part with its transposed type: shape
+    swapped and lowerTri <-> upperTri (the inference rule the paper prints);
   * reported mul_flops = 2 * multiplications; add_flops = structural non-zeros of the Add terms.
     (The factor 2 and the add_flops convention are bookkeeping of this project: parity unpinned by
     the paper, which only speaks of scalar multiplications.)
@@ -225,17 +227,38 @@ def _preorder_splits(tree) -> List[int]:
     return [split] + _preorder_splits(left) + _preorder_splits(right)
 
 
-def _paren(tree, kept: Sequence[int]) -> str:
+def _paren(tree, kept: Sequence[int], transposed: Sequence[bool] = ()) -> str:
     if isinstance(tree, int):
-        return str(kept[tree])
+        i = kept[tree]
+        return str(i) + ("^T" if transposed and transposed[i] else "")
     _, left, right = tree
-    return "(" + _paren(left, kept) + "*" + _paren(right, kept) + ")"
+    return "(" + _paren(left, kept, transposed) + "*" + _paren(right, kept, transposed) + ")"
 
 
-def plan(chain: Sequence[Tuple[int, int, int]], add: Sequence[Tuple[int, int, int]] = ()) -> Plan:
-    """Plan `X = prod(chain) + sum(add)`; operands are (rows, cols, property) triples."""
-    cdescs = [Desc(*c) for c in chain]
-    adescs = [Desc(*a) for a in add]
+def transpose_desc(d: Desc) -> Desc:
+    """Type of A^T given the type of A: shape swapped; paper Section 2, "Transformations", prints the
+    inference rule lowerTriangular(A) -> upperTriangular(A^T) (and symmetrically); general and Identity
+    keep their property."""
+    prop = {LOWER_TRI: UPPER_TRI, UPPER_TRI: LOWER_TRI}.get(d.prop, d.prop)
+    return Desc(d.cols, d.rows, prop)
+
+
+def plan(chain: Sequence[Tuple[int, int, int]], add: Sequence[Tuple[int, int, int]] = (),
+         chain_transposed: Sequence[bool] = (), add_transposed: Sequence[bool] = ()) -> Plan:
+    """Plan `X = prod(chain) + sum(add)`; operands are (rows, cols, property) triples of the STORED matrices.
+
+    `chain_transposed[i]` / `add_transposed[i]` say that the equation uses the transpose of that operand
+    (paper Table 1, "Transpose"); the plan then works with the transposed type and prints the operand as `i^T`.
+    """
+    stored_c = [Desc(*c) for c in chain]
+    stored_a = [Desc(*a) for a in add]
+    for d in stored_c + stored_a:               # the stored matrices must be well-typed themselves
+        if d.prop not in (GENERAL, LOWER_TRI, UPPER_TRI, IDENTITY):
+            raise OracleError("property", "unknown property")
+    tc = list(chain_transposed) + [False] * (len(stored_c) - len(chain_transposed))
+    ta = list(add_transposed) + [False] * (len(stored_a) - len(add_transposed))
+    cdescs = [transpose_desc(d) if t else d for d, t in zip(stored_c, tc)]
+    adescs = [transpose_desc(d) if t else d for d, t in zip(stored_a, ta)]
     _validate(cdescs, adescs)
     n = len(cdescs)
     rows, cols = cdescs[0].rows, cdescs[-1].cols
@@ -276,7 +299,7 @@ def plan(chain: Sequence[Tuple[int, int, int]], add: Sequence[Tuple[int, int, in
     _, product = emit(tree)
     assert sum(s.mults for s in steps) == cost
     result = Desc(rows, cols, sum_property(product.prop, [t.prop for t in adescs]))
-    return Plan(_paren(tree, kept), cost, 2 * cost, add_flops, tuple(steps), product, result, kept)
+    return Plan(_paren(tree, kept, tc), cost, 2 * cost, add_flops, tuple(steps), product, result, kept)
 
 
 def catalan(r: int) -> int:

@@ -89,6 +89,25 @@ def dense(arr: Optional[np.ndarray], desc: Tuple[int, int, int]) -> np.ndarray:
     return a
 
 
+def transposed_operands(arrays, descs, flags):
+    """Operands as the equation uses them: entry i transposed (array and descriptor) where flags[i] is set.
+
+    The transpose of a stored lowerTri matrix is upperTri and vice versa (the paper's printed inference
+    rule); Identity and general keep their property.  Dense storage is simply transposed with NumPy.
+    """
+    swap = {LOWER_TRI: UPPER_TRI, UPPER_TRI: LOWER_TRI}
+    out_a, out_d = [], []
+    flags = list(flags) + [False] * (len(descs) - len(flags))
+    for a, (r, c, p), t in zip(arrays, descs, flags):
+        if t:
+            out_a.append(None if a is None else np.ascontiguousarray(np.asarray(a).T))
+            out_d.append((c, r, swap.get(p, p)))
+        else:
+            out_a.append(a)
+            out_d.append((r, c, p))
+    return out_a, out_d
+
+
 def evaluate(chain: Sequence[Optional[np.ndarray]], chain_descs: Sequence[Tuple[int, int, int]],
              add: Sequence[Optional[np.ndarray]] = (), add_descs: Sequence[Tuple[int, int, int]] = (),
              rows: Optional[np.ndarray] = None, threads: Optional[int] = None

@@ -268,3 +268,37 @@ def test_invalid_equations_are_rejected(chain, add, code):
     with pytest.raises(op.OracleError) as e:
         op.plan(chain, add)
     assert e.value.code == code
+
+
+# ---------------------------------------------------------------- Transpose (paper Table 1; Section 2 inference rule)
+def test_transposed_operands_take_the_transposed_type():
+    # the rule the paper prints: lowerTriangular(A) -> upperTriangular(A^T)
+    assert op.transpose_desc(Desc(5, 5, L)) == Desc(5, 5, U)
+    assert op.transpose_desc(Desc(5, 5, U)) == Desc(5, 5, L)
+    assert op.transpose_desc(Desc(3, 7, G)) == Desc(7, 3, G)
+    assert op.transpose_desc(Desc(4, 4, I)) == Desc(4, 4, I)
+    # L^T * L^T is upperTri; L^T * L is general; structure of S(A^T) is the mirrored structure
+    assert op.plan([(6, 6, L), (6, 6, L)], chain_transposed=[True, True]).result_desc == Desc(6, 6, U)
+    assert op.plan([(6, 6, L), (6, 6, L)], chain_transposed=[True, False]).result_desc == Desc(6, 6, G)
+    for prop in (G, L, U, I):
+        tp = op.transpose_desc(Desc(5, 5, prop)).prop
+        for i in range(5):
+            for j in range(5):
+                assert op.in_structure(tp, i, j) == op.in_structure(prop, j, i)
+
+
+def test_transposes_change_shapes_costs_and_the_string():
+    # A (7 x 30) stored, used as A^T (30 x 7): the chain A^T * B * C with B 7 x 40, C 40 x 3
+    p = op.plan([(7, 30, G), (7, 40, G), (40, 3, G)], chain_transposed=[True, False, False])
+    assert p.paren == "(0^T*(1*2))"
+    assert p.mults == 7 * 40 * 3 + 30 * 7 * 3
+    assert p.result_desc == Desc(30, 3, G)
+    # a plan with transposes equals the plan of the explicitly transposed descriptors (up to the printed marks)
+    q = op.plan([(30, 7, G), (7, 40, G), (40, 3, G)])
+    assert q.mults == p.mults and q.paren == p.paren.replace("^T", "")
+    with pytest.raises(op.OracleError):
+        op.plan([(7, 30, G), (7, 40, G)])                        # without the transpose the shapes do not chain
+    # Add terms may be transposed too
+    p = op.plan([(4, 9, G)], [(9, 4, G)], add_transposed=[True])
+    assert p.result_desc == Desc(4, 9, G) and p.add_flops == 36
+    assert op.plan([(5, 5, L)], [(5, 5, U)], add_transposed=[True]).result_desc.prop == L

@@ -163,3 +163,22 @@ def test_generated_inputs_follow_the_storage_contract():
     big = wl.config_large_square(n=64)
     (_, a64, _, _), _ = wl.generate(big)
     assert abs(float(a64.std()) - 64 ** -0.5) < 0.02
+
+
+def test_transposed_operands_follow_the_transpose_identities():
+    # (A*B)^T = B^T * A^T, checked through the oracle's own transposed-operand path against NumPy
+    rng = np.random.default_rng(5)
+    a = rng.standard_normal((6, 9)).astype(np.float32)
+    b = rng.standard_normal((9, 4)).astype(np.float32)
+    arrs, descs = ov.transposed_operands([b, a], [(9, 4, G), (6, 9, G)], [True, True])
+    assert descs == [(4, 9, G), (9, 6, G)]
+    x, _ = ov.evaluate(arrs, descs)
+    assert np.allclose(x, (a.astype(np.float64) @ b.astype(np.float64)).T, rtol=1e-14)
+    # the transpose of a stored lower-triangular matrix is upper triangular, entry for entry
+    eq = wl.Equation("t", 12, (wl.Operand(7, 7, L),))
+    (l,), _ = wl.generate(eq)
+    (lt,), (d,) = ov.transposed_operands([l], eq.descs(), [True])
+    assert d == (7, 7, U) and np.array_equal(lt, l.T) and ov.off_structure_exactly_zero(lt, U)
+    # untouched operands are passed through
+    arrs, descs = ov.transposed_operands([a, None], [(6, 9, G), (9, 9, I)], [False, True])
+    assert arrs[0] is a and arrs[1] is None and descs[1] == (9, 9, I)

@@ -53,6 +53,8 @@ class Equation:
     chain: Sequence[Operand]
     add: Sequence[Operand] = field(default_factory=tuple)
     batch: int = 1  # > 1: `batch` independent instances sharing one plan
+    chain_t: Sequence[bool] = ()   # operand i of the chain enters the equation transposed (stored as given)
+    add_t: Sequence[bool] = ()
 
     def descs(self):
         return [(o.rows, o.cols, o.prop) for o in self.chain]
