@@ -93,6 +93,7 @@ typedef struct {
     int32_t kind;                    /* mom_kind_t */
     int32_t lhs_property, rhs_property, out_property;
     int32_t uses_tensor_cores;       /* 1: tcgen05 3xTF32 kernel, 0: FFMA kernel */
+    int32_t lhs_transposed, rhs_transposed;   /* the operand is an original chain operand used transposed */
     int64_t m, n, k;                 /* out is m x n, contraction length k */
     uint64_t useful_mults;           /* scalar multiplications with both factors structurally non-zero */
 } mom_step_t;
@@ -118,6 +119,16 @@ mom_status_t mom_matrix_desc(int64_t rows, int64_t cols, mom_property_t property
 mom_status_t mom_equation_plan(const mom_matrix_desc_t *chain, int32_t n_chain,
                                const mom_matrix_desc_t *add_terms, int32_t n_add,
                                mom_variant_t variant, mom_plan_t **out_plan);
+
+/* The same with Transpose (paper Table 1, "Transpose"; Section 2 prints the inference rule
+ * lowerTriangular(A) -> upperTriangular(A^T)): chain_transposed[i] != 0 means the equation uses the transpose
+ * of chain operand i, add_transposed[i] likewise for the Add terms; either array may be NULL (nothing
+ * transposed).  The descriptors describe the matrices AS STORED; a transposed operand takes part with its
+ * shape swapped and lowerTri <-> upperTri.  Nothing is moved in memory: the kernels read a transposed operand
+ * through its stored layout.  In the parenthesization string a transposed operand prints as "i^T". */
+mom_status_t mom_equation_plan_transposed(const mom_matrix_desc_t *chain, const int32_t *chain_transposed, int32_t n_chain,
+                                          const mom_matrix_desc_t *add_terms, const int32_t *add_transposed, int32_t n_add,
+                                          mom_variant_t variant, mom_plan_t **out_plan);
 
 /* mul_flops = 2 * (useful multiplications of the chosen parenthesization); add_flops = structural
  * non-zeros of the Add terms (an Identity term counts its n diagonal entries).  Either may be NULL. */

@@ -33,6 +33,7 @@ class Step(ctypes.Structure):
     _fields_ = [("lhs", ctypes.c_int32), ("rhs", ctypes.c_int32), ("out", ctypes.c_int32),
                 ("kind", ctypes.c_int32), ("lhs_property", ctypes.c_int32), ("rhs_property", ctypes.c_int32),
                 ("out_property", ctypes.c_int32), ("uses_tensor_cores", ctypes.c_int32),
+                ("lhs_transposed", ctypes.c_int32), ("rhs_transposed", ctypes.c_int32),
                 ("m", ctypes.c_int64), ("n", ctypes.c_int64), ("k", ctypes.c_int64),
                 ("useful_mults", ctypes.c_uint64)]
 
@@ -55,6 +56,9 @@ _sigs = {
     "mom_matrix_desc": [ctypes.c_int64, ctypes.c_int64, ctypes.c_int, ctypes.c_int, ctypes.POINTER(MatrixDesc)],
     "mom_equation_plan": [ctypes.POINTER(MatrixDesc), ctypes.c_int32, ctypes.POINTER(MatrixDesc), ctypes.c_int32,
                           ctypes.c_int, ctypes.POINTER(_P)],
+    "mom_equation_plan_transposed": [ctypes.POINTER(MatrixDesc), ctypes.POINTER(ctypes.c_int32), ctypes.c_int32,
+                                     ctypes.POINTER(MatrixDesc), ctypes.POINTER(ctypes.c_int32), ctypes.c_int32,
+                                     ctypes.c_int, ctypes.POINTER(_P)],
     "mom_plan_flops": [_P, ctypes.POINTER(ctypes.c_uint64), ctypes.POINTER(ctypes.c_uint64)],
     "mom_plan_parenthesization": [_P, ctypes.c_char_p, ctypes.c_size_t, ctypes.POINTER(ctypes.c_size_t)],
     "mom_plan_num_steps": [_P, ctypes.POINTER(ctypes.c_int32)],
@@ -228,6 +232,24 @@ def mom_equation_plan(chain: Sequence, add_terms: Sequence = (), variant: int = 
     st = _lib.mom_equation_plan(_desc_array(chain) if n_chain else None, n_chain,
                                 _desc_array(add_terms) if n_add else None, n_add, variant, ctypes.byref(handle))
     _check(st, "mom_equation_plan")
+    return Plan(handle.value, n_chain, n_add)
+
+
+def mom_equation_plan_transposed(chain: Sequence, chain_transposed: Optional[Sequence], add_terms: Sequence = (),
+                                 add_transposed: Optional[Sequence] = None, variant: int = VARIANT_3XTF32) -> Plan:
+    """As mom_equation_plan, with per-operand Transpose flags; descriptors describe the matrices as stored."""
+    handle = _P()
+    n_chain, n_add = len(chain), len(add_terms)
+
+    def flags(f, n):
+        if f is None or n == 0:
+            return None
+        f = list(f) + [False] * (n - len(f))
+        return (ctypes.c_int32 * n)(*[1 if x else 0 for x in f])
+    st = _lib.mom_equation_plan_transposed(_desc_array(chain) if n_chain else None, flags(chain_transposed, n_chain), n_chain,
+                                           _desc_array(add_terms) if n_add else None, flags(add_transposed, n_add), n_add,
+                                           variant, ctypes.byref(handle))
+    _check(st, "mom_equation_plan_transposed")
     return Plan(handle.value, n_chain, n_add)
 
 

@@ -16,6 +16,8 @@ struct AddTerms {
     const float *ptr[MAX_FUSED_ADD];     // NULL for an Identity term
     long long stride[MAX_FUSED_ADD];     // elements between batch instances
     int count;
+    unsigned transposed;                 // bit t: term t is stored transposed (cols x rows of X)
+    int rows;                            // rows of X (leading dimension of a transposed term)
 };
 
 // With dense zero-filled storage every product is C[r,c] = sum over l in [klo, khi) of A[r,l]*B[l,c],
@@ -47,7 +49,8 @@ __device__ __forceinline__ float finish_entry(float acc, const AddTerms &add, lo
     for (int t = 0; t < MAX_FUSED_ADD; ++t) {
         if (t < add.count) {
             const float *p = add.ptr[t];
-            v += p ? __ldg(p + batch * add.stride[t] + (long long)r * ld + c) : (r == c ? 1.0f : 0.0f);
+            const long long at = (add.transposed >> t) & 1u ? (long long)c * add.rows + r : (long long)r * ld + c;
+            v += p ? __ldg(p + batch * add.stride[t] + at) : (r == c ? 1.0f : 0.0f);
         }
     }
     return in_structure(out_prop, r, c) ? v : 0.0f;

@@ -114,7 +114,8 @@ mom_status_t execute_impl(const mom_plan *p, const float *const *chain_ptrs, con
         for (int i = 0; i < fp.n_ops; ++i) {
             const int id = p->kept[i];
             fp.ops[i] = FusedOperand{chain_ptrs[id], chain_strides ? chain_strides[id] : 0, (int)p->chain[id].rows,
-                                     (int)p->chain[id].cols, p->chain[id].property, p->fused_value_off[id], p->fused_value_ld[id]};
+                                     (int)p->chain[id].cols, p->chain[id].property, p->fused_value_off[id], p->fused_value_ld[id],
+                                     (int)p->chain_t[id]};
         }
         fp.n_steps = (int)p->steps.size();
         for (int s = 0; s < fp.n_steps; ++s) {
@@ -127,9 +128,12 @@ mom_status_t execute_impl(const mom_plan *p, const float *const *chain_ptrs, con
                                     stp.is_last ? 0 : p->fused_value_ld[stp.pub.out]};
         }
         fp.add.count = n_add;
+        fp.add.transposed = 0;
+        fp.add.rows = (int)rows;
         for (int i = 0; i < n_add; ++i) {
             fp.add.ptr[i] = p->add[i].property == MOM_IDENTITY ? nullptr : add_ptrs[i];
             fp.add.stride[i] = add_strides ? add_strides[i] : 0;
+            if (p->add_t[i]) fp.add.transposed |= 1u << i;
         }
         fp.out = out;
         fp.out_stride = out_stride;
@@ -162,10 +166,13 @@ mom_status_t execute_impl(const mom_plan *p, const float *const *chain_ptrs, con
         };
         auto add_terms = [&](int first, AddTerms *t) {
             t->count = 0;
+            t->transposed = 0;
+            t->rows = (int)rows;
             for (int i = first; i < n_add && t->count < MAX_FUSED_ADD; ++i, ++t->count) {
                 const long long s = add_strides ? add_strides[i] : 0;
                 t->ptr[t->count] = p->add[i].property == MOM_IDENTITY ? nullptr : add_ptrs[i] + b0 * s;
                 t->stride[t->count] = s;
+                if (p->add_t[i]) t->transposed |= 1u << t->count;
             }
             return first + t->count;
         };
@@ -180,7 +187,7 @@ mom_status_t execute_impl(const mom_plan *p, const float *const *chain_ptrs, con
                 e = launch_elementwise(nullptr, 0, 1, x, out_stride, (int)rows, (int)cols, p->result_desc.property, t, nb, stream);
             } else {
                 const Operand src = chain_op(p->kept[0]);
-                e = launch_elementwise(src.ptr, src.stride, 0, x, out_stride, (int)rows, (int)cols, p->result_desc.property, t, nb, stream);
+                e = launch_elementwise(src.ptr, src.stride, p->chain_t[p->kept[0]] ? 3 : 0, x, out_stride, (int)rows, (int)cols, p->result_desc.property, t, nb, stream);
             }
             if (e != cudaSuccess) return MOM_ERR_CUDA;
             ++launches;
@@ -204,6 +211,7 @@ mom_status_t execute_impl(const mom_plan *p, const float *const *chain_ptrs, con
             a.strideA = A.stride; a.strideB = B.stride;
             a.m = (int)stp.pub.m; a.n = (int)stp.pub.n; a.k = (int)stp.pub.k;
             a.pa = stp.pub.lhs_property; a.pb = stp.pub.rhs_property;
+            a.transA = stp.pub.lhs_transposed; a.transB = stp.pub.rhs_transposed;
             if (stp.is_last) {
                 a.C = x; a.strideC = out_stride;
                 a.pout = p->result_desc.property;
@@ -214,6 +222,8 @@ mom_status_t execute_impl(const mom_plan *p, const float *const *chain_ptrs, con
                 a.strideC = (long long)stp.pub.m * stp.pub.n;
                 a.pout = stp.pub.out_property;
                 a.add.count = 0;
+                a.add.transposed = 0;
+                a.add.rows = (int)stp.pub.m;
             }
             cudaEvent_t *ev = timing ? &p->dev->events[((size_t)(p->dev->timed_executes % TIMING_SLOTS) * ns + s) * 3] : nullptr;
             if (ev) cudaEventRecord(ev[0], stream);

@@ -24,9 +24,10 @@ constexpr int WARPS = THREADS / 32;
 // dimension ld.  Only the part inside the structure is read; the rest is zero-filled.  16-byte
 // asynchronous copies (cp.async) keep every load of every operand in flight at once; a copy with
 // source size 0 writes zeros.  The caller waits with cp_async_wait_all() + __syncthreads().
-__device__ void load_operand(float *__restrict__ dst, const float *__restrict__ src, int rows, int cols, int ld, int prop) {
+__device__ void load_operand(float *__restrict__ dst, const float *__restrict__ src, int rows, int cols, int ld, int prop,
+                             int transposed) {
     const int vec_per_row = (cols + 3) >> 2;
-    const bool vec_ok = (cols & 3) == 0 && (reinterpret_cast<uintptr_t>(src) & 15) == 0;
+    const bool vec_ok = !transposed && (cols & 3) == 0 && (reinterpret_cast<uintptr_t>(src) & 15) == 0;
     // thread -> (row, float4 column); when the row length divides the block the column stays fixed and
     // the row advances by a constant, which avoids a division per copy
     const bool regular = (THREADS % vec_per_row) == 0;
@@ -43,7 +44,12 @@ __device__ void load_operand(float *__restrict__ dst, const float *__restrict__ 
             asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(daddr), "l"(p), "r"(needed ? 16 : 0) : "memory");
         } else {
             float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (needed) {
+            if (needed && transposed) {          // stored cols x rows: entry (r, c) is at c * rows + r
+                if (c < cols) v.x = __ldg(src + (size_t)c * rows + r);
+                if (c + 1 < cols) v.y = __ldg(src + (size_t)(c + 1) * rows + r);
+                if (c + 2 < cols) v.z = __ldg(src + (size_t)(c + 2) * rows + r);
+                if (c + 3 < cols) v.w = __ldg(src + (size_t)(c + 3) * rows + r);
+            } else if (needed) {
                 if (c < cols) v.x = __ldg(p);
                 if (c + 1 < cols) v.y = __ldg(p + 1);
                 if (c + 2 < cols) v.z = __ldg(p + 2);
@@ -231,7 +237,7 @@ fused_small_kernel(const FusedPlan fp) {
     for (long long inst = blockIdx.x; inst < fp.batch; inst += gridDim.x) {
         for (int i = 0; i < fp.n_ops; ++i) {
             const FusedOperand &op = fp.ops[i];
-            load_operand(smem + op.smem_off, op.ptr + inst * op.stride, op.rows, op.cols, op.ld, op.prop);
+            load_operand(smem + op.smem_off, op.ptr + inst * op.stride, op.rows, op.cols, op.ld, op.prop, op.transposed);
         }
         cp_async_wait_all();
         __syncthreads();

@@ -17,6 +17,7 @@ struct FusedOperand {
     int rows, cols, prop;
     int smem_off;            // floats
     int ld;                  // leading dimension in shared memory (floats)
+    int transposed;          // stored as cols x rows; read transposed into shared memory
 };
 
 struct FusedStep {

@@ -13,13 +13,15 @@ struct ProductArgs {
     const float *B;
     float *C;
     int m, n, k;
-    int pa, pb, pout;                       // mom_property_t of A, B and of what is written to C
+    int pa, pb, pout;                       // mom_property_t of A, B (as used) and of what is written to C
+    int transA, transB;                     // the operand is stored transposed (k x m resp. n x k)
     long long strideA, strideB, strideC;    // elements between batch instances
     AddTerms add;
 };
 
 cudaError_t launch_product_ffma(const ProductArgs &a, int batch, cudaStream_t stream);
 
+// src_mode: 0 pointer, 1 Identity, 2 X itself (in place), 3 pointer to the transposed matrix (cols x rows)
 cudaError_t launch_elementwise(const float *src, long long src_stride, int src_mode, float *X, long long x_stride,
                                int rows, int cols, int out_prop, const AddTerms &add, int batch, cudaStream_t stream);
 

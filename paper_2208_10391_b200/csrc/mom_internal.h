@@ -51,8 +51,9 @@ struct DeviceState;   // launcher-owned, created on first execute (execute.cu)
 
 struct mom_plan {
     int32_t variant = 0;
-    std::vector<mom_matrix_desc_t> chain;      // original operands
+    std::vector<mom_matrix_desc_t> chain;      // original operands as the equation uses them (transposed type where flagged)
     std::vector<mom_matrix_desc_t> add;
+    std::vector<char> chain_t, add_t;          // operand enters transposed: stored shape is (cols x rows) of the entry above
     std::vector<int32_t> kept;                 // original indices surviving identity simplification
     std::string paren;
     uint64_t mults = 0;                        // useful multiplications of the chosen tree

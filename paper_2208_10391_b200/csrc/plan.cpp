@@ -120,16 +120,45 @@ mom_status_t mom_matrix_desc(int64_t rows, int64_t cols, mom_property_t property
 mom_status_t mom_equation_plan(const mom_matrix_desc_t *chain, int32_t n_chain,
                                const mom_matrix_desc_t *add_terms, int32_t n_add,
                                mom_variant_t variant, mom_plan_t **out_plan) {
-    if (!out_plan || !chain || n_chain < 1 || n_add < 0 || (n_add > 0 && !add_terms)) return MOM_ERR_INVALID_ARG;
+    return mom_equation_plan_transposed(chain, nullptr, n_chain, add_terms, nullptr, n_add, variant, out_plan);
+}
+
+mom_status_t mom_equation_plan_transposed(const mom_matrix_desc_t *stored_chain, const int32_t *chain_transposed, int32_t n_chain,
+                                          const mom_matrix_desc_t *stored_add, const int32_t *add_transposed, int32_t n_add,
+                                          mom_variant_t variant, mom_plan_t **out_plan) {
+    if (!out_plan || !stored_chain || n_chain < 1 || n_add < 0 || (n_add > 0 && !stored_add)) return MOM_ERR_INVALID_ARG;
     if ((int)variant < 0 || (int)variant > 2) return MOM_ERR_INVALID_ARG;
     for (int i = 0; i < n_chain; ++i) {
-        mom_status_t st = check_desc(chain[i]);
+        mom_status_t st = check_desc(stored_chain[i]);
         if (st != MOM_OK) return st;
     }
     for (int i = 0; i < n_add; ++i) {
-        mom_status_t st = check_desc(add_terms[i]);
+        mom_status_t st = check_desc(stored_add[i]);
         if (st != MOM_OK) return st;
     }
+    // A transposed operand takes part with its transposed type: shape swapped, lowerTri <-> upperTri
+    // (the inference rule of the paper's Section 2); from here on `chain` / `add_terms` are the types as used.
+    auto as_used = [](const mom_matrix_desc_t &d, bool t) {
+        if (!t) return d;
+        const int32_t prop = d.property == MOM_LOWER_TRI ? (int32_t)MOM_UPPER_TRI
+                             : d.property == MOM_UPPER_TRI ? (int32_t)MOM_LOWER_TRI : d.property;
+        return mom_matrix_desc_t{d.cols, d.rows, prop, d.dtype};
+    };
+    std::vector<mom_matrix_desc_t> chain_v, add_v;
+    std::vector<char> chain_t((size_t)n_chain, 0), add_t((size_t)n_add, 0);
+    try {
+        for (int i = 0; i < n_chain; ++i) {
+            chain_t[i] = chain_transposed && chain_transposed[i] != 0;
+            chain_v.push_back(as_used(stored_chain[i], chain_t[i] != 0));
+        }
+        for (int i = 0; i < n_add; ++i) {
+            add_t[i] = add_transposed && add_transposed[i] != 0;
+            add_v.push_back(as_used(stored_add[i], add_t[i] != 0));
+        }
+    } catch (const std::bad_alloc &) {
+        return MOM_ERR_ALLOC;
+    }
+    const mom_matrix_desc_t *chain = chain_v.data(), *add_terms = add_v.data();
     for (int i = 0; i + 1 < n_chain; ++i)
         if (chain[i].cols != chain[i + 1].rows) return MOM_ERR_SHAPE_MISMATCH;
     const int64_t rows = chain[0].rows, cols = chain[n_chain - 1].cols;
@@ -142,6 +171,8 @@ mom_status_t mom_equation_plan(const mom_matrix_desc_t *chain, int32_t n_chain,
         p->variant = (int32_t)variant;
         p->chain.assign(chain, chain + n_chain);
         if (n_add) p->add.assign(add_terms, add_terms + n_add);
+        p->chain_t = chain_t;
+        p->add_t = add_t;
         for (int i = 0; i < n_add; ++i) p->add_flops += nnz(add_terms[i]);
 
         // identity simplification: A*I -> A, I*A -> A, I*I -> I
@@ -190,7 +221,11 @@ mom_status_t mom_equation_plan(const mom_matrix_desc_t *chain, int32_t n_chain,
                 mom_plan *p; const std::vector<Node> &node; const std::vector<int> &split; int r; int32_t &next_id;
                 std::string &s;
                 int32_t run(int i, int j) {
-                    if (i == j) { s += std::to_string(p->kept[i]); return p->kept[i]; }
+                    if (i == j) {
+                        s += std::to_string(p->kept[i]);
+                        if (p->chain_t[p->kept[i]]) s += "^T";
+                        return p->kept[i];
+                    }
                     const int k = split[(size_t)i * r + j];
                     s += "(";
                     const int32_t l = run(i, k);
@@ -202,6 +237,8 @@ mom_status_t mom_equation_plan(const mom_matrix_desc_t *chain, int32_t n_chain,
                     std::memset(&st.pub, 0, sizeof(st.pub));
                     st.pub.lhs = l; st.pub.rhs = rr; st.pub.out = next_id++;
                     st.pub.lhs_property = a.prop; st.pub.rhs_property = b.prop; st.pub.out_property = o.prop;
+                    st.pub.lhs_transposed = l < (int32_t)p->chain.size() && p->chain_t[l];
+                    st.pub.rhs_transposed = rr < (int32_t)p->chain.size() && p->chain_t[rr];
                     st.pub.m = a.rows; st.pub.k = a.cols; st.pub.n = b.cols;
                     useful_mults(a.prop, b.prop, a.rows, a.cols, b.cols, &st.pub.useful_mults);
                     const bool ta = is_tri(a.prop), tb = is_tri(b.prop);

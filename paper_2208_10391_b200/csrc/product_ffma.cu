@@ -33,13 +33,16 @@ product_ffma_kernel(ProductArgs a) {
     // global -> shared mapping
     const int a_row = tid >> 1, a_k = (tid & 1) * 4;          // A tile: 128 rows x 8 k, one float4 along k
     const int b_k = tid >> 5, b_col = (tid & 31) * 4;         // B tile: 8 k x 128 cols, one float4 along n
-    const bool a_vec = (k % 4 == 0) && ((reinterpret_cast<uintptr_t>(A) & 15) == 0);
-    const bool b_vec = (n % 4 == 0) && ((reinterpret_cast<uintptr_t>(B) & 15) == 0);
+    const bool a_vec = !a.transA && (k % 4 == 0) && ((reinterpret_cast<uintptr_t>(A) & 15) == 0);
+    const bool b_vec = !a.transB && (n % 4 == 0) && ((reinterpret_cast<uintptr_t>(B) & 15) == 0);
 
     auto load_a = [&](int k0, float (&v)[4]) {
         const int r = r0 + a_row, kk = k0 + a_k;
         v[0] = v[1] = v[2] = v[3] = 0.0f;
-        if (r < m) {
+        if (r < m && a.transA) {                 // stored k x m: consecutive threads read consecutive rows r
+#pragma unroll
+            for (int i = 0; i < 4; ++i) if (kk + i < k) v[i] = __ldg(A + (long long)(kk + i) * m + r);
+        } else if (r < m) {
             const float *p = A + (long long)r * k + kk;
             if (a_vec && kk + 3 < k) {
                 const float4 t = __ldg(reinterpret_cast<const float4 *>(p));
@@ -53,7 +56,10 @@ product_ffma_kernel(ProductArgs a) {
     auto load_b = [&](int k0, float (&v)[4]) {
         const int kk = k0 + b_k, c = c0 + b_col;
         v[0] = v[1] = v[2] = v[3] = 0.0f;
-        if (kk < k) {
+        if (kk < k && a.transB) {                // stored n x k
+#pragma unroll
+            for (int i = 0; i < 4; ++i) if (c + i < n) v[i] = __ldg(B + (long long)(c + i) * k + kk);
+        } else if (kk < k) {
             const float *p = B + (long long)kk * n + c;
             if (b_vec && c + 3 < n) {
                 const float4 t = __ldg(reinterpret_cast<const float4 *>(p));
@@ -135,7 +141,7 @@ product_ffma_kernel(ProductArgs a) {
 }
 
 // X = src (+ Add terms), masked to the result's structure.  src_mode: 0 pointer, 1 Identity,
-// 2 X itself (in place; used to add terms beyond the fused limit).
+// 2 X itself (in place; used to add terms beyond the fused limit), 3 pointer to the transposed matrix.
 __global__ void __launch_bounds__(256)
 elementwise_kernel(const float *__restrict__ src, long long src_stride, int src_mode, float *X, long long x_stride,
                    int rows, int cols, int out_prop, AddTerms add) {
@@ -145,6 +151,7 @@ elementwise_kernel(const float *__restrict__ src, long long src_stride, int src_
         const int r = (int)(e / cols), c = (int)(e % cols);
         float v;
         if (src_mode == 0) v = __ldg(src + inst * src_stride + e);
+        else if (src_mode == 3) v = __ldg(src + inst * src_stride + (long long)c * rows + r);
         else if (src_mode == 1) v = (r == c) ? 1.0f : 0.0f;
         else v = X[inst * x_stride + e];
         X[inst * x_stride + e] = finish_entry(v, add, inst, r, c, cols, out_prop);

@@ -123,7 +123,13 @@ __device__ __forceinline__ void epilogue_chunk(const TcParams &prm, const CUtens
     const bool row_ok = r < prm.m;
     for (int a = 0; a < prm.add.count; ++a) {                   // Add terms, left to right
         const float *p = prm.add.ptr[a];
-        if (p) {
+        if (p && ((prm.add.transposed >> a) & 1u)) {             // term stored as n x m: column-wise reads
+            if (row_ok) {
+#pragma unroll
+                for (int j = 0; j < 32; ++j)
+                    if (col0 + j < prm.n) v[j] += __ldg(p + (long long)(col0 + j) * prm.m + r);
+            }
+        } else if (p) {
             if (row_ok) {
                 const float4 *src = reinterpret_cast<const float4 *>(p + (long long)r * prm.n + col0);
 #pragma unroll
@@ -804,12 +810,20 @@ mom_status_t tc_launch_step(const mom_plan &p, TcPlanState &s, int step, const P
     // operand planes: written by the producing step's epilogue, or split here from the f32 operand
     auto blocks = [](int x) { return (x + SPLIT_PIECE - 1) / SPLIT_PIECE; };
     int split_launches = 0;
+    // The MMA wants A as m x k and B as n x k (both K-major).  An operand stored the other way round
+    // (a transposed chain operand) only swaps which of the two split kernels reads it; the structure
+    // argument is the one of the matrix as stored (the transpose of a lower triangle is an upper one).
+    auto stored_prop = [](int prop_as_used) {
+        return prop_as_used == MOM_LOWER_TRI ? (int)MOM_UPPER_TRI : prop_as_used == MOM_UPPER_TRI ? (int)MOM_LOWER_TRI : prop_as_used;
+    };
     if (!st.a_planes_ready) {
-        split_planes_kernel<false><<<dim3(blocks(a.k), blocks(a.m)), 256, 0, stream>>>(a.A, a_hi, a_lo, a.m, a.k, a.pa);
+        if (!a.transA) split_planes_kernel<false><<<dim3(blocks(a.k), blocks(a.m)), 256, 0, stream>>>(a.A, a_hi, a_lo, a.m, a.k, a.pa);
+        else split_planes_kernel<true><<<dim3(blocks(a.m), blocks(a.k)), 256, 0, stream>>>(a.A, a_hi, a_lo, a.k, a.m, stored_prop(a.pa));
         ++split_launches;
     }
     if (!st.b_planes_ready) {
-        split_planes_kernel<true><<<dim3(blocks(a.n), blocks(a.k)), 256, 0, stream>>>(a.B, b_hi, b_lo, a.k, a.n, a.pb);
+        if (!a.transB) split_planes_kernel<true><<<dim3(blocks(a.n), blocks(a.k)), 256, 0, stream>>>(a.B, b_hi, b_lo, a.k, a.n, a.pb);
+        else split_planes_kernel<false><<<dim3(blocks(a.k), blocks(a.n)), 256, 0, stream>>>(a.B, b_hi, b_lo, a.n, a.k, stored_prop(a.pb));
         ++split_launches;
     }
     if (cudaGetLastError() != cudaSuccess) return MOM_ERR_CUDA;

@@ -21,7 +21,7 @@ def run_equation(eq: wl.Equation, variant: int, chain=None, add=None, via: str =
     """Plan and evaluate `eq` on the GPU; returns (X as numpy f32, plan, (chain, add) host arrays)."""
     if chain is None:
         chain, add = wl.generate(eq)
-    plan = mom.mom_equation_plan(eq.descs(), eq.add_descs(), variant)
+    plan = mom.mom_equation_plan_transposed(eq.descs(), eq.chain_t, eq.add_descs(), eq.add_t, variant)
     rd = plan.result_desc()
     batch = eq.batch
     shape = (batch, rd.rows, rd.cols) if batch > 1 else (rd.rows, rd.cols)
@@ -66,7 +66,7 @@ def run_equation(eq: wl.Equation, variant: int, chain=None, add=None, via: str =
 
 def check_against_oracle(eq: wl.Equation, x: np.ndarray, plan, chain, add, rows=None, instances=None, tol: float = TOL):
     """Element-wise parity with the fp64 oracle; returns the worst normwise error seen."""
-    want = op.plan(eq.descs(), eq.add_descs())
+    want = op.plan(eq.descs(), eq.add_descs(), eq.chain_t, eq.add_t)
     assert plan.parenthesization() == want.paren
     assert plan.flops() == (want.mul_flops, want.add_flops)
     prop = plan.result_desc().property
@@ -78,7 +78,9 @@ def check_against_oracle(eq: wl.Equation, x: np.ndarray, plan, chain, add, rows=
         c = [None if a is None else (a if b is None else a[b]) for a in chain]
         t = [None if a is None else (a if b is None else a[b]) for a in add]
         xb = x if b is None else x[b]
-        x_ref, d = ov.evaluate(c, eq.descs(), t, eq.add_descs(), rows=rows)
+        c, cd = ov.transposed_operands(c, eq.descs(), eq.chain_t)
+        t, td = ov.transposed_operands(t, eq.add_descs(), eq.add_t)
+        x_ref, d = ov.evaluate(c, cd, t, td, rows=rows)
         got = xb if rows is None else xb[rows]
         err = ov.normwise_error(got, x_ref, d)
         assert err <= tol, f"normwise error {err:.3e} > {tol:.1e} ({eq.name}, instance {b})"

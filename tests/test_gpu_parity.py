@@ -260,3 +260,50 @@ def test_argument_errors_are_reported_before_any_launch():
     assert status() == mom.OK
     torch.cuda.synchronize()
     assert plan.device_status() == (0, 0)
+
+
+# ---------------------------------------------------------------- Transpose (paper Table 1; Section 2 inference rule)
+TRANSPOSE_CASES = {
+    "At_B": (((200, 136, G), (200, 264, G)), (True, False), (), ()),
+    "A_Bt": (((136, 200, G), (264, 200, G)), (False, True), (), ()),
+    "At_Bt_plus_Ct": (((200, 136, G), (264, 200, G)), (True, True), ((264, 136, G),), (True,)),
+    "Lt_G": (((328, 328, L), (328, 72, G)), (True, False), (), ()),
+    "G_Ut": (((72, 328, G), (328, 328, U)), (False, True), (), ()),
+    "Lt_L": (((264, 264, L), (264, 264, L)), (True, False), (), ()),
+    "Lt_Lt_plus_Ut": (((264, 264, L), (264, 264, L)), (True, True), ((264, 264, L),), (True,)),
+    "chain": (((96, 200, G), (96, 96, U), (328, 96, G), (328, 40, G)), (True, True, True, False), ((200, 40, G), (40, 200, G)), (False, True)),
+    "zero_step": (((56, 120, G),), (True,), ((56, 120, G), (120, 56, G)), (True, False)),
+    "zero_step_Lt": (((64, 64, L),), (True,), ((64, 64, I),), (False,)),
+    "tiny_fused": (((64, 64, L), (32, 64, G), (48, 32, G)), (True, True, True), ((64, 48, G),), (False,)),
+    "odd_sizes": (((33, 21, G), (33, 33, U), (33, 18, G)), (True, True, False), ((18, 21, G),), (True,)),
+}
+
+
+@pytest.mark.parametrize("variant", VARIANTS + [mom.VARIANT_3XTF32], ids=VNAME.get)
+@pytest.mark.parametrize("name", sorted(TRANSPOSE_CASES))
+def test_transposed_operands(name, variant):
+    chain, ct, add, at = TRANSPOSE_CASES[name]
+    dist = lambda p: "uniform" if p != G else "normal"
+    eq = Equation(f"transpose_{name}", 80, tuple(Operand(r, c, p, dist(p)) for r, c, p in chain),
+                  tuple(Operand(r, c, p, dist(p)) for r, c, p in add), chain_t=ct, add_t=at)
+    _, x, plan = both(eq, variant)
+    if name == "Lt_Lt_plus_Ut":
+        assert plan.result_desc().property == U       # (L^T)(L^T) + (L)^T... every summand is upper triangular
+
+
+@pytest.mark.parametrize("variant", [mom.VARIANT_FFMA, mom.VARIANT_3XTF32], ids=VNAME.get)
+def test_transposed_operands_batched(variant):
+    eq = Equation("transpose_batched", 81, (Operand(64, 64, L), Operand(48, 64, G), Operand(48, 16, G)), (Operand(16, 64, G),),
+                  batch=40, chain_t=(True, True, False), add_t=(True,))
+    both(eq, variant)
+
+
+def test_transposed_operands_large_sampled_rows():
+    # large enough for the CTA-pair kernel: X = L^T * B^T + C with L stored lower triangular (used as upper)
+    m, n = 3336, 3592
+    eq = Equation("transpose_pair", 82, (Operand(m, m, L), Operand(n, m, G, "normal", 0.02)), (Operand(m, n, G, "normal"),),
+                  chain_t=(True, True))
+    x, plan, (chain, add) = run_equation(eq, mom.VARIANT_3XTF32)
+    assert plan.step(0).uses_tensor_cores and plan.step(0).lhs_property == U
+    rows = np.sort(np.random.default_rng(4).choice(m, size=32, replace=False))
+    check_against_oracle(eq, x, plan, chain, add, rows=rows)

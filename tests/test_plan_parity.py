@@ -131,3 +131,31 @@ def test_step_kinds():
     for (a, b), kind in cases.items():
         p = mom.mom_equation_plan([(8, 8, a), (8, 8, b)])
         assert p.step(0).kind == kind
+
+
+def test_transposed_operands_match_the_oracle():
+    rng = np.random.default_rng(17)
+    for seed in range(200):
+        eq = wl.random_equation(5000 + seed, max_len=7, max_dim=40)
+        ct = [bool(rng.integers(0, 2)) for _ in eq.chain]
+        at = [bool(rng.integers(0, 2)) for _ in eq.add]
+        # store the flagged operands transposed, so that the equation as used stays well-formed
+        swap = {mom.LOWER_TRI: mom.UPPER_TRI, mom.UPPER_TRI: mom.LOWER_TRI}
+        stored_c = [(c, r, swap.get(p, p)) if t else (r, c, p) for (r, c, p), t in zip(eq.descs(), ct)]
+        stored_a = [(c, r, swap.get(p, p)) if t else (r, c, p) for (r, c, p), t in zip(eq.add_descs(), at)]
+        want = op.plan(stored_c, stored_a, ct, at)
+        got = mom.mom_equation_plan_transposed(stored_c, ct, stored_a, at)
+        assert got.parenthesization() == want.paren
+        assert got.flops() == (want.mul_flops, want.add_flops)
+        rd = got.result_desc()
+        assert (rd.rows, rd.cols, rd.property) == (want.result_desc.rows, want.result_desc.cols, want.result_desc.prop)
+        for g, w in zip(got.steps(), want.steps):
+            assert (g.lhs, g.rhs, g.out, g.m, g.n, g.k, g.useful_mults) == (w.lhs, w.rhs, w.out, w.m, w.n, w.k, w.mults)
+            assert g.lhs_transposed == int(g.lhs < len(ct) and ct[g.lhs]) and g.rhs_transposed == int(g.rhs < len(ct) and ct[g.rhs])
+    # the paper's rule: the transpose of a lower-triangular matrix is upper triangular
+    p = mom.mom_equation_plan_transposed([(9, 9, mom.LOWER_TRI), (9, 9, mom.LOWER_TRI)], [True, True])
+    assert p.result_desc().property == mom.UPPER_TRI and p.parenthesization() == "(0^T*1^T)"
+    with pytest.raises(mom.MomError) as e:
+        mom.mom_equation_plan_transposed([(7, 30, 0), (7, 40, 0)], [False, False])
+    assert e.value.status == mom.ERR_SHAPE_MISMATCH
+    assert mom.mom_equation_plan_transposed([(7, 30, 0), (7, 40, 0)], [True, False]).result_desc().rows == 30
