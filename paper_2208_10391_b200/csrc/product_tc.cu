@@ -365,18 +365,20 @@ product_tc_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_con
 // CTA-pair variant (cta_group::2): two CTAs of a cluster share one 256 x 256 output tile.  Each CTA
 // loads its own 128 rows of A and only its own half (128 columns) of B -- the tensor cores of the pair
 // exchange the B halves -- so a stage is 64 KiB instead of 96 (three stages fit) and the L2 / shared
-// memory traffic per flop drops by a third.  The leader CTA (cluster rank 0) issues every MMA; each CTA
-// counts its own loads on its own "full" barrier and the peer relays completion to the leader with one
-// remote arrive per stage; tcgen05.commit with a CTA mask releases the stage in both CTAs and publishes
-// the accumulator to both epilogues; the peer's epilogue warps tell the leader over the cluster when an
-// accumulator may be overwritten.
+// memory traffic per flop drops by a third.  The leader CTA (cluster rank 0) issues every MMA.  Only the
+// leader's "full" barriers are used: the leader's producer arms one with the bytes of both CTAs' loads and
+// the peer's TMA loads report their bytes there (cta_group::2 form), so no thread-level message crosses
+// the pair on the way in.  (Two variants were slower: the peer also arriving remotely on that barrier, and
+// each CTA counting its own loads with a per-stage relay to the leader.)  tcgen05.commit with a CTA mask
+// releases the stage in both CTAs and publishes the accumulator to both epilogues; the peer's epilogue
+// warps tell the leader over the cluster when an accumulator may be overwritten.
 // ---------------------------------------------------------------------------------------------
 constexpr int P_BM = 2 * BM;                  // rows of a pair tile
 constexpr int P_STAGES = 3;
 constexpr int P_A_PLANE_BYTES = BM * BK * 4;          // 16 KiB: this CTA's 128 rows
 constexpr int P_B_PLANE_BYTES = (BN / 2) * BK * 4;    // 16 KiB: this CTA's 128 columns of B
 constexpr int P_STAGE_BYTES = 2 * P_A_PLANE_BYTES + 2 * P_B_PLANE_BYTES;   // 64 KiB
-constexpr int P_NUM_BARRIERS = 3 * P_STAGES + 4 + 1;
+constexpr int P_NUM_BARRIERS = 2 * P_STAGES + 4 + 1;
 constexpr int P_SMEM_BYTES = 1024 + P_STAGES * P_STAGE_BYTES + EPI_BYTES + 256;
 static_assert(P_SMEM_BYTES <= 227 * 1024, "shared memory budget");
 
@@ -395,7 +397,6 @@ product_tc_pair_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __gri
     auto tmem_full_bar = [&](int a) { return bars + 8 * (2 * P_STAGES + a); };
     auto tmem_empty_bar = [&](int a) { return bars + 8 * (2 * P_STAGES + 2 + a); };
     const uint32_t drain_bar = bars + 8 * (2 * P_STAGES + 4);
-    auto peer_ready_bar = [&](int s) { return bars + 8 * (2 * P_STAGES + 5 + s); };   // leader: the peer's stage has landed
     const uint32_t tmem_slot = bars + 8 * P_NUM_BARRIERS;
     volatile int *abort_flag = &abort_word;
 
@@ -405,11 +406,7 @@ product_tc_pair_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __gri
 
     if (threadIdx.x == 0) {
         abort_word = 0;
-        for (int s = 0; s < P_STAGES; ++s) {
-            ptx::mbar_init(full_bar(s), 1);
-            ptx::mbar_init(empty_bar(s), 1);
-            ptx::mbar_init(peer_ready_bar(s), 1);
-        }
+        for (int s = 0; s < P_STAGES; ++s) { ptx::mbar_init(full_bar(s), 1); ptx::mbar_init(empty_bar(s), 1); }
         ptx::mbar_init(tmem_full_bar(0), 1);
         ptx::mbar_init(tmem_full_bar(1), 1);
         ptx::mbar_init(tmem_empty_bar(0), 8);               // four epilogue warps in each CTA
@@ -439,16 +436,17 @@ product_tc_pair_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __gri
                 if (lane == 0) ok = wait_barrier(empty_bar(s), parity, abort_flag, prm.status, (1 << 24) | (s << 16) | (t & 0xFFFF));
                 ok = __shfl_sync(0xffffffffu, ok, 0);
                 if (!ok) break;
-                // each CTA counts its own loads on its own barrier (per-transaction updates of a barrier in the
-                // other SM were several times slower); the peer's MMA warp relays "landed" to the leader
-                if (lane == 0) ptx::mbar_arrive_expect_tx(full_bar(s), P_STAGE_BYTES);
+                // Both CTAs' loads are counted on the leader's barrier: the leader alone arms it with the bytes of
+                // the whole pair, the peer's TMA reports its bytes there (cta_group::2 form).
+                const uint32_t bar = rank == 0 ? full_bar(s) : ptx::map_to_cta(full_bar(s), 0);
+                if (lane == 0 && rank == 0) ptx::mbar_arrive_expect_tx(full_bar(s), 2 * P_STAGE_BYTES);
                 __syncwarp();
                 const uint32_t st = stage_addr(s);
                 const int a_row = tile.x + (int)rank * BM, b_row = tile.y + (int)rank * (BN / 2);
-                if (lane == 0) ptx::tma_load_2d(st, &map_a_hi, kb, a_row, full_bar(s));
-                else if (lane == 1) ptx::tma_load_2d(st + P_A_PLANE_BYTES, &map_a_lo, kb, a_row, full_bar(s));
-                else if (lane == 2) ptx::tma_load_2d(st + 2 * P_A_PLANE_BYTES, &map_b_hi, kb, b_row, full_bar(s));
-                else if (lane == 3) ptx::tma_load_2d(st + 2 * P_A_PLANE_BYTES + P_B_PLANE_BYTES, &map_b_lo, kb, b_row, full_bar(s));
+                if (lane == 0) ptx::tma_load_2d_pair(st, &map_a_hi, kb, a_row, bar);
+                else if (lane == 1) ptx::tma_load_2d_pair(st + P_A_PLANE_BYTES, &map_a_lo, kb, a_row, bar);
+                else if (lane == 2) ptx::tma_load_2d_pair(st + 2 * P_A_PLANE_BYTES, &map_b_hi, kb, b_row, bar);
+                else if (lane == 3) ptx::tma_load_2d_pair(st + 2 * P_A_PLANE_BYTES + P_B_PLANE_BYTES, &map_b_lo, kb, b_row, bar);
             }
         }
         // failure path: give loads that are still in flight time to land before this CTA's memory goes away
@@ -457,20 +455,6 @@ product_tc_pair_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __gri
             while (global_ns() - t0 < 200000ull) { }
         }
     } else if (warp == 1) {
-        // ------------------------------------------------------------------ peer CTA: relay "stage landed" to the leader
-        if (lane == 0 && rank != 0) {
-            uint32_t it = 0;
-            bool ok = true;
-            for (int t = pair; t < prm.num_tiles && ok; t += num_pairs) {
-                const int4 tile = prm.tiles[t];
-                for (int kb = tile.z; kb < tile.w; kb += BK, ++it) {
-                    const int s = it % P_STAGES;
-                    ok = wait_barrier(full_bar(s), (it / P_STAGES) & 1, abort_flag, prm.status, (7 << 24) | (s << 16) | (t & 0xFFFF));
-                    if (!ok) break;
-                    ptx::mbar_arrive_cluster(ptx::map_to_cta(peer_ready_bar(s), 0));
-                }
-            }
-        }
         // ------------------------------------------------------------------ MMA issuer (leader CTA, one thread)
         if (lane == 0 && rank == 0) {
             constexpr uint32_t idesc = ptx::instr_desc_tf32(P_BM, BN, 0, 0);
@@ -487,8 +471,7 @@ product_tc_pair_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __gri
                 uint32_t accumulate = 0;
                 for (int kb = tile.z; kb < tile.w; kb += BK, ++it) {
                     const int s = it % P_STAGES;
-                    ok = wait_barrier(full_bar(s), (it / P_STAGES) & 1, abort_flag, prm.status, (3 << 24) | (s << 16) | (t & 0xFFFF)) &&
-                         wait_barrier(peer_ready_bar(s), (it / P_STAGES) & 1, abort_flag, prm.status, (8 << 24) | (s << 16) | (t & 0xFFFF));
+                    ok = wait_barrier(full_bar(s), (it / P_STAGES) & 1, abort_flag, prm.status, (3 << 24) | (s << 16) | (t & 0xFFFF));
                     if (!ok) break;
                     ptx::tc_fence_after_sync();
                     const uint32_t a_hi = stage_addr(s), a_lo = a_hi + P_A_PLANE_BYTES;
