@@ -214,7 +214,7 @@ class ClockSampler:
 def time_equation(mom, torch, eq, variant, steps, warmup, stream, timing=False):
     """Device-resident timing of one configuration: returns dict with per-step ms list, plan, launches."""
     chain, add = wl.generate(eq)
-    plan = mom.mom_equation_plan(eq.descs(), eq.add_descs(), variant)
+    plan = mom.mom_equation_plan_transposed(eq.descs(), eq.chain_t, eq.add_descs(), eq.add_t, variant)
     rd = plan.result_desc()
     dchain = [None if a is None else torch.from_numpy(a).cuda() for a in chain]
     dadd = [None if a is None else torch.from_numpy(a).cuda() for a in add]
@@ -286,7 +286,8 @@ def run_gpu(args):
     if args.only:
         # one named configuration, nothing else: the small case for profiler captures
         cfgs = {c.name: c for c in (wl.config_tiny(), wl.config_five_general(), wl.config_property_heavy(),
-                                    wl.config_large_square(), wl.config_batched(), wl.config_paper_chain())}
+                                    wl.config_large_square(), wl.config_batched(), wl.config_paper_chain(),
+                                    wl.config_transposed())}
         cfg = cfgs[args.only]
         r = time_equation(mom, torch, cfg, variant, steps=args.steps, warmup=args.warmup, stream=stream, timing=cfg.batch == 1)
         print(json.dumps({"workload": cfg.name, "variant": args.variant, "ms": r["ms"], "useful_flops": r["useful_flops"],
@@ -420,7 +421,7 @@ def run_gpu(args):
         # ---- the other configurations, briefly (min of 5 as in the paper's Section 4, and the median)
         others = []
         for cfg in (wl.config_tiny(), wl.config_five_general(), wl.config_property_heavy(), wl.config_batched(),
-                    wl.config_paper_chain()):
+                    wl.config_paper_chain(), wl.config_transposed()):
             r = time_equation(mom, torch, cfg, variant, steps=20, warmup=3, stream=stream, timing=cfg.batch == 1)
             ms_min, ms_med = min(r["ms"]), statistics.median(r["ms"])
             entry = {"workload": cfg.name, "parenthesization": r["plan"].parenthesization(),

@@ -307,3 +307,11 @@ def test_transposed_operands_large_sampled_rows():
     assert plan.step(0).uses_tensor_cores and plan.step(0).lhs_property == U
     rows = np.sort(np.random.default_rng(4).choice(m, size=32, replace=False))
     check_against_oracle(eq, x, plan, chain, add, rows=rows)
+
+
+def test_config_transposed_full_size_sampled_rows():
+    eq = wl.config_transposed()
+    x, plan, (chain, add) = run_equation(eq, mom.VARIANT_3XTF32)
+    assert plan.parenthesization() == "(0^T*(1*(2^T*3)))"
+    rows = np.sort(np.random.default_rng(6).choice(4096, size=32, replace=False))
+    check_against_oracle(eq, x, plan, chain, add, rows=rows)

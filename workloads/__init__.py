@@ -158,6 +158,17 @@ def config_paper_chain(seed: int = 5) -> Equation:
         Operand(dims[i], dims[i + 1], GENERAL, "normal") for i in range(4)))
 
 
+def config_transposed(n: int = 4096, seed: int = 6) -> Equation:
+    """X = L^T * A * U^T * B + C^T, all n x n: the Transpose op on chain operands and on an Add term.
+
+    L is stored lower triangular (used as upper), U stored upper (used as lower)."""
+    s = float(n) ** -0.5
+    return Equation(f"LtAUtB_plus_Ct_{n}", seed, (
+        Operand(n, n, LOWER_TRI), Operand(n, n, GENERAL, "normal", s),
+        Operand(n, n, UPPER_TRI), Operand(n, n, GENERAL, "normal", s)), (Operand(n, n, GENERAL, "normal"),),
+        chain_t=(True, False, True, False), add_t=(True,))
+
+
 def config_listing2() -> Equation:
     """Listing 2 of the paper: two 5x5 lowerTri matrices filled with the constant 1."""
     return Equation("listing2_LL_5", 0, (
