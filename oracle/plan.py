@@ -308,3 +308,115 @@ def catalan(r: int) -> int:
     for i in range(r - 1):
         c = c * 2 * (2 * i + 1) // (i + 2)
     return c
+
+
+# ----------------------------------------------------------------------------------------------
+# sums of several Mul chains
+# ----------------------------------------------------------------------------------------------
+# Paper Section 2, "Operations": an Equation holds a bag of Mul and Add operations, both variadic, so
+# its value can be a sum of several products,  X = prod(chain_1) + ... + prod(chain_c);  a chain of
+# one factor is a plain Add term.  Readings taken here (the paper gives no rule):
+#   * Add is linear in each summand, so every chain is parenthesized on its own, exactly as `plan` does;
+#   * factors are numbered 0..F-1 across all chains in the order written, intermediates F.. in the order
+#     the chains' products are emitted (chain by chain, each in post-order);
+#   * reuse between chains: a product below the root of its chain's tree is computed once when the same
+#     run of factors (same matrix names, same transposition flags) was already multiplied by an earlier
+#     chain, also below that chain's root; its multiplications are then counted once.  A chain's root
+#     product is never shared: it is what the chain adds to X;
+#   * the result property folds `sum_property` over the chains' product types;
+#   * add_flops = structural non-zeros of every summand after the first.
+
+@dataclass(frozen=True)
+class SumPlan:
+    paren: str
+    mults: int
+    mul_flops: int
+    add_flops: int
+    steps: Tuple[Step, ...]        # global ids, reused products appear once
+    chain_values: Tuple[int, ...]  # per chain: id of its value (a factor id, a step's out), -1 for Identity
+    chain_descs: Tuple[Desc, ...]  # per chain: type of its product
+    result_desc: Desc
+    reused: int                    # products not emitted because an earlier chain computed them
+
+
+def plan_sum(chains: Sequence[Sequence[Tuple[int, int, int]]],
+             transposed: Sequence[Sequence[bool]] = (),
+             names: Sequence[Sequence[int]] = ()) -> SumPlan:
+    """Plan X = sum over chains of prod(chain).  `names[c][f]` identifies the matrix behind factor f of
+    chain c (equal names = the same stored matrix); without names every factor is its own matrix."""
+    if len(chains) < 1:
+        raise OracleError("invalid_arg", "no chain")
+    flags = [list(transposed[c]) if c < len(transposed) else [] for c in range(len(chains))]
+    flags = [f + [False] * (len(ch) - len(f)) for f, ch in zip(flags, chains)]
+    total = sum(len(ch) for ch in chains)
+    if names:
+        if [len(n) for n in names] != [len(ch) for ch in chains]:
+            raise OracleError("invalid_arg", "names do not match the chains")
+        by_name = {}
+        for ch, fl, nm in zip(chains, flags, names):
+            for d, n in zip(ch, nm):
+                if by_name.setdefault(n, tuple(d)) != tuple(d):
+                    raise OracleError("invalid_arg", "one name, two types")
+    else:
+        counter = iter(range(total))
+        names = [[next(counter) for _ in ch] for ch in chains]
+
+    plans = [plan(ch, (), fl) for ch, fl in zip(chains, flags)]
+    rows, cols = plans[0].product_desc.rows, plans[0].product_desc.cols
+    for p in plans[1:]:
+        if (p.product_desc.rows, p.product_desc.cols) != (rows, cols):
+            raise OracleError("shape_mismatch", "summands differ in shape")
+
+    steps: List[Step] = []
+    seen = {}                      # (names and flags of a factor run) -> global id of its product
+    reused = 0
+    next_id = total
+    base = 0
+    values: List[int] = []
+    parens: List[str] = []
+    for c, (p, ch) in enumerate(zip(plans, chains)):
+        n_local = len(ch)
+        span = {i: (i, i) for i in range(n_local)}          # local id -> factor positions covered
+        to_global = {i: base + i for i in range(n_local)}
+        for s in p.steps:
+            lo, hi = span[s.lhs][0], span[s.rhs][1]
+            span[s.out] = (lo, hi)
+            kept_run = tuple((names[c][i], flags[c][i]) for i in range(lo, hi + 1) if i in p.kept)
+            is_root = s is p.steps[-1]
+            if not is_root and kept_run in seen:
+                to_global[s.out] = seen[kept_run]
+                reused += 1
+                continue
+            gid = next_id
+            next_id += 1
+            to_global[s.out] = gid
+            if not is_root:
+                seen[kept_run] = gid
+            steps.append(Step(to_global[s.lhs], to_global[s.rhs], gid, s.m, s.n, s.k,
+                              s.lhs_prop, s.rhs_prop, s.out_prop, s.mults))
+        if p.steps:
+            values.append(to_global[p.steps[-1].out])
+        elif p.kept:
+            values.append(base + p.kept[0])
+        else:
+            values.append(-1)
+        # the chain's string with its factor numbers moved to the global numbering
+        out, num = [], ""
+        for chr_ in p.paren + "\0":
+            if chr_.isdigit():
+                num += chr_
+                continue
+            if num:
+                out.append(str(int(num) + base))
+                num = ""
+            if chr_ != "\0":
+                out.append(chr_)
+        parens.append("".join(out))
+        base += n_local
+
+    mults = sum(s.mults for s in steps)
+    descs = tuple(p.product_desc for p in plans)
+    result_prop = sum_property(descs[0].prop, [d.prop for d in descs[1:]])
+    add_flops = sum(structural_nonzeros(d) for d in descs[1:])
+    return SumPlan("+".join(parens), mults, 2 * mults, add_flops, tuple(steps), tuple(values), descs,
+                   Desc(rows, cols, result_prop), reused)

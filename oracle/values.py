@@ -138,6 +138,25 @@ def evaluate(chain: Sequence[Optional[np.ndarray]], chain_descs: Sequence[Tuple[
     return x, d
 
 
+def evaluate_sum(chains: Sequence[Sequence[Optional[np.ndarray]]],
+                 chain_descs: Sequence[Sequence[Tuple[int, int, int]]],
+                 rows: Optional[np.ndarray] = None, threads: Optional[int] = None
+                 ) -> Tuple[np.ndarray, np.ndarray]:
+    """(X_ref, D) of a sum of Mul chains, X = prod(chain_1) + ... + prod(chain_c)  (paper Section 2,
+    "Operations": Mul and Add are both variadic and an Equation holds a bag of them).
+
+    Every chain is evaluated by `evaluate` on its own, left to right, and the values are added in the
+    order written; D adds up the chains' denominators.  Operands are given as the equation uses them
+    (apply `transposed_operands` first where a factor enters transposed).
+    """
+    x = d = None
+    for mats, descs in zip(chains, chain_descs):
+        xc, dc = evaluate(mats, descs, rows=rows, threads=threads)
+        x = xc if x is None else x + xc
+        d = dc if d is None else d + dc
+    return x, d
+
+
 def evaluate_steps(chain: Sequence[Optional[np.ndarray]], chain_descs: Sequence[Tuple[int, int, int]],
                    steps, add: Sequence[Optional[np.ndarray]] = (),
                    add_descs: Sequence[Tuple[int, int, int]] = (), threads: Optional[int] = None) -> np.ndarray:
