@@ -130,8 +130,32 @@ mom_status_t mom_equation_plan_transposed(const mom_matrix_desc_t *chain, const 
                                           const mom_matrix_desc_t *add_terms, const int32_t *add_transposed, int32_t n_add,
                                           mom_variant_t variant, mom_plan_t **out_plan);
 
-/* mul_flops = 2 * (useful multiplications of the chosen parenthesization); add_flops = structural
- * non-zeros of the Add terms (an Identity term counts its n diagonal entries).  Either may be NULL. */
+/* Plan a sum of several Mul chains, X = prod(chain_0) + prod(chain_1) + ... (paper Section 2, "Operations":
+ * Mul and Add are both variadic and one Equation holds a bag of them).  A chain of one factor is a plain Add term.
+ *   factors            host array with all chains' factors one after the other, AS STORED (n = sum of chain_lengths)
+ *   factor_transposed  host array of n flags, or NULL: the equation uses the transpose of that factor
+ *   factor_names       host array of n integers, or NULL: factors with equal names are the same stored matrix
+ *                      (they must then have equal descriptors, and execute must be given equal pointers and strides
+ *                      for them); NULL means that nothing is known to be shared
+ *   chain_lengths      host array of n_chains >= 1 lengths, each >= 1
+ * Every chain is parenthesized on its own by the rules of mom_equation_plan.  With names, a product below the
+ * root of a chain's tree whose run of factors (names and transposition flags) an earlier chain has already
+ * multiplied, also below its root, is computed once and read by both; a chain's root product is never shared.
+ * Value ids in the steps: 0..n-1 are the factors in the order given, n.. the products in emission order (chain
+ * by chain, post-order, shared products once).  The parenthesization string joins the chains' strings with "+".
+ * The plan executes through mom_equation_execute / _batched / _host with chain_ptrs holding one pointer per
+ * factor (n_add = 0).  All chains must have X's shape.  Errors as mom_equation_plan. */
+mom_status_t mom_equation_plan_sum(const mom_matrix_desc_t *factors, const int32_t *factor_transposed,
+                                   const int32_t *factor_names, const int32_t *chain_lengths, int32_t n_chains,
+                                   mom_variant_t variant, mom_plan_t **out_plan);
+
+/* Number of products that mom_equation_plan_sum did not emit because an earlier chain computes them (0 for
+ * plans of the other entry points). */
+mom_status_t mom_plan_reused_products(const mom_plan_t *plan, int32_t *reused);
+
+/* mul_flops = 2 * (useful multiplications of the chosen parenthesization; over all chains, a shared product
+ * once); add_flops = structural non-zeros of every summand after the first chain: the Add terms (an Identity
+ * term counts its n diagonal entries) and the values of the further chains.  Either may be NULL. */
 mom_status_t mom_plan_flops(const mom_plan_t *plan, uint64_t *mul_flops, uint64_t *add_flops);
 
 /* The chosen parenthesization over ORIGINAL operand indices, e.g. "(0*(1*3))".  Eliminated Identity

@@ -59,6 +59,9 @@ _sigs = {
     "mom_equation_plan_transposed": [ctypes.POINTER(MatrixDesc), ctypes.POINTER(ctypes.c_int32), ctypes.c_int32,
                                      ctypes.POINTER(MatrixDesc), ctypes.POINTER(ctypes.c_int32), ctypes.c_int32,
                                      ctypes.c_int, ctypes.POINTER(_P)],
+    "mom_equation_plan_sum": [ctypes.POINTER(MatrixDesc), ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_int32),
+                              ctypes.POINTER(ctypes.c_int32), ctypes.c_int32, ctypes.c_int, ctypes.POINTER(_P)],
+    "mom_plan_reused_products": [_P, ctypes.POINTER(ctypes.c_int32)],
     "mom_plan_flops": [_P, ctypes.POINTER(ctypes.c_uint64), ctypes.POINTER(ctypes.c_uint64)],
     "mom_plan_parenthesization": [_P, ctypes.c_char_p, ctypes.c_size_t, ctypes.POINTER(ctypes.c_size_t)],
     "mom_plan_num_steps": [_P, ctypes.POINTER(ctypes.c_int32)],
@@ -153,6 +156,11 @@ class Plan:
         buf = ctypes.create_string_buffer(need.value)
         _check(_lib.mom_plan_parenthesization(self._h, buf, need.value, None), "mom_plan_parenthesization")
         return buf.value.decode()
+
+    def reused_products(self) -> int:
+        n = ctypes.c_int32()
+        _check(_lib.mom_plan_reused_products(self._h, ctypes.byref(n)), "mom_plan_reused_products")
+        return n.value
 
     def num_steps(self) -> int:
         n = ctypes.c_int32()
@@ -251,6 +259,26 @@ def mom_equation_plan_transposed(chain: Sequence, chain_transposed: Optional[Seq
                                            variant, ctypes.byref(handle))
     _check(st, "mom_equation_plan_transposed")
     return Plan(handle.value, n_chain, n_add)
+
+
+def mom_equation_plan_sum(chains: Sequence[Sequence], transposed: Optional[Sequence[Sequence]] = None,
+                          names: Optional[Sequence[Sequence[int]]] = None, variant: int = VARIANT_3XTF32) -> Plan:
+    """Plan X = sum over chains of prod(chain); the plan executes with one pointer per factor, chains flattened."""
+    handle = _P()
+    lengths = [len(c) for c in chains]
+    flat = [d for c in chains for d in c]
+    n = len(flat)
+    flags = None
+    if transposed is not None and n:
+        rows = [list(transposed[c]) if c < len(transposed) else [] for c in range(len(chains))]
+        rows = [r + [False] * (l - len(r)) for r, l in zip(rows, lengths)]
+        flags = (ctypes.c_int32 * n)(*[1 if x else 0 for r in rows for x in r])
+    name_arr = (ctypes.c_int32 * n)(*[int(x) for r in names for x in r]) if names is not None and n else None
+    len_arr = (ctypes.c_int32 * max(len(lengths), 1))(*lengths)
+    st = _lib.mom_equation_plan_sum(_desc_array(flat) if n else None, flags, name_arr, len_arr, len(lengths), variant,
+                                    ctypes.byref(handle))
+    _check(st, "mom_equation_plan_sum")
+    return Plan(handle.value, n, 0)
 
 
 def mom_product_3xtf32_noalloc(m: int, n: int, k: int, pa: int, pb: int, a_ptr: int, b_ptr: int, c_ptr: int,

@@ -17,6 +17,8 @@ struct AddTerms {
     long long stride[MAX_FUSED_ADD];     // elements between batch instances
     int count;
     unsigned transposed;                 // bit t: term t is stored transposed (cols x rows of X)
+    unsigned aliases_out;                // bit t: term t is X itself (a later chain adding to it): read past L1, never
+                                         // through the read-only path, and only by the thread that then writes the entry
     int rows;                            // rows of X (leading dimension of a transposed term)
 };
 
@@ -50,7 +52,9 @@ __device__ __forceinline__ float finish_entry(float acc, const AddTerms &add, lo
         if (t < add.count) {
             const float *p = add.ptr[t];
             const long long at = (add.transposed >> t) & 1u ? (long long)c * add.rows + r : (long long)r * ld + c;
-            v += p ? __ldg(p + batch * add.stride[t] + at) : (r == c ? 1.0f : 0.0f);
+            if (!p) v += r == c ? 1.0f : 0.0f;
+            else if ((add.aliases_out >> t) & 1u) v += __ldcg(p + batch * add.stride[t] + at);
+            else v += __ldg(p + batch * add.stride[t] + at);
         }
     }
     return in_structure(out_prop, r, c) ? v : 0.0f;

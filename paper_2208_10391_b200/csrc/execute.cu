@@ -78,6 +78,13 @@ mom_status_t execute_impl(const mom_plan *p, const float *const *chain_ptrs, con
         if (batch > 1 && (chain_strides[i] % 4 != 0 || chain_strides[i] < p->chain[i].rows * p->chain[i].cols))
             return MOM_ERR_INVALID_ARG;
     }
+    if (!p->names.empty()) {          // factors with one name are one matrix: a product shared between chains relies on it
+        for (int i = 0; i < n_chain; ++i)
+            for (int j = 0; j < i; ++j)
+                if (p->names[i] == p->names[j] && p->chain[i].property != MOM_IDENTITY &&
+                    (chain_ptrs[i] != chain_ptrs[j] || (batch > 1 && chain_strides[i] != chain_strides[j])))
+                    return MOM_ERR_INVALID_ARG;
+    }
     for (int i = 0; i < n_add; ++i) {
         if (p->add[i].property == MOM_IDENTITY) continue;
         if (!add_ptrs[i]) return MOM_ERR_INVALID_ARG;
@@ -158,36 +165,64 @@ mom_status_t execute_impl(const mom_plan *p, const float *const *chain_ptrs, con
     const int64_t group = any_tc ? 1 : (batch < 65535 ? batch : 65535);
     const size_t ws_inst = p->workspace_per_instance;
 
+    std::vector<const Summand *> simple;
+    bool has_products = false;
+    for (const Summand &sm : p->summands) {
+        if (sm.kind == SUM_STEP) has_products = true;
+        else simple.push_back(&sm);
+    }
+    const int n_simple = (int)simple.size();
+
     for (int64_t b0 = 0; b0 < batch; b0 += group) {
         const int nb = (int)((batch - b0 < group) ? batch - b0 : group);
         auto chain_op = [&](int id) {
             const long long s = chain_strides ? chain_strides[id] : 0;
             return Operand{chain_ptrs[id] ? chain_ptrs[id] + b0 * s : nullptr, s};
         };
+        float *x = out + b0 * out_stride;
+        // Summands that are not products (Add terms, chains that reduced to one factor or to Identity), in the
+        // order written; `simple[first..]` go into `t`, at most MAX_FUSED_ADD of them.  Returns the next index.
         auto add_terms = [&](int first, AddTerms *t) {
             t->count = 0;
             t->transposed = 0;
+            t->aliases_out = 0;
             t->rows = (int)rows;
-            for (int i = first; i < n_add && t->count < MAX_FUSED_ADD; ++i, ++t->count) {
-                const long long s = add_strides ? add_strides[i] : 0;
-                t->ptr[t->count] = p->add[i].property == MOM_IDENTITY ? nullptr : add_ptrs[i] + b0 * s;
-                t->stride[t->count] = s;
-                if (p->add_t[i]) t->transposed |= 1u << t->count;
+            int i = first;
+            for (; i < n_simple && t->count < MAX_FUSED_ADD; ++i, ++t->count) {
+                const Summand &sm = *simple[i];
+                if (sm.kind == SUM_IDENTITY || (sm.kind == SUM_TERM && p->add[sm.index].property == MOM_IDENTITY)) {
+                    t->ptr[t->count] = nullptr;
+                    t->stride[t->count] = 0;
+                } else if (sm.kind == SUM_TERM) {
+                    const long long s = add_strides ? add_strides[sm.index] : 0;
+                    t->ptr[t->count] = add_ptrs[sm.index] + b0 * s;
+                    t->stride[t->count] = s;
+                    if (p->add_t[sm.index]) t->transposed |= 1u << t->count;
+                } else {
+                    const Operand o = chain_op(sm.index);
+                    t->ptr[t->count] = o.ptr;
+                    t->stride[t->count] = o.stride;
+                    if (p->chain_t[sm.index]) t->transposed |= 1u << t->count;
+                }
             }
-            return first + t->count;
+            return i;
         };
-        float *x = out + b0 * out_stride;
         int added = 0;
 
-        if (ns == 0) {
+        if (!has_products) {
+            // X = first summand + the following ones
+            const Summand &sm = *simple[0];
             AddTerms t;
-            added = add_terms(0, &t);
+            added = add_terms(1, &t);
             cudaError_t e;
-            if (p->kept.empty()) {
+            if (sm.kind == SUM_IDENTITY || (sm.kind == SUM_TERM && p->add[sm.index].property == MOM_IDENTITY)) {
                 e = launch_elementwise(nullptr, 0, 1, x, out_stride, (int)rows, (int)cols, p->result_desc.property, t, nb, stream);
+            } else if (sm.kind == SUM_FACTOR) {
+                const Operand src = chain_op(sm.index);
+                e = launch_elementwise(src.ptr, src.stride, p->chain_t[sm.index] ? 3 : 0, x, out_stride, (int)rows, (int)cols, p->result_desc.property, t, nb, stream);
             } else {
-                const Operand src = chain_op(p->kept[0]);
-                e = launch_elementwise(src.ptr, src.stride, p->chain_t[p->kept[0]] ? 3 : 0, x, out_stride, (int)rows, (int)cols, p->result_desc.property, t, nb, stream);
+                const long long ss = add_strides ? add_strides[sm.index] : 0;
+                e = launch_elementwise(add_ptrs[sm.index] + b0 * ss, ss, p->add_t[sm.index] ? 3 : 0, x, out_stride, (int)rows, (int)cols, p->result_desc.property, t, nb, stream);
             }
             if (e != cudaSuccess) return MOM_ERR_CUDA;
             ++launches;
@@ -212,7 +247,17 @@ mom_status_t execute_impl(const mom_plan *p, const float *const *chain_ptrs, con
             a.m = (int)stp.pub.m; a.n = (int)stp.pub.n; a.k = (int)stp.pub.k;
             a.pa = stp.pub.lhs_property; a.pb = stp.pub.rhs_property;
             a.transA = stp.pub.lhs_transposed; a.transB = stp.pub.rhs_transposed;
-            if (stp.is_last) {
+            if (stp.is_last && stp.accumulate) {
+                // a later chain's product is added to what the earlier ones left in X
+                a.C = x; a.strideC = out_stride;
+                a.pout = p->result_desc.property;
+                a.add.count = 1;
+                a.add.ptr[0] = x;
+                a.add.stride[0] = out_stride;
+                a.add.transposed = 0;
+                a.add.aliases_out = 1u;
+                a.add.rows = (int)rows;
+            } else if (stp.is_last) {
                 a.C = x; a.strideC = out_stride;
                 a.pout = p->result_desc.property;
                 added = add_terms(0, &a.add);
@@ -223,6 +268,7 @@ mom_status_t execute_impl(const mom_plan *p, const float *const *chain_ptrs, con
                 a.pout = stp.pub.out_property;
                 a.add.count = 0;
                 a.add.transposed = 0;
+                a.add.aliases_out = 0;
                 a.add.rows = (int)stp.pub.m;
             }
             cudaEvent_t *ev = timing ? &p->dev->events[((size_t)(p->dev->timed_executes % TIMING_SLOTS) * ns + s) * 3] : nullptr;
@@ -242,8 +288,8 @@ mom_status_t execute_impl(const mom_plan *p, const float *const *chain_ptrs, con
         }
         (void)ws_inst;
 
-        // Add terms beyond the fused limit: X += T, a few at a time, in place
-        while (added < n_add) {
+        // summands beyond the fused limit: X += T, a few at a time, in place
+        while (added < n_simple) {
             AddTerms t;
             const int first = added;
             added = add_terms(first, &t);
@@ -304,6 +350,16 @@ mom_status_t mom_equation_execute_host(const mom_plan_t *plan, const float *cons
         return MOM_OK;
     };
     for (int i = 0; i < n_chain; ++i) {
+        int same = -1;                                 // a named matrix is copied once
+        if (!plan->names.empty())
+            for (int j = 0; j < i && same < 0; ++j)
+                if (plan->names[j] == plan->names[i]) same = j;
+        if (same >= 0) {
+            if (chain_host[i] != chain_host[same]) return MOM_ERR_INVALID_ARG;
+            cptr[i] = cptr[same];
+            cstride[i] = cstride[same];
+            continue;
+        }
         mom_status_t st = stage(plan->chain[i], chain_host[i], &cptr[i], &cstride[i]);
         if (st != MOM_OK) return st;
     }

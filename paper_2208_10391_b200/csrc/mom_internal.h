@@ -29,7 +29,8 @@ inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 struct StepImpl {
     mom_step_t pub;
-    bool is_last = false;           // carries the Add terms and writes X
+    bool is_last = false;           // root of its chain's tree: writes X (the first root also carries the Add terms)
+    bool accumulate = false;        // a later chain's root: adds its product to what X already holds
     // workspace byte offsets (per instance); SIZE_MAX = not used
     size_t out_off = SIZE_MAX;      // f32 intermediate written by this step (not for the last step)
     size_t a_hi_off = SIZE_MAX, a_lo_off = SIZE_MAX;   // split planes of the operands (tensor-core steps)
@@ -45,6 +46,13 @@ struct StepImpl {
     size_t partial_off = SIZE_MAX;
 };
 
+// One summand of X = sum of chain values + Add terms, in the order written.
+enum SummandKind { SUM_STEP = 0, SUM_FACTOR = 1, SUM_TERM = 2, SUM_IDENTITY = 3 };
+struct Summand {
+    int kind;       // SUM_STEP: a chain with products (index = its root step); SUM_FACTOR: a chain that reduced to
+    int index;      // one factor (index = factor id); SUM_TERM: Add term `index`; SUM_IDENTITY: a chain equal to I
+};
+
 struct DeviceState;   // launcher-owned, created on first execute (execute.cu)
 
 }  // namespace mom
@@ -54,7 +62,11 @@ struct mom_plan {
     std::vector<mom_matrix_desc_t> chain;      // original operands as the equation uses them (transposed type where flagged)
     std::vector<mom_matrix_desc_t> add;
     std::vector<char> chain_t, add_t;          // operand enters transposed: stored shape is (cols x rows) of the entry above
-    std::vector<int32_t> kept;                 // original indices surviving identity simplification
+    std::vector<int32_t> chain_begin;          // factors of chain c are [chain_begin[c], chain_begin[c + 1])
+    std::vector<int32_t> names;                // per factor: equal names = the same stored matrix (empty: all distinct)
+    std::vector<int32_t> kept;                 // factor indices surviving identity simplification
+    std::vector<mom::Summand> summands;        // what is added up into X, in the order written
+    int32_t reused = 0;                        // products not emitted because an earlier chain computed them
     std::string paren;
     uint64_t mults = 0;                        // useful multiplications of the chosen tree
     uint64_t add_flops = 0;

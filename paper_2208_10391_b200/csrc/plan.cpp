@@ -3,7 +3,10 @@
 // Pure host code: no CUDA call is made here.
 #include <algorithm>
 #include <cstring>
+#include <map>
 #include <new>
+#include <string>
+#include <vector>
 
 #include "fused_small.h"
 #include "mom_internal.h"
@@ -57,19 +60,17 @@ uint64_t nnz(const mom_matrix_desc_t &d) {
     return (uint64_t)d.rows * ((uint64_t)d.rows + 1) / 2;
 }
 
-// Property of chain value + T1 + ... + Tk.  A sum with terms is never Identity: an Identity summand
-// only contributes its diagonal footprint, which fits inside either triangle.
-int32_t sum_property(int32_t product, const std::vector<mom_matrix_desc_t> &terms) {
-    if (terms.empty()) return product;
+// Property of a sum of summands (chain values and Add terms).  A sum of two or more is never Identity: an
+// Identity summand only contributes its diagonal footprint, which fits inside either triangle.
+int32_t sum_property(const std::vector<int32_t> &props) {
+    if (props.size() == 1) return props[0];
     bool seen = false;
     int32_t acc = MOM_GENERAL;
-    auto fold = [&](int32_t p) {
-        if (p == MOM_IDENTITY) return;
+    for (int32_t p : props) {
+        if (p == MOM_IDENTITY) continue;
         if (!seen) { acc = p; seen = true; }
         else if (acc != p) acc = MOM_GENERAL;
-    };
-    fold(product);
-    for (const auto &t : terms) fold(t.property);
+    }
     return seen ? acc : (int32_t)MOM_LOWER_TRI;
 }
 
@@ -117,17 +118,22 @@ mom_status_t mom_matrix_desc(int64_t rows, int64_t cols, mom_property_t property
     return MOM_OK;
 }
 
-mom_status_t mom_equation_plan(const mom_matrix_desc_t *chain, int32_t n_chain,
-                               const mom_matrix_desc_t *add_terms, int32_t n_add,
-                               mom_variant_t variant, mom_plan_t **out_plan) {
-    return mom_equation_plan_transposed(chain, nullptr, n_chain, add_terms, nullptr, n_add, variant, out_plan);
-}
-
-mom_status_t mom_equation_plan_transposed(const mom_matrix_desc_t *stored_chain, const int32_t *chain_transposed, int32_t n_chain,
-                                          const mom_matrix_desc_t *stored_add, const int32_t *add_transposed, int32_t n_add,
-                                          mom_variant_t variant, mom_plan_t **out_plan) {
-    if (!out_plan || !stored_chain || n_chain < 1 || n_add < 0 || (n_add > 0 && !stored_add)) return MOM_ERR_INVALID_ARG;
+// Shared body of the planning entry points.  `factors` are all chains' stored factors one after the other,
+// `chain_len[c]` of them belong to chain c; `names` (optional) tells which factors are the same stored matrix.
+static mom_status_t plan_equation(const mom_matrix_desc_t *stored_chain, const int32_t *chain_transposed,
+                                  const int32_t *names, const int32_t *chain_len, int32_t n_chains,
+                                  const mom_matrix_desc_t *stored_add, const int32_t *add_transposed, int32_t n_add,
+                                  mom_variant_t variant, mom_plan_t **out_plan) {
+    if (!out_plan || !stored_chain || !chain_len || n_chains < 1 || n_add < 0 || (n_add > 0 && !stored_add))
+        return MOM_ERR_INVALID_ARG;
     if ((int)variant < 0 || (int)variant > 2) return MOM_ERR_INVALID_ARG;
+    int64_t total = 0;
+    for (int c = 0; c < n_chains; ++c) {
+        if (chain_len[c] < 1) return MOM_ERR_INVALID_ARG;
+        total += chain_len[c];
+        if (total > (1 << 20)) return MOM_ERR_INVALID_ARG;
+    }
+    const int n_chain = (int)total;
     for (int i = 0; i < n_chain; ++i) {
         mom_status_t st = check_desc(stored_chain[i]);
         if (st != MOM_OK) return st;
@@ -146,6 +152,7 @@ mom_status_t mom_equation_plan_transposed(const mom_matrix_desc_t *stored_chain,
     };
     std::vector<mom_matrix_desc_t> chain_v, add_v;
     std::vector<char> chain_t((size_t)n_chain, 0), add_t((size_t)n_add, 0);
+    std::vector<int32_t> begin;
     try {
         for (int i = 0; i < n_chain; ++i) {
             chain_t[i] = chain_transposed && chain_transposed[i] != 0;
@@ -155,13 +162,26 @@ mom_status_t mom_equation_plan_transposed(const mom_matrix_desc_t *stored_chain,
             add_t[i] = add_transposed && add_transposed[i] != 0;
             add_v.push_back(as_used(stored_add[i], add_t[i] != 0));
         }
+        begin.push_back(0);
+        for (int c = 0; c < n_chains; ++c) begin.push_back(begin.back() + chain_len[c]);
+        if (names) {                                   // one name, one stored type
+            std::map<int32_t, int> first;
+            for (int i = 0; i < n_chain; ++i) {
+                auto it = first.emplace(names[i], i).first;
+                const mom_matrix_desc_t &a = stored_chain[it->second], &b = stored_chain[i];
+                if (a.rows != b.rows || a.cols != b.cols || a.property != b.property) return MOM_ERR_INVALID_ARG;
+            }
+        }
     } catch (const std::bad_alloc &) {
         return MOM_ERR_ALLOC;
     }
     const mom_matrix_desc_t *chain = chain_v.data(), *add_terms = add_v.data();
-    for (int i = 0; i + 1 < n_chain; ++i)
-        if (chain[i].cols != chain[i + 1].rows) return MOM_ERR_SHAPE_MISMATCH;
-    const int64_t rows = chain[0].rows, cols = chain[n_chain - 1].cols;
+    for (int c = 0; c < n_chains; ++c)
+        for (int i = begin[c]; i + 1 < begin[c + 1]; ++i)
+            if (chain[i].cols != chain[i + 1].rows) return MOM_ERR_SHAPE_MISMATCH;
+    const int64_t rows = chain[0].rows, cols = chain[begin[1] - 1].cols;
+    for (int c = 1; c < n_chains; ++c)
+        if (chain[begin[c]].rows != rows || chain[begin[c + 1] - 1].cols != cols) return MOM_ERR_SHAPE_MISMATCH;
     for (int i = 0; i < n_add; ++i)
         if (add_terms[i].rows != rows || add_terms[i].cols != cols) return MOM_ERR_SHAPE_MISMATCH;
 
@@ -173,86 +193,132 @@ mom_status_t mom_equation_plan_transposed(const mom_matrix_desc_t *stored_chain,
         if (n_add) p->add.assign(add_terms, add_terms + n_add);
         p->chain_t = chain_t;
         p->add_t = add_t;
+        p->chain_begin = begin;
+        if (names) p->names.assign(names, names + n_chain);
         for (int i = 0; i < n_add; ++i) p->add_flops += nnz(add_terms[i]);
 
-        // identity simplification: A*I -> A, I*A -> A, I*I -> I
-        for (int i = 0; i < n_chain; ++i)
-            if (chain[i].property != MOM_IDENTITY) p->kept.push_back(i);
-        const int r = (int)p->kept.size();
+        int32_t next_id = n_chain;
+        std::map<std::vector<int64_t>, int32_t> seen;       // run of (name, transposed) -> id of its product
+        std::vector<int32_t> summand_props;
 
-        if (r == 0) {
-            p->paren = "I";
-            p->product_desc = mom_matrix_desc_t{rows, cols, MOM_IDENTITY, MOM_F32};
-        } else {
-            // dynamic program over the reduced chain
-            std::vector<Node> node((size_t)r * r);
-            std::vector<uint64_t> cost((size_t)r * r, 0);
-            std::vector<int> split((size_t)r * r, -1);
-            auto at = [r](int i, int j) { return (size_t)i * r + j; };
-            for (int i = 0; i < r; ++i) {
-                const auto &d = chain[p->kept[i]];
-                node[at(i, i)] = Node{d.rows, d.cols, d.property};
-            }
-            for (int len = 2; len <= r; ++len) {
-                for (int i = 0; i + len - 1 < r; ++i) {
-                    const int j = i + len - 1;
-                    bool have = false;
-                    uint64_t best = 0;
-                    int best_k = -1;
-                    for (int k = i; k < j; ++k) {
-                        const Node &a = node[at(i, k)], &b = node[at(k + 1, j)];
-                        uint64_t m;
-                        if (!useful_mults(a.prop, b.prop, a.rows, a.cols, b.cols, &m)) { delete p; return MOM_ERR_OVERFLOW; }
-                        const u128 c = (u128)cost[at(i, k)] + cost[at(k + 1, j)] + m;
-                        if (c >= (u128)COST_LIMIT) { delete p; return MOM_ERR_OVERFLOW; }
-                        if (!have || (uint64_t)c < best) { best = (uint64_t)c; best_k = k; have = true; }
-                    }
-                    cost[at(i, j)] = best;
-                    split[at(i, j)] = best_k;
-                    const Node &a = node[at(i, best_k)], &b = node[at(best_k + 1, j)];
-                    node[at(i, j)] = Node{a.rows, b.cols, join_property(a.prop, b.prop)};
-                }
-            }
-            p->mults = cost[at(0, r - 1)];
+        for (int c = 0; c < n_chains; ++c) {
+            if (c) p->paren += "+";
+            // identity simplification: A*I -> A, I*A -> A, I*I -> I
+            std::vector<int32_t> kept;
+            for (int i = begin[c]; i < begin[c + 1]; ++i)
+                if (chain[i].property != MOM_IDENTITY) kept.push_back(i);
+            p->kept.insert(p->kept.end(), kept.begin(), kept.end());
+            const int r = (int)kept.size();
+            mom_matrix_desc_t value_desc;
 
-            // post-order emission of the binary products; returns the id of the value of [i, j]
-            int32_t next_id = n_chain;
-            struct Emit {
-                mom_plan *p; const std::vector<Node> &node; const std::vector<int> &split; int r; int32_t &next_id;
-                std::string &s;
-                int32_t run(int i, int j) {
-                    if (i == j) {
-                        s += std::to_string(p->kept[i]);
-                        if (p->chain_t[p->kept[i]]) s += "^T";
-                        return p->kept[i];
-                    }
-                    const int k = split[(size_t)i * r + j];
-                    s += "(";
-                    const int32_t l = run(i, k);
-                    s += "*";
-                    const int32_t rr = run(k + 1, j);
-                    s += ")";
-                    const Node &a = node[(size_t)i * r + k], &b = node[(size_t)(k + 1) * r + j], &o = node[(size_t)i * r + j];
-                    mom::StepImpl st;
-                    std::memset(&st.pub, 0, sizeof(st.pub));
-                    st.pub.lhs = l; st.pub.rhs = rr; st.pub.out = next_id++;
-                    st.pub.lhs_property = a.prop; st.pub.rhs_property = b.prop; st.pub.out_property = o.prop;
-                    st.pub.lhs_transposed = l < (int32_t)p->chain.size() && p->chain_t[l];
-                    st.pub.rhs_transposed = rr < (int32_t)p->chain.size() && p->chain_t[rr];
-                    st.pub.m = a.rows; st.pub.k = a.cols; st.pub.n = b.cols;
-                    useful_mults(a.prop, b.prop, a.rows, a.cols, b.cols, &st.pub.useful_mults);
-                    const bool ta = is_tri(a.prop), tb = is_tri(b.prop);
-                    st.pub.kind = !ta && !tb ? MOM_KIND_GG : ta && !tb ? MOM_KIND_TG : !ta && tb ? MOM_KIND_GT
-                                  : a.prop == b.prop ? MOM_KIND_TT : MOM_KIND_TTMIX;
-                    p->steps.push_back(st);
-                    return st.pub.out;
+            if (r == 0) {
+                p->paren += "I";
+                value_desc = mom_matrix_desc_t{rows, cols, MOM_IDENTITY, MOM_F32};
+                p->summands.push_back(mom::Summand{mom::SUM_IDENTITY, 0});
+            } else {
+                // dynamic program over the reduced chain
+                std::vector<Node> node((size_t)r * r);
+                std::vector<uint64_t> cost((size_t)r * r, 0);
+                std::vector<int> split((size_t)r * r, -1);
+                auto at = [r](int i, int j) { return (size_t)i * r + j; };
+                for (int i = 0; i < r; ++i) {
+                    const auto &d = chain[kept[i]];
+                    node[at(i, i)] = Node{d.rows, d.cols, d.property};
                 }
-            } emit{p, node, split, r, next_id, p->paren};
-            emit.run(0, r - 1);
-            const Node &root = node[at(0, r - 1)];
-            p->product_desc = mom_matrix_desc_t{root.rows, root.cols, root.prop, MOM_F32};
+                for (int len = 2; len <= r; ++len) {
+                    for (int i = 0; i + len - 1 < r; ++i) {
+                        const int j = i + len - 1;
+                        bool have = false;
+                        uint64_t best = 0;
+                        int best_k = -1;
+                        for (int k = i; k < j; ++k) {
+                            const Node &a = node[at(i, k)], &b = node[at(k + 1, j)];
+                            uint64_t m;
+                            if (!useful_mults(a.prop, b.prop, a.rows, a.cols, b.cols, &m)) { delete p; return MOM_ERR_OVERFLOW; }
+                            const u128 cst = (u128)cost[at(i, k)] + cost[at(k + 1, j)] + m;
+                            if (cst >= (u128)COST_LIMIT) { delete p; return MOM_ERR_OVERFLOW; }
+                            if (!have || (uint64_t)cst < best) { best = (uint64_t)cst; best_k = k; have = true; }
+                        }
+                        cost[at(i, j)] = best;
+                        split[at(i, j)] = best_k;
+                        const Node &a = node[at(i, best_k)], &b = node[at(best_k + 1, j)];
+                        node[at(i, j)] = Node{a.rows, b.cols, join_property(a.prop, b.prop)};
+                    }
+                }
+
+                // Post-order emission of the binary products; returns the id of the value of [i, j].  A product
+                // below the root whose run of named factors an earlier chain already multiplied (also below its
+                // root) is not emitted again: its id is reused and only its text is written.
+                struct Emit {
+                    mom_plan *p; const std::vector<Node> &node; const std::vector<int> &split; int r; int32_t &next_id;
+                    const std::vector<int32_t> &kept; std::map<std::vector<int64_t>, int32_t> &seen; bool named;
+                    std::string &s;
+                    int32_t run(int i, int j, bool emit) {
+                        if (i == j) {
+                            s += std::to_string(kept[i]);
+                            if (p->chain_t[kept[i]]) s += "^T";
+                            return kept[i];
+                        }
+                        const bool root = i == 0 && j == r - 1;
+                        std::vector<int64_t> key;
+                        int32_t shared = -1;
+                        if (emit && named && !root) {
+                            for (int q = i; q <= j; ++q) key.push_back((int64_t)p->names[kept[q]] * 2 + (p->chain_t[kept[q]] ? 1 : 0));
+                            auto it = seen.find(key);
+                            if (it != seen.end()) { shared = it->second; p->reused += j - i; }
+                        }
+                        const bool emit_here = emit && shared < 0;
+                        const int k = split[(size_t)i * r + j];
+                        s += "(";
+                        const int32_t l = run(i, k, emit_here);
+                        s += "*";
+                        const int32_t rr = run(k + 1, j, emit_here);
+                        s += ")";
+                        if (!emit) return -1;
+                        if (shared >= 0) return shared;
+                        const Node &a = node[(size_t)i * r + k], &b = node[(size_t)(k + 1) * r + j], &o = node[(size_t)i * r + j];
+                        mom::StepImpl st;
+                        std::memset(&st.pub, 0, sizeof(st.pub));
+                        st.pub.lhs = l; st.pub.rhs = rr; st.pub.out = next_id++;
+                        st.pub.lhs_property = a.prop; st.pub.rhs_property = b.prop; st.pub.out_property = o.prop;
+                        st.pub.lhs_transposed = l < (int32_t)p->chain.size() && p->chain_t[l];
+                        st.pub.rhs_transposed = rr < (int32_t)p->chain.size() && p->chain_t[rr];
+                        st.pub.m = a.rows; st.pub.k = a.cols; st.pub.n = b.cols;
+                        useful_mults(a.prop, b.prop, a.rows, a.cols, b.cols, &st.pub.useful_mults);
+                        const bool ta = is_tri(a.prop), tb = is_tri(b.prop);
+                        st.pub.kind = !ta && !tb ? MOM_KIND_GG : ta && !tb ? MOM_KIND_TG : !ta && tb ? MOM_KIND_GT
+                                      : a.prop == b.prop ? MOM_KIND_TT : MOM_KIND_TTMIX;
+                        st.is_last = root;
+                        p->steps.push_back(st);
+                        if (named && !root) seen.emplace(std::move(key), st.pub.out);
+                        return st.pub.out;
+                    }
+                } emit{p, node, split, r, next_id, kept, seen, names != nullptr, p->paren};
+                emit.run(0, r - 1, true);
+                const Node &root = node[at(0, r - 1)];
+                value_desc = mom_matrix_desc_t{root.rows, root.cols, root.prop, MOM_F32};
+                if (r == 1) p->summands.push_back(mom::Summand{mom::SUM_FACTOR, kept[0]});
+                else p->summands.push_back(mom::Summand{mom::SUM_STEP, (int)p->steps.size() - 1});
+            }
+            if (c == 0) p->product_desc = value_desc;
+            else p->add_flops += nnz(value_desc);
+            summand_props.push_back(value_desc.property);
         }
-        p->result_desc = mom_matrix_desc_t{rows, cols, sum_property(p->product_desc.property, p->add), MOM_F32};
+        for (const auto &st : p->steps) {
+            const u128 sum = (u128)p->mults + st.pub.useful_mults;
+            if (sum >= (u128)COST_LIMIT) { delete p; return MOM_ERR_OVERFLOW; }
+            p->mults = (uint64_t)sum;
+        }
+        for (int i = 0; i < n_add; ++i) {
+            p->summands.push_back(mom::Summand{mom::SUM_TERM, i});
+            summand_props.push_back(add_terms[i].property);
+        }
+        p->result_desc = mom_matrix_desc_t{rows, cols, sum_property(summand_props), MOM_F32};
+        {                                               // every root after the first adds to what X holds
+            bool first = true;
+            for (auto &st : p->steps)
+                if (st.is_last) { st.accumulate = !first; first = false; }
+        }
 
         // kernel choice and workspace layout
         const int ns = (int)p->steps.size();
@@ -260,7 +326,6 @@ mom_status_t mom_equation_plan_transposed(const mom_matrix_desc_t *stored_chain,
         items.reserve((size_t)ns * 6);
         for (int s = 0; s < ns; ++s) {
             mom::StepImpl &st = p->steps[s];
-            st.is_last = (s == ns - 1);
             const int64_t m = st.pub.m, n = st.pub.n, k = st.pub.k;
             const bool addressable = (k % 4 == 0) && (n % 4 == 0);
             const bool worth_it = (double)m * (double)n * (double)k >= (double)(1 << 23);
@@ -278,11 +343,11 @@ mom_status_t mom_equation_plan_transposed(const mom_matrix_desc_t *stored_chain,
         for (int s = 0; s < ns; ++s) {
             mom::StepImpl &st = p->steps[s];
             const int64_t m = st.pub.m, n = st.pub.n, k = st.pub.k;
-            int consumer = -1;
+            int consumer = -1, consumers = 0;              // last step that reads this value (a reused product has several)
             for (int t = s + 1; t < ns; ++t)
-                if (p->steps[t].pub.lhs == st.pub.out || p->steps[t].pub.rhs == st.pub.out) { consumer = t; break; }
-            // a tensor-core producer writes a tensor-core consumer's operand planes itself
-            const bool fused_planes = consumer >= 0 && st.pub.uses_tensor_cores && p->steps[consumer].pub.uses_tensor_cores &&
+                if (p->steps[t].pub.lhs == st.pub.out || p->steps[t].pub.rhs == st.pub.out) { consumer = t; ++consumers; }
+            // a tensor-core producer writes its only consumer's operand planes itself when that is a tensor-core step too
+            const bool fused_planes = consumers == 1 && st.pub.uses_tensor_cores && p->steps[consumer].pub.uses_tensor_cores &&
                                       st.split_k == 1;
             if (fused_planes) {
                 mom::StepImpl &c = p->steps[consumer];
@@ -328,7 +393,7 @@ mom_status_t mom_equation_plan_transposed(const mom_matrix_desc_t *stored_chain,
             const int values = n_chain + ns;
             p->fused_value_off.assign(values, -1);
             size_t floats = 0;
-            bool ok = ns >= 1 && ns <= mom::FUSED_MAX_STEPS && (int)p->kept.size() <= mom::FUSED_MAX_OPERANDS &&
+            bool ok = n_chains == 1 && ns >= 1 && ns <= mom::FUSED_MAX_STEPS && (int)p->kept.size() <= mom::FUSED_MAX_OPERANDS &&
                       n_add <= mom::MAX_FUSED_ADD && !any_tc;
             // every value feeds exactly one product: remember on which side
             std::vector<char> is_rhs(values, 0);
@@ -360,6 +425,30 @@ mom_status_t mom_equation_plan_transposed(const mom_matrix_desc_t *stored_chain,
         return MOM_ERR_ALLOC;
     }
     *out_plan = p;
+    return MOM_OK;
+}
+
+mom_status_t mom_equation_plan(const mom_matrix_desc_t *chain, int32_t n_chain,
+                               const mom_matrix_desc_t *add_terms, int32_t n_add,
+                               mom_variant_t variant, mom_plan_t **out_plan) {
+    return mom_equation_plan_transposed(chain, nullptr, n_chain, add_terms, nullptr, n_add, variant, out_plan);
+}
+
+mom_status_t mom_equation_plan_transposed(const mom_matrix_desc_t *stored_chain, const int32_t *chain_transposed, int32_t n_chain,
+                                          const mom_matrix_desc_t *stored_add, const int32_t *add_transposed, int32_t n_add,
+                                          mom_variant_t variant, mom_plan_t **out_plan) {
+    return plan_equation(stored_chain, chain_transposed, nullptr, &n_chain, 1, stored_add, add_transposed, n_add, variant, out_plan);
+}
+
+mom_status_t mom_equation_plan_sum(const mom_matrix_desc_t *factors, const int32_t *factor_transposed,
+                                   const int32_t *factor_names, const int32_t *chain_lengths, int32_t n_chains,
+                                   mom_variant_t variant, mom_plan_t **out_plan) {
+    return plan_equation(factors, factor_transposed, factor_names, chain_lengths, n_chains, nullptr, nullptr, 0, variant, out_plan);
+}
+
+mom_status_t mom_plan_reused_products(const mom_plan_t *plan, int32_t *reused) {
+    if (!plan || !reused) return MOM_ERR_INVALID_ARG;
+    *reused = plan->reused;
     return MOM_OK;
 }
 

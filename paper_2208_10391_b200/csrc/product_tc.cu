@@ -135,7 +135,7 @@ __device__ __forceinline__ void epilogue_chunk(const TcParams &prm, const CUtens
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {
                     if (col0 + 4 * j < prm.n) {
-                        const float4 x = __ldg(src + j);
+                        const float4 x = ((prm.add.aliases_out >> a) & 1u) ? __ldcg(src + j) : __ldg(src + j);
                         v[4 * j] += x.x; v[4 * j + 1] += x.y; v[4 * j + 2] += x.z; v[4 * j + 3] += x.w;
                     }
                 }

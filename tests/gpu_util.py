@@ -89,3 +89,57 @@ def check_against_oracle(eq: wl.Equation, x: np.ndarray, plan, chain, add, rows=
         mask = ov.off_structure_mask(xb.shape[0], xb.shape[1], prop)
         assert np.all(xb.view(np.uint32)[mask] == 0), "off-structure entries must be +0.0f"
     return worst
+
+
+def run_sum_equation(eq: wl.SumEquation, variant: int, use_names: bool = True, poison_out: bool = True):
+    """Plan and evaluate a sum of chains on the GPU; returns (X, plan, per-chain host arrays)."""
+    arrays = wl.generate_sum(eq)
+    plan = mom.mom_equation_plan_sum(eq.descs(), eq.transposed, eq.names if use_names else None, variant)
+    rd = plan.result_desc()
+    n_out = rd.rows * rd.cols
+    stream = torch.cuda.current_stream().cuda_stream
+    dev = {}
+    ptrs = []
+    for chain, names in zip(arrays, eq.names):
+        for a, nm in zip(chain, names):
+            if a is None:
+                ptrs.append(None)
+                continue
+            if nm not in dev:
+                dev[nm] = torch.from_numpy(a).cuda()
+            ptrs.append(dev[nm].data_ptr())
+    ws_bytes = plan.workspace_bytes(1)
+    ws = torch.empty(max(ws_bytes, 256), dtype=torch.uint8, device="cuda")
+    guarded = torch.full((n_out + 2 * CANARY,), float("nan") if poison_out else 7.0, dtype=torch.float32, device="cuda")
+    guarded[:CANARY] = 12345.0
+    guarded[-CANARY:] = 12345.0
+    out = guarded[CANARY:CANARY + n_out]
+    plan.execute(ptrs, [], out.data_ptr(), ws.data_ptr() if ws_bytes else None, ws_bytes, stream)
+    torch.cuda.synchronize()
+    assert plan.device_status() == (0, 0), "a device-side wait timed out"
+    g = guarded.cpu().numpy()
+    assert np.all(g[:CANARY] == 12345.0) and np.all(g[-CANARY:] == 12345.0), "wrote outside the output buffer"
+    return g[CANARY:CANARY + n_out].reshape(rd.rows, rd.cols).copy(), plan, arrays
+
+
+def check_sum_against_oracle(eq: wl.SumEquation, x: np.ndarray, plan, arrays, use_names: bool = True, rows=None,
+                             tol: float = TOL):
+    want = op.plan_sum(eq.descs(), eq.transposed, eq.names if use_names else ())
+    assert plan.parenthesization() == want.paren
+    assert plan.flops() == (want.mul_flops, want.add_flops)
+    assert plan.reused_products() == want.reused
+    prop = plan.result_desc().property
+    assert prop == want.result_desc.prop
+    assert not np.isnan(x).any(), "part of the output was never written"
+    used_a, used_d = [], []
+    for chain, descs, flags in zip(arrays, eq.descs(), eq.transposed):
+        a, d = ov.transposed_operands(chain, descs, flags)
+        used_a.append(a)
+        used_d.append(d)
+    x_ref, den = ov.evaluate_sum(used_a, used_d, rows=rows)
+    got = x if rows is None else x[rows]
+    err = ov.normwise_error(got, x_ref, den)
+    assert err <= tol, f"normwise error {err:.3e} > {tol:.1e} ({eq.name})"
+    mask = ov.off_structure_mask(x.shape[0], x.shape[1], prop)
+    assert np.all(x.view(np.uint32)[mask] == 0), "off-structure entries must be +0.0f"
+    return err

@@ -159,3 +159,68 @@ def test_transposed_operands_match_the_oracle():
         mom.mom_equation_plan_transposed([(7, 30, 0), (7, 40, 0)], [False, False])
     assert e.value.status == mom.ERR_SHAPE_MISMATCH
     assert mom.mom_equation_plan_transposed([(7, 30, 0), (7, 40, 0)], [True, False]).result_desc().rows == 30
+
+
+# ---- sums of several chains ---------------------------------------------------------------------------
+
+def assert_same_sum_plan(chains, transposed=None, names=None, variant=mom.VARIANT_3XTF32):
+    want = op.plan_sum(chains, transposed or (), names or ())
+    got = mom.mom_equation_plan_sum(chains, transposed, names, variant)
+    assert got.parenthesization() == want.paren
+    assert got.flops() == (want.mul_flops, want.add_flops)
+    assert got.reused_products() == want.reused
+    rd = got.result_desc()
+    assert (rd.rows, rd.cols, rd.property) == (want.result_desc.rows, want.result_desc.cols, want.result_desc.prop)
+    steps = got.steps()
+    assert len(steps) == len(want.steps)
+    for g, w in zip(steps, want.steps):
+        assert (g.lhs, g.rhs, g.out, g.m, g.n, g.k) == (w.lhs, w.rhs, w.out, w.m, w.n, w.k)
+        assert (g.lhs_property, g.rhs_property, g.out_property, g.useful_mults) == (w.lhs_prop, w.rhs_prop, w.out_prop, w.mults)
+    return got, want
+
+
+def test_random_sums_of_chains_match_the_oracle():
+    shared = 0
+    for seed in range(400):
+        eq = wl.random_sum_equation(seed)
+        got, want = assert_same_sum_plan(eq.descs(), eq.transposed, eq.names)
+        shared += want.reused > 0
+        assert_same_sum_plan(eq.descs(), eq.transposed, None)        # nothing known to be shared
+    assert shared >= 20
+
+
+def test_sum_plan_shares_a_product_between_chains():
+    G = mom.GENERAL
+    a, b, c = (8, 50, G), (50, 8, G), (8, 100, G)
+    got, want = assert_same_sum_plan([[a, b, c], [a, b, c]], None, [[0, 1, 2], [0, 1, 3]])
+    assert got.reused_products() == 1 and got.num_steps() == 3
+    assert got.parenthesization() == "((0*1)*2)+((3*4)*5)"
+    # a shared run of three factors saves its two products
+    d = (100, 7, G)
+    got, _ = assert_same_sum_plan([[a, b, a, (50, 300, G)], [a, b, a, (50, 300, G)]], None, [[0, 1, 0, 2], [0, 1, 0, 3]])
+    assert got.reused_products() >= 1
+
+
+def test_sum_plan_of_one_chain_equals_the_chain_plan():
+    for seed in range(60):
+        eq = wl.random_equation(seed, max_len=7, max_dim=40, allow_add=False)
+        one = mom.mom_equation_plan(eq.descs())
+        many = mom.mom_equation_plan_sum([eq.descs()])
+        assert one.parenthesization() == many.parenthesization() and one.flops() == many.flops()
+
+
+@pytest.mark.parametrize("chains,names,status,code", [
+    ([], None, mom.ERR_INVALID_ARG, "invalid_arg"),
+    ([[(4, 5, 0)], [(5, 4, 0)]], None, mom.ERR_SHAPE_MISMATCH, "shape_mismatch"),
+    ([[(4, 5, 0), (4, 5, 0)]], None, mom.ERR_SHAPE_MISMATCH, "shape_mismatch"),
+    ([[(4, 4, 0)], [(4, 4, 1)]], [[0], [0]], mom.ERR_INVALID_ARG, "invalid_arg"),
+    ([[(4, 4, 0)], []], None, mom.ERR_INVALID_ARG, None),
+])
+def test_sum_plan_errors(chains, names, status, code):
+    with pytest.raises(mom.MomError) as e:
+        mom.mom_equation_plan_sum(chains, None, names)
+    assert e.value.status == status
+    if code is not None:
+        with pytest.raises(op.OracleError) as oe:
+            op.plan_sum(chains, (), names or ())
+        assert oe.value.code == code

@@ -216,3 +216,111 @@ def random_equation(seed: int, max_len: int = 6, max_dim: int = 96, allow_add: b
 
 def with_batch(eq: Equation, batch: int) -> Equation:
     return replace(eq, batch=batch, name=f"{eq.name}_x{batch}")
+
+
+# --------------------------------------------------------------------------
+# Sums of several Mul chains (paper Section 2, "Operations": Mul and Add are
+# variadic and one Equation holds a bag of them).
+# --------------------------------------------------------------------------
+
+@dataclass(frozen=True)
+class SumEquation:
+    """X = prod(chains[0]) + prod(chains[1]) + ...; a chain of one factor is a plain Add term.
+
+    names[c][f] identifies the stored matrix behind factor f of chain c: equal names mean the same
+    matrix (drawn once, keyed by its name); transposed[c][f] says the factor enters transposed.
+    """
+    name: str
+    seed: int
+    chains: Sequence[Sequence[Operand]]
+    transposed: Sequence[Sequence[bool]]
+    names: Sequence[Sequence[int]]
+
+    def descs(self):
+        return [[(o.rows, o.cols, o.prop) for o in chain] for chain in self.chains]
+
+
+def generate_sum(eq: SumEquation):
+    """Per chain, per factor: the stored float32 array (None for Identity); one array object per name."""
+    by_name = {}
+    out = []
+    for chain, names in zip(eq.chains, eq.names):
+        row = []
+        for o, nm in zip(chain, names):
+            if nm not in by_name:
+                by_name[nm] = generate_operand(o, eq.seed, nm)
+            row.append(by_name[nm])
+        out.append(row)
+    return out
+
+
+def random_sum_equation(seed: int, max_chains: int = 4, max_len: int = 5, max_dim: int = 48,
+                        dim_multiple: int = 1, share: float = 0.5) -> SumEquation:
+    """Random well-formed sum of chains.  With probability `share`/2 a chain starts with a run of factors
+    copied (same names and flags) from an earlier chain, so that shared products occur."""
+    rng = np.random.Generator(np.random.Philox(key=[int(seed), 0x5EED5]))
+    rows = int(rng.integers(1, max_dim // dim_multiple + 1)) * dim_multiple
+    cols = int(rng.integers(1, max_dim // dim_multiple + 1)) * dim_multiple
+    if rng.random() < 0.4:
+        cols = rows
+    chains, flags, names = [], [], []
+    next_name = 0
+
+    def new_factor(r, c):
+        nonlocal next_name
+        """One stored factor whose type AS USED is r x c, with a random property and transposition."""
+        kind = int(rng.integers(0, 7))
+        t = bool(rng.integers(0, 3) == 0)
+        if r == c and kind == 0:
+            o = Operand(r, r, LOWER_TRI)
+        elif r == c and kind == 1:
+            o = Operand(r, r, UPPER_TRI)
+        elif r == c and kind == 2:
+            o = Operand(r, r, IDENTITY)
+        else:
+            o = Operand(c, r, GENERAL) if t else Operand(r, c, GENERAL)
+        nm = next_name
+        next_name += 1
+        return o, t, nm
+
+    def used_shape(o, t):
+        return (o.cols, o.rows) if t else (o.rows, o.cols)
+
+    for c in range(int(rng.integers(1, max_chains + 1))):
+        length = int(rng.integers(1, max_len + 1))
+        ops, ts, nms = [], [], []
+        if chains and rng.random() < share:
+            src = int(rng.integers(0, len(chains)))
+            take = int(rng.integers(1, len(chains[src]) + 1))
+            if rng.random() < 0.5:                         # copy a prefix: its first factor has `rows` rows
+                ops, ts, nms = list(chains[src][:take]), list(flags[src][:take]), list(names[src][:take])
+        cur = used_shape(ops[-1], ts[-1])[1] if ops else rows
+        while len(ops) < length - 1 or not ops:
+            last = len(ops) >= length - 1
+            nxt = cols if last else int(rng.integers(1, max_dim // dim_multiple + 1)) * dim_multiple
+            if not last and rng.random() < 0.4:
+                nxt = cur
+            o, t, nm = new_factor(cur, nxt)
+            ops.append(o); ts.append(t); nms.append(nm)
+            cur = nxt
+        if cur != cols:                                    # a copied prefix that does not end on `cols`
+            o, t, nm = new_factor(cur, cols)
+            ops.append(o); ts.append(t); nms.append(nm)
+        chains.append(tuple(ops)); flags.append(tuple(ts)); names.append(tuple(nms))
+    return SumEquation(f"random_sum_{seed}", seed, tuple(chains), tuple(flags), tuple(names))
+
+
+def config_sum_shared(n: int = 4096, seed: int = 7) -> SumEquation:
+    """X = A*B*C + A*B*D, all general n x n: every tree ties, the left-nested one is taken, and A*B is
+    below the root in both chains, so it is multiplied once (3 products instead of 4)."""
+    g = Operand(n, n, GENERAL, "normal", 1.0 / np.sqrt(n))
+    return SumEquation(f"ABC_plus_ABD_{n}", seed, ((g, g, g), (g, g, g)), ((False,) * 3, (False,) * 3),
+                       ((0, 1, 2), (0, 1, 3)))
+
+
+def config_sum_triangular(n: int = 4096, seed: int = 8) -> SumEquation:
+    """X = L*A + B*U + C: L lowerTri, U upperTri, A, B, C general n x n."""
+    g = Operand(n, n, GENERAL, "normal", 1.0 / np.sqrt(n))
+    return SumEquation(f"LA_plus_BU_plus_C_{n}", seed,
+                       ((Operand(n, n, LOWER_TRI), g), (g, Operand(n, n, UPPER_TRI)), (g,)),
+                       ((False, False), (False, False), (False,)), ((0, 1), (2, 3), (4,)))
