@@ -213,10 +213,23 @@ class ClockSampler:
 
 def time_equation(mom, torch, eq, variant, steps, warmup, stream, timing=False):
     """Device-resident timing of one configuration: returns dict with per-step ms list, plan, launches."""
-    chain, add = wl.generate(eq)
-    plan = mom.mom_equation_plan_transposed(eq.descs(), eq.chain_t, eq.add_descs(), eq.add_t, variant)
+    if isinstance(eq, wl.SumEquation):
+        # a sum of chains: one device array per named matrix, one pointer per factor
+        arrays = wl.generate_sum(eq)
+        plan = mom.mom_equation_plan_sum(eq.descs(), eq.transposed, eq.names, variant)
+        by_name = {}
+        for row, names in zip(arrays, eq.names):
+            for a, nm in zip(row, names):
+                if a is not None and nm not in by_name:
+                    by_name[nm] = torch.from_numpy(a).cuda()
+        dchain = [None if a is None else by_name[nm] for row, names in zip(arrays, eq.names) for a, nm in zip(row, names)]
+        chain, add = [a for row in arrays for a in row], []
+        eq = wl.Equation(eq.name, eq.seed, tuple(o for c in eq.chains for o in c))     # batch 1, for the code below
+    else:
+        chain, add = wl.generate(eq)
+        plan = mom.mom_equation_plan_transposed(eq.descs(), eq.chain_t, eq.add_descs(), eq.add_t, variant)
+        dchain = [None if a is None else torch.from_numpy(a).cuda() for a in chain]
     rd = plan.result_desc()
-    dchain = [None if a is None else torch.from_numpy(a).cuda() for a in chain]
     dadd = [None if a is None else torch.from_numpy(a).cuda() for a in add]
     out = torch.empty((eq.batch, rd.rows, rd.cols), dtype=torch.float32, device="cuda")
     wsb = plan.workspace_bytes(eq.batch)
@@ -287,9 +300,10 @@ def run_gpu(args):
         # one named configuration, nothing else: the small case for profiler captures
         cfgs = {c.name: c for c in (wl.config_tiny(), wl.config_five_general(), wl.config_property_heavy(),
                                     wl.config_large_square(), wl.config_batched(), wl.config_paper_chain(),
-                                    wl.config_transposed())}
+                                    wl.config_transposed(), wl.config_sum_shared(), wl.config_sum_triangular())}
         cfg = cfgs[args.only]
-        r = time_equation(mom, torch, cfg, variant, steps=args.steps, warmup=args.warmup, stream=stream, timing=cfg.batch == 1)
+        r = time_equation(mom, torch, cfg, variant, steps=args.steps, warmup=args.warmup, stream=stream,
+                          timing=getattr(cfg, "batch", 1) == 1)
         print(json.dumps({"workload": cfg.name, "variant": args.variant, "ms": r["ms"], "useful_flops": r["useful_flops"],
                           "launches": r["launches"], "step_times_ms": r["step_times"][-1:] }))
         return
@@ -421,8 +435,9 @@ def run_gpu(args):
         # ---- the other configurations, briefly (min of 5 as in the paper's Section 4, and the median)
         others = []
         for cfg in (wl.config_tiny(), wl.config_five_general(), wl.config_property_heavy(), wl.config_batched(),
-                    wl.config_paper_chain(), wl.config_transposed()):
-            r = time_equation(mom, torch, cfg, variant, steps=20, warmup=3, stream=stream, timing=cfg.batch == 1)
+                    wl.config_paper_chain(), wl.config_transposed(), wl.config_sum_shared(), wl.config_sum_triangular()):
+            batch = getattr(cfg, "batch", 1)
+            r = time_equation(mom, torch, cfg, variant, steps=20, warmup=3, stream=stream, timing=batch == 1)
             ms_min, ms_med = min(r["ms"]), statistics.median(r["ms"])
             entry = {"workload": cfg.name, "parenthesization": r["plan"].parenthesization(),
                      "useful_flops": r["useful_flops"], "ms_min_of_20": ms_min, "ms_median": ms_med,
@@ -430,7 +445,7 @@ def run_gpu(args):
                      "gflops_at_median": r["useful_flops"] / (ms_med * 1e-3) / 1e9,
                      "frac_of_roofline_at_median": r["useful_flops"] / (ms_med * 1e-3) / 1e12 / peak,
                      "launches": r["launches"]}
-            if cfg.batch > 1:
+            if batch > 1:
                 per_inst = sum(o.rows * o.cols for o in list(cfg.chain) + list(cfg.add)) + rd_elems(r["plan"])
                 entry["hbm_gbs_at_median"] = per_inst * 4 * cfg.batch / (ms_med * 1e-3) / 1e9
                 entry["hbm_frac_of_measured_peak"] = entry["hbm_gbs_at_median"] / peaks["hbm_gbs"]

@@ -138,7 +138,7 @@ class Plan:
         self.destroy()
 
     def destroy(self) -> None:
-        if getattr(self, "_h", None) is not None and self._h.value:
+        if getattr(self, "_h", None) is not None and self._h.value and _lib is not None:   # None at interpreter exit
             _lib.mom_plan_destroy(self._h)
             self._h = _P(None)
 

@@ -6,6 +6,7 @@
 #include <map>
 #include <new>
 #include <string>
+#include <utility>
 #include <vector>
 
 #include "fused_small.h"
@@ -340,43 +341,79 @@ static mom_status_t plan_equation(const mom_matrix_desc_t *stored_chain, const i
                 }
             }
         }
+        // f32 intermediates, or planes written by the producer: a tensor-core producer writes its consumers' operand
+        // planes itself when every consumer is a tensor-core step that takes the value on the same side
         for (int s = 0; s < ns; ++s) {
             mom::StepImpl &st = p->steps[s];
-            const int64_t m = st.pub.m, n = st.pub.n, k = st.pub.k;
-            int consumer = -1, consumers = 0;              // last step that reads this value (a reused product has several)
-            for (int t = s + 1; t < ns; ++t)
-                if (p->steps[t].pub.lhs == st.pub.out || p->steps[t].pub.rhs == st.pub.out) { consumer = t; ++consumers; }
-            // a tensor-core producer writes its only consumer's operand planes itself when that is a tensor-core step too
-            const bool fused_planes = consumers == 1 && st.pub.uses_tensor_cores && p->steps[consumer].pub.uses_tensor_cores &&
-                                      st.split_k == 1;
-            if (fused_planes) {
-                mom::StepImpl &c = p->steps[consumer];
-                if (c.pub.lhs == st.pub.out) { st.planes_out = 1; c.a_planes_ready = true; }
-                else { st.planes_out = 2; c.b_planes_ready = true; }
-            } else if (!st.is_last) {
-                items.push_back(Interval{mom::align_up((size_t)m * n * sizeof(float), mom::WS_ALIGN), s, consumer < 0 ? ns - 1 : consumer, &st.out_off, 0});
+            const int64_t m = st.pub.m, n = st.pub.n;
+            int last_consumer = -1, as_lhs = 0, as_rhs = 0;   // a product shared between chains has several consumers
+            bool all_tc = true;
+            for (int t = s + 1; t < ns; ++t) {
+                const mom::StepImpl &c = p->steps[t];
+                if (c.pub.lhs != st.pub.out && c.pub.rhs != st.pub.out) continue;
+                last_consumer = t;
+                (c.pub.lhs == st.pub.out ? as_lhs : as_rhs)++;
+                all_tc &= c.pub.uses_tensor_cores != 0;
             }
-            if (st.pub.uses_tensor_cores) {
-                const size_t ab = mom::align_up((size_t)m * k * sizeof(float), mom::WS_ALIGN);
-                const size_t bb = mom::align_up((size_t)k * n * sizeof(float), mom::WS_ALIGN);
-                // planes written by an earlier step live from that step on
-                int a_from = s, b_from = s;
-                for (int t = 0; t < s; ++t) {
-                    if (p->steps[t].pub.out == st.pub.lhs && st.a_planes_ready) a_from = t;
-                    if (p->steps[t].pub.out == st.pub.rhs && st.b_planes_ready) b_from = t;
+            const bool fused_planes = last_consumer >= 0 && all_tc && (as_lhs == 0 || as_rhs == 0) &&
+                                      st.pub.uses_tensor_cores && st.split_k == 1;
+            if (fused_planes) {
+                st.planes_out = as_lhs ? 1 : 2;
+            } else if (!st.is_last) {
+                items.push_back(Interval{mom::align_up((size_t)m * n * sizeof(float), mom::WS_ALIGN), s,
+                                         last_consumer < 0 ? ns - 1 : last_consumer, &st.out_off, 0});
+            }
+        }
+        // Operand planes of the tensor-core steps.  Steps that take the same value on the same side (a shared
+        // product; a named factor with the same transposition) read one set of planes: the first of them owns
+        // the buffers, which then live until the last, and the others skip their split pass.
+        struct Shared { int owner; size_t hi_item, lo_item; };
+        std::map<std::pair<int64_t, int>, Shared> plane_sets;       // (value, side) -> owner
+        struct Copy { int step, side, owner; };
+        std::vector<Copy> copies;
+        for (int s = 0; s < ns; ++s) {
+            mom::StepImpl &st = p->steps[s];
+            if (!st.pub.uses_tensor_cores) continue;
+            const int64_t m = st.pub.m, n = st.pub.n, k = st.pub.k;
+            for (int side = 0; side < 2; ++side) {
+                const int32_t v = side == 0 ? st.pub.lhs : st.pub.rhs;
+                const size_t bytes = mom::align_up((size_t)(side == 0 ? m * k : k * n) * sizeof(float), mom::WS_ALIGN);
+                size_t *hi = side == 0 ? &st.a_hi_off : &st.b_hi_off, *lo = side == 0 ? &st.a_lo_off : &st.b_lo_off;
+                bool &ready = side == 0 ? st.a_planes_ready : st.b_planes_ready;
+                int from = s;
+                int64_t key = -1;                                    // -1: nothing to share with
+                if (v >= n_chain) {
+                    const int producer = v - n_chain;
+                    key = (int64_t)v << 1;
+                    if (p->steps[producer].planes_out) { from = producer; ready = true; }
+                } else if (names) {
+                    key = (((int64_t)names[v] << 1) | (chain_t[v] ? 1 : 0)) | ((int64_t)1 << 62);
                 }
-                items.push_back(Interval{ab, a_from, s, &st.a_hi_off, 0});
-                items.push_back(Interval{ab, a_from, s, &st.a_lo_off, 0});
-                items.push_back(Interval{bb, b_from, s, &st.b_hi_off, 0});
-                items.push_back(Interval{bb, b_from, s, &st.b_lo_off, 0});
-                if (st.split_k > 1) {
-                    const size_t slab_rows = (size_t)((m + mom::TC_BM - 1) / mom::TC_BM * mom::TC_BM);
-                    items.push_back(Interval{mom::align_up((size_t)st.split_k * slab_rows * n * sizeof(float), mom::WS_ALIGN), s, s, &st.partial_off, 0});
+                auto it = key >= 0 ? plane_sets.find({key, side}) : plane_sets.end();
+                if (it != plane_sets.end()) {
+                    items[it->second.hi_item].last = s;
+                    items[it->second.lo_item].last = s;
+                    copies.push_back(Copy{s, side, it->second.owner});
+                    ready = true;
+                    continue;
                 }
+                items.push_back(Interval{bytes, from, s, hi, 0});
+                items.push_back(Interval{bytes, from, s, lo, 0});
+                if (key >= 0) plane_sets[{key, side}] = Shared{s, items.size() - 2, items.size() - 1};
+            }
+            if (st.split_k > 1) {
+                const size_t slab_rows = (size_t)((m + mom::TC_BM - 1) / mom::TC_BM * mom::TC_BM);
+                items.push_back(Interval{mom::align_up((size_t)st.split_k * slab_rows * n * sizeof(float), mom::WS_ALIGN), s, s, &st.partial_off, 0});
             }
         }
         p->workspace_per_instance = pack(items);
-        for (int s = 0; s < ns; ++s) {                  // a producer's plane targets are its consumer's operand planes
+        for (const Copy &c : copies) {
+            mom::StepImpl &st = p->steps[c.step];
+            const mom::StepImpl &o = p->steps[c.owner];
+            if (c.side == 0) { st.a_hi_off = o.a_hi_off; st.a_lo_off = o.a_lo_off; }
+            else { st.b_hi_off = o.b_hi_off; st.b_lo_off = o.b_lo_off; }
+        }
+        for (int s = 0; s < ns; ++s) {                  // a producer's plane targets are its consumers' operand planes
             mom::StepImpl &st = p->steps[s];
             if (!st.planes_out) continue;
             for (int t = s + 1; t < ns; ++t) {

@@ -157,3 +157,15 @@ def test_sum_configurations_full_size_sampled_rows(eq):
     rows = np.random.default_rng(5).choice(x.shape[0], size=24, replace=False)
     rows = np.sort(np.concatenate([rows, [0, x.shape[0] - 1]]))
     check_sum_against_oracle(eq, x, plan, arrays, rows=rows)
+
+
+@pytest.mark.parametrize("variant", [mom.VARIANT_3XTF32, mom.VARIANT_3XTF32_FORCE])
+def test_named_factor_on_both_sides_and_in_both_orientations(variant):
+    # A is the left operand twice (one set of planes), the right operand once and enters transposed once
+    n = 392
+    a, g, l = (n, n, G), (n, n, G), (n, n, L)
+    eq = sum_eq("factor_reuse", [[a, g], [a, l], [g, a], [a, g], [l, a]],
+                transposed=((False, False), (False, False), (False, False), (True, False), (False, True)),
+                names=((0, 1), (0, 2), (3, 0), (0, 4), (2, 0)))
+    x, plan, arrays = run_sum_equation(eq, variant)
+    check_sum_against_oracle(eq, x, plan, arrays)

@@ -311,11 +311,11 @@ def random_sum_equation(seed: int, max_chains: int = 4, max_len: int = 5, max_di
 
 
 def config_sum_shared(n: int = 4096, seed: int = 7) -> SumEquation:
-    """X = A*B*C + A*B*D, all general n x n: every tree ties, the left-nested one is taken, and A*B is
+    """X = C*A*B + D*A*B, all general n x n: every tree ties, the right-nested one is taken, and A*B is
     below the root in both chains, so it is multiplied once (3 products instead of 4)."""
     g = Operand(n, n, GENERAL, "normal", 1.0 / np.sqrt(n))
-    return SumEquation(f"ABC_plus_ABD_{n}", seed, ((g, g, g), (g, g, g)), ((False,) * 3, (False,) * 3),
-                       ((0, 1, 2), (0, 1, 3)))
+    return SumEquation(f"CAB_plus_DAB_{n}", seed, ((g, g, g), (g, g, g)), ((False,) * 3, (False,) * 3),
+                       ((2, 0, 1), (3, 0, 1)))
 
 
 def config_sum_triangular(n: int = 4096, seed: int = 8) -> SumEquation:
