@@ -420,3 +420,115 @@ def plan_sum(chains: Sequence[Sequence[Tuple[int, int, int]]],
     add_flops = sum(structural_nonzeros(d) for d in descs[1:])
     return SumPlan("+".join(parens), mults, 2 * mults, add_flops, tuple(steps), tuple(values), descs,
                    Desc(rows, cols, result_prop), reused)
+
+
+# ----------------------------------------------------------------------------------------------
+# nested expressions
+# ----------------------------------------------------------------------------------------------
+# Paper Section 2, "Operations": the body of an Equation is a bag of Mul, Add and Transpose operations
+# that is walked from the yield, so Mul and Add may nest:  A*(B + C),  (A + B)^T * C,  ...
+# An expression is written here as a nested Python value:
+#     int i                     operand i of the operand table
+#     ("t", e)                  transpose of e
+#     ("mul", [e1, e2, ...])    product, left to right
+#     ("add", [e1, e2, ...])    sum
+# Readings (the paper gives no rule for any of this):
+#   * transposes are pushed down to the operands: (e1*e2)^T = e2^T*e1^T, (e1+e2)^T = e1^T+e2^T, (e^T)^T = e;
+#   * a product inside a product and a sum inside a sum are flattened (associativity);
+#   * a sum inside a product is MATERIALIZED: it is evaluated on its own (as a sum of chains, see `plan_sum`)
+#     into a temporary whose type is the sum's result type, and the temporary is one factor of the outer
+#     chain.  Nothing is distributed: A*(B+C) costs one product and one addition;
+#   * two nested sums with the same normal form are the same temporary, evaluated once;
+#   * sharing of products (`plan_sum`) works within one sum; operands are named by their index, a temporary
+#     by its normal form;
+#   * nested sums are planned before the sum that uses them, in order of first appearance;
+#   * in the string an operand prints as its index (with ^T), a temporary as [its sum's string].
+
+@dataclass(frozen=True)
+class ExprPlan:
+    paren: str
+    mults: int
+    mul_flops: int
+    add_flops: int
+    result_desc: Desc
+    products: Tuple[Tuple[int, int, int, int, int, int, int], ...]   # (m, n, k, lhs_prop, rhs_prop, out_prop, mults) in order
+    reused: int
+    temporaries: int       # distinct nested sums that were materialized
+
+
+def normalize_expr(expr, transposed: bool = False):
+    """Normal form: a sum = tuple of chains; a chain = tuple of factors; a factor = ("leaf", operand, t) or
+    ("sum", <normal form of the nested sum>)."""
+    if isinstance(expr, int):
+        return ((("leaf", expr, transposed),),)
+    kind = expr[0]
+    if kind == "t":
+        return normalize_expr(expr[1], not transposed)
+    children = list(expr[1])
+    if not children:
+        raise OracleError("invalid_arg", "operation without operands")
+    if kind == "add":
+        out = []
+        for c in children:
+            out.extend(normalize_expr(c, transposed))
+        return tuple(out)
+    if kind == "mul":
+        if transposed:
+            children.reverse()
+        chain = []
+        for c in children:
+            s = normalize_expr(c, transposed)
+            if len(s) == 1:
+                chain.extend(s[0])
+            else:
+                chain.append(("sum", s))
+        return (tuple(chain),)
+    raise OracleError("invalid_arg", f"unknown operation {kind!r}")
+
+
+def plan_expr(expr, operands: Sequence[Tuple[int, int, int]]) -> ExprPlan:
+    stored = [Desc(*d) for d in operands]
+    temporaries = {}                  # normal form -> (name, result Desc, string)
+    products: List[Tuple[int, ...]] = []
+    totals = {"mults": 0, "add": 0, "reused": 0}
+
+    def plan_one(sum_nf) -> Tuple[Desc, str]:
+        chains, flags, names, labels = [], [], [], []
+        for chain in sum_nf:
+            cd, cf, cn, cl = [], [], [], []
+            for f in chain:
+                if f[0] == "leaf":
+                    _, i, t = f
+                    if not 0 <= i < len(stored):
+                        raise OracleError("invalid_arg", "operand index out of range")
+                    cd.append(tuple(operands[i])); cf.append(t); cn.append(i); cl.append(str(i))
+                else:
+                    nf = f[1]
+                    if nf not in temporaries:
+                        desc, text = plan_one(nf)
+                        temporaries[nf] = (len(stored) + len(temporaries), desc, text)
+                    name, desc, text = temporaries[nf]
+                    cd.append((desc.rows, desc.cols, desc.prop)); cf.append(False); cn.append(name)
+                    cl.append("[" + text + "]")
+            chains.append(cd); flags.append(cf); names.append(cn); labels.extend(cl)
+        sp = plan_sum(chains, flags, names)
+        totals["mults"] += sp.mults
+        totals["add"] += sp.add_flops
+        totals["reused"] += sp.reused
+        products.extend((s.m, s.n, s.k, s.lhs_prop, s.rhs_prop, s.out_prop, s.mults) for s in sp.steps)
+        # positions -> labels
+        out, num = [], ""
+        for ch in sp.paren + "\0":
+            if ch.isdigit():
+                num += ch
+                continue
+            if num:
+                out.append(labels[int(num)])
+                num = ""
+            if ch != "\0":
+                out.append(ch)
+        return sp.result_desc, "".join(out)
+
+    desc, text = plan_one(normalize_expr(expr))
+    return ExprPlan(text, totals["mults"], 2 * totals["mults"], totals["add"], desc, tuple(products),
+                    totals["reused"], len(temporaries))

@@ -157,6 +157,37 @@ def evaluate_sum(chains: Sequence[Sequence[Optional[np.ndarray]]],
     return x, d
 
 
+def evaluate_expr(expr, arrays: Sequence[Optional[np.ndarray]], descs: Sequence[Tuple[int, int, int]],
+                  threads: Optional[int] = None) -> Tuple[np.ndarray, np.ndarray]:
+    """(X_ref, D) of a nested expression, by its plain definition (paper Section 2, "Operations": Mul, Add
+    and Transpose inside one Equation).  `expr` is an operand index, ("t", e), ("mul", [e...]) or
+    ("add", [e...]); operands are the stored matrices.  A product is multiplied left to right with the
+    fp64 triple loop, a sum is added left to right, a transpose is NumPy's.  D follows the same recursion
+    on absolute values: D(operand) = |A|, D(product) = product of the D's, D(sum) = sum of the D's.
+    """
+    def walk(e):
+        if isinstance(e, int):
+            a = dense(arrays[e], descs[e])
+            return a, np.abs(a)
+        kind = e[0]
+        if kind == "t":
+            x, d = walk(e[1])
+            return np.ascontiguousarray(x.T), np.ascontiguousarray(d.T)
+        parts = [walk(c) for c in e[1]]
+        x, d = parts[0]
+        for xc, dc in parts[1:]:
+            if kind == "mul":
+                x, d = matmul(x, xc, threads), matmul(d, dc, threads)
+            elif kind == "add":
+                x, d = x + xc, d + dc
+            else:
+                raise ValueError(f"unknown operation {kind!r}")
+        return x, d
+
+    x, d = walk(expr)
+    return np.array(x, dtype=np.float64, copy=True), np.array(d, dtype=np.float64, copy=True)
+
+
 def evaluate_steps(chain: Sequence[Optional[np.ndarray]], chain_descs: Sequence[Tuple[int, int, int]],
                    steps, add: Sequence[Optional[np.ndarray]] = (),
                    add_descs: Sequence[Tuple[int, int, int]] = (), threads: Optional[int] = None) -> np.ndarray:
