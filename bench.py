@@ -213,7 +213,13 @@ class ClockSampler:
 
 def time_equation(mom, torch, eq, variant, steps, warmup, stream, timing=False):
     """Device-resident timing of one configuration: returns dict with per-step ms list, plan, launches."""
-    if isinstance(eq, wl.SumEquation):
+    if isinstance(eq, wl.Expression):
+        # a nested expression: one pointer per operand of the table
+        chain, add = wl.generate_expression(eq), []
+        plan = mom.mom_expression_plan(eq.expr, eq.descs(), variant)
+        dchain = [None if a is None else torch.from_numpy(a).cuda() for a in chain]
+        eq = wl.Equation(eq.name, eq.seed, tuple(eq.operands))                          # batch 1, for the code below
+    elif isinstance(eq, wl.SumEquation):
         # a sum of chains: one device array per named matrix, one pointer per factor
         arrays = wl.generate_sum(eq)
         plan = mom.mom_equation_plan_sum(eq.descs(), eq.transposed, eq.names, variant)
@@ -300,7 +306,8 @@ def run_gpu(args):
         # one named configuration, nothing else: the small case for profiler captures
         cfgs = {c.name: c for c in (wl.config_tiny(), wl.config_five_general(), wl.config_property_heavy(),
                                     wl.config_large_square(), wl.config_batched(), wl.config_paper_chain(),
-                                    wl.config_transposed(), wl.config_sum_shared(), wl.config_sum_triangular())}
+                                    wl.config_transposed(), wl.config_sum_shared(), wl.config_sum_triangular(),
+                                    wl.config_expression())}
         cfg = cfgs[args.only]
         r = time_equation(mom, torch, cfg, variant, steps=args.steps, warmup=args.warmup, stream=stream,
                           timing=getattr(cfg, "batch", 1) == 1)
@@ -435,7 +442,8 @@ def run_gpu(args):
         # ---- the other configurations, briefly (min of 5 as in the paper's Section 4, and the median)
         others = []
         for cfg in (wl.config_tiny(), wl.config_five_general(), wl.config_property_heavy(), wl.config_batched(),
-                    wl.config_paper_chain(), wl.config_transposed(), wl.config_sum_shared(), wl.config_sum_triangular()):
+                    wl.config_paper_chain(), wl.config_transposed(), wl.config_sum_shared(), wl.config_sum_triangular(),
+                    wl.config_expression()):
             batch = getattr(cfg, "batch", 1)
             r = time_equation(mom, torch, cfg, variant, steps=20, warmup=3, stream=stream, timing=batch == 1)
             ms_min, ms_med = min(r["ms"]), statistics.median(r["ms"])

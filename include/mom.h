@@ -149,6 +149,45 @@ mom_status_t mom_equation_plan_sum(const mom_matrix_desc_t *factors, const int32
                                    const int32_t *factor_names, const int32_t *chain_lengths, int32_t n_chains,
                                    mom_variant_t variant, mom_plan_t **out_plan);
 
+/* Nested expressions (paper Section 2, "Operations": the body of an Equation is a bag of Mul, Add and Transpose
+ * operations walked from the yield, so they may nest: A*(B + C), (A + B)^T*C, ...).  The expression is a tree
+ * (or DAG) of nodes; node `root` is the value X. */
+typedef enum {
+    MOM_EXPR_OPERAND = 0,    /* operand `operand` of the operand table */
+    MOM_EXPR_MUL = 1,        /* product of its children, left to right */
+    MOM_EXPR_ADD = 2,        /* sum of its children */
+    MOM_EXPR_TRANSPOSE = 3   /* transpose of its single child */
+} mom_expr_kind_t;
+
+typedef struct {
+    int32_t kind;            /* mom_expr_kind_t */
+    int32_t operand;         /* MOM_EXPR_OPERAND: index into `operands`; otherwise ignored */
+    int32_t first_child;     /* the node's children are children[first_child .. first_child + n_children), each a */
+    int32_t n_children;      /* node index; ignored for MOM_EXPR_OPERAND */
+} mom_expr_node_t;
+
+/* Plan an expression.  Host only.
+ *   operands   host array of n_operands descriptors, the matrices AS STORED; an operand may be used many times
+ *   nodes      host array of n_nodes nodes;  children: host array of n_children node indices;  root: node of X
+ * What the planner does with the tree: transposes are pushed down to the operands ((e1*e2)^T = e2^T*e1^T,
+ * (e1+e2)^T = e1^T+e2^T); a product inside a product and a sum inside a sum are flattened; a sum inside a
+ * product is evaluated on its own, as by mom_equation_plan_sum, into a temporary in the workspace whose type is
+ * the sum's result type, and the temporary is one factor of the outer chain (nothing is distributed); nested
+ * sums with the same normal form are one temporary.  Products are shared within one sum as described for
+ * mom_equation_plan_sum, operands being named by their index.
+ * The plan executes through mom_equation_execute / _batched / _host with chain_ptrs holding ONE POINTER PER
+ * OPERAND (n_operands entries; an unused or Identity operand may be NULL) and no Add terms.
+ * In the parenthesization string an operand prints as its index (with ^T), a temporary as "[" its sum "]".
+ * Value ids in the steps count every factor of every chain (nested sums first) and then the products.
+ * Errors: INVALID_ARG (bad index, empty operation, a cycle), PROPERTY, DTYPE, SHAPE_MISMATCH, OVERFLOW, ALLOC. */
+mom_status_t mom_expression_plan(const mom_matrix_desc_t *operands, int32_t n_operands,
+                                 const mom_expr_node_t *nodes, int32_t n_nodes,
+                                 const int32_t *children, int32_t n_children, int32_t root,
+                                 mom_variant_t variant, mom_plan_t **out_plan);
+
+/* Number of nested sums the plan materializes (0 for plans of the other entry points). */
+mom_status_t mom_plan_temporaries(const mom_plan_t *plan, int32_t *temporaries);
+
 /* Number of products that mom_equation_plan_sum did not emit because an earlier chain computes them (0 for
  * plans of the other entry points). */
 mom_status_t mom_plan_reused_products(const mom_plan_t *plan, int32_t *reused);

@@ -38,6 +38,11 @@ class Step(ctypes.Structure):
                 ("useful_mults", ctypes.c_uint64)]
 
 
+class ExprNode(ctypes.Structure):
+    _fields_ = [("kind", ctypes.c_int32), ("operand", ctypes.c_int32), ("first_child", ctypes.c_int32),
+                ("n_children", ctypes.c_int32)]
+
+
 class MomError(RuntimeError):
     def __init__(self, status: int, where: str):
         self.status = int(status)
@@ -62,6 +67,10 @@ _sigs = {
     "mom_equation_plan_sum": [ctypes.POINTER(MatrixDesc), ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_int32),
                               ctypes.POINTER(ctypes.c_int32), ctypes.c_int32, ctypes.c_int, ctypes.POINTER(_P)],
     "mom_plan_reused_products": [_P, ctypes.POINTER(ctypes.c_int32)],
+    "mom_expression_plan": [ctypes.POINTER(MatrixDesc), ctypes.c_int32, ctypes.POINTER(ExprNode), ctypes.c_int32,
+                            ctypes.POINTER(ctypes.c_int32), ctypes.c_int32, ctypes.c_int32, ctypes.c_int,
+                            ctypes.POINTER(_P)],
+    "mom_plan_temporaries": [_P, ctypes.POINTER(ctypes.c_int32)],
     "mom_plan_flops": [_P, ctypes.POINTER(ctypes.c_uint64), ctypes.POINTER(ctypes.c_uint64)],
     "mom_plan_parenthesization": [_P, ctypes.c_char_p, ctypes.c_size_t, ctypes.POINTER(ctypes.c_size_t)],
     "mom_plan_num_steps": [_P, ctypes.POINTER(ctypes.c_int32)],
@@ -160,6 +169,11 @@ class Plan:
     def reused_products(self) -> int:
         n = ctypes.c_int32()
         _check(_lib.mom_plan_reused_products(self._h, ctypes.byref(n)), "mom_plan_reused_products")
+        return n.value
+
+    def temporaries(self) -> int:
+        n = ctypes.c_int32()
+        _check(_lib.mom_plan_temporaries(self._h, ctypes.byref(n)), "mom_plan_temporaries")
         return n.value
 
     def num_steps(self) -> int:
@@ -279,6 +293,38 @@ def mom_equation_plan_sum(chains: Sequence[Sequence], transposed: Optional[Seque
                                     ctypes.byref(handle))
     _check(st, "mom_equation_plan_sum")
     return Plan(handle.value, n, 0)
+
+
+EXPR_OPERAND, EXPR_MUL, EXPR_ADD, EXPR_TRANSPOSE = 0, 1, 2, 3
+
+
+def mom_expression_plan(expr, operands: Sequence, variant: int = VARIANT_3XTF32) -> Plan:
+    """Plan a nested expression: an operand index, ("t", e), ("mul", [e, ...]) or ("add", [e, ...]).
+
+    The plan executes with one pointer per operand.  This function only flattens the Python value into the
+    node and child arrays of the C call.
+    """
+    nodes: List[Tuple[int, int, int, int]] = []
+    children: List[int] = []
+
+    def emit(e) -> int:
+        if isinstance(e, int):
+            nodes.append((EXPR_OPERAND, e, 0, 0))
+            return len(nodes) - 1
+        kind = {"t": EXPR_TRANSPOSE, "mul": EXPR_MUL, "add": EXPR_ADD}.get(e[0], -1)
+        kids = [emit(c) for c in ([e[1]] if e[0] == "t" else e[1])]
+        nodes.append((kind, 0, len(children), len(kids)))
+        children.extend(kids)
+        return len(nodes) - 1
+
+    root = emit(expr)
+    node_arr = (ExprNode * len(nodes))(*[ExprNode(*n) for n in nodes])
+    child_arr = (ctypes.c_int32 * max(len(children), 1))(*children)
+    handle = _P()
+    st = _lib.mom_expression_plan(_desc_array(operands) if len(operands) else None, len(operands), node_arr, len(nodes),
+                                  child_arr, len(children), root, variant, ctypes.byref(handle))
+    _check(st, "mom_expression_plan")
+    return Plan(handle.value, len(operands), 0)
 
 
 def mom_product_3xtf32_noalloc(m: int, n: int, k: int, pa: int, pb: int, a_ptr: int, b_ptr: int, c_ptr: int,

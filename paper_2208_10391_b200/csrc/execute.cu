@@ -66,22 +66,22 @@ mom_status_t execute_impl(const mom_plan *p, const float *const *chain_ptrs, con
                           const float *const *add_ptrs, const int64_t *add_strides, float *out, int64_t out_stride,
                           int64_t batch, void *workspace, size_t workspace_bytes, cudaStream_t stream) {
     if (!p || !chain_ptrs || !out || batch < 1) return MOM_ERR_INVALID_ARG;
-    const int n_chain = (int)p->chain.size(), n_add = (int)p->add.size();
+    const int n_chain = (int)p->chain.size(), n_add = (int)p->add.size(), n_ptrs = (int)p->ptr_desc.size();
     if (n_add > 0 && !add_ptrs) return MOM_ERR_INVALID_ARG;
     if (batch > 1 && (!chain_strides || (n_add > 0 && !add_strides))) return MOM_ERR_INVALID_ARG;
     const int64_t rows = p->result_desc.rows, cols = p->result_desc.cols;
 
-    for (int i = 0; i < n_chain; ++i) {
-        if (p->chain[i].property == MOM_IDENTITY) continue;
+    for (int i = 0; i < n_ptrs; ++i) {
+        if (p->ptr_desc[i].property == MOM_IDENTITY) continue;
         if (!chain_ptrs[i]) return MOM_ERR_INVALID_ARG;
         if (!aligned16(chain_ptrs[i])) return MOM_ERR_ALIGNMENT;
-        if (batch > 1 && (chain_strides[i] % 4 != 0 || chain_strides[i] < p->chain[i].rows * p->chain[i].cols))
+        if (batch > 1 && (chain_strides[i] % 4 != 0 || chain_strides[i] < p->ptr_desc[i].rows * p->ptr_desc[i].cols))
             return MOM_ERR_INVALID_ARG;
     }
-    if (!p->names.empty()) {          // factors with one name are one matrix: a product shared between chains relies on it
-        for (int i = 0; i < n_chain; ++i)
+    if (!p->names.empty()) {          // entries with one name are one matrix: a product shared between chains relies on it
+        for (int i = 0; i < n_ptrs; ++i)
             for (int j = 0; j < i; ++j)
-                if (p->names[i] == p->names[j] && p->chain[i].property != MOM_IDENTITY &&
+                if (p->names[i] == p->names[j] && p->ptr_desc[i].property != MOM_IDENTITY &&
                     (chain_ptrs[i] != chain_ptrs[j] || (batch > 1 && chain_strides[i] != chain_strides[j])))
                     return MOM_ERR_INVALID_ARG;
     }
@@ -119,8 +119,8 @@ mom_status_t execute_impl(const mom_plan *p, const float *const *chain_ptrs, con
         std::memset(&fp, 0, sizeof(fp));
         fp.n_ops = (int)p->kept.size();
         for (int i = 0; i < fp.n_ops; ++i) {
-            const int id = p->kept[i];
-            fp.ops[i] = FusedOperand{chain_ptrs[id], chain_strides ? chain_strides[id] : 0, (int)p->chain[id].rows,
+            const int id = p->kept[i], slot = p->factor_ptr[id];
+            fp.ops[i] = FusedOperand{chain_ptrs[slot], chain_strides ? chain_strides[slot] : 0, (int)p->chain[id].rows,
                                      (int)p->chain[id].cols, p->chain[id].property, p->fused_value_off[id], p->fused_value_ld[id],
                                      (int)p->chain_t[id]};
         }
@@ -163,139 +163,152 @@ mom_status_t execute_impl(const mom_plan *p, const float *const *chain_ptrs, con
     }
     // instances per pass: all of them when every step can take grid.z batching, else one at a time
     const int64_t group = any_tc ? 1 : (batch < 65535 ? batch : 65535);
-    const size_t ws_inst = p->workspace_per_instance;
-
-    std::vector<const Summand *> simple;
-    bool has_products = false;
-    for (const Summand &sm : p->summands) {
-        if (sm.kind == SUM_STEP) has_products = true;
-        else simple.push_back(&sm);
-    }
-    const int n_simple = (int)simple.size();
+    char *const ws = static_cast<char *>(workspace);
 
     for (int64_t b0 = 0; b0 < batch; b0 += group) {
         const int nb = (int)((batch - b0 < group) ? batch - b0 : group);
+        // a factor: a stored matrix of the caller, or the temporary of a nested sum (instance-major in the workspace)
         auto chain_op = [&](int id) {
-            const long long s = chain_strides ? chain_strides[id] : 0;
-            return Operand{chain_ptrs[id] ? chain_ptrs[id] + b0 * s : nullptr, s};
-        };
-        float *x = out + b0 * out_stride;
-        // Summands that are not products (Add terms, chains that reduced to one factor or to Identity), in the
-        // order written; `simple[first..]` go into `t`, at most MAX_FUSED_ADD of them.  Returns the next index.
-        auto add_terms = [&](int first, AddTerms *t) {
-            t->count = 0;
-            t->transposed = 0;
-            t->aliases_out = 0;
-            t->rows = (int)rows;
-            int i = first;
-            for (; i < n_simple && t->count < MAX_FUSED_ADD; ++i, ++t->count) {
-                const Summand &sm = *simple[i];
-                if (sm.kind == SUM_IDENTITY || (sm.kind == SUM_TERM && p->add[sm.index].property == MOM_IDENTITY)) {
-                    t->ptr[t->count] = nullptr;
-                    t->stride[t->count] = 0;
-                } else if (sm.kind == SUM_TERM) {
-                    const long long s = add_strides ? add_strides[sm.index] : 0;
-                    t->ptr[t->count] = add_ptrs[sm.index] + b0 * s;
-                    t->stride[t->count] = s;
-                    if (p->add_t[sm.index]) t->transposed |= 1u << t->count;
-                } else {
-                    const Operand o = chain_op(sm.index);
-                    t->ptr[t->count] = o.ptr;
-                    t->stride[t->count] = o.stride;
-                    if (p->chain_t[sm.index]) t->transposed |= 1u << t->count;
-                }
+            if (p->factor_sum[id] >= 0) {
+                const SumInfo &t = p->sums[p->factor_sum[id]];
+                return Operand{reinterpret_cast<const float *>(ws + t.out_off * (size_t)nb), (long long)(t.desc.rows * t.desc.cols)};
             }
-            return i;
+            const int slot = p->factor_ptr[id];
+            const long long s = chain_strides ? chain_strides[slot] : 0;
+            return Operand{chain_ptrs[slot] ? chain_ptrs[slot] + b0 * s : nullptr, s};
         };
-        int added = 0;
 
-        if (!has_products) {
-            // X = first summand + the following ones
-            const Summand &sm = *simple[0];
-            AddTerms t;
-            added = add_terms(1, &t);
-            cudaError_t e;
-            if (sm.kind == SUM_IDENTITY || (sm.kind == SUM_TERM && p->add[sm.index].property == MOM_IDENTITY)) {
-                e = launch_elementwise(nullptr, 0, 1, x, out_stride, (int)rows, (int)cols, p->result_desc.property, t, nb, stream);
-            } else if (sm.kind == SUM_FACTOR) {
-                const Operand src = chain_op(sm.index);
-                e = launch_elementwise(src.ptr, src.stride, p->chain_t[sm.index] ? 3 : 0, x, out_stride, (int)rows, (int)cols, p->result_desc.property, t, nb, stream);
-            } else {
-                const long long ss = add_strides ? add_strides[sm.index] : 0;
-                e = launch_elementwise(add_ptrs[sm.index] + b0 * ss, ss, p->add_t[sm.index] ? 3 : 0, x, out_stride, (int)rows, (int)cols, p->result_desc.property, t, nb, stream);
+        for (size_t si = 0; si < p->sums.size(); ++si) {
+            const SumInfo &sum = p->sums[si];
+            const bool top = si + 1 == p->sums.size();
+            const int srows = (int)sum.desc.rows, scols = (int)sum.desc.cols;
+            // where this sum's value goes: X, or the temporary
+            float *x = top ? out + b0 * out_stride : reinterpret_cast<float *>(ws + sum.out_off * (size_t)nb);
+            const long long x_stride = top ? out_stride : (long long)srows * scols;
+
+            std::vector<const Summand *> simple;     // summands that are not products, in the order written
+            bool has_products = false;
+            for (const Summand &sm : sum.summands) {
+                if (sm.kind == SUM_STEP) has_products = true;
+                else simple.push_back(&sm);
             }
-            if (e != cudaSuccess) return MOM_ERR_CUDA;
-            ++launches;
-        }
-
-        for (int s = 0; s < ns; ++s) {
-            const StepImpl &stp = p->steps[s];
-            auto value = [&](int id) {
-                if (id < n_chain) return chain_op(id);
-                const StepImpl &prod = p->steps[id - n_chain];
-                const long long elems = (long long)prod.pub.m * prod.pub.n;
-                // grid.z batching keeps one copy of each intermediate per instance, instance-major
-                // (a tensor-core step that feeds another one leaves no f32 intermediate: its consumer reads planes)
-                if (prod.out_off == SIZE_MAX) return Operand{nullptr, elems};
-                return Operand{reinterpret_cast<const float *>(static_cast<char *>(workspace) + prod.out_off * (size_t)nb), elems};
+            const int n_simple = (int)simple.size();
+            auto is_identity = [&](const Summand &sm) {
+                return sm.kind == SUM_IDENTITY || (sm.kind == SUM_TERM && p->add[sm.index].property == MOM_IDENTITY);
             };
-            const Operand A = value(stp.pub.lhs), B = value(stp.pub.rhs);
-            ProductArgs a;
-            std::memset(&a, 0, sizeof(a));
-            a.A = A.ptr; a.B = B.ptr;
-            a.strideA = A.stride; a.strideB = B.stride;
-            a.m = (int)stp.pub.m; a.n = (int)stp.pub.n; a.k = (int)stp.pub.k;
-            a.pa = stp.pub.lhs_property; a.pb = stp.pub.rhs_property;
-            a.transA = stp.pub.lhs_transposed; a.transB = stp.pub.rhs_transposed;
-            if (stp.is_last && stp.accumulate) {
-                // a later chain's product is added to what the earlier ones left in X
-                a.C = x; a.strideC = out_stride;
-                a.pout = p->result_desc.property;
-                a.add.count = 1;
-                a.add.ptr[0] = x;
-                a.add.stride[0] = out_stride;
-                a.add.transposed = 0;
-                a.add.aliases_out = 1u;
-                a.add.rows = (int)rows;
-            } else if (stp.is_last) {
-                a.C = x; a.strideC = out_stride;
-                a.pout = p->result_desc.property;
-                added = add_terms(0, &a.add);
-            } else {
-                a.C = stp.out_off == SIZE_MAX ? nullptr
-                                              : reinterpret_cast<float *>(static_cast<char *>(workspace) + stp.out_off * (size_t)nb);
-                a.strideC = (long long)stp.pub.m * stp.pub.n;
-                a.pout = stp.pub.out_property;
-                a.add.count = 0;
-                a.add.transposed = 0;
-                a.add.aliases_out = 0;
-                a.add.rows = (int)stp.pub.m;
-            }
-            cudaEvent_t *ev = timing ? &p->dev->events[((size_t)(p->dev->timed_executes % TIMING_SLOTS) * ns + s) * 3] : nullptr;
-            if (ev) cudaEventRecord(ev[0], stream);
-            if (stp.pub.uses_tensor_cores) {
-                int used = 0;
-                st = tc_launch_step(*p, p->dev->tc, s, a, static_cast<char *>(workspace), p->dev->status, stream, &used,
-                                    ev ? ev[1] : nullptr);
-                if (st != MOM_OK) return st;
-                launches += used;
-            } else {
-                if (ev) cudaEventRecord(ev[1], stream);
-                if (launch_product_ffma(a, nb, stream) != cudaSuccess) return MOM_ERR_CUDA;
+            // `simple[first..]` go into `t`, at most MAX_FUSED_ADD of them; returns the next index
+            auto add_terms = [&](int first, AddTerms *t) {
+                t->count = 0;
+                t->transposed = 0;
+                t->aliases_out = 0;
+                t->rows = srows;
+                int i = first;
+                for (; i < n_simple && t->count < MAX_FUSED_ADD; ++i, ++t->count) {
+                    const Summand &sm = *simple[i];
+                    if (is_identity(sm)) {
+                        t->ptr[t->count] = nullptr;
+                        t->stride[t->count] = 0;
+                    } else if (sm.kind == SUM_TERM) {
+                        const long long s = add_strides ? add_strides[sm.index] : 0;
+                        t->ptr[t->count] = add_ptrs[sm.index] + b0 * s;
+                        t->stride[t->count] = s;
+                        if (p->add_t[sm.index]) t->transposed |= 1u << t->count;
+                    } else {
+                        const Operand o = chain_op(sm.index);
+                        t->ptr[t->count] = o.ptr;
+                        t->stride[t->count] = o.stride;
+                        if (p->chain_t[sm.index]) t->transposed |= 1u << t->count;
+                    }
+                }
+                return i;
+            };
+            int added = 0;
+
+            if (!has_products) {
+                // value = first summand + the following ones
+                const Summand &sm = *simple[0];
+                AddTerms t;
+                added = add_terms(1, &t);
+                cudaError_t e;
+                if (is_identity(sm)) {
+                    e = launch_elementwise(nullptr, 0, 1, x, x_stride, srows, scols, sum.desc.property, t, nb, stream);
+                } else if (sm.kind == SUM_FACTOR) {
+                    const Operand src = chain_op(sm.index);
+                    e = launch_elementwise(src.ptr, src.stride, p->chain_t[sm.index] ? 3 : 0, x, x_stride, srows, scols, sum.desc.property, t, nb, stream);
+                } else {
+                    const long long ss = add_strides ? add_strides[sm.index] : 0;
+                    e = launch_elementwise(add_ptrs[sm.index] + b0 * ss, ss, p->add_t[sm.index] ? 3 : 0, x, x_stride, srows, scols, sum.desc.property, t, nb, stream);
+                }
+                if (e != cudaSuccess) return MOM_ERR_CUDA;
                 ++launches;
             }
-            if (ev) cudaEventRecord(ev[2], stream);
-        }
-        (void)ws_inst;
 
-        // summands beyond the fused limit: X += T, a few at a time, in place
-        while (added < n_simple) {
-            AddTerms t;
-            const int first = added;
-            added = add_terms(first, &t);
-            if (launch_elementwise(nullptr, 0, 2, x, out_stride, (int)rows, (int)cols, p->result_desc.property, t, nb, stream) != cudaSuccess)
-                return MOM_ERR_CUDA;
-            ++launches;
+            for (int s = sum.step_begin; s < sum.step_end; ++s) {
+                const StepImpl &stp = p->steps[s];
+                auto value = [&](int id) {
+                    if (id < n_chain) return chain_op(id);
+                    const StepImpl &prod = p->steps[id - n_chain];
+                    const long long elems = (long long)prod.pub.m * prod.pub.n;
+                    // grid.z batching keeps one copy of each intermediate per instance, instance-major
+                    // (a tensor-core step that feeds another one leaves no f32 intermediate: its consumer reads planes)
+                    if (prod.out_off == SIZE_MAX) return Operand{nullptr, elems};
+                    return Operand{reinterpret_cast<const float *>(ws + prod.out_off * (size_t)nb), elems};
+                };
+                const Operand A = value(stp.pub.lhs), B = value(stp.pub.rhs);
+                ProductArgs a;
+                std::memset(&a, 0, sizeof(a));
+                a.A = A.ptr; a.B = B.ptr;
+                a.strideA = A.stride; a.strideB = B.stride;
+                a.m = (int)stp.pub.m; a.n = (int)stp.pub.n; a.k = (int)stp.pub.k;
+                a.pa = stp.pub.lhs_property; a.pb = stp.pub.rhs_property;
+                a.transA = stp.pub.lhs_transposed; a.transB = stp.pub.rhs_transposed;
+                if (stp.is_last && stp.accumulate) {
+                    // a later chain's product is added to what the earlier ones left in the sum's buffer
+                    a.C = x; a.strideC = x_stride;
+                    a.pout = sum.desc.property;
+                    a.add.count = 1;
+                    a.add.ptr[0] = x;
+                    a.add.stride[0] = x_stride;
+                    a.add.transposed = 0;
+                    a.add.aliases_out = 1u;
+                    a.add.rows = srows;
+                } else if (stp.is_last) {
+                    a.C = x; a.strideC = x_stride;
+                    a.pout = sum.desc.property;
+                    added = add_terms(0, &a.add);
+                } else {
+                    a.C = stp.out_off == SIZE_MAX ? nullptr : reinterpret_cast<float *>(ws + stp.out_off * (size_t)nb);
+                    a.strideC = (long long)stp.pub.m * stp.pub.n;
+                    a.pout = stp.pub.out_property;
+                    a.add.count = 0;
+                    a.add.transposed = 0;
+                    a.add.aliases_out = 0;
+                    a.add.rows = (int)stp.pub.m;
+                }
+                cudaEvent_t *ev = timing ? &p->dev->events[((size_t)(p->dev->timed_executes % TIMING_SLOTS) * ns + s) * 3] : nullptr;
+                if (ev) cudaEventRecord(ev[0], stream);
+                if (stp.pub.uses_tensor_cores) {
+                    int used = 0;
+                    st = tc_launch_step(*p, p->dev->tc, s, a, ws, p->dev->status, stream, &used, ev ? ev[1] : nullptr);
+                    if (st != MOM_OK) return st;
+                    launches += used;
+                } else {
+                    if (ev) cudaEventRecord(ev[1], stream);
+                    if (launch_product_ffma(a, nb, stream) != cudaSuccess) return MOM_ERR_CUDA;
+                    ++launches;
+                }
+                if (ev) cudaEventRecord(ev[2], stream);
+            }
+
+            // summands beyond the fused limit: value += T, a few at a time, in place
+            while (added < n_simple) {
+                AddTerms t;
+                const int first = added;
+                added = add_terms(first, &t);
+                if (launch_elementwise(nullptr, 0, 2, x, x_stride, srows, scols, sum.desc.property, t, nb, stream) != cudaSuccess)
+                    return MOM_ERR_CUDA;
+                ++launches;
+            }
         }
     }
     if (timing) ++p->dev->timed_executes;
@@ -333,7 +346,7 @@ mom_status_t mom_equation_execute_host(const mom_plan_t *plan, const float *cons
     mom_plan_host_staging_bytes(plan, batch, &need);
     if (!staging || staging_bytes < need) return MOM_ERR_WORKSPACE_TOO_SMALL;
     if (reinterpret_cast<uintptr_t>(staging) % mom::WS_ALIGN != 0) return MOM_ERR_ALIGNMENT;
-    const int n_chain = (int)plan->chain.size(), n_add = (int)plan->add.size();
+    const int n_chain = (int)plan->ptr_desc.size(), n_add = (int)plan->add.size();
     if (n_add > 0 && !add_host) return MOM_ERR_INVALID_ARG;
 
     char *cur = static_cast<char *>(staging);
@@ -360,7 +373,7 @@ mom_status_t mom_equation_execute_host(const mom_plan_t *plan, const float *cons
             cstride[i] = cstride[same];
             continue;
         }
-        mom_status_t st = stage(plan->chain[i], chain_host[i], &cptr[i], &cstride[i]);
+        mom_status_t st = stage(plan->ptr_desc[i], chain_host[i], &cptr[i], &cstride[i]);
         if (st != MOM_OK) return st;
     }
     for (int i = 0; i < n_add; ++i) {

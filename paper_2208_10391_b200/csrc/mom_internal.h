@@ -30,7 +30,8 @@ inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 struct StepImpl {
     mom_step_t pub;
     bool is_last = false;           // root of its chain's tree: writes X (the first root also carries the Add terms)
-    bool accumulate = false;        // a later chain's root: adds its product to what X already holds
+    bool accumulate = false;        // a later chain's root: adds its product to what the sum's buffer already holds
+    int sum = -1;                   // roots: index of the sum (mom_plan::sums) whose value they write
     // workspace byte offsets (per instance); SIZE_MAX = not used
     size_t out_off = SIZE_MAX;      // f32 intermediate written by this step (not for the last step)
     size_t a_hi_off = SIZE_MAX, a_lo_off = SIZE_MAX;   // split planes of the operands (tensor-core steps)
@@ -53,19 +54,32 @@ struct Summand {
     int index;      // one factor (index = factor id); SUM_TERM: Add term `index`; SUM_IDENTITY: a chain equal to I
 };
 
+// One sum of chains.  The last sum of a plan is the equation's value X; earlier ones are nested sums of an
+// expression (a sum inside a product), evaluated into a workspace temporary that is then a factor of a later chain.
+struct SumInfo {
+    std::vector<Summand> summands;          // what is added up, in the order written
+    int step_begin = 0, step_end = 0;       // the products emitted for this sum
+    mom_matrix_desc_t desc{};               // type of the value
+    size_t out_off = SIZE_MAX;              // workspace byte offset of the temporary (per instance); SIZE_MAX: X
+};
+
 struct DeviceState;   // launcher-owned, created on first execute (execute.cu)
 
 }  // namespace mom
 
 struct mom_plan {
     int32_t variant = 0;
-    std::vector<mom_matrix_desc_t> chain;      // original operands as the equation uses them (transposed type where flagged)
+    std::vector<mom_matrix_desc_t> chain;      // every factor of every chain as the equation uses it (transposed type where flagged)
+    std::vector<int32_t> factor_ptr;           // per factor: index into the caller's pointer array; -1 for a temporary
+    std::vector<int32_t> factor_sum;           // per factor: the nested sum whose temporary it is; -1 for a stored matrix
+    std::vector<mom_matrix_desc_t> ptr_desc;   // per entry of the caller's pointer array: the matrix as stored
     std::vector<mom_matrix_desc_t> add;
     std::vector<char> chain_t, add_t;          // operand enters transposed: stored shape is (cols x rows) of the entry above
     std::vector<int32_t> chain_begin;          // factors of chain c are [chain_begin[c], chain_begin[c + 1])
-    std::vector<int32_t> names;                // per factor: equal names = the same stored matrix (empty: all distinct)
+    std::vector<int32_t> names;                // per pointer entry: equal names = the same stored matrix (empty: all distinct)
     std::vector<int32_t> kept;                 // factor indices surviving identity simplification
-    std::vector<mom::Summand> summands;        // what is added up into X, in the order written
+    std::vector<mom::SumInfo> sums;            // nested sums first, X last
+    int32_t temporaries = 0;                   // nested sums that are materialized
     int32_t reused = 0;                        // products not emitted because an earlier chain computed them
     std::string paren;
     uint64_t mults = 0;                        // useful multiplications of the chosen tree

@@ -119,24 +119,37 @@ mom_status_t mom_matrix_desc(int64_t rows, int64_t cols, mom_property_t property
     return MOM_OK;
 }
 
-// Shared body of the planning entry points.  `factors` are all chains' stored factors one after the other,
-// `chain_len[c]` of them belong to chain c; `names` (optional) tells which factors are the same stored matrix.
-static mom_status_t plan_equation(const mom_matrix_desc_t *stored_chain, const int32_t *chain_transposed,
-                                  const int32_t *names, const int32_t *chain_len, int32_t n_chains,
-                                  const mom_matrix_desc_t *stored_add, const int32_t *add_transposed, int32_t n_add,
-                                  mom_variant_t variant, mom_plan_t **out_plan) {
-    if (!out_plan || !stored_chain || !chain_len || n_chains < 1 || n_add < 0 || (n_add > 0 && !stored_add))
-        return MOM_ERR_INVALID_ARG;
+// What the planning entry points hand to the shared planner: sums of chains in dependency order (a nested sum
+// before the sum that uses it; the last one is X).  A factor is a stored matrix (an entry of the caller's pointer
+// array, possibly transposed) or the temporary of an earlier sum.
+struct FactorIn {
+    int32_t ptr;        // entry of the pointer array, or -1
+    int32_t sub;        // earlier sum, or -1
+    bool t;             // enters transposed (stored matrices only)
+    int64_t name;       // equal names = the same value; -1: nothing known
+    std::string label;  // how a stored matrix prints in the parenthesization string
+};
+struct SumIn { std::vector<std::vector<FactorIn>> chains; };
+
+static mom_status_t plan_sums(const std::vector<mom_matrix_desc_t> &slots, const std::vector<SumIn> &sums_in,
+                              const int32_t *slot_names, const mom_matrix_desc_t *stored_add,
+                              const int32_t *add_transposed, int32_t n_add, mom_variant_t variant, mom_plan_t **out_plan) {
+    if (!out_plan || sums_in.empty() || n_add < 0 || (n_add > 0 && !stored_add)) return MOM_ERR_INVALID_ARG;
     if ((int)variant < 0 || (int)variant > 2) return MOM_ERR_INVALID_ARG;
     int64_t total = 0;
-    for (int c = 0; c < n_chains; ++c) {
-        if (chain_len[c] < 1) return MOM_ERR_INVALID_ARG;
-        total += chain_len[c];
-        if (total > (1 << 20)) return MOM_ERR_INVALID_ARG;
+    int n_chains = 0;
+    for (const SumIn &si : sums_in) {
+        if (si.chains.empty()) return MOM_ERR_INVALID_ARG;
+        for (const auto &c : si.chains) {
+            if (c.empty()) return MOM_ERR_INVALID_ARG;
+            total += (int64_t)c.size();
+            ++n_chains;
+            if (total > (1 << 20)) return MOM_ERR_INVALID_ARG;
+        }
     }
-    const int n_chain = (int)total;
-    for (int i = 0; i < n_chain; ++i) {
-        mom_status_t st = check_desc(stored_chain[i]);
+    const int n_chain = (int)total;                         // factors over all chains of all sums
+    for (const auto &d : slots) {
+        mom_status_t st = check_desc(d);
         if (st != MOM_OK) return st;
     }
     for (int i = 0; i < n_add; ++i) {
@@ -144,182 +157,214 @@ static mom_status_t plan_equation(const mom_matrix_desc_t *stored_chain, const i
         if (st != MOM_OK) return st;
     }
     // A transposed operand takes part with its transposed type: shape swapped, lowerTri <-> upperTri
-    // (the inference rule of the paper's Section 2); from here on `chain` / `add_terms` are the types as used.
+    // (the inference rule of the paper's Section 2); `chain` / `add_terms` hold the types as used.
     auto as_used = [](const mom_matrix_desc_t &d, bool t) {
         if (!t) return d;
         const int32_t prop = d.property == MOM_LOWER_TRI ? (int32_t)MOM_UPPER_TRI
                              : d.property == MOM_UPPER_TRI ? (int32_t)MOM_LOWER_TRI : d.property;
         return mom_matrix_desc_t{d.cols, d.rows, prop, d.dtype};
     };
-    std::vector<mom_matrix_desc_t> chain_v, add_v;
-    std::vector<char> chain_t((size_t)n_chain, 0), add_t((size_t)n_add, 0);
-    std::vector<int32_t> begin;
-    try {
-        for (int i = 0; i < n_chain; ++i) {
-            chain_t[i] = chain_transposed && chain_transposed[i] != 0;
-            chain_v.push_back(as_used(stored_chain[i], chain_t[i] != 0));
-        }
-        for (int i = 0; i < n_add; ++i) {
-            add_t[i] = add_transposed && add_transposed[i] != 0;
-            add_v.push_back(as_used(stored_add[i], add_t[i] != 0));
-        }
-        begin.push_back(0);
-        for (int c = 0; c < n_chains; ++c) begin.push_back(begin.back() + chain_len[c]);
-        if (names) {                                   // one name, one stored type
-            std::map<int32_t, int> first;
-            for (int i = 0; i < n_chain; ++i) {
-                auto it = first.emplace(names[i], i).first;
-                const mom_matrix_desc_t &a = stored_chain[it->second], &b = stored_chain[i];
+    if (slot_names) {                                       // one name, one stored type
+        try {
+            std::map<int32_t, size_t> first;
+            for (size_t i = 0; i < slots.size(); ++i) {
+                auto it = first.emplace(slot_names[i], i).first;
+                const mom_matrix_desc_t &a = slots[it->second], &b = slots[i];
                 if (a.rows != b.rows || a.cols != b.cols || a.property != b.property) return MOM_ERR_INVALID_ARG;
             }
+        } catch (const std::bad_alloc &) {
+            return MOM_ERR_ALLOC;
         }
-    } catch (const std::bad_alloc &) {
-        return MOM_ERR_ALLOC;
     }
-    const mom_matrix_desc_t *chain = chain_v.data(), *add_terms = add_v.data();
-    for (int c = 0; c < n_chains; ++c)
-        for (int i = begin[c]; i + 1 < begin[c + 1]; ++i)
-            if (chain[i].cols != chain[i + 1].rows) return MOM_ERR_SHAPE_MISMATCH;
-    const int64_t rows = chain[0].rows, cols = chain[begin[1] - 1].cols;
-    for (int c = 1; c < n_chains; ++c)
-        if (chain[begin[c]].rows != rows || chain[begin[c + 1] - 1].cols != cols) return MOM_ERR_SHAPE_MISMATCH;
-    for (int i = 0; i < n_add; ++i)
-        if (add_terms[i].rows != rows || add_terms[i].cols != cols) return MOM_ERR_SHAPE_MISMATCH;
 
     mom_plan *p = new (std::nothrow) mom_plan();
     if (!p) return MOM_ERR_ALLOC;
     try {
         p->variant = (int32_t)variant;
-        p->chain.assign(chain, chain + n_chain);
-        if (n_add) p->add.assign(add_terms, add_terms + n_add);
-        p->chain_t = chain_t;
-        p->add_t = add_t;
-        p->chain_begin = begin;
-        if (names) p->names.assign(names, names + n_chain);
-        for (int i = 0; i < n_add; ++i) p->add_flops += nnz(add_terms[i]);
+        p->ptr_desc = slots;
+        if (slot_names) p->names.assign(slot_names, slot_names + slots.size());
+        for (int i = 0; i < n_add; ++i) {
+            p->add_t.push_back(add_transposed && add_transposed[i] != 0);
+            p->add.push_back(as_used(stored_add[i], p->add_t.back() != 0));
+        }
+        p->chain_begin.push_back(0);
 
         int32_t next_id = n_chain;
-        std::map<std::vector<int64_t>, int32_t> seen;       // run of (name, transposed) -> id of its product
-        std::vector<int32_t> summand_props;
+        std::vector<std::string> sum_text(sums_in.size());
+        std::vector<int64_t> factor_name;                   // per factor, over all sums
 
-        for (int c = 0; c < n_chains; ++c) {
-            if (c) p->paren += "+";
-            // identity simplification: A*I -> A, I*A -> A, I*I -> I
-            std::vector<int32_t> kept;
-            for (int i = begin[c]; i < begin[c + 1]; ++i)
-                if (chain[i].property != MOM_IDENTITY) kept.push_back(i);
-            p->kept.insert(p->kept.end(), kept.begin(), kept.end());
-            const int r = (int)kept.size();
-            mom_matrix_desc_t value_desc;
+        for (size_t si = 0; si < sums_in.size(); ++si) {
+            const SumIn &in = sums_in[si];
+            const bool top = si + 1 == sums_in.size();
+            mom::SumInfo info;
+            info.step_begin = (int)p->steps.size();
+            std::map<std::vector<int64_t>, int32_t> seen;   // run of (name, transposed) -> id of its product
+            std::vector<int32_t> summand_props;
+            std::string &text = sum_text[si];
+            int64_t rows = 0, cols = 0;
 
-            if (r == 0) {
-                p->paren += "I";
-                value_desc = mom_matrix_desc_t{rows, cols, MOM_IDENTITY, MOM_F32};
-                p->summands.push_back(mom::Summand{mom::SUM_IDENTITY, 0});
-            } else {
-                // dynamic program over the reduced chain
-                std::vector<Node> node((size_t)r * r);
-                std::vector<uint64_t> cost((size_t)r * r, 0);
-                std::vector<int> split((size_t)r * r, -1);
-                auto at = [r](int i, int j) { return (size_t)i * r + j; };
-                for (int i = 0; i < r; ++i) {
-                    const auto &d = chain[kept[i]];
-                    node[at(i, i)] = Node{d.rows, d.cols, d.property};
-                }
-                for (int len = 2; len <= r; ++len) {
-                    for (int i = 0; i + len - 1 < r; ++i) {
-                        const int j = i + len - 1;
-                        bool have = false;
-                        uint64_t best = 0;
-                        int best_k = -1;
-                        for (int k = i; k < j; ++k) {
-                            const Node &a = node[at(i, k)], &b = node[at(k + 1, j)];
-                            uint64_t m;
-                            if (!useful_mults(a.prop, b.prop, a.rows, a.cols, b.cols, &m)) { delete p; return MOM_ERR_OVERFLOW; }
-                            const u128 cst = (u128)cost[at(i, k)] + cost[at(k + 1, j)] + m;
-                            if (cst >= (u128)COST_LIMIT) { delete p; return MOM_ERR_OVERFLOW; }
-                            if (!have || (uint64_t)cst < best) { best = (uint64_t)cst; best_k = k; have = true; }
-                        }
-                        cost[at(i, j)] = best;
-                        split[at(i, j)] = best_k;
-                        const Node &a = node[at(i, best_k)], &b = node[at(best_k + 1, j)];
-                        node[at(i, j)] = Node{a.rows, b.cols, join_property(a.prop, b.prop)};
+            for (size_t c = 0; c < in.chains.size(); ++c) {
+                if (c) text += "+";
+                // this chain's factors as used
+                const int begin = (int)p->chain.size();
+                std::vector<int64_t> fname;
+                std::vector<std::string> flabel;
+                for (const FactorIn &f : in.chains[c]) {
+                    if (f.sub >= 0) {
+                        if ((size_t)f.sub >= si) { delete p; return MOM_ERR_INVALID_ARG; }
+                        p->chain.push_back(p->sums[f.sub].desc);
+                        p->chain_t.push_back(0);
+                        flabel.push_back("[" + sum_text[f.sub] + "]");
+                    } else {
+                        if (f.ptr < 0 || (size_t)f.ptr >= slots.size()) { delete p; return MOM_ERR_INVALID_ARG; }
+                        p->chain.push_back(as_used(slots[f.ptr], f.t));
+                        p->chain_t.push_back(f.t ? 1 : 0);
+                        flabel.push_back(f.label);
                     }
+                    p->factor_ptr.push_back(f.sub >= 0 ? -1 : f.ptr);
+                    p->factor_sum.push_back(f.sub);
+                    fname.push_back(f.name);
+                    factor_name.push_back(f.name);
                 }
+                const int end = (int)p->chain.size();
+                p->chain_begin.push_back(end);
+                const mom_matrix_desc_t *chain = p->chain.data();
+                for (int i = begin; i + 1 < end; ++i)
+                    if (chain[i].cols != chain[i + 1].rows) { delete p; return MOM_ERR_SHAPE_MISMATCH; }
+                if (c == 0) { rows = chain[begin].rows; cols = chain[end - 1].cols; }
+                else if (chain[begin].rows != rows || chain[end - 1].cols != cols) { delete p; return MOM_ERR_SHAPE_MISMATCH; }
 
-                // Post-order emission of the binary products; returns the id of the value of [i, j].  A product
-                // below the root whose run of named factors an earlier chain already multiplied (also below its
-                // root) is not emitted again: its id is reused and only its text is written.
-                struct Emit {
-                    mom_plan *p; const std::vector<Node> &node; const std::vector<int> &split; int r; int32_t &next_id;
-                    const std::vector<int32_t> &kept; std::map<std::vector<int64_t>, int32_t> &seen; bool named;
-                    std::string &s;
-                    int32_t run(int i, int j, bool emit) {
-                        if (i == j) {
-                            s += std::to_string(kept[i]);
-                            if (p->chain_t[kept[i]]) s += "^T";
-                            return kept[i];
-                        }
-                        const bool root = i == 0 && j == r - 1;
-                        std::vector<int64_t> key;
-                        int32_t shared = -1;
-                        if (emit && named && !root) {
-                            for (int q = i; q <= j; ++q) key.push_back((int64_t)p->names[kept[q]] * 2 + (p->chain_t[kept[q]] ? 1 : 0));
-                            auto it = seen.find(key);
-                            if (it != seen.end()) { shared = it->second; p->reused += j - i; }
-                        }
-                        const bool emit_here = emit && shared < 0;
-                        const int k = split[(size_t)i * r + j];
-                        s += "(";
-                        const int32_t l = run(i, k, emit_here);
-                        s += "*";
-                        const int32_t rr = run(k + 1, j, emit_here);
-                        s += ")";
-                        if (!emit) return -1;
-                        if (shared >= 0) return shared;
-                        const Node &a = node[(size_t)i * r + k], &b = node[(size_t)(k + 1) * r + j], &o = node[(size_t)i * r + j];
-                        mom::StepImpl st;
-                        std::memset(&st.pub, 0, sizeof(st.pub));
-                        st.pub.lhs = l; st.pub.rhs = rr; st.pub.out = next_id++;
-                        st.pub.lhs_property = a.prop; st.pub.rhs_property = b.prop; st.pub.out_property = o.prop;
-                        st.pub.lhs_transposed = l < (int32_t)p->chain.size() && p->chain_t[l];
-                        st.pub.rhs_transposed = rr < (int32_t)p->chain.size() && p->chain_t[rr];
-                        st.pub.m = a.rows; st.pub.k = a.cols; st.pub.n = b.cols;
-                        useful_mults(a.prop, b.prop, a.rows, a.cols, b.cols, &st.pub.useful_mults);
-                        const bool ta = is_tri(a.prop), tb = is_tri(b.prop);
-                        st.pub.kind = !ta && !tb ? MOM_KIND_GG : ta && !tb ? MOM_KIND_TG : !ta && tb ? MOM_KIND_GT
-                                      : a.prop == b.prop ? MOM_KIND_TT : MOM_KIND_TTMIX;
-                        st.is_last = root;
-                        p->steps.push_back(st);
-                        if (named && !root) seen.emplace(std::move(key), st.pub.out);
-                        return st.pub.out;
+                // identity simplification: A*I -> A, I*A -> A, I*I -> I
+                std::vector<int32_t> kept;
+                for (int i = begin; i < end; ++i)
+                    if (chain[i].property != MOM_IDENTITY) kept.push_back(i);
+                p->kept.insert(p->kept.end(), kept.begin(), kept.end());
+                const int r = (int)kept.size();
+                mom_matrix_desc_t value_desc;
+
+                if (r == 0) {
+                    text += "I";
+                    value_desc = mom_matrix_desc_t{rows, cols, MOM_IDENTITY, MOM_F32};
+                    info.summands.push_back(mom::Summand{mom::SUM_IDENTITY, 0});
+                } else {
+                    // dynamic program over the reduced chain
+                    std::vector<Node> node((size_t)r * r);
+                    std::vector<uint64_t> cost((size_t)r * r, 0);
+                    std::vector<int> split((size_t)r * r, -1);
+                    auto at = [r](int i, int j) { return (size_t)i * r + j; };
+                    for (int i = 0; i < r; ++i) {
+                        const auto &d = chain[kept[i]];
+                        node[at(i, i)] = Node{d.rows, d.cols, d.property};
                     }
-                } emit{p, node, split, r, next_id, kept, seen, names != nullptr, p->paren};
-                emit.run(0, r - 1, true);
-                const Node &root = node[at(0, r - 1)];
-                value_desc = mom_matrix_desc_t{root.rows, root.cols, root.prop, MOM_F32};
-                if (r == 1) p->summands.push_back(mom::Summand{mom::SUM_FACTOR, kept[0]});
-                else p->summands.push_back(mom::Summand{mom::SUM_STEP, (int)p->steps.size() - 1});
+                    for (int len = 2; len <= r; ++len) {
+                        for (int i = 0; i + len - 1 < r; ++i) {
+                            const int j = i + len - 1;
+                            bool have = false;
+                            uint64_t best = 0;
+                            int best_k = -1;
+                            for (int k = i; k < j; ++k) {
+                                const Node &a = node[at(i, k)], &b = node[at(k + 1, j)];
+                                uint64_t m;
+                                if (!useful_mults(a.prop, b.prop, a.rows, a.cols, b.cols, &m)) { delete p; return MOM_ERR_OVERFLOW; }
+                                const u128 cst = (u128)cost[at(i, k)] + cost[at(k + 1, j)] + m;
+                                if (cst >= (u128)COST_LIMIT) { delete p; return MOM_ERR_OVERFLOW; }
+                                if (!have || (uint64_t)cst < best) { best = (uint64_t)cst; best_k = k; have = true; }
+                            }
+                            cost[at(i, j)] = best;
+                            split[at(i, j)] = best_k;
+                            const Node &a = node[at(i, best_k)], &b = node[at(best_k + 1, j)];
+                            node[at(i, j)] = Node{a.rows, b.cols, join_property(a.prop, b.prop)};
+                        }
+                    }
+
+                    // Post-order emission of the binary products; returns the id of the value of [i, j].  A product
+                    // below the root whose run of named factors an earlier chain of this sum already multiplied (also
+                    // below its root) is not emitted again: its id is reused and only its text is written.
+                    struct Emit {
+                        mom_plan *p; const std::vector<Node> &node; const std::vector<int> &split; int r; int32_t &next_id;
+                        const std::vector<int32_t> &kept; std::map<std::vector<int64_t>, int32_t> &seen;
+                        const std::vector<int64_t> &fname; const std::vector<std::string> &flabel; int begin; int n_factors;
+                        int sum_index; std::string &s;
+                        int32_t run(int i, int j, bool emit) {
+                            if (i == j) {
+                                s += flabel[kept[i] - begin];
+                                if (p->chain_t[kept[i]]) s += "^T";
+                                return kept[i];
+                            }
+                            const bool root = i == 0 && j == r - 1;
+                            std::vector<int64_t> key;
+                            int32_t shared = -1;
+                            bool named = true;
+                            for (int q = i; q <= j; ++q) named &= fname[kept[q] - begin] >= 0;
+                            if (emit && named && !root) {
+                                for (int q = i; q <= j; ++q) key.push_back(fname[kept[q] - begin] * 2 + (p->chain_t[kept[q]] ? 1 : 0));
+                                auto it = seen.find(key);
+                                if (it != seen.end()) { shared = it->second; p->reused += j - i; }
+                            }
+                            const bool emit_here = emit && shared < 0;
+                            const int k = split[(size_t)i * r + j];
+                            s += "(";
+                            const int32_t l = run(i, k, emit_here);
+                            s += "*";
+                            const int32_t rr = run(k + 1, j, emit_here);
+                            s += ")";
+                            if (!emit) return -1;
+                            if (shared >= 0) return shared;
+                            const Node &a = node[(size_t)i * r + k], &b = node[(size_t)(k + 1) * r + j], &o = node[(size_t)i * r + j];
+                            mom::StepImpl st;
+                            std::memset(&st.pub, 0, sizeof(st.pub));
+                            st.pub.lhs = l; st.pub.rhs = rr; st.pub.out = next_id++;
+                            st.pub.lhs_property = a.prop; st.pub.rhs_property = b.prop; st.pub.out_property = o.prop;
+                            st.pub.lhs_transposed = l < n_factors && p->chain_t[l];
+                            st.pub.rhs_transposed = rr < n_factors && p->chain_t[rr];
+                            st.pub.m = a.rows; st.pub.k = a.cols; st.pub.n = b.cols;
+                            useful_mults(a.prop, b.prop, a.rows, a.cols, b.cols, &st.pub.useful_mults);
+                            const bool ta = is_tri(a.prop), tb = is_tri(b.prop);
+                            st.pub.kind = !ta && !tb ? MOM_KIND_GG : ta && !tb ? MOM_KIND_TG : !ta && tb ? MOM_KIND_GT
+                                          : a.prop == b.prop ? MOM_KIND_TT : MOM_KIND_TTMIX;
+                            st.is_last = root;
+                            if (root) st.sum = sum_index;
+                            p->steps.push_back(st);
+                            if (named && !root) seen.emplace(std::move(key), st.pub.out);
+                            return st.pub.out;
+                        }
+                    } emit{p, node, split, r, next_id, kept, seen, fname, flabel, begin, n_chain, (int)si, text};
+                    emit.run(0, r - 1, true);
+                    const Node &root = node[at(0, r - 1)];
+                    value_desc = mom_matrix_desc_t{root.rows, root.cols, root.prop, MOM_F32};
+                    if (r == 1) info.summands.push_back(mom::Summand{mom::SUM_FACTOR, kept[0]});
+                    else info.summands.push_back(mom::Summand{mom::SUM_STEP, (int)p->steps.size() - 1});
+                }
+                if (c == 0) { if (top) p->product_desc = value_desc; }
+                else p->add_flops += nnz(value_desc);
+                summand_props.push_back(value_desc.property);
             }
-            if (c == 0) p->product_desc = value_desc;
-            else p->add_flops += nnz(value_desc);
-            summand_props.push_back(value_desc.property);
+            if (top) {
+                for (int i = 0; i < n_add; ++i) {
+                    if (p->add[i].rows != rows || p->add[i].cols != cols) { delete p; return MOM_ERR_SHAPE_MISMATCH; }
+                    p->add_flops += nnz(p->add[i]);
+                    info.summands.push_back(mom::Summand{mom::SUM_TERM, i});
+                    summand_props.push_back(p->add[i].property);
+                }
+            }
+            info.step_end = (int)p->steps.size();
+            info.desc = mom_matrix_desc_t{rows, cols, sum_property(summand_props), MOM_F32};
+            {                                           // every root after the first adds to what the sum's buffer holds
+                bool first = true;
+                for (int s = info.step_begin; s < info.step_end; ++s)
+                    if (p->steps[s].is_last) { p->steps[s].accumulate = !first; first = false; }
+            }
+            p->sums.push_back(std::move(info));
         }
+        p->paren = sum_text.back();
+        p->result_desc = p->sums.back().desc;
+        p->temporaries = (int32_t)p->sums.size() - 1;
         for (const auto &st : p->steps) {
             const u128 sum = (u128)p->mults + st.pub.useful_mults;
             if (sum >= (u128)COST_LIMIT) { delete p; return MOM_ERR_OVERFLOW; }
             p->mults = (uint64_t)sum;
         }
-        for (int i = 0; i < n_add; ++i) {
-            p->summands.push_back(mom::Summand{mom::SUM_TERM, i});
-            summand_props.push_back(add_terms[i].property);
-        }
-        p->result_desc = mom_matrix_desc_t{rows, cols, sum_property(summand_props), MOM_F32};
-        {                                               // every root after the first adds to what X holds
-            bool first = true;
-            for (auto &st : p->steps)
-                if (st.is_last) { st.accumulate = !first; first = false; }
-        }
+        const bool single_chain = sums_in.size() == 1 && n_chains == 1;
 
         // kernel choice and workspace layout
         const int ns = (int)p->steps.size();
@@ -364,6 +409,24 @@ static mom_status_t plan_equation(const mom_matrix_desc_t *stored_chain, const i
                                          last_consumer < 0 ? ns - 1 : last_consumer, &st.out_off, 0});
             }
         }
+        // temporaries of nested sums: written by their roots (or by one elementwise pass just before the next
+        // sum's first product), read as a factor by later products or as a summand of a later sum
+        for (size_t si = 0; si + 1 < p->sums.size(); ++si) {
+            mom::SumInfo &sum = p->sums[si];
+            const int last_step = ns > 0 ? ns - 1 : 0;
+            int last = std::min(sum.step_begin, last_step);
+            for (int t = 0; t < ns; ++t) {
+                const mom_step_t &c = p->steps[t].pub;
+                const bool reads = (c.lhs < n_chain && p->factor_sum[c.lhs] == (int)si) || (c.rhs < n_chain && p->factor_sum[c.rhs] == (int)si);
+                if (reads) last = std::max(last, t);
+            }
+            for (size_t sj = si + 1; sj < p->sums.size(); ++sj)
+                for (const mom::Summand &sm : p->sums[sj].summands)
+                    if (sm.kind == mom::SUM_FACTOR && p->factor_sum[sm.index] == (int)si)
+                        last = std::max(last, std::min(p->sums[sj].step_end, last_step));
+            items.push_back(Interval{mom::align_up((size_t)sum.desc.rows * sum.desc.cols * sizeof(float), mom::WS_ALIGN),
+                                     std::min(sum.step_begin, last_step), last, &sum.out_off, 0});
+        }
         // Operand planes of the tensor-core steps.  Steps that take the same value on the same side (a shared
         // product; a named factor with the same transposition) read one set of planes: the first of them owns
         // the buffers, which then live until the last, and the others skip their split pass.
@@ -386,8 +449,8 @@ static mom_status_t plan_equation(const mom_matrix_desc_t *stored_chain, const i
                     const int producer = v - n_chain;
                     key = (int64_t)v << 1;
                     if (p->steps[producer].planes_out) { from = producer; ready = true; }
-                } else if (names) {
-                    key = (((int64_t)names[v] << 1) | (chain_t[v] ? 1 : 0)) | ((int64_t)1 << 62);
+                } else if (factor_name[v] >= 0) {
+                    key = ((factor_name[v] << 1) | (p->chain_t[v] ? 1 : 0)) | ((int64_t)1 << 62);
                 }
                 auto it = key >= 0 ? plane_sets.find({key, side}) : plane_sets.end();
                 if (it != plane_sets.end()) {
@@ -430,7 +493,7 @@ static mom_status_t plan_equation(const mom_matrix_desc_t *stored_chain, const i
             const int values = n_chain + ns;
             p->fused_value_off.assign(values, -1);
             size_t floats = 0;
-            bool ok = n_chains == 1 && ns >= 1 && ns <= mom::FUSED_MAX_STEPS && (int)p->kept.size() <= mom::FUSED_MAX_OPERANDS &&
+            bool ok = single_chain && ns >= 1 && ns <= mom::FUSED_MAX_STEPS && (int)p->kept.size() <= mom::FUSED_MAX_OPERANDS &&
                       n_add <= mom::MAX_FUSED_ADD && !any_tc;
             // every value feeds exactly one product: remember on which side
             std::vector<char> is_rhs(values, 0);
@@ -439,8 +502,8 @@ static mom_status_t plan_equation(const mom_matrix_desc_t *stored_chain, const i
             if (ok) {
                 for (int id : p->kept) {
                     p->fused_value_off[id] = (int)floats;
-                    p->fused_value_ld[id] = mom::fused_ld((int)chain[id].cols, is_rhs[id] != 0);
-                    floats += (size_t)chain[id].rows * p->fused_value_ld[id];
+                    p->fused_value_ld[id] = mom::fused_ld((int)p->chain[id].cols, is_rhs[id] != 0);
+                    floats += (size_t)p->chain[id].rows * p->fused_value_ld[id];
                     if (floats * sizeof(float) > mom::FUSED_MAX_SMEM) { ok = false; break; }
                 }
             }
@@ -471,16 +534,142 @@ mom_status_t mom_equation_plan(const mom_matrix_desc_t *chain, int32_t n_chain,
     return mom_equation_plan_transposed(chain, nullptr, n_chain, add_terms, nullptr, n_add, variant, out_plan);
 }
 
+// one sum whose factors are the caller's array entries in order
+static mom_status_t plan_flat(const mom_matrix_desc_t *stored, const int32_t *transposed, const int32_t *names,
+                              const int32_t *chain_len, int32_t n_chains, const mom_matrix_desc_t *stored_add,
+                              const int32_t *add_transposed, int32_t n_add, mom_variant_t variant, mom_plan_t **out_plan) {
+    if (!out_plan || !stored || !chain_len || n_chains < 1) return MOM_ERR_INVALID_ARG;
+    try {
+        std::vector<SumIn> sums(1);
+        int64_t total = 0;
+        for (int c = 0; c < n_chains; ++c) {
+            if (chain_len[c] < 1 || total + chain_len[c] > (1 << 20)) return MOM_ERR_INVALID_ARG;
+            std::vector<FactorIn> chain;
+            for (int i = 0; i < chain_len[c]; ++i, ++total) {
+                const int32_t f = (int32_t)total;
+                chain.push_back(FactorIn{f, -1, transposed && transposed[f] != 0, names ? (int64_t)(uint32_t)names[f] : -1,
+                                         std::to_string(f)});
+            }
+            sums[0].chains.push_back(std::move(chain));
+        }
+        std::vector<mom_matrix_desc_t> slots(stored, stored + total);
+        return plan_sums(slots, sums, names, stored_add, add_transposed, n_add, variant, out_plan);
+    } catch (const std::bad_alloc &) {
+        return MOM_ERR_ALLOC;
+    }
+}
+
 mom_status_t mom_equation_plan_transposed(const mom_matrix_desc_t *stored_chain, const int32_t *chain_transposed, int32_t n_chain,
                                           const mom_matrix_desc_t *stored_add, const int32_t *add_transposed, int32_t n_add,
                                           mom_variant_t variant, mom_plan_t **out_plan) {
-    return plan_equation(stored_chain, chain_transposed, nullptr, &n_chain, 1, stored_add, add_transposed, n_add, variant, out_plan);
+    return plan_flat(stored_chain, chain_transposed, nullptr, &n_chain, 1, stored_add, add_transposed, n_add, variant, out_plan);
 }
 
 mom_status_t mom_equation_plan_sum(const mom_matrix_desc_t *factors, const int32_t *factor_transposed,
                                    const int32_t *factor_names, const int32_t *chain_lengths, int32_t n_chains,
                                    mom_variant_t variant, mom_plan_t **out_plan) {
-    return plan_equation(factors, factor_transposed, factor_names, chain_lengths, n_chains, nullptr, nullptr, 0, variant, out_plan);
+    return plan_flat(factors, factor_transposed, factor_names, chain_lengths, n_chains, nullptr, nullptr, 0, variant, out_plan);
+}
+
+// ---- nested expressions ------------------------------------------------------------------------------------
+namespace {
+
+// Normal form of an expression: transposes pushed down to the operands, products inside products and sums
+// inside sums flattened, and every sum inside a product registered as a sum of its own (identical ones once).
+struct Normalizer {
+    const mom_expr_node_t *nodes; int32_t n_nodes; const int32_t *children; int32_t n_children; int32_t n_operands;
+    std::vector<SumIn> sums;                          // registered nested sums, in dependency order
+    std::map<std::string, int32_t> known;             // serialized normal form -> index in `sums`
+    int64_t factors = 0;
+    mom_status_t err = MOM_OK;
+
+    static std::string serialize(const SumIn &s) {
+        std::string out;
+        for (const auto &c : s.chains) {
+            out += "(";
+            for (const FactorIn &f : c)
+                out += f.sub >= 0 ? "S" + std::to_string(f.sub) + ";" : "L" + std::to_string(f.ptr) + (f.t ? "t;" : ";");
+            out += ")";
+        }
+        return out;
+    }
+
+    SumIn run(int32_t node, bool t, int depth) {
+        SumIn out;
+        if (err != MOM_OK) return out;
+        if (node < 0 || node >= n_nodes || depth > n_nodes) { err = MOM_ERR_INVALID_ARG; return out; }
+        const mom_expr_node_t &nd = nodes[node];
+        if (nd.kind == MOM_EXPR_OPERAND) {
+            if (nd.operand < 0 || nd.operand >= n_operands) { err = MOM_ERR_INVALID_ARG; return out; }
+            if (++factors > (1 << 20)) { err = MOM_ERR_INVALID_ARG; return out; }
+            out.chains.push_back({FactorIn{nd.operand, -1, t, nd.operand, std::to_string(nd.operand)}});
+            return out;
+        }
+        if (nd.n_children < 1 || nd.first_child < 0 || (int64_t)nd.first_child + nd.n_children > n_children) {
+            err = MOM_ERR_INVALID_ARG;
+            return out;
+        }
+        const int32_t *ch = children + nd.first_child;
+        if (nd.kind == MOM_EXPR_TRANSPOSE) {
+            if (nd.n_children != 1) { err = MOM_ERR_INVALID_ARG; return out; }
+            return run(ch[0], !t, depth + 1);
+        }
+        if (nd.kind == MOM_EXPR_ADD) {
+            for (int i = 0; i < nd.n_children && err == MOM_OK; ++i) {
+                SumIn s = run(ch[i], t, depth + 1);
+                for (auto &c : s.chains) out.chains.push_back(std::move(c));
+            }
+            return out;
+        }
+        if (nd.kind != MOM_EXPR_MUL) { err = MOM_ERR_INVALID_ARG; return out; }
+        std::vector<FactorIn> chain;
+        for (int i = 0; i < nd.n_children && err == MOM_OK; ++i) {
+            SumIn s = run(ch[t ? nd.n_children - 1 - i : i], t, depth + 1);     // (e1*e2)^T = e2^T*e1^T
+            if (err != MOM_OK) break;
+            if (s.chains.size() == 1) {
+                for (auto &f : s.chains[0]) chain.push_back(std::move(f));
+            } else {
+                const std::string key = serialize(s);
+                auto it = known.find(key);
+                int32_t index;
+                if (it != known.end()) index = it->second;
+                else {
+                    index = (int32_t)sums.size();
+                    sums.push_back(std::move(s));
+                    known.emplace(key, index);
+                }
+                chain.push_back(FactorIn{-1, index, false, (int64_t)n_operands + index, std::string()});
+            }
+        }
+        out.chains.push_back(std::move(chain));
+        return out;
+    }
+};
+
+}  // namespace
+
+mom_status_t mom_expression_plan(const mom_matrix_desc_t *operands, int32_t n_operands,
+                                 const mom_expr_node_t *nodes, int32_t n_nodes,
+                                 const int32_t *children, int32_t n_children, int32_t root,
+                                 mom_variant_t variant, mom_plan_t **out_plan) {
+    if (!out_plan || !operands || n_operands < 1 || !nodes || n_nodes < 1 || n_children < 0 || (n_children > 0 && !children))
+        return MOM_ERR_INVALID_ARG;
+    try {
+        Normalizer nz{nodes, n_nodes, children, n_children, n_operands, {}, {}, 0, MOM_OK};
+        SumIn top = nz.run(root, false, 0);
+        if (nz.err != MOM_OK) return nz.err;
+        nz.sums.push_back(std::move(top));
+        std::vector<mom_matrix_desc_t> slots(operands, operands + n_operands);
+        return plan_sums(slots, nz.sums, nullptr, nullptr, nullptr, 0, variant, out_plan);
+    } catch (const std::bad_alloc &) {
+        return MOM_ERR_ALLOC;
+    }
+}
+
+mom_status_t mom_plan_temporaries(const mom_plan_t *plan, int32_t *temporaries) {
+    if (!plan || !temporaries) return MOM_ERR_INVALID_ARG;
+    *temporaries = plan->temporaries;
+    return MOM_OK;
 }
 
 mom_status_t mom_plan_reused_products(const mom_plan_t *plan, int32_t *reused) {
@@ -538,7 +727,7 @@ mom_status_t mom_plan_workspace_bytes(const mom_plan_t *plan, int64_t batch, siz
 mom_status_t mom_plan_host_staging_bytes(const mom_plan_t *plan, int64_t batch, size_t *bytes) {
     if (!plan || !bytes || batch < 1) return MOM_ERR_INVALID_ARG;
     size_t total = 0;
-    for (const auto &d : plan->chain)
+    for (const auto &d : plan->ptr_desc)
         if (d.property != MOM_IDENTITY) total += mom::align_up((size_t)d.rows * d.cols * sizeof(float) * batch, mom::WS_ALIGN);
     for (const auto &d : plan->add)
         if (d.property != MOM_IDENTITY) total += mom::align_up((size_t)d.rows * d.cols * sizeof(float) * batch, mom::WS_ALIGN);

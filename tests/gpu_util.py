@@ -143,3 +143,53 @@ def check_sum_against_oracle(eq: wl.SumEquation, x: np.ndarray, plan, arrays, us
     mask = ov.off_structure_mask(x.shape[0], x.shape[1], prop)
     assert np.all(x.view(np.uint32)[mask] == 0), "off-structure entries must be +0.0f"
     return err
+
+
+def run_expression(ex: wl.Expression, variant: int, via: str = "device"):
+    """Plan and evaluate a nested expression on the GPU; returns (X, plan, operand host arrays)."""
+    arrays = wl.generate_expression(ex)
+    plan = mom.mom_expression_plan(ex.expr, ex.descs(), variant)
+    rd = plan.result_desc()
+    n_out = rd.rows * rd.cols
+    stream = torch.cuda.current_stream().cuda_stream
+    if via == "host":
+        stage_bytes = plan.host_staging_bytes(1)
+        staging = torch.empty(max(stage_bytes, 256), dtype=torch.uint8, device="cuda")
+        pinned = [None if a is None else torch.from_numpy(a).pin_memory() for a in arrays]
+        out = torch.full((n_out,), float("nan"), dtype=torch.float32).pin_memory()
+        plan.execute_host([None if t is None else t.data_ptr() for t in pinned], [], out.data_ptr(), 1,
+                          staging.data_ptr(), stage_bytes, stream)
+        return out.numpy().reshape(rd.rows, rd.cols).copy(), plan, arrays
+    dev = to_device(arrays)
+    ws_bytes = plan.workspace_bytes(1)
+    ws = torch.full((max(ws_bytes, 256) // 4,), float("nan"), dtype=torch.float32, device="cuda")
+    guarded = torch.full((n_out + 2 * CANARY,), float("nan"), dtype=torch.float32, device="cuda")
+    guarded[:CANARY] = 12345.0
+    guarded[-CANARY:] = 12345.0
+    out = guarded[CANARY:CANARY + n_out]
+    plan.execute([None if t is None else t.data_ptr() for t in dev], [], out.data_ptr(),
+                 ws.data_ptr() if ws_bytes else None, ws_bytes, stream)
+    torch.cuda.synchronize()
+    assert plan.device_status() == (0, 0), "a device-side wait timed out"
+    g = guarded.cpu().numpy()
+    assert np.all(g[:CANARY] == 12345.0) and np.all(g[-CANARY:] == 12345.0), "wrote outside the output buffer"
+    return g[CANARY:CANARY + n_out].reshape(rd.rows, rd.cols).copy(), plan, arrays
+
+
+def check_expression_against_oracle(ex: wl.Expression, x: np.ndarray, plan, arrays, tol: float = TOL, sample_rows=None):
+    want = op.plan_expr(ex.expr, ex.descs())
+    assert plan.parenthesization() == want.paren
+    assert plan.flops() == (want.mul_flops, want.add_flops)
+    assert (plan.temporaries(), plan.reused_products()) == (want.temporaries, want.reused)
+    prop = plan.result_desc().property
+    assert prop == want.result_desc.prop
+    assert not np.isnan(x).any(), "part of the output was never written"
+    x_ref, den = ov.evaluate_expr(ex.expr, arrays, ex.descs())
+    if sample_rows is not None:
+        err = ov.normwise_error(x[sample_rows], x_ref[sample_rows], den[sample_rows])
+    else:
+        err = ov.normwise_error(x, x_ref, den)
+    assert err <= tol, f"normwise error {err:.3e} > {tol:.1e} ({ex.name})"
+    mask = ov.off_structure_mask(x.shape[0], x.shape[1], prop)
+    assert np.all(x.view(np.uint32)[mask] == 0), "off-structure entries must be +0.0f"
+    return err

@@ -224,3 +224,74 @@ def test_sum_plan_errors(chains, names, status, code):
         with pytest.raises(op.OracleError) as oe:
             op.plan_sum(chains, (), names or ())
         assert oe.value.code == code
+
+
+# ---- nested expressions -------------------------------------------------------------------------------
+
+def assert_same_expression_plan(expr, operands, variant=mom.VARIANT_3XTF32):
+    want = op.plan_expr(expr, operands)
+    got = mom.mom_expression_plan(expr, operands, variant)
+    assert got.parenthesization() == want.paren
+    assert got.flops() == (want.mul_flops, want.add_flops)
+    assert (got.temporaries(), got.reused_products()) == (want.temporaries, want.reused)
+    rd = got.result_desc()
+    assert (rd.rows, rd.cols, rd.property) == (want.result_desc.rows, want.result_desc.cols, want.result_desc.prop)
+    assert [(s.m, s.n, s.k, s.lhs_property, s.rhs_property, s.out_property, s.useful_mults) for s in got.steps()] == list(want.products)
+    return got, want
+
+
+def test_random_expressions_match_the_oracle():
+    nested = 0
+    for seed in range(500):
+        ex = wl.random_expression(seed)
+        _, want = assert_same_expression_plan(ex.expr, ex.descs())
+        nested += want.temporaries > 0
+    assert nested >= 100
+
+
+def test_expression_plan_examples():
+    G, L = mom.GENERAL, mom.LOWER_TRI
+    ops = [(10, 10, G)] * 3
+    got, _ = assert_same_expression_plan(("mul", [0, ("add", [1, 2])]), ops)
+    assert got.parenthesization() == "(0*[1+2])" and got.num_steps() == 1 and got.temporaries() == 1
+    # the same nested sum twice is one temporary; a product of the temporary is shared like any other
+    e = ("add", [("mul", [0, ("add", [1, 2]), 0]), ("mul", [0, ("add", [1, 2]), 1])])
+    got, want = assert_same_expression_plan(e, ops)
+    assert got.temporaries() == 1
+    # flattening and transposes
+    got, _ = assert_same_expression_plan(("t", ("mul", [("mul", [0, 1]), ("t", 2)])), ops)
+    assert got.parenthesization() == "(2*(1^T*0^T))"
+    assert_same_expression_plan(("mul", [0, ("add", [1, 2])]), [(10, 10, L)] * 3)
+    assert_same_expression_plan(wl.config_expression().expr, wl.config_expression().descs())
+
+
+@pytest.mark.parametrize("expr,operands,status,code", [
+    (("mul", [0, ("add", [1, 2])]), [(4, 5, 0), (5, 6, 0), (6, 5, 0)], mom.ERR_SHAPE_MISMATCH, "shape_mismatch"),
+    (("mul", [0, 7]), [(4, 5, 0)], mom.ERR_INVALID_ARG, "invalid_arg"),
+    (("add", []), [(4, 5, 0)], mom.ERR_INVALID_ARG, "invalid_arg"),
+    (("add", [0, ("t", 0)]), [(4, 5, 0)], mom.ERR_SHAPE_MISMATCH, "shape_mismatch"),
+])
+def test_expression_plan_errors(expr, operands, status, code):
+    with pytest.raises(mom.MomError) as e:
+        mom.mom_expression_plan(expr, operands)
+    assert e.value.status == status
+    with pytest.raises(op.OracleError) as oe:
+        op.plan_expr(expr, operands)
+    assert oe.value.code == code
+
+
+def test_expression_node_arrays_are_validated():
+    ops = mom._desc_array([(4, 4, 0)])
+    handle = ctypes.c_void_p()
+    lib = mom._lib
+    cyc = (mom.ExprNode * 1)(mom.ExprNode(mom.EXPR_TRANSPOSE, 0, 0, 1))          # a node that is its own child
+    kids = (ctypes.c_int32 * 1)(0)
+    assert lib.mom_expression_plan(ops, 1, cyc, 1, kids, 1, 0, 0, ctypes.byref(handle)) == mom.ERR_INVALID_ARG
+    bad = (mom.ExprNode * 1)(mom.ExprNode(mom.EXPR_MUL, 0, 0, 3))                # children out of range
+    assert lib.mom_expression_plan(ops, 1, bad, 1, kids, 1, 0, 0, ctypes.byref(handle)) == mom.ERR_INVALID_ARG
+    unk = (mom.ExprNode * 1)(mom.ExprNode(9, 0, 0, 1))
+    assert lib.mom_expression_plan(ops, 1, unk, 1, kids, 1, 0, 0, ctypes.byref(handle)) == mom.ERR_INVALID_ARG
+    leaf = (mom.ExprNode * 1)(mom.ExprNode(mom.EXPR_OPERAND, 0, 0, 0))
+    assert lib.mom_expression_plan(ops, 1, leaf, 1, kids, 0, 5, 0, ctypes.byref(handle)) == mom.ERR_INVALID_ARG
+    assert lib.mom_expression_plan(ops, 1, leaf, 1, kids, 0, 0, 0, ctypes.byref(handle)) == mom.OK
+    lib.mom_plan_destroy(handle)

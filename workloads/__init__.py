@@ -324,3 +324,75 @@ def config_sum_triangular(n: int = 4096, seed: int = 8) -> SumEquation:
     return SumEquation(f"LA_plus_BU_plus_C_{n}", seed,
                        ((Operand(n, n, LOWER_TRI), g), (g, Operand(n, n, UPPER_TRI)), (g,)),
                        ((False, False), (False, False), (False,)), ((0, 1), (2, 3), (4,)))
+
+
+# --------------------------------------------------------------------------
+# Nested expressions: an operand index, ("t", e), ("mul", [e, ...]) or
+# ("add", [e, ...]) over a table of operands (paper Section 2, "Operations").
+# --------------------------------------------------------------------------
+
+@dataclass(frozen=True)
+class Expression:
+    name: str
+    seed: int
+    operands: Sequence[Operand]
+    expr: object
+
+    def descs(self):
+        return [(o.rows, o.cols, o.prop) for o in self.operands]
+
+
+def generate_expression(ex: Expression):
+    """Stored float32 arrays of the operand table (None for Identity)."""
+    return [generate_operand(o, ex.seed, i) for i, o in enumerate(ex.operands)]
+
+
+def random_expression(seed: int, max_depth: int = 3, max_dim: int = 40, dim_multiple: int = 1) -> Expression:
+    """Random well-formed nested expression; operands are reused where an existing one has the needed type."""
+    rng = np.random.Generator(np.random.Philox(key=[int(seed), 0xE4B8]))
+    operands: List[Operand] = []
+
+    def dim():
+        return int(rng.integers(1, max_dim // dim_multiple + 1)) * dim_multiple
+
+    def leaf(r, c):
+        t = bool(rng.integers(0, 4) == 0)
+        sr, sc = (c, r) if t else (r, c)
+        same = [i for i, o in enumerate(operands) if (o.rows, o.cols) == (sr, sc)]
+        if same and rng.random() < 0.5:
+            i = int(rng.choice(same))
+        else:
+            kind = int(rng.integers(0, 7))
+            prop = {0: LOWER_TRI, 1: UPPER_TRI, 2: IDENTITY}.get(kind, GENERAL) if sr == sc else GENERAL
+            operands.append(Operand(sr, sc, prop, "normal" if kind == 3 else "uniform"))
+            i = len(operands) - 1
+        return ("t", i) if t else i
+
+    def gen(r, c, depth):
+        kind = int(rng.integers(0, 10)) if depth > 0 else 0
+        if kind <= 2:
+            return leaf(r, c)
+        if kind <= 5:
+            n = int(rng.integers(2, 4))
+            inner = [r] + [r if rng.random() < 0.3 else dim() for _ in range(n - 1)] + [c]
+            return ("mul", [gen(inner[i], inner[i + 1], depth - 1) for i in range(n)])
+        if kind <= 8:
+            return ("add", [gen(r, c, depth - 1) for _ in range(int(rng.integers(2, 4)))])
+        return ("t", gen(c, r, depth - 1))
+
+    r = dim()
+    c = r if rng.random() < 0.4 else dim()
+    top = int(rng.integers(0, 3))
+    if top == 0:
+        expr = ("mul", [gen(r, r, max_depth - 1), ("add", [gen(r, c, max_depth - 2), gen(r, c, max_depth - 2)])])
+    else:
+        expr = gen(r, c, max_depth)
+    return Expression(f"random_expr_{seed}", seed, tuple(operands), expr)
+
+
+def config_expression(n: int = 4096, seed: int = 9) -> Expression:
+    """X = (A + L) * (B + C^T) * U + D:  two nested sums, one chain of three factors, one Add term."""
+    g = Operand(n, n, GENERAL, "normal", 1.0 / np.sqrt(n))
+    ops = (g, Operand(n, n, LOWER_TRI), g, g, Operand(n, n, UPPER_TRI), g)
+    expr = ("add", [("mul", [("add", [0, 1]), ("add", [2, ("t", 3)]), 4]), 5])
+    return Expression(f"ApL_times_BpCt_times_U_plus_D_{n}", seed, ops, expr)
