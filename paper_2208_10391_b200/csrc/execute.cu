@@ -1,4 +1,5 @@
 // Launcher: walks a plan's steps and enqueues the kernels on the caller's stream.
+#include <algorithm>
 #include <cstdio>
 #include <cstring>
 #include <new>
@@ -18,7 +19,15 @@ struct DeviceState {
     // step timing: a ring of TIMING_SLOTS executes, 3 events per step (before pre-pass, before product, after)
     std::vector<cudaEvent_t> events;
     long long timed_executes = 0;       // executes recorded since timing was enabled
+    // host-staging entry point: uploads run on a stream of their own, one event per operand, so that the first
+    // products start while later operands are still on their way
+    cudaStream_t copy_stream = nullptr;
+    cudaEvent_t call_start = nullptr;
+    std::vector<cudaEvent_t> slot_ready, add_ready;
 };
+
+// events the launcher has to wait for before it first uses an operand (host-staging entry point only)
+struct StageEvents { const cudaEvent_t *slot; const cudaEvent_t *add; };
 
 constexpr int TIMING_SLOTS = 32;
 
@@ -29,6 +38,10 @@ void destroy_device_state(DeviceState *d) {
     if (d->device >= 0) cudaSetDevice(d->device);
     tc_release(d->tc);
     for (cudaEvent_t e : d->events) cudaEventDestroy(e);
+    for (cudaEvent_t e : d->slot_ready) cudaEventDestroy(e);
+    for (cudaEvent_t e : d->add_ready) cudaEventDestroy(e);
+    if (d->call_start) cudaEventDestroy(d->call_start);
+    if (d->copy_stream) cudaStreamDestroy(d->copy_stream);
     if (d->status) cudaFree(d->status);
     if (prev >= 0) cudaSetDevice(prev);
     delete d;
@@ -64,7 +77,8 @@ struct Operand { const float *ptr; long long stride; };
 
 mom_status_t execute_impl(const mom_plan *p, const float *const *chain_ptrs, const int64_t *chain_strides,
                           const float *const *add_ptrs, const int64_t *add_strides, float *out, int64_t out_stride,
-                          int64_t batch, void *workspace, size_t workspace_bytes, cudaStream_t stream) {
+                          int64_t batch, void *workspace, size_t workspace_bytes, cudaStream_t stream,
+                          const StageEvents *staged = nullptr) {
     if (!p || !chain_ptrs || !out || batch < 1) return MOM_ERR_INVALID_ARG;
     const int n_chain = (int)p->chain.size(), n_add = (int)p->add.size(), n_ptrs = (int)p->ptr_desc.size();
     if (n_add > 0 && !add_ptrs) return MOM_ERR_INVALID_ARG;
@@ -72,7 +86,7 @@ mom_status_t execute_impl(const mom_plan *p, const float *const *chain_ptrs, con
     const int64_t rows = p->result_desc.rows, cols = p->result_desc.cols;
 
     for (int i = 0; i < n_ptrs; ++i) {
-        if (p->ptr_desc[i].property == MOM_IDENTITY) continue;
+        if (p->ptr_desc[i].property == MOM_IDENTITY || !p->slot_used[i]) continue;
         if (!chain_ptrs[i]) return MOM_ERR_INVALID_ARG;
         if (!aligned16(chain_ptrs[i])) return MOM_ERR_ALIGNMENT;
         if (batch > 1 && (chain_strides[i] % 4 != 0 || chain_strides[i] < p->ptr_desc[i].rows * p->ptr_desc[i].cols))
@@ -81,7 +95,7 @@ mom_status_t execute_impl(const mom_plan *p, const float *const *chain_ptrs, con
     if (!p->names.empty()) {          // entries with one name are one matrix: a product shared between chains relies on it
         for (int i = 0; i < n_ptrs; ++i)
             for (int j = 0; j < i; ++j)
-                if (p->names[i] == p->names[j] && p->ptr_desc[i].property != MOM_IDENTITY &&
+                if (p->names[i] == p->names[j] && p->ptr_desc[i].property != MOM_IDENTITY && p->slot_used[i] && p->slot_used[j] &&
                     (chain_ptrs[i] != chain_ptrs[j] || (batch > 1 && chain_strides[i] != chain_strides[j])))
                     return MOM_ERR_INVALID_ARG;
     }
@@ -114,7 +128,28 @@ mom_status_t execute_impl(const mom_plan *p, const float *const *chain_ptrs, con
         if (st != MOM_OK) return st;
     }
 
+    // operands that are still being uploaded: wait (on the stream) before the first launch that reads them
+    std::vector<char> slot_waited(n_ptrs, 0), add_waited(n_add, 0);
+    auto need_slot = [&](int slot) {
+        if (!staged || slot < 0 || slot_waited[slot] || p->ptr_desc[slot].property == MOM_IDENTITY || !p->slot_used[slot]) return;
+        slot_waited[slot] = 1;
+        cudaStreamWaitEvent(stream, staged->slot[slot], 0);
+    };
+    auto need_value = [&](int id) { if (id < n_chain) need_slot(p->factor_ptr[id]); };
+    auto need_summands = [&](const SumInfo &sum) {
+        if (!staged) return;
+        for (const Summand &sm : sum.summands) {
+            if (sm.kind == SUM_FACTOR) need_value(sm.index);
+            if (sm.kind == SUM_TERM && !add_waited[sm.index] && p->add[sm.index].property != MOM_IDENTITY) {
+                add_waited[sm.index] = 1;
+                cudaStreamWaitEvent(stream, staged->add[sm.index], 0);
+            }
+        }
+    };
+
     if (p->fused_ok) {
+        for (int i = 0; i < n_ptrs; ++i) need_slot(i);
+        need_summands(p->sums.back());
         FusedPlan fp;
         std::memset(&fp, 0, sizeof(fp));
         fp.n_ops = (int)p->kept.size();
@@ -225,6 +260,7 @@ mom_status_t execute_impl(const mom_plan *p, const float *const *chain_ptrs, con
             int added = 0;
 
             if (!has_products) {
+                need_summands(sum);
                 // value = first summand + the following ones
                 const Summand &sm = *simple[0];
                 AddTerms t;
@@ -254,6 +290,9 @@ mom_status_t execute_impl(const mom_plan *p, const float *const *chain_ptrs, con
                     if (prod.out_off == SIZE_MAX) return Operand{nullptr, elems};
                     return Operand{reinterpret_cast<const float *>(ws + prod.out_off * (size_t)nb), elems};
                 };
+                need_value(stp.pub.lhs);
+                need_value(stp.pub.rhs);
+                if (stp.is_last && !stp.accumulate) need_summands(sum);
                 const Operand A = value(stp.pub.lhs), B = value(stp.pub.rhs);
                 ProductArgs a;
                 std::memset(&a, 0, sizeof(a));
@@ -349,37 +388,80 @@ mom_status_t mom_equation_execute_host(const mom_plan_t *plan, const float *cons
     const int n_chain = (int)plan->ptr_desc.size(), n_add = (int)plan->add.size();
     if (n_add > 0 && !add_host) return MOM_ERR_INVALID_ARG;
 
+    int device = 0;
+    mom_status_t est = mom::check_arch(&device);
+    if (est != MOM_OK) return est;
+    est = mom::ensure_device_state(plan, device);
+    if (est != MOM_OK) return est;
+    mom::DeviceState *dev = plan->dev;
+    if (!dev->copy_stream) {
+        if (cudaStreamCreateWithFlags(&dev->copy_stream, cudaStreamNonBlocking) != cudaSuccess) return MOM_ERR_CUDA;
+        if (cudaEventCreateWithFlags(&dev->call_start, cudaEventDisableTiming) != cudaSuccess) return MOM_ERR_CUDA;
+    }
+    while ((int)dev->slot_ready.size() < n_chain || (int)dev->add_ready.size() < n_add) {
+        cudaEvent_t e = nullptr;
+        if (cudaEventCreateWithFlags(&e, cudaEventDisableTiming) != cudaSuccess) return MOM_ERR_CUDA;
+        ((int)dev->slot_ready.size() < n_chain ? dev->slot_ready : dev->add_ready).push_back(e);
+    }
+    // uploads start once the caller's stream has reached this call (the staging area may still be in use before)
+    if (cudaEventRecord(dev->call_start, stream) != cudaSuccess) return MOM_ERR_CUDA;
+    if (cudaStreamWaitEvent(dev->copy_stream, dev->call_start, 0) != cudaSuccess) return MOM_ERR_CUDA;
+
     char *cur = static_cast<char *>(staging);
     std::vector<const float *> cptr(n_chain, nullptr), aptr(n_add, nullptr);
     std::vector<int64_t> cstride(n_chain, 0), astride(n_add, 0);
-    auto stage = [&](const mom_matrix_desc_t &d, const float *host, const float **dev, int64_t *stride) -> mom_status_t {
-        if (d.property == MOM_IDENTITY) return MOM_OK;
-        if (!host) return MOM_ERR_INVALID_ARG;
-        const size_t bytes = (size_t)d.rows * d.cols * sizeof(float) * batch;
-        if (cudaMemcpyAsync(cur, host, bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess) return MOM_ERR_CUDA;
-        *dev = reinterpret_cast<const float *>(cur);
-        *stride = d.rows * d.cols;
-        cur += mom::align_up(bytes, mom::WS_ALIGN);
-        return MOM_OK;
-    };
-    for (int i = 0; i < n_chain; ++i) {
-        int same = -1;                                 // a named matrix is copied once
-        if (!plan->names.empty())
-            for (int j = 0; j < i && same < 0; ++j)
-                if (plan->names[j] == plan->names[i]) same = j;
-        if (same >= 0) {
-            if (chain_host[i] != chain_host[same]) return MOM_ERR_INVALID_ARG;
-            cptr[i] = cptr[same];
-            cstride[i] = cstride[same];
+    std::vector<size_t> cbytes(n_chain, 0);
+    std::vector<int> same_as(n_chain, -1);
+    for (int i = 0; i < n_chain; ++i) {                  // addresses in the staging area, in the order given
+        const mom_matrix_desc_t &d = plan->ptr_desc[i];
+        if (d.property == MOM_IDENTITY) continue;
+        if (!plan->names.empty())                        // a named matrix is copied once
+            for (int j = 0; j < i && same_as[i] < 0; ++j)
+                if (plan->names[j] == plan->names[i]) same_as[i] = j;
+        if (same_as[i] >= 0) {
+            if (chain_host[i] != chain_host[same_as[i]]) return MOM_ERR_INVALID_ARG;
+            cptr[i] = cptr[same_as[i]];
+            cstride[i] = cstride[same_as[i]];
             continue;
         }
-        mom_status_t st = stage(plan->ptr_desc[i], chain_host[i], &cptr[i], &cstride[i]);
-        if (st != MOM_OK) return st;
+        if (!plan->slot_used[i]) continue;               // an operand no factor refers to is not uploaded
+        if (!chain_host[i]) return MOM_ERR_INVALID_ARG;
+        cbytes[i] = (size_t)d.rows * d.cols * sizeof(float) * batch;
+        cptr[i] = reinterpret_cast<const float *>(cur);
+        cstride[i] = d.rows * d.cols;
+        cur += mom::align_up(cbytes[i], mom::WS_ALIGN);
+    }
+    // upload in the order of first use by the plan's products, so that the first products can start early
+    std::vector<int> first_use(n_chain, (int)plan->steps.size());
+    for (size_t s = 0; s < plan->steps.size(); ++s)
+        for (int32_t v : {plan->steps[s].pub.lhs, plan->steps[s].pub.rhs})
+            if (v < (int32_t)plan->factor_ptr.size() && plan->factor_ptr[v] >= 0)
+                first_use[plan->factor_ptr[v]] = std::min(first_use[plan->factor_ptr[v]], (int)s);
+    for (int i = 0; i < n_chain; ++i)                    // a matrix given under several entries is needed when the first is
+        if (same_as[i] >= 0) first_use[same_as[i]] = std::min(first_use[same_as[i]], first_use[i]);
+    std::vector<int> order(n_chain);
+    for (int i = 0; i < n_chain; ++i) order[i] = i;
+    std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return first_use[a] < first_use[b]; });
+    for (int i : order) {
+        if (same_as[i] >= 0) continue;
+        if (cbytes[i] && cudaMemcpyAsync(const_cast<float *>(cptr[i]), chain_host[i], cbytes[i], cudaMemcpyHostToDevice, dev->copy_stream) != cudaSuccess)
+            return MOM_ERR_CUDA;
+        if (cudaEventRecord(dev->slot_ready[i], dev->copy_stream) != cudaSuccess) return MOM_ERR_CUDA;
+        for (int j = i + 1; j < n_chain; ++j)
+            if (same_as[j] == i && cudaEventRecord(dev->slot_ready[j], dev->copy_stream) != cudaSuccess) return MOM_ERR_CUDA;
     }
     for (int i = 0; i < n_add; ++i) {
-        mom_status_t st = stage(plan->add[i], add_host[i], &aptr[i], &astride[i]);
-        if (st != MOM_OK) return st;
+        const mom_matrix_desc_t &d = plan->add[i];
+        if (d.property == MOM_IDENTITY) continue;
+        if (!add_host[i]) return MOM_ERR_INVALID_ARG;
+        const size_t bytes = (size_t)d.rows * d.cols * sizeof(float) * batch;
+        if (cudaMemcpyAsync(cur, add_host[i], bytes, cudaMemcpyHostToDevice, dev->copy_stream) != cudaSuccess) return MOM_ERR_CUDA;
+        if (cudaEventRecord(dev->add_ready[i], dev->copy_stream) != cudaSuccess) return MOM_ERR_CUDA;
+        aptr[i] = reinterpret_cast<const float *>(cur);
+        astride[i] = d.rows * d.cols;
+        cur += mom::align_up(bytes, mom::WS_ALIGN);
     }
+    const mom::StageEvents staged{dev->slot_ready.data(), dev->add_ready.data()};
     float *x = reinterpret_cast<float *>(cur);
     const int64_t xelems = plan->result_desc.rows * plan->result_desc.cols;
     const size_t xbytes = (size_t)xelems * sizeof(float) * batch;
@@ -393,9 +475,9 @@ mom_status_t mom_equation_execute_host(const mom_plan_t *plan, const float *cons
     for (int i = 0; i < n_add; ++i) strides_ok &= astride[i] % 4 == 0;
     mom_status_t st = MOM_OK;
     if (batch == 1) {
-        st = mom::execute_impl(plan, cptr.data(), nullptr, aptr.data(), nullptr, x, 0, 1, cur, ws_bytes, stream);
+        st = mom::execute_impl(plan, cptr.data(), nullptr, aptr.data(), nullptr, x, 0, 1, cur, ws_bytes, stream, &staged);
     } else if (strides_ok) {
-        st = mom::execute_impl(plan, cptr.data(), cstride.data(), aptr.data(), astride.data(), x, xelems, batch, cur, ws_bytes, stream);
+        st = mom::execute_impl(plan, cptr.data(), cstride.data(), aptr.data(), astride.data(), x, xelems, batch, cur, ws_bytes, stream, &staged);
     } else {
         return MOM_ERR_ALIGNMENT;
     }

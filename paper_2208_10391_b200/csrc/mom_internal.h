@@ -73,6 +73,7 @@ struct mom_plan {
     std::vector<int32_t> factor_ptr;           // per factor: index into the caller's pointer array; -1 for a temporary
     std::vector<int32_t> factor_sum;           // per factor: the nested sum whose temporary it is; -1 for a stored matrix
     std::vector<mom_matrix_desc_t> ptr_desc;   // per entry of the caller's pointer array: the matrix as stored
+    std::vector<char> slot_used;               // per entry: some factor refers to it (an unused operand may be NULL)
     std::vector<mom_matrix_desc_t> add;
     std::vector<char> chain_t, add_t;          // operand enters transposed: stored shape is (cols x rows) of the entry above
     std::vector<int32_t> chain_begin;          // factors of chain c are [chain_begin[c], chain_begin[c + 1])

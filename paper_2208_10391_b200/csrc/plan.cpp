@@ -356,6 +356,9 @@ static mom_status_t plan_sums(const std::vector<mom_matrix_desc_t> &slots, const
             }
             p->sums.push_back(std::move(info));
         }
+        p->slot_used.assign(slots.size(), 0);
+        for (int32_t f : p->factor_ptr)
+            if (f >= 0) p->slot_used[f] = 1;
         p->paren = sum_text.back();
         p->result_desc = p->sums.back().desc;
         p->temporaries = (int32_t)p->sums.size() - 1;
