@@ -20,7 +20,11 @@ Readings taken where the paper is silent (each also listed in the design notes):
     structurally non-zero (non-strict triangles: the diagonal is an ordinary entry);
   * Identity operands are removed before the enumeration and never appear in the result string;
   * ties: the tree whose pre-order list of split positions is lexicographically smallest;
-  * property of a product = join in  Identity < {lowerTri, upperTri} < general;
+  * property of a product = join in  Identity < Diagonal < {lowerTri, upperTri} < general;
+  * Diagonal (one of the "more properties" the paper's conclusion announces; the paper prints no rule
+    for it): a square matrix stored densely whose entries off the diagonal are zero.  Unlike Identity
+    its diagonal is data, so it is never simplified away; D*A costs one multiplication per structural
+    entry of A; the transpose of a Diagonal matrix is Diagonal;
   * a transposed operand (paper Table 1, "Transpose") takes part with its transposed type: shape
     swapped and lowerTri <-> upperTri (the inference rule the paper prints);
   * reported mul_flops = 2 * multiplications; add_flops = structural non-zeros of the Add terms.
@@ -32,7 +36,8 @@ from __future__ import annotations
 from dataclasses import dataclass
 from typing import List, Optional, Sequence, Tuple
 
-GENERAL, LOWER_TRI, UPPER_TRI, IDENTITY = 0, 1, 2, 3
+GENERAL, LOWER_TRI, UPPER_TRI, IDENTITY, DIAGONAL = 0, 1, 2, 3, 4
+PROPERTIES = (GENERAL, LOWER_TRI, UPPER_TRI, IDENTITY, DIAGONAL)
 
 
 class OracleError(ValueError):
@@ -88,7 +93,7 @@ def in_structure(prop: int, i: int, j: int) -> bool:
         return i >= j
     if prop == UPPER_TRI:
         return i <= j
-    if prop == IDENTITY:
+    if prop in (IDENTITY, DIAGONAL):
         return i == j
     raise OracleError("property", f"unknown property {prop}")
 
@@ -103,7 +108,7 @@ def structural_nonzeros(d: Desc) -> int:
         return d.rows * d.cols
     if d.prop in (LOWER_TRI, UPPER_TRI):
         return d.rows * (d.rows + 1) // 2
-    return d.rows
+    return d.rows                   # Identity, Diagonal
 
 
 def brute_force_mults(a: Desc, b: Desc) -> int:
@@ -127,6 +132,10 @@ def product_mults(a: Desc, b: Desc) -> int:
     tb = b.prop in (LOWER_TRI, UPPER_TRI)
     if a.prop == IDENTITY or b.prop == IDENTITY:
         return 0
+    if a.prop == DIAGONAL:         # row l of B is scaled by d_l: one multiplication per structural entry of B
+        return structural_nonzeros(b)
+    if b.prop == DIAGONAL:         # column l of A is scaled by d_l
+        return structural_nonzeros(a)
     if not ta and not tb:
         return a.rows * a.cols * b.cols
     if ta and not tb:
@@ -142,12 +151,16 @@ def product_mults(a: Desc, b: Desc) -> int:
 
 
 def join(p: int, q: int) -> int:
-    """Property of a product: least upper bound in Identity < {lowerTri, upperTri} < general."""
+    """Property of a product: least upper bound in Identity < Diagonal < {lowerTri, upperTri} < general."""
     if p == IDENTITY:
         return q
     if q == IDENTITY:
         return p
     if p == q:
+        return p
+    if p == DIAGONAL:
+        return q
+    if q == DIAGONAL:
         return p
     return GENERAL
 
@@ -156,17 +169,14 @@ def sum_property(product_prop: int, add_props: Sequence[int]) -> int:
     """Property of (chain value) + T1 + ... + Tk.  With no terms it is the product's own property.
 
     A sum with at least one term is never typed Identity (I + I = 2I): an Identity summand counts
-    through its footprint, which fits either triangle.  All-Identity sums are reported lowerTri.
+    through its footprint, the diagonal, so it is joined as a Diagonal matrix.  The result is the
+    least type that holds every summand's footprint: Diagonal < {lowerTri, upperTri} < general.
     """
     if not add_props:
         return product_prop
-    props = [product_prop] + list(add_props)
-    concrete = [p for p in props if p != IDENTITY]
-    if not concrete:
-        return LOWER_TRI
-    out = concrete[0]
-    for p in concrete[1:]:
-        out = p if p == out else GENERAL
+    out = DIAGONAL
+    for p in [product_prop] + list(add_props):
+        out = join(out, DIAGONAL if p == IDENTITY else p)
     return out
 
 
@@ -180,10 +190,10 @@ def _validate(chain: Sequence[Desc], add: Sequence[Desc]) -> None:
     for d in list(chain) + list(add):
         if d.rows < 1 or d.cols < 1:
             raise OracleError("invalid_arg", "non-positive dimension")
-        if d.prop not in (GENERAL, LOWER_TRI, UPPER_TRI, IDENTITY):
+        if d.prop not in PROPERTIES:
             raise OracleError("property", "unknown property")
         if d.prop != GENERAL and d.rows != d.cols:
-            raise OracleError("property", "triangular / Identity matrices are square")
+            raise OracleError("property", "triangular / Diagonal / Identity matrices are square")
     for a, b in zip(chain[:-1], chain[1:]):
         if a.cols != b.rows:
             raise OracleError("shape_mismatch", "inner dimensions differ")
@@ -237,8 +247,8 @@ def _paren(tree, kept: Sequence[int], transposed: Sequence[bool] = ()) -> str:
 
 def transpose_desc(d: Desc) -> Desc:
     """Type of A^T given the type of A: shape swapped; paper Section 2, "Transformations", prints the
-    inference rule lowerTriangular(A) -> upperTriangular(A^T) (and symmetrically); general and Identity
-    keep their property."""
+    inference rule lowerTriangular(A) -> upperTriangular(A^T) (and symmetrically); general, Diagonal and
+    Identity keep their property."""
     prop = {LOWER_TRI: UPPER_TRI, UPPER_TRI: LOWER_TRI}.get(d.prop, d.prop)
     return Desc(d.cols, d.rows, prop)
 
@@ -253,7 +263,7 @@ def plan(chain: Sequence[Tuple[int, int, int]], add: Sequence[Tuple[int, int, in
     stored_c = [Desc(*c) for c in chain]
     stored_a = [Desc(*a) for a in add]
     for d in stored_c + stored_a:               # the stored matrices must be well-typed themselves
-        if d.prop not in (GENERAL, LOWER_TRI, UPPER_TRI, IDENTITY):
+        if d.prop not in PROPERTIES:
             raise OracleError("property", "unknown property")
     tc = list(chain_transposed) + [False] * (len(stored_c) - len(chain_transposed))
     ta = list(add_transposed) + [False] * (len(stored_a) - len(add_transposed))

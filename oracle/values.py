@@ -18,7 +18,7 @@ from typing import List, Optional, Sequence, Tuple
 
 import numpy as np
 
-GENERAL, LOWER_TRI, UPPER_TRI, IDENTITY = 0, 1, 2, 3
+GENERAL, LOWER_TRI, UPPER_TRI, IDENTITY, DIAGONAL = 0, 1, 2, 3, 4
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "matmul_f64.c")
@@ -93,7 +93,7 @@ def transposed_operands(arrays, descs, flags):
     """Operands as the equation uses them: entry i transposed (array and descriptor) where flags[i] is set.
 
     The transpose of a stored lowerTri matrix is upperTri and vice versa (the paper's printed inference
-    rule); Identity and general keep their property.  Dense storage is simply transposed with NumPy.
+    rule); Identity, Diagonal and general keep their property.  Dense storage is simply transposed with NumPy.
     """
     swap = {LOWER_TRI: UPPER_TRI, UPPER_TRI: LOWER_TRI}
     out_a, out_d = [], []
@@ -231,7 +231,7 @@ def off_structure_mask(rows: int, cols: int, prop: int, row_index: Optional[np.n
         return i < j
     if prop == UPPER_TRI:
         return i > j
-    if prop == IDENTITY:
+    if prop in (IDENTITY, DIAGONAL):
         return i != j
     raise ValueError("unknown property")
 

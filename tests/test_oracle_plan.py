@@ -10,7 +10,7 @@ import pytest
 
 from conftest import golden
 from oracle import plan as op
-from oracle.plan import GENERAL as G, LOWER_TRI as L, UPPER_TRI as U, IDENTITY as I, Desc
+from oracle.plan import GENERAL as G, LOWER_TRI as L, UPPER_TRI as U, IDENTITY as I, DIAGONAL as D, Desc
 import workloads as wl
 
 
@@ -58,7 +58,7 @@ def test_listing2_product_is_typed_lower_triangular():
 
 
 # ---------------------------------------------------------------- cost model
-@pytest.mark.parametrize("pa,pb", list(itertools.product([G, L, U], repeat=2)))
+@pytest.mark.parametrize("pa,pb", list(itertools.product([G, L, U, D], repeat=2)))
 def test_closed_form_mults_equal_brute_force_count(pa, pb):
     for n in range(1, 8):
         shapes = [(n, n, n)]
@@ -79,7 +79,7 @@ def test_closed_form_mults_equal_brute_force_count(pa, pb):
 
 def test_brute_force_count_against_dense_indicator_product():
     # the count of useful multiplications equals the sum of entries of S(A) * S(B) (0/1 matrices)
-    for pa, pb in itertools.product([G, L, U], repeat=2):
+    for pa, pb in itertools.product([G, L, U, D], repeat=2):
         n = 6
         sa = np.array([[op.in_structure(pa, i, j) for j in range(n)] for i in range(n)], dtype=np.int64)
         sb = np.array([[op.in_structure(pb, i, j) for j in range(n)] for i in range(n)], dtype=np.int64)
@@ -87,7 +87,7 @@ def test_brute_force_count_against_dense_indicator_product():
 
 
 def test_structural_nonzeros():
-    for prop in (G, L, U, I):
+    for prop in (G, L, U, I, D):
         for n in (1, 2, 5, 9):
             d = Desc(n, n, prop)
             assert op.structural_nonzeros(d) == op.brute_force_nonzeros(d)
@@ -102,7 +102,9 @@ def test_identity_costs_nothing_and_join_rules():
     assert op.join(G, L) == G and op.join(U, G) == G
     assert op.join(I, L) == L and op.join(U, I) == U and op.join(I, I) == I
     # join is associative and commutative, so a sub-chain's property does not depend on its tree
-    for a, b, c in itertools.product([G, L, U, I], repeat=3):
+    assert op.join(D, D) == D and op.join(D, L) == L and op.join(U, D) == U and op.join(D, G) == G
+    assert op.join(I, D) == D and op.join(D, I) == D
+    for a, b, c in itertools.product([G, L, U, I, D], repeat=3):
         assert op.join(op.join(a, b), c) == op.join(a, op.join(b, c))
         assert op.join(a, b) == op.join(b, a)
 
@@ -111,7 +113,7 @@ def test_product_structure_rule_matches_boolean_products():
     # the structure of a product of 0/1 structure matrices is inside the joined property's structure,
     # and fills it completely
     n = 5
-    for pa, pb in itertools.product([G, L, U, I], repeat=2):
+    for pa, pb in itertools.product([G, L, U, I, D], repeat=2):
         sa = np.array([[op.in_structure(pa, i, j) for j in range(n)] for i in range(n)], dtype=np.int64)
         sb = np.array([[op.in_structure(pb, i, j) for j in range(n)] for i in range(n)], dtype=np.int64)
         got = (sa @ sb) > 0
@@ -248,7 +250,13 @@ def test_sum_property():
     assert op.plan([(4, 4, L), (4, 4, L)], [(4, 4, L)]).result_desc.prop == L
     assert op.plan([(4, 4, L), (4, 4, L)], [(4, 4, U)]).result_desc.prop == G
     assert op.plan([(4, 4, L), (4, 4, L)], [(4, 4, I)]).result_desc.prop == L
-    assert op.plan([(4, 4, I)], [(4, 4, I)]).result_desc.prop == L
+    assert op.plan([(4, 4, I)], [(4, 4, I)]).result_desc.prop == D       # I + I = 2I: a diagonal matrix
+    assert op.plan([(4, 4, D)], [(4, 4, I)]).result_desc.prop == D
+    assert op.plan([(4, 4, D)], [(4, 4, L)]).result_desc.prop == L
+    assert op.plan([(4, 4, D), (4, 4, U)], [(4, 4, D)]).result_desc.prop == U
+    assert op.plan([(4, 4, L)], [(4, 4, D), (4, 4, U)]).result_desc.prop == G
+    assert op.plan([(4, 4, D)], []).result_desc.prop == D
+    assert op.plan([(4, 4, U)], [(4, 4, D)]).add_flops == 4
     assert op.plan([(4, 4, I)], [(4, 4, U), (4, 4, I)]).result_desc.prop == U
     assert op.plan([(4, 4, I)], []).result_desc.prop == I
     assert op.plan([(4, 4, U)], [(4, 4, G)]).add_flops == 16
@@ -260,6 +268,7 @@ def test_sum_property():
     ([(0, 3, G)], [], "invalid_arg"),
     ([(3, 4, L)], [], "property"),
     ([(3, 4, I)], [], "property"),
+    ([(3, 4, D)], [], "property"),
     ([(3, 3, 7)], [], "property"),
     ([(3, 4, G), (5, 3, G)], [], "shape_mismatch"),
     ([(3, 4, G)], [(3, 5, G)], "shape_mismatch"),

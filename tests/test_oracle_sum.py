@@ -6,7 +6,7 @@ import pytest
 
 from oracle import plan as op
 from oracle import values as ov
-from oracle.plan import GENERAL as G, LOWER_TRI as L, UPPER_TRI as U, IDENTITY as I
+from oracle.plan import GENERAL as G, LOWER_TRI as L, UPPER_TRI as U, IDENTITY as I, DIAGONAL as D
 
 
 def rnd(rng, rows, cols, prop=G):
@@ -15,6 +15,8 @@ def rnd(rng, rows, cols, prop=G):
         a = np.tril(a)
     if prop == U:
         a = np.triu(a)
+    if prop == D:
+        a = np.diag(np.diag(a))
     return a
 
 
@@ -74,7 +76,8 @@ def test_chains_of_one_factor_behave_like_add_terms():
 
 
 @pytest.mark.parametrize("props", [((L, L), (L, L)), ((L, L), (U, U)), ((L, G), (L, L)), ((U, U), (U, I)),
-                                   ((I, I), (I, I)), ((L, I), (I, I)), ((I, I), (U, U))])
+                                   ((I, I), (I, I)), ((L, I), (I, I)), ((I, I), (U, U)),
+                                   ((D, D), (I, I)), ((D, L), (D, I)), ((D, U), (L, D)), ((G, D), (D, D))])
 def test_result_property_is_the_tightest_that_holds_the_numeric_pattern(props):
     # With positive entries nothing cancels, so the non-zero pattern of the numeric value is the true
     # structure; the inferred property must contain it and no tighter property may.
@@ -85,14 +88,15 @@ def test_result_property_is_the_tightest_that_holds_the_numeric_pattern(props):
     x, _ = ov.evaluate_sum(mats, chains)
     sp = op.plan_sum(chains)
     pattern = x != 0
-    holds = {p: not pattern[ov.off_structure_mask(n, n, p)].any() for p in (G, L, U, I)}
-    assert holds[sp.result_desc.prop]
-    if sp.result_desc.prop == G:
+    holds = {p: not pattern[ov.off_structure_mask(n, n, p)].any() for p in (G, L, U, D)}
+    got = sp.result_desc.prop
+    assert got != I and holds[got]              # a sum of at least two summands is never typed Identity (I + I = 2 I)
+    if got == G:
         assert not holds[L] and not holds[U]
-    else:                       # a sum of at least two summands is never typed Identity (I + I = 2 I)
-        assert sp.result_desc.prop in (L, U)
-        diagonal_only = holds[I]
-        assert diagonal_only or not holds[U if sp.result_desc.prop == L else L]
+    elif got in (L, U):
+        assert not holds[D]
+    else:
+        assert got == D
 
 
 def test_reuse_of_a_shared_product_counts_it_once():

@@ -11,8 +11,8 @@ one compile-time property (paper Section 2, "Matrix Attribute" and "Types").
 
 Storage convention for generated data (paper Section 2: the property dictates
 how the dense buffer is filled): dense row-major float32; entries outside a
-triangular operand's structure are ``+0.0``; Identity operands are never
-materialised (``None``).
+triangular or diagonal operand's structure are ``+0.0``; Identity operands are
+never materialised (``None``).
 
 Random stream: NumPy's Philox counter-based generator keyed by
 ``(seed, operand index)``; operand indices count the chain first, then the
@@ -25,8 +25,9 @@ from typing import List, Optional, Sequence
 
 import numpy as np
 
-GENERAL, LOWER_TRI, UPPER_TRI, IDENTITY = 0, 1, 2, 3
-PROPERTY_NAMES = {GENERAL: "general", LOWER_TRI: "lowerTri", UPPER_TRI: "upperTri", IDENTITY: "Identity"}
+GENERAL, LOWER_TRI, UPPER_TRI, IDENTITY, DIAGONAL = 0, 1, 2, 3, 4
+PROPERTY_NAMES = {GENERAL: "general", LOWER_TRI: "lowerTri", UPPER_TRI: "upperTri", IDENTITY: "Identity",
+                  DIAGONAL: "diagonal"}
 
 
 @dataclass(frozen=True)
@@ -37,7 +38,8 @@ class Operand:
           "normal"   -> N(0, sigma^2)
           "ones"     -> every structural entry 1 (the paper's Listing 2 fill)
     Triangular operands always use: strict part from `dist`, diagonal 1 + U(0, 1)
-    (except dist == "ones"), other half exactly zero.
+    (except dist == "ones"), other half exactly zero.  Diagonal operands: diagonal
+    1 + U(0, 1) (or ones), everything else exactly zero.
     """
     rows: int
     cols: int
@@ -83,15 +85,16 @@ def generate_operand(op: Operand, seed: int, index: int, batch: int = 1) -> Opti
     rng = np.random.Generator(np.random.Philox(key=[int(seed), int(index)]))
     shape = (batch, op.rows, op.cols) if batch > 1 else (op.rows, op.cols)
     m = _draw(rng, shape, op.dist, op.sigma)
-    if op.prop in (LOWER_TRI, UPPER_TRI):
+    if op.prop in (LOWER_TRI, UPPER_TRI, DIAGONAL):
         if op.rows != op.cols:
-            raise ValueError("triangular operands are square")
+            raise ValueError("triangular and diagonal operands are square")
         n = op.rows
         if op.dist != "ones":
             diag = np.float32(1.0) + rng.random(shape[:-1], dtype=np.float32)
             idx = np.arange(n)
             m[..., idx, idx] = diag
-        keep = np.tril(np.ones((n, n), dtype=bool)) if op.prop == LOWER_TRI else np.triu(np.ones((n, n), dtype=bool))
+        keep = (np.tril(np.ones((n, n), dtype=bool)) if op.prop == LOWER_TRI else
+                np.triu(np.ones((n, n), dtype=bool)) if op.prop == UPPER_TRI else np.eye(n, dtype=bool))
         m = np.where(keep, m, np.float32(0.0)).astype(np.float32)
     return np.ascontiguousarray(m, dtype=np.float32)
 
@@ -176,19 +179,22 @@ def config_listing2() -> Equation:
 
 
 def random_equation(seed: int, max_len: int = 6, max_dim: int = 96, allow_add: bool = True,
-                    dim_multiple: int = 1) -> Equation:
+                    dim_multiple: int = 1, diagonal: bool = False) -> Equation:
     """A random well-formed equation (for property tests): random length, dims, properties.
 
     Triangular / Identity operands are only placed where the neighbouring dimensions are equal,
-    which the generator arranges by repeating a dimension.
+    which the generator arranges by repeating a dimension.  With `diagonal` about a quarter of the
+    operands and Add terms are Diagonal (the streams without it are unchanged).
     """
-    rng = np.random.Generator(np.random.Philox(key=[int(seed), 0xC0FFEE]))
+    rng = np.random.Generator(np.random.Philox(key=[int(seed), 0xD1A6 if diagonal else 0xC0FFEE]))
     n = int(rng.integers(1, max_len + 1))
     chain: List[Operand] = []
     cur = int(rng.integers(1, max_dim // dim_multiple + 1)) * dim_multiple
     for _ in range(n):
-        kind = int(rng.integers(0, 6))
-        if kind == 0:
+        kind = int(rng.integers(0, 8 if diagonal else 6))
+        if kind >= 6:
+            chain.append(Operand(cur, cur, DIAGONAL))
+        elif kind == 0:
             chain.append(Operand(cur, cur, LOWER_TRI))
         elif kind == 1:
             chain.append(Operand(cur, cur, UPPER_TRI))
@@ -202,8 +208,10 @@ def random_equation(seed: int, max_len: int = 6, max_dim: int = 96, allow_add: b
     add: List[Operand] = []
     if allow_add:
         for _ in range(int(rng.integers(0, 3))):
-            kind = int(rng.integers(0, 5))
-            if rows == cols and kind == 0:
+            kind = int(rng.integers(0, 7 if diagonal else 5))
+            if rows == cols and kind >= 5:
+                add.append(Operand(rows, cols, DIAGONAL))
+            elif rows == cols and kind == 0:
                 add.append(Operand(rows, cols, LOWER_TRI))
             elif rows == cols and kind == 1:
                 add.append(Operand(rows, cols, UPPER_TRI))
