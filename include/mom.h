@@ -40,7 +40,7 @@ extern "C" {
 typedef enum {
     MOM_OK = 0,
     MOM_ERR_INVALID_ARG = 1,         /* null pointer, n_chain < 1, rows/cols < 1, bad enum, batch < 1 */
-    MOM_ERR_PROPERTY = 2,            /* triangular or Identity descriptor that is not square          */
+    MOM_ERR_PROPERTY = 2,            /* triangular, Diagonal or Identity descriptor that is not square */
     MOM_ERR_DTYPE = 3,               /* element type other than f32                                   */
     MOM_ERR_SHAPE_MISMATCH = 4,      /* inner dimensions differ, or an Add term's shape != X's shape  */
     MOM_ERR_OVERFLOW = 5,            /* a multiplication count does not fit in 63 bits                */
@@ -55,8 +55,13 @@ typedef enum {
 } mom_status_t;
 
 /* Paper Section 2, "Matrix Attribute" / "Types".  Triangles are non-strict and non-unit: the diagonal
- * is an ordinary stored entry (Listing 2 fills the diagonal with the fill value). */
-typedef enum { MOM_GENERAL = 0, MOM_LOWER_TRI = 1, MOM_UPPER_TRI = 2, MOM_IDENTITY = 3 } mom_property_t;
+ * is an ordinary stored entry (Listing 2 fills the diagonal with the fill value).
+ * MOM_DIAGONAL is one of the further properties the paper's conclusion announces (it prints no rule for
+ * it): a square matrix, stored densely like every other operand, whose entries off the diagonal are zeros.
+ * Unlike Identity its diagonal is data: it is never simplified away, D*A costs one multiplication per
+ * structural entry of A and runs as a scaling pass, D^T = D, and the lattice of product and sum types is
+ * Identity < Diagonal < {lowerTri, upperTri} < general. */
+typedef enum { MOM_GENERAL = 0, MOM_LOWER_TRI = 1, MOM_UPPER_TRI = 2, MOM_IDENTITY = 3, MOM_DIAGONAL = 4 } mom_property_t;
 typedef enum { MOM_F32 = 0 } mom_dtype_t;
 
 /* Arithmetic used by the product kernels.
@@ -77,7 +82,8 @@ typedef enum {
     MOM_KIND_TG = 1,     /* triangular * general                               */
     MOM_KIND_GT = 2,     /* general * triangular                               */
     MOM_KIND_TT = 3,     /* L*L or U*U: result keeps the triangle              */
-    MOM_KIND_TTMIX = 4   /* L*U or U*L: result is general                      */
+    MOM_KIND_TTMIX = 4,  /* L*U or U*L: result is general                      */
+    MOM_KIND_SCALE = 5   /* a Diagonal operand on either side: rows or columns of the other operand are scaled */
 } mom_kind_t;
 
 typedef struct {
@@ -92,7 +98,7 @@ typedef struct {
     int32_t lhs, rhs, out;
     int32_t kind;                    /* mom_kind_t */
     int32_t lhs_property, rhs_property, out_property;
-    int32_t uses_tensor_cores;       /* 1: tcgen05 3xTF32 kernel, 0: FFMA kernel */
+    int32_t uses_tensor_cores;       /* 1: tcgen05 3xTF32 kernel, 0: FFMA kernel (MOM_KIND_SCALE: the scaling kernel) */
     int32_t lhs_transposed, rhs_transposed;   /* the operand is an original chain operand used transposed */
     int64_t m, n, k;                 /* out is m x n, contraction length k */
     uint64_t useful_mults;           /* scalar multiplications with both factors structurally non-zero */

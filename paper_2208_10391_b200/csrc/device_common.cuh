@@ -26,21 +26,22 @@ struct AddTerms {
 // where the range for an output tile rows [r0,r1) x cols [c0,c1) is the intersection of the
 // operands' structural ranges:
 //   A lowerTri: l < r1      A upperTri: l >= r0      B lowerTri: l >= c0      B upperTri: l < c1
+//   A Diagonal: r0 <= l < r1                         B Diagonal: c0 <= l < c1
 // An empty range means the tile is structurally zero.
 __host__ __device__ inline void tile_k_range(int pa, int pb, int r0, int r1, int c0, int c1, int k,
                                              int *klo, int *khi) {
     int lo = 0, hi = k;
-    if (pa == MOM_UPPER_TRI && r0 > lo) lo = r0;
-    if (pb == MOM_LOWER_TRI && c0 > lo) lo = c0;
-    if (pa == MOM_LOWER_TRI && r1 < hi) hi = r1;
-    if (pb == MOM_UPPER_TRI && c1 < hi) hi = c1;
+    if ((pa == MOM_UPPER_TRI || pa == MOM_DIAGONAL) && r0 > lo) lo = r0;
+    if ((pb == MOM_LOWER_TRI || pb == MOM_DIAGONAL) && c0 > lo) lo = c0;
+    if ((pa == MOM_LOWER_TRI || pa == MOM_DIAGONAL) && r1 < hi) hi = r1;
+    if ((pb == MOM_UPPER_TRI || pb == MOM_DIAGONAL) && c1 < hi) hi = c1;
     *klo = lo;
     *khi = hi;
 }
 
 __host__ __device__ inline bool in_structure(int prop, int r, int c) {
     return prop == MOM_GENERAL || (prop == MOM_LOWER_TRI && r >= c) || (prop == MOM_UPPER_TRI && r <= c) ||
-           (prop == MOM_IDENTITY && r == c);
+           ((prop == MOM_IDENTITY || prop == MOM_DIAGONAL) && r == c);
 }
 
 // value of the equation at (r, c) given the chain's value `acc` there
@@ -58,6 +59,40 @@ __device__ __forceinline__ float finish_entry(float acc, const AddTerms &add, lo
         }
     }
     return in_structure(out_prop, r, c) ? v : 0.0f;
+}
+
+// The same for four consecutive entries (r, c .. c+3) of a row, for the kernels that are bound by memory
+// traffic: a compact loop over the terms (no unrolling: these kernels are tiny and must stay in the
+// instruction cache), one 16-byte load per term where its layout allows.  `n` is the row length of X
+// (entries at or beyond it are left alone), `vec` says that ld is a multiple of 4 (so that a term's
+// row segment is 16-byte aligned whenever the term's base is).
+__device__ __forceinline__ void finish_row4(float (&v)[4], const AddTerms &add, long long batch, int r, int c,
+                                             int ld, int n, int out_prop, bool vec) {
+#pragma unroll 1
+    for (int t = 0; t < add.count; ++t) {
+        const float *p = add.ptr[t];
+        if (!p) {                                            // Identity term
+#pragma unroll
+            for (int j = 0; j < 4; ++j) v[j] += r == c + j ? 1.0f : 0.0f;
+            continue;
+        }
+        p += batch * add.stride[t];
+        const bool tr = (add.transposed >> t) & 1u, alias = (add.aliases_out >> t) & 1u;
+        if (!tr && vec && c + 3 < n && (reinterpret_cast<uintptr_t>(p) & 15) == 0) {
+            const float4 *q = reinterpret_cast<const float4 *>(p + (long long)r * ld + c);
+            const float4 x = alias ? __ldcg(q) : __ldg(q);
+            v[0] += x.x; v[1] += x.y; v[2] += x.z; v[3] += x.w;
+        } else {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                if (c + j >= n) continue;
+                const long long at = tr ? (long long)(c + j) * add.rows + r : (long long)r * ld + c + j;
+                v[j] += alias ? __ldcg(p + at) : __ldg(p + at);
+            }
+        }
+    }
+#pragma unroll
+    for (int j = 0; j < 4; ++j) v[j] = in_structure(out_prop, r, c + j) ? v[j] : 0.0f;
 }
 
 }  // namespace mom

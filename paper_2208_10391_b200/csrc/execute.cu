@@ -333,7 +333,8 @@ mom_status_t execute_impl(const mom_plan *p, const float *const *chain_ptrs, con
                     launches += used;
                 } else {
                     if (ev) cudaEventRecord(ev[1], stream);
-                    if (launch_product_ffma(a, nb, stream) != cudaSuccess) return MOM_ERR_CUDA;
+                    const cudaError_t e = stp.pub.kind == MOM_KIND_SCALE ? launch_scale(a, nb, stream) : launch_product_ffma(a, nb, stream);
+                    if (e != cudaSuccess) return MOM_ERR_CUDA;
                     ++launches;
                 }
                 if (ev) cudaEventRecord(ev[2], stream);

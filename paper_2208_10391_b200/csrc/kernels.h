@@ -21,6 +21,9 @@ struct ProductArgs {
 
 cudaError_t launch_product_ffma(const ProductArgs &a, int batch, cudaStream_t stream);
 
+// The same product when A or B is Diagonal: a row or column scaling of the other operand (one pass).
+cudaError_t launch_scale(const ProductArgs &a, int batch, cudaStream_t stream);
+
 // src_mode: 0 pointer, 1 Identity, 2 X itself (in place), 3 pointer to the transposed matrix (cols x rows)
 cudaError_t launch_elementwise(const float *src, long long src_stride, int src_mode, float *X, long long x_stride,
                                int rows, int cols, int out_prop, const AddTerms &add, int batch, cudaStream_t stream);

@@ -19,11 +19,22 @@ constexpr uint64_t COST_LIMIT = (uint64_t)1 << 63;
 
 bool is_tri(int32_t p) { return p == MOM_LOWER_TRI || p == MOM_UPPER_TRI; }
 
-// Least upper bound in  Identity < {lowerTri, upperTri} < general  (paper Listing 3 types L*L as lowerTri).
+// Least upper bound in  Identity < Diagonal < {lowerTri, upperTri} < general  (paper Listing 3 types L*L as lowerTri).
 int32_t join_property(int32_t p, int32_t q) {
     if (p == MOM_IDENTITY) return q;
     if (q == MOM_IDENTITY) return p;
-    return p == q ? p : (int32_t)MOM_GENERAL;
+    if (p == q) return p;
+    if (p == MOM_DIAGONAL) return q;
+    if (q == MOM_DIAGONAL) return p;
+    return (int32_t)MOM_GENERAL;
+}
+
+// structural non-zeros of an r x c matrix with property p (triangular, Diagonal and Identity are square)
+unsigned __int128 structural_entries(int32_t p, int64_t r, int64_t c) {
+    const unsigned __int128 R = (unsigned __int128)r, C = (unsigned __int128)c;
+    if (p == MOM_GENERAL) return R * C;
+    if (p == MOM_LOWER_TRI || p == MOM_UPPER_TRI) return R * (R + 1) / 2;
+    return R;
 }
 
 // Scalar multiplications a_il * b_lj of an (m x k)(k x n) product in which both factors are
@@ -31,7 +42,11 @@ int32_t join_property(int32_t p, int32_t q) {
 bool useful_mults(int32_t pa, int32_t pb, int64_t m, int64_t k, int64_t n, uint64_t *out) {
     u128 v;
     const u128 M = (u128)m, K = (u128)k, N = (u128)n;
-    if (!is_tri(pa) && !is_tri(pb)) {
+    if (pa == MOM_DIAGONAL) {
+        v = structural_entries(pb, k, n);          // D*B scales the rows of B: one multiplication per entry of B
+    } else if (pb == MOM_DIAGONAL) {
+        v = structural_entries(pa, m, k);          // A*D scales the columns of A
+    } else if (!is_tri(pa) && !is_tri(pb)) {
         v = M * K * N;
     } else if (is_tri(pa) && !is_tri(pb)) {
         v = N * (K * (K + 1) / 2);                 // row i of A has i+1 (or k-i) non-zeros
@@ -49,30 +64,21 @@ bool useful_mults(int32_t pa, int32_t pb, int64_t m, int64_t k, int64_t n, uint6
 
 mom_status_t check_desc(const mom_matrix_desc_t &d) {
     if (d.rows < 1 || d.cols < 1) return MOM_ERR_INVALID_ARG;
-    if (d.property < MOM_GENERAL || d.property > MOM_IDENTITY) return MOM_ERR_INVALID_ARG;
+    if (d.property < MOM_GENERAL || d.property > MOM_DIAGONAL) return MOM_ERR_INVALID_ARG;
     if (d.dtype != MOM_F32) return MOM_ERR_DTYPE;
     if (d.property != MOM_GENERAL && d.rows != d.cols) return MOM_ERR_PROPERTY;
     return MOM_OK;
 }
 
-uint64_t nnz(const mom_matrix_desc_t &d) {
-    if (d.property == MOM_GENERAL) return (uint64_t)d.rows * (uint64_t)d.cols;
-    if (d.property == MOM_IDENTITY) return (uint64_t)d.rows;
-    return (uint64_t)d.rows * ((uint64_t)d.rows + 1) / 2;
-}
+uint64_t nnz(const mom_matrix_desc_t &d) { return (uint64_t)structural_entries(d.property, d.rows, d.cols); }
 
 // Property of a sum of summands (chain values and Add terms).  A sum of two or more is never Identity: an
-// Identity summand only contributes its diagonal footprint, which fits inside either triangle.
+// Identity summand contributes its diagonal footprint and is joined as a Diagonal matrix.
 int32_t sum_property(const std::vector<int32_t> &props) {
     if (props.size() == 1) return props[0];
-    bool seen = false;
-    int32_t acc = MOM_GENERAL;
-    for (int32_t p : props) {
-        if (p == MOM_IDENTITY) continue;
-        if (!seen) { acc = p; seen = true; }
-        else if (acc != p) acc = MOM_GENERAL;
-    }
-    return seen ? acc : (int32_t)MOM_LOWER_TRI;
+    int32_t acc = MOM_DIAGONAL;
+    for (int32_t p : props) acc = join_property(acc, p == MOM_IDENTITY ? (int32_t)MOM_DIAGONAL : p);
+    return acc;
 }
 
 struct Node { int64_t rows, cols; int32_t prop; };
@@ -320,7 +326,8 @@ static mom_status_t plan_sums(const std::vector<mom_matrix_desc_t> &slots, const
                             st.pub.m = a.rows; st.pub.k = a.cols; st.pub.n = b.cols;
                             useful_mults(a.prop, b.prop, a.rows, a.cols, b.cols, &st.pub.useful_mults);
                             const bool ta = is_tri(a.prop), tb = is_tri(b.prop);
-                            st.pub.kind = !ta && !tb ? MOM_KIND_GG : ta && !tb ? MOM_KIND_TG : !ta && tb ? MOM_KIND_GT
+                            st.pub.kind = a.prop == MOM_DIAGONAL || b.prop == MOM_DIAGONAL ? MOM_KIND_SCALE
+                                          : !ta && !tb ? MOM_KIND_GG : ta && !tb ? MOM_KIND_TG : !ta && tb ? MOM_KIND_GT
                                           : a.prop == b.prop ? MOM_KIND_TT : MOM_KIND_TTMIX;
                             st.is_last = root;
                             if (root) st.sum = sum_index;
@@ -379,7 +386,8 @@ static mom_status_t plan_sums(const std::vector<mom_matrix_desc_t> &slots, const
             const bool addressable = (k % 4 == 0) && (n % 4 == 0);
             const bool worth_it = (double)m * (double)n * (double)k >= (double)(1 << 23);
             st.pub.uses_tensor_cores =
-                (variant == MOM_VARIANT_3XTF32 && addressable && worth_it) || ((int)variant == 2 && addressable);
+                st.pub.kind != MOM_KIND_SCALE &&        // a Diagonal operand: one scaling pass, bound by HBM
+                ((variant == MOM_VARIANT_3XTF32 && addressable && worth_it) || ((int)variant == 2 && addressable));
             if (st.pub.uses_tensor_cores) {
                 // few output tiles, long contraction: split k over otherwise idle SMs
                 const int64_t tiles = ((m + mom::TC_BM - 1) / mom::TC_BM) * ((n + mom::TC_BN - 1) / mom::TC_BN);
@@ -759,7 +767,7 @@ const char *mom_status_string(mom_status_t s) {
     switch (s) {
         case MOM_OK: return "ok";
         case MOM_ERR_INVALID_ARG: return "invalid argument";
-        case MOM_ERR_PROPERTY: return "triangular and Identity matrices must be square";
+        case MOM_ERR_PROPERTY: return "triangular, Diagonal and Identity matrices must be square";
         case MOM_ERR_DTYPE: return "unsupported element type";
         case MOM_ERR_SHAPE_MISMATCH: return "shape mismatch";
         case MOM_ERR_OVERFLOW: return "multiplication count overflows 63 bits";

@@ -142,23 +142,142 @@ product_ffma_kernel(ProductArgs a) {
 
 // X = src (+ Add terms), masked to the result's structure.  src_mode: 0 pointer, 1 Identity,
 // 2 X itself (in place; used to add terms beyond the fused limit), 3 pointer to the transposed matrix.
-__global__ void __launch_bounds__(256)
+// Bound by HBM: a thread takes four consecutive columns of four rows per pass (16-byte accesses where
+// the layout allows, all loads of a pass issued before its first store).
+constexpr int EW_TX = 64, EW_TY = 4, EW_ROWS = 4;
+
+__global__ void __launch_bounds__(EW_TX * EW_TY)
 elementwise_kernel(const float *__restrict__ src, long long src_stride, int src_mode, float *X, long long x_stride,
                    int rows, int cols, int out_prop, AddTerms add) {
     const long long inst = blockIdx.z;
-    const long long total = (long long)rows * cols;
-    for (long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (long long)gridDim.x * blockDim.x) {
-        const int r = (int)(e / cols), c = (int)(e % cols);
-        float v;
-        if (src_mode == 0) v = __ldg(src + inst * src_stride + e);
-        else if (src_mode == 3) v = __ldg(src + inst * src_stride + (long long)c * rows + r);
-        else if (src_mode == 1) v = (r == c) ? 1.0f : 0.0f;
-        else v = X[inst * x_stride + e];
-        X[inst * x_stride + e] = finish_entry(v, add, inst, r, c, cols, out_prop);
+    const float *S = src_mode == 2 ? X + inst * x_stride : src + inst * src_stride;
+    float *Xi = X + inst * x_stride;
+    const bool ld4 = (cols & 3) == 0;
+    const bool vec_x = ld4 && (reinterpret_cast<uintptr_t>(Xi) & 15) == 0;
+    const bool vec_s = vec_x && (src_mode == 2 || (src_mode == 0 && (reinterpret_cast<uintptr_t>(S) & 15) == 0));
+    const int c = (blockIdx.x * EW_TX + threadIdx.x) * 4;
+    if (c >= cols) return;
+    for (int rb = blockIdx.y * (EW_TY * EW_ROWS) + threadIdx.y; rb < rows; rb += gridDim.y * (EW_TY * EW_ROWS)) {
+        float v[EW_ROWS][4];
+#pragma unroll
+        for (int i = 0; i < EW_ROWS; ++i) {
+            const int r = rb + i * EW_TY;
+            v[i][0] = v[i][1] = v[i][2] = v[i][3] = 0.f;
+            if (r >= rows) continue;
+            if (src_mode == 1) {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) v[i][j] = r == c + j ? 1.0f : 0.0f;
+            } else if (vec_s) {
+                const float4 *q = reinterpret_cast<const float4 *>(S + (long long)r * cols + c);
+                const float4 t = src_mode == 2 ? __ldcg(q) : __ldg(q);      // X itself is never read through the read-only path
+                v[i][0] = t.x; v[i][1] = t.y; v[i][2] = t.z; v[i][3] = t.w;
+            } else {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    if (c + j >= cols) continue;
+                    if (src_mode == 3) v[i][j] = __ldg(S + (long long)(c + j) * rows + r);
+                    else if (src_mode == 2) v[i][j] = __ldcg(S + (long long)r * cols + c + j);
+                    else v[i][j] = __ldg(S + (long long)r * cols + c + j);
+                }
+            }
+        }
+#pragma unroll
+        for (int i = 0; i < EW_ROWS; ++i) {
+            const int r = rb + i * EW_TY;
+            if (r >= rows) continue;
+            finish_row4(v[i], add, inst, r, c, cols, cols, out_prop, ld4);
+            float *p = Xi + (long long)r * cols + c;
+            if (vec_x) {
+                *reinterpret_cast<float4 *>(p) = make_float4(v[i][0], v[i][1], v[i][2], v[i][3]);
+            } else {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) if (c + j < cols) p[j] = v[i][j];
+            }
+        }
+    }
+}
+
+// Product with a Diagonal operand: C = D*B scales row r of B by d_r, C = A*D scales column c of A by d_c
+// (+ Add terms, structure mask).  One pass over the other operand, bound by HBM: a thread takes four
+// consecutive columns of a row (one 16-byte load and store where the layout allows), only the diagonal of
+// D and the structural part of the other operand are read.
+constexpr int SCALE_TX = 64, SCALE_TY = 4;
+
+__global__ void __launch_bounds__(SCALE_TX * SCALE_TY)
+scale_kernel(ProductArgs a) {
+    const long long inst = blockIdx.z;
+    const bool left = a.pa == MOM_DIAGONAL;                 // D on the left: the other operand is B
+    const float *__restrict__ D = (left ? a.A : a.B) + inst * (left ? a.strideA : a.strideB);
+    const float *__restrict__ S = (left ? a.B : a.A) + inst * (left ? a.strideB : a.strideA);
+    const int ps = left ? a.pb : a.pa;
+    const bool trans = left ? a.transB != 0 : a.transA != 0;   // S is stored n x m
+    float *__restrict__ C = a.C + inst * a.strideC;
+    const int m = a.m, n = a.n;
+    const long long dstep = (long long)a.k + 1;             // D is k x k: d_i sits at i * (k + 1)
+    const bool vec = !trans && (n & 3) == 0 && ((reinterpret_cast<uintptr_t>(S) | reinterpret_cast<uintptr_t>(C)) & 15) == 0;
+    const int c = (blockIdx.x * SCALE_TX + threadIdx.x) * 4;
+    if (c >= n) return;
+    float dc[4] = {0.f, 0.f, 0.f, 0.f};                     // D on the right: this thread's four columns keep their factors
+    if (!left) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) if (c + j < n) dc[j] = __ldg(D + (c + j) * dstep);
+    }
+    // four rows per thread and pass: their loads are all issued before the first store
+    constexpr int ROWS = 4;
+    for (int rb = blockIdx.y * (SCALE_TY * ROWS) + threadIdx.y; rb < m; rb += gridDim.y * (SCALE_TY * ROWS)) {
+        float s[ROWS][4];
+        float dr[ROWS];
+#pragma unroll
+        for (int i = 0; i < ROWS; ++i) {
+            const int r = rb + i * SCALE_TY;
+            s[i][0] = s[i][1] = s[i][2] = s[i][3] = 0.f;
+            dr[i] = 0.f;
+            if (r >= m) continue;
+            // the four entries lie inside S's structure?  (outside, the stored zeros need not be read)
+            const bool any = ps == MOM_GENERAL || (ps == MOM_LOWER_TRI && c <= r) || (ps == MOM_UPPER_TRI && c + 3 >= r) ||
+                             (ps == MOM_DIAGONAL && c <= r && c + 3 >= r);
+            if (any) {
+                if (vec) {
+                    const float4 t = __ldg(reinterpret_cast<const float4 *>(S + (long long)r * n + c));
+                    s[i][0] = t.x; s[i][1] = t.y; s[i][2] = t.z; s[i][3] = t.w;
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 4; ++j)
+                        if (c + j < n) s[i][j] = __ldg(trans ? S + (long long)(c + j) * m + r : S + (long long)r * n + c + j);
+                }
+            }
+            if (left) dr[i] = __ldg(D + r * dstep);
+        }
+#pragma unroll
+        for (int i = 0; i < ROWS; ++i) {
+            const int r = rb + i * SCALE_TY;
+            if (r >= m) continue;
+            float v[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) v[j] = (left ? dr[i] : dc[j]) * s[i][j];
+            finish_row4(v, a.add, inst, r, c, n, n, a.pout, (n & 3) == 0);
+            float *p = C + (long long)r * n + c;
+            if (vec) {
+                *reinterpret_cast<float4 *>(p) = make_float4(v[0], v[1], v[2], v[3]);
+            } else {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) if (c + j < n) p[j] = v[j];
+            }
+        }
     }
 }
 
 }  // namespace
+
+cudaError_t launch_scale(const ProductArgs &a, int batch, cudaStream_t stream) {
+    const int gx = (a.n + SCALE_TX * 4 - 1) / (SCALE_TX * 4);
+    int gy = (a.m + SCALE_TY * 4 - 1) / (SCALE_TY * 4);     // a CTA pass covers 16 rows
+    const int want = (148 * 16 + gx - 1) / gx;              // a few CTAs per SM; rows beyond that are looped over
+    if (gy > want) gy = want;
+    if (gy < 1) gy = 1;
+    scale_kernel<<<dim3(gx, gy, batch), dim3(SCALE_TX, SCALE_TY), 0, stream>>>(a);
+    return cudaGetLastError();
+}
 
 cudaError_t launch_product_ffma(const ProductArgs &a, int batch, cudaStream_t stream) {
     dim3 grid((a.n + BN - 1) / BN, (a.m + BM - 1) / BM, batch);
@@ -168,12 +287,12 @@ cudaError_t launch_product_ffma(const ProductArgs &a, int batch, cudaStream_t st
 
 cudaError_t launch_elementwise(const float *src, long long src_stride, int src_mode, float *X, long long x_stride,
                                int rows, int cols, int out_prop, const AddTerms &add, int batch, cudaStream_t stream) {
-    const long long total = (long long)rows * cols;
-    long long blocks = (total + 255) / 256;
-    if (blocks > 148 * 16) blocks = 148 * 16;
-    if (blocks < 1) blocks = 1;
-    dim3 grid((unsigned)blocks, 1, batch);
-    elementwise_kernel<<<grid, 256, 0, stream>>>(src, src_stride, src_mode, X, x_stride, rows, cols, out_prop, add);
+    const int gx = (cols + EW_TX * 4 - 1) / (EW_TX * 4);
+    int gy = (rows + EW_TY * EW_ROWS - 1) / (EW_TY * EW_ROWS);
+    const int want = (148 * 16 + gx - 1) / gx;              // a few CTAs per SM; rows beyond that are looped over
+    if (gy > want) gy = want;
+    if (gy < 1) gy = 1;
+    elementwise_kernel<<<dim3(gx, gy, batch), dim3(EW_TX, EW_TY), 0, stream>>>(src, src_stride, src_mode, X, x_stride, rows, cols, out_prop, add);
     return cudaGetLastError();
 }
 

@@ -54,6 +54,21 @@ def test_random_equations_match_the_oracle():
         assert_same_plan(eq.descs(), eq.add_descs())
 
 
+def test_random_equations_with_diagonal_operands_match_the_oracle():
+    diag = 0
+    for seed in range(300):
+        eq = wl.random_equation(seed, max_len=9, max_dim=50, diagonal=True)
+        got, _ = assert_same_plan(eq.descs(), eq.add_descs())
+        diag += any(got.step(i).kind == mom.KIND_SCALE for i in range(got.num_steps()))
+    assert diag > 100
+    # equal dimensions: many ties between the sides a Diagonal factor can join
+    rng = np.random.default_rng(4)
+    for _ in range(60):
+        chain = [(12, 12, int(rng.integers(0, 5))) for _ in range(int(rng.integers(2, 9)))]
+        add = [(12, 12, int(rng.integers(0, 5))) for _ in range(int(rng.integers(0, 3)))]
+        assert_same_plan(chain, add)
+
+
 def test_long_chains_with_many_ties():
     # equal dimensions everywhere: every tree of an all-general chain ties; mixed properties tie partially
     rng = np.random.default_rng(3)
@@ -128,9 +143,15 @@ def test_step_kinds():
     L, U, G = mom.LOWER_TRI, mom.UPPER_TRI, mom.GENERAL
     cases = {(G, G): mom.KIND_GG, (L, G): mom.KIND_TG, (U, G): mom.KIND_TG, (G, L): mom.KIND_GT, (G, U): mom.KIND_GT,
              (L, L): mom.KIND_TT, (U, U): mom.KIND_TT, (L, U): mom.KIND_TTMIX, (U, L): mom.KIND_TTMIX}
+    D = mom.DIAGONAL
+    cases.update({(D, G): mom.KIND_SCALE, (G, D): mom.KIND_SCALE, (D, L): mom.KIND_SCALE, (U, D): mom.KIND_SCALE, (D, D): mom.KIND_SCALE})
     for (a, b), kind in cases.items():
         p = mom.mom_equation_plan([(8, 8, a), (8, 8, b)])
         assert p.step(0).kind == kind
+        assert not (kind == mom.KIND_SCALE and p.step(0).uses_tensor_cores)
+    # a scaling never runs on tensor cores, whatever its size
+    p = mom.mom_equation_plan([(4096, 4096, D), (4096, 4096, G)])
+    assert p.step(0).kind == mom.KIND_SCALE and not p.step(0).uses_tensor_cores
 
 
 def test_transposed_operands_match_the_oracle():
@@ -187,6 +208,9 @@ def test_random_sums_of_chains_match_the_oracle():
         shared += want.reused > 0
         assert_same_sum_plan(eq.descs(), eq.transposed, None)        # nothing known to be shared
     assert shared >= 20
+    for seed in range(200):                                          # with Diagonal factors
+        eq = wl.random_sum_equation(seed, diagonal=True)
+        assert_same_sum_plan(eq.descs(), eq.transposed, eq.names)
 
 
 def test_sum_plan_shares_a_product_between_chains():
@@ -247,6 +271,9 @@ def test_random_expressions_match_the_oracle():
         _, want = assert_same_expression_plan(ex.expr, ex.descs())
         nested += want.temporaries > 0
     assert nested >= 100
+    for seed in range(200):                                          # with Diagonal operands
+        ex = wl.random_expression(seed, diagonal=True)
+        assert_same_expression_plan(ex.expr, ex.descs())
 
 
 def test_expression_plan_examples():

@@ -172,6 +172,15 @@ def config_transposed(n: int = 4096, seed: int = 6) -> Equation:
         chain_t=(True, False, True, False), add_t=(True,))
 
 
+def config_diagonal(n: int = 4096, seed: int = 10) -> Equation:
+    """X = L * D * A * U + C: a Diagonal factor between a triangle and a general matrix (it joins the
+    triangle: n(n+1)/2 multiplications instead of n^2), then two triangular x general products."""
+    s = 1.0 / np.sqrt(n)
+    return Equation(f"LDAU_plus_C_{n}", seed, (
+        Operand(n, n, LOWER_TRI), Operand(n, n, DIAGONAL), Operand(n, n, GENERAL, "normal", s), Operand(n, n, UPPER_TRI)),
+        (Operand(n, n, GENERAL, "normal"),))
+
+
 def config_listing2() -> Equation:
     """Listing 2 of the paper: two 5x5 lowerTri matrices filled with the constant 1."""
     return Equation("listing2_LL_5", 0, (
@@ -263,10 +272,11 @@ def generate_sum(eq: SumEquation):
 
 
 def random_sum_equation(seed: int, max_chains: int = 4, max_len: int = 5, max_dim: int = 48,
-                        dim_multiple: int = 1, share: float = 0.5) -> SumEquation:
+                        dim_multiple: int = 1, share: float = 0.5, diagonal: bool = False) -> SumEquation:
     """Random well-formed sum of chains.  With probability `share`/2 a chain starts with a run of factors
-    copied (same names and flags) from an earlier chain, so that shared products occur."""
-    rng = np.random.Generator(np.random.Philox(key=[int(seed), 0x5EED5]))
+    copied (same names and flags) from an earlier chain, so that shared products occur.  With `diagonal`
+    some square factors are Diagonal (the streams without it are unchanged)."""
+    rng = np.random.Generator(np.random.Philox(key=[int(seed), 0x5D1A6 if diagonal else 0x5EED5]))
     rows = int(rng.integers(1, max_dim // dim_multiple + 1)) * dim_multiple
     cols = int(rng.integers(1, max_dim // dim_multiple + 1)) * dim_multiple
     if rng.random() < 0.4:
@@ -277,9 +287,11 @@ def random_sum_equation(seed: int, max_chains: int = 4, max_len: int = 5, max_di
     def new_factor(r, c):
         nonlocal next_name
         """One stored factor whose type AS USED is r x c, with a random property and transposition."""
-        kind = int(rng.integers(0, 7))
+        kind = int(rng.integers(0, 9 if diagonal else 7))
         t = bool(rng.integers(0, 3) == 0)
-        if r == c and kind == 0:
+        if r == c and kind >= 7:
+            o = Operand(r, r, DIAGONAL)
+        elif r == c and kind == 0:
             o = Operand(r, r, LOWER_TRI)
         elif r == c and kind == 1:
             o = Operand(r, r, UPPER_TRI)
@@ -355,9 +367,11 @@ def generate_expression(ex: Expression):
     return [generate_operand(o, ex.seed, i) for i, o in enumerate(ex.operands)]
 
 
-def random_expression(seed: int, max_depth: int = 3, max_dim: int = 40, dim_multiple: int = 1) -> Expression:
-    """Random well-formed nested expression; operands are reused where an existing one has the needed type."""
-    rng = np.random.Generator(np.random.Philox(key=[int(seed), 0xE4B8]))
+def random_expression(seed: int, max_depth: int = 3, max_dim: int = 40, dim_multiple: int = 1,
+                      diagonal: bool = False) -> Expression:
+    """Random well-formed nested expression; operands are reused where an existing one has the needed type.
+    With `diagonal` some square operands are Diagonal (the streams without it are unchanged)."""
+    rng = np.random.Generator(np.random.Philox(key=[int(seed), 0xED1A6 if diagonal else 0xE4B8]))
     operands: List[Operand] = []
 
     def dim():
@@ -370,8 +384,8 @@ def random_expression(seed: int, max_depth: int = 3, max_dim: int = 40, dim_mult
         if same and rng.random() < 0.5:
             i = int(rng.choice(same))
         else:
-            kind = int(rng.integers(0, 7))
-            prop = {0: LOWER_TRI, 1: UPPER_TRI, 2: IDENTITY}.get(kind, GENERAL) if sr == sc else GENERAL
+            kind = int(rng.integers(0, 9 if diagonal else 7))
+            prop = {0: LOWER_TRI, 1: UPPER_TRI, 2: IDENTITY, 7: DIAGONAL, 8: DIAGONAL}.get(kind, GENERAL) if sr == sc else GENERAL
             operands.append(Operand(sr, sc, prop, "normal" if kind == 3 else "uniform"))
             i = len(operands) - 1
         return ("t", i) if t else i
