@@ -2,7 +2,9 @@
 // one instance per CTA, with the operands and all intermediates resident in shared memory.  Batched
 // small equations are bound by HBM traffic, so each operand is read exactly once (only the
 // structural part of triangular operands), nothing intermediate touches global memory, and several
-// CTAs per SM overlap one instance's loads with another's arithmetic.
+// CTAs per SM overlap one instance's loads with another's arithmetic.  The kernel is bound by
+// instruction issue as much as by memory, so the per-instance code is kept short: the epilogue loops over
+// the Add terms instead of unrolling them, and the low part of the operand split is not rounded.
 //
 // Two arithmetic variants of the products:
 //   MMA   warp-level mma.sync m16n8k8 tf32 with the 3xTF32 split done in registers on the
@@ -70,9 +72,12 @@ __device__ __forceinline__ void cp_async_wait_all() {
 // last kept place to the magnitude, clear the 13 dropped bits.  (The cvt.rna.tf32.f32 instruction gives
 // the same result but issues at conversion-pipe rate, which made it the bottleneck of this kernel.)
 __device__ __forceinline__ uint32_t round_tf32_bits(float a) { return (__float_as_uint(a) + 0x1000u) & 0xFFFFE000u; }
+// The low part a - hi is exact in f32 and is handed to the MMA as it is: the tensor core reads only the
+// tf32 part of an operand register (sign, exponent, 10 mantissa bits), i.e. it drops bits that are worth
+// at most 2^-21 of a -- the size of the lo*lo term this scheme leaves out anyway.
 __device__ __forceinline__ void split_tf32(float a, uint32_t &hi, uint32_t &lo) {
     hi = round_tf32_bits(a);
-    lo = round_tf32_bits(a - __uint_as_float(hi));
+    lo = __float_as_uint(a - __uint_as_float(hi));
 }
 
 __device__ __forceinline__ void mma_tf32(float (&d)[4], const uint32_t (&a)[4], const uint32_t (&b)[2]) {
@@ -81,26 +86,54 @@ __device__ __forceinline__ void mma_tf32(float (&d)[4], const uint32_t (&a)[4], 
                  : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b[0]), "r"(b[1]));
 }
 
+// What the kernel's loop hands to the products of one instance.
+struct Instance {
+    long long inst;
+    float *smem;
+};
+__device__ __forceinline__ float *at(const Instance &in, int off) { return in.smem + off; }
+
+// the equation's value at (r, c) and (r, c + 1) given the chain's values there: Add terms left to right
+// in a compact loop, then the structure mask
+__device__ __forceinline__ void finish_pair(const FusedPlan &fp, const Instance &in, int r, int c, int n, int pout, bool two,
+                                            float &x0, float &x1) {
+#pragma unroll 1
+    for (int t = 0; t < fp.add.count; ++t) {
+        const float *p = fp.add.ptr[t];
+        if (!p) {
+            x0 += r == c ? 1.0f : 0.0f;
+            x1 += r == c + 1 ? 1.0f : 0.0f;
+            continue;
+        }
+        p += in.inst * fp.add.stride[t];
+        const bool tr = (fp.add.transposed >> t) & 1u;
+        x0 += __ldg(p + (tr ? (long long)c * fp.add.rows + r : (long long)r * n + c));
+        if (two) x1 += __ldg(p + (tr ? (long long)(c + 1) * fp.add.rows + r : (long long)r * n + c + 1));
+    }
+    x0 = in_structure(pout, r, c) ? x0 : 0.0f;
+    x1 = in_structure(pout, r, c + 1) ? x1 : 0.0f;
+}
+
 // store one output entry pair (r, c), (r, c+1) of a step: into shared memory for an intermediate
 // (masked to its structure, padded columns zero) or, on the last step, into X with the Add terms
-__device__ __forceinline__ void store_pair(const FusedPlan &fp, const FusedStep &st, float *smem, long long inst, int r, int c,
+__device__ __forceinline__ void store_pair(const FusedPlan &fp, const FusedStep &st, const Instance &in, int r, int c,
                                            float v0, float v1) {
     if (r >= st.m) return;
     if (st.out_off >= 0) {
         if (c >= st.ldc) return;
-        float *C = smem + st.out_off + r * st.ldc + c;
+        float *C = at(in, st.out_off) + r * st.ldc + c;
         C[0] = (c < st.n && in_structure(st.pout, r, c)) ? v0 : 0.f;
         if (c + 1 < st.ldc) C[1] = (c + 1 < st.n && in_structure(st.pout, r, c + 1)) ? v1 : 0.f;
     } else {
         if (c >= st.n) return;
-        float *X = fp.out + inst * fp.out_stride + (size_t)r * st.n + c;
-        const float x0 = finish_entry(v0, fp.add, inst, r, c, st.n, st.pout);
-        if (c + 1 < st.n) {
-            const float x1 = finish_entry(v1, fp.add, inst, r, c + 1, st.n, st.pout);
-            if ((reinterpret_cast<uintptr_t>(X) & 7) == 0) *reinterpret_cast<float2 *>(X) = make_float2(x0, x1);
-            else { X[0] = x0; X[1] = x1; }
+        float *X = fp.out + in.inst * fp.out_stride + (size_t)r * st.n + c;
+        const bool two = c + 1 < st.n;
+        finish_pair(fp, in, r, c, st.n, st.pout, two, v0, v1);
+        if (two) {
+            if ((reinterpret_cast<uintptr_t>(X) & 7) == 0) *reinterpret_cast<float2 *>(X) = make_float2(v0, v1);
+            else { X[0] = v0; X[1] = v1; }
         } else {
-            X[0] = x0;
+            X[0] = v0;
         }
     }
 }
@@ -110,9 +143,9 @@ __device__ __forceinline__ void store_pair(const FusedPlan &fp, const FusedStep 
 // terms (lo*hi, hi*lo) and the main term (hi*hi) go to separate accumulators: two independent MMA
 // chains per 8-column tile instead of one three times as long.
 template <int NTW>
-__device__ void product_mma_whole(const FusedPlan &fp, const FusedStep &st, float *smem, long long inst) {
-    const float *__restrict__ A = smem + st.a_off;
-    const float *__restrict__ B = smem + st.b_off;
+__device__ void product_mma_whole(const FusedPlan &fp, const FusedStep &st, const Instance &in) {
+    const float *__restrict__ A = at(in, st.a_off);
+    const float *__restrict__ B = at(in, st.b_off);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
     constexpr int TW = 8 * NTW;
     const int tiles_n = st.n / TW, tiles = (st.m >> 4) * tiles_n;
@@ -148,22 +181,22 @@ __device__ void product_mma_whole(const FusedPlan &fp, const FusedStep &st, floa
         }
 #pragma unroll
         for (int j = 0; j < NTW; ++j) {
-            store_pair(fp, st, smem, inst, r0 + g, c0 + 8 * j + 2 * t, main_acc[j][0] + small_acc[j][0], main_acc[j][1] + small_acc[j][1]);
-            store_pair(fp, st, smem, inst, r0 + g + 8, c0 + 8 * j + 2 * t, main_acc[j][2] + small_acc[j][2], main_acc[j][3] + small_acc[j][3]);
+            store_pair(fp, st, in, r0 + g, c0 + 8 * j + 2 * t, main_acc[j][0] + small_acc[j][0], main_acc[j][1] + small_acc[j][1]);
+            store_pair(fp, st, in, r0 + g + 8, c0 + 8 * j + 2 * t, main_acc[j][2] + small_acc[j][2], main_acc[j][3] + small_acc[j][3]);
         }
     }
 }
 
 // One product on tensor cores: 16 x 16 output tiles dealt round-robin to the warps.
-__device__ void product_mma(const FusedPlan &fp, const FusedStep &st, float *smem, long long inst) {
+__device__ void product_mma(const FusedPlan &fp, const FusedStep &st, const Instance &in) {
     if (((st.m | st.n) & 15) == 0 && (st.k & 7) == 0) {
         // with few 16 x 16 tiles, 16 x 8 tiles give every warp of the CTA something to do
-        if ((st.m >> 4) * (st.n >> 4) < WARPS) product_mma_whole<1>(fp, st, smem, inst);
-        else product_mma_whole<2>(fp, st, smem, inst);
+        if ((st.m >> 4) * (st.n >> 4) < WARPS) product_mma_whole<1>(fp, st, in);
+        else product_mma_whole<2>(fp, st, in);
         return;
     }
-    const float *__restrict__ A = smem + st.a_off;
-    const float *__restrict__ B = smem + st.b_off;
+    const float *__restrict__ A = at(in, st.a_off);
+    const float *__restrict__ B = at(in, st.b_off);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
     const int tiles_n = (st.n + 15) >> 4, tiles = ((st.m + 15) >> 4) * tiles_n;
     for (int tile = warp; tile < tiles; tile += WARPS) {
@@ -198,16 +231,16 @@ __device__ void product_mma(const FusedPlan &fp, const FusedStep &st, float *sme
         }
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
-            store_pair(fp, st, smem, inst, r0 + g, c0 + 8 * h + 2 * t, acc[h][0], acc[h][1]);
-            store_pair(fp, st, smem, inst, r0 + g + 8, c0 + 8 * h + 2 * t, acc[h][2], acc[h][3]);
+            store_pair(fp, st, in, r0 + g, c0 + 8 * h + 2 * t, acc[h][0], acc[h][1]);
+            store_pair(fp, st, in, r0 + g + 8, c0 + 8 * h + 2 * t, acc[h][2], acc[h][3]);
         }
     }
 }
 
 // One product with plain FMA: cells of 2 rows x 4 columns dealt round-robin to the threads.
-__device__ void product_ffma(const FusedPlan &fp, const FusedStep &st, float *smem, long long inst) {
-    const float *__restrict__ A = smem + st.a_off;
-    const float *__restrict__ B = smem + st.b_off;
+__device__ void product_ffma(const FusedPlan &fp, const FusedStep &st, const Instance &in) {
+    const float *__restrict__ A = at(in, st.a_off);
+    const float *__restrict__ B = at(in, st.b_off);
     const int cells_per_row = (st.n + 3) >> 2, row_pairs = (st.m + 1) >> 1;
     for (int cell = threadIdx.x; cell < row_pairs * cells_per_row; cell += THREADS) {
         const int r = (cell / cells_per_row) << 1, c = (cell % cells_per_row) << 2;
@@ -222,20 +255,23 @@ __device__ void product_ffma(const FusedPlan &fp, const FusedStep &st, float *sm
             a0[0] = fmaf(x0, b.x, a0[0]); a0[1] = fmaf(x0, b.y, a0[1]); a0[2] = fmaf(x0, b.z, a0[2]); a0[3] = fmaf(x0, b.w, a0[3]);
             a1[0] = fmaf(x1, b.x, a1[0]); a1[1] = fmaf(x1, b.y, a1[1]); a1[2] = fmaf(x1, b.z, a1[2]); a1[3] = fmaf(x1, b.w, a1[3]);
         }
-        store_pair(fp, st, smem, inst, r, c, a0[0], a0[1]);
-        store_pair(fp, st, smem, inst, r, c + 2, a0[2], a0[3]);
+        store_pair(fp, st, in, r, c, a0[0], a0[1]);
+        store_pair(fp, st, in, r, c + 2, a0[2], a0[3]);
         if (two) {
-            store_pair(fp, st, smem, inst, r + 1, c, a1[0], a1[1]);
-            store_pair(fp, st, smem, inst, r + 1, c + 2, a1[2], a1[3]);
+            store_pair(fp, st, in, r + 1, c, a1[0], a1[1]);
+            store_pair(fp, st, in, r + 1, c + 2, a1[2], a1[3]);
         }
     }
 }
 
 template <bool MMA>
-__global__ void __launch_bounds__(THREADS)
+__global__ void __launch_bounds__(THREADS, 4)
 fused_small_kernel(const FusedPlan fp) {
     extern __shared__ __align__(16) float smem[];
+    Instance in;
+    in.smem = smem;
     for (long long inst = blockIdx.x; inst < fp.batch; inst += gridDim.x) {
+        in.inst = inst;
         for (int i = 0; i < fp.n_ops; ++i) {
             const FusedOperand &op = fp.ops[i];
             load_operand(smem + op.smem_off, op.ptr + inst * op.stride, op.rows, op.cols, op.ld, op.prop, op.transposed);
@@ -243,8 +279,8 @@ fused_small_kernel(const FusedPlan fp) {
         cp_async_wait_all();
         __syncthreads();
         for (int s = 0; s < fp.n_steps; ++s) {
-            if (MMA) product_mma(fp, fp.steps[s], smem, inst);
-            else product_ffma(fp, fp.steps[s], smem, inst);
+            if (MMA) product_mma(fp, fp.steps[s], in);
+            else product_ffma(fp, fp.steps[s], in);
             __syncthreads();
         }
     }
