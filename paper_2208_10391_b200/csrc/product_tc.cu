@@ -696,11 +696,16 @@ mom_status_t tc_prepare(const mom_plan &p, TcPlanState &s) {
                     }
                 }
             }
-        // Order.  Unequal tiles (triangular operands): heaviest first, so that the persistent CTAs, which
-        // take tiles round-robin, finish together; structurally zero tiles last.  Equal tiles (general
-        // operands): tiles that run at the same time should share operand panels in L2, so they are
-        // grouped into super-tiles of SUPER_ROWS x SUPER_COLS tiles (about one wave of CTAs, equal bytes
-        // of A and B panels).  (Super-tiles for unequal tiles cost more in imbalance than they saved.)
+        // Order.  Tiles that run at the same time should share operand panels in L2: the output is cut into
+        // bands of BAND tile rows, bands are visited heaviest first (triangular operands make them unequal),
+        // and inside a band the tiles go column by column, every other band backwards.  A wave of CTAs
+        // (or CTA pairs) then covers BAND rows x about units / BAND columns, a near-square block in bytes
+        // of A and B panels, wherever the wave starts.  Structurally zero tiles come last.
+        // Equal tiles are taken round-robin in that order.  Unequal tiles are dealt out by list scheduling on
+        // the host: each tile, in that order, to the unit with the least work so far; the last few waves'
+        // worth of tiles are taken heaviest first so that the units finish together.  Unit u then owns table
+        // entries u, u + units, u + 2*units, ...; rounds a unit has no tile for hold a dummy entry that lies
+        // outside the matrix (nothing loaded or stored).
         bool uniform = true;
         for (const int4 &t : tab) uniform &= (t.w - t.z) == (tab[0].w - tab[0].z);
         int sms = 0;
@@ -711,11 +716,35 @@ mom_status_t tc_prepare(const mom_plan &p, TcPlanState &s) {
         }
         const int units = std::max(1, std::min((int)tab.size(), s.steps[i].pair ? sms / 2 : sms));   // CTAs, or CTA pairs
         s.steps[i].units = units;
+        if (split <= 1) {
+            const int band = s.steps[i].pair ? 8 : 16;                 // tile rows per band (2048 rows)
+            const int n_bands = ((m + tile_rows - 1) / tile_rows + band - 1) / band;
+            auto band_of = [&](const int4 &t) { return (t.x & TILE_ROW_MASK) / tile_rows / band; };
+            std::vector<long long> band_work(n_bands, 0);
+            for (const int4 &t : tab) band_work[band_of(t)] += t.w - t.z;
+            std::vector<int> by_work(n_bands), rank(n_bands);
+            for (int b2 = 0; b2 < n_bands; ++b2) by_work[b2] = b2;
+            std::stable_sort(by_work.begin(), by_work.end(), [&](int x, int y) { return band_work[x] > band_work[y]; });
+            for (int r2 = 0; r2 < n_bands; ++r2) rank[by_work[r2]] = r2;
+            std::stable_sort(tab.begin(), tab.end(), [&](const int4 &x, const int4 &y) {
+                const bool zx = x.w <= x.z, zy = y.w <= y.z;
+                if (zx != zy) return zy;
+                const int rx = rank[band_of(x)], ry = rank[band_of(y)];
+                if (rx != ry) return rx < ry;
+                if (x.y != y.y) return (rx & 1) ? x.y > y.y : x.y < y.y;
+                return (x.x & TILE_ROW_MASK) < (y.x & TILE_ROW_MASK);
+            });
+        }
         if (!uniform) {
-            // Longest-processing-time list scheduling on the host: tiles by decreasing cost, each to the unit
-            // with the least work so far.  Unit u then owns table entries u, u + units, u + 2*units, ...; rounds
-            // a unit has no tile for hold a dummy entry that lies outside the matrix (nothing loaded or stored).
-            std::stable_sort(tab.begin(), tab.end(), [](const int4 &a, const int4 &b) { return (a.w - a.z) > (b.w - b.z); });
+            if (split <= 1) {
+                size_t busy = 0;
+                while (busy < tab.size() && tab[busy].w > tab[busy].z) ++busy;
+                const size_t tail = std::min(busy, (size_t)3 * units);
+                std::stable_sort(tab.begin() + (busy - tail), tab.begin() + busy,
+                                 [](const int4 &x, const int4 &y) { return (x.w - x.z) > (y.w - y.z); });
+            } else {
+                std::stable_sort(tab.begin(), tab.end(), [](const int4 &x, const int4 &y) { return (x.w - x.z) > (y.w - y.z); });
+            }
             constexpr long long TILE_OVERHEAD = 3 * BK;         // epilogue and pipeline fill, in k units
             std::vector<std::vector<int4>> mine(units);
             std::vector<long long> load(units, 0);
@@ -732,19 +761,6 @@ mom_status_t tc_prepare(const mom_plan &p, TcPlanState &s) {
             tab.assign(rounds * units, dummy);
             for (int u = 0; u < units; ++u)
                 for (size_t r = 0; r < mine[u].size(); ++r) tab[r * units + u] = mine[u][r];
-        } else {
-            constexpr int SUPER_ROWS = 16, SUPER_COLS = 8;
-            const int super_cols = ((n + BN - 1) / BN + SUPER_COLS - 1) / SUPER_COLS;
-            auto super_of = [&](const int4 &t) { return ((t.x & TILE_ROW_MASK) / BM / SUPER_ROWS) * super_cols + (t.y / BN / SUPER_COLS); };
-            std::vector<long long> super_work((size_t)(((m + BM - 1) / BM + SUPER_ROWS - 1) / SUPER_ROWS + 1) * super_cols, 0);
-            for (const int4 &t : tab) super_work[super_of(t)] += t.w - t.z;
-            std::stable_sort(tab.begin(), tab.end(), [&](const int4 &a, const int4 &b) {
-                const bool za = a.w <= a.z, zb = b.w <= b.z;
-                if (za != zb) return zb;
-                const int sa = super_of(a), sb = super_of(b);
-                if (sa != sb) return super_work[sa] != super_work[sb] ? super_work[sa] > super_work[sb] : sa < sb;
-                return (a.w - a.z) > (b.w - b.z);
-            });
         }
         total += tab.size();
     }
