@@ -65,16 +65,20 @@ typedef enum { MOM_GENERAL = 0, MOM_LOWER_TRI = 1, MOM_UPPER_TRI = 2, MOM_IDENTI
 typedef enum { MOM_F32 = 0 } mom_dtype_t;
 
 /* Arithmetic used by the product kernels.
- *   MOM_VARIANT_3XTF32: tcgen05 tensor-core MMA (kind::tf32) on operands split as a = hi + lo,
- *       accumulating lo*hi + hi*lo + hi*hi in f32 (f32-level accuracy).  Products whose shapes
- *       cannot be addressed by TMA (a leading dimension that is not a multiple of 4 elements) run
- *       on the FFMA kernel instead.
- *       Small products (m*n*k < 2^23) also run on the FFMA kernel: the operand split and the
- *       tensor pipeline's set-up cost more than they save there.
+ *   MOM_VARIANT_3XTF32: tensor-core MMA (kind::tf32 / .tf32) on operands split as a = hi + lo,
+ *       accumulating lo*hi + hi*lo + hi*hi in f32 (f32-level accuracy).  Large products
+ *       (m*n*k >= 3 * 2^26) whose shapes TMA can address (leading dimensions that are multiples of 4
+ *       elements) run on the tcgen05 kernel (operand planes, TMA, tensor memory).  Smaller products and
+ *       the other shapes run on the warp-level kernel (mma.sync on the operands as stored, one launch per
+ *       product): below that size the tcgen05 path's extra passes cost more than they save.
  *   MOM_VARIANT_FFMA: plain f32 fused multiply-add on CUDA cores.
- *   MOM_VARIANT_3XTF32_FORCE: as 3XTF32 but without the size rule (every TMA-addressable product
- *       runs on tensor cores); meant for testing the tensor-core kernel on small shapes. */
-typedef enum { MOM_VARIANT_3XTF32 = 0, MOM_VARIANT_FFMA = 1, MOM_VARIANT_3XTF32_FORCE = 2 } mom_variant_t;
+ *   MOM_VARIANT_3XTF32_FORCE: every TMA-addressable product runs on the tcgen05 kernel, the others on
+ *       the FFMA kernel; meant for testing the tcgen05 kernel on small shapes.
+ *   MOM_VARIANT_3XTF32_WARP: every product runs on the warp-level kernel; meant for testing it on
+ *       large shapes.
+ * Whatever the variant, equations small enough for shared memory run as one fused launch, and products
+ * with a Diagonal factor run on the scaling kernel. */
+typedef enum { MOM_VARIANT_3XTF32 = 0, MOM_VARIANT_FFMA = 1, MOM_VARIANT_3XTF32_FORCE = 2, MOM_VARIANT_3XTF32_WARP = 3 } mom_variant_t;
 
 /* Kind of a binary product, by which operands are triangular. */
 typedef enum {
@@ -98,7 +102,7 @@ typedef struct {
     int32_t lhs, rhs, out;
     int32_t kind;                    /* mom_kind_t */
     int32_t lhs_property, rhs_property, out_property;
-    int32_t uses_tensor_cores;       /* 1: tcgen05 3xTF32 kernel, 0: FFMA kernel (MOM_KIND_SCALE: the scaling kernel) */
+    int32_t uses_tensor_cores;       /* 1: tcgen05 3xTF32 kernel, 2: warp-level 3xTF32 kernel, 0: FFMA kernel (MOM_KIND_SCALE: the scaling kernel) */
     int32_t lhs_transposed, rhs_transposed;   /* the operand is an original chain operand used transposed */
     int64_t m, n, k;                 /* out is m x n, contraction length k */
     uint64_t useful_mults;           /* scalar multiplications with both factors structurally non-zero */

@@ -14,7 +14,7 @@ from typing import List, Optional, Sequence, Tuple
 
 GENERAL, LOWER_TRI, UPPER_TRI, IDENTITY, DIAGONAL = 0, 1, 2, 3, 4
 F32 = 0
-VARIANT_3XTF32, VARIANT_FFMA, VARIANT_3XTF32_FORCE = 0, 1, 2
+VARIANT_3XTF32, VARIANT_FFMA, VARIANT_3XTF32_FORCE, VARIANT_3XTF32_WARP = 0, 1, 2, 3
 KIND_GG, KIND_TG, KIND_GT, KIND_TT, KIND_TTMIX, KIND_SCALE = 0, 1, 2, 3, 4, 5
 
 (OK, ERR_INVALID_ARG, ERR_PROPERTY, ERR_DTYPE, ERR_SHAPE_MISMATCH, ERR_OVERFLOW, ERR_ALLOC,

@@ -61,6 +61,21 @@ __device__ __forceinline__ float finish_entry(float acc, const AddTerms &add, lo
     return in_structure(out_prop, r, c) ? v : 0.0f;
 }
 
+// The same with a loop over the terms instead of unrolled code (for kernels whose epilogue runs once per
+// thread and should stay small).
+__device__ __forceinline__ float finish_entry_compact(float acc, const AddTerms &add, long long batch, int r, int c,
+                                                       int ld, int out_prop) {
+    float v = acc;
+#pragma unroll 1
+    for (int t = 0; t < add.count; ++t) {
+        const float *p = add.ptr[t];
+        if (!p) { v += r == c ? 1.0f : 0.0f; continue; }
+        p += batch * add.stride[t] + ((add.transposed >> t) & 1u ? (long long)c * add.rows + r : (long long)r * ld + c);
+        v += (add.aliases_out >> t) & 1u ? __ldcg(p) : __ldg(p);
+    }
+    return in_structure(out_prop, r, c) ? v : 0.0f;
+}
+
 // The same for four consecutive entries (r, c .. c+3) of a row, for the kernels that are bound by memory
 // traffic: a compact loop over the terms (no unrolling: these kernels are tiny and must stay in the
 // instruction cache), one 16-byte load per term where its layout allows.  `n` is the row length of X

@@ -122,7 +122,7 @@ mom_status_t execute_impl(const mom_plan *p, const float *const *chain_ptrs, con
     if (st != MOM_OK) return st;
 
     bool any_tc = false;
-    for (const auto &s : p->steps) any_tc |= s.pub.uses_tensor_cores != 0;
+    for (const auto &s : p->steps) any_tc |= s.pub.uses_tensor_cores == 1;
     if (any_tc) {
         st = tc_prepare(*p, p->dev->tc);
         if (st != MOM_OK) return st;
@@ -326,14 +326,16 @@ mom_status_t execute_impl(const mom_plan *p, const float *const *chain_ptrs, con
                 }
                 cudaEvent_t *ev = timing ? &p->dev->events[((size_t)(p->dev->timed_executes % TIMING_SLOTS) * ns + s) * 3] : nullptr;
                 if (ev) cudaEventRecord(ev[0], stream);
-                if (stp.pub.uses_tensor_cores) {
+                if (stp.pub.uses_tensor_cores == 1) {
                     int used = 0;
                     st = tc_launch_step(*p, p->dev->tc, s, a, ws, p->dev->status, stream, &used, ev ? ev[1] : nullptr);
                     if (st != MOM_OK) return st;
                     launches += used;
                 } else {
                     if (ev) cudaEventRecord(ev[1], stream);
-                    const cudaError_t e = stp.pub.kind == MOM_KIND_SCALE ? launch_scale(a, nb, stream) : launch_product_ffma(a, nb, stream);
+                    const cudaError_t e = stp.pub.kind == MOM_KIND_SCALE ? launch_scale(a, nb, stream)
+                                          : stp.pub.uses_tensor_cores == 2 ? launch_product_mma(a, nb, stream)
+                                                                           : launch_product_ffma(a, nb, stream);
                     if (e != cudaSuccess) return MOM_ERR_CUDA;
                     ++launches;
                 }

@@ -21,6 +21,10 @@ struct ProductArgs {
 
 cudaError_t launch_product_ffma(const ProductArgs &a, int batch, cudaStream_t stream);
 
+// The same product on the warp-level tensor-core kernel (mma.sync, 3xTF32 split in registers): one launch,
+// operands read as stored, contraction split over a thread-block cluster when the output has few tiles.
+cudaError_t launch_product_mma(const ProductArgs &a, int batch, cudaStream_t stream);
+
 // The same product when A or B is Diagonal: a row or column scaling of the other operand (one pass).
 cudaError_t launch_scale(const ProductArgs &a, int batch, cudaStream_t stream);
 

@@ -141,7 +141,7 @@ static mom_status_t plan_sums(const std::vector<mom_matrix_desc_t> &slots, const
                               const int32_t *slot_names, const mom_matrix_desc_t *stored_add,
                               const int32_t *add_transposed, int32_t n_add, mom_variant_t variant, mom_plan_t **out_plan) {
     if (!out_plan || sums_in.empty() || n_add < 0 || (n_add > 0 && !stored_add)) return MOM_ERR_INVALID_ARG;
-    if ((int)variant < 0 || (int)variant > 2) return MOM_ERR_INVALID_ARG;
+    if ((int)variant < 0 || (int)variant > 3) return MOM_ERR_INVALID_ARG;
     int64_t total = 0;
     int n_chains = 0;
     for (const SumIn &si : sums_in) {
@@ -384,11 +384,15 @@ static mom_status_t plan_sums(const std::vector<mom_matrix_desc_t> &slots, const
             mom::StepImpl &st = p->steps[s];
             const int64_t m = st.pub.m, n = st.pub.n, k = st.pub.k;
             const bool addressable = (k % 4 == 0) && (n % 4 == 0);
-            const bool worth_it = (double)m * (double)n * (double)k >= (double)(1 << 23);
-            st.pub.uses_tensor_cores =
-                st.pub.kind != MOM_KIND_SCALE &&        // a Diagonal operand: one scaling pass, bound by HBM
-                ((variant == MOM_VARIANT_3XTF32 && addressable && worth_it) || ((int)variant == 2 && addressable));
-            if (st.pub.uses_tensor_cores) {
+            // below this size the tcgen05 path's extra launches (operand splits, split-K reduction) cost more
+            // than its faster mainloop saves; the warp-level kernel is one launch
+            const bool large = (double)m * (double)n * (double)k >= 3.0 * (double)(1 << 26);
+            if (st.pub.kind == MOM_KIND_SCALE) st.pub.uses_tensor_cores = 0;       // a Diagonal operand: one scaling pass, bound by HBM
+            else if (variant == MOM_VARIANT_3XTF32) st.pub.uses_tensor_cores = addressable && large ? 1 : 2;
+            else if (variant == MOM_VARIANT_3XTF32_FORCE) st.pub.uses_tensor_cores = addressable ? 1 : 0;
+            else if (variant == MOM_VARIANT_3XTF32_WARP) st.pub.uses_tensor_cores = 2;
+            else st.pub.uses_tensor_cores = 0;
+            if (st.pub.uses_tensor_cores == 1) {
                 // few output tiles, long contraction: split k over otherwise idle SMs
                 const int64_t tiles = ((m + mom::TC_BM - 1) / mom::TC_BM) * ((n + mom::TC_BN - 1) / mom::TC_BN);
                 if (tiles <= 37 && k >= 512) {
@@ -409,10 +413,10 @@ static mom_status_t plan_sums(const std::vector<mom_matrix_desc_t> &slots, const
                 if (c.pub.lhs != st.pub.out && c.pub.rhs != st.pub.out) continue;
                 last_consumer = t;
                 (c.pub.lhs == st.pub.out ? as_lhs : as_rhs)++;
-                all_tc &= c.pub.uses_tensor_cores != 0;
+                all_tc &= c.pub.uses_tensor_cores == 1;
             }
             const bool fused_planes = last_consumer >= 0 && all_tc && (as_lhs == 0 || as_rhs == 0) &&
-                                      st.pub.uses_tensor_cores && st.split_k == 1;
+                                      st.pub.uses_tensor_cores == 1 && st.split_k == 1;
             if (fused_planes) {
                 st.planes_out = as_lhs ? 1 : 2;
             } else if (!st.is_last) {
@@ -447,7 +451,7 @@ static mom_status_t plan_sums(const std::vector<mom_matrix_desc_t> &slots, const
         std::vector<Copy> copies;
         for (int s = 0; s < ns; ++s) {
             mom::StepImpl &st = p->steps[s];
-            if (!st.pub.uses_tensor_cores) continue;
+            if (st.pub.uses_tensor_cores != 1) continue;
             const int64_t m = st.pub.m, n = st.pub.n, k = st.pub.k;
             for (int side = 0; side < 2; ++side) {
                 const int32_t v = side == 0 ? st.pub.lhs : st.pub.rhs;
@@ -500,12 +504,12 @@ static mom_status_t plan_sums(const std::vector<mom_matrix_desc_t> &slots, const
         // Small equations run as one fused kernel with every operand and intermediate in shared memory.
         {
             bool any_tc = false;
-            for (const auto &st : p->steps) any_tc |= st.pub.uses_tensor_cores != 0;
+            for (const auto &st : p->steps) any_tc |= st.pub.uses_tensor_cores == 1;
             const int values = n_chain + ns;
             p->fused_value_off.assign(values, -1);
             size_t floats = 0;
             bool ok = single_chain && ns >= 1 && ns <= mom::FUSED_MAX_STEPS && (int)p->kept.size() <= mom::FUSED_MAX_OPERANDS &&
-                      n_add <= mom::MAX_FUSED_ADD && !any_tc;
+                      n_add <= mom::MAX_FUSED_ADD && !any_tc && variant != MOM_VARIANT_3XTF32_WARP;
             // every value feeds exactly one product: remember on which side
             std::vector<char> is_rhs(values, 0);
             for (const auto &st : p->steps) is_rhs[st.pub.rhs] = 1;
@@ -729,7 +733,7 @@ mom_status_t mom_plan_workspace_bytes(const mom_plan_t *plan, int64_t batch, siz
     // workspace; all-FFMA plans run up to 65535 instances per launch and keep one copy of each
     // intermediate per instance.
     bool any_tc = false;
-    for (const auto &s : plan->steps) any_tc |= s.pub.uses_tensor_cores != 0;
+    for (const auto &s : plan->steps) any_tc |= s.pub.uses_tensor_cores == 1;
     const int64_t group = any_tc ? 1 : (batch < 65535 ? batch : 65535);
     *bytes = plan->workspace_per_instance * (size_t)group;
     return MOM_OK;

@@ -669,7 +669,7 @@ mom_status_t tc_prepare(const mom_plan &p, TcPlanState &s) {
     size_t total = 0;
     for (int i = 0; i < ns; ++i) {
         const mom_step_t &st = p.steps[i].pub;
-        if (!st.uses_tensor_cores) continue;
+        if (st.uses_tensor_cores != 1) continue;
         const int m = (int)st.m, n = (int)st.n, k = (int)st.k;
         std::vector<int4> &tab = tables[i];
         // CTA pairs (256-row tiles) once there are enough of them to occupy most of the GPU's 74 pairs

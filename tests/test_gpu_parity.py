@@ -13,8 +13,8 @@ from gpu_util import run_equation, check_against_oracle, TOL
 
 pytestmark = pytest.mark.gpu
 
-VARIANTS = [mom.VARIANT_FFMA, mom.VARIANT_3XTF32_FORCE]
-VNAME = {mom.VARIANT_FFMA: "ffma", mom.VARIANT_3XTF32_FORCE: "tc", mom.VARIANT_3XTF32: "auto"}
+VARIANTS = [mom.VARIANT_FFMA, mom.VARIANT_3XTF32_FORCE, mom.VARIANT_3XTF32_WARP]
+VNAME = {mom.VARIANT_FFMA: "ffma", mom.VARIANT_3XTF32_FORCE: "tc", mom.VARIANT_3XTF32: "auto", mom.VARIANT_3XTF32_WARP: "warp"}
 
 
 def both(eq, variant, **kw):
@@ -62,6 +62,7 @@ def test_split_k_products(pa, pb):
     eq = Equation(f"splitk_{pa}{pb}", 60, (Operand(am, ak, pa, "normal" if pa == G else "uniform"),
                                            Operand(bk, bn, pb, "normal" if pb == G else "uniform")), add)
     both(eq, mom.VARIANT_3XTF32_FORCE)
+    both(eq, mom.VARIANT_3XTF32_WARP)       # the warp-level kernel splits the contraction over a thread-block cluster
     # the same product as the inner step of a chain whose next step is a tensor-core step too
     eq = Equation(f"splitk_chain_{pa}{pb}", 61, (Operand(200, am, G, "normal"), Operand(am, ak, pa, "normal" if pa == G else "uniform"),
                                                  Operand(bk, bn, pb, "normal" if pb == G else "uniform")))
@@ -121,7 +122,7 @@ def test_pair_kernel_ragged_shapes(case):
     else:
         eq = Equation("pair_chain", 72, (Operand(m, m, U), Operand(m, k, G, "normal", 0.02), Operand(k, k, L), Operand(k, n, G, "normal", 0.02)))
     x, plan, (chain, add) = run_equation(eq, mom.VARIANT_3XTF32)
-    assert all(s.uses_tensor_cores for s in plan.steps())
+    assert all(s.uses_tensor_cores == 1 for s in plan.steps())
     rows = np.sort(np.random.default_rng(3).choice(m, size=40, replace=False))
     rows[:6] = [0, 127, 128, 255, 256, m - 1]
     check_against_oracle(eq, x, plan, chain, add, rows=np.sort(rows))
@@ -304,7 +305,7 @@ def test_transposed_operands_large_sampled_rows():
     eq = Equation("transpose_pair", 82, (Operand(m, m, L), Operand(n, m, G, "normal", 0.02)), (Operand(m, n, G, "normal"),),
                   chain_t=(True, True))
     x, plan, (chain, add) = run_equation(eq, mom.VARIANT_3XTF32)
-    assert plan.step(0).uses_tensor_cores and plan.step(0).lhs_property == U
+    assert plan.step(0).uses_tensor_cores == 1 and plan.step(0).lhs_property == U
     rows = np.sort(np.random.default_rng(4).choice(m, size=32, replace=False))
     check_against_oracle(eq, x, plan, chain, add, rows=rows)
 

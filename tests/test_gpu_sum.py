@@ -12,7 +12,7 @@ from gpu_util import run_sum_equation, check_sum_against_oracle, TOL
 
 pytestmark = pytest.mark.gpu
 
-VARIANTS = [mom.VARIANT_3XTF32, mom.VARIANT_FFMA, mom.VARIANT_3XTF32_FORCE]
+VARIANTS = [mom.VARIANT_3XTF32, mom.VARIANT_FFMA, mom.VARIANT_3XTF32_FORCE, mom.VARIANT_3XTF32_WARP]
 
 
 def sum_eq(name, chains, transposed=None, names=None, seed=11):
@@ -88,8 +88,12 @@ def test_rectangular_chains_on_several_tiles(variant):
 def test_split_k_roots_accumulate():
     # few output tiles and a long contraction: both roots run split over k and the second adds to X
     eq = sum_eq("splitk", [[(128, 4096, G), (4096, 256, G)], [(128, 2048, G), (2048, 256, G)]])
+    x, plan, arrays = run_sum_equation(eq, mom.VARIANT_3XTF32_FORCE)
+    assert all(s.uses_tensor_cores == 1 for s in plan.steps())
+    check_sum_against_oracle(eq, x, plan, arrays)
+    # the same roots on the warp-level kernel: the contraction is split over a thread-block cluster
     x, plan, arrays = run_sum_equation(eq, mom.VARIANT_3XTF32)
-    assert all(s.uses_tensor_cores for s in plan.steps())
+    assert all(s.uses_tensor_cores == 2 for s in plan.steps())
     check_sum_against_oracle(eq, x, plan, arrays)
 
 

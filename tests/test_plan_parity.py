@@ -129,11 +129,19 @@ def test_workspace_covers_intermediates_and_planes():
     p = mom.mom_equation_plan(eq.descs(), (), mom.VARIANT_3XTF32)
     assert all(s.uses_tensor_cores == 1 for s in p.steps())
     assert p.workspace_bytes() >= 2 * n * n * 4 + 4 * n * n * 4
-    # shapes TMA cannot address fall back to FFMA; tiny products too
+    # shapes TMA cannot address fall back to FFMA when the tcgen05 kernel is forced; in the default variant they
+    # and all small products run on the warp-level kernel (one launch per product)
     p = mom.mom_equation_plan([(5, 5, 1), (5, 5, 1)], (), mom.VARIANT_3XTF32_FORCE)
     assert p.step(0).uses_tensor_cores == 0
     p = mom.mom_equation_plan(wl.config_tiny().descs(), (), mom.VARIANT_3XTF32)
-    assert all(s.uses_tensor_cores == 0 for s in p.steps())
+    assert all(s.uses_tensor_cores == 2 for s in p.steps())
+    p = mom.mom_equation_plan(wl.config_paper_chain().descs(), (), mom.VARIANT_3XTF32)
+    up = lambda b: (b + 255) // 256 * 256          # two f32 intermediates, no operand planes
+    assert all(s.uses_tensor_cores == 2 for s in p.steps()) and p.workspace_bytes() == up(900 * 100 * 4) + up(1100 * 100 * 4)
+    p = mom.mom_equation_plan([(1001, 1001, 0), (1001, 1001, 0)], (), mom.VARIANT_3XTF32)
+    assert p.step(0).uses_tensor_cores == 2
+    p = mom.mom_equation_plan(wl.config_property_heavy().descs(), (), mom.VARIANT_3XTF32_WARP)
+    assert all(s.uses_tensor_cores == 2 for s in p.steps())
     p = mom.mom_equation_plan(wl.config_tiny().descs(), (), mom.VARIANT_3XTF32_FORCE)
     assert all(s.uses_tensor_cores == 1 for s in p.steps())
     assert mom.mom_equation_plan(wl.config_tiny_identity_left().descs()).workspace_bytes() == 0
