@@ -16,6 +16,8 @@ struct DeviceState {
     int device = -1;
     int32_t *status = nullptr;          // device: {code, detail, 0, 0}
     TcPlanState tc;                     // tile tables of tensor-core steps
+    uint2 *fused_table = nullptr;       // copy table of the fused small-equation kernel
+    std::vector<int> fused_tab_begin, fused_tab_end;    // per kept operand: its rows of the table
     // step timing: a ring of TIMING_SLOTS executes, 3 events per step (before pre-pass, before product, after)
     std::vector<cudaEvent_t> events;
     long long timed_executes = 0;       // executes recorded since timing was enabled
@@ -43,6 +45,7 @@ void destroy_device_state(DeviceState *d) {
     if (d->call_start) cudaEventDestroy(d->call_start);
     if (d->copy_stream) cudaStreamDestroy(d->copy_stream);
     if (d->status) cudaFree(d->status);
+    if (d->fused_table) cudaFree(d->fused_table);
     if (prev >= 0) cudaSetDevice(prev);
     delete d;
 }
@@ -153,11 +156,31 @@ mom_status_t execute_impl(const mom_plan *p, const float *const *chain_ptrs, con
         FusedPlan fp;
         std::memset(&fp, 0, sizeof(fp));
         fp.n_ops = (int)p->kept.size();
+        DeviceState *dev = p->dev;
+        if (dev->fused_tab_begin.empty()) {
+            // first execute: the copy table of every operand that is read as stored in whole 16-byte pieces
+            // (operand pointers and instance strides are 16-byte aligned, checked above)
+            std::vector<uint2> table;
+            dev->fused_tab_begin.assign(fp.n_ops, 0);
+            dev->fused_tab_end.assign(fp.n_ops, 0);
+            for (int i = 0; i < fp.n_ops; ++i) {
+                const int id = p->kept[i];
+                if (p->chain_t[id] || p->chain[id].cols % 4 != 0) continue;
+                dev->fused_tab_begin[i] = (int)(table.size() / FUSED_THREADS);
+                dev->fused_tab_end[i] = dev->fused_tab_begin[i] + fused_copy_table((int)p->chain[id].rows, (int)p->chain[id].cols, p->chain[id].property,
+                                                                                    p->fused_value_off[id], p->fused_value_ld[id], table);
+            }
+            if (!table.empty()) {
+                if (cudaMalloc(&dev->fused_table, table.size() * sizeof(uint2)) != cudaSuccess) return MOM_ERR_ALLOC;
+                if (cudaMemcpy(dev->fused_table, table.data(), table.size() * sizeof(uint2), cudaMemcpyHostToDevice) != cudaSuccess) return MOM_ERR_CUDA;
+            }
+        }
+        fp.copy_table = dev->fused_table;
         for (int i = 0; i < fp.n_ops; ++i) {
             const int id = p->kept[i], slot = p->factor_ptr[id];
             fp.ops[i] = FusedOperand{chain_ptrs[slot], chain_strides ? chain_strides[slot] : 0, (int)p->chain[id].rows,
                                      (int)p->chain[id].cols, p->chain[id].property, p->fused_value_off[id], p->fused_value_ld[id],
-                                     (int)p->chain_t[id]};
+                                     (int)p->chain_t[id], dev->fused_tab_begin[i], dev->fused_tab_end[i]};
         }
         fp.n_steps = (int)p->steps.size();
         for (int s = 0; s < fp.n_steps; ++s) {

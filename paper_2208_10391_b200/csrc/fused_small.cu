@@ -19,7 +19,7 @@ namespace mom {
 
 namespace {
 
-constexpr int THREADS = 256;
+constexpr int THREADS = FUSED_THREADS;
 constexpr int WARPS = THREADS / 32;
 
 // Copy one operand (rows x cols, row-major, leading dimension cols) into shared memory with leading
@@ -270,11 +270,22 @@ fused_small_kernel(const FusedPlan fp) {
     extern __shared__ __align__(16) float smem[];
     Instance in;
     in.smem = smem;
+    const uint32_t smem_base = static_cast<uint32_t>(__cvta_generic_to_shared(smem));
     for (long long inst = blockIdx.x; inst < fp.batch; inst += gridDim.x) {
         in.inst = inst;
         for (int i = 0; i < fp.n_ops; ++i) {
             const FusedOperand &op = fp.ops[i];
-            load_operand(smem + op.smem_off, op.ptr + inst * op.stride, op.rows, op.cols, op.ld, op.prop, op.transposed);
+            const float *src = op.ptr + inst * op.stride;
+            if (op.tab_end > op.tab_begin) {
+                const uint2 *e = fp.copy_table + (size_t)op.tab_begin * THREADS + threadIdx.x;
+                for (int row = op.tab_begin; row < op.tab_end; ++row, e += THREADS) {
+                    const uint2 c = __ldg(e);
+                    if (c.x != FUSED_COPY_NONE)
+                        asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(smem_base + (c.x & ~15u)), "l"(src + c.y), "r"((c.x & 1u) ? 16 : 0) : "memory");
+                }
+            } else {
+                load_operand(smem + op.smem_off, src, op.rows, op.cols, op.ld, op.prop, op.transposed);
+            }
         }
         cp_async_wait_all();
         __syncthreads();
@@ -290,6 +301,21 @@ int g_sm_count = 0;
 int g_max_smem[2] = {0, 0};
 
 }  // namespace
+
+int fused_copy_table(int rows, int cols, int prop, int smem_off, int ld, std::vector<uint2> &table) {
+    const size_t first = table.size();
+    const bool lower = prop == MOM_LOWER_TRI || prop == MOM_DIAGONAL, upper = prop == MOM_UPPER_TRI || prop == MOM_DIAGONAL;
+    for (int r = 0; r < rows; ++r) {
+        const int block = r & ~15;
+        for (int c = 0; c < cols; c += 4) {
+            if ((lower && c >= block + 16) || (upper && c + 3 < block)) continue;      // never read by any product
+            const bool needed = !((lower && c > r) || (upper && c + 3 < r));
+            table.push_back(make_uint2((uint32_t)(smem_off + r * ld + c) * 4u | (needed ? 1u : 0u), (uint32_t)(r * cols + c)));
+        }
+    }
+    while ((table.size() - first) % FUSED_THREADS != 0) table.push_back(make_uint2(FUSED_COPY_NONE, 0));
+    return (int)((table.size() - first) / FUSED_THREADS);
+}
 
 cudaError_t launch_fused_small(const FusedPlan &fp, size_t smem_bytes, cudaStream_t stream) {
     if (!g_sm_count) {

@@ -3,6 +3,8 @@
 
 #include <cuda_runtime.h>
 
+#include <vector>
+
 #include "device_common.cuh"
 
 namespace mom {
@@ -18,6 +20,7 @@ struct FusedOperand {
     int smem_off;            // floats
     int ld;                  // leading dimension in shared memory (floats)
     int transposed;          // stored as cols x rows; read transposed into shared memory
+    int tab_begin, tab_end;  // rows of the copy table that fetch this operand; empty: the generic loader does it
 };
 
 struct FusedStep {
@@ -37,7 +40,20 @@ struct FusedPlan {
     long long out_stride;
     long long batch;
     int use_mma;             // 1: tensor-core mma.sync with the 3xTF32 split, 0: plain FMA
+    const uint2 *copy_table; // device: FUSED_THREADS entries per row, see fused_copy_table()
 };
+
+constexpr int FUSED_THREADS = 256;
+constexpr uint32_t FUSED_COPY_NONE = 0xFFFFFFFFu;
+
+// Copy table of an operand that is read as stored with rows of whole 16-byte pieces: where every 16-byte
+// piece of one instance goes, worked out once on the host so that the kernel (bound by instruction issue)
+// spends a load and an add per copy instead of index arithmetic.  Entry (row, thread): x = byte offset in
+// shared memory | 1 if the piece meets the operand's structure (else it is zero-filled without a read),
+// y = offset in floats from the instance's first element; x = FUSED_COPY_NONE: nothing to do.  Pieces that no
+// product can read (beyond the 16-column block of a triangular row's diagonal) get no entry.
+// Appends whole rows to `table` and returns the number of rows appended.
+int fused_copy_table(int rows, int cols, int prop, int smem_off, int ld, std::vector<uint2> &table);
 
 // Leading dimension (floats) of a matrix with `cols` columns held in shared memory.  A value is read
 // by exactly one product, as its left or its right operand; the padding makes that product's
