@@ -304,6 +304,13 @@ mom_status_t execute_impl(const mom_plan *p, const float *const *chain_ptrs, con
 
             for (int s = sum.step_begin; s < sum.step_end; ++s) {
                 const StepImpl &stp = p->steps[s];
+                if (stp.folded) {                        // a scaling done by its reader's operand-split pass: nothing to launch
+                    if (timing) {
+                        cudaEvent_t *fe = &p->dev->events[((size_t)(p->dev->timed_executes % TIMING_SLOTS) * ns + s) * 3];
+                        for (int q = 0; q < 3; ++q) cudaEventRecord(fe[q], stream);
+                    }
+                    continue;
+                }
                 auto value = [&](int id) {
                     if (id < n_chain) return chain_op(id);
                     const StepImpl &prod = p->steps[id - n_chain];
@@ -313,17 +320,33 @@ mom_status_t execute_impl(const mom_plan *p, const float *const *chain_ptrs, con
                     if (prod.out_off == SIZE_MAX) return Operand{nullptr, elems};
                     return Operand{reinterpret_cast<const float *>(ws + prod.out_off * (size_t)nb), elems};
                 };
-                need_value(stp.pub.lhs);
-                need_value(stp.pub.rhs);
                 if (stp.is_last && !stp.accumulate) need_summands(sum);
-                const Operand A = value(stp.pub.lhs), B = value(stp.pub.rhs);
                 ProductArgs a;
                 std::memset(&a, 0, sizeof(a));
-                a.A = A.ptr; a.B = B.ptr;
-                a.strideA = A.stride; a.strideB = B.stride;
                 a.m = (int)stp.pub.m; a.n = (int)stp.pub.n; a.k = (int)stp.pub.k;
                 a.pa = stp.pub.lhs_property; a.pb = stp.pub.rhs_property;
-                a.transA = stp.pub.lhs_transposed; a.transB = stp.pub.rhs_transposed;
+                // an operand: the value itself, or d * S / S * d of a folded scaling step (S read as stored, d handed
+                // to the split pass)
+                auto operand = [&](int id, int fold, const float **ptr, long long *stride, int *trans, int own_trans,
+                                   const float **scale, long long *scale_step, int *scale_rows) {
+                    if (fold < 0) {
+                        need_value(id);
+                        const Operand o = value(id);
+                        *ptr = o.ptr; *stride = o.stride; *trans = own_trans;
+                        return;
+                    }
+                    const mom_step_t &sc = p->steps[fold].pub;
+                    const bool left = sc.lhs_property == MOM_DIAGONAL;          // d * S
+                    const int s_id = left ? sc.rhs : sc.lhs, d_id = left ? sc.lhs : sc.rhs;
+                    need_value(s_id);
+                    need_value(d_id);
+                    const Operand o = value(s_id), d = value(d_id);
+                    *ptr = o.ptr; *stride = o.stride;
+                    *trans = left ? sc.rhs_transposed : sc.lhs_transposed;
+                    *scale = d.ptr; *scale_step = sc.k + 1; *scale_rows = left ? 1 : 0;
+                };
+                operand(stp.pub.lhs, stp.fold_a, &a.A, &a.strideA, &a.transA, stp.pub.lhs_transposed, &a.scaleA, &a.scaleA_step, &a.scaleA_rows);
+                operand(stp.pub.rhs, stp.fold_b, &a.B, &a.strideB, &a.transB, stp.pub.rhs_transposed, &a.scaleB, &a.scaleB_step, &a.scaleB_rows);
                 if (stp.is_last && stp.accumulate) {
                     // a later chain's product is added to what the earlier ones left in the sum's buffer
                     a.C = x; a.strideC = x_stride;

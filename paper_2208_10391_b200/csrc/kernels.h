@@ -17,6 +17,11 @@ struct ProductArgs {
     int transA, transB;                     // the operand is stored transposed (k x m resp. n x k)
     long long strideA, strideB, strideC;    // elements between batch instances
     AddTerms add;
+    // tensor-core path only: the operand is d * A (rows of A as used scaled, scale_rows != 0) or A * d (columns);
+    // d points at a dense Diagonal matrix whose entries are scale_step floats apart; NULL: no scaling
+    const float *scaleA, *scaleB;
+    long long scaleA_step, scaleB_step;
+    int scaleA_rows, scaleB_rows;
 };
 
 cudaError_t launch_product_ffma(const ProductArgs &a, int batch, cudaStream_t stream);

@@ -45,6 +45,11 @@ struct StepImpl {
     // different CTAs; the slices' partial sums go to scratch and a small kernel adds them up.
     int split_k = 1;
     size_t partial_off = SIZE_MAX;
+    // A scaling step (Diagonal factor) whose only reader is a tensor-core step is folded into that step's
+    // operand-split pass: it launches nothing and has no buffer; the reader splits d * S instead of S.
+    bool folded = false;
+    int fold_into = -1;             // folded step: the tensor-core step that reads it
+    int fold_a = -1, fold_b = -1;   // tensor-core step: the folded scaling step behind its left / right operand
 };
 
 // One summand of X = sum of chain values + Add terms, in the order written.

@@ -401,6 +401,22 @@ static mom_status_t plan_sums(const std::vector<mom_matrix_desc_t> &slots, const
                 }
             }
         }
+        // A scaling step read by exactly one tensor-core step is folded into that step's operand-split pass.
+        for (int s = 0; s < ns; ++s) {
+            mom::StepImpl &st = p->steps[s];
+            if (st.pub.kind != MOM_KIND_SCALE || st.is_last) continue;
+            if (st.pub.lhs_property == MOM_DIAGONAL && st.pub.rhs_property == MOM_DIAGONAL) continue;
+            int readers = 0, reader = -1;
+            for (int t = s + 1; t < ns; ++t)
+                if (p->steps[t].pub.lhs == st.pub.out || p->steps[t].pub.rhs == st.pub.out) { ++readers; reader = t; }
+            if (readers != 1 || p->steps[reader].pub.uses_tensor_cores != 1) continue;
+            if (p->steps[reader].pub.lhs == st.pub.out && p->steps[reader].pub.rhs == st.pub.out) continue;
+            st.folded = true;
+            st.fold_into = reader;
+            (p->steps[reader].pub.lhs == st.pub.out ? p->steps[reader].fold_a : p->steps[reader].fold_b) = s;
+        }
+        // the step at which a reader really reads its operands: a folded step's operands are read by its target
+        auto read_at = [&](int t) { return p->steps[t].folded ? p->steps[t].fold_into : t; };
         // f32 intermediates, or planes written by the producer: a tensor-core producer writes its consumers' operand
         // planes itself when every consumer is a tensor-core step that takes the value on the same side
         for (int s = 0; s < ns; ++s) {
@@ -411,7 +427,7 @@ static mom_status_t plan_sums(const std::vector<mom_matrix_desc_t> &slots, const
             for (int t = s + 1; t < ns; ++t) {
                 const mom::StepImpl &c = p->steps[t];
                 if (c.pub.lhs != st.pub.out && c.pub.rhs != st.pub.out) continue;
-                last_consumer = t;
+                last_consumer = std::max(last_consumer, read_at(t));
                 (c.pub.lhs == st.pub.out ? as_lhs : as_rhs)++;
                 all_tc &= c.pub.uses_tensor_cores == 1;
             }
@@ -419,7 +435,7 @@ static mom_status_t plan_sums(const std::vector<mom_matrix_desc_t> &slots, const
                                       st.pub.uses_tensor_cores == 1 && st.split_k == 1;
             if (fused_planes) {
                 st.planes_out = as_lhs ? 1 : 2;
-            } else if (!st.is_last) {
+            } else if (!st.is_last && !st.folded) {
                 items.push_back(Interval{mom::align_up((size_t)m * n * sizeof(float), mom::WS_ALIGN), s,
                                          last_consumer < 0 ? ns - 1 : last_consumer, &st.out_off, 0});
             }
@@ -433,7 +449,7 @@ static mom_status_t plan_sums(const std::vector<mom_matrix_desc_t> &slots, const
             for (int t = 0; t < ns; ++t) {
                 const mom_step_t &c = p->steps[t].pub;
                 const bool reads = (c.lhs < n_chain && p->factor_sum[c.lhs] == (int)si) || (c.rhs < n_chain && p->factor_sum[c.rhs] == (int)si);
-                if (reads) last = std::max(last, t);
+                if (reads) last = std::max(last, read_at(t));
             }
             for (size_t sj = si + 1; sj < p->sums.size(); ++sj)
                 for (const mom::Summand &sm : p->sums[sj].summands)

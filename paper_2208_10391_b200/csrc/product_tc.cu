@@ -552,9 +552,19 @@ product_tc_pair_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __gri
 // needs it: the plain path needs cols % 4 == 0, the transposing path rows % 4 == 0.
 constexpr int SPLIT_PIECE = 64;
 
+// Optional scaling folded into the split (a product with a Diagonal factor whose only reader is this
+// operand): entry (r, c) of the matrix as stored is multiplied by d[r] (by_row) or d[c] before it is split;
+// d's entries are `step` floats apart (the diagonal of a dense matrix).  d == NULL: no scaling.
+struct SplitScale {
+    const float *d;
+    long long step;
+    int by_row;
+};
+
 template <bool TRANSPOSE>
 __global__ void __launch_bounds__(256)
-split_planes_kernel(const float *__restrict__ src, float *__restrict__ hi, float *__restrict__ lo, int rows, int cols, int prop) {
+split_planes_kernel(const float *__restrict__ src, float *__restrict__ hi, float *__restrict__ lo, int rows, int cols, int prop,
+                    SplitScale sc) {
     const int pr = blockIdx.y * SPLIT_PIECE, pc = blockIdx.x * SPLIT_PIECE;
     const int br = pr / SPLIT_BLOCK * SPLIT_BLOCK, bc = pc / SPLIT_BLOCK * SPLIT_BLOCK;
     if (prop == MOM_LOWER_TRI && bc > br + SPLIT_BLOCK - 1) return;     // block wholly above the diagonal
@@ -566,7 +576,16 @@ split_planes_kernel(const float *__restrict__ src, float *__restrict__ hi, float
             const int r = pr + (e >> 4), c = pc + ((e & 15) << 2);
             if (r < rows && c < cols) {
                 const size_t off = (size_t)r * cols + c;
-                const float4 a = __ldg(reinterpret_cast<const float4 *>(src + off));
+                float4 a = __ldg(reinterpret_cast<const float4 *>(src + off));
+                if (sc.d) {
+                    if (sc.by_row) {
+                        const float f = __ldg(sc.d + r * sc.step);
+                        a.x *= f; a.y *= f; a.z *= f; a.w *= f;
+                    } else {
+                        a.x *= __ldg(sc.d + c * sc.step); a.y *= __ldg(sc.d + (c + 1) * sc.step);
+                        a.z *= __ldg(sc.d + (c + 2) * sc.step); a.w *= __ldg(sc.d + (c + 3) * sc.step);
+                    }
+                }
                 float4 h, l;
                 h.x = ptx::to_tf32(a.x); h.y = ptx::to_tf32(a.y); h.z = ptx::to_tf32(a.z); h.w = ptx::to_tf32(a.w);
                 l.x = ptx::to_tf32(a.x - h.x); l.y = ptx::to_tf32(a.y - h.y); l.z = ptx::to_tf32(a.z - h.z); l.w = ptx::to_tf32(a.w - h.w);
@@ -580,7 +599,9 @@ split_planes_kernel(const float *__restrict__ src, float *__restrict__ hi, float
         for (int i = 0; i < 16; ++i) {
             const int e = threadIdx.x + 256 * i;                         // 64 x 64 scalars, row-contiguous reads
             const int r = e >> 6, c = e & 63;
-            tile[r][c] = (pr + r < rows && pc + c < cols) ? __ldg(src + (size_t)(pr + r) * cols + pc + c) : 0.0f;
+            float v = (pr + r < rows && pc + c < cols) ? __ldg(src + (size_t)(pr + r) * cols + pc + c) : 0.0f;
+            if (sc.d && pr + r < rows && pc + c < cols) v *= __ldg(sc.d + (sc.by_row ? pr + r : pc + c) * sc.step);
+            tile[r][c] = v;
         }
         __syncthreads();
 #pragma unroll
@@ -815,14 +836,17 @@ mom_status_t tc_launch_step(const mom_plan &p, TcPlanState &s, int step, const P
     auto stored_prop = [](int prop_as_used) {
         return prop_as_used == MOM_LOWER_TRI ? (int)MOM_UPPER_TRI : prop_as_used == MOM_UPPER_TRI ? (int)MOM_LOWER_TRI : prop_as_used;
     };
+    // a folded scaling: rows of the operand as used <-> rows of the matrix as stored unless it is stored transposed
+    const SplitScale sa{a.scaleA, a.scaleA_step, a.scaleA ? (a.scaleA_rows != 0) != (a.transA != 0) : 0};
+    const SplitScale sb{a.scaleB, a.scaleB_step, a.scaleB ? (a.scaleB_rows != 0) != (a.transB != 0) : 0};
     if (!st.a_planes_ready) {
-        if (!a.transA) split_planes_kernel<false><<<dim3(blocks(a.k), blocks(a.m)), 256, 0, stream>>>(a.A, a_hi, a_lo, a.m, a.k, a.pa);
-        else split_planes_kernel<true><<<dim3(blocks(a.m), blocks(a.k)), 256, 0, stream>>>(a.A, a_hi, a_lo, a.k, a.m, stored_prop(a.pa));
+        if (!a.transA) split_planes_kernel<false><<<dim3(blocks(a.k), blocks(a.m)), 256, 0, stream>>>(a.A, a_hi, a_lo, a.m, a.k, a.pa, sa);
+        else split_planes_kernel<true><<<dim3(blocks(a.m), blocks(a.k)), 256, 0, stream>>>(a.A, a_hi, a_lo, a.k, a.m, stored_prop(a.pa), sa);
         ++split_launches;
     }
     if (!st.b_planes_ready) {
-        if (!a.transB) split_planes_kernel<true><<<dim3(blocks(a.n), blocks(a.k)), 256, 0, stream>>>(a.B, b_hi, b_lo, a.k, a.n, a.pb);
-        else split_planes_kernel<false><<<dim3(blocks(a.k), blocks(a.n)), 256, 0, stream>>>(a.B, b_hi, b_lo, a.n, a.k, stored_prop(a.pb));
+        if (!a.transB) split_planes_kernel<true><<<dim3(blocks(a.n), blocks(a.k)), 256, 0, stream>>>(a.B, b_hi, b_lo, a.k, a.n, a.pb, sb);
+        else split_planes_kernel<false><<<dim3(blocks(a.k), blocks(a.n)), 256, 0, stream>>>(a.B, b_hi, b_lo, a.n, a.k, stored_prop(a.pb), sb);
         ++split_launches;
     }
     if (cudaGetLastError() != cudaSuccess) return MOM_ERR_CUDA;
@@ -1080,8 +1104,8 @@ extern "C" mom_status_t mom_product_3xtf32_noalloc(int64_t m64, int64_t n64, int
 
     auto blocks = [](int x) { return (x + SPLIT_PIECE - 1) / SPLIT_PIECE; };
     noalloc_build_tiles_kernel<<<(unsigned)((tiles + 127) / 128), 128, 0, stream>>>(table, m, n, k, (int)pa, (int)pb);
-    split_planes_kernel<false><<<dim3(blocks(k), blocks(m)), 256, 0, stream>>>(A, a_hi, a_lo, m, k, (int)pa);
-    split_planes_kernel<true><<<dim3(blocks(n), blocks(k)), 256, 0, stream>>>(B, b_hi, b_lo, k, n, (int)pb);
+    split_planes_kernel<false><<<dim3(blocks(k), blocks(m)), 256, 0, stream>>>(A, a_hi, a_lo, m, k, (int)pa, SplitScale{nullptr, 0, 0});
+    split_planes_kernel<true><<<dim3(blocks(n), blocks(k)), 256, 0, stream>>>(B, b_hi, b_lo, k, n, (int)pb, SplitScale{nullptr, 0, 0});
     if (cudaGetLastError() != cudaSuccess) return MOM_ERR_CUDA;
 
     CUtensorMap ma_hi, ma_lo, mb_hi, mb_lo, mc;

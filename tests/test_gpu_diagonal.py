@@ -59,6 +59,32 @@ def test_scalings_inside_chains(variant):
         both(Equation("dd_plus", 39, (Operand(n, n, D), Operand(n, n, D)), tuple(terms)), variant)
 
 
+@pytest.mark.parametrize("trans", [False, True])
+@pytest.mark.parametrize("side", ["left_row", "left_col", "right_row", "right_col"])
+def test_scaling_folded_into_the_operand_split(side, trans):
+    # a scaling whose only reader is a tensor-core product costs no launch: the reader's split pass scales as it
+    # reads.  The scaled matrix is the product's left or right operand, scaled by rows (D*S) or by columns (S*D),
+    # stored as used or transposed.
+    m, k, n = 264, 392, 520
+    g = lambda r, c: Operand(c, r, G, "normal") if trans else Operand(r, c, G, "normal")
+    if side == "left_row":      # (D * A) * B with a tall B, so that D joins A
+        chain, ct = (Operand(m, m, D), g(m, k), Operand(k, n, G, "normal")), (False, trans, False)
+    elif side == "left_col":    # (A * D) * B
+        chain, ct = (g(m, k), Operand(k, k, D), Operand(k, n + 400, G, "normal")), (trans, False, False)
+    elif side == "right_row":   # A * (D * B)
+        chain, ct = (Operand(m + 400, k, G, "normal"), Operand(k, k, D), g(k, n)), (False, False, trans)
+    else:                       # A * (B * D)
+        chain, ct = (Operand(m + 400, k, G, "normal"), g(k, n), Operand(n, n, D)), (False, trans, False)
+    eq = Equation(f"fold_{side}_{int(trans)}", 50, chain, (), 1, ct)
+    _, x, plan = both(eq, mom.VARIANT_3XTF32_FORCE)
+    kinds = [plan.step(i).kind for i in range(plan.num_steps())]
+    assert kinds.count(mom.KIND_SCALE) == 1 and plan.step(kinds.index(mom.KIND_SCALE)).out != plan.step(plan.num_steps() - 1).out
+    assert plan.last_launch_count() == 3        # two operand splits and the product; no scaling launch
+    # the other kernels take the scaled matrix from memory: same values
+    both(eq, mom.VARIANT_3XTF32_WARP)
+    both(eq, mom.VARIANT_FFMA)
+
+
 @pytest.mark.parametrize("variant", VARIANTS, ids=VNAME.get)
 def test_zero_step_plans_with_diagonals(variant):
     n = 33
