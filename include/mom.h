@@ -250,6 +250,11 @@ mom_status_t mom_equation_execute_batched(const mom_plan_t *plan, const float *c
  * Add terms, X, and the workspace, for `batch` instances. */
 mom_status_t mom_plan_host_staging_bytes(const mom_plan_t *plan, int64_t batch, size_t *bytes);
 
+/* Bytes mom_equation_execute_host copies from the host per call: every used operand and Add term once (a
+ * named matrix once); of a large triangular operand (batch == 1, at least 1024 rows) only the blocks of 256
+ * rows up to (from) the diagonal block are copied, the rest of its device copy is zero-filled on the device. */
+mom_status_t mom_plan_host_upload_bytes(const mom_plan_t *plan, int64_t batch, size_t *bytes);
+
 /* Same evaluation with HOST operands and a HOST result: copies the operands into `staging` (device,
  * 256-byte aligned, at least mom_plan_host_staging_bytes), runs the plan, copies X back into
  * out_host, all on `stream`; returns after the stream has been synchronised.  Instances are packed

@@ -82,6 +82,7 @@ _sigs = {
                                      ctypes.POINTER(ctypes.c_int64), _P, ctypes.c_int64, ctypes.c_int64, _P,
                                      ctypes.c_size_t, _P],
     "mom_plan_host_staging_bytes": [_P, ctypes.c_int64, ctypes.POINTER(ctypes.c_size_t)],
+    "mom_plan_host_upload_bytes": [_P, ctypes.c_int64, ctypes.POINTER(ctypes.c_size_t)],
     "mom_equation_execute_host": [_P, ctypes.POINTER(_P), ctypes.POINTER(_P), _P, ctypes.c_int64, _P,
                                   ctypes.c_size_t, _P],
     "mom_plan_device_status": [_P, ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_int32)],
@@ -202,6 +203,11 @@ class Plan:
     def host_staging_bytes(self, batch: int = 1) -> int:
         b = ctypes.c_size_t()
         _check(_lib.mom_plan_host_staging_bytes(self._h, batch, ctypes.byref(b)), "mom_plan_host_staging_bytes")
+        return b.value
+
+    def host_upload_bytes(self, batch: int = 1) -> int:
+        b = ctypes.c_size_t()
+        _check(_lib.mom_plan_host_upload_bytes(self._h, batch, ctypes.byref(b)), "mom_plan_host_upload_bytes")
         return b.value
 
     def device_status(self) -> Tuple[int, int]:

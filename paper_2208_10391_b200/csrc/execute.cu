@@ -33,6 +33,21 @@ struct StageEvents { const cudaEvent_t *slot; const cudaEvent_t *add; };
 
 constexpr int TIMING_SLOTS = 32;
 
+// host-staging entry point: triangular operands of at least UPLOAD_MIN rows are uploaded in blocks of UPLOAD_BLOCK rows
+constexpr int64_t UPLOAD_BLOCK = 256, UPLOAD_MIN = 1024;
+inline bool triangular_upload(const mom_matrix_desc_t &d, int64_t batch) {
+    return batch == 1 && d.rows >= UPLOAD_MIN && (d.property == MOM_LOWER_TRI || d.property == MOM_UPPER_TRI);
+}
+inline size_t upload_bytes(const mom_matrix_desc_t &d, int64_t batch) {
+    if (!triangular_upload(d, batch)) return (size_t)d.rows * d.cols * sizeof(float) * batch;
+    size_t total = 0;
+    for (int64_t r0 = 0; r0 < d.rows; r0 += UPLOAD_BLOCK) {
+        const int64_t r1 = std::min<int64_t>(d.rows, r0 + UPLOAD_BLOCK);
+        total += (size_t)(r1 - r0) * (size_t)(d.property == MOM_LOWER_TRI ? r1 : d.rows - r0) * sizeof(float);
+    }
+    return total;
+}
+
 void destroy_device_state(DeviceState *d) {
     if (!d) return;
     int prev = -1;
@@ -493,7 +508,21 @@ mom_status_t mom_equation_execute_host(const mom_plan_t *plan, const float *cons
     std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return first_use[a] < first_use[b]; });
     for (int i : order) {
         if (same_as[i] >= 0) continue;
-        if (cbytes[i] && cudaMemcpyAsync(const_cast<float *>(cptr[i]), chain_host[i], cbytes[i], cudaMemcpyHostToDevice, dev->copy_stream) != cudaSuccess)
+        if (cbytes[i] && mom::triangular_upload(plan->ptr_desc[i], batch)) {
+            // a large triangular operand: the host buffer holds zeros outside the triangle (storage contract), so
+            // only the 256-row blocks' columns up to (from) the diagonal block cross the bus; the rest is zero-filled here
+            const mom_matrix_desc_t &d = plan->ptr_desc[i];
+            float *dst = const_cast<float *>(cptr[i]);
+            const int64_t n = d.rows;
+            if (cudaMemsetAsync(dst, 0, cbytes[i], dev->copy_stream) != cudaSuccess) return MOM_ERR_CUDA;
+            for (int64_t r0 = 0; r0 < n; r0 += mom::UPLOAD_BLOCK) {
+                const int64_t r1 = std::min(n, r0 + mom::UPLOAD_BLOCK);
+                const int64_t c0 = d.property == MOM_LOWER_TRI ? 0 : r0, c1 = d.property == MOM_LOWER_TRI ? r1 : n;
+                if (cudaMemcpy2DAsync(dst + r0 * n + c0, (size_t)n * sizeof(float), chain_host[i] + r0 * n + c0, (size_t)n * sizeof(float),
+                                      (size_t)(c1 - c0) * sizeof(float), (size_t)(r1 - r0), cudaMemcpyHostToDevice, dev->copy_stream) != cudaSuccess)
+                    return MOM_ERR_CUDA;
+            }
+        } else if (cbytes[i] && cudaMemcpyAsync(const_cast<float *>(cptr[i]), chain_host[i], cbytes[i], cudaMemcpyHostToDevice, dev->copy_stream) != cudaSuccess)
             return MOM_ERR_CUDA;
         if (cudaEventRecord(dev->slot_ready[i], dev->copy_stream) != cudaSuccess) return MOM_ERR_CUDA;
         for (int j = i + 1; j < n_chain; ++j)
@@ -533,6 +562,24 @@ mom_status_t mom_equation_execute_host(const mom_plan_t *plan, const float *cons
     if (st != MOM_OK) return st;
     if (cudaMemcpyAsync(out_host, x, xbytes, cudaMemcpyDeviceToHost, stream) != cudaSuccess) return MOM_ERR_CUDA;
     if (cudaStreamSynchronize(stream) != cudaSuccess) return MOM_ERR_CUDA;
+    return MOM_OK;
+}
+
+mom_status_t mom_plan_host_upload_bytes(const mom_plan_t *plan, int64_t batch, size_t *bytes) {
+    if (!plan || !bytes || batch < 1) return MOM_ERR_INVALID_ARG;
+    size_t total = 0;
+    const int n = (int)plan->ptr_desc.size();
+    for (int i = 0; i < n; ++i) {
+        const mom_matrix_desc_t &d = plan->ptr_desc[i];
+        if (d.property == MOM_IDENTITY || !plan->slot_used[i]) continue;
+        bool seen = false;                               // a named matrix is copied once
+        if (!plan->names.empty())
+            for (int j = 0; j < i && !seen; ++j) seen = plan->names[j] == plan->names[i] && plan->slot_used[j];
+        if (!seen) total += mom::upload_bytes(d, batch);
+    }
+    for (const auto &d : plan->add)
+        if (d.property != MOM_IDENTITY) total += (size_t)d.rows * d.cols * sizeof(float) * batch;
+    *bytes = total;
     return MOM_OK;
 }
 

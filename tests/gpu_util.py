@@ -29,7 +29,7 @@ def run_equation(eq: wl.Equation, variant: int, chain=None, add=None, via: str =
     stream = torch.cuda.current_stream().cuda_stream
     if via == "host":
         stage_bytes = plan.host_staging_bytes(batch)
-        staging = torch.empty(max(stage_bytes, 256), dtype=torch.uint8, device="cuda")
+        staging = torch.full((max(stage_bytes, 256),), 255, dtype=torch.uint8, device="cuda")   # NaN patterns: nothing stale may be read
         pinned = [None if a is None else torch.from_numpy(a).pin_memory() for a in chain]
         pinned_add = [None if a is None else torch.from_numpy(a).pin_memory() for a in add]
         out = torch.full((n_out,), float("nan"), dtype=torch.float32).pin_memory()

@@ -225,6 +225,26 @@ def test_random_equations(variant):
         both(eq, variant)
 
 
+def test_host_entry_point_uploads_large_triangles_by_blocks():
+    # triangular operands of 1024 rows or more cross the bus only up to (from) their diagonal blocks of 256 rows;
+    # the device copy is completed with zeros, so the result is the device entry point's, bit for bit
+    n = 1288                                 # not a multiple of the block
+    eq = Equation("host_tri", 90, (Operand(n, n, L), Operand(n, n, G, "normal", 0.03), Operand(n, n, U)), (Operand(n, n, G, "normal"),))
+    chain, add = wl.generate(eq)
+    xd, plan, _ = run_equation(eq, mom.VARIANT_3XTF32, chain, add, via="device")
+    xh, _, _ = run_equation(eq, mom.VARIANT_3XTF32, chain, add, via="host")
+    assert np.array_equal(xd, xh)
+    full = 4 * n * n * 4
+    blocks = [(r0, min(n, r0 + 256)) for r0 in range(0, n, 256)]
+    lower = sum((r1 - r0) * r1 for r0, r1 in blocks) * 4
+    upper = sum((r1 - r0) * (n - r0) for r0, r1 in blocks) * 4
+    assert plan.host_upload_bytes(1) == full - 2 * n * n * 4 + lower + upper < 0.85 * full
+    # a stale staging area must not leak into the zero-filled part: run once more after poisoning is done by run_equation
+    xh2, _, _ = run_equation(eq, mom.VARIANT_FFMA, chain, add, via="host")
+    xd2, _, _ = run_equation(eq, mom.VARIANT_FFMA, chain, add, via="device")
+    assert np.array_equal(xd2, xh2)
+
+
 @pytest.mark.parametrize("variant", VARIANTS, ids=VNAME.get)
 def test_host_entry_point_matches_device_entry_point(variant):
     for eq in (wl.config_tiny(), wl.config_batched(batch=9), wl.config_property_heavy(n=264)):
