@@ -25,6 +25,15 @@ Readings taken where the paper is silent (each also listed in the design notes):
     for it): a square matrix stored densely whose entries off the diagonal are zero.  Unlike Identity
     its diagonal is data, so it is never simplified away; D*A costs one multiplication per structural
     entry of A; the transpose of a Diagonal matrix is Diagonal;
+  * Symmetric (another of those properties, again without a printed rule): a square matrix stored densely
+    in full with a_ij = a_ji.  Its structure is full, so it costs what a general matrix costs; S^T = S; a
+    product with a Symmetric factor is general (S*I = S); a sum of Symmetric, Diagonal and Identity
+    summands is Symmetric;
+  * Gram products: when the factors are named (equal names = the same matrix) and a sub-chain reads
+    Y * Y^T factor by factor (second half = first half reversed, every factor transposed; Symmetric and
+    Diagonal factors are their own transposes), its value is Symmetric whatever the tree, and the tree that
+    splits it in the middle computes only Y and then the lower triangle of Y * Y^T: the right half costs
+    nothing and the product costs the multiplications of the entries (i, j) with i >= j;
   * a transposed operand (paper Table 1, "Transpose") takes part with its transposed type: shape
     swapped and lowerTri <-> upperTri (the inference rule the paper prints);
   * reported mul_flops = 2 * multiplications; add_flops = structural non-zeros of the Add terms.
@@ -36,8 +45,8 @@ from __future__ import annotations
 from dataclasses import dataclass
 from typing import List, Optional, Sequence, Tuple
 
-GENERAL, LOWER_TRI, UPPER_TRI, IDENTITY, DIAGONAL = 0, 1, 2, 3, 4
-PROPERTIES = (GENERAL, LOWER_TRI, UPPER_TRI, IDENTITY, DIAGONAL)
+GENERAL, LOWER_TRI, UPPER_TRI, IDENTITY, DIAGONAL, SYMMETRIC = 0, 1, 2, 3, 4, 5
+PROPERTIES = (GENERAL, LOWER_TRI, UPPER_TRI, IDENTITY, DIAGONAL, SYMMETRIC)
 
 
 class OracleError(ValueError):
@@ -67,6 +76,7 @@ class Step:
     rhs_prop: int
     out_prop: int
     mults: int
+    gram: bool = False   # out = lhs * lhs^T (rhs is the same value, read transposed); only entries i >= j are counted
 
 
 @dataclass(frozen=True)
@@ -87,7 +97,7 @@ class Plan:
 
 def in_structure(prop: int, i: int, j: int) -> bool:
     """Is entry (i, j) a structural non-zero of a matrix with this property?"""
-    if prop == GENERAL:
+    if prop in (GENERAL, SYMMETRIC):
         return True
     if prop == LOWER_TRI:
         return i >= j
@@ -104,7 +114,7 @@ def brute_force_nonzeros(d: Desc) -> int:
 
 
 def structural_nonzeros(d: Desc) -> int:
-    if d.prop == GENERAL:
+    if d.prop in (GENERAL, SYMMETRIC):
         return d.rows * d.cols
     if d.prop in (LOWER_TRI, UPPER_TRI):
         return d.rows * (d.rows + 1) // 2
@@ -150,12 +160,29 @@ def product_mults(a: Desc, b: Desc) -> int:
     return n * (n + 1) * (2 * n + 1) // 6   # L*U, U*L: sum of squares
 
 
+def brute_force_gram_mults(y: Desc) -> int:
+    """#{(i, l, j): i >= j, (i, l) in S(Y) and (j, l) in S(Y)}: the multiplications of the lower triangle of Y*Y^T."""
+    return sum(1 for i in range(y.rows) for j in range(i + 1) for l in range(y.cols)
+               if in_structure(y.prop, i, l) and in_structure(y.prop, j, l))
+
+
+def gram_mults(y: Desc) -> int:
+    """The same in closed form (Y general, Symmetric or triangular)."""
+    if y.prop in (LOWER_TRI, UPPER_TRI):
+        n = y.rows
+        return n * (n + 1) * (n + 2) // 6
+    return y.cols * y.rows * (y.rows + 1) // 2
+
+
 def join(p: int, q: int) -> int:
-    """Property of a product: least upper bound in Identity < Diagonal < {lowerTri, upperTri} < general."""
+    """Property of a product: least upper bound in Identity < Diagonal < {lowerTri, upperTri} < general;
+    a product with a Symmetric factor is general (only S*I = S)."""
     if p == IDENTITY:
         return q
     if q == IDENTITY:
         return p
+    if SYMMETRIC in (p, q):
+        return GENERAL
     if p == q:
         return p
     if p == DIAGONAL:
@@ -174,9 +201,12 @@ def sum_property(product_prop: int, add_props: Sequence[int]) -> int:
     """
     if not add_props:
         return product_prop
+    props = [DIAGONAL if p == IDENTITY else p for p in [product_prop] + list(add_props)]
+    if SYMMETRIC in props:          # Symmetric + (Symmetric | Diagonal) is Symmetric; a triangle or a general summand breaks it
+        return SYMMETRIC if all(p in (SYMMETRIC, DIAGONAL) for p in props) else GENERAL
     out = DIAGONAL
-    for p in [product_prop] + list(add_props):
-        out = join(out, DIAGONAL if p == IDENTITY else p)
+    for p in props:
+        out = join(out, p)
     return out
 
 
@@ -193,7 +223,7 @@ def _validate(chain: Sequence[Desc], add: Sequence[Desc]) -> None:
         if d.prop not in PROPERTIES:
             raise OracleError("property", "unknown property")
         if d.prop != GENERAL and d.rows != d.cols:
-            raise OracleError("property", "triangular / Diagonal / Identity matrices are square")
+            raise OracleError("property", "triangular / Diagonal / Symmetric / Identity matrices are square")
     for a, b in zip(chain[:-1], chain[1:]):
         if a.cols != b.rows:
             raise OracleError("shape_mismatch", "inner dimensions differ")
@@ -220,13 +250,40 @@ def all_trees(lo: int, hi: int):
                 yield (split, left, right)
 
 
-def _tree_desc_cost(tree, descs: Sequence[Desc]) -> Tuple[Desc, int]:
+def _span(tree) -> Tuple[int, int]:
+    if isinstance(tree, int):
+        return tree, tree
+    _, left, right = tree
+    return _span(left)[0], _span(right)[1]
+
+
+def _reads_as_gram(lo: int, hi: int, descs: Sequence[Desc], ident) -> bool:
+    """Do the factors lo..hi read Y * Y^T?  `ident[i]` = (name, transposed) of factor i, or None when nothing
+    is known about it.  Factor hi - q must be the transpose of factor lo + q: the same matrix with the other
+    flag, or the same matrix with any flag when it is its own transpose (Symmetric, Diagonal)."""
+    if ident is None or (hi - lo + 1) % 2:
+        return False
+    for q in range((hi - lo + 1) // 2):
+        a, b = ident[lo + q], ident[hi - q]
+        if a is None or b is None or a[0] != b[0]:
+            return False
+        if a[1] == b[1] and descs[lo + q].prop not in (SYMMETRIC, DIAGONAL):
+            return False
+    return True
+
+
+def _tree_desc_cost(tree, descs: Sequence[Desc], ident=None) -> Tuple[Desc, int]:
     if isinstance(tree, int):
         return descs[tree], 0
-    _, left, right = tree
-    dl, cl = _tree_desc_cost(left, descs)
-    dr, cr = _tree_desc_cost(right, descs)
-    node = Desc(dl.rows, dr.cols, join(dl.prop, dr.prop))
+    split, left, right = tree
+    lo, hi = _span(tree)
+    dl, cl = _tree_desc_cost(left, descs, ident)
+    dr, cr = _tree_desc_cost(right, descs, ident)
+    prop = join(dl.prop, dr.prop)
+    gram = prop == GENERAL and _reads_as_gram(lo, hi, descs, ident)
+    node = Desc(dl.rows, dr.cols, SYMMETRIC if gram else prop)
+    if gram and 2 * split == lo + hi - 1:           # split in the middle: the right half is never computed
+        return node, cl + gram_mults(dl)
     return node, cl + cr + product_mults(dl, dr)
 
 
@@ -247,18 +304,21 @@ def _paren(tree, kept: Sequence[int], transposed: Sequence[bool] = ()) -> str:
 
 def transpose_desc(d: Desc) -> Desc:
     """Type of A^T given the type of A: shape swapped; paper Section 2, "Transformations", prints the
-    inference rule lowerTriangular(A) -> upperTriangular(A^T) (and symmetrically); general, Diagonal and
-    Identity keep their property."""
+    inference rule lowerTriangular(A) -> upperTriangular(A^T) (and symmetrically); general, Diagonal,
+    Symmetric and Identity keep their property."""
     prop = {LOWER_TRI: UPPER_TRI, UPPER_TRI: LOWER_TRI}.get(d.prop, d.prop)
     return Desc(d.cols, d.rows, prop)
 
 
 def plan(chain: Sequence[Tuple[int, int, int]], add: Sequence[Tuple[int, int, int]] = (),
-         chain_transposed: Sequence[bool] = (), add_transposed: Sequence[bool] = ()) -> Plan:
+         chain_transposed: Sequence[bool] = (), add_transposed: Sequence[bool] = (),
+         names: Optional[Sequence[int]] = None) -> Plan:
     """Plan `X = prod(chain) + sum(add)`; operands are (rows, cols, property) triples of the STORED matrices.
 
     `chain_transposed[i]` / `add_transposed[i]` say that the equation uses the transpose of that operand
     (paper Table 1, "Transpose"); the plan then works with the transposed type and prints the operand as `i^T`.
+    `names[i]` identifies the matrix behind chain operand i (equal names = the same matrix); only with names can
+    a sub-chain be recognised as a Gram product Y * Y^T.
     """
     stored_c = [Desc(*c) for c in chain]
     stored_a = [Desc(*a) for a in add]
@@ -282,9 +342,10 @@ def plan(chain: Sequence[Tuple[int, int, int]], add: Sequence[Tuple[int, int, in
                     Desc(rows, cols, sum_property(IDENTITY, [t.prop for t in adescs])), kept)
 
     reduced = [cdescs[i] for i in kept]
+    ident = None if names is None else [(names[i], bool(tc[i])) for i in kept]
     best = None
     for tree in all_trees(0, len(reduced) - 1):
-        _, cost = _tree_desc_cost(tree, reduced)
+        _, cost = _tree_desc_cost(tree, reduced, ident)
         key = (cost, _preorder_splits(tree))
         if best is None or key < best[0]:
             best = (key, tree)
@@ -296,10 +357,19 @@ def plan(chain: Sequence[Tuple[int, int, int]], add: Sequence[Tuple[int, int, in
     def emit(t) -> Tuple[int, Desc]:
         if isinstance(t, int):
             return kept[t], reduced[t]
-        _, left, right = t
+        split, left, right = t
+        lo, hi = _span(t)
         lid, ld = emit(left)
+        oid_prop = _tree_desc_cost(t, reduced, ident)[0].prop
+        if oid_prop == SYMMETRIC and 2 * split == lo + hi - 1 and _reads_as_gram(lo, hi, reduced, ident):
+            # Y * Y^T: the right half is the same value read transposed; nothing is emitted for it
+            rt = transpose_desc(ld)
+            oid = next_id[0]
+            next_id[0] += 1
+            steps.append(Step(lid, lid, oid, ld.rows, ld.rows, ld.cols, ld.prop, rt.prop, SYMMETRIC, gram_mults(ld), True))
+            return oid, Desc(ld.rows, ld.rows, SYMMETRIC)
         rid, rd = emit(right)
-        out = Desc(ld.rows, rd.cols, join(ld.prop, rd.prop))
+        out = Desc(ld.rows, rd.cols, oid_prop)
         oid = next_id[0]
         next_id[0] += 1
         steps.append(Step(lid, rid, oid, ld.rows, rd.cols, ld.cols, ld.prop, rd.prop, out.prop,
@@ -371,7 +441,7 @@ def plan_sum(chains: Sequence[Sequence[Tuple[int, int, int]]],
         counter = iter(range(total))
         names = [[next(counter) for _ in ch] for ch in chains]
 
-    plans = [plan(ch, (), fl) for ch, fl in zip(chains, flags)]
+    plans = [plan(ch, (), fl, (), nm) for ch, fl, nm in zip(chains, flags, names)]
     rows, cols = plans[0].product_desc.rows, plans[0].product_desc.cols
     for p in plans[1:]:
         if (p.product_desc.rows, p.product_desc.cols) != (rows, cols):
@@ -386,12 +456,16 @@ def plan_sum(chains: Sequence[Sequence[Tuple[int, int, int]]],
     parens: List[str] = []
     for c, (p, ch) in enumerate(zip(plans, chains)):
         n_local = len(ch)
-        span = {i: (i, i) for i in range(n_local)}          # local id -> factor positions covered
+        # local id -> the run of (name, transposed) factors it multiplies; the right half of a Gram product
+        # Y * Y^T is Y's run reversed with every flag flipped
+        run = {i: ((names[c][i], flags[c][i]),) for i in range(n_local)}
         to_global = {i: base + i for i in range(n_local)}
         for s in p.steps:
-            lo, hi = span[s.lhs][0], span[s.rhs][1]
-            span[s.out] = (lo, hi)
-            kept_run = tuple((names[c][i], flags[c][i]) for i in range(lo, hi + 1) if i in p.kept)
+            if s.gram:
+                run[s.out] = run[s.lhs] + tuple((nm, not fl) for nm, fl in reversed(run[s.lhs]))
+            else:
+                run[s.out] = run[s.lhs] + run[s.rhs]
+            kept_run = run[s.out]
             is_root = s is p.steps[-1]
             if not is_root and kept_run in seen:
                 to_global[s.out] = seen[kept_run]
@@ -403,7 +477,7 @@ def plan_sum(chains: Sequence[Sequence[Tuple[int, int, int]]],
             if not is_root:
                 seen[kept_run] = gid
             steps.append(Step(to_global[s.lhs], to_global[s.rhs], gid, s.m, s.n, s.k,
-                              s.lhs_prop, s.rhs_prop, s.out_prop, s.mults))
+                              s.lhs_prop, s.rhs_prop, s.out_prop, s.mults, s.gram))
         if p.steps:
             values.append(to_global[p.steps[-1].out])
         elif p.kept:

@@ -18,7 +18,7 @@ from typing import List, Optional, Sequence, Tuple
 
 import numpy as np
 
-GENERAL, LOWER_TRI, UPPER_TRI, IDENTITY, DIAGONAL = 0, 1, 2, 3, 4
+GENERAL, LOWER_TRI, UPPER_TRI, IDENTITY, DIAGONAL, SYMMETRIC = 0, 1, 2, 3, 4, 5
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "matmul_f64.c")
@@ -93,7 +93,7 @@ def transposed_operands(arrays, descs, flags):
     """Operands as the equation uses them: entry i transposed (array and descriptor) where flags[i] is set.
 
     The transpose of a stored lowerTri matrix is upperTri and vice versa (the paper's printed inference
-    rule); Identity, Diagonal and general keep their property.  Dense storage is simply transposed with NumPy.
+    rule); Identity, Diagonal, Symmetric and general keep their property.  Dense storage is simply transposed with NumPy.
     """
     swap = {LOWER_TRI: UPPER_TRI, UPPER_TRI: LOWER_TRI}
     out_a, out_d = [], []
@@ -200,7 +200,8 @@ def evaluate_steps(chain: Sequence[Optional[np.ndarray]], chain_descs: Sequence[
             for i in range(len(chain))}
     last = None
     for s in steps:
-        vals[s.out] = matmul(vals[s.lhs], vals[s.rhs], threads)
+        rhs = np.ascontiguousarray(vals[s.lhs].T) if getattr(s, "gram", False) else vals[s.rhs]   # Y * Y^T
+        vals[s.out] = matmul(vals[s.lhs], rhs, threads)
         last = s.out
     if last is None:
         kept = [i for i in range(len(chain)) if chain_descs[i][2] != IDENTITY]
@@ -225,7 +226,7 @@ def off_structure_mask(rows: int, cols: int, prop: int, row_index: Optional[np.n
     """Boolean mask of entries that lie OUTSIDE the structure of `prop` (must hold exact zeros)."""
     i = (np.arange(rows) if row_index is None else np.asarray(row_index))[:, None]
     j = np.arange(cols)[None, :]
-    if prop == GENERAL:
+    if prop in (GENERAL, SYMMETRIC):
         return np.zeros((i.shape[0], cols), dtype=bool)
     if prop == LOWER_TRI:
         return i < j

@@ -25,9 +25,9 @@ from typing import List, Optional, Sequence
 
 import numpy as np
 
-GENERAL, LOWER_TRI, UPPER_TRI, IDENTITY, DIAGONAL = 0, 1, 2, 3, 4
+GENERAL, LOWER_TRI, UPPER_TRI, IDENTITY, DIAGONAL, SYMMETRIC = 0, 1, 2, 3, 4, 5
 PROPERTY_NAMES = {GENERAL: "general", LOWER_TRI: "lowerTri", UPPER_TRI: "upperTri", IDENTITY: "Identity",
-                  DIAGONAL: "diagonal"}
+                  DIAGONAL: "diagonal", SYMMETRIC: "symmetric"}
 
 
 @dataclass(frozen=True)
@@ -39,7 +39,8 @@ class Operand:
           "ones"     -> every structural entry 1 (the paper's Listing 2 fill)
     Triangular operands always use: strict part from `dist`, diagonal 1 + U(0, 1)
     (except dist == "ones"), other half exactly zero.  Diagonal operands: diagonal
-    1 + U(0, 1) (or ones), everything else exactly zero.
+    1 + U(0, 1) (or ones), everything else exactly zero.  Symmetric operands: the lower triangle
+    from `dist`, mirrored into the upper one (exactly symmetric in float32).
     """
     rows: int
     cols: int
@@ -96,6 +97,11 @@ def generate_operand(op: Operand, seed: int, index: int, batch: int = 1) -> Opti
         keep = (np.tril(np.ones((n, n), dtype=bool)) if op.prop == LOWER_TRI else
                 np.triu(np.ones((n, n), dtype=bool)) if op.prop == UPPER_TRI else np.eye(n, dtype=bool))
         m = np.where(keep, m, np.float32(0.0)).astype(np.float32)
+    if op.prop == SYMMETRIC:
+        if op.rows != op.cols:
+            raise ValueError("symmetric operands are square")
+        low = np.tril(m)
+        m = low + np.swapaxes(np.tril(m, -1), -1, -2)
     return np.ascontiguousarray(m, dtype=np.float32)
 
 
