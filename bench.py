@@ -307,7 +307,7 @@ def run_gpu(args):
         cfgs = {c.name: c for c in (wl.config_tiny(), wl.config_five_general(), wl.config_property_heavy(),
                                     wl.config_large_square(), wl.config_batched(), wl.config_paper_chain(),
                                     wl.config_transposed(), wl.config_sum_shared(), wl.config_sum_triangular(),
-                                    wl.config_expression(), wl.config_diagonal())}
+                                    wl.config_expression(), wl.config_diagonal(), wl.config_gram())}
         cfg = cfgs[args.only]
         r = time_equation(mom, torch, cfg, variant, steps=args.steps, warmup=args.warmup, stream=stream,
                           timing=getattr(cfg, "batch", 1) == 1)
@@ -443,7 +443,7 @@ def run_gpu(args):
         others = []
         for cfg in (wl.config_tiny(), wl.config_five_general(), wl.config_property_heavy(), wl.config_batched(),
                     wl.config_paper_chain(), wl.config_transposed(), wl.config_sum_shared(), wl.config_sum_triangular(),
-                    wl.config_expression(), wl.config_diagonal()):
+                    wl.config_expression(), wl.config_diagonal(), wl.config_gram()):
             batch = getattr(cfg, "batch", 1)
             r = time_equation(mom, torch, cfg, variant, steps=20, warmup=3, stream=stream, timing=batch == 1)
             ms_min, ms_med = min(r["ms"]), statistics.median(r["ms"])

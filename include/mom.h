@@ -40,7 +40,7 @@ extern "C" {
 typedef enum {
     MOM_OK = 0,
     MOM_ERR_INVALID_ARG = 1,         /* null pointer, n_chain < 1, rows/cols < 1, bad enum, batch < 1 */
-    MOM_ERR_PROPERTY = 2,            /* triangular, Diagonal or Identity descriptor that is not square */
+    MOM_ERR_PROPERTY = 2,            /* triangular, Diagonal, Symmetric or Identity descriptor that is not square */
     MOM_ERR_DTYPE = 3,               /* element type other than f32                                   */
     MOM_ERR_SHAPE_MISMATCH = 4,      /* inner dimensions differ, or an Add term's shape != X's shape  */
     MOM_ERR_OVERFLOW = 5,            /* a multiplication count does not fit in 63 bits                */
@@ -60,8 +60,16 @@ typedef enum {
  * it): a square matrix, stored densely like every other operand, whose entries off the diagonal are zeros.
  * Unlike Identity its diagonal is data: it is never simplified away, D*A costs one multiplication per
  * structural entry of A and runs as a scaling pass, D^T = D, and the lattice of product and sum types is
- * Identity < Diagonal < {lowerTri, upperTri} < general. */
-typedef enum { MOM_GENERAL = 0, MOM_LOWER_TRI = 1, MOM_UPPER_TRI = 2, MOM_IDENTITY = 3, MOM_DIAGONAL = 4 } mom_property_t;
+ * Identity < Diagonal < {lowerTri, upperTri} < general.
+ * MOM_SYMMETRIC is another such property: a square matrix stored densely IN FULL (both triangles) with
+ * a_ij = a_ji; the library relies on that and does not check it.  Its structure is full, so it costs what a
+ * general matrix costs; S^T = S; a product with a Symmetric factor is general; a sum of Symmetric, Diagonal
+ * and Identity summands is Symmetric.  Symmetric values also arise inside plans: where factor names are known
+ * (mom_equation_plan_sum with names, mom_expression_plan), a sub-chain that reads Y * Y^T factor by factor
+ * is typed Symmetric, and the tree that splits it in the middle computes Y once and then only the lower
+ * triangle of Y * Y^T (MOM_KIND_GRAM): the right half is never multiplied.  A computed Symmetric value is
+ * symmetric up to rounding in its diagonal blocks and exactly symmetric elsewhere (mirrored). */
+typedef enum { MOM_GENERAL = 0, MOM_LOWER_TRI = 1, MOM_UPPER_TRI = 2, MOM_IDENTITY = 3, MOM_DIAGONAL = 4, MOM_SYMMETRIC = 5 } mom_property_t;
 typedef enum { MOM_F32 = 0 } mom_dtype_t;
 
 /* Arithmetic used by the product kernels.
@@ -87,7 +95,8 @@ typedef enum {
     MOM_KIND_GT = 2,     /* general * triangular                               */
     MOM_KIND_TT = 3,     /* L*L or U*U: result keeps the triangle              */
     MOM_KIND_TTMIX = 4,  /* L*U or U*L: result is general                      */
-    MOM_KIND_SCALE = 5   /* a Diagonal operand on either side: rows or columns of the other operand are scaled */
+    MOM_KIND_SCALE = 5,  /* a Diagonal operand on either side: rows or columns of the other operand are scaled */
+    MOM_KIND_GRAM = 6    /* Y * Y^T: rhs is the same value as lhs, read transposed; useful_mults counts entries i >= j */
 } mom_kind_t;
 
 typedef struct {
@@ -103,7 +112,7 @@ typedef struct {
     int32_t kind;                    /* mom_kind_t */
     int32_t lhs_property, rhs_property, out_property;
     int32_t uses_tensor_cores;       /* 1: tcgen05 3xTF32 kernel, 2: warp-level 3xTF32 kernel, 0: FFMA kernel (MOM_KIND_SCALE: the scaling kernel) */
-    int32_t lhs_transposed, rhs_transposed;   /* the operand is an original chain operand used transposed */
+    int32_t lhs_transposed, rhs_transposed;   /* the operand is read transposed (an original chain operand used transposed; the rhs of MOM_KIND_GRAM) */
     int64_t m, n, k;                 /* out is m x n, contraction length k */
     uint64_t useful_mults;           /* scalar multiplications with both factors structurally non-zero */
 } mom_step_t;

@@ -12,10 +12,10 @@ import ctypes
 import os
 from typing import List, Optional, Sequence, Tuple
 
-GENERAL, LOWER_TRI, UPPER_TRI, IDENTITY, DIAGONAL = 0, 1, 2, 3, 4
+GENERAL, LOWER_TRI, UPPER_TRI, IDENTITY, DIAGONAL, SYMMETRIC = 0, 1, 2, 3, 4, 5
 F32 = 0
 VARIANT_3XTF32, VARIANT_FFMA, VARIANT_3XTF32_FORCE, VARIANT_3XTF32_WARP = 0, 1, 2, 3
-KIND_GG, KIND_TG, KIND_GT, KIND_TT, KIND_TTMIX, KIND_SCALE = 0, 1, 2, 3, 4, 5
+KIND_GG, KIND_TG, KIND_GT, KIND_TT, KIND_TTMIX, KIND_SCALE, KIND_GRAM = 0, 1, 2, 3, 4, 5, 6
 
 (OK, ERR_INVALID_ARG, ERR_PROPERTY, ERR_DTYPE, ERR_SHAPE_MISMATCH, ERR_OVERFLOW, ERR_ALLOC,
  ERR_WORKSPACE_TOO_SMALL, ERR_ALIGNMENT, ERR_ARCH, ERR_CUDA, ERR_DEVICE_TIMEOUT, ERR_BUFFER_TOO_SMALL,

@@ -40,7 +40,7 @@ __host__ __device__ inline void tile_k_range(int pa, int pb, int r0, int r1, int
 }
 
 __host__ __device__ inline bool in_structure(int prop, int r, int c) {
-    return prop == MOM_GENERAL || (prop == MOM_LOWER_TRI && r >= c) || (prop == MOM_UPPER_TRI && r <= c) ||
+    return prop == MOM_GENERAL || prop == MOM_SYMMETRIC || (prop == MOM_LOWER_TRI && r >= c) || (prop == MOM_UPPER_TRI && r <= c) ||
            ((prop == MOM_IDENTITY || prop == MOM_DIAGONAL) && r == c);
 }
 

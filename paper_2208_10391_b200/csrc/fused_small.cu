@@ -38,7 +38,7 @@ __device__ void load_operand(float *__restrict__ dst, const float *__restrict__ 
     for (int e = threadIdx.x; e < rows * vec_per_row; e += THREADS, r += r_step) {
         if (!regular) { r = e / vec_per_row; c = (e - r * vec_per_row) << 2; }
         // columns [c, c+4) intersect the structure of row r?
-        const bool needed = prop == MOM_GENERAL || (prop == MOM_LOWER_TRI && c <= r) || (prop == MOM_UPPER_TRI && c + 3 >= r) ||
+        const bool needed = prop == MOM_GENERAL || prop == MOM_SYMMETRIC || (prop == MOM_LOWER_TRI && c <= r) || (prop == MOM_UPPER_TRI && c + 3 >= r) ||
                             (prop == MOM_DIAGONAL && c <= r && c + 3 >= r);
         float *d = dst + r * ld + c;
         const float *p = src + (size_t)r * cols + c;

@@ -47,6 +47,7 @@ struct StepImpl {
     size_t partial_off = SIZE_MAX;
     // A scaling step (Diagonal factor) whose only reader is a tensor-core step is folded into that step's
     // operand-split pass: it launches nothing and has no buffer; the reader splits d * S instead of S.
+    bool mirror = false;            // Gram product on the tensor-core kernel: lower tiles computed, upper ones mirrored
     bool folded = false;
     int fold_into = -1;             // folded step: the tensor-core step that reads it
     int fold_a = -1, fold_b = -1;   // tensor-core step: the folded scaling step behind its left / right operand

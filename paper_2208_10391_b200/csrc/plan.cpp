@@ -23,6 +23,7 @@ bool is_tri(int32_t p) { return p == MOM_LOWER_TRI || p == MOM_UPPER_TRI; }
 int32_t join_property(int32_t p, int32_t q) {
     if (p == MOM_IDENTITY) return q;
     if (q == MOM_IDENTITY) return p;
+    if (p == MOM_SYMMETRIC || q == MOM_SYMMETRIC) return (int32_t)MOM_GENERAL;   // S*S, D*S, ... are not symmetric in general
     if (p == q) return p;
     if (p == MOM_DIAGONAL) return q;
     if (q == MOM_DIAGONAL) return p;
@@ -32,10 +33,14 @@ int32_t join_property(int32_t p, int32_t q) {
 // structural non-zeros of an r x c matrix with property p (triangular, Diagonal and Identity are square)
 unsigned __int128 structural_entries(int32_t p, int64_t r, int64_t c) {
     const unsigned __int128 R = (unsigned __int128)r, C = (unsigned __int128)c;
-    if (p == MOM_GENERAL) return R * C;
+    if (p == MOM_GENERAL || p == MOM_SYMMETRIC) return R * C;
     if (p == MOM_LOWER_TRI || p == MOM_UPPER_TRI) return R * (R + 1) / 2;
     return R;
 }
+
+// Multiplications of the lower triangle (i >= j) of Y * Y^T, Y m x k: k m(m+1)/2 for a full Y, n(n+1)(n+2)/6 for a
+// triangular one.  Returns false on overflow.
+bool gram_mults(int32_t py, int64_t m, int64_t k, uint64_t *out);
 
 // Scalar multiplications a_il * b_lj of an (m x k)(k x n) product in which both factors are
 // structurally non-zero.  Triangular operands are square.  Returns false on overflow.
@@ -62,9 +67,17 @@ bool useful_mults(int32_t pa, int32_t pb, int64_t m, int64_t k, int64_t n, uint6
     return true;
 }
 
+bool gram_mults(int32_t py, int64_t m, int64_t k, uint64_t *out) {
+    const u128 M = (u128)m, K = (u128)k;
+    const u128 v = is_tri(py) ? M * (M + 1) * (M + 2) / 6 : K * (M * (M + 1) / 2);
+    if (v >= (u128)COST_LIMIT) return false;
+    *out = (uint64_t)v;
+    return true;
+}
+
 mom_status_t check_desc(const mom_matrix_desc_t &d) {
     if (d.rows < 1 || d.cols < 1) return MOM_ERR_INVALID_ARG;
-    if (d.property < MOM_GENERAL || d.property > MOM_DIAGONAL) return MOM_ERR_INVALID_ARG;
+    if (d.property < MOM_GENERAL || d.property > MOM_SYMMETRIC) return MOM_ERR_INVALID_ARG;
     if (d.dtype != MOM_F32) return MOM_ERR_DTYPE;
     if (d.property != MOM_GENERAL && d.rows != d.cols) return MOM_ERR_PROPERTY;
     return MOM_OK;
@@ -76,6 +89,12 @@ uint64_t nnz(const mom_matrix_desc_t &d) { return (uint64_t)structural_entries(d
 // Identity summand contributes its diagonal footprint and is joined as a Diagonal matrix.
 int32_t sum_property(const std::vector<int32_t> &props) {
     if (props.size() == 1) return props[0];
+    bool any_symmetric = false, only_symmetric_like = true;      // Symmetric + (Symmetric | Diagonal | Identity) is Symmetric
+    for (int32_t p : props) {
+        any_symmetric |= p == MOM_SYMMETRIC;
+        only_symmetric_like &= p == MOM_SYMMETRIC || p == MOM_DIAGONAL || p == MOM_IDENTITY;
+    }
+    if (any_symmetric) return only_symmetric_like ? (int32_t)MOM_SYMMETRIC : (int32_t)MOM_GENERAL;
     int32_t acc = MOM_DIAGONAL;
     for (int32_t p : props) acc = join_property(acc, p == MOM_IDENTITY ? (int32_t)MOM_DIAGONAL : p);
     return acc;
@@ -262,24 +281,49 @@ static mom_status_t plan_sums(const std::vector<mom_matrix_desc_t> &slots, const
                         const auto &d = chain[kept[i]];
                         node[at(i, i)] = Node{d.rows, d.cols, d.property};
                     }
+                    // Does the reduced run [i, j] read Y * Y^T factor by factor?  Factor j - q must be the transpose of
+                    // factor i + q: the same named matrix with the other flag, or with any flag when it is its own
+                    // transpose (Symmetric, Diagonal).
+                    auto reads_as_gram = [&](int i, int j) {
+                        if ((j - i + 1) % 2) return false;
+                        for (int q = 0; q < (j - i + 1) / 2; ++q) {
+                            const int a = kept[i + q], b = kept[j - q];
+                            if (fname[a - begin] < 0 || fname[a - begin] != fname[b - begin]) return false;
+                            const int32_t pa = chain[a].property;
+                            if (p->chain_t[a] == p->chain_t[b] && pa != MOM_SYMMETRIC && pa != MOM_DIAGONAL) return false;
+                        }
+                        return true;
+                    };
+                    std::vector<char> gram((size_t)r * r, 0);       // [i, j] is a Gram product (typed Symmetric whatever its tree)
                     for (int len = 2; len <= r; ++len) {
                         for (int i = 0; i + len - 1 < r; ++i) {
                             const int j = i + len - 1;
+                            // the type of [i, j] does not depend on its tree: join of the factors' types, Symmetric for a Gram run
+                            int32_t prop = node[at(i, i)].prop;
+                            for (int q = i + 1; q <= j; ++q) prop = join_property(prop, node[at(q, q)].prop);
+                            const bool is_gram = prop == MOM_GENERAL && reads_as_gram(i, j);
+                            gram[at(i, j)] = is_gram;
                             bool have = false;
                             uint64_t best = 0;
                             int best_k = -1;
                             for (int k = i; k < j; ++k) {
                                 const Node &a = node[at(i, k)], &b = node[at(k + 1, j)];
                                 uint64_t m;
-                                if (!useful_mults(a.prop, b.prop, a.rows, a.cols, b.cols, &m)) { delete p; return MOM_ERR_OVERFLOW; }
-                                const u128 cst = (u128)cost[at(i, k)] + cost[at(k + 1, j)] + m;
+                                u128 cst;
+                                if (is_gram && 2 * k == i + j - 1) {            // split in the middle: the right half is never computed
+                                    if (!gram_mults(a.prop, a.rows, a.cols, &m)) { delete p; return MOM_ERR_OVERFLOW; }
+                                    cst = (u128)cost[at(i, k)] + m;
+                                } else {
+                                    if (!useful_mults(a.prop, b.prop, a.rows, a.cols, b.cols, &m)) { delete p; return MOM_ERR_OVERFLOW; }
+                                    cst = (u128)cost[at(i, k)] + cost[at(k + 1, j)] + m;
+                                }
                                 if (cst >= (u128)COST_LIMIT) { delete p; return MOM_ERR_OVERFLOW; }
                                 if (!have || (uint64_t)cst < best) { best = (uint64_t)cst; best_k = k; have = true; }
                             }
                             cost[at(i, j)] = best;
                             split[at(i, j)] = best_k;
                             const Node &a = node[at(i, best_k)], &b = node[at(best_k + 1, j)];
-                            node[at(i, j)] = Node{a.rows, b.cols, join_property(a.prop, b.prop)};
+                            node[at(i, j)] = Node{a.rows, b.cols, is_gram ? (int32_t)MOM_SYMMETRIC : prop};
                         }
                     }
 
@@ -290,53 +334,113 @@ static mom_status_t plan_sums(const std::vector<mom_matrix_desc_t> &slots, const
                         mom_plan *p; const std::vector<Node> &node; const std::vector<int> &split; int r; int32_t &next_id;
                         const std::vector<int32_t> &kept; std::map<std::vector<int64_t>, int32_t> &seen;
                         const std::vector<int64_t> &fname; const std::vector<std::string> &flabel; int begin; int n_factors;
-                        int sum_index; std::string &s;
-                        int32_t run(int i, int j, bool emit) {
+                        int sum_index; std::string &s; const std::vector<char> &gram;
+                        // `key` receives the run of (name, transposed) factors the value multiplies (empty when a factor has
+                        // no name); the right half of a Gram product Y * Y^T is Y's run reversed with every flag flipped
+                        int32_t run(int i, int j, bool emit, std::vector<int64_t> &key) {
+                            key.clear();
                             if (i == j) {
                                 s += flabel[kept[i] - begin];
                                 if (p->chain_t[kept[i]]) s += "^T";
+                                if (fname[kept[i] - begin] >= 0) key.push_back(fname[kept[i] - begin] * 2 + (p->chain_t[kept[i]] ? 1 : 0));
                                 return kept[i];
                             }
                             const bool root = i == 0 && j == r - 1;
-                            std::vector<int64_t> key;
-                            int32_t shared = -1;
+                            const int k = split[(size_t)i * r + j];
+                            const bool is_gram = gram[(size_t)i * r + j] && 2 * k == i + j - 1;
                             bool named = true;
                             for (int q = i; q <= j; ++q) named &= fname[kept[q] - begin] >= 0;
-                            if (emit && named && !root) {
-                                for (int q = i; q <= j; ++q) key.push_back(fname[kept[q] - begin] * 2 + (p->chain_t[kept[q]] ? 1 : 0));
-                                auto it = seen.find(key);
-                                if (it != seen.end()) { shared = it->second; p->reused += j - i; }
-                            }
-                            const bool emit_here = emit && shared < 0;
-                            const int k = split[(size_t)i * r + j];
+                            // text first (both halves as written), with nothing emitted; then the products
+                            const size_t text_at = s.size();
+                            std::vector<int64_t> kl, kr;
                             s += "(";
-                            const int32_t l = run(i, k, emit_here);
+                            run(i, k, false, kl);
                             s += "*";
-                            const int32_t rr = run(k + 1, j, emit_here);
+                            if (is_gram) right_nested(k + 1, j);  // never multiplied: every tree costs the same, the first in the tie order is written
+                            else run(k + 1, j, false, kr);
                             s += ")";
-                            if (!emit) return -1;
-                            if (shared >= 0) return shared;
+                            if (!emit) {
+                                if (named) {
+                                    key = kl;
+                                    if (is_gram) for (size_t q = kl.size(); q-- > 0;) key.push_back(kl[q] ^ 1);
+                                    else key.insert(key.end(), kr.begin(), kr.end());
+                                }
+                                return -1;
+                            }
+                            const std::string text = s.substr(text_at);
+                            s.resize(text_at);
+                            std::string scratch;
+                            std::swap(s, scratch);                // emission below must not write the text twice
+                            int32_t l, rr;
+                            {
+                                std::vector<int64_t> k2;
+                                if (named) {
+                                    key = kl;
+                                    if (is_gram) for (size_t q = kl.size(); q-- > 0;) key.push_back(kl[q] ^ 1);
+                                    else key.insert(key.end(), kr.begin(), kr.end());
+                                }
+                                int32_t shared = -1;
+                                if (named && !root) {
+                                    auto it = seen.find(key);
+                                    if (it != seen.end()) { shared = it->second; p->reused += count_products(i, j); }
+                                }
+                                if (shared >= 0) {
+                                    std::swap(s, scratch);
+                                    s += text;
+                                    return shared;
+                                }
+                                l = run(i, k, true, k2);
+                                rr = is_gram ? l : run(k + 1, j, true, k2);
+                            }
+                            std::swap(s, scratch);
+                            s += text;
                             const Node &a = node[(size_t)i * r + k], &b = node[(size_t)(k + 1) * r + j], &o = node[(size_t)i * r + j];
                             mom::StepImpl st;
                             std::memset(&st.pub, 0, sizeof(st.pub));
                             st.pub.lhs = l; st.pub.rhs = rr; st.pub.out = next_id++;
-                            st.pub.lhs_property = a.prop; st.pub.rhs_property = b.prop; st.pub.out_property = o.prop;
+                            st.pub.lhs_property = a.prop; st.pub.out_property = o.prop;
                             st.pub.lhs_transposed = l < n_factors && p->chain_t[l];
-                            st.pub.rhs_transposed = rr < n_factors && p->chain_t[rr];
-                            st.pub.m = a.rows; st.pub.k = a.cols; st.pub.n = b.cols;
-                            useful_mults(a.prop, b.prop, a.rows, a.cols, b.cols, &st.pub.useful_mults);
-                            const bool ta = is_tri(a.prop), tb = is_tri(b.prop);
-                            st.pub.kind = a.prop == MOM_DIAGONAL || b.prop == MOM_DIAGONAL ? MOM_KIND_SCALE
-                                          : !ta && !tb ? MOM_KIND_GG : ta && !tb ? MOM_KIND_TG : !ta && tb ? MOM_KIND_GT
-                                          : a.prop == b.prop ? MOM_KIND_TT : MOM_KIND_TTMIX;
+                            st.pub.m = a.rows; st.pub.k = a.cols;
+                            if (is_gram) {
+                                // Y * Y^T: the right operand is the left one read transposed
+                                st.pub.rhs_property = a.prop == MOM_LOWER_TRI ? (int32_t)MOM_UPPER_TRI
+                                                      : a.prop == MOM_UPPER_TRI ? (int32_t)MOM_LOWER_TRI : a.prop;
+                                st.pub.rhs_transposed = l < n_factors ? !p->chain_t[l] : 1;
+                                st.pub.n = a.rows;
+                                gram_mults(a.prop, a.rows, a.cols, &st.pub.useful_mults);
+                                st.pub.kind = MOM_KIND_GRAM;
+                            } else {
+                                st.pub.rhs_property = b.prop;
+                                st.pub.rhs_transposed = rr < n_factors && p->chain_t[rr];
+                                st.pub.n = b.cols;
+                                useful_mults(a.prop, b.prop, a.rows, a.cols, b.cols, &st.pub.useful_mults);
+                                const bool ta = is_tri(a.prop), tb = is_tri(b.prop);
+                                st.pub.kind = a.prop == MOM_DIAGONAL || b.prop == MOM_DIAGONAL ? MOM_KIND_SCALE
+                                              : !ta && !tb ? MOM_KIND_GG : ta && !tb ? MOM_KIND_TG : !ta && tb ? MOM_KIND_GT
+                                              : a.prop == b.prop ? MOM_KIND_TT : MOM_KIND_TTMIX;
+                            }
                             st.is_last = root;
                             if (root) st.sum = sum_index;
                             p->steps.push_back(st);
-                            if (named && !root) seen.emplace(std::move(key), st.pub.out);
+                            if (named && !root) seen.emplace(key, st.pub.out);
                             return st.pub.out;
                         }
-                    } emit{p, node, split, r, next_id, kept, seen, fname, flabel, begin, n_chain, (int)si, text};
-                    emit.run(0, r - 1, true);
+                        void right_nested(int i, int j) {
+                            if (i < j) s += "(";
+                            s += flabel[kept[i] - begin];
+                            if (p->chain_t[kept[i]]) s += "^T";
+                            if (i < j) { s += "*"; right_nested(i + 1, j); s += ")"; }
+                        }
+                        // binary products in the chosen tree of [i, j] (a Gram node's right half has none)
+                        int count_products(int i, int j) const {
+                            if (i == j) return 0;
+                            const int k = split[(size_t)i * r + j];
+                            const bool is_gram = gram[(size_t)i * r + j] && 2 * k == i + j - 1;
+                            return 1 + count_products(i, k) + (is_gram ? 0 : count_products(k + 1, j));
+                        }
+                    } emit{p, node, split, r, next_id, kept, seen, fname, flabel, begin, n_chain, (int)si, text, gram};
+                    std::vector<int64_t> root_key;
+                    emit.run(0, r - 1, true, root_key);
                     const Node &root = node[at(0, r - 1)];
                     value_desc = mom_matrix_desc_t{root.rows, root.cols, root.prop, MOM_F32};
                     if (r == 1) info.summands.push_back(mom::Summand{mom::SUM_FACTOR, kept[0]});
@@ -431,8 +535,13 @@ static mom_status_t plan_sums(const std::vector<mom_matrix_desc_t> &slots, const
                 (c.pub.lhs == st.pub.out ? as_lhs : as_rhs)++;
                 all_tc &= c.pub.uses_tensor_cores == 1;
             }
+            // (a Gram product keeps its f32 output: its epilogue mirrors the lower triangle into the upper one)
             const bool fused_planes = last_consumer >= 0 && all_tc && (as_lhs == 0 || as_rhs == 0) &&
-                                      st.pub.uses_tensor_cores == 1 && st.split_k == 1;
+                                      st.pub.uses_tensor_cores == 1 && st.split_k == 1 && st.pub.kind != MOM_KIND_GRAM;
+            // mirrored Gram product: only the tiles on and below the diagonal are computed; needs a plain f32 result
+            // without Add terms (a root that is its sum's only summand, or an intermediate)
+            st.mirror = st.pub.kind == MOM_KIND_GRAM && st.pub.uses_tensor_cores == 1 && st.split_k == 1 &&
+                        (!st.is_last || (!st.accumulate && p->sums[st.sum].summands.size() == 1));
             if (fused_planes) {
                 st.planes_out = as_lhs ? 1 : 2;
             } else if (!st.is_last && !st.folded) {
@@ -470,6 +579,12 @@ static mom_status_t plan_sums(const std::vector<mom_matrix_desc_t> &slots, const
             if (st.pub.uses_tensor_cores != 1) continue;
             const int64_t m = st.pub.m, n = st.pub.n, k = st.pub.k;
             for (int side = 0; side < 2; ++side) {
+                if (side == 1 && st.pub.kind == MOM_KIND_GRAM) {
+                    // Y * Y^T: the right operand's planes (n x k, K-major) are the left operand's
+                    copies.push_back(Copy{s, 1, -1});
+                    st.b_planes_ready = true;
+                    continue;
+                }
                 const int32_t v = side == 0 ? st.pub.lhs : st.pub.rhs;
                 const size_t bytes = mom::align_up((size_t)(side == 0 ? m * k : k * n) * sizeof(float), mom::WS_ALIGN);
                 size_t *hi = side == 0 ? &st.a_hi_off : &st.b_hi_off, *lo = side == 0 ? &st.a_lo_off : &st.b_lo_off;
@@ -502,10 +617,17 @@ static mom_status_t plan_sums(const std::vector<mom_matrix_desc_t> &slots, const
         }
         p->workspace_per_instance = pack(items);
         for (const Copy &c : copies) {
+            if (c.owner < 0) continue;
             mom::StepImpl &st = p->steps[c.step];
             const mom::StepImpl &o = p->steps[c.owner];
             if (c.side == 0) { st.a_hi_off = o.a_hi_off; st.a_lo_off = o.a_lo_off; }
             else { st.b_hi_off = o.b_hi_off; st.b_lo_off = o.b_lo_off; }
+        }
+        for (const Copy &c : copies) {                  // Gram products: right planes = left planes (set above by now)
+            if (c.owner >= 0) continue;
+            mom::StepImpl &st = p->steps[c.step];
+            st.b_hi_off = st.a_hi_off;
+            st.b_lo_off = st.a_lo_off;
         }
         for (int s = 0; s < ns; ++s) {                  // a producer's plane targets are its consumers' operand planes
             mom::StepImpl &st = p->steps[s];
@@ -519,13 +641,13 @@ static mom_status_t plan_sums(const std::vector<mom_matrix_desc_t> &slots, const
 
         // Small equations run as one fused kernel with every operand and intermediate in shared memory.
         {
-            bool any_tc = false;
-            for (const auto &st : p->steps) any_tc |= st.pub.uses_tensor_cores == 1;
+            bool any_tc = false, any_gram = false;      // (a Gram product reads one value on both sides: the layout below gives a value one side)
+            for (const auto &st : p->steps) { any_tc |= st.pub.uses_tensor_cores == 1; any_gram |= st.pub.kind == MOM_KIND_GRAM; }
             const int values = n_chain + ns;
             p->fused_value_off.assign(values, -1);
             size_t floats = 0;
             bool ok = single_chain && ns >= 1 && ns <= mom::FUSED_MAX_STEPS && (int)p->kept.size() <= mom::FUSED_MAX_OPERANDS &&
-                      n_add <= mom::MAX_FUSED_ADD && !any_tc && variant != MOM_VARIANT_3XTF32_WARP;
+                      n_add <= mom::MAX_FUSED_ADD && !any_tc && variant != MOM_VARIANT_3XTF32_WARP && !any_gram;
             // every value feeds exactly one product: remember on which side
             std::vector<char> is_rhs(values, 0);
             for (const auto &st : p->steps) is_rhs[st.pub.rhs] = 1;
@@ -787,7 +909,7 @@ const char *mom_status_string(mom_status_t s) {
     switch (s) {
         case MOM_OK: return "ok";
         case MOM_ERR_INVALID_ARG: return "invalid argument";
-        case MOM_ERR_PROPERTY: return "triangular, Diagonal and Identity matrices must be square";
+        case MOM_ERR_PROPERTY: return "triangular, Diagonal, Symmetric and Identity matrices must be square";
         case MOM_ERR_DTYPE: return "unsupported element type";
         case MOM_ERR_SHAPE_MISMATCH: return "shape mismatch";
         case MOM_ERR_OVERFLOW: return "multiplication count overflows 63 bits";

@@ -234,7 +234,7 @@ scale_kernel(ProductArgs a) {
             dr[i] = 0.f;
             if (r >= m) continue;
             // the four entries lie inside S's structure?  (outside, the stored zeros need not be read)
-            const bool any = ps == MOM_GENERAL || (ps == MOM_LOWER_TRI && c <= r) || (ps == MOM_UPPER_TRI && c + 3 >= r) ||
+            const bool any = ps == MOM_GENERAL || ps == MOM_SYMMETRIC || (ps == MOM_LOWER_TRI && c <= r) || (ps == MOM_UPPER_TRI && c + 3 >= r) ||
                              (ps == MOM_DIAGONAL && c <= r && c + 3 >= r);
             if (any) {
                 if (vec) {

@@ -94,6 +94,8 @@ struct TcParams {
     int pout;
     int out_mode;            // 0: f32 result through map_c; 1: hi/lo planes (map_c, map_c2); 2: transposed hi/lo planes
     int slice_rows;          // split-K: rows between the partial-sum slabs of consecutive k-slices (0: no split)
+    int mirror;              // Gram product Y * Y^T (CTA-pair kernel, out_mode 0, no Add terms): the table holds the tiles on and
+                             // below the diagonal; a tile below it is also written transposed to its mirror position
     AddTerms add;
     int32_t *status;
 };
@@ -119,7 +121,7 @@ __device__ __forceinline__ uint32_t round_tf32_bits(float a) { return (__float_a
 
 __device__ __forceinline__ void epilogue_chunk(const TcParams &prm, const CUtensorMap *map_c, const CUtensorMap *map_c2,
                                                float (&v)[32], int r, int row0, int col0, int lane, uint32_t stage_buf,
-                                               uint32_t &store_it) {
+                                               uint32_t &store_it, bool mirror_this = false) {
     const bool row_ok = r < prm.m;
     for (int a = 0; a < prm.add.count; ++a) {                   // Add terms, left to right
         const float *p = prm.add.ptr[a];
@@ -149,13 +151,14 @@ __device__ __forceinline__ void epilogue_chunk(const TcParams &prm, const CUtens
 #pragma unroll
         for (int j = 0; j < 32; ++j) v[j] = in_structure(prm.pout, r, col0 + j) ? v[j] : 0.0f;
     }
-    const int passes = prm.out_mode == 0 ? 1 : 2;                // f32, or hi then lo
+    const int passes = prm.out_mode == 0 ? (mirror_this ? 2 : 1) : 2;   // f32 (and its mirror image), or hi then lo
 #pragma unroll 1
     for (int pass = 0; pass < passes; ++pass) {
         const uint32_t buf = stage_buf + (store_it & 1) * EPI_BOX_BYTES;
         if (lane == 0) ptx::tma_store_wait_read<1>();            // the store that last read this buffer is done
         __syncwarp();
-        if (prm.out_mode != 2) {
+        const bool transposed_box = prm.out_mode == 2 || (prm.out_mode == 0 && pass == 1);
+        if (!transposed_box) {
             // 32 rows of 128 bytes: 16-byte chunk j of row i stored at chunk j ^ (i & 7)
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
@@ -175,7 +178,7 @@ __device__ __forceinline__ void epilogue_chunk(const TcParams &prm, const CUtens
             for (int j = 0; j < 32; ++j) {
                 const float x = v[j];
                 const float hi = __uint_as_float(round_tf32_bits(x));
-                const float w = pass == 0 ? hi : __uint_as_float(round_tf32_bits(x - hi));
+                const float w = prm.out_mode == 0 ? x : pass == 0 ? hi : __uint_as_float(round_tf32_bits(x - hi));
                 const uint32_t dst = buf + j * 128 + ((((uint32_t)lane >> 2) ^ (j & 7)) << 4) + ((lane & 3) << 2);
                 asm volatile("st.shared.f32 [%0], %1;" ::"r"(dst), "f"(w) : "memory");
             }
@@ -183,8 +186,8 @@ __device__ __forceinline__ void epilogue_chunk(const TcParams &prm, const CUtens
         ptx::fence_proxy_async_smem();
         __syncwarp();
         if (lane == 0) {
-            const CUtensorMap *map = pass == 0 ? map_c : map_c2;
-            if (prm.out_mode != 2) ptx::tma_store_2d(map, col0, row0, buf);
+            const CUtensorMap *map = pass == 0 || prm.out_mode == 0 ? map_c : map_c2;
+            if (!transposed_box) ptx::tma_store_2d(map, col0, row0, buf);
             else ptx::tma_store_2d(map, row0, col0, buf);
             ptx::tma_store_commit();
         }
@@ -527,7 +530,9 @@ product_tc_pair_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __gri
 #pragma unroll
                     for (int j = 0; j < 32; ++j) v[j] = 0.0f;
                 }
-                if (rows_left > 0) epilogue_chunk(prm, &map_c, &map_c2, v, r, row0, col0, lane, stage_buf, store_it);
+                if (rows_left > 0)
+                    epilogue_chunk(prm, &map_c, &map_c2, v, r, row0, col0, lane, stage_buf, store_it,
+                                   prm.mirror != 0 && tile.y < (tile.x & TILE_ROW_MASK));
             }
             if (!zero_tile) {
                 ptx::tc_fence_before_sync();
@@ -699,8 +704,11 @@ mom_status_t tc_prepare(const mom_plan &p, TcPlanState &s) {
         const int split = p.steps[i].split_k;
         if (split > 1) s.steps[i].pair = false;
         const int tile_rows = s.steps[i].pair ? P_BM : BM;
+        // a mirrored Gram product computes the tiles on and below the diagonal only (square 256 x 256 pair tiles)
+        s.steps[i].mirror = p.steps[i].mirror && s.steps[i].pair;
         for (int r0 = 0; r0 < m; r0 += tile_rows)
             for (int c0 = 0; c0 < n; c0 += BN) {
+                if (s.steps[i].mirror && c0 > r0) continue;
                 int klo, khi;
                 tile_k_range(st.lhs_property, st.rhs_property, r0, std::min(r0 + tile_rows, m), c0, std::min(c0 + BN, n), k, &klo, &khi);
                 if (klo >= khi) { klo = 0; khi = 0; }
@@ -883,6 +891,8 @@ mom_status_t tc_launch_step(const mom_plan &p, TcPlanState &s, int step, const P
     prm.pout = st.split_k > 1 ? (int)MOM_GENERAL : a.pout;      // split-K: mask and Add terms are applied by the reduction
     prm.out_mode = st.planes_out;
     prm.slice_rows = slice_rows;
+    if (s.steps[step].mirror && (a.add.count != 0 || st.planes_out != 0)) return MOM_ERR_INVALID_ARG;   // the planner never asks for this
+    prm.mirror = s.steps[step].mirror ? 1 : 0;
     prm.add = a.add;
     if (st.split_k > 1) prm.add.count = 0;
     prm.status = status;
@@ -1123,6 +1133,7 @@ extern "C" mom_status_t mom_product_3xtf32_noalloc(int64_t m64, int64_t n64, int
     prm.pout = pa == MOM_GENERAL || pb == MOM_GENERAL || pa != pb ? (int)MOM_GENERAL : (int)pa;
     prm.out_mode = 0;
     prm.slice_rows = 0;
+    prm.mirror = 0;
     prm.add.count = 0;
     prm.status = status;
     product_tc_kernel<<<std::min(prm.num_tiles, g_sm_count), THREADS, SMEM_BYTES, stream>>>(ma_hi, ma_lo, mb_hi, mb_lo, mc, mc, prm);

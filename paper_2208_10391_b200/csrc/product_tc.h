@@ -12,6 +12,7 @@ struct TcStepState {
     int4 *tiles = nullptr;      // device: work-sorted tile table {row0, col0, k_begin, k_end}
     int num_tiles = 0;
     bool pair = false;          // tiles are 256 rows high and run on CTA pairs (cta_group::2)
+    bool mirror = false;        // Gram product: tiles on and below the diagonal only, the others written as mirror images
     int units = 1;              // CTAs (or CTA pairs) the table was laid out for: unit u owns entries u, u + units, ...
 };
 

@@ -221,6 +221,31 @@ def test_random_sums_of_chains_match_the_oracle():
         assert_same_sum_plan(eq.descs(), eq.transposed, eq.names)
 
 
+def test_gram_products_match_the_oracle():
+    grams = shared = 0
+    for seed in range(400):
+        eq = wl.random_gram_sum(seed)
+        got, want = assert_same_sum_plan(eq.descs(), eq.transposed, eq.names)
+        grams += any(s.gram for s in want.steps)
+        shared += want.reused > 0
+        for g, w in zip(got.steps(), want.steps):
+            assert (g.kind == mom.KIND_GRAM) == w.gram
+            if w.gram:
+                assert g.lhs == g.rhs and g.rhs_transposed != g.lhs_transposed
+        assert_same_sum_plan(eq.descs(), eq.transposed, None)          # without names there is no Gram product
+    assert grams >= 250 and shared >= 40
+    A, S = (10, 4, mom.GENERAL), (10, 10, mom.SYMMETRIC)
+    got, want = assert_same_sum_plan([[A, A], [S]], [[False, True], [False]], [[0, 0], [1]])
+    assert got.parenthesization() == "(0*1^T)+2" and got.flops() == (2 * 220, 100) and got.result_desc().property == mom.SYMMETRIC
+    got, _ = assert_same_sum_plan([[A, A]], [[False, True]], None)
+    assert got.flops()[0] == 2 * 400 and got.result_desc().property == mom.GENERAL
+    eq = wl.config_gram()
+    got, want = assert_same_sum_plan(eq.descs(), eq.transposed, eq.names)
+    n, k = 4096, 2048
+    assert got.parenthesization() == "((0*1)*(2^T*3^T))+4" and want.mults == n * k * k + k * n * (n + 1) // 2
+    assert [s.kind for s in got.steps()] == [mom.KIND_GG, mom.KIND_GRAM] and got.result_desc().property == mom.SYMMETRIC
+
+
 def test_sum_plan_shares_a_product_between_chains():
     G = mom.GENERAL
     a, b, c = (8, 50, G), (50, 8, G), (8, 100, G)

@@ -336,6 +336,57 @@ def random_sum_equation(seed: int, max_chains: int = 4, max_len: int = 5, max_di
     return SumEquation(f"random_sum_{seed}", seed, tuple(chains), tuple(flags), tuple(names))
 
 
+def random_gram_sum(seed: int, max_dim: int = 40, dim_multiple: int = 1) -> SumEquation:
+    """Random sum of chains in which Gram products occur: every chain is (prefix) * Y-factors * mirrored
+    Y-factors * (suffix), where the mirrored half names the same matrices with the transposition flags
+    flipped (or, for Symmetric and Diagonal factors, sometimes kept); later chains often reuse the first
+    chain's Y, so that Gram products and their halves are shared between chains."""
+    rng = np.random.Generator(np.random.Philox(key=[int(seed), 0x6AA3]))
+    dim = lambda: int(rng.integers(1, max_dim // dim_multiple + 1)) * dim_multiple
+    next_name = [0]
+
+    def factor(r, c):
+        """(stored operand, transposed flag, name) of a new matrix used as r x c"""
+        kind = int(rng.integers(0, 8))
+        t = bool(rng.integers(0, 2))
+        if r == c and kind < 4:
+            o = Operand(r, r, (LOWER_TRI, UPPER_TRI, SYMMETRIC, DIAGONAL)[kind])
+        else:
+            o = Operand(c, r, GENERAL, "normal") if t else Operand(r, c, GENERAL, "normal")
+        next_name[0] += 1
+        return o, t, next_name[0]
+
+    n = dim()                                              # every chain's value is n x n
+    halves = []
+    chains, flags, names = [], [], []
+    for c in range(int(rng.integers(1, 4))):
+        if halves and rng.random() < 0.6:
+            half = halves[int(rng.integers(0, len(halves)))]
+        else:
+            half, cur = [], n
+            for q in range(int(rng.integers(1, 4))):
+                nxt = cur if rng.random() < 0.4 else dim()
+                half.append(factor(cur, nxt))
+                cur = nxt
+            halves.append(half)
+        mirrored = [(o, (t if o.prop in (SYMMETRIC, DIAGONAL) and rng.random() < 0.5 else not t), nm) for o, t, nm in reversed(half)]
+        body = list(half) + mirrored
+        if rng.random() < 0.3:                             # a square factor in front or behind breaks the symmetry of the chain
+            extra = factor(n, n)
+            body = [extra] + body if rng.random() < 0.5 else body + [extra]
+        chains.append(tuple(o for o, _, _ in body)); flags.append(tuple(t for _, t, _ in body)); names.append(tuple(nm for _, _, nm in body))
+    return SumEquation(f"random_gram_{seed}", seed, tuple(chains), tuple(flags), tuple(names))
+
+
+def config_gram(n: int = 4096, k: int = 2048, seed: int = 11) -> SumEquation:
+    """X = A * B * B^T * A^T + S: A n x k, B k x k general, S Symmetric.  The chain reads Y * Y^T with Y = A * B:
+    one general product, then only the lower triangle of Y * Y^T (mirrored), plus a Symmetric summand."""
+    a = Operand(n, k, GENERAL, "normal", 1.0 / np.sqrt(k))
+    b = Operand(k, k, GENERAL, "normal", 1.0 / np.sqrt(k))
+    return SumEquation(f"ABBtAt_plus_S_{n}", seed, ((a, b, b, a), (Operand(n, n, SYMMETRIC, "normal"),)),
+                       ((False, False, True, True), (False,)), ((0, 1, 1, 0), (2,)))
+
+
 def config_sum_shared(n: int = 4096, seed: int = 7) -> SumEquation:
     """X = C*A*B + D*A*B, all general n x n: every tree ties, the right-nested one is taken, and A*B is
     below the root in both chains, so it is multiplied once (3 products instead of 4)."""
