@@ -538,10 +538,11 @@ static mom_status_t plan_sums(const std::vector<mom_matrix_desc_t> &slots, const
             // (a Gram product keeps its f32 output: its epilogue mirrors the lower triangle into the upper one)
             const bool fused_planes = last_consumer >= 0 && all_tc && (as_lhs == 0 || as_rhs == 0) &&
                                       st.pub.uses_tensor_cores == 1 && st.split_k == 1 && st.pub.kind != MOM_KIND_GRAM;
-            // mirrored Gram product: only the tiles on and below the diagonal are computed; needs a plain f32 result
-            // without Add terms (a root that is its sum's only summand, or an intermediate)
+            // mirrored Gram product: only the tiles on and below the diagonal are computed, the others are written as
+            // mirror images; needs a plain f32 result, and as a root a Symmetric sum (then every fused summand is
+            // Symmetric, Diagonal or Identity, so the mirror image of entry (i, j) is the value of entry (j, i))
             st.mirror = st.pub.kind == MOM_KIND_GRAM && st.pub.uses_tensor_cores == 1 && st.split_k == 1 &&
-                        (!st.is_last || (!st.accumulate && p->sums[st.sum].summands.size() == 1));
+                        (!st.is_last || (!st.accumulate && p->sums[st.sum].desc.property == MOM_SYMMETRIC));
             if (fused_planes) {
                 st.planes_out = as_lhs ? 1 : 2;
             } else if (!st.is_last && !st.folded) {

@@ -94,7 +94,7 @@ struct TcParams {
     int pout;
     int out_mode;            // 0: f32 result through map_c; 1: hi/lo planes (map_c, map_c2); 2: transposed hi/lo planes
     int slice_rows;          // split-K: rows between the partial-sum slabs of consecutive k-slices (0: no split)
-    int mirror;              // Gram product Y * Y^T (CTA-pair kernel, out_mode 0, no Add terms): the table holds the tiles on and
+    int mirror;              // Gram product Y * Y^T (CTA-pair kernel, out_mode 0, Symmetric Add terms only): the table holds the tiles on and
                              // below the diagonal; a tile below it is also written transposed to its mirror position
     AddTerms add;
     int32_t *status;
@@ -891,7 +891,7 @@ mom_status_t tc_launch_step(const mom_plan &p, TcPlanState &s, int step, const P
     prm.pout = st.split_k > 1 ? (int)MOM_GENERAL : a.pout;      // split-K: mask and Add terms are applied by the reduction
     prm.out_mode = st.planes_out;
     prm.slice_rows = slice_rows;
-    if (s.steps[step].mirror && (a.add.count != 0 || st.planes_out != 0)) return MOM_ERR_INVALID_ARG;   // the planner never asks for this
+    if (s.steps[step].mirror && st.planes_out != 0) return MOM_ERR_INVALID_ARG;   // the planner never asks for this
     prm.mirror = s.steps[step].mirror ? 1 : 0;
     prm.add = a.add;
     if (st.split_k > 1) prm.add.count = 0;
