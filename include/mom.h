@@ -75,7 +75,7 @@ typedef enum { MOM_F32 = 0 } mom_dtype_t;
 /* Arithmetic used by the product kernels.
  *   MOM_VARIANT_3XTF32: tensor-core MMA (kind::tf32 / .tf32) on operands split as a = hi + lo,
  *       accumulating lo*hi + hi*lo + hi*hi in f32 (f32-level accuracy).  Large products
- *       (m*n*k >= 3 * 2^26) whose shapes TMA can address (leading dimensions that are multiples of 4
+ *       (m*n*k >= 6 * 2^26) whose shapes TMA can address (leading dimensions that are multiples of 4
  *       elements) run on the tcgen05 kernel (operand planes, TMA, tensor memory).  Smaller products and
  *       the other shapes run on the warp-level kernel (mma.sync on the operands as stored, one launch per
  *       product): below that size the tcgen05 path's extra passes cost more than they save.

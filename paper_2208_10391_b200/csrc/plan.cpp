@@ -490,7 +490,7 @@ static mom_status_t plan_sums(const std::vector<mom_matrix_desc_t> &slots, const
             const bool addressable = (k % 4 == 0) && (n % 4 == 0);
             // below this size the tcgen05 path's extra launches (operand splits, split-K reduction) cost more
             // than its faster mainloop saves; the warp-level kernel is one launch
-            const bool large = (double)m * (double)n * (double)k >= 3.0 * (double)(1 << 26);
+            const bool large = (double)m * (double)n * (double)k >= 6.0 * (double)(1 << 26);
             if (st.pub.kind == MOM_KIND_SCALE) st.pub.uses_tensor_cores = 0;       // a Diagonal operand: one scaling pass, bound by HBM
             else if (variant == MOM_VARIANT_3XTF32) st.pub.uses_tensor_cores = addressable && large ? 1 : 2;
             else if (variant == MOM_VARIANT_3XTF32_FORCE) st.pub.uses_tensor_cores = addressable ? 1 : 0;
