@@ -179,10 +179,77 @@ __device__ void product_mma_whole(const FusedPlan &fp, const FusedStep &st, cons
                 mma_tf32(small_acc[j], a_hi, b_lo);
             }
         }
+        // Whole tiles need no bounds checks, and all addresses derive from one base: entries (ra, c), (ra, c + 1),
+        // (ra + 8, c), (ra + 8, c + 1) with c = c0 + 8 j + 2 t.  Row lengths are multiples of 8 here, so pairs are
+        // 8-byte aligned.
+        const int ra = r0 + g, c = c0 + 2 * t;
+        const bool masked = st.pout != MOM_GENERAL && st.pout != MOM_SYMMETRIC;
+        if (st.out_off >= 0) {
+            float *C = at(in, st.out_off) + ra * st.ldc + c;
 #pragma unroll
-        for (int j = 0; j < NTW; ++j) {
-            store_pair(fp, st, in, r0 + g, c0 + 8 * j + 2 * t, main_acc[j][0] + small_acc[j][0], main_acc[j][1] + small_acc[j][1]);
-            store_pair(fp, st, in, r0 + g + 8, c0 + 8 * j + 2 * t, main_acc[j][2] + small_acc[j][2], main_acc[j][3] + small_acc[j][3]);
+            for (int j = 0; j < NTW; ++j) {
+                float2 lo2 = make_float2(main_acc[j][0] + small_acc[j][0], main_acc[j][1] + small_acc[j][1]);
+                float2 hi2 = make_float2(main_acc[j][2] + small_acc[j][2], main_acc[j][3] + small_acc[j][3]);
+                if (masked) {
+                    const int cc = c + 8 * j;
+                    lo2.x = in_structure(st.pout, ra, cc) ? lo2.x : 0.f;       lo2.y = in_structure(st.pout, ra, cc + 1) ? lo2.y : 0.f;
+                    hi2.x = in_structure(st.pout, ra + 8, cc) ? hi2.x : 0.f;   hi2.y = in_structure(st.pout, ra + 8, cc + 1) ? hi2.y : 0.f;
+                }
+                *reinterpret_cast<float2 *>(C + 8 * j) = lo2;
+                *reinterpret_cast<float2 *>(C + 8 * st.ldc + 8 * j) = hi2;
+            }
+        } else if (fp.add.transposed == 0 && (reinterpret_cast<uintptr_t>(fp.out) & 7) == 0 && (fp.out_stride & 1) == 0) {
+            const long long at0 = (long long)ra * st.n + c, at8 = at0 + 8LL * st.n;
+            float2 lo2[NTW], hi2[NTW];
+#pragma unroll
+            for (int j = 0; j < NTW; ++j) {
+                lo2[j] = make_float2(main_acc[j][0] + small_acc[j][0], main_acc[j][1] + small_acc[j][1]);
+                hi2[j] = make_float2(main_acc[j][2] + small_acc[j][2], main_acc[j][3] + small_acc[j][3]);
+            }
+#pragma unroll 1
+            for (int term = 0; term < fp.add.count; ++term) {                  // Add terms, left to right
+                const float *p = fp.add.ptr[term];
+                if (!p) {                                                       // Identity
+#pragma unroll
+                    for (int j = 0; j < NTW; ++j) {
+                        const int cc = c + 8 * j;
+                        lo2[j].x += ra == cc ? 1.f : 0.f;       lo2[j].y += ra == cc + 1 ? 1.f : 0.f;
+                        hi2[j].x += ra + 8 == cc ? 1.f : 0.f;   hi2[j].y += ra + 8 == cc + 1 ? 1.f : 0.f;
+                    }
+                    continue;
+                }
+                p += in.inst * fp.add.stride[term];
+                const bool vec = (reinterpret_cast<uintptr_t>(p) & 7) == 0;
+#pragma unroll
+                for (int j = 0; j < NTW; ++j) {
+                    float2 x, y;
+                    if (vec) {
+                        x = __ldg(reinterpret_cast<const float2 *>(p + at0 + 8 * j));
+                        y = __ldg(reinterpret_cast<const float2 *>(p + at8 + 8 * j));
+                    } else {
+                        x = make_float2(__ldg(p + at0 + 8 * j), __ldg(p + at0 + 8 * j + 1));
+                        y = make_float2(__ldg(p + at8 + 8 * j), __ldg(p + at8 + 8 * j + 1));
+                    }
+                    lo2[j].x += x.x; lo2[j].y += x.y; hi2[j].x += y.x; hi2[j].y += y.y;
+                }
+            }
+            float *X = fp.out + in.inst * fp.out_stride;
+#pragma unroll
+            for (int j = 0; j < NTW; ++j) {
+                if (masked) {
+                    const int cc = c + 8 * j;
+                    lo2[j].x = in_structure(st.pout, ra, cc) ? lo2[j].x : 0.f;       lo2[j].y = in_structure(st.pout, ra, cc + 1) ? lo2[j].y : 0.f;
+                    hi2[j].x = in_structure(st.pout, ra + 8, cc) ? hi2[j].x : 0.f;   hi2[j].y = in_structure(st.pout, ra + 8, cc + 1) ? hi2[j].y : 0.f;
+                }
+                *reinterpret_cast<float2 *>(X + at0 + 8 * j) = lo2[j];
+                *reinterpret_cast<float2 *>(X + at8 + 8 * j) = hi2[j];
+            }
+        } else {
+#pragma unroll
+            for (int j = 0; j < NTW; ++j) {
+                store_pair(fp, st, in, r0 + g, c0 + 8 * j + 2 * t, main_acc[j][0] + small_acc[j][0], main_acc[j][1] + small_acc[j][1]);
+                store_pair(fp, st, in, r0 + g + 8, c0 + 8 * j + 2 * t, main_acc[j][2] + small_acc[j][2], main_acc[j][3] + small_acc[j][3]);
+            }
         }
     }
 }
@@ -190,9 +257,9 @@ __device__ void product_mma_whole(const FusedPlan &fp, const FusedStep &st, cons
 // One product on tensor cores: 16 x 16 output tiles dealt round-robin to the warps.
 __device__ void product_mma(const FusedPlan &fp, const FusedStep &st, const Instance &in) {
     if (((st.m | st.n) & 15) == 0 && (st.k & 7) == 0) {
-        // with few 16 x 16 tiles, 16 x 8 tiles give every warp of the CTA something to do
-        if ((st.m >> 4) * (st.n >> 4) < WARPS) product_mma_whole<1>(fp, st, in);
-        else product_mma_whole<2>(fp, st, in);
+        // 16 x 16 tiles per warp also when that leaves warps idle: the kernel is bound by instruction issue, and a
+        // 16 x 16 tile shares the left fragments (and their splits) between its two column halves
+        product_mma_whole<2>(fp, st, in);
         return;
     }
     const float *__restrict__ A = at(in, st.a_off);
