@@ -732,7 +732,8 @@ mom_status_t tc_prepare(const mom_plan &p, TcPlanState &s) {
         // of A and B panels, wherever the wave starts.  Structurally zero tiles come last.
         // Equal tiles are taken round-robin in that order.  Unequal tiles are dealt out by list scheduling on
         // the host: each tile, in that order, to the unit with the least work so far; the last few waves'
-        // worth of tiles are taken heaviest first so that the units finish together.  Unit u then owns table
+        // worth of tiles (all of them when there are only a few waves) are taken heaviest first so that the
+        // units finish together.  Unit u then owns table
         // entries u, u + units, u + 2*units, ...; rounds a unit has no tile for hold a dummy entry that lies
         // outside the matrix (nothing loaded or stored).
         bool uniform = true;
@@ -768,7 +769,8 @@ mom_status_t tc_prepare(const mom_plan &p, TcPlanState &s) {
             if (split <= 1) {
                 size_t busy = 0;
                 while (busy < tab.size() && tab[busy].w > tab[busy].z) ++busy;
-                const size_t tail = std::min(busy, (size_t)3 * units);
+                // with few waves of tiles the makespan matters more than locality: everything heaviest first
+                const size_t tail = busy <= (size_t)6 * units ? busy : (size_t)3 * units;
                 std::stable_sort(tab.begin() + (busy - tail), tab.begin() + busy,
                                  [](const int4 &x, const int4 &y) { return (x.w - x.z) > (y.w - y.z); });
             } else {
