@@ -462,6 +462,20 @@ def run_gpu(args):
             torch.cuda.empty_cache()
         result["all_configs"] = others
 
+        # ---- the FFMA comparison variant on the property-heavy configuration, against the FP32 FMA peak
+        if args.variant == "3xtf32":
+            cfg = wl.config_property_heavy()
+            r = time_equation(mom, torch, cfg, mom.VARIANT_FFMA, steps=10, warmup=3, stream=stream, timing=False)
+            ms_med = statistics.median(r["ms"])
+            clock_mhz = result.get("clocks", {}).get("sm_max_mhz") or 1965.0
+            ffma_peak = torch.cuda.get_device_properties(local).multi_processor_count * 128 * 2 * clock_mhz * 1e6 / 1e12
+            tf = r["useful_flops"] / (ms_med * 1e-3) / 1e12
+            result["ffma_variant"] = {"workload": cfg.name, "ms_median": ms_med, "tflops_useful": tf,
+                                      "peak_tflops": ffma_peak, "peak_is": "SMs x 128 lanes x 2 x max SM clock",
+                                      "frac": tf / ffma_peak, "frac_of_probe": (tf / probes["ffma_tflops"]) if isinstance(probes.get("ffma_tflops"), float) else None}
+            del r
+            torch.cuda.empty_cache()
+
         # ---- CPU baseline: the oracle on a bounded sample of the same workload
         result["cpu_baseline"] = cpu_baseline(eq, chain, add, useful, n_rows=256)
 

@@ -147,6 +147,21 @@ def test_workspace_covers_intermediates_and_planes():
     assert mom.mom_equation_plan(wl.config_tiny_identity_left().descs()).workspace_bytes() == 0
 
 
+def test_host_upload_bytes_count_triangles_by_blocks():
+    n = 1288
+    blocks = [(r0, min(n, r0 + 256)) for r0 in range(0, n, 256)]
+    lower = sum((r1 - r0) * r1 for r0, r1 in blocks) * 4
+    upper = sum((r1 - r0) * (n - r0) for r0, r1 in blocks) * 4
+    L, U, G, I = mom.LOWER_TRI, mom.UPPER_TRI, mom.GENERAL, mom.IDENTITY
+    p = mom.mom_equation_plan([(n, n, L), (n, n, I), (n, n, G), (n, n, U)], [(n, n, G)])
+    assert p.host_upload_bytes(1) == lower + upper + 2 * n * n * 4           # Identity is never copied
+    assert p.host_upload_bytes(3) == 3 * 5 * n * n * 4 - 3 * n * n * 4       # batches are copied in full
+    small = mom.mom_equation_plan([(512, 512, L), (512, 512, G)])
+    assert small.host_upload_bytes(1) == 2 * 512 * 512 * 4                   # below 1024 rows: one plain copy
+    shared = mom.mom_equation_plan_sum([[(64, 64, G), (64, 64, G)], [(64, 64, G)]], None, [[0, 1], [0]])
+    assert shared.host_upload_bytes(1) == 2 * 64 * 64 * 4                    # a named matrix once
+
+
 def test_step_kinds():
     L, U, G = mom.LOWER_TRI, mom.UPPER_TRI, mom.GENERAL
     cases = {(G, G): mom.KIND_GG, (L, G): mom.KIND_TG, (U, G): mom.KIND_TG, (G, L): mom.KIND_GT, (G, U): mom.KIND_GT,
