@@ -90,6 +90,9 @@ def test_identity_only_and_single_operand():
     ([(0, 3, 0)], [], mom.ERR_INVALID_ARG, "invalid_arg"),
     ([(3, 4, 1)], [], mom.ERR_PROPERTY, "property"),
     ([(3, 4, 3)], [], mom.ERR_PROPERTY, "property"),
+    ([(3, 4, 4)], [], mom.ERR_PROPERTY, "property"),
+    ([(3, 4, 5)], [], mom.ERR_PROPERTY, "property"),
+    ([(3, 3, 0)], [(3, 3, 6)], mom.ERR_INVALID_ARG, "property"),
     ([(3, 4, 0), (5, 3, 0)], [], mom.ERR_SHAPE_MISMATCH, "shape_mismatch"),
     ([(3, 4, 0)], [(3, 5, 0)], mom.ERR_SHAPE_MISMATCH, "shape_mismatch"),
 ])
@@ -117,6 +120,12 @@ def test_more_errors():
         mom.mom_equation_plan([(big, big, 0), (big, big, 0)], [])
     assert e.value.status == mom.ERR_OVERFLOW
     assert mom.status_string(mom.ERR_OVERFLOW)
+    with pytest.raises(mom.MomError) as e:                      # a Gram product's multiplication count overflows too
+        mom.mom_equation_plan_sum([[(big, big, 0), (big, big, 0)]], [[False, True]], [[0, 0]])
+    assert e.value.status == mom.ERR_OVERFLOW
+    with pytest.raises(mom.MomError) as e:
+        mom.mom_equation_plan([(4, 4, 0)], [], 4)               # unknown variant
+    assert e.value.status == mom.ERR_INVALID_ARG
 
 
 def test_workspace_covers_intermediates_and_planes():
