@@ -23,13 +23,15 @@ struct DeviceState {
     long long timed_executes = 0;       // executes recorded since timing was enabled
     // host-staging entry point: uploads run on a stream of their own, one event per operand, so that the first
     // products start while later operands are still on their way
-    cudaStream_t copy_stream = nullptr;
-    cudaEvent_t call_start = nullptr;
+    cudaStream_t copy_stream = nullptr, back_stream = nullptr;
+    cudaEvent_t call_start = nullptr, first_rows_done = nullptr, back_done = nullptr;
     std::vector<cudaEvent_t> slot_ready, add_ready;
 };
 
 // events the launcher has to wait for before it first uses an operand (host-staging entry point only)
-struct StageEvents { const cudaEvent_t *slot; const cudaEvent_t *add; };
+// and, the other way, an event the launcher records once the first rows of X are final (first_rows is set to their
+// number, 0 when X is only final at the end)
+struct StageEvents { const cudaEvent_t *slot; const cudaEvent_t *add; cudaEvent_t first_rows_done; int *first_rows; };
 
 constexpr int TIMING_SLOTS = 32;
 
@@ -58,7 +60,10 @@ void destroy_device_state(DeviceState *d) {
     for (cudaEvent_t e : d->slot_ready) cudaEventDestroy(e);
     for (cudaEvent_t e : d->add_ready) cudaEventDestroy(e);
     if (d->call_start) cudaEventDestroy(d->call_start);
+    if (d->first_rows_done) cudaEventDestroy(d->first_rows_done);
+    if (d->back_done) cudaEventDestroy(d->back_done);
     if (d->copy_stream) cudaStreamDestroy(d->copy_stream);
+    if (d->back_stream) cudaStreamDestroy(d->back_stream);
     if (d->status) cudaFree(d->status);
     if (d->fused_table) cudaFree(d->fused_table);
     if (prev >= 0) cudaSetDevice(prev);
@@ -389,7 +394,20 @@ mom_status_t execute_impl(const mom_plan *p, const float *const *chain_ptrs, con
                 if (ev) cudaEventRecord(ev[0], stream);
                 if (stp.pub.uses_tensor_cores == 1) {
                     int used = 0;
-                    st = tc_launch_step(*p, p->dev->tc, s, a, ws, p->dev->status, stream, &used, ev ? ev[1] : nullptr);
+                    // the host-staging entry point copies the first rows of X back while the rest is still computed:
+                    // the product that writes X then runs as two launches (only when nothing is added to X afterwards)
+                    const bool two_parts = staged && staged->first_rows && top && stp.is_last && !stp.accumulate &&
+                                           added >= n_simple && batch == 1 && p->dev->tc.steps[s].part_row > 0;
+                    if (two_parts) {
+                        st = tc_launch_step(*p, p->dev->tc, s, a, ws, p->dev->status, stream, &used, ev ? ev[1] : nullptr, 1);
+                        if (st != MOM_OK) return st;
+                        launches += used;
+                        if (cudaEventRecord(staged->first_rows_done, stream) != cudaSuccess) return MOM_ERR_CUDA;
+                        *staged->first_rows = p->dev->tc.steps[s].part_row;
+                        st = tc_launch_step(*p, p->dev->tc, s, a, ws, p->dev->status, stream, &used, nullptr, 2);
+                    } else {
+                        st = tc_launch_step(*p, p->dev->tc, s, a, ws, p->dev->status, stream, &used, ev ? ev[1] : nullptr);
+                    }
                     if (st != MOM_OK) return st;
                     launches += used;
                 } else {
@@ -460,7 +478,10 @@ mom_status_t mom_equation_execute_host(const mom_plan_t *plan, const float *cons
     mom::DeviceState *dev = plan->dev;
     if (!dev->copy_stream) {
         if (cudaStreamCreateWithFlags(&dev->copy_stream, cudaStreamNonBlocking) != cudaSuccess) return MOM_ERR_CUDA;
+        if (cudaStreamCreateWithFlags(&dev->back_stream, cudaStreamNonBlocking) != cudaSuccess) return MOM_ERR_CUDA;
         if (cudaEventCreateWithFlags(&dev->call_start, cudaEventDisableTiming) != cudaSuccess) return MOM_ERR_CUDA;
+        if (cudaEventCreateWithFlags(&dev->first_rows_done, cudaEventDisableTiming) != cudaSuccess) return MOM_ERR_CUDA;
+        if (cudaEventCreateWithFlags(&dev->back_done, cudaEventDisableTiming) != cudaSuccess) return MOM_ERR_CUDA;
     }
     while ((int)dev->slot_ready.size() < n_chain || (int)dev->add_ready.size() < n_add) {
         cudaEvent_t e = nullptr;
@@ -539,7 +560,8 @@ mom_status_t mom_equation_execute_host(const mom_plan_t *plan, const float *cons
         astride[i] = d.rows * d.cols;
         cur += mom::align_up(bytes, mom::WS_ALIGN);
     }
-    const mom::StageEvents staged{dev->slot_ready.data(), dev->add_ready.data()};
+    int first_rows = 0;
+    const mom::StageEvents staged{dev->slot_ready.data(), dev->add_ready.data(), dev->first_rows_done, &first_rows};
     float *x = reinterpret_cast<float *>(cur);
     const int64_t xelems = plan->result_desc.rows * plan->result_desc.cols;
     const size_t xbytes = (size_t)xelems * sizeof(float) * batch;
@@ -560,7 +582,18 @@ mom_status_t mom_equation_execute_host(const mom_plan_t *plan, const float *cons
         return MOM_ERR_ALIGNMENT;
     }
     if (st != MOM_OK) return st;
-    if (cudaMemcpyAsync(out_host, x, xbytes, cudaMemcpyDeviceToHost, stream) != cudaSuccess) return MOM_ERR_CUDA;
+    if (first_rows > 0) {
+        // the first rows of X are final before the last launch ends: they travel on a stream of their own meanwhile
+        const size_t head = (size_t)first_rows * plan->result_desc.cols * sizeof(float);
+        if (cudaStreamWaitEvent(dev->back_stream, dev->first_rows_done, 0) != cudaSuccess) return MOM_ERR_CUDA;
+        if (cudaMemcpyAsync(out_host, x, head, cudaMemcpyDeviceToHost, dev->back_stream) != cudaSuccess) return MOM_ERR_CUDA;
+        if (cudaEventRecord(dev->back_done, dev->back_stream) != cudaSuccess) return MOM_ERR_CUDA;
+        if (cudaMemcpyAsync(reinterpret_cast<char *>(out_host) + head, reinterpret_cast<char *>(x) + head, xbytes - head,
+                            cudaMemcpyDeviceToHost, stream) != cudaSuccess) return MOM_ERR_CUDA;
+        if (cudaStreamWaitEvent(stream, dev->back_done, 0) != cudaSuccess) return MOM_ERR_CUDA;
+    } else if (cudaMemcpyAsync(out_host, x, xbytes, cudaMemcpyDeviceToHost, stream) != cudaSuccess) {
+        return MOM_ERR_CUDA;
+    }
     if (cudaStreamSynchronize(stream) != cudaSuccess) return MOM_ERR_CUDA;
     return MOM_OK;
 }

@@ -691,8 +691,14 @@ mom_status_t tc_prepare(const mom_plan &p, TcPlanState &s) {
     if (s.ready) return MOM_OK;
     const int ns = (int)p.steps.size();
     s.steps.assign(ns, TcStepState{});
-    std::vector<std::vector<int4>> tables(ns);
+    std::vector<std::vector<int4>> tables(ns), part_tables[2] = {std::vector<std::vector<int4>>(ns), std::vector<std::vector<int4>>(ns)};
     size_t total = 0;
+    int sms = 0;
+    {
+        int dev = 0;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    }
     for (int i = 0; i < ns; ++i) {
         const mom_step_t &st = p.steps[i].pub;
         if (st.uses_tensor_cores != 1) continue;
@@ -736,63 +742,72 @@ mom_status_t tc_prepare(const mom_plan &p, TcPlanState &s) {
         // units finish together.  Unit u then owns table
         // entries u, u + units, u + 2*units, ...; rounds a unit has no tile for hold a dummy entry that lies
         // outside the matrix (nothing loaded or stored).
-        bool uniform = true;
-        for (const int4 &t : tab) uniform &= (t.w - t.z) == (tab[0].w - tab[0].z);
-        int sms = 0;
-        {
-            int dev = 0;
-            cudaGetDevice(&dev);
-            cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-        }
-        const int units = std::max(1, std::min((int)tab.size(), s.steps[i].pair ? sms / 2 : sms));   // CTAs, or CTA pairs
-        s.steps[i].units = units;
-        if (split <= 1) {
-            const int band = s.steps[i].pair ? 8 : 16;                 // tile rows per band (2048 rows)
-            const int n_bands = ((m + tile_rows - 1) / tile_rows + band - 1) / band;
-            auto band_of = [&](const int4 &t) { return (t.x & TILE_ROW_MASK) / tile_rows / band; };
-            std::vector<long long> band_work(n_bands, 0);
-            for (const int4 &t : tab) band_work[band_of(t)] += t.w - t.z;
-            std::vector<int> by_work(n_bands), rank(n_bands);
-            for (int b2 = 0; b2 < n_bands; ++b2) by_work[b2] = b2;
-            std::stable_sort(by_work.begin(), by_work.end(), [&](int x, int y) { return band_work[x] > band_work[y]; });
-            for (int r2 = 0; r2 < n_bands; ++r2) rank[by_work[r2]] = r2;
-            std::stable_sort(tab.begin(), tab.end(), [&](const int4 &x, const int4 &y) {
-                const bool zx = x.w <= x.z, zy = y.w <= y.z;
-                if (zx != zy) return zy;
-                const int rx = rank[band_of(x)], ry = rank[band_of(y)];
-                if (rx != ry) return rx < ry;
-                if (x.y != y.y) return (rx & 1) ? x.y > y.y : x.y < y.y;
-                return (x.x & TILE_ROW_MASK) < (y.x & TILE_ROW_MASK);
-            });
-        }
-        if (!uniform) {
+        auto order = [&](std::vector<int4> &tab) -> int {    // orders `tab` in place, returns the units it was laid out for
+            if (tab.empty()) return 1;
+            bool uniform = true;
+            for (const int4 &t : tab) uniform &= (t.w - t.z) == (tab[0].w - tab[0].z);
+            const int units = std::max(1, std::min((int)tab.size(), s.steps[i].pair ? sms / 2 : sms));   // CTAs, or CTA pairs
             if (split <= 1) {
-                size_t busy = 0;
-                while (busy < tab.size() && tab[busy].w > tab[busy].z) ++busy;
-                // with few waves of tiles the makespan matters more than locality: everything heaviest first
-                const size_t tail = busy <= (size_t)6 * units ? busy : (size_t)3 * units;
-                std::stable_sort(tab.begin() + (busy - tail), tab.begin() + busy,
-                                 [](const int4 &x, const int4 &y) { return (x.w - x.z) > (y.w - y.z); });
-            } else {
-                std::stable_sort(tab.begin(), tab.end(), [](const int4 &x, const int4 &y) { return (x.w - x.z) > (y.w - y.z); });
+                const int band = s.steps[i].pair ? 8 : 16;                 // tile rows per band (2048 rows)
+                const int n_bands = ((m + tile_rows - 1) / tile_rows + band - 1) / band;
+                auto band_of = [&](const int4 &t) { return (t.x & TILE_ROW_MASK) / tile_rows / band; };
+                std::vector<long long> band_work(n_bands, 0);
+                for (const int4 &t : tab) band_work[band_of(t)] += t.w - t.z;
+                std::vector<int> by_work(n_bands), rank(n_bands);
+                for (int b2 = 0; b2 < n_bands; ++b2) by_work[b2] = b2;
+                std::stable_sort(by_work.begin(), by_work.end(), [&](int x, int y) { return band_work[x] > band_work[y]; });
+                for (int r2 = 0; r2 < n_bands; ++r2) rank[by_work[r2]] = r2;
+                std::stable_sort(tab.begin(), tab.end(), [&](const int4 &x, const int4 &y) {
+                    const bool zx = x.w <= x.z, zy = y.w <= y.z;
+                    if (zx != zy) return zy;
+                    const int rx = rank[band_of(x)], ry = rank[band_of(y)];
+                    if (rx != ry) return rx < ry;
+                    if (x.y != y.y) return (rx & 1) ? x.y > y.y : x.y < y.y;
+                    return (x.x & TILE_ROW_MASK) < (y.x & TILE_ROW_MASK);
+                });
             }
-            constexpr long long TILE_OVERHEAD = 3 * BK;         // epilogue and pipeline fill, in k units
-            std::vector<std::vector<int4>> mine(units);
-            std::vector<long long> load(units, 0);
-            for (const int4 &t : tab) {
-                int best = 0;
-                for (int u = 1; u < units; ++u)
-                    if (load[u] < load[best]) best = u;
-                mine[best].push_back(t);
-                load[best] += (t.w - t.z) + TILE_OVERHEAD;
+            if (!uniform) {
+                if (split <= 1) {
+                    size_t busy = 0;
+                    while (busy < tab.size() && tab[busy].w > tab[busy].z) ++busy;
+                    // with few waves of tiles the makespan matters more than locality: everything heaviest first
+                    const size_t tail = busy <= (size_t)6 * units ? busy : (size_t)3 * units;
+                    std::stable_sort(tab.begin() + (busy - tail), tab.begin() + busy,
+                                     [](const int4 &x, const int4 &y) { return (x.w - x.z) > (y.w - y.z); });
+                } else {
+                    std::stable_sort(tab.begin(), tab.end(), [](const int4 &x, const int4 &y) { return (x.w - x.z) > (y.w - y.z); });
+                }
+                constexpr long long TILE_OVERHEAD = 3 * BK;         // epilogue and pipeline fill, in k units
+                std::vector<std::vector<int4>> mine(units);
+                std::vector<long long> load(units, 0);
+                for (const int4 &t : tab) {
+                    int best = 0;
+                    for (int u = 1; u < units; ++u)
+                        if (load[u] < load[best]) best = u;
+                    mine[best].push_back(t);
+                    load[best] += (t.w - t.z) + TILE_OVERHEAD;
+                }
+                size_t rounds = 0;
+                for (const auto &v : mine) rounds = std::max(rounds, v.size());
+                const int4 dummy = make_int4(TILE_ROW_MASK & ~(P_BM - 1), n + BN, 0, 0);
+                tab.assign(rounds * units, dummy);
+                for (int u = 0; u < units; ++u)
+                    for (size_t r = 0; r < mine[u].size(); ++r) tab[r * units + u] = mine[u][r];
             }
-            size_t rounds = 0;
-            for (const auto &v : mine) rounds = std::max(rounds, v.size());
-            const int4 dummy = make_int4(TILE_ROW_MASK & ~(P_BM - 1), n + BN, 0, 0);
-            tab.assign(rounds * units, dummy);
-            for (int u = 0; u < units; ++u)
-                for (size_t r = 0; r < mine[u].size(); ++r) tab[r * units + u] = mine[u][r];
+            return units;
+        };
+        // the product that writes X, when it is large and plain: also as two row ranges (see TcStepState)
+        const bool top_root = p.steps[i].is_last && !p.steps[i].accumulate && p.steps[i].sum + 1 == (int)p.sums.size();
+        if (top_root && s.steps[i].pair && split <= 1 && !s.steps[i].mirror && m >= 2048) {
+            const int row = std::max(P_BM, (int)(0.4 * m) / P_BM * P_BM);
+            for (const int4 &t : tab) part_tables[(t.x & TILE_ROW_MASK) < row ? 0 : 1][i].push_back(t);
+            s.steps[i].part_row = row;
+            for (int q = 0; q < 2; ++q) {
+                s.steps[i].part_units[q] = order(part_tables[q][i]);
+                total += part_tables[q][i].size();
+            }
         }
+        s.steps[i].units = order(tab);
         total += tab.size();
     }
     if (total == 0) { s.ready = true; return MOM_OK; }
@@ -808,6 +823,18 @@ mom_status_t tc_prepare(const mom_plan &p, TcPlanState &s) {
         s.steps[i].tiles = cur;
         s.steps[i].num_tiles = (int)tables[i].size();
         cur += tables[i].size();
+        for (int q = 0; q < 2; ++q) {
+            const std::vector<int4> &pt = part_tables[q][i];
+            if (pt.empty()) continue;
+            if (cudaMemcpy(cur, pt.data(), pt.size() * sizeof(int4), cudaMemcpyHostToDevice) != cudaSuccess) {
+                cudaFree(s.block);
+                s.block = nullptr;
+                return MOM_ERR_CUDA;
+            }
+            s.steps[i].part_tiles[q] = cur;
+            s.steps[i].part_num[q] = (int)pt.size();
+            cur += pt.size();
+        }
     }
     s.ready = true;
     return MOM_OK;
@@ -821,9 +848,13 @@ void tc_release(TcPlanState &s) {
 }
 
 mom_status_t tc_launch_step(const mom_plan &p, TcPlanState &s, int step, const ProductArgs &a, char *workspace,
-                            int32_t *status, cudaStream_t stream, int *launches, cudaEvent_t before_product) {
+                            int32_t *status, cudaStream_t stream, int *launches, cudaEvent_t before_product, int part) {
     const StepImpl &st = p.steps[step];
     if (!s.ready || step >= (int)s.steps.size() || !s.steps[step].tiles) return MOM_ERR_INVALID_ARG;
+    if (part < 0 || part > 2 || (part > 0 && (s.steps[step].part_row == 0 || !s.steps[step].part_tiles[part - 1]))) return MOM_ERR_INVALID_ARG;
+    const int4 *tiles = part ? s.steps[step].part_tiles[part - 1] : s.steps[step].tiles;
+    const int num_tiles = part ? s.steps[step].part_num[part - 1] : s.steps[step].num_tiles;
+    const int units = part ? s.steps[step].part_units[part - 1] : s.steps[step].units;
     if (!g_sm_count) {
         int dev = 0;
         cudaGetDevice(&dev);
@@ -849,12 +880,12 @@ mom_status_t tc_launch_step(const mom_plan &p, TcPlanState &s, int step, const P
     // a folded scaling: rows of the operand as used <-> rows of the matrix as stored unless it is stored transposed
     const SplitScale sa{a.scaleA, a.scaleA_step, a.scaleA ? (a.scaleA_rows != 0) != (a.transA != 0) : 0};
     const SplitScale sb{a.scaleB, a.scaleB_step, a.scaleB ? (a.scaleB_rows != 0) != (a.transB != 0) : 0};
-    if (!st.a_planes_ready) {
+    if (!st.a_planes_ready && part != 2) {
         if (!a.transA) split_planes_kernel<false><<<dim3(blocks(a.k), blocks(a.m)), 256, 0, stream>>>(a.A, a_hi, a_lo, a.m, a.k, a.pa, sa);
         else split_planes_kernel<true><<<dim3(blocks(a.m), blocks(a.k)), 256, 0, stream>>>(a.A, a_hi, a_lo, a.k, a.m, stored_prop(a.pa), sa);
         ++split_launches;
     }
-    if (!st.b_planes_ready) {
+    if (!st.b_planes_ready && part != 2) {
         if (!a.transB) split_planes_kernel<true><<<dim3(blocks(a.n), blocks(a.k)), 256, 0, stream>>>(a.B, b_hi, b_lo, a.k, a.n, a.pb, sb);
         else split_planes_kernel<false><<<dim3(blocks(a.k), blocks(a.n)), 256, 0, stream>>>(a.B, b_hi, b_lo, a.n, a.k, stored_prop(a.pb), sb);
         ++split_launches;
@@ -886,8 +917,8 @@ mom_status_t tc_launch_step(const mom_plan &p, TcPlanState &s, int step, const P
     if (!ok) return MOM_ERR_CUDA;
 
     TcParams prm;
-    prm.tiles = s.steps[step].tiles;
-    prm.num_tiles = s.steps[step].num_tiles;
+    prm.tiles = tiles;
+    prm.num_tiles = num_tiles;
     prm.m = a.m;
     prm.n = a.n;
     prm.pout = st.split_k > 1 ? (int)MOM_GENERAL : a.pout;      // split-K: mask and Add terms are applied by the reduction
@@ -926,11 +957,11 @@ mom_status_t tc_launch_step(const mom_plan &p, TcPlanState &s, int step, const P
             if (cudaOccupancyMaxActiveClusters(&n, product_tc_pair_kernel, &cfg) != cudaSuccess || n < 1) return MOM_ERR_CUDA;
             max_pairs = n;
         }
-        if (max_pairs < s.steps[step].units) return MOM_ERR_CUDA;   // the table was laid out for co-resident pairs
-        cfg.gridDim = dim3(2 * s.steps[step].units);
+        if (max_pairs < units) return MOM_ERR_CUDA;   // the table was laid out for co-resident pairs
+        cfg.gridDim = dim3(2 * units);
         if (cudaLaunchKernelEx(&cfg, product_tc_pair_kernel, ma_hi, ma_lo, mb_hi, mb_lo, mc, mc2, prm) != cudaSuccess) return MOM_ERR_CUDA;
     } else {
-        const int grid = std::min(s.steps[step].units, g_sm_count);
+        const int grid = std::min(units, g_sm_count);
         product_tc_kernel<<<grid, THREADS, SMEM_BYTES, stream>>>(ma_hi, ma_lo, mb_hi, mb_lo, mc, mc2, prm);
     }
     if (cudaGetLastError() != cudaSuccess) return MOM_ERR_CUDA;

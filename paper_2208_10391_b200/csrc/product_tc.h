@@ -13,6 +13,12 @@ struct TcStepState {
     int num_tiles = 0;
     bool pair = false;          // tiles are 256 rows high and run on CTA pairs (cta_group::2)
     bool mirror = false;        // Gram product: tiles on and below the diagonal only, the others written as mirror images
+    // The product that writes X can also run as two launches, rows [0, part_row) first: the host-staging entry
+    // point copies those rows back while the second launch runs.  part_row == 0: no such tables.
+    int part_row = 0;
+    int4 *part_tiles[2] = {nullptr, nullptr};
+    int part_num[2] = {0, 0};
+    int part_units[2] = {1, 1};
     int units = 1;              // CTAs (or CTA pairs) the table was laid out for: unit u owns entries u, u + units, ...
 };
 
@@ -27,8 +33,9 @@ mom_status_t tc_prepare(const mom_plan &p, TcPlanState &s);
 
 // Enqueues the operand splits and the product kernel of step `step`.  `before_product`, when not
 // null, is recorded on the stream between the splits and the product kernel.
+// `part`: 0 the whole product; 1 the operand splits and the rows [0, part_row); 2 the remaining rows (no splits).
 mom_status_t tc_launch_step(const mom_plan &p, TcPlanState &s, int step, const ProductArgs &a, char *workspace,
-                            int32_t *status, cudaStream_t stream, int *launches, cudaEvent_t before_product);
+                            int32_t *status, cudaStream_t stream, int *launches, cudaEvent_t before_product, int part = 0);
 
 void tc_release(TcPlanState &s);
 

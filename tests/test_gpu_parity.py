@@ -245,6 +245,20 @@ def test_host_entry_point_uploads_large_triangles_by_blocks():
     assert np.array_equal(xd2, xh2)
 
 
+def test_host_entry_point_copies_the_first_rows_back_early():
+    # from 2048 rows on, the product that writes X runs as two launches in the host entry point (rows up to a
+    # multiple of 256 near 40 % first) and the first rows travel back during the second launch; same bits as one launch
+    for n, add in ((2312, ()), (2048, (Operand(2048, 2048, G, "normal"),))):
+        eq = Equation(f"host_parts_{n}", 91, (Operand(n, n, L), Operand(n, n, G, "normal", 0.02)), add)
+        chain, terms = wl.generate(eq)
+        xd, plan, _ = run_equation(eq, mom.VARIANT_3XTF32, chain, terms, via="device")
+        xh, plan_h, _ = run_equation(eq, mom.VARIANT_3XTF32, chain, terms, via="host")
+        assert np.array_equal(xd, xh)
+        assert plan_h.last_launch_count() == plan.last_launch_count() + 1
+        rows = np.sort(np.random.default_rng(8).choice(n, size=24, replace=False))
+        check_against_oracle(eq, xh, plan_h, chain, terms, rows=rows)
+
+
 @pytest.mark.parametrize("variant", VARIANTS, ids=VNAME.get)
 def test_host_entry_point_matches_device_entry_point(variant):
     for eq in (wl.config_tiny(), wl.config_batched(batch=9), wl.config_property_heavy(n=264)):
