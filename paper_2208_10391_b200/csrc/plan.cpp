@@ -499,7 +499,7 @@ static mom_status_t plan_sums(const std::vector<mom_matrix_desc_t> &slots, const
             if (st.pub.uses_tensor_cores == 1) {
                 // few output tiles, long contraction: split k over otherwise idle SMs
                 const int64_t tiles = ((m + mom::TC_BM - 1) / mom::TC_BM) * ((n + mom::TC_BN - 1) / mom::TC_BN);
-                if (tiles <= 37 && k >= 512) {
+                if ((tiles <= 37 && k >= 512) || (tiles <= 74 && k >= 1024)) {      // up to half of the SMs busy otherwise
                     int64_t split = std::min<int64_t>(std::min<int64_t>(148 / tiles, k / 128), 32);
                     if (split >= 2) st.split_k = (int)split;
                 }
