@@ -567,10 +567,9 @@ struct SplitScale {
 };
 
 template <bool TRANSPOSE>
-__global__ void __launch_bounds__(256)
-split_planes_kernel(const float *__restrict__ src, float *__restrict__ hi, float *__restrict__ lo, int rows, int cols, int prop,
-                    SplitScale sc) {
-    const int pr = blockIdx.y * SPLIT_PIECE, pc = blockIdx.x * SPLIT_PIECE;
+__device__ __forceinline__ void split_piece(const float *__restrict__ src, float *__restrict__ hi, float *__restrict__ lo, int rows,
+                                            int cols, int prop, const SplitScale &sc, int piece_x, int piece_y) {
+    const int pr = piece_y * SPLIT_PIECE, pc = piece_x * SPLIT_PIECE;
     const int br = pr / SPLIT_BLOCK * SPLIT_BLOCK, bc = pc / SPLIT_BLOCK * SPLIT_BLOCK;
     if (prop == MOM_LOWER_TRI && bc > br + SPLIT_BLOCK - 1) return;     // block wholly above the diagonal
     if (prop == MOM_UPPER_TRI && br > bc + SPLIT_BLOCK - 1) return;     // wholly below
@@ -624,6 +623,31 @@ split_planes_kernel(const float *__restrict__ src, float *__restrict__ hi, float
             }
         }
     }
+}
+
+template <bool TRANSPOSE>
+__global__ void __launch_bounds__(256)
+split_planes_kernel(const float *__restrict__ src, float *__restrict__ hi, float *__restrict__ lo, int rows, int cols, int prop,
+                    SplitScale sc) {
+    split_piece<TRANSPOSE>(src, hi, lo, rows, cols, prop, sc, blockIdx.x, blockIdx.y);
+}
+
+// Both operands of one product in ONE launch (a launch costs about as much as splitting a few MB): the first
+// pieces_a CTAs split the left operand, the others the right one.
+struct SplitJob {
+    const float *src;
+    float *hi, *lo;
+    int rows, cols, prop, transpose, pieces_x;
+    SplitScale sc;
+};
+__global__ void __launch_bounds__(256)
+split_both_kernel(SplitJob a, SplitJob b, int pieces_a) {
+    const bool first = (int)blockIdx.x < pieces_a;
+    const SplitJob &j = first ? a : b;
+    const int piece = first ? blockIdx.x : blockIdx.x - pieces_a;
+    const int px = piece % j.pieces_x, py = piece / j.pieces_x;
+    if (j.transpose) split_piece<true>(j.src, j.hi, j.lo, j.rows, j.cols, j.prop, j.sc, px, py);
+    else split_piece<false>(j.src, j.hi, j.lo, j.rows, j.cols, j.prop, j.sc, px, py);
 }
 
 // Split-K: sum the k-slices' partial results, then the usual finish (Add terms, structure mask).
@@ -880,14 +904,20 @@ mom_status_t tc_launch_step(const mom_plan &p, TcPlanState &s, int step, const P
     // a folded scaling: rows of the operand as used <-> rows of the matrix as stored unless it is stored transposed
     const SplitScale sa{a.scaleA, a.scaleA_step, a.scaleA ? (a.scaleA_rows != 0) != (a.transA != 0) : 0};
     const SplitScale sb{a.scaleB, a.scaleB_step, a.scaleB ? (a.scaleB_rows != 0) != (a.transB != 0) : 0};
-    if (!st.a_planes_ready && part != 2) {
-        if (!a.transA) split_planes_kernel<false><<<dim3(blocks(a.k), blocks(a.m)), 256, 0, stream>>>(a.A, a_hi, a_lo, a.m, a.k, a.pa, sa);
-        else split_planes_kernel<true><<<dim3(blocks(a.m), blocks(a.k)), 256, 0, stream>>>(a.A, a_hi, a_lo, a.k, a.m, stored_prop(a.pa), sa);
+    // as stored: rows x cols and the property of the matrix the kernel reads
+    const SplitJob ja{a.A, a_hi, a_lo, a.transA ? a.k : a.m, a.transA ? a.m : a.k, a.transA ? stored_prop(a.pa) : a.pa, a.transA ? 1 : 0,
+                      blocks(a.transA ? a.m : a.k), sa};
+    const SplitJob jb{a.B, b_hi, b_lo, a.transB ? a.n : a.k, a.transB ? a.k : a.n, a.transB ? stored_prop(a.pb) : a.pb, a.transB ? 0 : 1,
+                      blocks(a.transB ? a.k : a.n), sb};
+    const bool do_a = !st.a_planes_ready && part != 2, do_b = !st.b_planes_ready && part != 2;
+    auto pieces = [&](const SplitJob &j) { return j.pieces_x * blocks(j.rows); };
+    if (do_a && do_b) {
+        split_both_kernel<<<pieces(ja) + pieces(jb), 256, 0, stream>>>(ja, jb, pieces(ja));
         ++split_launches;
-    }
-    if (!st.b_planes_ready && part != 2) {
-        if (!a.transB) split_planes_kernel<true><<<dim3(blocks(a.n), blocks(a.k)), 256, 0, stream>>>(a.B, b_hi, b_lo, a.k, a.n, a.pb, sb);
-        else split_planes_kernel<false><<<dim3(blocks(a.k), blocks(a.n)), 256, 0, stream>>>(a.B, b_hi, b_lo, a.n, a.k, stored_prop(a.pb), sb);
+    } else if (do_a || do_b) {
+        const SplitJob &j = do_a ? ja : jb;
+        if (j.transpose) split_planes_kernel<true><<<dim3(j.pieces_x, blocks(j.rows)), 256, 0, stream>>>(j.src, j.hi, j.lo, j.rows, j.cols, j.prop, j.sc);
+        else split_planes_kernel<false><<<dim3(j.pieces_x, blocks(j.rows)), 256, 0, stream>>>(j.src, j.hi, j.lo, j.rows, j.cols, j.prop, j.sc);
         ++split_launches;
     }
     if (cudaGetLastError() != cudaSuccess) return MOM_ERR_CUDA;
