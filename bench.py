@@ -211,6 +211,21 @@ class ClockSampler:
                 "power_w_max": max(power) if power else None, "samples": len(sm), "reasons": sorted(reasons)}
 
 
+def planning_us(mom, eq, variant, repeats=15):
+    """Host time of one planning call through the binding (median of `repeats`), in microseconds."""
+    ts = []
+    for _ in range(repeats):
+        t0 = time.perf_counter()
+        if isinstance(eq, wl.Expression):
+            mom.mom_expression_plan(eq.expr, eq.descs(), variant)
+        elif isinstance(eq, wl.SumEquation):
+            mom.mom_equation_plan_sum(eq.descs(), eq.transposed, eq.names, variant)
+        else:
+            mom.mom_equation_plan_transposed(eq.descs(), eq.chain_t, eq.add_descs(), eq.add_t, variant)
+        ts.append((time.perf_counter() - t0) * 1e6)
+    return statistics.median(ts)
+
+
 def time_equation(mom, torch, eq, variant, steps, warmup, stream, timing=False):
     """Device-resident timing of one configuration: returns dict with per-step ms list, plan, launches."""
     if isinstance(eq, wl.Expression):
@@ -398,7 +413,8 @@ def run_gpu(args):
         "data": "synthetic",
         "config": {"workload": eq.name, "equation": "X = L*A*U*B, 8192x8192 f32, seed 3",
                    "parenthesization": plan.parenthesization(), "useful_flops": useful, "variant": args.variant,
-                   "l2": "operands (1 GiB) exceed L2; no flush", "parallelism": f"{world} independent replicas"},
+                   "l2": "operands (1 GiB) exceed L2; no flush", "parallelism": f"{world} independent replicas",
+                   "plan_us": planning_us(mom, eq, variant)},
         "clocks": clocks, "gpu_launches": launches, "roofline": roofline,
         "roofline_whole_equation_frac": (value / world / 1e3) / peak,
     }
@@ -452,7 +468,7 @@ def run_gpu(args):
                      "gflops_at_min": r["useful_flops"] / (ms_min * 1e-3) / 1e9,
                      "gflops_at_median": r["useful_flops"] / (ms_med * 1e-3) / 1e9,
                      "frac_of_roofline_at_median": r["useful_flops"] / (ms_med * 1e-3) / 1e12 / peak,
-                     "launches": r["launches"]}
+                     "launches": r["launches"], "plan_us": planning_us(mom, cfg, variant)}
             if batch > 1:
                 per_inst = sum(o.rows * o.cols for o in list(cfg.chain) + list(cfg.add)) + rd_elems(r["plan"])
                 entry["hbm_gbs_at_median"] = per_inst * 4 * cfg.batch / (ms_med * 1e-3) / 1e9
