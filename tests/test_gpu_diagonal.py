@@ -114,6 +114,10 @@ def test_batched_equations_with_diagonals(variant):
     assert plan.last_launch_count() == 1
     eq = Equation("b_large", 45, (Operand(200, 200, D), Operand(200, 200, G, "normal"), Operand(200, 200, U)), (), batch=5)
     both(eq, variant)
+    # tensor-core steps walk the instances one at a time; the folded scaling follows each instance's own D and S
+    both(eq, mom.VARIANT_3XTF32_FORCE)
+    eq = Equation("b_fold", 46, (Operand(264, 392, G, "normal"), Operand(392, 392, D), Operand(392, 520, G, "normal")), (Operand(264, 520, G),), batch=3)
+    both(eq, mom.VARIANT_3XTF32_FORCE)
 
 
 @pytest.mark.parametrize("variant", VARIANTS, ids=VNAME.get)
