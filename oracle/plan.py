@@ -34,8 +34,15 @@ Readings taken where the paper is silent (each also listed in the design notes):
     Diagonal factors are their own transposes), its value is Symmetric whatever the tree, and the tree that
     splits it in the middle computes only Y and then the lower triangle of Y * Y^T: the right half costs
     nothing and the product costs the multiplications of the entries (i, j) with i >= j;
+  * strictly triangular and unit triangular (two more of those properties; no printed rule): square, stored
+    densely; a strictly triangular matrix also has zeros on its diagonal, a unit triangular one has ones there
+    (stored as 1.0).  An entry known to be 1 needs no multiplication, exactly as Identity needs none: a
+    multiplication a_il * b_lj counts only when both entries are structural non-zeros and neither is a known 1.
+    So a unit triangle costs what the strict one costs.  Within one orientation a product's diagonal is the
+    product of the diagonals (zero if either is zero, one if both are one); in a sum the diagonals add
+    (zero + zero = zero, zero + one = one, anything else is ordinary data), so I + strictly lower = unit lower;
   * a transposed operand (paper Table 1, "Transpose") takes part with its transposed type: shape
-    swapped and lowerTri <-> upperTri (the inference rule the paper prints);
+    swapped and lowerTri <-> upperTri (the inference rule the paper prints), likewise for the strict and unit kinds;
   * reported mul_flops = 2 * multiplications; add_flops = structural non-zeros of the Add terms.
     (The factor 2 and the add_flops convention are bookkeeping of this project: parity unpinned by
     the paper, which only speaks of scalar multiplications.)
@@ -46,7 +53,11 @@ from dataclasses import dataclass
 from typing import List, Optional, Sequence, Tuple
 
 GENERAL, LOWER_TRI, UPPER_TRI, IDENTITY, DIAGONAL, SYMMETRIC = 0, 1, 2, 3, 4, 5
-PROPERTIES = (GENERAL, LOWER_TRI, UPPER_TRI, IDENTITY, DIAGONAL, SYMMETRIC)
+STRICT_LOWER, STRICT_UPPER, UNIT_LOWER, UNIT_UPPER = 6, 7, 8, 9
+PROPERTIES = (GENERAL, LOWER_TRI, UPPER_TRI, IDENTITY, DIAGONAL, SYMMETRIC,
+              STRICT_LOWER, STRICT_UPPER, UNIT_LOWER, UNIT_UPPER)
+LOWER_KINDS = (LOWER_TRI, STRICT_LOWER, UNIT_LOWER)
+UPPER_KINDS = (UPPER_TRI, STRICT_UPPER, UNIT_UPPER)
 
 
 class OracleError(ValueError):
@@ -99,13 +110,27 @@ def in_structure(prop: int, i: int, j: int) -> bool:
     """Is entry (i, j) a structural non-zero of a matrix with this property?"""
     if prop in (GENERAL, SYMMETRIC):
         return True
-    if prop == LOWER_TRI:
+    if prop in (LOWER_TRI, UNIT_LOWER):
         return i >= j
-    if prop == UPPER_TRI:
+    if prop in (UPPER_TRI, UNIT_UPPER):
         return i <= j
+    if prop == STRICT_LOWER:
+        return i > j
+    if prop == STRICT_UPPER:
+        return i < j
     if prop in (IDENTITY, DIAGONAL):
         return i == j
     raise OracleError("property", f"unknown property {prop}")
+
+
+def known_one(prop: int, i: int, j: int) -> bool:
+    """Is entry (i, j) known to be 1 from the type alone?  (The diagonal of Identity and of the unit triangles.)"""
+    return i == j and prop in (IDENTITY, UNIT_LOWER, UNIT_UPPER)
+
+
+def multiplies(prop: int, i: int, j: int) -> bool:
+    """Does entry (i, j) take part in multiplications: a structural non-zero that is not a known 1?"""
+    return in_structure(prop, i, j) and not known_one(prop, i, j)
 
 
 def brute_force_nonzeros(d: Desc) -> int:
@@ -116,21 +141,32 @@ def brute_force_nonzeros(d: Desc) -> int:
 def structural_nonzeros(d: Desc) -> int:
     if d.prop in (GENERAL, SYMMETRIC):
         return d.rows * d.cols
-    if d.prop in (LOWER_TRI, UPPER_TRI):
+    if d.prop in (LOWER_TRI, UPPER_TRI, UNIT_LOWER, UNIT_UPPER):
         return d.rows * (d.rows + 1) // 2
+    if d.prop in (STRICT_LOWER, STRICT_UPPER):
+        return d.rows * (d.rows - 1) // 2
     return d.rows                   # Identity, Diagonal
 
 
+def multiplying_entries(d: Desc) -> int:
+    """Structural non-zeros that are not known ones (what a Diagonal factor has to scale)."""
+    if d.prop == IDENTITY:
+        return 0
+    if d.prop in (UNIT_LOWER, UNIT_UPPER):
+        return d.rows * (d.rows - 1) // 2
+    return structural_nonzeros(d)
+
+
 def brute_force_mults(a: Desc, b: Desc) -> int:
-    """#{(i, l, j): (i, l) in S(A) and (l, j) in S(B)} by counting, for tiny shapes."""
+    """#{(i, l, j): (i, l) and (l, j) both structural non-zeros, neither a known 1} by counting, for tiny shapes."""
     assert a.cols == b.rows
     count = 0
     for i in range(a.rows):
         for l in range(a.cols):
-            if not in_structure(a.prop, i, l):
+            if not multiplies(a.prop, i, l):
                 continue
             for j in range(b.cols):
-                if in_structure(b.prop, l, j):
+                if multiplies(b.prop, l, j):
                     count += 1
     return count
 
@@ -138,58 +174,93 @@ def brute_force_mults(a: Desc, b: Desc) -> int:
 def product_mults(a: Desc, b: Desc) -> int:
     """Useful scalar multiplications of A*B in closed form (both operands non-Identity)."""
     assert a.cols == b.rows
-    ta = a.prop in (LOWER_TRI, UPPER_TRI)
-    tb = b.prop in (LOWER_TRI, UPPER_TRI)
+    ta = a.prop in LOWER_KINDS + UPPER_KINDS
+    tb = b.prop in LOWER_KINDS + UPPER_KINDS
     if a.prop == IDENTITY or b.prop == IDENTITY:
         return 0
-    if a.prop == DIAGONAL:         # row l of B is scaled by d_l: one multiplication per structural entry of B
-        return structural_nonzeros(b)
+    if a.prop == DIAGONAL:         # row l of B is scaled by d_l: one multiplication per multiplying entry of B
+        return multiplying_entries(b)
     if b.prop == DIAGONAL:         # column l of A is scaled by d_l
-        return structural_nonzeros(a)
+        return multiplying_entries(a)
     if not ta and not tb:
         return a.rows * a.cols * b.cols
+    # a strict or unit triangle multiplies with the entries strictly off its diagonal only
+    sa = 0 if a.prop in (LOWER_TRI, UPPER_TRI) else 1
+    sb = 0 if b.prop in (LOWER_TRI, UPPER_TRI) else 1
     if ta and not tb:
         n = a.rows
-        return b.cols * n * (n + 1) // 2
+        return b.cols * (n * (n + 1) // 2 - sa * n)
     if tb and not ta:
         n = b.rows
-        return a.rows * n * (n + 1) // 2
+        return a.rows * (n * (n + 1) // 2 - sb * n)
     n = a.rows
-    if a.prop == b.prop:           # L*L or U*U: sum over l of (#rows below l) * (#cols left of l) ...
-        return n * (n + 1) * (n + 2) // 6
-    return n * (n + 1) * (2 * n + 1) // 6   # L*U, U*L: sum of squares
+    if (a.prop in LOWER_KINDS) == (b.prop in LOWER_KINDS):
+        # L*L: triples i >= l + sa, l >= j + sb: choose three of n + 2 - sa - sb places
+        t = n + 2 - sa - sb
+        return t * (t - 1) * (t - 2) // 6
+    # L*U (U*L): column l of A and row l of B both hold t = n - l (l + 1) entries, less the excluded diagonal:
+    # sum over t = 1..n of (t - sa)(t - sb)
+    return n * (n + 1) * (2 * n + 1) // 6 - (sa + sb) * n * (n + 1) // 2 + sa * sb * n
 
 
 def brute_force_gram_mults(y: Desc) -> int:
     """#{(i, l, j): i >= j, (i, l) in S(Y) and (j, l) in S(Y)}: the multiplications of the lower triangle of Y*Y^T."""
     return sum(1 for i in range(y.rows) for j in range(i + 1) for l in range(y.cols)
-               if in_structure(y.prop, i, l) and in_structure(y.prop, j, l))
+               if multiplies(y.prop, i, l) and multiplies(y.prop, j, l))
 
 
 def gram_mults(y: Desc) -> int:
-    """The same in closed form (Y general, Symmetric or triangular)."""
+    """The same in closed form (Y general, Symmetric or one of the triangular kinds)."""
     if y.prop in (LOWER_TRI, UPPER_TRI):
         n = y.rows
         return n * (n + 1) * (n + 2) // 6
+    if y.prop in LOWER_KINDS + UPPER_KINDS:     # strict or unit: the diagonal takes no part
+        n = y.rows
+        return (n + 1) * n * (n - 1) // 6
     return y.cols * y.rows * (y.rows + 1) // 2
+
+
+def _region(p: int) -> str:
+    """Where the structural non-zeros may lie: 'D'iagonal, 'L'ower, 'U'pper, 'S'ymmetric (full), 'G'eneral (full)."""
+    if p in LOWER_KINDS:
+        return "L"
+    if p in UPPER_KINDS:
+        return "U"
+    return {GENERAL: "G", SYMMETRIC: "S", IDENTITY: "D", DIAGONAL: "D"}[p]
+
+
+def _diagonal(p: int) -> str:
+    """What the type says about the diagonal: 'zero', 'one' or ordinary 'data'."""
+    if p in (STRICT_LOWER, STRICT_UPPER):
+        return "zero"
+    if p in (IDENTITY, UNIT_LOWER, UNIT_UPPER):
+        return "one"
+    return "data"
+
+
+def _triangle(region: str, diagonal: str) -> int:
+    kinds = {"data": (LOWER_TRI, UPPER_TRI), "zero": (STRICT_LOWER, STRICT_UPPER), "one": (UNIT_LOWER, UNIT_UPPER)}
+    return kinds[diagonal][0 if region == "L" else 1]
 
 
 def join(p: int, q: int) -> int:
     """Property of a product: least upper bound in Identity < Diagonal < {lowerTri, upperTri} < general;
-    a product with a Symmetric factor is general (only S*I = S)."""
+    a product with a Symmetric factor is general (only S*I = S).  Inside one triangle the diagonal of the
+    product is the entrywise product of the diagonals: zero if either is zero, one if both are one."""
     if p == IDENTITY:
         return q
     if q == IDENTITY:
         return p
     if SYMMETRIC in (p, q):
         return GENERAL
-    if p == q:
-        return p
-    if p == DIAGONAL:
-        return q
-    if q == DIAGONAL:
-        return p
-    return GENERAL
+    rp, rq = _region(p), _region(q)
+    if rp == "D" and rq == "D":
+        return DIAGONAL
+    region = rq if rp == "D" else rp if rq == "D" else rp if rp == rq else "G"
+    if region not in ("L", "U"):
+        return GENERAL
+    dp, dq = _diagonal(p), _diagonal(q)
+    return _triangle(region, "zero" if "zero" in (dp, dq) else "one" if dp == dq == "one" else "data")
 
 
 def sum_property(product_prop: int, add_props: Sequence[int]) -> int:
@@ -201,13 +272,20 @@ def sum_property(product_prop: int, add_props: Sequence[int]) -> int:
     """
     if not add_props:
         return product_prop
-    props = [DIAGONAL if p == IDENTITY else p for p in [product_prop] + list(add_props)]
-    if SYMMETRIC in props:          # Symmetric + (Symmetric | Diagonal) is Symmetric; a triangle or a general summand breaks it
-        return SYMMETRIC if all(p in (SYMMETRIC, DIAGONAL) for p in props) else GENERAL
-    out = DIAGONAL
-    for p in props:
-        out = join(out, p)
-    return out
+    summands = [product_prop] + list(add_props)
+    if SYMMETRIC in summands:       # Symmetric + (Symmetric | Diagonal | Identity) is Symmetric; a triangle or a general summand breaks it
+        return SYMMETRIC if all(p in (SYMMETRIC, DIAGONAL, IDENTITY) for p in summands) else GENERAL
+    regions = {_region(p) for p in summands}
+    if "G" in regions or {"L", "U"} <= regions:
+        return GENERAL
+    if regions == {"D"}:
+        return DIAGONAL
+    # one triangle (plus diagonal summands): the diagonals add up
+    diagonal = "zero"
+    for p in summands:
+        d = _diagonal(p)
+        diagonal = d if diagonal == "zero" else diagonal if d == "zero" else "data"
+    return _triangle("L" if "L" in regions else "U", diagonal)
 
 
 # ----------------------------------------------------------------------------------------------
@@ -306,8 +384,9 @@ def transpose_desc(d: Desc) -> Desc:
     """Type of A^T given the type of A: shape swapped; paper Section 2, "Transformations", prints the
     inference rule lowerTriangular(A) -> upperTriangular(A^T) (and symmetrically); general, Diagonal,
     Symmetric and Identity keep their property."""
-    prop = {LOWER_TRI: UPPER_TRI, UPPER_TRI: LOWER_TRI}.get(d.prop, d.prop)
-    return Desc(d.cols, d.rows, prop)
+    swap = {LOWER_TRI: UPPER_TRI, UPPER_TRI: LOWER_TRI, STRICT_LOWER: STRICT_UPPER, STRICT_UPPER: STRICT_LOWER,
+            UNIT_LOWER: UNIT_UPPER, UNIT_UPPER: UNIT_LOWER}
+    return Desc(d.cols, d.rows, swap.get(d.prop, d.prop))
 
 
 def plan(chain: Sequence[Tuple[int, int, int]], add: Sequence[Tuple[int, int, int]] = (),

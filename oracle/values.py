@@ -19,6 +19,7 @@ from typing import List, Optional, Sequence, Tuple
 import numpy as np
 
 GENERAL, LOWER_TRI, UPPER_TRI, IDENTITY, DIAGONAL, SYMMETRIC = 0, 1, 2, 3, 4, 5
+STRICT_LOWER, STRICT_UPPER, UNIT_LOWER, UNIT_UPPER = 6, 7, 8, 9
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "matmul_f64.c")
@@ -93,9 +94,11 @@ def transposed_operands(arrays, descs, flags):
     """Operands as the equation uses them: entry i transposed (array and descriptor) where flags[i] is set.
 
     The transpose of a stored lowerTri matrix is upperTri and vice versa (the paper's printed inference
-    rule); Identity, Diagonal, Symmetric and general keep their property.  Dense storage is simply transposed with NumPy.
+    rule), likewise the strict and the unit triangles; Identity, Diagonal, Symmetric and general keep their
+    property.  Dense storage is simply transposed with NumPy.
     """
-    swap = {LOWER_TRI: UPPER_TRI, UPPER_TRI: LOWER_TRI}
+    swap = {LOWER_TRI: UPPER_TRI, UPPER_TRI: LOWER_TRI, STRICT_LOWER: STRICT_UPPER, STRICT_UPPER: STRICT_LOWER,
+            UNIT_LOWER: UNIT_UPPER, UNIT_UPPER: UNIT_LOWER}
     out_a, out_d = [], []
     flags = list(flags) + [False] * (len(descs) - len(flags))
     for a, (r, c, p), t in zip(arrays, descs, flags):
@@ -228,13 +231,27 @@ def off_structure_mask(rows: int, cols: int, prop: int, row_index: Optional[np.n
     j = np.arange(cols)[None, :]
     if prop in (GENERAL, SYMMETRIC):
         return np.zeros((i.shape[0], cols), dtype=bool)
-    if prop == LOWER_TRI:
+    if prop in (LOWER_TRI, UNIT_LOWER):
         return i < j
-    if prop == UPPER_TRI:
+    if prop in (UPPER_TRI, UNIT_UPPER):
         return i > j
+    if prop == STRICT_LOWER:
+        return i <= j
+    if prop == STRICT_UPPER:
+        return i >= j
     if prop in (IDENTITY, DIAGONAL):
         return i != j
     raise ValueError("unknown property")
+
+
+def unit_diagonal_exactly_one(x: np.ndarray, prop: int, row_index: Optional[np.ndarray] = None) -> bool:
+    """True iff the property fixes no diagonal of ones, or every diagonal entry of x (rows `row_index`) is exactly 1."""
+    if prop not in (UNIT_LOWER, UNIT_UPPER):
+        return True
+    x = np.asarray(x)
+    rows = np.arange(x.shape[-2]) if row_index is None else np.asarray(row_index)
+    inside = rows < x.shape[-1]
+    return bool(np.all(x[..., np.nonzero(inside)[0], rows[inside]] == 1.0))
 
 
 def off_structure_exactly_zero(x: np.ndarray, prop: int, row_index: Optional[np.ndarray] = None) -> bool:

@@ -269,7 +269,9 @@ def test_sum_property():
     ([(3, 4, L)], [], "property"),
     ([(3, 4, I)], [], "property"),
     ([(3, 4, D)], [], "property"),
-    ([(3, 3, 7)], [], "property"),
+    ([(3, 3, 10)], [], "property"),
+    ([(3, 4, 6)], [], "property"),
+    ([(3, 4, 9)], [], "property"),
     ([(3, 4, G), (5, 3, G)], [], "shape_mismatch"),
     ([(3, 4, G)], [(3, 5, G)], "shape_mismatch"),
 ])

@@ -26,8 +26,11 @@ from typing import List, Optional, Sequence
 import numpy as np
 
 GENERAL, LOWER_TRI, UPPER_TRI, IDENTITY, DIAGONAL, SYMMETRIC = 0, 1, 2, 3, 4, 5
+STRICT_LOWER, STRICT_UPPER, UNIT_LOWER, UNIT_UPPER = 6, 7, 8, 9
 PROPERTY_NAMES = {GENERAL: "general", LOWER_TRI: "lowerTri", UPPER_TRI: "upperTri", IDENTITY: "Identity",
-                  DIAGONAL: "diagonal", SYMMETRIC: "symmetric"}
+                  DIAGONAL: "diagonal", SYMMETRIC: "symmetric", STRICT_LOWER: "strictLowerTri",
+                  STRICT_UPPER: "strictUpperTri", UNIT_LOWER: "unitLowerTri", UNIT_UPPER: "unitUpperTri"}
+_TRIANGLE_KINDS = (STRICT_LOWER, STRICT_UPPER, UNIT_LOWER, UNIT_UPPER)
 
 
 @dataclass(frozen=True)
@@ -97,6 +100,17 @@ def generate_operand(op: Operand, seed: int, index: int, batch: int = 1) -> Opti
         keep = (np.tril(np.ones((n, n), dtype=bool)) if op.prop == LOWER_TRI else
                 np.triu(np.ones((n, n), dtype=bool)) if op.prop == UPPER_TRI else np.eye(n, dtype=bool))
         m = np.where(keep, m, np.float32(0.0)).astype(np.float32)
+    if op.prop in _TRIANGLE_KINDS:
+        # strictly triangular: zeros on the diagonal; unit triangular: ones there, stored as 1.0
+        if op.rows != op.cols:
+            raise ValueError("triangular operands are square")
+        n = op.rows
+        lower = op.prop in (STRICT_LOWER, UNIT_LOWER)
+        keep = np.tril(np.ones((n, n), dtype=bool), -1) if lower else np.triu(np.ones((n, n), dtype=bool), 1)
+        m = np.where(keep, m, np.float32(0.0)).astype(np.float32)
+        if op.prop in (UNIT_LOWER, UNIT_UPPER):
+            idx = np.arange(n)
+            m[..., idx, idx] = np.float32(1.0)
     if op.prop == SYMMETRIC:
         if op.rows != op.cols:
             raise ValueError("symmetric operands are square")
@@ -194,20 +208,24 @@ def config_listing2() -> Equation:
 
 
 def random_equation(seed: int, max_len: int = 6, max_dim: int = 96, allow_add: bool = True,
-                    dim_multiple: int = 1, diagonal: bool = False) -> Equation:
+                    dim_multiple: int = 1, diagonal: bool = False, kinds: bool = False) -> Equation:
     """A random well-formed equation (for property tests): random length, dims, properties.
 
     Triangular / Identity operands are only placed where the neighbouring dimensions are equal,
     which the generator arranges by repeating a dimension.  With `diagonal` about a quarter of the
-    operands and Add terms are Diagonal (the streams without it are unchanged).
+    operands and Add terms are Diagonal (the streams without it are unchanged).  With `kinds` a third of them
+    are strictly or unit triangular (a stream of its own, Diagonal included).
     """
-    rng = np.random.Generator(np.random.Philox(key=[int(seed), 0xD1A6 if diagonal else 0xC0FFEE]))
+    diagonal = diagonal or kinds
+    rng = np.random.Generator(np.random.Philox(key=[int(seed), 0x7D1A6 if kinds else 0xD1A6 if diagonal else 0xC0FFEE]))
     n = int(rng.integers(1, max_len + 1))
     chain: List[Operand] = []
     cur = int(rng.integers(1, max_dim // dim_multiple + 1)) * dim_multiple
     for _ in range(n):
-        kind = int(rng.integers(0, 8 if diagonal else 6))
-        if kind >= 6:
+        kind = int(rng.integers(0, 12 if kinds else 8 if diagonal else 6))
+        if kind >= 8:
+            chain.append(Operand(cur, cur, _TRIANGLE_KINDS[kind - 8]))
+        elif kind >= 6:
             chain.append(Operand(cur, cur, DIAGONAL))
         elif kind == 0:
             chain.append(Operand(cur, cur, LOWER_TRI))
@@ -223,8 +241,10 @@ def random_equation(seed: int, max_len: int = 6, max_dim: int = 96, allow_add: b
     add: List[Operand] = []
     if allow_add:
         for _ in range(int(rng.integers(0, 3))):
-            kind = int(rng.integers(0, 7 if diagonal else 5))
-            if rows == cols and kind >= 5:
+            kind = int(rng.integers(0, 11 if kinds else 7 if diagonal else 5))
+            if rows == cols and kind >= 7:
+                add.append(Operand(rows, cols, _TRIANGLE_KINDS[kind - 7]))
+            elif rows == cols and kind >= 5:
                 add.append(Operand(rows, cols, DIAGONAL))
             elif rows == cols and kind == 0:
                 add.append(Operand(rows, cols, LOWER_TRI))
@@ -278,11 +298,14 @@ def generate_sum(eq: SumEquation):
 
 
 def random_sum_equation(seed: int, max_chains: int = 4, max_len: int = 5, max_dim: int = 48,
-                        dim_multiple: int = 1, share: float = 0.5, diagonal: bool = False) -> SumEquation:
+                        dim_multiple: int = 1, share: float = 0.5, diagonal: bool = False,
+                        kinds: bool = False) -> SumEquation:
     """Random well-formed sum of chains.  With probability `share`/2 a chain starts with a run of factors
     copied (same names and flags) from an earlier chain, so that shared products occur.  With `diagonal`
-    some square factors are Diagonal (the streams without it are unchanged)."""
-    rng = np.random.Generator(np.random.Philox(key=[int(seed), 0x5D1A6 if diagonal else 0x5EED5]))
+    some square factors are Diagonal (the streams without it are unchanged); with `kinds` some are strictly or
+    unit triangular as well (a stream of its own)."""
+    diagonal = diagonal or kinds
+    rng = np.random.Generator(np.random.Philox(key=[int(seed), 0x75D1A6 if kinds else 0x5D1A6 if diagonal else 0x5EED5]))
     rows = int(rng.integers(1, max_dim // dim_multiple + 1)) * dim_multiple
     cols = int(rng.integers(1, max_dim // dim_multiple + 1)) * dim_multiple
     if rng.random() < 0.4:
@@ -293,9 +316,11 @@ def random_sum_equation(seed: int, max_chains: int = 4, max_len: int = 5, max_di
     def new_factor(r, c):
         nonlocal next_name
         """One stored factor whose type AS USED is r x c, with a random property and transposition."""
-        kind = int(rng.integers(0, 9 if diagonal else 7))
+        kind = int(rng.integers(0, 13 if kinds else 9 if diagonal else 7))
         t = bool(rng.integers(0, 3) == 0)
-        if r == c and kind >= 7:
+        if r == c and kind >= 9:
+            o = Operand(r, r, _TRIANGLE_KINDS[kind - 9])
+        elif r == c and kind >= 7:
             o = Operand(r, r, DIAGONAL)
         elif r == c and kind == 0:
             o = Operand(r, r, LOWER_TRI)
@@ -425,10 +450,12 @@ def generate_expression(ex: Expression):
 
 
 def random_expression(seed: int, max_depth: int = 3, max_dim: int = 40, dim_multiple: int = 1,
-                      diagonal: bool = False) -> Expression:
+                      diagonal: bool = False, kinds: bool = False) -> Expression:
     """Random well-formed nested expression; operands are reused where an existing one has the needed type.
-    With `diagonal` some square operands are Diagonal (the streams without it are unchanged)."""
-    rng = np.random.Generator(np.random.Philox(key=[int(seed), 0xED1A6 if diagonal else 0xE4B8]))
+    With `diagonal` some square operands are Diagonal (the streams without it are unchanged); with `kinds` some
+    are strictly or unit triangular as well (a stream of its own)."""
+    diagonal = diagonal or kinds
+    rng = np.random.Generator(np.random.Philox(key=[int(seed), 0x7ED1A6 if kinds else 0xED1A6 if diagonal else 0xE4B8]))
     operands: List[Operand] = []
 
     def dim():
@@ -441,8 +468,9 @@ def random_expression(seed: int, max_depth: int = 3, max_dim: int = 40, dim_mult
         if same and rng.random() < 0.5:
             i = int(rng.choice(same))
         else:
-            kind = int(rng.integers(0, 9 if diagonal else 7))
-            prop = {0: LOWER_TRI, 1: UPPER_TRI, 2: IDENTITY, 7: DIAGONAL, 8: DIAGONAL}.get(kind, GENERAL) if sr == sc else GENERAL
+            kind = int(rng.integers(0, 13 if kinds else 9 if diagonal else 7))
+            prop = {0: LOWER_TRI, 1: UPPER_TRI, 2: IDENTITY, 7: DIAGONAL, 8: DIAGONAL, 9: STRICT_LOWER, 10: STRICT_UPPER,
+                    11: UNIT_LOWER, 12: UNIT_UPPER}.get(kind, GENERAL) if sr == sc else GENERAL
             operands.append(Operand(sr, sc, prop, "normal" if kind == 3 else "uniform"))
             i = len(operands) - 1
         return ("t", i) if t else i
