@@ -68,8 +68,19 @@ typedef enum {
  * (mom_equation_plan_sum with names, mom_expression_plan), a sub-chain that reads Y * Y^T factor by factor
  * is typed Symmetric, and the tree that splits it in the middle computes Y once and then only the lower
  * triangle of Y * Y^T (MOM_KIND_GRAM): the right half is never multiplied.  A computed Symmetric value is
- * symmetric up to rounding in its diagonal blocks and exactly symmetric elsewhere (mirrored). */
-typedef enum { MOM_GENERAL = 0, MOM_LOWER_TRI = 1, MOM_UPPER_TRI = 2, MOM_IDENTITY = 3, MOM_DIAGONAL = 4, MOM_SYMMETRIC = 5 } mom_property_t;
+ * symmetric up to rounding in its diagonal blocks and exactly symmetric elsewhere (mirrored).
+ * MOM_STRICT_LOWER / MOM_STRICT_UPPER and MOM_UNIT_LOWER / MOM_UNIT_UPPER are two more such properties: square
+ * triangular matrices, stored densely, whose diagonal holds zeros (strict) or ones (unit; stored as 1.0f, the
+ * library relies on that and does not check it).  An entry known to be 1 needs no multiplication, as with
+ * Identity: a multiplication counts only when both entries are structural non-zeros and neither is a known 1,
+ * so a unit triangle costs what the strict one costs.  Within one orientation the diagonal of a product is the
+ * product of the diagonals (strict if either factor is strict, unit if both are unit); in a sum the diagonals add
+ * (strict + strict = strict, strict + unit or Identity = unit, anything else an ordinary triangle); the transpose
+ * swaps lower and upper and keeps the kind.  The kernels treat them as the enclosing ordinary triangle: a strict
+ * result's diagonal is computed as a sum of products with an exact zero factor (+0 for finite inputs), a unit
+ * result's diagonal as 1*1 plus such zeros (exactly 1). */
+typedef enum { MOM_GENERAL = 0, MOM_LOWER_TRI = 1, MOM_UPPER_TRI = 2, MOM_IDENTITY = 3, MOM_DIAGONAL = 4, MOM_SYMMETRIC = 5,
+               MOM_STRICT_LOWER = 6, MOM_STRICT_UPPER = 7, MOM_UNIT_LOWER = 8, MOM_UNIT_UPPER = 9 } mom_property_t;
 typedef enum { MOM_F32 = 0 } mom_dtype_t;
 
 /* Arithmetic used by the product kernels.

@@ -38,14 +38,15 @@ constexpr int TIMING_SLOTS = 32;
 // host-staging entry point: triangular operands of at least UPLOAD_MIN rows are uploaded in blocks of UPLOAD_BLOCK rows
 constexpr int64_t UPLOAD_BLOCK = 256, UPLOAD_MIN = 1024;
 inline bool triangular_upload(const mom_matrix_desc_t &d, int64_t batch) {
-    return batch == 1 && d.rows >= UPLOAD_MIN && (d.property == MOM_LOWER_TRI || d.property == MOM_UPPER_TRI);
+    const int32_t kp = kernel_property(d.property);        // strict and unit triangles lie inside the ordinary one
+    return batch == 1 && d.rows >= UPLOAD_MIN && (kp == MOM_LOWER_TRI || kp == MOM_UPPER_TRI);
 }
 inline size_t upload_bytes(const mom_matrix_desc_t &d, int64_t batch) {
     if (!triangular_upload(d, batch)) return (size_t)d.rows * d.cols * sizeof(float) * batch;
     size_t total = 0;
     for (int64_t r0 = 0; r0 < d.rows; r0 += UPLOAD_BLOCK) {
         const int64_t r1 = std::min<int64_t>(d.rows, r0 + UPLOAD_BLOCK);
-        total += (size_t)(r1 - r0) * (size_t)(d.property == MOM_LOWER_TRI ? r1 : d.rows - r0) * sizeof(float);
+        total += (size_t)(r1 - r0) * (size_t)(kernel_property(d.property) == MOM_LOWER_TRI ? r1 : d.rows - r0) * sizeof(float);
     }
     return total;
 }
@@ -187,7 +188,7 @@ mom_status_t execute_impl(const mom_plan *p, const float *const *chain_ptrs, con
                 const int id = p->kept[i];
                 if (p->chain_t[id] || p->chain[id].cols % 4 != 0) continue;
                 dev->fused_tab_begin[i] = (int)(table.size() / FUSED_THREADS);
-                dev->fused_tab_end[i] = dev->fused_tab_begin[i] + fused_copy_table((int)p->chain[id].rows, (int)p->chain[id].cols, p->chain[id].property,
+                dev->fused_tab_end[i] = dev->fused_tab_begin[i] + fused_copy_table((int)p->chain[id].rows, (int)p->chain[id].cols, kernel_property(p->chain[id].property),
                                                                                     p->fused_value_off[id], p->fused_value_ld[id], table);
             }
             if (!table.empty()) {
@@ -199,7 +200,7 @@ mom_status_t execute_impl(const mom_plan *p, const float *const *chain_ptrs, con
         for (int i = 0; i < fp.n_ops; ++i) {
             const int id = p->kept[i], slot = p->factor_ptr[id];
             fp.ops[i] = FusedOperand{chain_ptrs[slot], chain_strides ? chain_strides[slot] : 0, (int)p->chain[id].rows,
-                                     (int)p->chain[id].cols, p->chain[id].property, p->fused_value_off[id], p->fused_value_ld[id],
+                                     (int)p->chain[id].cols, kernel_property(p->chain[id].property), p->fused_value_off[id], p->fused_value_ld[id],
                                      (int)p->chain_t[id], dev->fused_tab_begin[i], dev->fused_tab_end[i]};
         }
         fp.n_steps = (int)p->steps.size();
@@ -207,8 +208,8 @@ mom_status_t execute_impl(const mom_plan *p, const float *const *chain_ptrs, con
             const StepImpl &stp = p->steps[s];
             fp.steps[s] = FusedStep{p->fused_value_off[stp.pub.lhs], p->fused_value_off[stp.pub.rhs],
                                     stp.is_last ? -1 : p->fused_value_off[stp.pub.out], (int)stp.pub.m, (int)stp.pub.n,
-                                    (int)stp.pub.k, stp.pub.lhs_property, stp.pub.rhs_property,
-                                    stp.is_last ? p->result_desc.property : stp.pub.out_property,
+                                    (int)stp.pub.k, kernel_property(stp.pub.lhs_property), kernel_property(stp.pub.rhs_property),
+                                    kernel_property(stp.is_last ? p->result_desc.property : stp.pub.out_property),
                                     p->fused_value_ld[stp.pub.lhs], p->fused_value_ld[stp.pub.rhs],
                                     stp.is_last ? 0 : p->fused_value_ld[stp.pub.out]};
         }
@@ -310,13 +311,13 @@ mom_status_t execute_impl(const mom_plan *p, const float *const *chain_ptrs, con
                 added = add_terms(1, &t);
                 cudaError_t e;
                 if (is_identity(sm)) {
-                    e = launch_elementwise(nullptr, 0, 1, x, x_stride, srows, scols, sum.desc.property, t, nb, stream);
+                    e = launch_elementwise(nullptr, 0, 1, x, x_stride, srows, scols, kernel_property(sum.desc.property), t, nb, stream);
                 } else if (sm.kind == SUM_FACTOR) {
                     const Operand src = chain_op(sm.index);
-                    e = launch_elementwise(src.ptr, src.stride, p->chain_t[sm.index] ? 3 : 0, x, x_stride, srows, scols, sum.desc.property, t, nb, stream);
+                    e = launch_elementwise(src.ptr, src.stride, p->chain_t[sm.index] ? 3 : 0, x, x_stride, srows, scols, kernel_property(sum.desc.property), t, nb, stream);
                 } else {
                     const long long ss = add_strides ? add_strides[sm.index] : 0;
-                    e = launch_elementwise(add_ptrs[sm.index] + b0 * ss, ss, p->add_t[sm.index] ? 3 : 0, x, x_stride, srows, scols, sum.desc.property, t, nb, stream);
+                    e = launch_elementwise(add_ptrs[sm.index] + b0 * ss, ss, p->add_t[sm.index] ? 3 : 0, x, x_stride, srows, scols, kernel_property(sum.desc.property), t, nb, stream);
                 }
                 if (e != cudaSuccess) return MOM_ERR_CUDA;
                 ++launches;
@@ -344,7 +345,7 @@ mom_status_t execute_impl(const mom_plan *p, const float *const *chain_ptrs, con
                 ProductArgs a;
                 std::memset(&a, 0, sizeof(a));
                 a.m = (int)stp.pub.m; a.n = (int)stp.pub.n; a.k = (int)stp.pub.k;
-                a.pa = stp.pub.lhs_property; a.pb = stp.pub.rhs_property;
+                a.pa = kernel_property(stp.pub.lhs_property); a.pb = kernel_property(stp.pub.rhs_property);
                 // an operand: the value itself, or d * S / S * d of a folded scaling step (S read as stored, d handed
                 // to the split pass)
                 auto operand = [&](int id, int fold, const float **ptr, long long *stride, int *trans, int own_trans,
@@ -370,7 +371,7 @@ mom_status_t execute_impl(const mom_plan *p, const float *const *chain_ptrs, con
                 if (stp.is_last && stp.accumulate) {
                     // a later chain's product is added to what the earlier ones left in the sum's buffer
                     a.C = x; a.strideC = x_stride;
-                    a.pout = sum.desc.property;
+                    a.pout = kernel_property(sum.desc.property);
                     a.add.count = 1;
                     a.add.ptr[0] = x;
                     a.add.stride[0] = x_stride;
@@ -379,12 +380,12 @@ mom_status_t execute_impl(const mom_plan *p, const float *const *chain_ptrs, con
                     a.add.rows = srows;
                 } else if (stp.is_last) {
                     a.C = x; a.strideC = x_stride;
-                    a.pout = sum.desc.property;
+                    a.pout = kernel_property(sum.desc.property);
                     added = add_terms(0, &a.add);
                 } else {
                     a.C = stp.out_off == SIZE_MAX ? nullptr : reinterpret_cast<float *>(ws + stp.out_off * (size_t)nb);
                     a.strideC = (long long)stp.pub.m * stp.pub.n;
-                    a.pout = stp.pub.out_property;
+                    a.pout = kernel_property(stp.pub.out_property);
                     a.add.count = 0;
                     a.add.transposed = 0;
                     a.add.aliases_out = 0;
@@ -426,7 +427,7 @@ mom_status_t execute_impl(const mom_plan *p, const float *const *chain_ptrs, con
                 AddTerms t;
                 const int first = added;
                 added = add_terms(first, &t);
-                if (launch_elementwise(nullptr, 0, 2, x, x_stride, srows, scols, sum.desc.property, t, nb, stream) != cudaSuccess)
+                if (launch_elementwise(nullptr, 0, 2, x, x_stride, srows, scols, kernel_property(sum.desc.property), t, nb, stream) != cudaSuccess)
                     return MOM_ERR_CUDA;
                 ++launches;
             }
@@ -538,7 +539,8 @@ mom_status_t mom_equation_execute_host(const mom_plan_t *plan, const float *cons
             if (cudaMemsetAsync(dst, 0, cbytes[i], dev->copy_stream) != cudaSuccess) return MOM_ERR_CUDA;
             for (int64_t r0 = 0; r0 < n; r0 += mom::UPLOAD_BLOCK) {
                 const int64_t r1 = std::min(n, r0 + mom::UPLOAD_BLOCK);
-                const int64_t c0 = d.property == MOM_LOWER_TRI ? 0 : r0, c1 = d.property == MOM_LOWER_TRI ? r1 : n;
+                const bool lower = mom::kernel_property(d.property) == MOM_LOWER_TRI;
+                const int64_t c0 = lower ? 0 : r0, c1 = lower ? r1 : n;
                 if (cudaMemcpy2DAsync(dst + r0 * n + c0, (size_t)n * sizeof(float), chain_host[i] + r0 * n + c0, (size_t)n * sizeof(float),
                                       (size_t)(c1 - c0) * sizeof(float), (size_t)(r1 - r0), cudaMemcpyHostToDevice, dev->copy_stream) != cudaSuccess)
                     return MOM_ERR_CUDA;

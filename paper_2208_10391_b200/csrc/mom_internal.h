@@ -27,6 +27,27 @@ constexpr size_t WS_ALIGN = 256;
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
+// Type of A^T: lower and upper swap (the inference rule of the paper's Section 2), the kind of diagonal stays.
+inline int32_t transpose_property(int32_t p) {
+    switch (p) {
+        case MOM_LOWER_TRI: return MOM_UPPER_TRI;
+        case MOM_UPPER_TRI: return MOM_LOWER_TRI;
+        case MOM_STRICT_LOWER: return MOM_STRICT_UPPER;
+        case MOM_STRICT_UPPER: return MOM_STRICT_LOWER;
+        case MOM_UNIT_LOWER: return MOM_UNIT_UPPER;
+        case MOM_UNIT_UPPER: return MOM_UNIT_LOWER;
+        default: return p;
+    }
+}
+
+// The structure the kernels work with: a strict or unit triangle is handled as the ordinary triangle around it
+// (its diagonal holds stored zeros or ones; products with them give exact zeros and ones).
+inline int32_t kernel_property(int32_t p) {
+    if (p == MOM_STRICT_LOWER || p == MOM_UNIT_LOWER) return MOM_LOWER_TRI;
+    if (p == MOM_STRICT_UPPER || p == MOM_UNIT_UPPER) return MOM_UPPER_TRI;
+    return p;
+}
+
 struct StepImpl {
     mom_step_t pub;
     bool is_last = false;           // root of its chain's tree: writes X (the first root also carries the Add terms)

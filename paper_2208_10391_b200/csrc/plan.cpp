@@ -17,50 +17,83 @@ namespace {
 using u128 = unsigned __int128;
 constexpr uint64_t COST_LIMIT = (uint64_t)1 << 63;
 
-bool is_tri(int32_t p) { return p == MOM_LOWER_TRI || p == MOM_UPPER_TRI; }
+bool is_lower(int32_t p) { return p == MOM_LOWER_TRI || p == MOM_STRICT_LOWER || p == MOM_UNIT_LOWER; }
+bool is_upper(int32_t p) { return p == MOM_UPPER_TRI || p == MOM_STRICT_UPPER || p == MOM_UNIT_UPPER; }
+bool is_tri(int32_t p) { return is_lower(p) || is_upper(p); }
+
+// What a type states about its diagonal.
+enum Diag { DIAG_DATA = 0, DIAG_ZERO = 1, DIAG_ONE = 2 };
+Diag diag_of(int32_t p) {
+    if (p == MOM_STRICT_LOWER || p == MOM_STRICT_UPPER) return DIAG_ZERO;
+    if (p == MOM_UNIT_LOWER || p == MOM_UNIT_UPPER || p == MOM_IDENTITY) return DIAG_ONE;
+    return DIAG_DATA;
+}
+int32_t triangle(bool lower, Diag d) {
+    if (d == DIAG_ZERO) return lower ? MOM_STRICT_LOWER : MOM_STRICT_UPPER;
+    if (d == DIAG_ONE) return lower ? MOM_UNIT_LOWER : MOM_UNIT_UPPER;
+    return lower ? MOM_LOWER_TRI : MOM_UPPER_TRI;
+}
 
 // Least upper bound in  Identity < Diagonal < {lowerTri, upperTri} < general  (paper Listing 3 types L*L as lowerTri).
+// Inside one orientation the product's diagonal is the entrywise product of the factors' diagonals.
 int32_t join_property(int32_t p, int32_t q) {
     if (p == MOM_IDENTITY) return q;
     if (q == MOM_IDENTITY) return p;
     if (p == MOM_SYMMETRIC || q == MOM_SYMMETRIC) return (int32_t)MOM_GENERAL;   // S*S, D*S, ... are not symmetric in general
-    if (p == q) return p;
-    if (p == MOM_DIAGONAL) return q;
-    if (q == MOM_DIAGONAL) return p;
-    return (int32_t)MOM_GENERAL;
+    if (p == MOM_GENERAL || q == MOM_GENERAL) return (int32_t)MOM_GENERAL;
+    if (p == MOM_DIAGONAL && q == MOM_DIAGONAL) return (int32_t)MOM_DIAGONAL;
+    const bool lower = is_lower(p) || is_lower(q), upper = is_upper(p) || is_upper(q);
+    if (lower && upper) return (int32_t)MOM_GENERAL;
+    const Diag dp = diag_of(p), dq = diag_of(q);
+    return triangle(lower, dp == DIAG_ZERO || dq == DIAG_ZERO ? DIAG_ZERO : dp == DIAG_ONE && dq == DIAG_ONE ? DIAG_ONE : DIAG_DATA);
 }
 
-// structural non-zeros of an r x c matrix with property p (triangular, Diagonal and Identity are square)
+// structural non-zeros of an r x c matrix with property p (every property but general is square)
 unsigned __int128 structural_entries(int32_t p, int64_t r, int64_t c) {
     const unsigned __int128 R = (unsigned __int128)r, C = (unsigned __int128)c;
     if (p == MOM_GENERAL || p == MOM_SYMMETRIC) return R * C;
-    if (p == MOM_LOWER_TRI || p == MOM_UPPER_TRI) return R * (R + 1) / 2;
+    if (diag_of(p) == DIAG_ZERO) return R * (R - 1) / 2;
+    if (is_tri(p)) return R * (R + 1) / 2;
     return R;
+}
+
+// of those, the entries that are not known to be 1 (the ones a multiplication needs)
+unsigned __int128 multiplying_entries(int32_t p, int64_t r, int64_t c) {
+    if (p == MOM_IDENTITY) return 0;
+    if (p == MOM_UNIT_LOWER || p == MOM_UNIT_UPPER) return (unsigned __int128)r * (unsigned __int128)(r - 1) / 2;
+    return structural_entries(p, r, c);
 }
 
 // Multiplications of the lower triangle (i >= j) of Y * Y^T, Y m x k: k m(m+1)/2 for a full Y, n(n+1)(n+2)/6 for a
 // triangular one.  Returns false on overflow.
 bool gram_mults(int32_t py, int64_t m, int64_t k, uint64_t *out);
 
-// Scalar multiplications a_il * b_lj of an (m x k)(k x n) product in which both factors are
-// structurally non-zero.  Triangular operands are square.  Returns false on overflow.
+// Scalar multiplications a_il * b_lj of an (m x k)(k x n) product in which both factors are structurally
+// non-zero and neither is known to be 1.  Triangular operands are square.  Returns false on overflow.
 bool useful_mults(int32_t pa, int32_t pb, int64_t m, int64_t k, int64_t n, uint64_t *out) {
     u128 v;
     const u128 M = (u128)m, K = (u128)k, N = (u128)n;
+    // a strict or unit triangle takes part with the entries off its diagonal only: e of its K diagonal entries drop out
+    const u128 ea = pa == MOM_LOWER_TRI || pa == MOM_UPPER_TRI ? 0 : 1, eb = pb == MOM_LOWER_TRI || pb == MOM_UPPER_TRI ? 0 : 1;
     if (pa == MOM_DIAGONAL) {
-        v = structural_entries(pb, k, n);          // D*B scales the rows of B: one multiplication per entry of B
+        v = multiplying_entries(pb, k, n);         // D*B scales the rows of B: one multiplication per entry of B
     } else if (pb == MOM_DIAGONAL) {
-        v = structural_entries(pa, m, k);          // A*D scales the columns of A
+        v = multiplying_entries(pa, m, k);         // A*D scales the columns of A
     } else if (!is_tri(pa) && !is_tri(pb)) {
         v = M * K * N;
     } else if (is_tri(pa) && !is_tri(pb)) {
-        v = N * (K * (K + 1) / 2);                 // row i of A has i+1 (or k-i) non-zeros
+        v = N * (K * (K + 1) / 2 - ea * K);        // row i of A has i+1 (or k-i) non-zeros, one fewer without the diagonal
     } else if (!is_tri(pa) && is_tri(pb)) {
-        v = M * (K * (K + 1) / 2);
-    } else if (pa == pb) {
-        v = K * (K + 1) * (K + 2) / 6;             // sum_l (l+1)(k-l) over the shared triangle
+        v = M * (K * (K + 1) / 2 - eb * K);
+    } else if (is_lower(pa) == is_lower(pb)) {
+        // sum_l (k - l - ea)(l + 1 - eb), l = 0..k-1; with ea = eb = 0 this is k(k+1)(k+2)/6
+        const u128 s1 = K * (K - 1) / 2, s2 = (K - 1) * K * (2 * K - 1) / 6;        // sum of l and of l^2
+        // (K - ea)(1 - eb) K + ((K - ea) - (1 - eb)) s1 - s2
+        const u128 c0 = K - ea, c1 = 1 - eb;
+        v = c0 * c1 * K + c0 * s1 - s2 - c1 * s1;
     } else {
-        v = K * (K + 1) * (2 * K + 1) / 6;         // sum_l (l+1)^2 : opposite triangles
+        // sum_t (t - ea)(t - eb), t = 1..k; with ea = eb = 0 the sum of squares k(k+1)(2k+1)/6
+        v = K * (K + 1) * (2 * K + 1) / 6 + ea * eb * K - (ea + eb) * (K * (K + 1) / 2);
     }
     if (v >= (u128)COST_LIMIT) return false;
     *out = (uint64_t)v;
@@ -69,7 +102,9 @@ bool useful_mults(int32_t pa, int32_t pb, int64_t m, int64_t k, int64_t n, uint6
 
 bool gram_mults(int32_t py, int64_t m, int64_t k, uint64_t *out) {
     const u128 M = (u128)m, K = (u128)k;
-    const u128 v = is_tri(py) ? M * (M + 1) * (M + 2) / 6 : K * (M * (M + 1) / 2);
+    // triangular Y: triples i >= j >= l (lower) of a shared column l; without the diagonal i >= j > l
+    const u128 v = !is_tri(py) ? K * (M * (M + 1) / 2)
+                   : py == MOM_LOWER_TRI || py == MOM_UPPER_TRI ? M * (M + 1) * (M + 2) / 6 : (M + 1) * M * (M - 1) / 6;
     if (v >= (u128)COST_LIMIT) return false;
     *out = (uint64_t)v;
     return true;
@@ -77,7 +112,7 @@ bool gram_mults(int32_t py, int64_t m, int64_t k, uint64_t *out) {
 
 mom_status_t check_desc(const mom_matrix_desc_t &d) {
     if (d.rows < 1 || d.cols < 1) return MOM_ERR_INVALID_ARG;
-    if (d.property < MOM_GENERAL || d.property > MOM_SYMMETRIC) return MOM_ERR_INVALID_ARG;
+    if (d.property < MOM_GENERAL || d.property > MOM_UNIT_UPPER) return MOM_ERR_INVALID_ARG;
     if (d.dtype != MOM_F32) return MOM_ERR_DTYPE;
     if (d.property != MOM_GENERAL && d.rows != d.cols) return MOM_ERR_PROPERTY;
     return MOM_OK;
@@ -95,9 +130,18 @@ int32_t sum_property(const std::vector<int32_t> &props) {
         only_symmetric_like &= p == MOM_SYMMETRIC || p == MOM_DIAGONAL || p == MOM_IDENTITY;
     }
     if (any_symmetric) return only_symmetric_like ? (int32_t)MOM_SYMMETRIC : (int32_t)MOM_GENERAL;
-    int32_t acc = MOM_DIAGONAL;
-    for (int32_t p : props) acc = join_property(acc, p == MOM_IDENTITY ? (int32_t)MOM_DIAGONAL : p);
-    return acc;
+    bool lower = false, upper = false;
+    Diag d = DIAG_ZERO;                             // the diagonals add up: 0 + x = x, anything else is data
+    for (int32_t p : props) {
+        if (p == MOM_GENERAL) return (int32_t)MOM_GENERAL;
+        lower |= is_lower(p);
+        upper |= is_upper(p);
+        const Diag dp = diag_of(p);
+        d = d == DIAG_ZERO ? dp : dp == DIAG_ZERO ? d : DIAG_DATA;
+    }
+    if (lower && upper) return (int32_t)MOM_GENERAL;
+    if (!lower && !upper) return (int32_t)MOM_DIAGONAL;
+    return triangle(lower, d);
 }
 
 struct Node { int64_t rows, cols; int32_t prop; };
@@ -185,9 +229,7 @@ static mom_status_t plan_sums(const std::vector<mom_matrix_desc_t> &slots, const
     // (the inference rule of the paper's Section 2); `chain` / `add_terms` hold the types as used.
     auto as_used = [](const mom_matrix_desc_t &d, bool t) {
         if (!t) return d;
-        const int32_t prop = d.property == MOM_LOWER_TRI ? (int32_t)MOM_UPPER_TRI
-                             : d.property == MOM_UPPER_TRI ? (int32_t)MOM_LOWER_TRI : d.property;
-        return mom_matrix_desc_t{d.cols, d.rows, prop, d.dtype};
+        return mom_matrix_desc_t{d.cols, d.rows, mom::transpose_property(d.property), d.dtype};
     };
     if (slot_names) {                                       // one name, one stored type
         try {
@@ -403,8 +445,7 @@ static mom_status_t plan_sums(const std::vector<mom_matrix_desc_t> &slots, const
                             st.pub.m = a.rows; st.pub.k = a.cols;
                             if (is_gram) {
                                 // Y * Y^T: the right operand is the left one read transposed
-                                st.pub.rhs_property = a.prop == MOM_LOWER_TRI ? (int32_t)MOM_UPPER_TRI
-                                                      : a.prop == MOM_UPPER_TRI ? (int32_t)MOM_LOWER_TRI : a.prop;
+                                st.pub.rhs_property = mom::transpose_property(a.prop);
                                 st.pub.rhs_transposed = l < n_factors ? !p->chain_t[l] : 1;
                                 st.pub.n = a.rows;
                                 gram_mults(a.prop, a.rows, a.cols, &st.pub.useful_mults);
@@ -417,7 +458,7 @@ static mom_status_t plan_sums(const std::vector<mom_matrix_desc_t> &slots, const
                                 const bool ta = is_tri(a.prop), tb = is_tri(b.prop);
                                 st.pub.kind = a.prop == MOM_DIAGONAL || b.prop == MOM_DIAGONAL ? MOM_KIND_SCALE
                                               : !ta && !tb ? MOM_KIND_GG : ta && !tb ? MOM_KIND_TG : !ta && tb ? MOM_KIND_GT
-                                              : a.prop == b.prop ? MOM_KIND_TT : MOM_KIND_TTMIX;
+                                              : is_lower(a.prop) == is_lower(b.prop) ? MOM_KIND_TT : MOM_KIND_TTMIX;
                             }
                             st.is_last = root;
                             if (root) st.sum = sum_index;

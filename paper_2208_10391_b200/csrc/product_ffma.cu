@@ -349,7 +349,9 @@ scale_kernel(ProductArgs a) {
             if (r >= m) continue;
             float v[4];
 #pragma unroll
-            for (int j = 0; j < 4; ++j) v[j] = (left ? dr[i] : dc[j]) * s[i][j];
+            // (+ 0.0f: a product with a stored zero is +0 whatever the sign of d, so the diagonal of a strictly
+            // triangular result holds +0.0f like every entry outside a structure)
+            for (int j = 0; j < 4; ++j) v[j] = fmaf(left ? dr[i] : dc[j], s[i][j], 0.0f);
             finish_row4(v, a.add, inst, r, c, n, n, a.pout, (n & 3) == 0);
             float *p = C + (long long)r * n + c;
             if (vec) {

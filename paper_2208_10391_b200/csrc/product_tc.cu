@@ -740,7 +740,7 @@ mom_status_t tc_prepare(const mom_plan &p, TcPlanState &s) {
             for (int c0 = 0; c0 < n; c0 += BN) {
                 if (s.steps[i].mirror && c0 > r0) continue;
                 int klo, khi;
-                tile_k_range(st.lhs_property, st.rhs_property, r0, std::min(r0 + tile_rows, m), c0, std::min(c0 + BN, n), k, &klo, &khi);
+                tile_k_range(kernel_property(st.lhs_property), kernel_property(st.rhs_property), r0, std::min(r0 + tile_rows, m), c0, std::min(c0 + BN, n), k, &klo, &khi);
                 if (klo >= khi) { klo = 0; khi = 0; }
                 klo = klo / BK * BK;                      // leading extra elements are stored zeros
                 if (split <= 1) {

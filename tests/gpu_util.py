@@ -88,6 +88,7 @@ def check_against_oracle(eq: wl.Equation, x: np.ndarray, plan, chain, add, rows=
         # entries outside the result's structure: exactly +0.0f (all 32 bits clear)
         mask = ov.off_structure_mask(xb.shape[0], xb.shape[1], prop)
         assert np.all(xb.view(np.uint32)[mask] == 0), "off-structure entries must be +0.0f"
+        assert ov.unit_diagonal_exactly_one(xb, prop), "the diagonal of a unit triangular result must be exactly 1"
     return worst
 
 
@@ -142,6 +143,7 @@ def check_sum_against_oracle(eq: wl.SumEquation, x: np.ndarray, plan, arrays, us
     assert err <= tol, f"normwise error {err:.3e} > {tol:.1e} ({eq.name})"
     mask = ov.off_structure_mask(x.shape[0], x.shape[1], prop)
     assert np.all(x.view(np.uint32)[mask] == 0), "off-structure entries must be +0.0f"
+    assert ov.unit_diagonal_exactly_one(x, prop), "the diagonal of a unit triangular result must be exactly 1"
     return err
 
 
@@ -192,4 +194,5 @@ def check_expression_against_oracle(ex: wl.Expression, x: np.ndarray, plan, arra
     assert err <= tol, f"normwise error {err:.3e} > {tol:.1e} ({ex.name})"
     mask = ov.off_structure_mask(x.shape[0], x.shape[1], prop)
     assert np.all(x.view(np.uint32)[mask] == 0), "off-structure entries must be +0.0f"
+    assert ov.unit_diagonal_exactly_one(x, prop), "the diagonal of a unit triangular result must be exactly 1"
     return err

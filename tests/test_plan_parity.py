@@ -69,6 +69,30 @@ def test_random_equations_with_diagonal_operands_match_the_oracle():
         assert_same_plan(chain, add)
 
 
+def test_random_equations_with_strict_and_unit_triangles_match_the_oracle():
+    for seed in range(300):
+        eq = wl.random_equation(seed, max_len=9, max_dim=50, kinds=True)
+        assert_same_plan(eq.descs(), eq.add_descs())
+    # equal dimensions, every property: ties and every pair of types in the cost and type rules
+    rng = np.random.default_rng(6)
+    for _ in range(150):
+        chain = [(9, 9, int(rng.integers(0, 10))) for _ in range(int(rng.integers(1, 8)))]
+        add = [(9, 9, int(rng.integers(0, 10))) for _ in range(int(rng.integers(0, 4)))]
+        assert_same_plan(chain, add)
+    for pa in range(10):                                             # each pair, on its own and transposed
+        for pb in range(10):
+            assert_same_plan([(7, 7, pa), (7, 7, pb)])
+            assert_same_plan([(7, 7, pa)], [(7, 7, pb)])
+            assert_same_sum_plan([[(7, 7, pa), (7, 7, pb)]], [[True, False]], None)
+            assert_same_sum_plan([[(7, 7, pa), (7, 7, pb), (7, 7, pb), (7, 7, pa)]], [[False, False, True, True]], [[0, 1, 1, 0]])
+    for seed in range(150):
+        eq = wl.random_sum_equation(seed, kinds=True)
+        assert_same_sum_plan(eq.descs(), eq.transposed, eq.names)
+    for seed in range(150):
+        ex = wl.random_expression(seed, kinds=True)
+        assert_same_expression_plan(ex.expr, ex.descs())
+
+
 def test_long_chains_with_many_ties():
     # equal dimensions everywhere: every tree of an all-general chain ties; mixed properties tie partially
     rng = np.random.default_rng(3)
@@ -92,7 +116,9 @@ def test_identity_only_and_single_operand():
     ([(3, 4, 3)], [], mom.ERR_PROPERTY, "property"),
     ([(3, 4, 4)], [], mom.ERR_PROPERTY, "property"),
     ([(3, 4, 5)], [], mom.ERR_PROPERTY, "property"),
-    ([(3, 3, 0)], [(3, 3, 6)], mom.ERR_INVALID_ARG, "property"),
+    ([(3, 3, 0)], [(3, 3, 10)], mom.ERR_INVALID_ARG, "property"),
+    ([(3, 4, 6)], [], mom.ERR_PROPERTY, "property"),
+    ([(3, 4, 9)], [], mom.ERR_PROPERTY, "property"),
     ([(3, 4, 0), (5, 3, 0)], [], mom.ERR_SHAPE_MISMATCH, "shape_mismatch"),
     ([(3, 4, 0)], [(3, 5, 0)], mom.ERR_SHAPE_MISMATCH, "shape_mismatch"),
 ])
