@@ -137,6 +137,27 @@ typedef struct CUstream_st *mom_stream_t;    /* a CUDA stream handle (cudaStream
 mom_status_t mom_matrix_desc(int64_t rows, int64_t cols, mom_property_t property, mom_dtype_t dtype,
                              mom_matrix_desc_t *out /* host */);
 
+/* Column-slab split of one equation over `world` devices (paper Section 5 names non-rectangular iteration spaces and
+ * other containers as future work; this is the data-parallel split that needs neither).  Column j of
+ * X = M1*...*Mn + T1 + ... + Tk depends on column j of Mn and of every Tk only, so device `rank` evaluates
+ *     X[:, begin:end] = M1 * ... * M(n-1) * Mn[:, begin:end] + T1[:, begin:end] + ... + Tk[:, begin:end]
+ * as an ordinary equation of its own, with no exchange between devices; the slabs of X are the result (gathered
+ * by the caller where the whole X is wanted).
+ * mom_column_slab: the slab of device `rank`: the `cols` columns are cut into units of `multiple` columns (the last
+ * unit may be short) and the units are dealt out contiguously, as evenly as whole units allow; *begin == *end
+ * means the device has nothing to do.  multiple = 4 keeps every slab addressable by the tensor-core kernel.
+ * Errors: INVALID_ARG (cols < 1, world < 1, rank outside [0, world), multiple < 1, NULL outputs). */
+mom_status_t mom_column_slab(int64_t cols, int32_t rank, int32_t world, int64_t multiple, int64_t *begin, int64_t *end);
+
+/* Descriptor of the STORED matrix that holds columns [begin, end) of an operand as used: `stored` describes the
+ * whole operand as stored, `transposed` says the equation uses its transpose (then the slab is rows
+ * [begin, end) of the stored matrix, contiguous in memory).  The whole operand keeps its property; a proper slab
+ * is general (a slab of a triangular, Diagonal, Symmetric or Identity matrix is stored densely with its zeros and
+ * ones, the caller's copy).  Errors: those of mom_matrix_desc for `stored`, INVALID_ARG (NULL, begin < 0,
+ * end <= begin, end beyond the operand's columns as used). */
+mom_status_t mom_column_slab_desc(const mom_matrix_desc_t *stored, int32_t transposed, int64_t begin, int64_t end,
+                                  mom_matrix_desc_t *slab);
+
 /* Plan X = prod(chain) + sum(add_terms) (paper Section 2, "Transformations").  Host only: makes no
  * CUDA call and works on a machine without a GPU.
  *   chain      host array of n_chain >= 1 descriptors, left to right

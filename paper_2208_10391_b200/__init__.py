@@ -60,6 +60,10 @@ _lib = ctypes.CDLL(LIB_PATH)
 _P = ctypes.c_void_p
 _sigs = {
     "mom_matrix_desc": [ctypes.c_int64, ctypes.c_int64, ctypes.c_int, ctypes.c_int, ctypes.POINTER(MatrixDesc)],
+    "mom_column_slab": [ctypes.c_int64, ctypes.c_int32, ctypes.c_int32, ctypes.c_int64, ctypes.POINTER(ctypes.c_int64),
+                        ctypes.POINTER(ctypes.c_int64)],
+    "mom_column_slab_desc": [ctypes.POINTER(MatrixDesc), ctypes.c_int32, ctypes.c_int64, ctypes.c_int64,
+                             ctypes.POINTER(MatrixDesc)],
     "mom_equation_plan": [ctypes.POINTER(MatrixDesc), ctypes.c_int32, ctypes.POINTER(MatrixDesc), ctypes.c_int32,
                           ctypes.c_int, ctypes.POINTER(_P)],
     "mom_equation_plan_transposed": [ctypes.POINTER(MatrixDesc), ctypes.POINTER(ctypes.c_int32), ctypes.c_int32,
@@ -126,6 +130,69 @@ def mom_matrix_desc(rows: int, cols: int, prop: int = GENERAL, dtype: int = F32)
     d = MatrixDesc()
     _check(_lib.mom_matrix_desc(rows, cols, prop, dtype, ctypes.byref(d)), "mom_matrix_desc")
     return d
+
+
+def _as_desc(d) -> MatrixDesc:
+    if isinstance(d, MatrixDesc):
+        return d
+    return MatrixDesc(int(d[0]), int(d[1]), int(d[2]), F32 if len(d) < 4 else int(d[3]))
+
+
+def mom_column_slab(cols: int, rank: int, world: int, multiple: int = 4) -> Tuple[int, int]:
+    """Columns [begin, end) of X that device `rank` of `world` evaluates (begin == end: nothing to do)."""
+    b, e = ctypes.c_int64(), ctypes.c_int64()
+    _check(_lib.mom_column_slab(cols, rank, world, multiple, ctypes.byref(b), ctypes.byref(e)), "mom_column_slab")
+    return b.value, e.value
+
+
+def mom_column_slab_desc(stored, transposed: bool, begin: int, end: int) -> MatrixDesc:
+    """Descriptor of the stored matrix that holds columns [begin, end) of an operand as used."""
+    src, out = _as_desc(stored), MatrixDesc()
+    _check(_lib.mom_column_slab_desc(ctypes.byref(src), 1 if transposed else 0, begin, end, ctypes.byref(out)),
+           "mom_column_slab_desc")
+    return out
+
+
+def column_slab_equation(chain: Sequence, add_terms: Sequence, rank: int, world: int, chain_transposed: Sequence = (),
+                         add_transposed: Sequence = (), multiple: int = 4):
+    """Descriptors of device `rank`'s slab equation: the chain with its last operand cut to the slab's columns and
+    every Add term likewise.  Returns (chain, add_terms, begin, end), or None when the slab is empty.  Marshalling
+    only: the bounds and the slab descriptors come from the library."""
+    chain = [_as_desc(d) for d in chain]
+    add_terms = [_as_desc(d) for d in add_terms]
+    ct = list(chain_transposed) + [False] * (len(chain) - len(chain_transposed))
+    at = list(add_transposed) + [False] * (len(add_terms) - len(add_transposed))
+    cols = chain[-1].rows if ct[-1] else chain[-1].cols
+    begin, end = mom_column_slab(cols, rank, world, multiple)
+    if begin == end:
+        return None
+    chain[-1] = mom_column_slab_desc(chain[-1], ct[-1], begin, end)
+    add_terms = [mom_column_slab_desc(d, t, begin, end) for d, t in zip(add_terms, at)]
+    return chain, add_terms, begin, end
+
+
+def gather_column_slabs(x_slab, rows: int, cols: int, rank: int, world: int, multiple: int = 4, group=None):
+    """All-gather of the devices' slabs of X into the whole rows x cols matrix on every rank (torch.distributed;
+    NCCL on GPUs).  `x_slab` is this rank's rows x (end - begin) tensor, or None for an empty slab.  The slabs are
+    padded to the widest one for the collective; no arithmetic happens here."""
+    import torch
+    import torch.distributed as dist
+    bounds = [mom_column_slab(cols, r, world, multiple) for r in range(world)]
+    width = max(e - b for b, e in bounds)
+    like = x_slab if x_slab is not None else None
+    if like is None:
+        raise ValueError("gather_column_slabs needs a tensor to take device and dtype from; pass an empty one")
+    buf = torch.zeros((rows, width), dtype=like.dtype, device=like.device)
+    b, e = bounds[rank]
+    if e > b:
+        buf[:, :e - b] = x_slab
+    parts = [torch.empty_like(buf) for _ in range(world)]
+    dist.all_gather(parts, buf, group=group)
+    x = torch.empty((rows, cols), dtype=like.dtype, device=like.device)
+    for (b, e), part in zip(bounds, parts):
+        if e > b:
+            x[:, b:e] = part[:, :e - b]
+    return x
 
 
 def _desc_array(descs: Sequence) -> "ctypes.Array":

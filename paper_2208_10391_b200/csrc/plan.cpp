@@ -188,6 +188,30 @@ mom_status_t mom_matrix_desc(int64_t rows, int64_t cols, mom_property_t property
     return MOM_OK;
 }
 
+mom_status_t mom_column_slab(int64_t cols, int32_t rank, int32_t world, int64_t multiple, int64_t *begin, int64_t *end) {
+    if (!begin || !end || cols < 1 || world < 1 || rank < 0 || rank >= world || multiple < 1) return MOM_ERR_INVALID_ARG;
+    const unsigned __int128 units = ((unsigned __int128)cols + (unsigned __int128)multiple - 1) / (unsigned __int128)multiple;
+    const unsigned __int128 u0 = units * (unsigned __int128)rank / (unsigned __int128)world;
+    const unsigned __int128 u1 = units * (unsigned __int128)(rank + 1) / (unsigned __int128)world;
+    const unsigned __int128 b = u0 * (unsigned __int128)multiple, e = u1 * (unsigned __int128)multiple;
+    *begin = (int64_t)std::min<unsigned __int128>(b, (unsigned __int128)cols);
+    *end = (int64_t)std::min<unsigned __int128>(e, (unsigned __int128)cols);
+    return MOM_OK;
+}
+
+mom_status_t mom_column_slab_desc(const mom_matrix_desc_t *stored, int32_t transposed, int64_t begin, int64_t end,
+                                  mom_matrix_desc_t *slab) {
+    if (!stored || !slab) return MOM_ERR_INVALID_ARG;
+    mom_status_t st = check_desc(*stored);
+    if (st != MOM_OK) return st;
+    const int64_t used_cols = transposed ? stored->rows : stored->cols;
+    if (begin < 0 || end <= begin || end > used_cols) return MOM_ERR_INVALID_ARG;
+    if (begin == 0 && end == used_cols) { *slab = *stored; return MOM_OK; }
+    *slab = transposed ? mom_matrix_desc_t{end - begin, stored->cols, MOM_GENERAL, stored->dtype}
+                       : mom_matrix_desc_t{stored->rows, end - begin, MOM_GENERAL, stored->dtype};
+    return MOM_OK;
+}
+
 // What the planning entry points hand to the shared planner: sums of chains in dependency order (a nested sum
 // before the sum that uses it; the last one is X).  A factor is a stored matrix (an entry of the caller's pointer
 // array, possibly transposed) or the temporary of an earlier sum.
