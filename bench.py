@@ -63,8 +63,48 @@ def measured_traffic():
     return TRAFFIC_CAPTURE["bytes_per_launch"] if sha == TRAFFIC_CAPTURE["kernel_source_sha256_16"] else None
 
 
+def sum_over_ranks(value: float, world: int, device="cpu") -> float:
+    """Sum of a per-rank quantity (every rank gets it); a no-op for one rank."""
+    if world <= 1:
+        return float(value)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.SUM)
+    return float(t.item())
+
+
+def split_job_gflops(useful_flops_this_rank: int, world: int, ms_per_step: float, device="cpu") -> float:
+    """One equation cut into column slabs: the job's throughput is all slabs' work over the slowest rank's time."""
+    return sum_over_ranks(float(useful_flops_this_rank), world, device) / (ms_per_step * 1e-3) / 1e9
+
+
 def headline_equation() -> wl.Equation:
     return wl.config_large_square()
+
+
+def column_slab_of(mom, eq: wl.Equation, rank: int, world: int):
+    """This rank's share of `eq` under the column-slab split: (slab equation, begin, end); the last factor and the
+    Add terms keep their distribution, their columns are [begin, end) of the whole operand's."""
+    got = mom.column_slab_equation(eq.descs(), eq.add_descs(), rank, world, eq.chain_t, eq.add_t)
+    if got is None:
+        raise SystemExit(f"rank {rank} of {world} has no columns of {eq.name}")
+    cd, ad, begin, end = got
+    last = eq.chain[-1]
+    ops = tuple(eq.chain[:-1]) + (wl.Operand(cd[-1].rows, cd[-1].cols, cd[-1].property, last.dist, last.sigma),)
+    terms = tuple(wl.Operand(d.rows, d.cols, d.property, t.dist, t.sigma) for d, t in zip(ad, eq.add))
+    return wl.Equation(f"{eq.name}_cols{begin}_{end}", eq.seed, ops, terms, chain_t=eq.chain_t, add_t=eq.add_t), begin, end
+
+
+def cut_columns(eq: wl.Equation, chain, add, begin: int, end: int):
+    """Host arrays of the slab equation, cut from the whole equation's arrays (views made contiguous)."""
+    import numpy as np
+    ct = list(eq.chain_t) + [False] * (len(chain) - len(eq.chain_t))
+    at = list(eq.add_t) + [False] * (len(add) - len(eq.add_t))
+
+    def cut(a, t):
+        return np.ascontiguousarray(a[begin:end, :] if t else a[:, begin:end])
+    return list(chain[:-1]) + [cut(chain[-1], ct[-1])], [cut(a, t) for a, t in zip(add, at)]
 
 
 def measured_peaks():
@@ -313,6 +353,11 @@ def run_gpu(args):
     peaks = measured_peaks()
 
     eq = headline_equation()
+    whole_eq, slab = eq, None
+    if args.split == "columns" and not args.only:
+        # one equation over all ranks: this rank evaluates its columns of X, no exchange between ranks
+        eq, b, e = column_slab_of(mom, whole_eq, rank, world)
+        slab = (b, e)
     sampler = ClockSampler(local)
     if not args.only:
         sampler.start()
@@ -341,7 +386,9 @@ def run_gpu(args):
     plan = warm["plan"]
     del warm
     torch.cuda.empty_cache()
-    chain, add = wl.generate(eq)
+    chain, add = wl.generate(whole_eq)
+    if slab and slab != (0, rd_cols(whole_eq)):
+        chain, add = cut_columns(whole_eq, chain, add, *slab)
     dchain = [None if a is None else torch.from_numpy(a).cuda() for a in chain]
     dadd = [None if a is None else torch.from_numpy(a).cuda() for a in add]
     rd = plan.result_desc()
@@ -382,7 +429,7 @@ def run_gpu(args):
     ms_per_step = total_ms / args.steps
     mul, addf = plan.flops()
     useful = mul + addf
-    value = whole_job_gflops(useful, world, ms_per_step)
+    value = split_job_gflops(useful, world, ms_per_step, "cuda") if slab else whole_job_gflops(useful, world, ms_per_step)
 
     # ---- roofline of the dominant kernel (the product kernel): useful FLOPs of its launches / their device time
     steps_info = plan.steps()
@@ -408,12 +455,14 @@ def run_gpu(args):
 
     result = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
-        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "strong" if slab else "weak", "vs_baseline": None,
         "dtype": "f32 (3xTF32 tensor-core split)" if args.variant == "3xtf32" else "f32",
         "data": "synthetic",
         "config": {"workload": eq.name, "equation": "X = L*A*U*B, 8192x8192 f32, seed 3",
                    "parenthesization": plan.parenthesization(), "useful_flops": useful, "variant": args.variant,
-                   "l2": "operands (1 GiB) exceed L2; no flush", "parallelism": f"{world} independent replicas",
+                   "l2": "operands (1 GiB) exceed L2; no flush",
+                   "parallelism": (f"one equation, column slabs of X over {world} ranks (this rank: columns {slab[0]}..{slab[1]}), no exchange"
+                                   if slab else f"{world} independent replicas"),
                    "plan_us": planning_us(mom, eq, variant)},
         "clocks": clocks, "gpu_launches": launches, "roofline": roofline,
         "roofline_whole_equation_frac": (value / world / 1e3) / peak,
@@ -501,6 +550,12 @@ def run_gpu(args):
         dist.destroy_process_group()
 
 
+def rd_cols(eq: wl.Equation) -> int:
+    """Columns of the equation's result: those of its last factor as used."""
+    t = list(eq.chain_t) + [False] * (len(eq.chain) - len(eq.chain_t))
+    return eq.chain[-1].rows if t[-1] else eq.chain[-1].cols
+
+
 def rd_elems(plan):
     d = plan.result_desc()
     return d.rows * d.cols
@@ -513,6 +568,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--variant", default="3xtf32", choices=["3xtf32", "ffma"])
+    ap.add_argument("--split", default="none", choices=["none", "columns"],
+                    help="columns: the ranks share ONE headline equation, each evaluating a column slab of X (strong scaling); "
+                         "none: every rank evaluates its own replica (weak scaling)")
     ap.add_argument("--only", default=None, help="time just this workload (by name) and print a short JSON line")
     args = ap.parse_args()
     if args.impl == "reference":

@@ -19,7 +19,8 @@ def _worker(rank, world, port, out):
     dist.barrier()
     ms = bench.max_over_ranks(10.0 + 5.0 * rank, world)          # rank 1 is the slow one
     value = bench.whole_job_gflops(2_000_000_000, world, ms)
-    out.put((rank, ms, value))
+    split_value = bench.split_job_gflops(1_000_000_000 * (rank + 1), world, ms)      # slabs of unequal work
+    out.put((rank, ms, value, split_value))
     dist.barrier()
     dist.destroy_process_group()
 
@@ -35,9 +36,10 @@ def test_two_ranks_report_the_slowest_time_and_the_summed_work():
     for p in procs:
         p.join(timeout=60)
         assert p.exitcode == 0
-    for rank, ms, value in results:
+    for rank, ms, value, split_value in results:
         assert ms == 15.0                                            # max over ranks, seen by both
         assert value == pytest.approx(2 * 2e9 / 15e-3 / 1e9)        # two replicas' work over that time
+        assert split_value == pytest.approx(3e9 / 15e-3 / 1e9)      # one equation: the slabs' work summed, same time
 
 
 def test_single_rank_is_a_no_op():
@@ -45,3 +47,23 @@ def test_single_rank_is_a_no_op():
     import bench
     assert bench.max_over_ranks(7.5, 1) == 7.5
     assert bench.whole_job_gflops(10**9, 1, 1.0) == pytest.approx(1000.0)
+    assert bench.split_job_gflops(10**9, 1, 1.0) == pytest.approx(1000.0)
+
+
+def test_column_slab_of_the_headline_equation():
+    sys.path.insert(0, ROOT)
+    import numpy as np
+    import bench
+    import paper_2208_10391_b200 as mom
+    import workloads as wl
+    eq = wl.config_large_square(n=64)
+    chain, add = wl.generate(eq)
+    widths = 0
+    for rank in range(4):
+        seq, b, e = bench.column_slab_of(mom, eq, rank, 4)
+        assert (b, e) == (16 * rank, 16 * rank + 16)
+        assert seq.descs()[:-1] == eq.descs()[:-1] and seq.descs()[-1] == (64, 16, wl.GENERAL)
+        c, a = bench.cut_columns(eq, chain, add, b, e)
+        assert np.array_equal(c[-1], chain[-1][:, b:e]) and c[-1].flags["C_CONTIGUOUS"] and c[0] is chain[0]
+        widths += e - b
+    assert widths == bench.rd_cols(eq) == 64
