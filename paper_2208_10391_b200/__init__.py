@@ -173,25 +173,23 @@ def column_slab_equation(chain: Sequence, add_terms: Sequence, rank: int, world:
 
 def gather_column_slabs(x_slab, rows: int, cols: int, rank: int, world: int, multiple: int = 4, group=None):
     """All-gather of the devices' slabs of X into the whole rows x cols matrix on every rank (torch.distributed;
-    NCCL on GPUs).  `x_slab` is this rank's rows x (end - begin) tensor, or None for an empty slab.  The slabs are
-    padded to the widest one for the collective; no arithmetic happens here."""
+    NCCL on GPUs).  `x_slab` is this rank's rows x (end - begin) tensor (rows x 0 for an empty slab: it still
+    supplies device and dtype).  The slabs are padded to the widest one for the collective; no arithmetic happens
+    here."""
     import torch
     import torch.distributed as dist
     bounds = [mom_column_slab(cols, r, world, multiple) for r in range(world)]
-    width = max(e - b for b, e in bounds)
-    like = x_slab if x_slab is not None else None
-    if like is None:
-        raise ValueError("gather_column_slabs needs a tensor to take device and dtype from; pass an empty one")
-    buf = torch.zeros((rows, width), dtype=like.dtype, device=like.device)
     b, e = bounds[rank]
-    if e > b:
-        buf[:, :e - b] = x_slab
+    if tuple(x_slab.shape) != (rows, e - b):
+        raise ValueError(f"rank {rank} holds columns {b}..{e} of {rows} x {cols}, not a tensor of shape {tuple(x_slab.shape)}")
+    width = max(hi - lo for lo, hi in bounds)
+    buf = torch.zeros((rows, width), dtype=x_slab.dtype, device=x_slab.device)
+    buf[:, :e - b] = x_slab
     parts = [torch.empty_like(buf) for _ in range(world)]
     dist.all_gather(parts, buf, group=group)
-    x = torch.empty((rows, cols), dtype=like.dtype, device=like.device)
-    for (b, e), part in zip(bounds, parts):
-        if e > b:
-            x[:, b:e] = part[:, :e - b]
+    x = torch.empty((rows, cols), dtype=x_slab.dtype, device=x_slab.device)
+    for (lo, hi), part in zip(bounds, parts):
+        x[:, lo:hi] = part[:, :hi - lo]
     return x
 
 
