@@ -25,13 +25,17 @@ struct DeviceState {
     // products start while later operands are still on their way
     cudaStream_t copy_stream = nullptr, back_stream = nullptr;
     cudaEvent_t call_start = nullptr, first_rows_done = nullptr, back_done = nullptr;
-    std::vector<cudaEvent_t> slot_ready, add_ready;
+    std::vector<cudaEvent_t> slot_ready, add_ready, slot_head;
 };
 
 // events the launcher has to wait for before it first uses an operand (host-staging entry point only)
 // and, the other way, an event the launcher records once the first rows of X are final (first_rows is set to their
 // number, 0 when X is only final at the end)
-struct StageEvents { const cudaEvent_t *slot; const cudaEvent_t *add; cudaEvent_t first_rows_done; int *first_rows; };
+struct StageEvents {
+    const cudaEvent_t *slot; const cudaEvent_t *add; cudaEvent_t first_rows_done; int *first_rows;
+    // operands uploaded in two pieces: slot_head[i] is recorded once rows [0, slot_head_rows[i]) have arrived (0: one piece)
+    const cudaEvent_t *slot_head; const int *slot_head_rows;
+};
 
 constexpr int TIMING_SLOTS = 32;
 
@@ -59,6 +63,7 @@ void destroy_device_state(DeviceState *d) {
     tc_release(d->tc);
     for (cudaEvent_t e : d->events) cudaEventDestroy(e);
     for (cudaEvent_t e : d->slot_ready) cudaEventDestroy(e);
+    for (cudaEvent_t e : d->slot_head) cudaEventDestroy(e);
     for (cudaEvent_t e : d->add_ready) cudaEventDestroy(e);
     if (d->call_start) cudaEventDestroy(d->call_start);
     if (d->first_rows_done) cudaEventDestroy(d->first_rows_done);
@@ -348,10 +353,15 @@ mom_status_t execute_impl(const mom_plan *p, const float *const *chain_ptrs, con
                 a.pa = kernel_property(stp.pub.lhs_property); a.pb = kernel_property(stp.pub.rhs_property);
                 // an operand: the value itself, or d * S / S * d of a folded scaling step (S read as stored, d handed
                 // to the split pass)
+                // a left operand that arrives in two pieces: the first launch waits for its first rows only
+                const int lhs_slot = stp.pub.lhs < n_chain ? p->factor_ptr[stp.pub.lhs] : -1;
+                const bool lhs_in_pieces = staged && batch == 1 && stp.pub.uses_tensor_cores == 1 && lhs_slot >= 0 && !slot_waited[lhs_slot] &&
+                                           stp.pub.rhs != stp.pub.lhs &&
+                                           p->dev->tc.steps[s].split_a_by_part && staged->slot_head_rows[lhs_slot] == p->dev->tc.steps[s].part_row;
                 auto operand = [&](int id, int fold, const float **ptr, long long *stride, int *trans, int own_trans,
                                    const float **scale, long long *scale_step, int *scale_rows) {
                     if (fold < 0) {
-                        need_value(id);
+                        if (!(lhs_in_pieces && id == stp.pub.lhs)) need_value(id);
                         const Operand o = value(id);
                         *ptr = o.ptr; *stride = o.stride; *trans = own_trans;
                         return;
@@ -397,9 +407,18 @@ mom_status_t execute_impl(const mom_plan *p, const float *const *chain_ptrs, con
                     int used = 0;
                     // the host-staging entry point copies the first rows of X back while the rest is still computed:
                     // the product that writes X then runs as two launches (only when nothing is added to X afterwards)
-                    const bool two_parts = staged && staged->first_rows && top && stp.is_last && !stp.accumulate &&
+                    bool later_root = false;          // another chain's product is added to X after this one
+                    for (int t = s + 1; t < sum.step_end; ++t) later_root |= p->steps[t].is_last;
+                    const bool two_parts = staged && staged->first_rows && top && stp.is_last && !stp.accumulate && !later_root &&
                                            added >= n_simple && batch == 1 && p->dev->tc.steps[s].part_row > 0;
-                    if (two_parts) {
+                    if (lhs_in_pieces) {
+                        if (cudaStreamWaitEvent(stream, staged->slot_head[lhs_slot], 0) != cudaSuccess) return MOM_ERR_CUDA;
+                        st = tc_launch_step(*p, p->dev->tc, s, a, ws, p->dev->status, stream, &used, ev ? ev[1] : nullptr, 1);
+                        if (st != MOM_OK) return st;
+                        launches += used;
+                        need_slot(lhs_slot);                                               // the whole operand
+                        st = tc_launch_step(*p, p->dev->tc, s, a, ws, p->dev->status, stream, &used, nullptr, 2);
+                    } else if (two_parts) {
                         st = tc_launch_step(*p, p->dev->tc, s, a, ws, p->dev->status, stream, &used, ev ? ev[1] : nullptr, 1);
                         if (st != MOM_OK) return st;
                         launches += used;
@@ -484,6 +503,17 @@ mom_status_t mom_equation_execute_host(const mom_plan_t *plan, const float *cons
         if (cudaEventCreateWithFlags(&dev->first_rows_done, cudaEventDisableTiming) != cudaSuccess) return MOM_ERR_CUDA;
         if (cudaEventCreateWithFlags(&dev->back_done, cudaEventDisableTiming) != cudaSuccess) return MOM_ERR_CUDA;
     }
+    bool any_tc = false;
+    for (const auto &s : plan->steps) any_tc |= s.pub.uses_tensor_cores == 1;
+    if (any_tc) {
+        est = mom::tc_prepare(*plan, dev->tc);
+        if (est != MOM_OK) return est;
+    }
+    while ((int)dev->slot_head.size() < n_chain) {
+        cudaEvent_t e = nullptr;
+        if (cudaEventCreateWithFlags(&e, cudaEventDisableTiming) != cudaSuccess) return MOM_ERR_CUDA;
+        dev->slot_head.push_back(e);
+    }
     while ((int)dev->slot_ready.size() < n_chain || (int)dev->add_ready.size() < n_add) {
         cudaEvent_t e = nullptr;
         if (cudaEventCreateWithFlags(&e, cudaEventDisableTiming) != cudaSuccess) return MOM_ERR_CUDA;
@@ -528,9 +558,27 @@ mom_status_t mom_equation_execute_host(const mom_plan_t *plan, const float *cons
     std::vector<int> order(n_chain);
     for (int i = 0; i < n_chain; ++i) order[i] = i;
     std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return first_use[a] < first_use[b]; });
+    // a general operand that a tensor-core product inside the plan reads as its left factor in two row ranges travels in
+    // two pieces, with an event between them: that product starts on the first rows while the others are on their way
+    std::vector<int> head_rows(n_chain, 0);
+    if (any_tc && batch == 1)
+        for (size_t s = 0; s < plan->steps.size(); ++s) {
+            const int32_t v = plan->steps[s].pub.lhs;
+            if (!dev->tc.steps[s].split_a_by_part || v >= (int32_t)plan->factor_ptr.size()) continue;
+            const int slot = plan->factor_ptr[v];
+            if (slot >= 0 && same_as[slot] < 0 && cbytes[slot] && first_use[slot] == (int)s && !mom::triangular_upload(plan->ptr_desc[slot], batch))
+                head_rows[slot] = dev->tc.steps[s].part_row;
+        }
     for (int i : order) {
         if (same_as[i] >= 0) continue;
-        if (cbytes[i] && mom::triangular_upload(plan->ptr_desc[i], batch)) {
+        if (cbytes[i] && head_rows[i] > 0) {
+            const size_t head = (size_t)head_rows[i] * plan->ptr_desc[i].cols * sizeof(float);
+            char *dst = reinterpret_cast<char *>(const_cast<float *>(cptr[i]));
+            const char *src = reinterpret_cast<const char *>(chain_host[i]);
+            if (cudaMemcpyAsync(dst, src, head, cudaMemcpyHostToDevice, dev->copy_stream) != cudaSuccess) return MOM_ERR_CUDA;
+            if (cudaEventRecord(dev->slot_head[i], dev->copy_stream) != cudaSuccess) return MOM_ERR_CUDA;
+            if (cudaMemcpyAsync(dst + head, src + head, cbytes[i] - head, cudaMemcpyHostToDevice, dev->copy_stream) != cudaSuccess) return MOM_ERR_CUDA;
+        } else if (cbytes[i] && mom::triangular_upload(plan->ptr_desc[i], batch)) {
             // a large triangular operand: the host buffer holds zeros outside the triangle (storage contract), so
             // only the 256-row blocks' columns up to (from) the diagonal block cross the bus; the rest is zero-filled here
             const mom_matrix_desc_t &d = plan->ptr_desc[i];
@@ -563,7 +611,8 @@ mom_status_t mom_equation_execute_host(const mom_plan_t *plan, const float *cons
         cur += mom::align_up(bytes, mom::WS_ALIGN);
     }
     int first_rows = 0;
-    const mom::StageEvents staged{dev->slot_ready.data(), dev->add_ready.data(), dev->first_rows_done, &first_rows};
+    const mom::StageEvents staged{dev->slot_ready.data(), dev->add_ready.data(), dev->first_rows_done, &first_rows,
+                                  dev->slot_head.data(), head_rows.data()};
     float *x = reinterpret_cast<float *>(cur);
     const int64_t xelems = plan->result_desc.rows * plan->result_desc.cols;
     const size_t xbytes = (size_t)xelems * sizeof(float) * batch;

@@ -831,6 +831,21 @@ mom_status_t tc_prepare(const mom_plan &p, TcPlanState &s) {
                 total += part_tables[q][i].size();
             }
         }
+        // a product inside the plan whose left operand is a stored general matrix, read as stored and split here: two
+        // row ranges as well, so that a caller who is still uploading that operand can start on its first half
+        const int n_factors = (int)p.factor_ptr.size();
+        const bool stored_lhs = st.lhs >= 0 && st.lhs < n_factors && p.factor_ptr[st.lhs] >= 0 && !st.lhs_transposed &&
+                                st.lhs_property == MOM_GENERAL && !p.steps[i].a_planes_ready && p.steps[i].fold_a < 0;
+        if (!p.steps[i].is_last && stored_lhs && s.steps[i].pair && split <= 1 && !s.steps[i].mirror && m >= 2048) {
+            const int row = std::max(P_BM, (m / 2) / P_BM * P_BM);
+            for (const int4 &t : tab) part_tables[(t.x & TILE_ROW_MASK) < row ? 0 : 1][i].push_back(t);
+            s.steps[i].part_row = row;
+            s.steps[i].split_a_by_part = true;
+            for (int q = 0; q < 2; ++q) {
+                s.steps[i].part_units[q] = order(part_tables[q][i]);
+                total += part_tables[q][i].size();
+            }
+        }
         s.steps[i].units = order(tab);
         total += tab.size();
     }
@@ -905,11 +920,19 @@ mom_status_t tc_launch_step(const mom_plan &p, TcPlanState &s, int step, const P
     const SplitScale sa{a.scaleA, a.scaleA_step, a.scaleA ? (a.scaleA_rows != 0) != (a.transA != 0) : 0};
     const SplitScale sb{a.scaleB, a.scaleB_step, a.scaleB ? (a.scaleB_rows != 0) != (a.transB != 0) : 0};
     // as stored: rows x cols and the property of the matrix the kernel reads
-    const SplitJob ja{a.A, a_hi, a_lo, a.transA ? a.k : a.m, a.transA ? a.m : a.k, a.transA ? stored_prop(a.pa) : a.pa, a.transA ? 1 : 0,
-                      blocks(a.transA ? a.m : a.k), sa};
+    SplitJob ja{a.A, a_hi, a_lo, a.transA ? a.k : a.m, a.transA ? a.m : a.k, a.transA ? stored_prop(a.pa) : a.pa, a.transA ? 1 : 0,
+                blocks(a.transA ? a.m : a.k), sa};
+    const bool a_by_part = part > 0 && s.steps[step].split_a_by_part;     // a general m x k matrix read as stored
+    if (a_by_part) {
+        const int row = s.steps[step].part_row, r0 = part == 1 ? 0 : row;
+        ja.src += (size_t)r0 * a.k;
+        ja.hi += (size_t)r0 * a.k;
+        ja.lo += (size_t)r0 * a.k;
+        ja.rows = part == 1 ? row : a.m - row;
+    }
     const SplitJob jb{a.B, b_hi, b_lo, a.transB ? a.n : a.k, a.transB ? a.k : a.n, a.transB ? stored_prop(a.pb) : a.pb, a.transB ? 0 : 1,
                       blocks(a.transB ? a.k : a.n), sb};
-    const bool do_a = !st.a_planes_ready && part != 2, do_b = !st.b_planes_ready && part != 2;
+    const bool do_a = !st.a_planes_ready && (part != 2 || a_by_part), do_b = !st.b_planes_ready && part != 2;
     auto pieces = [&](const SplitJob &j) { return j.pieces_x * blocks(j.rows); };
     if (do_a && do_b) {
         split_both_kernel<<<pieces(ja) + pieces(jb), 256, 0, stream>>>(ja, jb, pieces(ja));

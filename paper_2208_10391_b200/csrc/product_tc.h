@@ -19,6 +19,10 @@ struct TcStepState {
     int4 *part_tiles[2] = {nullptr, nullptr};
     int part_num[2] = {0, 0};
     int part_units[2] = {1, 1};
+    // A product that is not the one writing X, whose left operand is a general matrix read as stored: the same two row
+    // ranges let the host-staging entry point upload that operand in two pieces and start on the first one while the
+    // second is still on its way; then each launch splits its own rows of the operand.  False: splits happen in part 1.
+    bool split_a_by_part = false;
     int units = 1;              // CTAs (or CTA pairs) the table was laid out for: unit u owns entries u, u + units, ...
 };
 
@@ -33,7 +37,8 @@ mom_status_t tc_prepare(const mom_plan &p, TcPlanState &s);
 
 // Enqueues the operand splits and the product kernel of step `step`.  `before_product`, when not
 // null, is recorded on the stream between the splits and the product kernel.
-// `part`: 0 the whole product; 1 the operand splits and the rows [0, part_row); 2 the remaining rows (no splits).
+// `part`: 0 the whole product; 1 the operand splits and the rows [0, part_row); 2 the remaining rows (no splits,
+// unless split_a_by_part: then part 1 splits the left operand's rows [0, part_row) and part 2 the others).
 mom_status_t tc_launch_step(const mom_plan &p, TcPlanState &s, int step, const ProductArgs &a, char *workspace,
                             int32_t *status, cudaStream_t stream, int *launches, cudaEvent_t before_product, int part = 0);
 

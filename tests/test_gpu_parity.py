@@ -9,7 +9,7 @@ torch = pytest.importorskip("torch")
 import paper_2208_10391_b200 as mom
 import workloads as wl
 from workloads import GENERAL as G, LOWER_TRI as L, UPPER_TRI as U, IDENTITY as I, Operand, Equation
-from gpu_util import run_equation, check_against_oracle, TOL
+from gpu_util import run_equation, check_against_oracle, run_expression, check_expression_against_oracle, TOL
 
 pytestmark = pytest.mark.gpu
 
@@ -257,6 +257,34 @@ def test_host_entry_point_copies_the_first_rows_back_early():
         assert plan_h.last_launch_count() == plan.last_launch_count() + 1
         rows = np.sort(np.random.default_rng(8).choice(n, size=24, replace=False))
         check_against_oracle(eq, xh, plan_h, chain, terms, rows=rows)
+
+
+def test_host_entry_point_starts_on_the_first_rows_of_a_left_operand_still_on_its_way():
+    # L*A*U*B (the benchmark's shape): the product A*(U*B) lies inside the plan and reads the stored general A as its
+    # left factor; in the host entry point A travels in two pieces and the product runs as two launches, each
+    # splitting its own rows of A (one launch and one split pass more), then the product that writes X as two
+    # launches as well.  Same bits as the device entry point's single launches.
+    for n in (2312, 2048):
+        eq = wl.config_large_square(n=n)
+        chain, terms = wl.generate(eq)
+        xd, plan, _ = run_equation(eq, mom.VARIANT_3XTF32, chain, terms, via="device")
+        xh, plan_h, _ = run_equation(eq, mom.VARIANT_3XTF32, chain, terms, via="host")
+        assert plan.parenthesization() == "(0*(1*(2*3)))"
+        assert np.array_equal(xd, xh)
+        assert plan_h.last_launch_count() == plan.last_launch_count() + 3
+        xh2, _, _ = run_equation(eq, mom.VARIANT_3XTF32, chain, terms, via="host")       # events and pieces are reusable
+        assert np.array_equal(xd, xh2)
+        rows = np.sort(np.random.default_rng(9).choice(n, size=24, replace=False))
+        check_against_oracle(eq, xh, plan_h, chain, terms, rows=rows)
+    # two chains write X one after the other: the first one's rows are not final when its product ends, so nothing is
+    # copied back early; the stored A is the left factor of both roots: A*(U*B) + A*L
+    n = 2048
+    g = Operand(n, n, G, "normal", 0.02)
+    ex = wl.Expression("two_uses", 92, (g, Operand(n, n, U), g, Operand(n, n, L)), ("add", [("mul", [0, 1, 2]), ("mul", [0, 3])]))
+    xd, plan_d, arrays = run_expression(ex, mom.VARIANT_3XTF32, via="device")
+    xh, plan_h, _ = run_expression(ex, mom.VARIANT_3XTF32, via="host")
+    assert np.array_equal(xd, xh) and plan_h.last_launch_count() == plan_d.last_launch_count()
+    check_expression_against_oracle(ex, xh, plan_h, arrays, sample_rows=np.arange(0, n, 97))
 
 
 @pytest.mark.parametrize("variant", VARIANTS, ids=VNAME.get)
