@@ -299,8 +299,9 @@ mom_status_t mom_plan_host_upload_bytes(const mom_plan_t *plan, int64_t batch, s
 /* Same evaluation with HOST operands and a HOST result: copies the operands into `staging` (device,
  * 256-byte aligned, at least mom_plan_host_staging_bytes), runs the plan, copies X back into
  * out_host, all on `stream` (and on two copy streams the plan owns, ordered against `stream` by events: uploads run
- * ahead of the products that need them, and the first rows of a large X travel back while its last rows are still
- * being computed); returns after the stream has been synchronised.  Instances are packed
+ * ahead of the products that need them, a large general operand that an inner tensor-core product reads as its left
+ * factor arrives in two pieces and that product starts on the first, and the first rows of a large X travel back
+ * while its last rows are still being computed); returns after the stream has been synchronised.  Instances are packed
  * (stride rows*cols).  Pinned host memory makes the copies asynchronous; pageable memory also works. */
 mom_status_t mom_equation_execute_host(const mom_plan_t *plan, const float *const *chain_host,
                                        const float *const *add_host, float *out_host, int64_t batch,
