@@ -23,7 +23,10 @@ product_ffma_kernel(ProductArgs a) {
     const float *__restrict__ B = a.B + inst * a.strideB;
     float *__restrict__ C = a.C + inst * a.strideC;
     const int m = a.m, n = a.n, k = a.k;
-    const int r0 = blockIdx.y * BM, c0 = blockIdx.x * BN;
+    // tile rows of a lower triangular A get heavier downwards: start them from the bottom, so that the longest tiles
+    // are not the last ones to be scheduled
+    const int by = a.pa == MOM_LOWER_TRI ? (int)(gridDim.y - 1 - blockIdx.y) : (int)blockIdx.y;
+    const int r0 = by * BM, c0 = blockIdx.x * BN;
     const int r1 = min(r0 + BM, m), c1 = min(c0 + BN, n);
 
     int klo, khi;
