@@ -128,10 +128,8 @@ product_ffma_kernel(ProductArgs a) {
         for (int h = 0; h < 2; ++h) {
             const int c = c0 + h * 64 + tx * 4;
             if (c >= n) continue;
-            float v[4];
-#pragma unroll
-            for (int j = 0; j < 4; ++j)
-                v[j] = (c + j < n) ? finish_entry(acc[i][h * 4 + j], a.add, inst, r, c + j, n, a.pout) : 0.0f;
+            float v[4] = {acc[i][h * 4], acc[i][h * 4 + 1], acc[i][h * 4 + 2], acc[i][h * 4 + 3]};
+            finish_row4(v, a.add, inst, r, c, n, n, a.pout, (n & 3) == 0);     // compact: the epilogue stays small in the instruction cache
             float *p = C + (long long)r * n + c;
             if (c_vec && c + 3 < n) {
                 *reinterpret_cast<float4 *>(p) = make_float4(v[0], v[1], v[2], v[3]);
