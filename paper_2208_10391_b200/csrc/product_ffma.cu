@@ -10,9 +10,9 @@ namespace mom {
 
 namespace {
 
-constexpr int BM = 128, BN = 128, BK = 8, THREADS = 256;
+constexpr int BM = 128, BN = 128, BK = 16, THREADS = 256;     // a k-block is loaded as two halves of 8
 
-__global__ void __launch_bounds__(THREADS)
+__global__ void __launch_bounds__(THREADS, 2)
 product_ffma_kernel(ProductArgs a) {
     __shared__ __align__(16) float As[2][BK][BM];     // k-major: As[k][row]
     __shared__ __align__(16) float Bs[2][BK][BN];
@@ -73,10 +73,10 @@ product_ffma_kernel(ProductArgs a) {
             }
         }
     };
-    auto store_tiles = [&](int buf, const float (&va)[4], const float (&vb)[4]) {
+    auto store_tiles = [&](int buf, int half, const float (&va)[4], const float (&vb)[4]) {
 #pragma unroll
-        for (int i = 0; i < 4; ++i) As[buf][a_k + i][a_row] = va[i];
-        *reinterpret_cast<float4 *>(&Bs[buf][b_k][b_col]) = make_float4(vb[0], vb[1], vb[2], vb[3]);
+        for (int i = 0; i < 4; ++i) As[buf][half * 8 + a_k + i][a_row] = va[i];
+        *reinterpret_cast<float4 *>(&Bs[buf][half * 8 + b_k][b_col]) = make_float4(vb[0], vb[1], vb[2], vb[3]);
     };
 
     // each thread owns rows {ty*4..+3, 64+ty*4..+3} x cols {tx*4..+3, 64+tx*4..+3}
@@ -88,15 +88,18 @@ product_ffma_kernel(ProductArgs a) {
         for (int j = 0; j < 8; ++j) acc[i][j] = 0.0f;
 
     if (klo < khi) {
-        float va[4], vb[4];
+        float va[4], vb[4], va2[4], vb2[4];
         load_a(klo, va);
         load_b(klo, vb);
-        store_tiles(0, va, vb);
+        load_a(klo + 8, va2);
+        load_b(klo + 8, vb2);
+        store_tiles(0, 0, va, vb);
+        store_tiles(0, 1, va2, vb2);
         __syncthreads();
         int buf = 0;
         for (int k0 = klo; k0 < khi; k0 += BK) {
             const bool more = k0 + BK < khi;
-            if (more) { load_a(k0 + BK, va); load_b(k0 + BK, vb); }
+            if (more) { load_a(k0 + BK, va); load_b(k0 + BK, vb); load_a(k0 + BK + 8, va2); load_b(k0 + BK + 8, vb2); }
 #pragma unroll
             for (int kk = 0; kk < BK; ++kk) {
                 const float4 a0 = *reinterpret_cast<const float4 *>(&As[buf][kk][ty * 4]);
@@ -111,7 +114,8 @@ product_ffma_kernel(ProductArgs a) {
                     for (int j = 0; j < 8; ++j) acc[i][j] = fmaf(ar[i], br[j], acc[i][j]);
             }
             if (more) {
-                store_tiles(buf ^ 1, va, vb);
+                store_tiles(buf ^ 1, 0, va, vb);
+                store_tiles(buf ^ 1, 1, va2, vb2);
                 __syncthreads();
                 buf ^= 1;
             }
