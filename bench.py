@@ -122,28 +122,45 @@ def measured_peaks():
 # ------------------------------------------------------------------------------------------------
 
 def oracle_sample_seconds(eq, chain, add, rows):
-    """Time the oracle on `rows` of X (left-to-right fp64 triple loops); returns (seconds, threads used)."""
+    """Time the oracle on `rows` of X (left-to-right fp64 triple loops); returns (seconds, threads used, X_ref rows, D rows)."""
     from oracle import values as ov
     t0 = time.perf_counter()
-    ov.evaluate([None if c is None else (c[0] if eq.batch > 1 else c) for c in chain], eq.descs(),
-                [None if a is None else (a[0] if eq.batch > 1 else a) for a in add], eq.add_descs(), rows=rows)
-    return time.perf_counter() - t0, ov.threads_used()
+    x_ref, den = ov.evaluate([None if c is None else (c[0] if eq.batch > 1 else c) for c in chain], eq.descs(),
+                             [None if a is None else (a[0] if eq.batch > 1 else a) for a in add], eq.add_descs(), rows=rows)
+    return time.perf_counter() - t0, ov.threads_used(), x_ref, den
 
 
-def cpu_baseline(eq, chain, add, useful_flops_per_instance, n_rows):
+def sample_rows(total_rows: int, slab: int = 32):
+    """One row out of every 32 (drawn inside each slab with a fixed seed): every tile row and every epilogue warp's slab
+    of the product kernels' output is represented."""
+    rng = np.random.default_rng(0)
+    return np.array([min(total_rows - 1, r0 + int(rng.integers(0, slab))) for r0 in range(0, total_rows, slab)], dtype=np.int64)
+
+
+def cpu_baseline(eq, chain, add, useful_flops_per_instance, rows, x_rows=None, x_off_structure_ok=None, result_prop=None):
+    """The oracle timed on `rows` of X; when `x_rows` (those rows of the X the timed GPU steps left) is given, the same
+    oracle values also give the run's own parity figure."""
     from oracle import plan as op
+    from oracle import values as ov
     t0 = time.perf_counter()
     op.plan(eq.descs(), eq.add_descs())
     plan_s = time.perf_counter() - t0
     total_rows = eq.chain[0].rows
-    rows = np.sort(np.random.default_rng(0).choice(total_rows, size=min(n_rows, total_rows), replace=False))
-    secs, threads = oracle_sample_seconds(eq, chain, add, rows)
+    secs, threads, x_ref, den = oracle_sample_seconds(eq, chain, add, rows)
     frac = len(rows) / total_rows
     value = useful_flops_per_instance * frac / (secs + plan_s) / 1e9
-    return {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle",
-            "sample": f"{len(rows)} of {total_rows} rows of X (one instance), exhaustive plan + left-to-right fp64 "
-                      f"triple loops incl. the error denominator; useful FLOPs scaled by the row fraction; "
-                      f"{secs + plan_s:.2f} s"}
+    out = {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle",
+           "sample": f"{len(rows)} of {total_rows} rows of X (one in every 32; one instance), exhaustive plan + left-to-right fp64 "
+                     f"triple loops incl. the error denominator; useful FLOPs scaled by the row fraction; "
+                     f"{secs + plan_s:.2f} s"}
+    parity = None
+    if x_rows is not None:
+        parity = {"normwise_err": ov.normwise_error(x_rows, x_ref, den), "bound": 1e-5, "rows_compared": int(len(rows)),
+                  "of_rows": int(total_rows), "nan_free": bool(not np.isnan(x_rows).any()),
+                  "off_structure_exact_zero": x_off_structure_ok,
+                  "what": "X left by the timed steps against the fp64 oracle on the sampled rows: ||X - X_ref||_F / ||D||_F"}
+        parity["ok"] = bool(parity["normwise_err"] <= 1e-5 and parity["nan_free"] and x_off_structure_ok is not False)
+    return out, parity
 
 
 def run_reference(args):
@@ -161,7 +178,7 @@ def run_reference(args):
     threads = 1
     for i in range(args.warmup + args.steps):
         rows = np.sort(np.random.default_rng(i).choice(total_rows, size=n_rows, replace=False))
-        secs, threads = oracle_sample_seconds(eq, chain, add, rows)
+        secs, threads, _, _ = oracle_sample_seconds(eq, chain, add, rows)
         if i >= args.warmup:
             times.append(secs)
     mean_s = sum(times) / len(times)
@@ -326,12 +343,23 @@ def time_equation(mom, torch, eq, variant, steps, warmup, stream, timing=False):
                 except mom.MomError:        # fused single-kernel plans have no per-step events
                     step_times.append([])
         stream.synchronize()
+        # the same steps back to back (nothing waits for the host between them): what a caller who enqueues equation
+        # after equation sees; the per-step figures above expose every launch gap when `timing` synchronises each step
+        b0, b1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        if timing:
+            plan.enable_step_timing(False)
+        b0.record(stream)
+        for _ in range(steps):
+            run()
+        b1.record(stream)
+        stream.synchronize()
     ms = [e0.elapsed_time(e1) for e0, e1 in events]
+    ms_b2b = b0.elapsed_time(b1) / steps
     status = plan.device_status()
     if status != (0, 0):
         raise RuntimeError(f"device-side wait timed out: {status}")
     mul, addf = plan.flops()
-    return {"ms": ms, "plan": plan, "useful_flops": (mul + addf) * eq.batch, "launches": plan.last_launch_count(),
+    return {"ms": ms, "ms_back_to_back": ms_b2b, "plan": plan, "useful_flops": (mul + addf) * eq.batch, "launches": plan.last_launch_count(),
             "step_times": step_times, "host": (chain, add), "keep": (dchain, dadd, out, ws)}
 
 
@@ -425,6 +453,15 @@ def run_gpu(args):
         prod_ms[i], pre_ms[i] = a, b
     if plan.device_status() != (0, 0):
         raise RuntimeError("device-side wait timed out")
+    # the X the timed steps left: the rows the oracle will compute below, and the exact-zero check of everything
+    # outside the result's structure (whole matrix, on the device)
+    parity_rows = sample_rows(rd.rows)
+    x_rows = out[torch.from_numpy(parity_rows).cuda()].cpu().numpy()
+    bits = out.view(torch.int32)
+    prop = rd.property
+    x_off_ok = (bool((torch.triu(bits, 1) == 0).all()) if prop in (wl.LOWER_TRI,) else
+                bool((torch.tril(bits, -1) == 0).all()) if prop in (wl.UPPER_TRI,) else True)
+    del bits
     total_ms = max_over_ranks(total_ms, world, "cuda")
     ms_per_step = total_ms / args.steps
     mul, addf = plan.flops()
@@ -435,24 +472,45 @@ def run_gpu(args):
     steps_info = plan.steps()
     prod_total_ms = sum(prod_ms)
     achieved_tflops = useful / (prod_total_ms * 1e-3) / 1e12 if prod_total_ms > 0 else None
+    timed_s = total_ms * 1e-3
     if args.variant == "3xtf32":
-        peak = peaks["bf16_sustained"] * TF32_OVER_BF16 / 3.0
-        peak_note = (f"{peaks['source']} sustained bf16 {peaks['bf16_sustained']} TFLOP/s x nominal tf32/bf16 ratio "
-                     f"{TF32_OVER_BF16:.4f} / 3 MMAs per useful product")
+        # effective 3xTF32 peak = tf32 dense peak / 3 MMAs per useful product; tf32 peak = measured bf16 peak carried over
+        # by the nominal tf32 : bf16 ratio.  Which measured bf16 figure: the sustained one (a seconds-long loop under the
+        # power cap) when this run's timed region is itself at least a second long, else the burst one.
+        peak_burst = peaks["bf16_burst"] * TF32_OVER_BF16 / 3.0
+        peak_sustained = peaks["bf16_sustained"] * TF32_OVER_BF16 / 3.0
+        use_sustained = timed_s >= 1.0
+        peak = peak_sustained if use_sustained else peak_burst
+        peak_note = (f"{peaks['source']} {'sustained' if use_sustained else 'burst'} bf16 "
+                     f"{peaks['bf16_sustained'] if use_sustained else peaks['bf16_burst']} TFLOP/s x nominal tf32/bf16 ratio "
+                     f"{TF32_OVER_BF16:.4f} / 3 MMAs per useful product; timed region {timed_s:.2f} s")
         bound = "tensor"
     else:
         props = torch.cuda.get_device_properties(local)
         mhz = clocks["sm_mhz"] or 1965.0
         peak = props.multi_processor_count * 128 * 2 * mhz * 1e6 / 1e12
+        peak_burst = peak_sustained = peak
         peak_note = f"{props.multi_processor_count} SMs x 128 FP32 lanes x 2 x median SM clock {mhz} MHz"
         bound = "alu"
+    whole_tflops = useful / (ms_per_step * 1e-3) / 1e12
     roofline = {"bound": bound, "achieved": achieved_tflops, "peak": peak, "unit": "TFLOP/s",
                 "frac": (achieved_tflops / peak) if achieved_tflops else None,
+                "frac_is": "product launches of the step (useful FLOPs / their device time) over `peak`",
+                "frac_burst": (achieved_tflops / peak_burst) if achieved_tflops else None,
+                "frac_sustained": (achieved_tflops / peak_sustained) if achieved_tflops else None,
+                "frac_whole_equation": whole_tflops / peak,
+                "frac_whole_equation_is": "all launches of the step, operand-split passes included, over `peak`",
                 "traffic": measured_traffic() if args.variant == "3xtf32" else None,
                 "kernel": "product_tc_pair_kernel" if args.variant == "3xtf32" else "product_ffma_kernel",
                 "launches_per_step": n_steps, "product_ms_per_step": prod_ms, "prepass_ms_per_step": pre_ms,
                 "peak_is": peak_note}
 
+    slab_price = None
+    if slab:
+        # what the cut costs in arithmetic: a proper slab of a triangular last factor is general (its zeros are multiplied)
+        # and a narrow slab may be parenthesized differently; all slabs' useful FLOPs over the whole equation's
+        wp = mom.mom_equation_plan_transposed(whole_eq.descs(), whole_eq.chain_t, whole_eq.add_descs(), whole_eq.add_t, variant)
+        slab_price = sum_over_ranks(float(useful), world, "cuda") / float(sum(wp.flops()))
     result = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "strong" if slab else "weak", "vs_baseline": None,
@@ -465,8 +523,9 @@ def run_gpu(args):
                                    if slab else f"{world} independent replicas"),
                    "plan_us": planning_us(mom, eq, variant)},
         "clocks": clocks, "gpu_launches": launches, "roofline": roofline,
-        "roofline_whole_equation_frac": (value / world / 1e3) / peak,
     }
+    if slab_price is not None:
+        result["config"]["slab_flops_over_whole_equation"] = slab_price
 
     if rank == 0 and world == 1:
         # ---- probes: sustained tcgen05 kind::tf32 rate and FFMA rate on this GPU
@@ -479,7 +538,12 @@ def run_gpu(args):
                 probes[name] = f"unavailable: {e}"
         result["probes"] = probes
         if isinstance(probes.get("tf32_tflops"), float) and args.variant == "3xtf32" and achieved_tflops:
-            result["roofline"]["frac_of_probe"] = achieved_tflops / (probes["tf32_tflops"] / 3.0)
+            # the library's own kind::tf32 issue loop on resident tiles (runs at the full clock: it draws little power);
+            # the second figure scales it to the median SM clock of the timed region
+            probe_peak = probes["tf32_tflops"] / 3.0
+            result["roofline"]["frac_of_probe"] = achieved_tflops / probe_peak
+            if clocks.get("sm_mhz") and clocks.get("sm_max_mhz"):
+                result["roofline"]["frac_of_probe_at_run_clock"] = achieved_tflops / (probe_peak * clocks["sm_mhz"] / clocks["sm_max_mhz"])
 
         # ---- e2e: host operands in pinned memory, H2D + execute + D2H inside the timed region
         stage_b = plan.host_staging_bytes(1)
@@ -514,9 +578,11 @@ def run_gpu(args):
             ms_min, ms_med = min(r["ms"]), statistics.median(r["ms"])
             entry = {"workload": cfg.name, "parenthesization": r["plan"].parenthesization(),
                      "useful_flops": r["useful_flops"], "ms_min_of_20": ms_min, "ms_median": ms_med,
+                     "ms_back_to_back": r["ms_back_to_back"],
+                     "gflops_back_to_back": r["useful_flops"] / (r["ms_back_to_back"] * 1e-3) / 1e9,
                      "gflops_at_min": r["useful_flops"] / (ms_min * 1e-3) / 1e9,
                      "gflops_at_median": r["useful_flops"] / (ms_med * 1e-3) / 1e9,
-                     "frac_of_roofline_at_median": r["useful_flops"] / (ms_med * 1e-3) / 1e12 / peak,
+                     "frac_of_burst_roofline_at_median": r["useful_flops"] / (ms_med * 1e-3) / 1e12 / peak_burst,
                      "launches": r["launches"], "plan_us": planning_us(mom, cfg, variant)}
             if batch > 1:
                 per_inst = sum(o.rows * o.cols for o in list(cfg.chain) + list(cfg.add)) + rd_elems(r["plan"])
@@ -542,11 +608,59 @@ def run_gpu(args):
             torch.cuda.empty_cache()
 
         # ---- CPU baseline: the oracle on a bounded sample of the same workload
-        result["cpu_baseline"] = cpu_baseline(eq, chain, add, useful, n_rows=256)
+        result["cpu_baseline"], result["parity"] = cpu_baseline(eq, chain, add, useful, parity_rows, x_rows, x_off_ok)
 
     if rank == 0:
         print(json.dumps(result))
     if world > 1:
+        dist.destroy_process_group()
+
+
+def launcher_command(argv, gpus: int, port: int):
+    """The command that starts `gpus` ranks of this script on one node (one process per GPU)."""
+    return [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={gpus}",
+            "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + list(argv)
+
+
+def free_port() -> int:
+    import socket
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        return sk.getsockname()[1]
+
+
+def run_check_launch(args):
+    """Start-up and bookkeeping only, no GPU and no measurement: every rank joins a gloo group, plans its share of the
+    headline equation (planning is host-only) and the ranks agree on the slowest rank's (made-up) time and on the summed
+    work; rank 0 prints one JSON line.  This is what a machine without GPUs can check of the multi-rank path."""
+    import torch.distributed as dist
+    import paper_2208_10391_b200 as mom
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if world > 1:
+        dist.init_process_group("gloo")
+    variant = {"3xtf32": mom.VARIANT_3XTF32, "ffma": mom.VARIANT_FFMA}[args.variant]
+    whole = headline_equation()
+    whole_plan = mom.mom_equation_plan_transposed(whole.descs(), whole.chain_t, whole.add_descs(), whole.add_t, variant)
+    whole_useful = sum(whole_plan.flops())
+    eq, slab = whole, None
+    if args.split == "columns":
+        eq, b, e = column_slab_of(mom, whole, rank, world)
+        slab = (b, e)
+    plan = mom.mom_equation_plan_transposed(eq.descs(), eq.chain_t, eq.add_descs(), eq.add_t, variant)
+    useful = sum(plan.flops())
+    ms = max_over_ranks(10.0 + rank, world)                       # a made-up per-rank time: the slowest rank's counts
+    total = sum_over_ranks(float(useful), world)
+    value = split_job_gflops(useful, world, ms) if slab else whole_job_gflops(useful, world, ms)
+    cols = sum_over_ranks(float(slab[1] - slab[0]) if slab else 0.0, world)
+    if rank == 0:
+        print(json.dumps({"check_launch": True, "n_gpus": world, "gpus_asked": args.gpus, "split": args.split,
+                          "ms_slowest_rank": ms, "value": value, "useful_flops_all_ranks": total,
+                          "useful_flops_whole_equation": whole_useful, "columns_all_ranks": cols,
+                          "slab_flops_over_whole": total / whole_useful if slab else None,
+                          "rank0_parenthesization": plan.parenthesization()}))
+    if world > 1:
+        dist.barrier()
         dist.destroy_process_group()
 
 
@@ -564,7 +678,9 @@ def rd_elems(plan):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--steps", type=int, default=250,
+                    help="timed steps of the headline equation (250 steps are about 2.3 s: long enough for the power-capped "
+                         "steady state, so that the sustained measured peak is the right roofline denominator)")
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--variant", default="3xtf32", choices=["3xtf32", "ffma"])
@@ -572,9 +688,17 @@ def main():
                     help="columns: the ranks share ONE headline equation, each evaluating a column slab of X (strong scaling); "
                          "none: every rank evaluates its own replica (weak scaling)")
     ap.add_argument("--only", default=None, help="time just this workload (by name) and print a short JSON line")
+    ap.add_argument("--check-launch", action="store_true",
+                    help="start the ranks, join a gloo group, plan each rank's share and report the bookkeeping; no GPU, no timing")
     args = ap.parse_args()
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and not (args.impl == "reference"):
+        # started as a plain script: start one rank per GPU ourselves and hand over
+        cmd = launcher_command(sys.argv[1:], args.gpus, free_port())
+        raise SystemExit(subprocess.call(cmd))
     if args.impl == "reference":
         run_reference(args)
+    elif args.check_launch:
+        run_check_launch(args)
     else:
         run_gpu(args)
 

@@ -14,8 +14,19 @@
  * property-specialised sm_100a kernel and fuses the Add terms into the last product.
  *
  * Conventions
- *   - Every function returns mom_status_t (except mom_status_string); nothing throws; there is no
- *     global state.  Output arguments are written only on MOM_OK unless stated otherwise.
+ *   - Every function returns mom_status_t (except mom_status_string); nothing throws.  Output arguments
+ *     are written only on MOM_OK unless stated otherwise.
+ *   - State.  Planning is a pure function of its arguments and may run from any number of threads at
+ *     once.  The library keeps two pieces of process-wide state, both per GPU and both behind a mutex:
+ *     a table of hardware facts and one-time kernel settings (SM count, shared-memory limits raised with
+ *     cudaFuncSetAttribute), filled when a device is first used, so one process may run plans on several
+ *     GPUs; and the fixed scratch array of mom_product_3xtf32_noalloc.  A plan's parenthesization, steps and
+ *     sizes never change after creation; the plan also owns launcher state (tile tables, a status word,
+ *     timing events, copy streams) that is created at its first execute on a device and rebuilt if the plan
+ *     is later executed on another device.  The execute calls take a per-plan lock while they enqueue, so
+ *     several threads may execute one plan (on one device); mom_plan_last_launch_count, the step timers and
+ *     mom_plan_device_status then describe whichever call came last.  A plan must not be destroyed while
+ *     another thread is inside a call on it.
  *   - "host" / "device" below says which address space a pointer must belong to.
  *   - Matrix storage (device): dense row-major f32, leading dimension == cols, base address aligned
  *     to 16 bytes.  Entries outside a triangular operand's structure must be stored as zeros (paper
@@ -25,7 +36,9 @@
  *   - The result X is always written as a full dense rows x cols matrix; entries outside the
  *     result's inferred structure are written as +0.0f.  X must not alias any input or the workspace.
  *   - Execution is asynchronous on the given stream.  All argument errors are reported before
- *     anything is enqueued.
+ *     anything is enqueued (mom_equation_execute_host included: no copy from the caller's buffers
+ *     starts before its arguments have been checked, and if a CUDA call fails later it waits for the copies
+ *     already enqueued before it returns the error).
  */
 #ifndef MOM_H_
 #define MOM_H_
@@ -128,12 +141,12 @@ typedef struct {
     uint64_t useful_mults;           /* scalar multiplications with both factors structurally non-zero */
 } mom_step_t;
 
-typedef struct mom_plan mom_plan_t;          /* opaque; host memory; immutable once created */
+typedef struct mom_plan mom_plan_t;          /* opaque; host memory; what was planned never changes (see "State" above) */
 typedef struct CUstream_st *mom_stream_t;    /* a CUDA stream handle (cudaStream_t) */
 
 /* Fill a descriptor (paper Section 2, "Types": property, static shape, element type).
  * Errors: INVALID_ARG (out NULL, rows/cols < 1, unknown property), PROPERTY (non-square triangular or
- * Identity), DTYPE. */
+ * Identity), DTYPE, LIMIT (rows or cols above 2^31 - 1025: the kernels index with 32-bit integers). */
 mom_status_t mom_matrix_desc(int64_t rows, int64_t cols, mom_property_t property, mom_dtype_t dtype,
                              mom_matrix_desc_t *out /* host */);
 
@@ -166,7 +179,10 @@ mom_status_t mom_column_slab_desc(const mom_matrix_desc_t *stored, int32_t trans
  * The multiplication count of a product counts a_il*b_lj only when both factors are structurally
  * non-zero; Identity operands are removed first; among equal-cost parenthesizations the split
  * positions are compared outermost-first, left subtree before right, smallest wins.
- * Errors: INVALID_ARG, PROPERTY, DTYPE, SHAPE_MISMATCH, OVERFLOW, ALLOC. */
+ * Errors: INVALID_ARG, PROPERTY, DTYPE, LIMIT, SHAPE_MISMATCH, OVERFLOW, ALLOC.
+ * Size limits: a dimension above 2^31 - 1025 is refused (LIMIT); a product with more than 2^24 - 1024 rows or
+ * columns never runs on the tcgen05 kernel (its tile table keeps a row index in 24 bits) but on the warp-level
+ * or FFMA kernel. */
 mom_status_t mom_equation_plan(const mom_matrix_desc_t *chain, int32_t n_chain,
                                const mom_matrix_desc_t *add_terms, int32_t n_add,
                                mom_variant_t variant, mom_plan_t **out_plan);
@@ -254,6 +270,9 @@ mom_status_t mom_plan_flops(const mom_plan_t *plan, uint64_t *mul_flops, uint64_
  * size including the NUL.  BUFFER_TOO_SMALL if cap < needed (needed is still written). */
 mom_status_t mom_plan_parenthesization(const mom_plan_t *plan, char *buf, size_t cap, size_t *needed);
 
+/* The binary products the variadic Mul was rewritten into (paper Section 2, "Operations": after the symbolic
+ * walk the equation is rematerialised as binary multiplications in the optimal order): their number, and
+ * product i in execution order (post-order of the tree; 0 <= i < n).  Errors: INVALID_ARG. */
 mom_status_t mom_plan_num_steps(const mom_plan_t *plan, int32_t *n);
 mom_status_t mom_plan_step(const mom_plan_t *plan, int32_t i, mom_step_t *out);
 
@@ -262,7 +281,9 @@ mom_status_t mom_plan_result_desc(const mom_plan_t *plan, mom_matrix_desc_t *out
 
 /* Bytes of device workspace mom_equation_execute[_batched] needs for `batch` instances: room for
  * the intermediates (each also as hi/lo planes for tensor-core steps), the split planes of the
- * operands of tensor-core steps, and split-K partial sums.  May be 0. */
+ * operands of tensor-core steps, and split-K partial sums.  May be 0.  (The paper has no counterpart: its
+ * bufferization allocates every intermediate with malloc, Section 2, "Matrix Attribute"; here the caller
+ * lends one buffer and the plan packs the intermediates into it by live range.)  Errors: INVALID_ARG. */
 mom_status_t mom_plan_workspace_bytes(const mom_plan_t *plan, int64_t batch, size_t *bytes);
 
 /* Evaluate one equation.
@@ -313,6 +334,15 @@ mom_status_t mom_equation_execute_host(const mom_plan_t *plan, const float *cons
  * leaves cleanly, so the context stays usable.  Reading clears the word. */
 mom_status_t mom_plan_device_status(const mom_plan_t *plan, int32_t *code, int32_t *detail);
 
+/* Self-test of the failure route above, without breaking anything: enqueues one tiny kernel in which a single
+ * thread waits -- with the very wait routine of the product kernels -- on a barrier that nothing ever signals.
+ * After `limit_ms` (0 < limit_ms <= 1000) the wait gives up, records {MOM_ERR_DEVICE_TIMEOUT, detail} in this
+ * plan's status block and the kernel ends by itself; once the stream has been synchronised,
+ * mom_plan_device_status reports it (and clears it) and the plan executes as before.  (The paper has no
+ * counterpart.)  Creates the plan's device state if no execute has done so yet.  Errors: INVALID_ARG, ARCH,
+ * ALLOC, CUDA. */
+mom_status_t mom_probe_wait_timeout(const mom_plan_t *plan, double limit_ms, int32_t detail, mom_stream_t stream);
+
 /* Number of kernels the most recent execute of this plan enqueued (0 before the first). */
 mom_status_t mom_plan_last_launch_count(const mom_plan_t *plan, int32_t *launches);
 
@@ -325,7 +355,11 @@ mom_status_t mom_plan_last_launch_count(const mom_plan_t *plan, int32_t *launche
 mom_status_t mom_plan_enable_step_timing(mom_plan_t *plan, int32_t enable);
 mom_status_t mom_plan_step_times(const mom_plan_t *plan, int32_t i, float *product_ms, float *prepass_ms);
 
-mom_status_t mom_plan_destroy(mom_plan_t *plan);   /* NULL is accepted */
+/* Releases the plan and the launcher state it owns (device block, events, copy streams).  The paper has no
+ * counterpart (its plans are compiled code).  NULL is accepted.  Must not run while another thread is inside a
+ * call on the same plan.  Kernels of this plan that are still in flight are waited for (the device block is
+ * released with cudaFree, which returns once the device has finished with it). */
+mom_status_t mom_plan_destroy(mom_plan_t *plan);
 
 const char *mom_status_string(mom_status_t status);
 

@@ -91,6 +91,7 @@ _sigs = {
     "mom_equation_execute_host": [_P, ctypes.POINTER(_P), ctypes.POINTER(_P), _P, ctypes.c_int64, _P,
                                   ctypes.c_size_t, _P],
     "mom_plan_device_status": [_P, ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_int32)],
+    "mom_probe_wait_timeout": [_P, ctypes.c_double, ctypes.c_int32, _P],
     "mom_plan_last_launch_count": [_P, ctypes.POINTER(ctypes.c_int32)],
     "mom_plan_enable_step_timing": [_P, ctypes.c_int32],
     "mom_plan_step_times": [_P, ctypes.c_int32, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_float)],
@@ -280,6 +281,10 @@ class Plan:
         code, detail = ctypes.c_int32(), ctypes.c_int32()
         _check(_lib.mom_plan_device_status(self._h, ctypes.byref(code), ctypes.byref(detail)), "mom_plan_device_status")
         return code.value, detail.value
+
+    def probe_wait_timeout(self, limit_ms: float, detail: int, stream: int = 0) -> None:
+        """Enqueue the bounded-wait self-test: a wait nothing satisfies gives up after `limit_ms`."""
+        _check(_lib.mom_probe_wait_timeout(self._h, float(limit_ms), int(detail), _P(stream)), "mom_probe_wait_timeout")
 
     def last_launch_count(self) -> int:
         n = ctypes.c_int32()

@@ -1,0 +1,44 @@
+// Per-device facts and one-time settings (SM count, kernel attributes that CUDA keeps per device), shared by
+// every launcher.  A process may use the library on several GPUs: nothing here is cached across devices.
+#pragma once
+
+#include <mutex>
+
+#include <cuda_runtime.h>
+
+namespace mom {
+
+constexpr int MAX_DEVICES = 64;
+
+struct DeviceInfo {
+    int sm_count = 0;
+    int max_pairs = 0;               // co-resident clusters of the CTA-pair kernel (0: not asked yet)
+    bool tc_attr = false;            // dynamic shared-memory limit raised for the tensor-core kernels on this device
+    bool pair_attr = false;
+    bool chain_attr = false;
+    int fused_max_smem[2] = {0, 0};  // largest dynamic shared-memory size set for the fused small-equation kernels
+    int batched_max_smem = 0;
+};
+
+// Entry of the device that is current on the calling thread (SM count filled in), or nullptr when the
+// ordinal is beyond MAX_DEVICES or the runtime call fails.  The entry is only read or changed while the
+// caller holds device_info_mutex().
+DeviceInfo *current_device_info(int *device = nullptr);
+std::mutex &device_info_mutex();
+
+// cudaFuncSetAttribute(MaxDynamicSharedMemorySize) once per device, remembered in `*done`.
+template <typename Kernel>
+cudaError_t raise_smem_limit_once(Kernel kernel, int bytes, bool DeviceInfo::*done) {
+    std::lock_guard<std::mutex> lock(device_info_mutex());
+    DeviceInfo *info = current_device_info();
+    if (!info) return cudaErrorInvalidDevice;
+    if (info->*done) return cudaSuccess;
+    const cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    if (e == cudaSuccess) info->*done = true;
+    return e;
+}
+
+// SM count of the current device (0 on failure).
+int current_sm_count();
+
+}  // namespace mom

@@ -465,6 +465,8 @@ extern "C" {
 mom_status_t mom_equation_execute(const mom_plan_t *plan, const float *const *chain_ptrs,
                                   const float *const *add_ptrs, float *out,
                                   void *workspace, size_t workspace_bytes, mom_stream_t stream) {
+    if (!plan) return MOM_ERR_INVALID_ARG;
+    std::lock_guard<std::mutex> lock(plan->exec_mutex);
     return mom::execute_impl(plan, chain_ptrs, nullptr, add_ptrs, nullptr, out, 0, 1, workspace, workspace_bytes,
                              reinterpret_cast<cudaStream_t>(stream));
 }
@@ -474,6 +476,8 @@ mom_status_t mom_equation_execute_batched(const mom_plan_t *plan, const float *c
                                           const int64_t *add_strides, float *out, int64_t out_stride,
                                           int64_t batch, void *workspace, size_t workspace_bytes,
                                           mom_stream_t stream) {
+    if (!plan) return MOM_ERR_INVALID_ARG;
+    std::lock_guard<std::mutex> lock(plan->exec_mutex);
     return mom::execute_impl(plan, chain_ptrs, chain_strides, add_ptrs, add_strides, out, out_stride, batch,
                              workspace, workspace_bytes, reinterpret_cast<cudaStream_t>(stream));
 }
@@ -482,6 +486,7 @@ mom_status_t mom_equation_execute_host(const mom_plan_t *plan, const float *cons
                                        const float *const *add_host, float *out_host, int64_t batch,
                                        void *staging, size_t staging_bytes, mom_stream_t stream_) {
     if (!plan || !chain_host || !out_host || batch < 1) return MOM_ERR_INVALID_ARG;
+    std::lock_guard<std::mutex> lock(plan->exec_mutex);
     cudaStream_t stream = reinterpret_cast<cudaStream_t>(stream_);
     size_t need = 0;
     mom_plan_host_staging_bytes(plan, batch, &need);
@@ -489,6 +494,30 @@ mom_status_t mom_equation_execute_host(const mom_plan_t *plan, const float *cons
     if (reinterpret_cast<uintptr_t>(staging) % mom::WS_ALIGN != 0) return MOM_ERR_ALIGNMENT;
     const int n_chain = (int)plan->ptr_desc.size(), n_add = (int)plan->add.size();
     if (n_add > 0 && !add_host) return MOM_ERR_INVALID_ARG;
+    // every argument error is found here, before the first copy is enqueued
+    std::vector<int> same_as(n_chain, -1);
+    bool strides_ok = (plan->result_desc.rows * plan->result_desc.cols) % 4 == 0;
+    for (int i = 0; i < n_chain; ++i) {
+        const mom_matrix_desc_t &d = plan->ptr_desc[i];
+        if (d.property == MOM_IDENTITY) continue;
+        if (!plan->names.empty())                        // a named matrix is one buffer, copied once
+            for (int j = 0; j < i && same_as[i] < 0; ++j)
+                if (plan->names[j] == plan->names[i]) same_as[i] = j;
+        if (same_as[i] >= 0) {
+            if (chain_host[i] != chain_host[same_as[i]]) return MOM_ERR_INVALID_ARG;
+            continue;
+        }
+        if (!plan->slot_used[i]) continue;
+        if (!chain_host[i]) return MOM_ERR_INVALID_ARG;
+        strides_ok &= (d.rows * d.cols) % 4 == 0;
+    }
+    for (int i = 0; i < n_add; ++i) {
+        if (plan->add[i].property == MOM_IDENTITY) continue;
+        if (!add_host[i]) return MOM_ERR_INVALID_ARG;
+        strides_ok &= (plan->add[i].rows * plan->add[i].cols) % 4 == 0;
+    }
+    // instance strides that are not multiples of 4 elements cannot be batched in place
+    if (batch > 1 && !strides_ok) return MOM_ERR_ALIGNMENT;
 
     int device = 0;
     mom_status_t est = mom::check_arch(&device);
@@ -519,131 +548,129 @@ mom_status_t mom_equation_execute_host(const mom_plan_t *plan, const float *cons
         if (cudaEventCreateWithFlags(&e, cudaEventDisableTiming) != cudaSuccess) return MOM_ERR_CUDA;
         ((int)dev->slot_ready.size() < n_chain ? dev->slot_ready : dev->add_ready).push_back(e);
     }
-    // uploads start once the caller's stream has reached this call (the staging area may still be in use before)
-    if (cudaEventRecord(dev->call_start, stream) != cudaSuccess) return MOM_ERR_CUDA;
-    if (cudaStreamWaitEvent(dev->copy_stream, dev->call_start, 0) != cudaSuccess) return MOM_ERR_CUDA;
+    // From here on copies from the caller's host buffers may be in flight: an error return first waits for them, so
+    // that the caller may free or reuse those buffers (and the staging area) as soon as the call has returned.
+    auto enqueue = [&]() -> mom_status_t {
+        // uploads start once the caller's stream has reached this call (the staging area may still be in use before)
+        if (cudaEventRecord(dev->call_start, stream) != cudaSuccess) return MOM_ERR_CUDA;
+        if (cudaStreamWaitEvent(dev->copy_stream, dev->call_start, 0) != cudaSuccess) return MOM_ERR_CUDA;
 
-    char *cur = static_cast<char *>(staging);
-    std::vector<const float *> cptr(n_chain, nullptr), aptr(n_add, nullptr);
-    std::vector<int64_t> cstride(n_chain, 0), astride(n_add, 0);
-    std::vector<size_t> cbytes(n_chain, 0);
-    std::vector<int> same_as(n_chain, -1);
-    for (int i = 0; i < n_chain; ++i) {                  // addresses in the staging area, in the order given
-        const mom_matrix_desc_t &d = plan->ptr_desc[i];
-        if (d.property == MOM_IDENTITY) continue;
-        if (!plan->names.empty())                        // a named matrix is copied once
-            for (int j = 0; j < i && same_as[i] < 0; ++j)
-                if (plan->names[j] == plan->names[i]) same_as[i] = j;
-        if (same_as[i] >= 0) {
-            if (chain_host[i] != chain_host[same_as[i]]) return MOM_ERR_INVALID_ARG;
-            cptr[i] = cptr[same_as[i]];
-            cstride[i] = cstride[same_as[i]];
-            continue;
-        }
-        if (!plan->slot_used[i]) continue;               // an operand no factor refers to is not uploaded
-        if (!chain_host[i]) return MOM_ERR_INVALID_ARG;
-        cbytes[i] = (size_t)d.rows * d.cols * sizeof(float) * batch;
-        cptr[i] = reinterpret_cast<const float *>(cur);
-        cstride[i] = d.rows * d.cols;
-        cur += mom::align_up(cbytes[i], mom::WS_ALIGN);
-    }
-    // upload in the order of first use by the plan's products, so that the first products can start early
-    std::vector<int> first_use(n_chain, (int)plan->steps.size());
-    for (size_t s = 0; s < plan->steps.size(); ++s)
-        for (int32_t v : {plan->steps[s].pub.lhs, plan->steps[s].pub.rhs})
-            if (v < (int32_t)plan->factor_ptr.size() && plan->factor_ptr[v] >= 0)
-                first_use[plan->factor_ptr[v]] = std::min(first_use[plan->factor_ptr[v]], (int)s);
-    for (int i = 0; i < n_chain; ++i)                    // a matrix given under several entries is needed when the first is
-        if (same_as[i] >= 0) first_use[same_as[i]] = std::min(first_use[same_as[i]], first_use[i]);
-    std::vector<int> order(n_chain);
-    for (int i = 0; i < n_chain; ++i) order[i] = i;
-    std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return first_use[a] < first_use[b]; });
-    // a general operand that a tensor-core product inside the plan reads as its left factor in two row ranges travels in
-    // two pieces, with an event between them: that product starts on the first rows while the others are on their way
-    std::vector<int> head_rows(n_chain, 0);
-    if (any_tc && batch == 1)
-        for (size_t s = 0; s < plan->steps.size(); ++s) {
-            const int32_t v = plan->steps[s].pub.lhs;
-            if (!dev->tc.steps[s].split_a_by_part || v >= (int32_t)plan->factor_ptr.size()) continue;
-            const int slot = plan->factor_ptr[v];
-            if (slot >= 0 && same_as[slot] < 0 && cbytes[slot] && first_use[slot] == (int)s && !mom::triangular_upload(plan->ptr_desc[slot], batch))
-                head_rows[slot] = dev->tc.steps[s].part_row;
-        }
-    for (int i : order) {
-        if (same_as[i] >= 0) continue;
-        if (cbytes[i] && head_rows[i] > 0) {
-            const size_t head = (size_t)head_rows[i] * plan->ptr_desc[i].cols * sizeof(float);
-            char *dst = reinterpret_cast<char *>(const_cast<float *>(cptr[i]));
-            const char *src = reinterpret_cast<const char *>(chain_host[i]);
-            if (cudaMemcpyAsync(dst, src, head, cudaMemcpyHostToDevice, dev->copy_stream) != cudaSuccess) return MOM_ERR_CUDA;
-            if (cudaEventRecord(dev->slot_head[i], dev->copy_stream) != cudaSuccess) return MOM_ERR_CUDA;
-            if (cudaMemcpyAsync(dst + head, src + head, cbytes[i] - head, cudaMemcpyHostToDevice, dev->copy_stream) != cudaSuccess) return MOM_ERR_CUDA;
-        } else if (cbytes[i] && mom::triangular_upload(plan->ptr_desc[i], batch)) {
-            // a large triangular operand: the host buffer holds zeros outside the triangle (storage contract), so
-            // only the 256-row blocks' columns up to (from) the diagonal block cross the bus; the rest is zero-filled here
+        char *cur = static_cast<char *>(staging);
+        std::vector<const float *> cptr(n_chain, nullptr), aptr(n_add, nullptr);
+        std::vector<int64_t> cstride(n_chain, 0), astride(n_add, 0);
+        std::vector<size_t> cbytes(n_chain, 0);
+        for (int i = 0; i < n_chain; ++i) {                  // addresses in the staging area, in the order given
             const mom_matrix_desc_t &d = plan->ptr_desc[i];
-            float *dst = const_cast<float *>(cptr[i]);
-            const int64_t n = d.rows;
-            if (cudaMemsetAsync(dst, 0, cbytes[i], dev->copy_stream) != cudaSuccess) return MOM_ERR_CUDA;
-            for (int64_t r0 = 0; r0 < n; r0 += mom::UPLOAD_BLOCK) {
-                const int64_t r1 = std::min(n, r0 + mom::UPLOAD_BLOCK);
-                const bool lower = mom::kernel_property(d.property) == MOM_LOWER_TRI;
-                const int64_t c0 = lower ? 0 : r0, c1 = lower ? r1 : n;
-                if (cudaMemcpy2DAsync(dst + r0 * n + c0, (size_t)n * sizeof(float), chain_host[i] + r0 * n + c0, (size_t)n * sizeof(float),
-                                      (size_t)(c1 - c0) * sizeof(float), (size_t)(r1 - r0), cudaMemcpyHostToDevice, dev->copy_stream) != cudaSuccess)
-                    return MOM_ERR_CUDA;
+            if (d.property == MOM_IDENTITY) continue;
+            if (same_as[i] >= 0) {                           // a named matrix is copied once
+                cptr[i] = cptr[same_as[i]];
+                cstride[i] = cstride[same_as[i]];
+                continue;
             }
-        } else if (cbytes[i] && cudaMemcpyAsync(const_cast<float *>(cptr[i]), chain_host[i], cbytes[i], cudaMemcpyHostToDevice, dev->copy_stream) != cudaSuccess)
+            if (!plan->slot_used[i]) continue;               // an operand no factor refers to is not uploaded
+            cbytes[i] = (size_t)d.rows * d.cols * sizeof(float) * batch;
+            cptr[i] = reinterpret_cast<const float *>(cur);
+            cstride[i] = d.rows * d.cols;
+            cur += mom::align_up(cbytes[i], mom::WS_ALIGN);
+        }
+        // upload in the order of first use by the plan's products, so that the first products can start early
+        std::vector<int> first_use(n_chain, (int)plan->steps.size());
+        for (size_t s = 0; s < plan->steps.size(); ++s)
+            for (int32_t v : {plan->steps[s].pub.lhs, plan->steps[s].pub.rhs})
+                if (v < (int32_t)plan->factor_ptr.size() && plan->factor_ptr[v] >= 0)
+                    first_use[plan->factor_ptr[v]] = std::min(first_use[plan->factor_ptr[v]], (int)s);
+        for (int i = 0; i < n_chain; ++i)                    // a matrix given under several entries is needed when the first is
+            if (same_as[i] >= 0) first_use[same_as[i]] = std::min(first_use[same_as[i]], first_use[i]);
+        std::vector<int> order(n_chain);
+        for (int i = 0; i < n_chain; ++i) order[i] = i;
+        std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return first_use[a] < first_use[b]; });
+        // a general operand that a tensor-core product inside the plan reads as its left factor in two row ranges travels in
+        // two pieces, with an event between them: that product starts on the first rows while the others are on their way
+        std::vector<int> head_rows(n_chain, 0);
+        if (any_tc && batch == 1)
+            for (size_t s = 0; s < plan->steps.size(); ++s) {
+                const int32_t v = plan->steps[s].pub.lhs;
+                if (!dev->tc.steps[s].split_a_by_part || v >= (int32_t)plan->factor_ptr.size()) continue;
+                const int slot = plan->factor_ptr[v];
+                if (slot >= 0 && same_as[slot] < 0 && cbytes[slot] && first_use[slot] == (int)s && !mom::triangular_upload(plan->ptr_desc[slot], batch))
+                    head_rows[slot] = dev->tc.steps[s].part_row;
+            }
+        for (int i : order) {
+            if (same_as[i] >= 0) continue;
+            if (cbytes[i] && head_rows[i] > 0) {
+                const size_t head = (size_t)head_rows[i] * plan->ptr_desc[i].cols * sizeof(float);
+                char *dst = reinterpret_cast<char *>(const_cast<float *>(cptr[i]));
+                const char *src = reinterpret_cast<const char *>(chain_host[i]);
+                if (cudaMemcpyAsync(dst, src, head, cudaMemcpyHostToDevice, dev->copy_stream) != cudaSuccess) return MOM_ERR_CUDA;
+                if (cudaEventRecord(dev->slot_head[i], dev->copy_stream) != cudaSuccess) return MOM_ERR_CUDA;
+                if (cudaMemcpyAsync(dst + head, src + head, cbytes[i] - head, cudaMemcpyHostToDevice, dev->copy_stream) != cudaSuccess) return MOM_ERR_CUDA;
+            } else if (cbytes[i] && mom::triangular_upload(plan->ptr_desc[i], batch)) {
+                // a large triangular operand: the host buffer holds zeros outside the triangle (storage contract), so
+                // only the 256-row blocks' columns up to (from) the diagonal block cross the bus; the rest is zero-filled here
+                const mom_matrix_desc_t &d = plan->ptr_desc[i];
+                float *dst = const_cast<float *>(cptr[i]);
+                const int64_t n = d.rows;
+                if (cudaMemsetAsync(dst, 0, cbytes[i], dev->copy_stream) != cudaSuccess) return MOM_ERR_CUDA;
+                for (int64_t r0 = 0; r0 < n; r0 += mom::UPLOAD_BLOCK) {
+                    const int64_t r1 = std::min(n, r0 + mom::UPLOAD_BLOCK);
+                    const bool lower = mom::kernel_property(d.property) == MOM_LOWER_TRI;
+                    const int64_t c0 = lower ? 0 : r0, c1 = lower ? r1 : n;
+                    if (cudaMemcpy2DAsync(dst + r0 * n + c0, (size_t)n * sizeof(float), chain_host[i] + r0 * n + c0, (size_t)n * sizeof(float),
+                                          (size_t)(c1 - c0) * sizeof(float), (size_t)(r1 - r0), cudaMemcpyHostToDevice, dev->copy_stream) != cudaSuccess)
+                        return MOM_ERR_CUDA;
+                }
+            } else if (cbytes[i] && cudaMemcpyAsync(const_cast<float *>(cptr[i]), chain_host[i], cbytes[i], cudaMemcpyHostToDevice, dev->copy_stream) != cudaSuccess)
+                return MOM_ERR_CUDA;
+            if (cudaEventRecord(dev->slot_ready[i], dev->copy_stream) != cudaSuccess) return MOM_ERR_CUDA;
+            for (int j = i + 1; j < n_chain; ++j)
+                if (same_as[j] == i && cudaEventRecord(dev->slot_ready[j], dev->copy_stream) != cudaSuccess) return MOM_ERR_CUDA;
+        }
+        for (int i = 0; i < n_add; ++i) {
+            const mom_matrix_desc_t &d = plan->add[i];
+            if (d.property == MOM_IDENTITY) continue;
+            const size_t bytes = (size_t)d.rows * d.cols * sizeof(float) * batch;
+            if (cudaMemcpyAsync(cur, add_host[i], bytes, cudaMemcpyHostToDevice, dev->copy_stream) != cudaSuccess) return MOM_ERR_CUDA;
+            if (cudaEventRecord(dev->add_ready[i], dev->copy_stream) != cudaSuccess) return MOM_ERR_CUDA;
+            aptr[i] = reinterpret_cast<const float *>(cur);
+            astride[i] = d.rows * d.cols;
+            cur += mom::align_up(bytes, mom::WS_ALIGN);
+        }
+        int first_rows = 0;
+        const mom::StageEvents staged{dev->slot_ready.data(), dev->add_ready.data(), dev->first_rows_done, &first_rows,
+                                      dev->slot_head.data(), head_rows.data()};
+        float *x = reinterpret_cast<float *>(cur);
+        const int64_t xelems = plan->result_desc.rows * plan->result_desc.cols;
+        const size_t xbytes = (size_t)xelems * sizeof(float) * batch;
+        cur += mom::align_up(xbytes, mom::WS_ALIGN);
+        size_t ws_bytes = 0;
+        mom_plan_workspace_bytes(plan, batch, &ws_bytes);
+        mom_status_t st = MOM_OK;
+        if (batch == 1) {
+            st = mom::execute_impl(plan, cptr.data(), nullptr, aptr.data(), nullptr, x, 0, 1, cur, ws_bytes, stream, &staged);
+        } else {
+            st = mom::execute_impl(plan, cptr.data(), cstride.data(), aptr.data(), astride.data(), x, xelems, batch, cur, ws_bytes, stream, &staged);
+        }
+        if (st != MOM_OK) return st;
+        if (first_rows > 0) {
+            // the first rows of X are final before the last launch ends: they travel on a stream of their own meanwhile
+            const size_t head = (size_t)first_rows * plan->result_desc.cols * sizeof(float);
+            if (cudaStreamWaitEvent(dev->back_stream, dev->first_rows_done, 0) != cudaSuccess) return MOM_ERR_CUDA;
+            if (cudaMemcpyAsync(out_host, x, head, cudaMemcpyDeviceToHost, dev->back_stream) != cudaSuccess) return MOM_ERR_CUDA;
+            if (cudaEventRecord(dev->back_done, dev->back_stream) != cudaSuccess) return MOM_ERR_CUDA;
+            if (cudaMemcpyAsync(reinterpret_cast<char *>(out_host) + head, reinterpret_cast<char *>(x) + head, xbytes - head,
+                                cudaMemcpyDeviceToHost, stream) != cudaSuccess) return MOM_ERR_CUDA;
+            if (cudaStreamWaitEvent(stream, dev->back_done, 0) != cudaSuccess) return MOM_ERR_CUDA;
+        } else if (cudaMemcpyAsync(out_host, x, xbytes, cudaMemcpyDeviceToHost, stream) != cudaSuccess) {
             return MOM_ERR_CUDA;
-        if (cudaEventRecord(dev->slot_ready[i], dev->copy_stream) != cudaSuccess) return MOM_ERR_CUDA;
-        for (int j = i + 1; j < n_chain; ++j)
-            if (same_as[j] == i && cudaEventRecord(dev->slot_ready[j], dev->copy_stream) != cudaSuccess) return MOM_ERR_CUDA;
-    }
-    for (int i = 0; i < n_add; ++i) {
-        const mom_matrix_desc_t &d = plan->add[i];
-        if (d.property == MOM_IDENTITY) continue;
-        if (!add_host[i]) return MOM_ERR_INVALID_ARG;
-        const size_t bytes = (size_t)d.rows * d.cols * sizeof(float) * batch;
-        if (cudaMemcpyAsync(cur, add_host[i], bytes, cudaMemcpyHostToDevice, dev->copy_stream) != cudaSuccess) return MOM_ERR_CUDA;
-        if (cudaEventRecord(dev->add_ready[i], dev->copy_stream) != cudaSuccess) return MOM_ERR_CUDA;
-        aptr[i] = reinterpret_cast<const float *>(cur);
-        astride[i] = d.rows * d.cols;
-        cur += mom::align_up(bytes, mom::WS_ALIGN);
-    }
-    int first_rows = 0;
-    const mom::StageEvents staged{dev->slot_ready.data(), dev->add_ready.data(), dev->first_rows_done, &first_rows,
-                                  dev->slot_head.data(), head_rows.data()};
-    float *x = reinterpret_cast<float *>(cur);
-    const int64_t xelems = plan->result_desc.rows * plan->result_desc.cols;
-    const size_t xbytes = (size_t)xelems * sizeof(float) * batch;
-    cur += mom::align_up(xbytes, mom::WS_ALIGN);
-    size_t ws_bytes = 0;
-    mom_plan_workspace_bytes(plan, batch, &ws_bytes);
-    // strides that are not multiples of 4 elements cannot be batched in place; such instances are rare
-    // (odd-sized matrices) and are handled one call at a time
-    bool strides_ok = xelems % 4 == 0;
-    for (int i = 0; i < n_chain; ++i) strides_ok &= cstride[i] % 4 == 0;
-    for (int i = 0; i < n_add; ++i) strides_ok &= astride[i] % 4 == 0;
-    mom_status_t st = MOM_OK;
-    if (batch == 1) {
-        st = mom::execute_impl(plan, cptr.data(), nullptr, aptr.data(), nullptr, x, 0, 1, cur, ws_bytes, stream, &staged);
-    } else if (strides_ok) {
-        st = mom::execute_impl(plan, cptr.data(), cstride.data(), aptr.data(), astride.data(), x, xelems, batch, cur, ws_bytes, stream, &staged);
-    } else {
-        return MOM_ERR_ALIGNMENT;
-    }
-    if (st != MOM_OK) return st;
-    if (first_rows > 0) {
-        // the first rows of X are final before the last launch ends: they travel on a stream of their own meanwhile
-        const size_t head = (size_t)first_rows * plan->result_desc.cols * sizeof(float);
-        if (cudaStreamWaitEvent(dev->back_stream, dev->first_rows_done, 0) != cudaSuccess) return MOM_ERR_CUDA;
-        if (cudaMemcpyAsync(out_host, x, head, cudaMemcpyDeviceToHost, dev->back_stream) != cudaSuccess) return MOM_ERR_CUDA;
-        if (cudaEventRecord(dev->back_done, dev->back_stream) != cudaSuccess) return MOM_ERR_CUDA;
-        if (cudaMemcpyAsync(reinterpret_cast<char *>(out_host) + head, reinterpret_cast<char *>(x) + head, xbytes - head,
-                            cudaMemcpyDeviceToHost, stream) != cudaSuccess) return MOM_ERR_CUDA;
-        if (cudaStreamWaitEvent(stream, dev->back_done, 0) != cudaSuccess) return MOM_ERR_CUDA;
-    } else if (cudaMemcpyAsync(out_host, x, xbytes, cudaMemcpyDeviceToHost, stream) != cudaSuccess) {
-        return MOM_ERR_CUDA;
+        }
+        return MOM_OK;
+    };
+    const mom_status_t status = enqueue();
+    if (status != MOM_OK) {
+        cudaStreamSynchronize(dev->copy_stream);
+        cudaStreamSynchronize(dev->back_stream);
+        cudaStreamSynchronize(stream);
+        return status;
     }
     if (cudaStreamSynchronize(stream) != cudaSuccess) return MOM_ERR_CUDA;
     return MOM_OK;
@@ -695,8 +722,22 @@ mom_status_t mom_plan_step_times(const mom_plan_t *plan, int32_t i, float *produ
     return MOM_OK;
 }
 
+mom_status_t mom_probe_wait_timeout(const mom_plan_t *plan, double limit_ms, int32_t detail, mom_stream_t stream) {
+    if (!plan || !(limit_ms > 0.0) || limit_ms > 1000.0) return MOM_ERR_INVALID_ARG;
+    std::lock_guard<std::mutex> lock(plan->exec_mutex);
+    int device = 0;
+    mom_status_t st = mom::check_arch(&device);
+    if (st != MOM_OK) return st;
+    st = mom::ensure_device_state(plan, device);
+    if (st != MOM_OK) return st;
+    const unsigned long long limit_ns = (unsigned long long)(limit_ms * 1.0e6);
+    return mom::launch_wait_timeout_probe(plan->dev->status, limit_ns, detail, reinterpret_cast<cudaStream_t>(stream)) == cudaSuccess
+               ? MOM_OK : MOM_ERR_CUDA;
+}
+
 mom_status_t mom_plan_device_status(const mom_plan_t *plan, int32_t *code, int32_t *detail) {
     if (!plan || !code) return MOM_ERR_INVALID_ARG;
+    std::lock_guard<std::mutex> lock(plan->exec_mutex);
     int32_t host[4] = {0, 0, 0, 0};
     if (plan->dev && plan->dev->status) {
         if (cudaMemcpy(host, plan->dev->status, sizeof(host), cudaMemcpyDeviceToHost) != cudaSuccess) return MOM_ERR_CUDA;

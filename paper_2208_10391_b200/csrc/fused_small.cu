@@ -13,6 +13,7 @@
 //   FFMA  plain f32 FMA on cells of 2 rows x 4 columns.
 #include <cstring>
 
+#include "device_info.h"
 #include "fused_small.h"
 
 namespace mom {
@@ -364,9 +365,6 @@ fused_small_kernel(const FusedPlan fp) {
     }
 }
 
-int g_sm_count = 0;
-int g_max_smem[2] = {0, 0};
-
 }  // namespace
 
 int fused_copy_table(int rows, int cols, int prop, int smem_off, int ld, std::vector<uint2> &table) {
@@ -385,23 +383,25 @@ int fused_copy_table(int rows, int cols, int prop, int smem_off, int ld, std::ve
 }
 
 cudaError_t launch_fused_small(const FusedPlan &fp, size_t smem_bytes, cudaStream_t stream) {
-    if (!g_sm_count) {
-        int dev = 0;
-        cudaGetDevice(&dev);
-        cudaDeviceGetAttribute(&g_sm_count, cudaDevAttrMultiProcessorCount, dev);
-    }
     const int v = fp.use_mma ? 1 : 0;
-    if ((int)smem_bytes > g_max_smem[v]) {
-        cudaError_t e = v ? cudaFuncSetAttribute(fused_small_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes)
-                          : cudaFuncSetAttribute(fused_small_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
-        if (e != cudaSuccess) return e;
-        g_max_smem[v] = (int)smem_bytes;
+    int sm_count = 0;
+    {
+        std::lock_guard<std::mutex> lock(device_info_mutex());
+        DeviceInfo *info = current_device_info();
+        if (!info) return cudaErrorInvalidDevice;
+        sm_count = info->sm_count;
+        if ((int)smem_bytes > info->fused_max_smem[v]) {
+            cudaError_t e = v ? cudaFuncSetAttribute(fused_small_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes)
+                              : cudaFuncSetAttribute(fused_small_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
+            if (e != cudaSuccess) return e;
+            info->fused_max_smem[v] = (int)smem_bytes;
+        }
     }
     // enough CTAs to fill every SM several times over; each walks instances with a grid stride
     long long per_sm = smem_bytes ? (long long)(220 * 1024) / (long long)smem_bytes : 8;
     if (per_sm > 8) per_sm = 8;
     if (per_sm < 1) per_sm = 1;
-    long long grid = (long long)g_sm_count * per_sm;
+    long long grid = (long long)sm_count * per_sm;
     if (grid > fp.batch) grid = fp.batch;
     if (v) fused_small_kernel<true><<<(unsigned)grid, THREADS, smem_bytes, stream>>>(fp);
     else fused_small_kernel<false><<<(unsigned)grid, THREADS, smem_bytes, stream>>>(fp);

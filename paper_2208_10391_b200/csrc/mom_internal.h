@@ -3,6 +3,7 @@
 
 #include <cstddef>
 #include <cstdint>
+#include <mutex>
 #include <string>
 #include <vector>
 
@@ -24,6 +25,12 @@ constexpr int FF_BM = 128;
 constexpr int FF_BN = 128;
 
 constexpr size_t WS_ALIGN = 256;
+
+// Largest rows / cols a descriptor may have: every kernel indexes rows, columns and k with 32-bit integers.
+constexpr int64_t MAX_DIMENSION = 2147483647 - 1024;
+// Largest m (and n) of a product on the tcgen05 kernel: a tile-table entry keeps the tile's first row in 24 bits
+// and a padding entry sits at row 2^24 - 256, which must lie outside every matrix.
+constexpr int64_t TC_MAX_ROWS = (1 << 24) - 1024;
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
@@ -121,6 +128,10 @@ struct mom_plan {
     size_t fused_smem_bytes = 0;
     std::vector<int> fused_value_off;          // shared-memory offset (floats) per value id; -1 = not resident
     std::vector<int> fused_value_ld;           // shared-memory leading dimension (floats) per value id
+    // launcher state: created at the first execute on a device, rebuilt when the plan moves to another device;
+    // `exec_mutex` serialises the host side of execute calls on one plan (enqueueing only: the kernels of two
+    // calls on different streams still overlap on the GPU)
+    mutable std::mutex exec_mutex;
     mutable mom::DeviceState *dev = nullptr;
     mutable int32_t last_launches = 0;
     bool step_timing = false;

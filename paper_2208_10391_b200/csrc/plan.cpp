@@ -115,6 +115,7 @@ mom_status_t check_desc(const mom_matrix_desc_t &d) {
     if (d.property < MOM_GENERAL || d.property > MOM_UNIT_UPPER) return MOM_ERR_INVALID_ARG;
     if (d.dtype != MOM_F32) return MOM_ERR_DTYPE;
     if (d.property != MOM_GENERAL && d.rows != d.cols) return MOM_ERR_PROPERTY;
+    if (d.rows > mom::MAX_DIMENSION || d.cols > mom::MAX_DIMENSION) return MOM_ERR_LIMIT;   // the kernels index with 32-bit integers
     return MOM_OK;
 }
 
@@ -552,7 +553,8 @@ static mom_status_t plan_sums(const std::vector<mom_matrix_desc_t> &slots, const
         for (int s = 0; s < ns; ++s) {
             mom::StepImpl &st = p->steps[s];
             const int64_t m = st.pub.m, n = st.pub.n, k = st.pub.k;
-            const bool addressable = (k % 4 == 0) && (n % 4 == 0);
+            // what TMA can address (16-byte row pitch) and the tile table can hold (first row of a tile in 24 bits)
+            const bool addressable = (k % 4 == 0) && (n % 4 == 0) && m <= mom::TC_MAX_ROWS && n <= mom::TC_MAX_ROWS;
             // below this size the tcgen05 path's extra launches (operand splits, split-K reduction) cost more
             // than its faster mainloop saves; the warp-level kernel is one launch
             const bool large = (double)m * (double)n * (double)k >= 6.0 * (double)(1 << 26);

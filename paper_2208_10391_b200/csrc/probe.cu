@@ -1,6 +1,7 @@
 // Sustained instruction-rate probes: the denominators of the reported roofline fractions.
 #include <cuda_runtime.h>
 
+#include "device_info.h"
 #include "mom.h"
 #include "tc_probe.h"
 
@@ -40,15 +41,7 @@ mom_status_t time_kernel(cudaStream_t stream, double *ms_out, void (*launch)(cud
     return MOM_OK;
 }
 
-int g_sms = 0;
-int sm_count() {
-    if (!g_sms) {
-        int dev = 0;
-        cudaGetDevice(&dev);
-        cudaDeviceGetAttribute(&g_sms, cudaDevAttrMultiProcessorCount, dev);
-    }
-    return g_sms;
-}
+int sm_count() { return mom::current_sm_count(); }
 
 void launch_ffma(cudaStream_t s, int iters, void *arg) {
     ffma_probe_kernel<<<sm_count() * 8, 256, 0, s>>>(static_cast<float *>(arg), iters, 1.0f);

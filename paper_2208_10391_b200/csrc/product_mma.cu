@@ -9,6 +9,7 @@
 #include <cooperative_groups.h>
 
 #include "device_common.cuh"
+#include "device_info.h"
 #include "kernels.h"
 
 namespace mom {
@@ -198,22 +199,17 @@ product_mma_kernel(const ProductArgs a, const int split, const int tiles_n) {
     cluster.sync();                                          // nobody leaves while a peer may still read its tile
 }
 
-int g_sm_count = 0;
-
 }  // namespace
 
 cudaError_t launch_product_mma(const ProductArgs &a, int batch, cudaStream_t stream) {
-    if (!g_sm_count) {
-        int dev = 0;
-        cudaGetDevice(&dev);
-        cudaDeviceGetAttribute(&g_sm_count, cudaDevAttrMultiProcessorCount, dev);
-    }
+    const int sm_count = current_sm_count();
+    if (sm_count < 1) return cudaErrorInvalidDevice;
     const int tiles_n = (a.n + BN - 1) / BN;
     const long long tiles = (long long)((a.m + BM - 1) / BM) * tiles_n;
     // few tiles and a long contraction: split k over a cluster, as long as every slice keeps a few k-blocks
     // (the longest structural k-range of a tile is at most k)
     int split = 1;
-    const long long resident = 4LL * g_sm_count;
+    const long long resident = 4LL * sm_count;
     while (split < MAX_SPLIT && tiles * batch * split * 2 <= resident && a.k / (split * 2) >= 4 * BK) split *= 2;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(tiles * split), 1, (unsigned)batch);

@@ -24,6 +24,7 @@
 
 #include <cuda.h>
 
+#include "device_info.h"
 #include "product_tc.h"
 #include "tc_probe.h"
 #include "tc_ptx.cuh"
@@ -66,7 +67,8 @@ __device__ __forceinline__ unsigned long long global_ns() {
 }
 
 // Bounded wait: false when the limit was reached (records the failure) or another role gave up.
-__device__ __forceinline__ bool wait_barrier(uint32_t bar, uint32_t parity, volatile int *abort_flag, int32_t *status, int detail) {
+__device__ __forceinline__ bool wait_barrier(uint32_t bar, uint32_t parity, volatile int *abort_flag, int32_t *status, int detail,
+                                             unsigned long long limit_ns = WAIT_LIMIT_NS) {
     unsigned long long start = 0;
     for (uint32_t i = 0;; ++i) {
         if (ptx::mbar_try_wait(bar, parity)) return true;
@@ -74,7 +76,7 @@ __device__ __forceinline__ bool wait_barrier(uint32_t bar, uint32_t parity, vola
             if (*abort_flag) return false;
             const unsigned long long now = global_ns();
             if (start == 0) start = now;
-            else if (now - start > WAIT_LIMIT_NS) break;
+            else if (now - start > limit_ns) break;
         }
     }
     if (atomicCAS(status, 0, (int)MOM_ERR_DEVICE_TIMEOUT) == 0) status[1] = detail;
@@ -706,9 +708,6 @@ bool make_map(CUtensorMap *map, const void *ptr, int rows, int cols, int box_row
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-int g_sm_count = 0;
-bool g_attr_set = false;
-
 }  // namespace
 
 mom_status_t tc_prepare(const mom_plan &p, TcPlanState &s) {
@@ -894,16 +893,9 @@ mom_status_t tc_launch_step(const mom_plan &p, TcPlanState &s, int step, const P
     const int4 *tiles = part ? s.steps[step].part_tiles[part - 1] : s.steps[step].tiles;
     const int num_tiles = part ? s.steps[step].part_num[part - 1] : s.steps[step].num_tiles;
     const int units = part ? s.steps[step].part_units[part - 1] : s.steps[step].units;
-    if (!g_sm_count) {
-        int dev = 0;
-        cudaGetDevice(&dev);
-        cudaDeviceGetAttribute(&g_sm_count, cudaDevAttrMultiProcessorCount, dev);
-    }
-    if (!g_attr_set) {
-        if (cudaFuncSetAttribute(product_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess)
-            return MOM_ERR_CUDA;
-        g_attr_set = true;
-    }
+    const int sm_count = current_sm_count();
+    if (sm_count < 1) return MOM_ERR_CUDA;
+    if (raise_smem_limit_once(product_tc_kernel, SMEM_BYTES, &DeviceInfo::tc_attr) != cudaSuccess) return MOM_ERR_CUDA;
     float *a_hi = reinterpret_cast<float *>(workspace + st.a_hi_off), *a_lo = reinterpret_cast<float *>(workspace + st.a_lo_off);
     float *b_hi = reinterpret_cast<float *>(workspace + st.b_hi_off), *b_lo = reinterpret_cast<float *>(workspace + st.b_lo_off);
 
@@ -983,15 +975,10 @@ mom_status_t tc_launch_step(const mom_plan &p, TcPlanState &s, int step, const P
     if (st.split_k > 1) prm.add.count = 0;
     prm.status = status;
     if (s.steps[step].pair) {
-        static bool pair_attr_set = false;
-        if (!pair_attr_set) {
-            if (cudaFuncSetAttribute(product_tc_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, P_SMEM_BYTES) != cudaSuccess)
-                return MOM_ERR_CUDA;
-            pair_attr_set = true;
-        }
+        if (raise_smem_limit_once(product_tc_pair_kernel, P_SMEM_BYTES, &DeviceInfo::pair_attr) != cudaSuccess) return MOM_ERR_CUDA;
         cudaLaunchConfig_t cfg;
         std::memset(&cfg, 0, sizeof(cfg));
-        cfg.gridDim = dim3(g_sm_count / 2 * 2);
+        cfg.gridDim = dim3(sm_count / 2 * 2);
         cfg.blockDim = dim3(THREADS);
         cfg.dynamicSmemBytes = P_SMEM_BYTES;
         cfg.stream = stream;
@@ -1004,29 +991,59 @@ mom_status_t tc_launch_step(const mom_plan &p, TcPlanState &s, int step, const P
         cfg.numAttrs = 1;
         // A persistent grid must not exceed what is co-resident: not every SM can host half of a CTA pair
         // (the pair must sit on one TPC), so ask how many clusters fit instead of assuming SMs / 2.
-        static int max_pairs = 0;
-        if (!max_pairs) {
-            int n = 0;
-            if (cudaOccupancyMaxActiveClusters(&n, product_tc_pair_kernel, &cfg) != cudaSuccess || n < 1) return MOM_ERR_CUDA;
-            max_pairs = n;
+        int max_pairs = 0;
+        {
+            std::lock_guard<std::mutex> lock(device_info_mutex());
+            DeviceInfo *info = current_device_info();
+            if (!info) return MOM_ERR_CUDA;
+            if (!info->max_pairs) {
+                int n = 0;
+                if (cudaOccupancyMaxActiveClusters(&n, product_tc_pair_kernel, &cfg) != cudaSuccess || n < 1) return MOM_ERR_CUDA;
+                info->max_pairs = n;
+            }
+            max_pairs = info->max_pairs;
         }
         if (max_pairs < units) return MOM_ERR_CUDA;   // the table was laid out for co-resident pairs
         cfg.gridDim = dim3(2 * units);
         if (cudaLaunchKernelEx(&cfg, product_tc_pair_kernel, ma_hi, ma_lo, mb_hi, mb_lo, mc, mc2, prm) != cudaSuccess) return MOM_ERR_CUDA;
     } else {
-        const int grid = std::min(units, g_sm_count);
+        const int grid = std::min(units, sm_count);
         product_tc_kernel<<<grid, THREADS, SMEM_BYTES, stream>>>(ma_hi, ma_lo, mb_hi, mb_lo, mc, mc2, prm);
     }
     if (cudaGetLastError() != cudaSuccess) return MOM_ERR_CUDA;
     *launches = 1 + split_launches;
     if (st.split_k > 1) {
         const long long vecs = (long long)a.m * (a.n / 4);
-        const int blocks_r = (int)std::min<long long>((vecs + 255) / 256, (long long)g_sm_count * 8);
+        const int blocks_r = (int)std::min<long long>((vecs + 255) / 256, (long long)sm_count * 8);
         splitk_reduce_kernel<<<blocks_r, 256, 0, stream>>>(partial, st.split_k, slice_rows, a.C, a.m, a.n, a.pout, a.add);
         if (cudaGetLastError() != cudaSuccess) return MOM_ERR_CUDA;
         ++*launches;
     }
     return MOM_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Self-test of the bounded wait: one thread waits, with the product kernels' own wait_barrier, on an mbarrier
+// that nothing ever arrives on.  The wait gives up after `limit_ns`, records MOM_ERR_DEVICE_TIMEOUT and
+// `detail` in the status block exactly as a product kernel would, and the kernel returns by itself.
+// ---------------------------------------------------------------------------------------------
+namespace {
+__global__ void __launch_bounds__(32, 1) wait_timeout_kernel(int32_t *status, unsigned long long limit_ns, int detail) {
+    __shared__ __align__(8) unsigned long long barrier_word;
+    __shared__ int abort_word;
+    if (threadIdx.x == 0) {
+        abort_word = 0;
+        const uint32_t bar = ptx::smem_u32(&barrier_word);
+        ptx::mbar_init(bar, 1);
+        ptx::fence_barrier_init();
+        wait_barrier(bar, 0, &abort_word, status, detail, limit_ns);
+    }
+}
+}  // namespace
+
+cudaError_t launch_wait_timeout_probe(int32_t *status, unsigned long long limit_ns, int detail, cudaStream_t stream) {
+    wait_timeout_kernel<<<1, 32, 0, stream>>>(status, limit_ns, detail);
+    return cudaGetLastError();
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -1182,12 +1199,9 @@ extern "C" mom_status_t mom_product_3xtf32_noalloc(int64_t m64, int64_t n64, int
         if (cudaGetSymbolAddress(&p, g_noalloc_scratch) != cudaSuccess || !p) return MOM_ERR_CUDA;
         g_noalloc_device_ptr[dev] = static_cast<unsigned char *>(p);
     }
-    if (!g_sm_count) cudaDeviceGetAttribute(&g_sm_count, cudaDevAttrMultiProcessorCount, dev);
-    if (!g_attr_set) {
-        if (cudaFuncSetAttribute(product_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess)
-            return MOM_ERR_CUDA;
-        g_attr_set = true;
-    }
+    const int sm_count = current_sm_count();
+    if (sm_count < 1) return MOM_ERR_CUDA;
+    if (raise_smem_limit_once(product_tc_kernel, SMEM_BYTES, &DeviceInfo::tc_attr) != cudaSuccess) return MOM_ERR_CUDA;
     cudaStream_t stream = reinterpret_cast<cudaStream_t>(stream_);
     unsigned char *base = g_noalloc_device_ptr[dev];
     float *a_hi = reinterpret_cast<float *>(base), *a_lo = reinterpret_cast<float *>(base + a_bytes);
@@ -1222,6 +1236,6 @@ extern "C" mom_status_t mom_product_3xtf32_noalloc(int64_t m64, int64_t n64, int
     prm.mirror = 0;
     prm.add.count = 0;
     prm.status = status;
-    product_tc_kernel<<<std::min(prm.num_tiles, g_sm_count), THREADS, SMEM_BYTES, stream>>>(ma_hi, ma_lo, mb_hi, mb_lo, mc, mc, prm);
+    product_tc_kernel<<<std::min(prm.num_tiles, sm_count), THREADS, SMEM_BYTES, stream>>>(ma_hi, ma_lo, mb_hi, mb_lo, mc, mc, prm);
     return cudaGetLastError() == cudaSuccess ? MOM_OK : MOM_ERR_CUDA;
 }

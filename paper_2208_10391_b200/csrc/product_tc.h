@@ -44,4 +44,8 @@ mom_status_t tc_launch_step(const mom_plan &p, TcPlanState &s, int step, const P
 
 void tc_release(TcPlanState &s);
 
+// One thread waits with the product kernels' bounded wait on a barrier nothing arrives on; after `limit_ns` it
+// records {MOM_ERR_DEVICE_TIMEOUT, detail} in `status` (device, 4 ints) and the kernel ends.
+cudaError_t launch_wait_timeout_probe(int32_t *status, unsigned long long limit_ns, int detail, cudaStream_t stream);
+
 }  // namespace mom

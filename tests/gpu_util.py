@@ -13,6 +13,19 @@ TOL = 1e-5          # normwise bound ||X - X_ref||_F / || |M1|...|Mn| + sum|Ti| 
 CANARY = 64         # guard floats on each side of the output buffer
 
 
+def stratified_rows(m: int, seed: int, slab: int = 32, extra=()):
+    """One row out of every `slab` consecutive rows (drawn at random inside the slab), plus `extra` rows.
+
+    The tensor-core kernels write the output in tiles of 128 or 256 rows, each epilogue warp a slab of 32 rows:
+    with one row per slab every tile row and every warp's slab of a large output is compared with the oracle,
+    at a cost the oracle can afford (m / 32 vector-matrix chains).
+    """
+    rng = np.random.default_rng(seed)
+    rows = [min(m - 1, r0 + int(rng.integers(0, slab))) for r0 in range(0, m, slab)]
+    rows += [r for r in extra if 0 <= r < m]
+    return np.unique(np.array(rows, dtype=np.int64))
+
+
 def to_device(arrs):
     return [None if a is None else torch.from_numpy(a).cuda() for a in arrs]
 

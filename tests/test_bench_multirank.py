@@ -67,3 +67,36 @@ def test_column_slab_of_the_headline_equation():
         assert np.array_equal(c[-1], chain[-1][:, b:e]) and c[-1].flags["C_CONTIGUOUS"] and c[0] is chain[0]
         widths += e - b
     assert widths == bench.rd_cols(eq) == 64
+
+
+@pytest.mark.parametrize("split", ["none", "columns"])
+def test_bench_starts_its_own_ranks(split):
+    # `python bench.py --gpus 2` (no torchrun around it) starts two ranks itself; --check-launch keeps them off the GPU:
+    # gloo group, each rank plans its share, the slowest rank's time and the summed work are agreed on
+    import json
+    import subprocess
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    proc = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--check-launch", "--split", split],
+                          capture_output=True, text=True, timeout=600, env=env, cwd=ROOT)
+    assert proc.returncode == 0, proc.stderr[-2000:]
+    lines = [l for l in proc.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1                                         # rank 0 alone prints
+    r = json.loads(lines[0])
+    assert r["n_gpus"] == 2 and r["gpus_asked"] == 2 and r["ms_slowest_rank"] == 11.0
+    whole = r["useful_flops_whole_equation"]
+    if split == "columns":
+        assert r["columns_all_ranks"] == 8192 and r["useful_flops_all_ranks"] == whole     # B is general: the cut is free
+        assert r["slab_flops_over_whole"] == 1.0
+        assert r["value"] == pytest.approx(whole / 11e-3 / 1e9)
+    else:
+        assert r["useful_flops_all_ranks"] == 2 * whole
+        assert r["value"] == pytest.approx(2 * whole / 11e-3 / 1e9)
+
+
+def test_launcher_command_is_one_process_per_gpu_on_the_loopback_address():
+    sys.path.insert(0, ROOT)
+    import bench
+    cmd = bench.launcher_command(["--gpus", "4", "--steps", "7"], 4, 29876)
+    assert cmd[1:3] == ["-m", "torch.distributed.run"] and "--nproc-per-node=4" in cmd and "--nnodes=1" in cmd
+    assert cmd[cmd.index("--master-addr") + 1] == "127.0.0.1" and cmd[cmd.index("--master-port") + 1] == "29876"
+    assert cmd[-4:] == ["--gpus", "4", "--steps", "7"] and cmd[-5].endswith("bench.py")

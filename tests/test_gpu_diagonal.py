@@ -11,7 +11,7 @@ import paper_2208_10391_b200 as mom
 import workloads as wl
 from workloads import GENERAL as G, LOWER_TRI as L, UPPER_TRI as U, IDENTITY as I, DIAGONAL as D, Operand, Equation
 from gpu_util import (run_equation, check_against_oracle, run_sum_equation, check_sum_against_oracle, run_expression,
-                      check_expression_against_oracle)
+                      check_expression_against_oracle, stratified_rows)
 
 pytestmark = pytest.mark.gpu
 
@@ -143,5 +143,4 @@ def test_config_diagonal_full_size_sampled_rows():
     eq = wl.config_diagonal()
     x, plan, (chain, add) = run_equation(eq, mom.VARIANT_3XTF32)
     assert [plan.step(i).kind for i in range(plan.num_steps())].count(mom.KIND_SCALE) == 1
-    rows = np.sort(np.random.default_rng(5).choice(eq.chain[0].rows, size=48, replace=False))
-    check_against_oracle(eq, x, plan, chain, add, rows=rows)
+    check_against_oracle(eq, x, plan, chain, add, rows=stratified_rows(eq.chain[0].rows, 5))

@@ -9,7 +9,7 @@ torch = pytest.importorskip("torch")
 import paper_2208_10391_b200 as mom
 import workloads as wl
 from workloads import GENERAL as G, LOWER_TRI as L, UPPER_TRI as U, IDENTITY as I, Operand, Equation
-from gpu_util import run_equation, check_against_oracle, run_expression, check_expression_against_oracle, TOL
+from gpu_util import run_equation, check_against_oracle, run_expression, check_expression_against_oracle, stratified_rows, TOL
 
 pytestmark = pytest.mark.gpu
 
@@ -123,27 +123,38 @@ def test_pair_kernel_ragged_shapes(case):
         eq = Equation("pair_chain", 72, (Operand(m, m, U), Operand(m, k, G, "normal", 0.02), Operand(k, k, L), Operand(k, n, G, "normal", 0.02)))
     x, plan, (chain, add) = run_equation(eq, mom.VARIANT_3XTF32)
     assert all(s.uses_tensor_cores == 1 for s in plan.steps())
-    rows = np.sort(np.random.default_rng(3).choice(m, size=40, replace=False))
-    rows[:6] = [0, 127, 128, 255, 256, m - 1]
-    check_against_oracle(eq, x, plan, chain, add, rows=np.sort(rows))
+    # one row in every 32-row slab: every pair-tile row and every epilogue warp's slab is compared
+    check_against_oracle(eq, x, plan, chain, add, rows=stratified_rows(m, 3, extra=[0, 127, 128, 255, 256, m - 1]))
+
+
+@pytest.mark.parametrize("pa,pb", list(itertools.product([G, L, U], repeat=2)))
+def test_pair_kernel_whole_output(pa, pb):
+    # the smallest products the CTA-pair kernel takes (48 pair tiles of 256 x 256), every property pair, compared with
+    # the oracle on the WHOLE output: every tile, every k-range of the tile table, every epilogue slab
+    m, n = 2048, 1536
+    if pa != G and pb != G:
+        m = n = 2048                                      # both factors are square
+    k = m if pa != G else n if pb != G else 1152
+    op = lambda r, c, p: Operand(r, c, p, "normal", 0.05) if p == G else Operand(r, c, p)
+    eq = Equation(f"pair_full_{pa}{pb}", 73, (op(m, k, pa), op(k, n, pb)), (Operand(m, n, G, "normal"),) if pa == G else ())
+    x, plan, (chain, add) = run_equation(eq, mom.VARIANT_3XTF32_FORCE)
+    assert plan.step(0).uses_tensor_cores == 1 and (m // 256) * (n // 256) >= 48
+    check_against_oracle(eq, x, plan, chain, add)
 
 
 @pytest.mark.parametrize("variant", [mom.VARIANT_3XTF32, mom.VARIANT_FFMA], ids=VNAME.get)
 def test_config_property_heavy_full_size_sampled_rows(variant):
     eq = wl.config_property_heavy()
     x, plan, (chain, add) = run_equation(eq, variant)
-    rows = np.random.default_rng(0).choice(4096, size=48, replace=False)
-    rows[:4] = [0, 127, 128, 4095]
-    check_against_oracle(eq, x, plan, chain, add, rows=np.sort(rows))
+    check_against_oracle(eq, x, plan, chain, add, rows=stratified_rows(4096, 0, extra=[0, 127, 128, 4095]))
 
 
 @pytest.mark.parametrize("variant", [mom.VARIANT_3XTF32], ids=VNAME.get)
 def test_config_large_square_full_size_sampled_rows(variant):
     eq = wl.config_large_square()
     x, plan, (chain, add) = run_equation(eq, variant)
-    rows = np.random.default_rng(1).choice(8192, size=24, replace=False)
-    rows[:4] = [0, 127, 128, 8191]
-    check_against_oracle(eq, x, plan, chain, add, rows=np.sort(rows))
+    # 256 rows, one in every 32-row slab: all 32 pair-tile rows and all 256 epilogue-warp slabs of X
+    check_against_oracle(eq, x, plan, chain, add, rows=stratified_rows(8192, 1, extra=[0, 127, 128, 8191]))
 
 
 @pytest.mark.parametrize("variant", VARIANTS + [mom.VARIANT_3XTF32], ids=VNAME.get)
@@ -255,8 +266,7 @@ def test_host_entry_point_copies_the_first_rows_back_early():
         xh, plan_h, _ = run_equation(eq, mom.VARIANT_3XTF32, chain, terms, via="host")
         assert np.array_equal(xd, xh)
         assert plan_h.last_launch_count() == plan.last_launch_count() + 1
-        rows = np.sort(np.random.default_rng(8).choice(n, size=24, replace=False))
-        check_against_oracle(eq, xh, plan_h, chain, terms, rows=rows)
+        check_against_oracle(eq, xh, plan_h, chain, terms, rows=stratified_rows(n, 8))
 
 
 def test_host_entry_point_starts_on_the_first_rows_of_a_left_operand_still_on_its_way():
@@ -274,8 +284,7 @@ def test_host_entry_point_starts_on_the_first_rows_of_a_left_operand_still_on_it
         assert plan_h.last_launch_count() == plan.last_launch_count() + 3
         xh2, _, _ = run_equation(eq, mom.VARIANT_3XTF32, chain, terms, via="host")       # events and pieces are reusable
         assert np.array_equal(xd, xh2)
-        rows = np.sort(np.random.default_rng(9).choice(n, size=24, replace=False))
-        check_against_oracle(eq, xh, plan_h, chain, terms, rows=rows)
+        check_against_oracle(eq, xh, plan_h, chain, terms, rows=stratified_rows(n, 9))
     # two chains write X one after the other: the first one's rows are not final when its product ends, so nothing is
     # copied back early; the stored A is the left factor of both roots: A*(U*B) + A*L
     n = 2048
@@ -284,7 +293,7 @@ def test_host_entry_point_starts_on_the_first_rows_of_a_left_operand_still_on_it
     xd, plan_d, arrays = run_expression(ex, mom.VARIANT_3XTF32, via="device")
     xh, plan_h, _ = run_expression(ex, mom.VARIANT_3XTF32, via="host")
     assert np.array_equal(xd, xh) and plan_h.last_launch_count() == plan_d.last_launch_count()
-    check_expression_against_oracle(ex, xh, plan_h, arrays, sample_rows=np.arange(0, n, 97))
+    check_expression_against_oracle(ex, xh, plan_h, arrays, sample_rows=stratified_rows(n, 10))
 
 
 @pytest.mark.parametrize("variant", VARIANTS, ids=VNAME.get)
@@ -368,13 +377,11 @@ def test_transposed_operands_large_sampled_rows():
                   chain_t=(True, True))
     x, plan, (chain, add) = run_equation(eq, mom.VARIANT_3XTF32)
     assert plan.step(0).uses_tensor_cores == 1 and plan.step(0).lhs_property == U
-    rows = np.sort(np.random.default_rng(4).choice(m, size=32, replace=False))
-    check_against_oracle(eq, x, plan, chain, add, rows=rows)
+    check_against_oracle(eq, x, plan, chain, add, rows=stratified_rows(m, 4))
 
 
 def test_config_transposed_full_size_sampled_rows():
     eq = wl.config_transposed()
     x, plan, (chain, add) = run_equation(eq, mom.VARIANT_3XTF32)
     assert plan.parenthesization() == "(0^T*(1*(2^T*3)))"
-    rows = np.sort(np.random.default_rng(6).choice(4096, size=32, replace=False))
-    check_against_oracle(eq, x, plan, chain, add, rows=rows)
+    check_against_oracle(eq, x, plan, chain, add, rows=stratified_rows(4096, 6))

@@ -8,7 +8,7 @@ from oracle import plan as op
 from oracle import values as ov
 import workloads as wl
 from workloads import Operand, SumEquation, GENERAL as G, LOWER_TRI as L, UPPER_TRI as U, IDENTITY as I
-from gpu_util import run_sum_equation, check_sum_against_oracle, TOL
+from gpu_util import run_sum_equation, check_sum_against_oracle, stratified_rows, TOL
 
 pytestmark = pytest.mark.gpu
 
@@ -158,9 +158,7 @@ def test_sum_through_the_host_entry_point():
 @pytest.mark.parametrize("eq", [wl.config_sum_shared(), wl.config_sum_triangular()], ids=lambda e: e.name)
 def test_sum_configurations_full_size_sampled_rows(eq):
     x, plan, arrays = run_sum_equation(eq, mom.VARIANT_3XTF32)
-    rows = np.random.default_rng(5).choice(x.shape[0], size=24, replace=False)
-    rows = np.sort(np.concatenate([rows, [0, x.shape[0] - 1]]))
-    check_sum_against_oracle(eq, x, plan, arrays, rows=rows)
+    check_sum_against_oracle(eq, x, plan, arrays, rows=stratified_rows(x.shape[0], 5, extra=[0, x.shape[0] - 1]))
 
 
 @pytest.mark.parametrize("variant", [mom.VARIANT_3XTF32, mom.VARIANT_3XTF32_FORCE])

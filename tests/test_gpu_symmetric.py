@@ -9,7 +9,7 @@ import paper_2208_10391_b200 as mom
 import workloads as wl
 from workloads import (GENERAL as G, LOWER_TRI as L, UPPER_TRI as U, IDENTITY as I, DIAGONAL as D, SYMMETRIC as S, Operand,
                        Equation, SumEquation)
-from gpu_util import run_equation, check_against_oracle, run_sum_equation, check_sum_against_oracle
+from gpu_util import run_equation, check_against_oracle, run_sum_equation, check_sum_against_oracle, stratified_rows
 
 pytestmark = pytest.mark.gpu
 
@@ -72,9 +72,7 @@ def test_large_gram_product_is_mirrored(shape, terms):
     steps = plan.steps()
     assert [s.kind for s in steps] == [mom.KIND_GG, mom.KIND_GRAM] and all(s.uses_tensor_cores == 1 for s in steps)
     assert plan.result_desc().property == S
-    rows = np.sort(np.random.default_rng(7).choice(n, size=40, replace=False))
-    rows[:5] = [0, 255, 256, 257, n - 1]
-    check_sum_against_oracle(eq, x, plan, arrays, rows=np.sort(rows))
+    check_sum_against_oracle(eq, x, plan, arrays, rows=stratified_rows(n, 7, extra=[0, 255, 256, 257, n - 1]))
     pair_tiles = ((n + 255) // 256) ** 2               # the CTA-pair kernel (and with it the mirroring) needs 48 tiles of 256 x 256
     if pair_tiles >= 48:
         # mirror images are exact copies: outside the 256 x 256 diagonal blocks the result is exactly symmetric

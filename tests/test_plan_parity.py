@@ -405,3 +405,44 @@ def test_expression_node_arrays_are_validated():
     assert lib.mom_expression_plan(ops, 1, leaf, 1, kids, 0, 5, 0, ctypes.byref(handle)) == mom.ERR_INVALID_ARG
     assert lib.mom_expression_plan(ops, 1, leaf, 1, kids, 0, 0, 0, ctypes.byref(handle)) == mom.OK
     lib.mom_plan_destroy(handle)
+
+
+def test_size_limits_of_the_library():
+    D = lambda r, c: (r, c, wl.GENERAL)
+    # every kernel indexes with 32-bit integers: larger dimensions are refused when the plan is made
+    big = 2 ** 31
+    with pytest.raises(mom.MomError) as e:
+        mom.mom_matrix_desc(big, 8)
+    assert e.value.status == mom.ERR_LIMIT
+    with pytest.raises(mom.MomError) as e:
+        mom.mom_equation_plan([D(8, big), D(big, 8)], [], mom.VARIANT_3XTF32)
+    assert e.value.status == mom.ERR_LIMIT
+    # the tcgen05 kernel's tile table keeps a tile's first row in 24 bits: a taller (or wider) product goes to
+    # the warp-level kernel (default variant) or the FFMA kernel (forced variant), never to the tcgen05 kernel
+    tall = 2 ** 24
+    for m, n in ((tall, 64), (64, tall), (tall - 1024 + 4, 64)):
+        for variant, want in ((mom.VARIANT_3XTF32, 2), (mom.VARIANT_3XTF32_FORCE, 0)):
+            plan = mom.mom_equation_plan([D(m, 64), D(64, n)], [], variant)
+            assert plan.step(0).uses_tensor_cores == want
+    plan = mom.mom_equation_plan([D(tall - 1024, 64), D(64, 64)], [], mom.VARIANT_3XTF32)
+    assert plan.step(0).uses_tensor_cores == 1           # m*n*k is above the size rule and the rows fit the table
+
+
+def test_planning_from_several_threads():
+    # planning is a pure function of its arguments: the same plans whether made one by one or from eight threads at once
+    import threading
+    eqs = [wl.random_equation(seed, max_len=9, max_dim=50) for seed in range(64)]
+    want = [(p.parenthesization(), p.flops()) for p in (mom.mom_equation_plan(e.descs(), e.add_descs(), mom.VARIANT_3XTF32) for e in eqs)]
+    got = [[None] * len(eqs) for _ in range(8)]
+    def work(slot):
+        for rep in range(5):
+            for i, e in enumerate(eqs):
+                p = mom.mom_equation_plan(e.descs(), e.add_descs(), mom.VARIANT_3XTF32)
+                got[slot][i] = (p.parenthesization(), p.flops())
+                del p                                      # destroys the plan (no device state was ever created)
+    threads = [threading.Thread(target=work, args=(s,)) for s in range(8)]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    assert all(g == want for g in got)
