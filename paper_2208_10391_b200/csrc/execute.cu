@@ -5,6 +5,7 @@
 #include <new>
 #include <vector>
 
+#include "batched_chain.h"
 #include "fused_small.h"
 #include "kernels.h"
 #include "mom_internal.h"
@@ -102,6 +103,62 @@ mom_status_t ensure_device_state(const mom_plan *p, int device) {
 
 bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
 
+// A plan the batched-chain kernel can run: a right-nested chain M_S * (... (M_1 * B)) of stored, untransposed
+// factors with whole 16-row blocks and a right end of 8 or 16 columns, Add terms not transposed, many instances.
+bool batched_chain_plan(const mom_plan *p, int64_t batch, const float *const *chain_ptrs, const int64_t *chain_strides,
+                        const float *const *add_ptrs, const int64_t *add_strides, float *out, int64_t out_stride,
+                        BatchedChainPlan *bp) {
+    if (!p->fused_ok || p->variant == MOM_VARIANT_FFMA || batch < BC_MIN_BATCH || p->sums.size() != 1) return false;
+    const int S = (int)p->steps.size(), n_chain = (int)p->chain.size(), n_add = (int)p->add.size();
+    if (S < 1 || S > BC_MAX_STEPS || n_add > MAX_FUSED_ADD) return false;
+    for (const Summand &sm : p->sums[0].summands)
+        if (sm.kind != SUM_STEP && sm.kind != SUM_TERM) return false;
+    for (int i = 0; i < n_add; ++i)
+        if (p->add_t[i]) return false;
+    const int n = (int)p->steps[0].pub.n;
+    if ((n != 8 && n != 16) || !p->steps[S - 1].is_last) return false;
+    std::memset(bp, 0, sizeof(*bp));
+    for (int s = 0; s < S; ++s) {
+        const mom_step_t &st = p->steps[s].pub;
+        if (st.kind == MOM_KIND_SCALE || st.kind == MOM_KIND_GRAM || p->steps[s].folded || p->steps[s].accumulate) return false;
+        if (st.lhs < 0 || st.lhs >= n_chain || st.lhs_transposed || p->chain_t[st.lhs] || p->factor_ptr[st.lhs] < 0) return false;
+        if (s == 0 ? (st.rhs < 0 || st.rhs >= n_chain || st.rhs_transposed || p->chain_t[st.rhs] || p->factor_ptr[st.rhs] < 0)
+                   : st.rhs != p->steps[s - 1].pub.out) return false;
+        if (st.m % 16 || st.m > BC_MAX_DIM || st.k % 16 || st.k > BC_MAX_DIM || st.n != n) return false;
+        const int pa = kernel_property(st.lhs_property), pb = kernel_property(st.rhs_property);
+        if (pa == MOM_DIAGONAL || pa == MOM_IDENTITY || pb == MOM_DIAGONAL || pb == MOM_IDENTITY) return false;
+        BatchedChainStep &b = bp->steps[s];
+        const int slot = p->factor_ptr[st.lhs];
+        b.lhs = chain_ptrs[slot];
+        b.lhs_stride = chain_strides ? chain_strides[slot] : 0;
+        b.m = (int)st.m;
+        b.k = (int)st.k;
+        unsigned char needed[4] = {0, 0, 0, 0};
+        for (int rb = 0; rb < b.m / 16; ++rb) {
+            int klo, khi;
+            tile_k_range(pa, pb, 16 * rb, 16 * rb + 16, 0, n, b.k, &klo, &khi);
+            for (int c = klo / 16; c < (khi + 15) / 16; ++c) needed[rb] |= (unsigned char)(1u << c);
+        }
+        batched_chain_assign(needed, b.m / 16, &b);
+    }
+    const int rslot = p->factor_ptr[p->steps[0].pub.rhs];
+    bp->n_steps = S;
+    bp->rhs = chain_ptrs[rslot];
+    bp->rhs_stride = chain_strides ? chain_strides[rslot] : 0;
+    bp->n = n;
+    bp->add.count = n_add;
+    bp->add.rows = (int)p->result_desc.rows;
+    for (int i = 0; i < n_add; ++i) {
+        bp->add.ptr[i] = p->add[i].property == MOM_IDENTITY ? nullptr : add_ptrs[i];
+        bp->add.stride[i] = add_strides ? add_strides[i] : 0;
+    }
+    bp->out = out;
+    bp->out_stride = out_stride;
+    bp->pout = kernel_property(p->result_desc.property);
+    bp->batch = batch;
+    return true;
+}
+
 struct Operand { const float *ptr; long long stride; };
 
 mom_status_t execute_impl(const mom_plan *p, const float *const *chain_ptrs, const int64_t *chain_strides,
@@ -179,6 +236,13 @@ mom_status_t execute_impl(const mom_plan *p, const float *const *chain_ptrs, con
     if (p->fused_ok) {
         for (int i = 0; i < n_ptrs; ++i) need_slot(i);
         need_summands(p->sums.back());
+        BatchedChainPlan bp;
+        if (batched_chain_plan(p, batch, chain_ptrs, chain_strides, add_ptrs, add_strides, out, out_stride, &bp)) {
+            // many instances of a right-nested chain: two warps per instance, operands streamed through registers
+            if (launch_batched_chain(bp, stream) != cudaSuccess) return MOM_ERR_CUDA;
+            p->last_launches = 1;
+            return MOM_OK;
+        }
         FusedPlan fp;
         std::memset(&fp, 0, sizeof(fp));
         fp.n_ops = (int)p->kept.size();

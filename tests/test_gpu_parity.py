@@ -182,6 +182,55 @@ def test_batched_small_chains(n, variant):
         both(eq, variant)
 
 
+BATCHED_CHAINS = {
+    # name: (chain of (rows, cols, property), Add terms, instances): right-nested plans with a right end of 8 or 16 columns
+    "LAB_plus_C": (((64, 64, L), (64, 64, G), (64, 16, G)), ((64, 16, G),), 300),
+    "UAB": (((64, 64, U), (64, 64, G), (64, 16, G)), (), 257),
+    "one_product_n8": (((48, 32, G), (32, 8, G)), ((48, 8, G), (48, 8, G)), 513),
+    "four_products": (((32, 64, G), (64, 64, L), (64, 48, G), (48, 48, U), (48, 16, G)), ((32, 16, G),), 260),
+    "square_result": (((16, 16, L), (16, 16, L)), ((16, 16, I), (16, 16, L)), 1000),
+    "upper_right_end": (((64, 16, G), (16, 16, U), (16, 16, U)), (), 256),
+    "mixed_heights": (((16, 48, G), (48, 64, G), (64, 64, L), (64, 8, G)), ((16, 8, G), (16, 8, G), (16, 8, G)), 333),
+}
+
+
+@pytest.mark.parametrize("variant", [mom.VARIANT_3XTF32], ids=VNAME.get)
+@pytest.mark.parametrize("name", sorted(BATCHED_CHAINS))
+def test_batched_right_nested_chains(name, variant):
+    # many instances of M_S*(...(M_1*B)) with whole 16-row blocks: the kernel that gives two warps to each instance and
+    # streams the factors through registers; every instance compared with the oracle
+    chain, add, batch = BATCHED_CHAINS[name]
+    dist = lambda p: "uniform" if p != G else "normal"
+    eq = Equation(f"batched_chain_{name}", 50, tuple(Operand(r, c, p, dist(p)) for r, c, p in chain),
+                  tuple(Operand(r, c, p, dist(p)) for r, c, p in add), batch=batch)
+    _, x, plan = both(eq, variant)
+    assert plan.last_launch_count() == 1
+    # fewer instances than the kernel is worth: the one-CTA-per-instance kernel gives the same values within the bound
+    small = Equation(f"batched_chain_{name}_few", 50, eq.chain, eq.add, batch=7)
+    both(small, variant)
+
+
+def test_batched_chain_with_padding_and_poisoned_gaps():
+    # instance strides larger than the matrices, NaNs in the gaps: nothing outside an instance is read or written
+    eq = wl.config_batched(batch=384)
+    chain, add = wl.generate(eq)
+    plan = mom.mom_equation_plan(eq.descs(), eq.add_descs(), mom.VARIANT_3XTF32)
+    pad = 12
+    def padded(a):
+        flat = np.full((a.shape[0], a[0].size + pad), np.nan, dtype=np.float32)
+        flat[:, :a[0].size] = a.reshape(a.shape[0], -1)
+        return torch.from_numpy(flat).cuda()
+    dc, da = [padded(a) for a in chain], [padded(a) for a in add]
+    out = torch.full((384, 64 * 16 + pad), float("nan"), dtype=torch.float32, device="cuda")
+    plan.execute_batched([t.data_ptr() for t in dc], [t.shape[1] for t in dc], [t.data_ptr() for t in da],
+                         [t.shape[1] for t in da], out.data_ptr(), out.shape[1], 384, None, 0,
+                         torch.cuda.current_stream().cuda_stream)
+    torch.cuda.synchronize()
+    o = out.cpu().numpy()
+    assert np.isnan(o[:, 64 * 16:]).all()
+    check_against_oracle(eq, o[:, :64 * 16].reshape(384, 64, 16), plan, chain, add)
+
+
 @pytest.mark.parametrize("variant", VARIANTS, ids=VNAME.get)
 def test_batched_with_padding_between_instances(variant):
     eq = wl.config_batched(batch=5)
