@@ -399,7 +399,8 @@ def run_gpu(args):
         cfg = cfgs[args.only]
         r = time_equation(mom, torch, cfg, variant, steps=args.steps, warmup=args.warmup, stream=stream,
                           timing=getattr(cfg, "batch", 1) == 1)
-        print(json.dumps({"workload": cfg.name, "variant": args.variant, "ms": r["ms"], "useful_flops": r["useful_flops"],
+        print(json.dumps({"workload": cfg.name, "variant": args.variant, "ms": r["ms"], "ms_back_to_back": r["ms_back_to_back"],
+                          "useful_flops": r["useful_flops"],
                           "launches": r["launches"], "step_times_ms": r["step_times"][-1:] }))
         return
 

@@ -11,9 +11,9 @@
 //     one 16-byte load per row, every 32-byte sector fully used -- and the right operand's fragments follow the
 //     same renumbering.  The loads of the next product's (or the next instance's) left factor are issued before
 //     the current block is multiplied, so each warp keeps up to sixteen 16-byte loads in flight all the time.
-//   - The right end B is fetched the same way (scalar loads, whole sectors); an intermediate is written to a
-//     4.5 KB shared-memory buffer of the pair in accumulator layout and read back as the next product's right
-//     fragments (padded rows: conflict-free).
+//   - The right end B of the NEXT instance is copied asynchronously (cp.async) into a 4.5 KB shared-memory buffer of
+//     the pair while the current instance is multiplied; an intermediate is written to such a buffer in accumulator
+//     layout; both are read back as right fragments (rows padded by two floats: conflict-free).
 //   - Blocks of 16 x 16 that lie outside a triangular factor's structure are neither loaded nor multiplied.
 //   - 3xTF32 on the fragments: a = hi + lo, accumulate lo*hi + hi*lo + hi*hi in f32 (hi rounded to tf32 on the bit
 //     pattern; lo = a - hi handed over unrounded: the MMA ignores the bits below tf32, worth at most 2^-21 of a,
@@ -33,7 +33,7 @@ namespace {
 
 constexpr int BC_THREADS = 128;                 // four warps: two instances in flight per CTA
 constexpr int BC_PAIRS = BC_THREADS / 64;
-constexpr int BC_CTAS_PER_SM = 3;
+constexpr int BC_CTAS_PER_SM = 4;
 constexpr int T_PAD = 2;                        // extra floats per row of an intermediate in shared memory
 constexpr int T_FLOATS = BC_MAX_DIM * (BC_MAX_N + T_PAD);
 
@@ -42,10 +42,11 @@ __device__ __forceinline__ float4 load_once_f4(const float *p) {     // streamed
     asm volatile("ld.global.nc.L1::no_allocate.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(p));
     return v;
 }
-__device__ __forceinline__ float load_once_f1(const float *p) {
-    float v;
-    asm volatile("ld.global.nc.f32 %0, [%1];" : "=f"(v) : "l"(p));
-    return v;
+__device__ __forceinline__ void copy_async_8(float *dst_shared, const float *src) {
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"((uint32_t)__cvta_generic_to_shared(dst_shared)), "l"(src) : "memory");
+}
+__device__ __forceinline__ void copy_async_wait_all() {
+    asm volatile("cp.async.commit_group;\n\tcp.async.wait_group 0;" ::: "memory");
 }
 __device__ __forceinline__ float2 load_once_f2(const float *p) {
     float2 v;
@@ -69,7 +70,8 @@ __device__ __forceinline__ void mma_tf32(float (&d)[4], const uint32_t (&a)[4], 
 template <int NT>
 __global__ void __launch_bounds__(BC_THREADS, BC_CTAS_PER_SM)
 batched_chain_kernel(const BatchedChainPlan bp) {
-    __shared__ __align__(16) float tbuf[BC_PAIRS][2][T_FLOATS];
+    __shared__ __align__(16) float tbuf[BC_PAIRS][2][T_FLOATS];      // intermediates: product s reads [s & 1], writes [(s + 1) & 1]
+    __shared__ __align__(16) float bbuf[BC_PAIRS][2][T_FLOATS];      // the right end B of this instance and of the next
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
     const int pair = warp >> 1, w = warp & 1;
     constexpr int LD = 8 * NT + T_PAD;
@@ -78,7 +80,6 @@ batched_chain_kernel(const BatchedChainPlan bp) {
     long long inst = (long long)blockIdx.x * BC_PAIRS + pair;
 
     float4 buf[2][4][2];             // [slot][16-column chunk][row g / row g + 8] of the left factor
-    float bfrag[4][2][2][NT];        // the right end B as fragments: [chunk][k-step][entry][column tile]
 
     // 16-byte loads of one row block of a left factor (only the chunks that its structure needs)
     auto issue_lhs = [&](auto slot, int s, long long at) {
@@ -96,25 +97,19 @@ batched_chain_kernel(const BatchedChainPlan bp) {
                 buf[q][c][1] = load_once_f4(row1 + 16 * c);
             }
     };
-    // the right end of instance `at`, in the renumbered fragment order (see the head of the file)
-    auto issue_rhs = [&](long long at) {
-        const float *b = bp.rhs + at * bp.rhs_stride + g;
-        const int chunks = bp.steps[0].k >> 4;
-#pragma unroll
-        for (int c = 0; c < 4; ++c)
-            if (c < chunks) {
-#pragma unroll
-                for (int j = 0; j < 2; ++j)
-#pragma unroll
-                    for (int e = 0; e < 2; ++e)
-#pragma unroll
-                        for (int nt = 0; nt < NT; ++nt)
-                            bfrag[c][j][e][nt] = load_once_f1(b + (16 * c + 4 * t + 2 * j + e) * (8 * NT) + 8 * nt);
-            }
+    // this warp's half of the right end of instance `at`, 8 bytes per copy (the padded rows are 8-byte aligned)
+    auto issue_rhs = [&](long long at, int parity) {
+        const float *b = bp.rhs + at * bp.rhs_stride;
+        float *dst = bbuf[pair][parity];
+        const int pieces = bp.steps[0].k * 4 * NT;
+        for (int p = 32 * w + lane; p < pieces; p += 64) {
+            const int row = p / (4 * NT), col = 2 * (p % (4 * NT));
+            copy_async_8(dst + row * LD + col, b + row * (8 * NT) + col);
+        }
     };
 
     // one row block of product s: multiply, then hand the block on (intermediate) or finish it (X)
-    auto process = [&](auto slot, int s, long long at) {
+    auto process = [&](auto slot, int s, long long at, int parity) {
         constexpr int q = decltype(slot)::value;
         const BatchedChainStep &st = bp.steps[s];
         const int rb = st.rb[w][q];
@@ -138,26 +133,18 @@ batched_chain_kernel(const BatchedChainPlan bp) {
         for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
             for (int i = 0; i < 4; ++i) acc[nt][i] = 0.0f;
-        const float *rhs_t = tbuf[pair][s & 1];
+        const float *rhs = s == 0 ? bbuf[pair][parity] : tbuf[pair][s & 1];
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
             if (!((mask >> c) & 1u)) continue;
+            // right fragments in the renumbered order: k-step j, entry e is row 16 c + 4 t + 2 j + e
             float b[2][2][NT];
-            if (s == 0) {
 #pragma unroll
-                for (int j = 0; j < 2; ++j)
+            for (int j = 0; j < 2; ++j)
 #pragma unroll
-                    for (int e = 0; e < 2; ++e)
+                for (int e = 0; e < 2; ++e)
 #pragma unroll
-                        for (int nt = 0; nt < NT; ++nt) b[j][e][nt] = bfrag[c][j][e][nt];
-            } else {
-#pragma unroll
-                for (int j = 0; j < 2; ++j)
-#pragma unroll
-                    for (int e = 0; e < 2; ++e)
-#pragma unroll
-                        for (int nt = 0; nt < NT; ++nt) b[j][e][nt] = rhs_t[(16 * c + 4 * t + 2 * j + e) * LD + g + 8 * nt];
-            }
+                    for (int nt = 0; nt < NT; ++nt) b[j][e][nt] = rhs[(16 * c + 4 * t + 2 * j + e) * LD + g + 8 * nt];
             const float4 v0 = buf[q][c][0], v1 = buf[q][c][1];
 #pragma unroll
             for (int j = 0; j < 2; ++j) {
@@ -227,13 +214,17 @@ batched_chain_kernel(const BatchedChainPlan bp) {
 
     using Slot0 = std::integral_constant<int, 0>;
     using Slot1 = std::integral_constant<int, 1>;
+    int parity = 0;
     if (inst < bp.batch) {
-        issue_rhs(inst);
+        issue_rhs(inst, 0);
         issue_lhs(Slot0{}, 0, inst);
         issue_lhs(Slot1{}, 0, inst);
+        copy_async_wait_all();
     }
-    for (; inst < bp.batch; inst += pairs_total) {
+    pair_barrier(pair);                                  // both halves of B are in place
+    for (; inst < bp.batch; inst += pairs_total, parity ^= 1) {
         const long long next_inst = inst + pairs_total;
+        if (next_inst < bp.batch) issue_rhs(next_inst, parity ^ 1);
 #pragma unroll 1
         for (int s = 0; s < S; ++s) {
             // what this warp loads next: the following product of this instance, or the first one of its next instance
@@ -241,13 +232,13 @@ batched_chain_kernel(const BatchedChainPlan bp) {
             const int ns = wraps ? 0 : s + 1;
             const long long ni = wraps ? next_inst : inst;
             const bool more = ni < bp.batch;
-            process(Slot0{}, s, inst);
+            process(Slot0{}, s, inst, parity);
             if (more) issue_lhs(Slot0{}, ns, ni);
-            process(Slot1{}, s, inst);
+            process(Slot1{}, s, inst, parity);
             if (more) issue_lhs(Slot1{}, ns, ni);
-            if (s == 0 && next_inst < bp.batch) issue_rhs(next_inst);
-            // the intermediate changes hands (and, after the last product, its buffer may be written again)
-            if (S > 1) pair_barrier(pair);
+            // the intermediate changes hands; after the last product the next instance's B must have landed
+            if (wraps) copy_async_wait_all();
+            pair_barrier(pair);
         }
     }
 }
