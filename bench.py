@@ -283,8 +283,9 @@ def planning_us(mom, eq, variant, repeats=15):
     return statistics.median(ts)
 
 
-def time_equation(mom, torch, eq, variant, steps, warmup, stream, timing=False):
-    """Device-resident timing of one configuration: returns dict with per-step ms list, plan, launches."""
+def time_equation(mom, torch, eq, variant, steps, warmup, stream, timing=False, chain_storage=None):
+    """Device-resident timing of one configuration: returns dict with per-step ms list, plan, launches.
+    chain_storage (plain chains only): mom.STORAGE_PACKED entries hand that triangular operand over as a packed container."""
     if isinstance(eq, wl.Expression):
         # a nested expression: one pointer per operand of the table
         chain, add = wl.generate_expression(eq), []
@@ -303,6 +304,12 @@ def time_equation(mom, torch, eq, variant, steps, warmup, stream, timing=False):
         dchain = [None if a is None else by_name[nm] for row, names in zip(arrays, eq.names) for a, nm in zip(row, names)]
         chain, add = [a for row in arrays for a in row], []
         eq = wl.Equation(eq.name, eq.seed, tuple(o for c in eq.chains for o in c))     # batch 1, for the code below
+    elif chain_storage is not None:
+        chain, add = wl.generate(eq)
+        plan = mom.mom_equation_plan_stored(eq.descs(), eq.chain_t, chain_storage, eq.add_descs(), eq.add_t, None, mom.STORAGE_DENSE, variant)
+        lower = (wl.LOWER_TRI, wl.STRICT_LOWER, wl.UNIT_LOWER)
+        chain = [a if s == mom.STORAGE_DENSE or a is None else wl.pack_triangle(a, o.prop in lower) for a, o, s in zip(chain, eq.chain, chain_storage)]
+        dchain = [None if a is None else torch.from_numpy(a).cuda() for a in chain]
     else:
         chain, add = wl.generate(eq)
         plan = mom.mom_equation_plan_transposed(eq.descs(), eq.chain_t, eq.add_descs(), eq.add_t, variant)
@@ -359,7 +366,8 @@ def time_equation(mom, torch, eq, variant, steps, warmup, stream, timing=False):
     if status != (0, 0):
         raise RuntimeError(f"device-side wait timed out: {status}")
     mul, addf = plan.flops()
-    return {"ms": ms, "ms_back_to_back": ms_b2b, "plan": plan, "useful_flops": (mul + addf) * eq.batch, "launches": plan.last_launch_count(),
+    stored_bytes = 4 * (sum(t.numel() for t in dchain if t is not None) + sum(t.numel() for t in dadd if t is not None) + out.numel())
+    return {"ms": ms, "ms_back_to_back": ms_b2b, "plan": plan, "stored_bytes": stored_bytes, "useful_flops": (mul + addf) * eq.batch, "launches": plan.last_launch_count(),
             "step_times": step_times, "host": (chain, add), "keep": (dchain, dadd, out, ws)}
 
 
@@ -587,11 +595,27 @@ def run_gpu(args):
                      "launches": r["launches"], "plan_us": planning_us(mom, cfg, variant)}
             if batch > 1:
                 per_inst = sum(o.rows * o.cols for o in list(cfg.chain) + list(cfg.add)) + rd_elems(r["plan"])
+                entry["bytes_per_instance"] = per_inst * 4
                 entry["hbm_gbs_at_median"] = per_inst * 4 * cfg.batch / (ms_med * 1e-3) / 1e9
                 entry["hbm_frac_of_measured_peak"] = entry["hbm_gbs_at_median"] / peaks["hbm_gbs"]
             others.append(entry)
             del r
             torch.cuda.empty_cache()
+            if batch > 1 and args.variant == "3xtf32":
+                # the same equations with L_i handed over as a packed triangle (2176 instead of 4096 entries per instance)
+                storage = [mom.STORAGE_PACKED if o.prop == wl.LOWER_TRI else mom.STORAGE_DENSE for o in cfg.chain]
+                r = time_equation(mom, torch, cfg, variant, steps=20, warmup=3, stream=stream, chain_storage=storage)
+                ms_med = statistics.median(r["ms"])
+                per_inst = r["stored_bytes"] // cfg.batch
+                others.append({"workload": cfg.name + "_packedL", "parenthesization": r["plan"].parenthesization(),
+                               "useful_flops": r["useful_flops"], "ms_min_of_20": min(r["ms"]), "ms_median": ms_med,
+                               "ms_back_to_back": r["ms_back_to_back"], "launches": r["launches"],
+                               "workspace_bytes": r["plan"].workspace_bytes(cfg.batch), "bytes_per_instance": per_inst,
+                               "hbm_gbs_at_median": per_inst * cfg.batch / (ms_med * 1e-3) / 1e9,
+                               "hbm_frac_of_measured_peak": per_inst * cfg.batch / (ms_med * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                               "dense_bytes_frac_of_measured_peak": entry["bytes_per_instance"] * cfg.batch / (ms_med * 1e-3) / 1e9 / peaks["hbm_gbs"]})
+                del r
+                torch.cuda.empty_cache()
         result["all_configs"] = others
 
         # ---- the FFMA comparison variant on the property-heavy configuration, against the FP32 FMA peak

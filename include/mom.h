@@ -197,6 +197,45 @@ mom_status_t mom_equation_plan_transposed(const mom_matrix_desc_t *chain, const 
                                           const mom_matrix_desc_t *add_terms, const int32_t *add_transposed, int32_t n_add,
                                           mom_variant_t variant, mom_plan_t **out_plan);
 
+/* Storage of a matrix in device (or host) memory.  The paper materialises every matrix as a dense buffer and names
+ * "more appropriate containers" as future work (Section 2, "Matrix Attribute"; the conclusion speaks of
+ * non-rectangular iteration spaces).  MOM_STORAGE_PACKED is such a container for triangular matrices (lowerTri,
+ * upperTri and their strict and unit kinds): only the triangle is kept, row by row, every stored row a whole number
+ * of 16-byte groups so that rows stay addressable by 16-byte accesses:
+ *     lower triangle, n x n: row i holds columns [0, 4 * (i / 4 + 1))
+ *     upper triangle, n x n: row i holds columns [4 * (i / 4), n rounded up to a multiple of 4)
+ * Rows follow each other without gaps.  The stored entries outside the triangle (fewer than four per row, next to
+ * the diagonal) and those beyond column n - 1 are padding: zeros in operands (the library relies on it), +0.0f in
+ * results.  A packed n x n triangle takes about n (n + 4) / 2 entries instead of n * n. */
+typedef enum { MOM_STORAGE_DENSE = 0, MOM_STORAGE_PACKED = 1 } mom_storage_t;
+
+/* Size of the packed container of a rows x rows triangle with the given property, in f32 entries, and where row
+ * `row` sits in it: *offset = position of its first stored entry, columns [*first_col, *end_col).
+ * Errors: INVALID_ARG (NULL, rows < 1, row outside [0, rows)), PROPERTY (not a triangular property), LIMIT. */
+mom_status_t mom_packed_elements(int64_t rows, mom_property_t property, int64_t *elements);
+mom_status_t mom_packed_row(int64_t rows, mom_property_t property, int64_t row, int64_t *offset, int64_t *first_col,
+                            int64_t *end_col);
+
+/* mom_equation_plan_transposed with a storage per operand, per Add term and for the result.
+ *   chain_storage / add_storage   host arrays of mom_storage_t (NULL: all dense); a packed operand must be triangular
+ *   result_storage                MOM_STORAGE_PACKED: X is written as a packed triangle; the equation's inferred
+ *                                 result type must then be triangular (PROPERTY otherwise)
+ * Descriptors still describe the matrices as stored (a packed lower triangle used transposed takes part as an upper
+ * one).  The plan is the same as for dense storage (storage changes neither costs nor parenthesization).  Execution:
+ * the operand-split pass of the tcgen05 kernel and the batched small-chain kernel read packed operands in place, and
+ * the tcgen05 kernel writes a packed X in place (tiles outside the triangle are not written at all); every other
+ * kernel gets a dense copy in the workspace (one unpacking pass per packed operand) or leaves a dense X there that a
+ * packing pass copies out -- mom_plan_workspace_bytes includes that room.  In mom_equation_execute_batched the
+ * instance stride of a packed matrix must be at least its packed size (and a multiple of 4).
+ * Errors: those of mom_equation_plan_transposed, PROPERTY (packed storage of a matrix that is not triangular). */
+mom_status_t mom_equation_plan_stored(const mom_matrix_desc_t *chain, const int32_t *chain_transposed, const int32_t *chain_storage,
+                                      int32_t n_chain, const mom_matrix_desc_t *add_terms, const int32_t *add_transposed,
+                                      const int32_t *add_storage, int32_t n_add, mom_storage_t result_storage,
+                                      mom_variant_t variant, mom_plan_t **out_plan);
+
+/* Number of f32 entries of X as the plan writes it: rows * cols of the result descriptor, or the packed size. */
+mom_status_t mom_plan_result_elements(const mom_plan_t *plan, int64_t *elements);
+
 /* Plan a sum of several Mul chains, X = prod(chain_0) + prod(chain_1) + ... (paper Section 2, "Operations":
  * Mul and Add are both variadic and one Equation holds a bag of them).  A chain of one factor is a plain Add term.
  *   factors            host array with all chains' factors one after the other, AS STORED (n = sum of chain_lengths)

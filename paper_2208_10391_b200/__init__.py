@@ -16,6 +16,7 @@ GENERAL, LOWER_TRI, UPPER_TRI, IDENTITY, DIAGONAL, SYMMETRIC = 0, 1, 2, 3, 4, 5
 STRICT_LOWER, STRICT_UPPER, UNIT_LOWER, UNIT_UPPER = 6, 7, 8, 9
 F32 = 0
 VARIANT_3XTF32, VARIANT_FFMA, VARIANT_3XTF32_FORCE, VARIANT_3XTF32_WARP = 0, 1, 2, 3
+STORAGE_DENSE, STORAGE_PACKED = 0, 1
 KIND_GG, KIND_TG, KIND_GT, KIND_TT, KIND_TTMIX, KIND_SCALE, KIND_GRAM = 0, 1, 2, 3, 4, 5, 6
 
 (OK, ERR_INVALID_ARG, ERR_PROPERTY, ERR_DTYPE, ERR_SHAPE_MISMATCH, ERR_OVERFLOW, ERR_ALLOC,
@@ -69,6 +70,13 @@ _sigs = {
     "mom_equation_plan_transposed": [ctypes.POINTER(MatrixDesc), ctypes.POINTER(ctypes.c_int32), ctypes.c_int32,
                                      ctypes.POINTER(MatrixDesc), ctypes.POINTER(ctypes.c_int32), ctypes.c_int32,
                                      ctypes.c_int, ctypes.POINTER(_P)],
+    "mom_packed_elements": [ctypes.c_int64, ctypes.c_int, ctypes.POINTER(ctypes.c_int64)],
+    "mom_packed_row": [ctypes.c_int64, ctypes.c_int, ctypes.c_int64, ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_int64),
+                       ctypes.POINTER(ctypes.c_int64)],
+    "mom_equation_plan_stored": [ctypes.POINTER(MatrixDesc), ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_int32), ctypes.c_int32,
+                                 ctypes.POINTER(MatrixDesc), ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_int32), ctypes.c_int32,
+                                 ctypes.c_int, ctypes.c_int, ctypes.POINTER(_P)],
+    "mom_plan_result_elements": [_P, ctypes.POINTER(ctypes.c_int64)],
     "mom_equation_plan_sum": [ctypes.POINTER(MatrixDesc), ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_int32),
                               ctypes.POINTER(ctypes.c_int32), ctypes.c_int32, ctypes.c_int, ctypes.POINTER(_P)],
     "mom_plan_reused_products": [_P, ctypes.POINTER(ctypes.c_int32)],
@@ -272,6 +280,12 @@ class Plan:
         _check(_lib.mom_plan_host_staging_bytes(self._h, batch, ctypes.byref(b)), "mom_plan_host_staging_bytes")
         return b.value
 
+    def result_elements(self) -> int:
+        """f32 entries of X as the plan writes it (rows * cols, or the packed size)."""
+        n = ctypes.c_int64()
+        _check(_lib.mom_plan_result_elements(self._h, ctypes.byref(n)), "mom_plan_result_elements")
+        return n.value
+
     def host_upload_bytes(self, batch: int = 1) -> int:
         b = ctypes.c_size_t()
         _check(_lib.mom_plan_host_upload_bytes(self._h, batch, ctypes.byref(b)), "mom_plan_host_upload_bytes")
@@ -350,6 +364,40 @@ def mom_equation_plan_transposed(chain: Sequence, chain_transposed: Optional[Seq
                                            variant, ctypes.byref(handle))
     _check(st, "mom_equation_plan_transposed")
     return Plan(handle.value, n_chain, n_add)
+
+
+def mom_equation_plan_stored(chain: Sequence, chain_transposed: Optional[Sequence], chain_storage: Optional[Sequence],
+                             add_terms: Sequence = (), add_transposed: Optional[Sequence] = None,
+                             add_storage: Optional[Sequence] = None, result_storage: int = STORAGE_DENSE,
+                             variant: int = VARIANT_3XTF32) -> Plan:
+    """As mom_equation_plan_transposed, with a storage (dense or packed triangle) per operand, per Add term and for X."""
+    handle = _P()
+    n_chain, n_add = len(chain), len(add_terms)
+
+    def ints(f, n):
+        if f is None or n == 0:
+            return None
+        f = list(f) + [0] * (n - len(f))
+        return (ctypes.c_int32 * n)(*[int(x) for x in f])
+    st = _lib.mom_equation_plan_stored(_desc_array(chain) if n_chain else None, ints(chain_transposed, n_chain), ints(chain_storage, n_chain),
+                                       n_chain, _desc_array(add_terms) if n_add else None, ints(add_transposed, n_add),
+                                       ints(add_storage, n_add), n_add, int(result_storage), variant, ctypes.byref(handle))
+    _check(st, "mom_equation_plan_stored")
+    return Plan(handle.value, n_chain, n_add)
+
+
+def mom_packed_elements(rows: int, prop: int) -> int:
+    """f32 entries of the packed container of a rows x rows triangle."""
+    n = ctypes.c_int64()
+    _check(_lib.mom_packed_elements(rows, prop, ctypes.byref(n)), "mom_packed_elements")
+    return n.value
+
+
+def mom_packed_row(rows: int, prop: int, row: int) -> Tuple[int, int, int]:
+    """(offset, first column, end column) of row `row` in the packed container."""
+    off, first, end = ctypes.c_int64(), ctypes.c_int64(), ctypes.c_int64()
+    _check(_lib.mom_packed_row(rows, prop, row, ctypes.byref(off), ctypes.byref(first), ctypes.byref(end)), "mom_packed_row")
+    return off.value, first.value, end.value
 
 
 def mom_equation_plan_sum(chains: Sequence[Sequence], transposed: Optional[Sequence[Sequence]] = None,

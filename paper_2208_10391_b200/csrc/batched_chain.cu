@@ -26,6 +26,7 @@
 
 #include "batched_chain.h"
 #include "device_info.h"
+#include "packed.cuh"
 
 namespace mom {
 
@@ -88,6 +89,20 @@ batched_chain_kernel(const BatchedChainPlan bp) {
         const int rb = st.rb[w][q];
         if (rb < 0) return;
         const unsigned mask = st.chunks[w][q];
+        if (st.packed) {
+            // a packed triangle: each row's stored columns start at its own offset; what the container does not hold
+            // (beyond the diagonal's group of four) is zero and is not loaded
+            const PackedRow p0 = packed_row(st.packed == 1, st.m, 16 * rb + g), p1 = packed_row(st.packed == 1, st.m, 16 * rb + g + 8);
+            const float *row0 = st.lhs + at * st.lhs_stride + p0.offset - p0.first, *row1 = st.lhs + at * st.lhs_stride + p1.offset - p1.first;
+#pragma unroll
+            for (int c = 0; c < 4; ++c)
+                if ((mask >> c) & 1u) {
+                    const int col = 16 * c + 4 * t;
+                    buf[q][c][0] = col >= p0.first && col < p0.end ? load_once_f4(row0 + col) : make_float4(0.f, 0.f, 0.f, 0.f);
+                    buf[q][c][1] = col >= p1.first && col < p1.end ? load_once_f4(row1 + col) : make_float4(0.f, 0.f, 0.f, 0.f);
+                }
+            return;
+        }
         const float *row0 = st.lhs + at * st.lhs_stride + (long long)(16 * rb + g) * st.k + 4 * t;
         const float *row1 = row0 + 8 * st.k;
 #pragma unroll

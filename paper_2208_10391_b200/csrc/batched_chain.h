@@ -11,12 +11,12 @@ namespace mom {
 constexpr int BC_MAX_STEPS = 4;
 constexpr int BC_MAX_DIM = 64;       // rows and contraction length of every product
 constexpr int BC_MAX_N = 16;         // columns of the right end (and of every intermediate and of X)
-constexpr long long BC_MIN_BATCH = 256;
 
 struct BatchedChainStep {
     const float *lhs;                // the left factor of this product, m x k, row-major as stored (one instance)
     long long lhs_stride;            // elements between instances
     int m, k;
+    int packed;                      // 0: dense; 1 / 2: a packed lower / upper triangle (m == k) read in place
     // work split of the step's 16-row blocks over the two warps of an instance: warp w handles row blocks
     // rb[w][0] and rb[w][1] (-1: none); chunks[w][q] has bit c set when that row block needs columns
     // [16 c, 16 c + 16) of the left factor (blocks wholly outside a triangular factor's structure are skipped)

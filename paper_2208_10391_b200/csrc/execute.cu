@@ -42,12 +42,13 @@ constexpr int TIMING_SLOTS = 32;
 
 // host-staging entry point: triangular operands of at least UPLOAD_MIN rows are uploaded in blocks of UPLOAD_BLOCK rows
 constexpr int64_t UPLOAD_BLOCK = 256, UPLOAD_MIN = 1024;
-inline bool triangular_upload(const mom_matrix_desc_t &d, int64_t batch) {
+inline bool triangular_upload(const mom_matrix_desc_t &d, int64_t batch, int32_t storage = MOM_STORAGE_DENSE) {
+    if (storage != MOM_STORAGE_DENSE) return false;          // a packed triangle crosses the bus as it is
     const int32_t kp = kernel_property(d.property);        // strict and unit triangles lie inside the ordinary one
     return batch == 1 && d.rows >= UPLOAD_MIN && (kp == MOM_LOWER_TRI || kp == MOM_UPPER_TRI);
 }
-inline size_t upload_bytes(const mom_matrix_desc_t &d, int64_t batch) {
-    if (!triangular_upload(d, batch)) return (size_t)d.rows * d.cols * sizeof(float) * batch;
+inline size_t upload_bytes(const mom_matrix_desc_t &d, int64_t batch, int32_t storage = MOM_STORAGE_DENSE) {
+    if (!triangular_upload(d, batch, storage)) return (size_t)stored_elements(d, storage) * sizeof(float) * batch;
     size_t total = 0;
     for (int64_t r0 = 0; r0 < d.rows; r0 += UPLOAD_BLOCK) {
         const int64_t r1 = std::min<int64_t>(d.rows, r0 + UPLOAD_BLOCK);
@@ -103,36 +104,32 @@ mom_status_t ensure_device_state(const mom_plan *p, int device) {
 
 bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
 
+// Per call: which of the caller's pointers are packed triangles that the kernels read (or write) in place.
+struct StorageCall {
+    std::vector<char> slot_packed;
+    bool out_packed = false;
+};
+
 // A plan the batched-chain kernel can run: a right-nested chain M_S * (... (M_1 * B)) of stored, untransposed
 // factors with whole 16-row blocks and a right end of 8 or 16 columns, Add terms not transposed, many instances.
 bool batched_chain_plan(const mom_plan *p, int64_t batch, const float *const *chain_ptrs, const int64_t *chain_strides,
                         const float *const *add_ptrs, const int64_t *add_strides, float *out, int64_t out_stride,
-                        BatchedChainPlan *bp) {
-    if (!p->fused_ok || p->variant == MOM_VARIANT_FFMA || batch < BC_MIN_BATCH || p->sums.size() != 1) return false;
-    const int S = (int)p->steps.size(), n_chain = (int)p->chain.size(), n_add = (int)p->add.size();
-    if (S < 1 || S > BC_MAX_STEPS || n_add > MAX_FUSED_ADD) return false;
-    for (const Summand &sm : p->sums[0].summands)
-        if (sm.kind != SUM_STEP && sm.kind != SUM_TERM) return false;
-    for (int i = 0; i < n_add; ++i)
-        if (p->add_t[i]) return false;
+                        BatchedChainPlan *bp, const StorageCall *sc = nullptr) {
+    if (sc && sc->out_packed) return false;
+    if (batch < BATCHED_CHAIN_MIN_BATCH || !batched_chain_shape(*p)) return false;
+    const int S = (int)p->steps.size(), n_add = (int)p->add.size();
     const int n = (int)p->steps[0].pub.n;
-    if ((n != 8 && n != 16) || !p->steps[S - 1].is_last) return false;
     std::memset(bp, 0, sizeof(*bp));
     for (int s = 0; s < S; ++s) {
         const mom_step_t &st = p->steps[s].pub;
-        if (st.kind == MOM_KIND_SCALE || st.kind == MOM_KIND_GRAM || p->steps[s].folded || p->steps[s].accumulate) return false;
-        if (st.lhs < 0 || st.lhs >= n_chain || st.lhs_transposed || p->chain_t[st.lhs] || p->factor_ptr[st.lhs] < 0) return false;
-        if (s == 0 ? (st.rhs < 0 || st.rhs >= n_chain || st.rhs_transposed || p->chain_t[st.rhs] || p->factor_ptr[st.rhs] < 0)
-                   : st.rhs != p->steps[s - 1].pub.out) return false;
-        if (st.m % 16 || st.m > BC_MAX_DIM || st.k % 16 || st.k > BC_MAX_DIM || st.n != n) return false;
         const int pa = kernel_property(st.lhs_property), pb = kernel_property(st.rhs_property);
-        if (pa == MOM_DIAGONAL || pa == MOM_IDENTITY || pb == MOM_DIAGONAL || pb == MOM_IDENTITY) return false;
         BatchedChainStep &b = bp->steps[s];
         const int slot = p->factor_ptr[st.lhs];
         b.lhs = chain_ptrs[slot];
         b.lhs_stride = chain_strides ? chain_strides[slot] : 0;
         b.m = (int)st.m;
         b.k = (int)st.k;
+        b.packed = sc && sc->slot_packed[slot] ? (pa == MOM_LOWER_TRI ? 1 : 2) : 0;
         unsigned char needed[4] = {0, 0, 0, 0};
         for (int rb = 0; rb < b.m / 16; ++rb) {
             int klo, khi;
@@ -142,6 +139,7 @@ bool batched_chain_plan(const mom_plan *p, int64_t batch, const float *const *ch
         batched_chain_assign(needed, b.m / 16, &b);
     }
     const int rslot = p->factor_ptr[p->steps[0].pub.rhs];
+    if (sc && sc->slot_packed[rslot]) return false;          // the right end is read dense
     bp->n_steps = S;
     bp->rhs = chain_ptrs[rslot];
     bp->rhs_stride = chain_strides ? chain_strides[rslot] : 0;
@@ -161,10 +159,10 @@ bool batched_chain_plan(const mom_plan *p, int64_t batch, const float *const *ch
 
 struct Operand { const float *ptr; long long stride; };
 
-mom_status_t execute_impl(const mom_plan *p, const float *const *chain_ptrs, const int64_t *chain_strides,
+mom_status_t execute_core(const mom_plan *p, const float *const *chain_ptrs, const int64_t *chain_strides,
                           const float *const *add_ptrs, const int64_t *add_strides, float *out, int64_t out_stride,
                           int64_t batch, void *workspace, size_t workspace_bytes, cudaStream_t stream,
-                          const StageEvents *staged = nullptr) {
+                          const StageEvents *staged = nullptr, const StorageCall *sc = nullptr) {
     if (!p || !chain_ptrs || !out || batch < 1) return MOM_ERR_INVALID_ARG;
     const int n_chain = (int)p->chain.size(), n_add = (int)p->add.size(), n_ptrs = (int)p->ptr_desc.size();
     if (n_add > 0 && !add_ptrs) return MOM_ERR_INVALID_ARG;
@@ -175,7 +173,8 @@ mom_status_t execute_impl(const mom_plan *p, const float *const *chain_ptrs, con
         if (p->ptr_desc[i].property == MOM_IDENTITY || !p->slot_used[i]) continue;
         if (!chain_ptrs[i]) return MOM_ERR_INVALID_ARG;
         if (!aligned16(chain_ptrs[i])) return MOM_ERR_ALIGNMENT;
-        if (batch > 1 && (chain_strides[i] % 4 != 0 || chain_strides[i] < p->ptr_desc[i].rows * p->ptr_desc[i].cols))
+        const bool in_place = sc && sc->slot_packed[i];
+        if (batch > 1 && (chain_strides[i] % 4 != 0 || chain_strides[i] < stored_elements(p->ptr_desc[i], in_place ? MOM_STORAGE_PACKED : MOM_STORAGE_DENSE)))
             return MOM_ERR_INVALID_ARG;
     }
     if (!p->names.empty()) {          // entries with one name are one matrix: a product shared between chains relies on it
@@ -192,7 +191,8 @@ mom_status_t execute_impl(const mom_plan *p, const float *const *chain_ptrs, con
         if (batch > 1 && (add_strides[i] % 4 != 0 || add_strides[i] < rows * cols)) return MOM_ERR_INVALID_ARG;
     }
     if (!aligned16(out)) return MOM_ERR_ALIGNMENT;
-    if (batch > 1 && (out_stride % 4 != 0 || out_stride < rows * cols)) return MOM_ERR_INVALID_ARG;
+    if (batch > 1 && (out_stride % 4 != 0 || out_stride < stored_elements(p->result_desc, sc && sc->out_packed ? MOM_STORAGE_PACKED : MOM_STORAGE_DENSE)))
+        return MOM_ERR_INVALID_ARG;
 
     size_t need = 0;
     mom_plan_workspace_bytes(p, batch, &need);
@@ -237,12 +237,15 @@ mom_status_t execute_impl(const mom_plan *p, const float *const *chain_ptrs, con
         for (int i = 0; i < n_ptrs; ++i) need_slot(i);
         need_summands(p->sums.back());
         BatchedChainPlan bp;
-        if (batched_chain_plan(p, batch, chain_ptrs, chain_strides, add_ptrs, add_strides, out, out_stride, &bp)) {
+        if (batched_chain_plan(p, batch, chain_ptrs, chain_strides, add_ptrs, add_strides, out, out_stride, &bp, sc)) {
             // many instances of a right-nested chain: two warps per instance, operands streamed through registers
             if (launch_batched_chain(bp, stream) != cudaSuccess) return MOM_ERR_CUDA;
             p->last_launches = 1;
             return MOM_OK;
         }
+        if (sc)                                               // the shared-memory kernel below reads dense operands only
+            for (char in_place : sc->slot_packed)
+                if (in_place) return MOM_ERR_INVALID_ARG;
         FusedPlan fp;
         std::memset(&fp, 0, sizeof(fp));
         fp.n_ops = (int)p->kept.size();
@@ -423,11 +426,12 @@ mom_status_t execute_impl(const mom_plan *p, const float *const *chain_ptrs, con
                                            stp.pub.rhs != stp.pub.lhs &&
                                            p->dev->tc.steps[s].split_a_by_part && staged->slot_head_rows[lhs_slot] == p->dev->tc.steps[s].part_row;
                 auto operand = [&](int id, int fold, const float **ptr, long long *stride, int *trans, int own_trans,
-                                   const float **scale, long long *scale_step, int *scale_rows) {
+                                   const float **scale, long long *scale_step, int *scale_rows, int *packed) {
                     if (fold < 0) {
                         if (!(lhs_in_pieces && id == stp.pub.lhs)) need_value(id);
                         const Operand o = value(id);
                         *ptr = o.ptr; *stride = o.stride; *trans = own_trans;
+                        *packed = sc && id < n_chain && p->factor_ptr[id] >= 0 && sc->slot_packed[p->factor_ptr[id]];
                         return;
                     }
                     const mom_step_t &sc = p->steps[fold].pub;
@@ -440,8 +444,9 @@ mom_status_t execute_impl(const mom_plan *p, const float *const *chain_ptrs, con
                     *trans = left ? sc.rhs_transposed : sc.lhs_transposed;
                     *scale = d.ptr; *scale_step = sc.k + 1; *scale_rows = left ? 1 : 0;
                 };
-                operand(stp.pub.lhs, stp.fold_a, &a.A, &a.strideA, &a.transA, stp.pub.lhs_transposed, &a.scaleA, &a.scaleA_step, &a.scaleA_rows);
-                operand(stp.pub.rhs, stp.fold_b, &a.B, &a.strideB, &a.transB, stp.pub.rhs_transposed, &a.scaleB, &a.scaleB_step, &a.scaleB_rows);
+                operand(stp.pub.lhs, stp.fold_a, &a.A, &a.strideA, &a.transA, stp.pub.lhs_transposed, &a.scaleA, &a.scaleA_step, &a.scaleA_rows, &a.packedA);
+                operand(stp.pub.rhs, stp.fold_b, &a.B, &a.strideB, &a.transB, stp.pub.rhs_transposed, &a.scaleB, &a.scaleB_step, &a.scaleB_rows, &a.packedB);
+                if ((a.packedA || a.packedB) && stp.pub.uses_tensor_cores != 1) return MOM_ERR_INVALID_ARG;   // only the split pass reads packed operands in place
                 if (stp.is_last && stp.accumulate) {
                     // a later chain's product is added to what the earlier ones left in the sum's buffer
                     a.C = x; a.strideC = x_stride;
@@ -455,6 +460,7 @@ mom_status_t execute_impl(const mom_plan *p, const float *const *chain_ptrs, con
                 } else if (stp.is_last) {
                     a.C = x; a.strideC = x_stride;
                     a.pout = kernel_property(sum.desc.property);
+                    a.packedC = top && sc && sc->out_packed;
                     added = add_terms(0, &a.add);
                 } else {
                     a.C = stp.out_off == SIZE_MAX ? nullptr : reinterpret_cast<float *>(ws + stp.out_off * (size_t)nb);
@@ -473,7 +479,7 @@ mom_status_t execute_impl(const mom_plan *p, const float *const *chain_ptrs, con
                     // the product that writes X then runs as two launches (only when nothing is added to X afterwards)
                     bool later_root = false;          // another chain's product is added to X after this one
                     for (int t = s + 1; t < sum.step_end; ++t) later_root |= p->steps[t].is_last;
-                    const bool two_parts = staged && staged->first_rows && top && stp.is_last && !stp.accumulate && !later_root &&
+                    const bool two_parts = staged && staged->first_rows && !a.packedC && top && stp.is_last && !stp.accumulate && !later_root &&
                                            added >= n_simple && batch == 1 && p->dev->tc.steps[s].part_row > 0;
                     if (lhs_in_pieces) {
                         if (cudaStreamWaitEvent(stream, staged->slot_head[lhs_slot], 0) != cudaSuccess) return MOM_ERR_CUDA;
@@ -521,6 +527,111 @@ mom_status_t execute_impl(const mom_plan *p, const float *const *chain_ptrs, con
     return MOM_OK;
 }
 
+
+// The storage layer around execute_core: packed operands that no kernel of this plan reads in place are unpacked into
+// dense copies behind the plan's own workspace, a packed X that is not written in place is computed dense there and
+// packed at the end; everything else goes through untouched.
+mom_status_t execute_impl(const mom_plan *p, const float *const *chain_ptrs, const int64_t *chain_strides,
+                          const float *const *add_ptrs, const int64_t *add_strides, float *out, int64_t out_stride,
+                          int64_t batch, void *workspace, size_t workspace_bytes, cudaStream_t stream,
+                          const StageEvents *staged = nullptr) {
+    if (!p) return MOM_ERR_INVALID_ARG;
+    if (p->ptr_storage.empty() && p->result_storage == MOM_STORAGE_DENSE)
+        return execute_core(p, chain_ptrs, chain_strides, add_ptrs, add_strides, out, out_stride, batch, workspace, workspace_bytes, stream, staged);
+    if (!chain_ptrs || !out || batch < 1) return MOM_ERR_INVALID_ARG;
+    const int n_ptrs = (int)p->ptr_desc.size(), n_add = (int)p->add.size();
+    if (n_add > 0 && !add_ptrs) return MOM_ERR_INVALID_ARG;
+    if (batch > 1 && (!chain_strides || (n_add > 0 && !add_strides))) return MOM_ERR_INVALID_ARG;
+    if (batch > 65535) return MOM_ERR_LIMIT;                 // the packing passes take the instances in grid.z
+
+    // every argument is checked before the first unpacking pass is enqueued
+    auto packed_size = [](const mom_matrix_desc_t &d) { return stored_elements(d, MOM_STORAGE_PACKED); };
+    for (int i = 0; i < n_ptrs; ++i) {
+        if (slot_storage(*p, i) != MOM_STORAGE_PACKED || !p->slot_used[i]) continue;
+        if (!chain_ptrs[i]) return MOM_ERR_INVALID_ARG;
+        if (!aligned16(chain_ptrs[i])) return MOM_ERR_ALIGNMENT;
+        if (batch > 1 && (chain_strides[i] % 4 != 0 || chain_strides[i] < packed_size(p->ptr_desc[i]))) return MOM_ERR_INVALID_ARG;
+    }
+    for (int i = 0; i < n_add; ++i) {
+        if (term_storage(*p, i) != MOM_STORAGE_PACKED) continue;
+        if (!add_ptrs[i]) return MOM_ERR_INVALID_ARG;
+        if (!aligned16(add_ptrs[i])) return MOM_ERR_ALIGNMENT;
+        if (batch > 1 && (add_strides[i] % 4 != 0 || add_strides[i] < packed_size(p->add[i]))) return MOM_ERR_INVALID_ARG;
+    }
+    if (!aligned16(out)) return MOM_ERR_ALIGNMENT;
+    if (p->result_storage == MOM_STORAGE_PACKED && batch > 1 && (out_stride % 4 != 0 || out_stride < packed_size(p->result_desc)))
+        return MOM_ERR_INVALID_ARG;
+    size_t need = 0;
+    mom_plan_workspace_bytes(p, batch, &need);
+    if (need > 0) {
+        if (!workspace || workspace_bytes < need) return MOM_ERR_WORKSPACE_TOO_SMALL;
+        if (reinterpret_cast<uintptr_t>(workspace) % WS_ALIGN != 0) return MOM_ERR_ALIGNMENT;
+    }
+    int device = 0;
+    mom_status_t st = check_arch(&device);
+    if (st != MOM_OK) return st;
+
+    const StorageLayout layout = storage_layout(*p, batch);
+    char *const region = static_cast<char *>(workspace) + (need - layout.bytes);
+    StorageCall sc;
+    sc.slot_packed.assign(n_ptrs, 0);
+    std::vector<const float *> cptr(chain_ptrs, chain_ptrs + n_ptrs), aptr(n_add, nullptr);
+    std::vector<int64_t> cstride(n_ptrs, 0), astride(n_add, 0);
+    for (int i = 0; i < n_ptrs; ++i) cstride[i] = chain_strides ? chain_strides[i] : 0;
+    for (int i = 0; i < n_add; ++i) { aptr[i] = add_ptrs[i]; astride[i] = add_strides ? add_strides[i] : 0; }
+
+    // which packed operands are read in place (the same rule that sized the workspace)
+    for (int i = 0; i < n_ptrs; ++i) sc.slot_packed[i] = storage_in_place(*p, i, batch);
+
+    int extra_launches = 0;
+    for (int i = 0; i < n_ptrs; ++i) {
+        if (slot_storage(*p, i) != MOM_STORAGE_PACKED || !p->slot_used[i] || sc.slot_packed[i]) continue;
+        if (layout.slot_off[i] == SIZE_MAX) return MOM_ERR_INVALID_ARG;
+        if (staged && cudaStreamWaitEvent(stream, staged->slot[i], 0) != cudaSuccess) return MOM_ERR_CUDA;
+        const mom_matrix_desc_t &d = p->ptr_desc[i];
+        float *dense = reinterpret_cast<float *>(region + layout.slot_off[i]);
+        if (launch_unpack(cptr[i], cstride[i], dense, dense_copy_stride(d), (int)d.rows, is_lower_kind(d.property), (int)batch, stream) != cudaSuccess)
+            return MOM_ERR_CUDA;
+        ++extra_launches;
+        cptr[i] = dense;
+        cstride[i] = dense_copy_stride(d);
+    }
+    if (!p->names.empty())                                   // entries with one name stay one matrix after the substitution
+        for (int i = 0; i < n_ptrs; ++i)
+            for (int j = 0; j < i; ++j)
+                if (p->names[i] == p->names[j] && chain_ptrs[i] == chain_ptrs[j] && p->slot_used[i] && p->slot_used[j]) { cptr[i] = cptr[j]; cstride[i] = cstride[j]; }
+    for (int i = 0; i < n_add; ++i) {
+        if (term_storage(*p, i) != MOM_STORAGE_PACKED) continue;
+        if (staged && cudaStreamWaitEvent(stream, staged->add[i], 0) != cudaSuccess) return MOM_ERR_CUDA;
+        const mom_matrix_desc_t &d = p->add[i];
+        float *dense = reinterpret_cast<float *>(region + layout.add_off[i]);
+        if (launch_unpack(aptr[i], astride[i], dense, dense_copy_stride(d), (int)d.rows, is_lower_kind(d.property), (int)batch, stream) != cudaSuccess)
+            return MOM_ERR_CUDA;
+        ++extra_launches;
+        aptr[i] = dense;
+        astride[i] = dense_copy_stride(d);
+    }
+    float *x = out;
+    int64_t x_stride = out_stride;
+    const mom_matrix_desc_t &rd = p->result_desc;
+    if (p->result_storage == MOM_STORAGE_PACKED) {
+        if (p->result_native) {
+            sc.out_packed = true;
+        } else {
+            x = reinterpret_cast<float *>(region + layout.x_off);
+            x_stride = dense_copy_stride(rd);
+        }
+    }
+    st = execute_core(p, cptr.data(), cstride.data(), aptr.data(), astride.data(), x, x_stride, batch, workspace, workspace_bytes, stream, staged, &sc);
+    if (st != MOM_OK) return st;
+    if (x != out) {
+        if (launch_pack(x, x_stride, out, out_stride, (int)rd.rows, is_lower_kind(rd.property), (int)batch, stream) != cudaSuccess) return MOM_ERR_CUDA;
+        ++extra_launches;
+    }
+    p->last_launches += extra_launches;
+    return MOM_OK;
+}
+
 }  // namespace
 }  // namespace mom
 
@@ -560,7 +671,7 @@ mom_status_t mom_equation_execute_host(const mom_plan_t *plan, const float *cons
     if (n_add > 0 && !add_host) return MOM_ERR_INVALID_ARG;
     // every argument error is found here, before the first copy is enqueued
     std::vector<int> same_as(n_chain, -1);
-    bool strides_ok = (plan->result_desc.rows * plan->result_desc.cols) % 4 == 0;
+    bool strides_ok = mom::stored_elements(plan->result_desc, plan->result_storage) % 4 == 0;
     for (int i = 0; i < n_chain; ++i) {
         const mom_matrix_desc_t &d = plan->ptr_desc[i];
         if (d.property == MOM_IDENTITY) continue;
@@ -573,12 +684,12 @@ mom_status_t mom_equation_execute_host(const mom_plan_t *plan, const float *cons
         }
         if (!plan->slot_used[i]) continue;
         if (!chain_host[i]) return MOM_ERR_INVALID_ARG;
-        strides_ok &= (d.rows * d.cols) % 4 == 0;
+        strides_ok &= mom::stored_elements(d, mom::slot_storage(*plan, i)) % 4 == 0;
     }
     for (int i = 0; i < n_add; ++i) {
         if (plan->add[i].property == MOM_IDENTITY) continue;
         if (!add_host[i]) return MOM_ERR_INVALID_ARG;
-        strides_ok &= (plan->add[i].rows * plan->add[i].cols) % 4 == 0;
+        strides_ok &= mom::stored_elements(plan->add[i], mom::term_storage(*plan, i)) % 4 == 0;
     }
     // instance strides that are not multiples of 4 elements cannot be batched in place
     if (batch > 1 && !strides_ok) return MOM_ERR_ALIGNMENT;
@@ -632,9 +743,9 @@ mom_status_t mom_equation_execute_host(const mom_plan_t *plan, const float *cons
                 continue;
             }
             if (!plan->slot_used[i]) continue;               // an operand no factor refers to is not uploaded
-            cbytes[i] = (size_t)d.rows * d.cols * sizeof(float) * batch;
+            cbytes[i] = (size_t)mom::stored_elements(d, mom::slot_storage(*plan, i)) * sizeof(float) * batch;
             cptr[i] = reinterpret_cast<const float *>(cur);
-            cstride[i] = d.rows * d.cols;
+            cstride[i] = mom::stored_elements(d, mom::slot_storage(*plan, i));
             cur += mom::align_up(cbytes[i], mom::WS_ALIGN);
         }
         // upload in the order of first use by the plan's products, so that the first products can start early
@@ -656,7 +767,7 @@ mom_status_t mom_equation_execute_host(const mom_plan_t *plan, const float *cons
                 const int32_t v = plan->steps[s].pub.lhs;
                 if (!dev->tc.steps[s].split_a_by_part || v >= (int32_t)plan->factor_ptr.size()) continue;
                 const int slot = plan->factor_ptr[v];
-                if (slot >= 0 && same_as[slot] < 0 && cbytes[slot] && first_use[slot] == (int)s && !mom::triangular_upload(plan->ptr_desc[slot], batch))
+                if (slot >= 0 && same_as[slot] < 0 && cbytes[slot] && first_use[slot] == (int)s && !mom::triangular_upload(plan->ptr_desc[slot], batch) && mom::slot_storage(*plan, slot) == MOM_STORAGE_DENSE)
                     head_rows[slot] = dev->tc.steps[s].part_row;
             }
         for (int i : order) {
@@ -668,7 +779,7 @@ mom_status_t mom_equation_execute_host(const mom_plan_t *plan, const float *cons
                 if (cudaMemcpyAsync(dst, src, head, cudaMemcpyHostToDevice, dev->copy_stream) != cudaSuccess) return MOM_ERR_CUDA;
                 if (cudaEventRecord(dev->slot_head[i], dev->copy_stream) != cudaSuccess) return MOM_ERR_CUDA;
                 if (cudaMemcpyAsync(dst + head, src + head, cbytes[i] - head, cudaMemcpyHostToDevice, dev->copy_stream) != cudaSuccess) return MOM_ERR_CUDA;
-            } else if (cbytes[i] && mom::triangular_upload(plan->ptr_desc[i], batch)) {
+            } else if (cbytes[i] && mom::triangular_upload(plan->ptr_desc[i], batch, mom::slot_storage(*plan, i))) {
                 // a large triangular operand: the host buffer holds zeros outside the triangle (storage contract), so
                 // only the 256-row blocks' columns up to (from) the diagonal block cross the bus; the rest is zero-filled here
                 const mom_matrix_desc_t &d = plan->ptr_desc[i];
@@ -692,18 +803,19 @@ mom_status_t mom_equation_execute_host(const mom_plan_t *plan, const float *cons
         for (int i = 0; i < n_add; ++i) {
             const mom_matrix_desc_t &d = plan->add[i];
             if (d.property == MOM_IDENTITY) continue;
-            const size_t bytes = (size_t)d.rows * d.cols * sizeof(float) * batch;
+            const size_t bytes = (size_t)mom::stored_elements(d, mom::term_storage(*plan, i)) * sizeof(float) * batch;
             if (cudaMemcpyAsync(cur, add_host[i], bytes, cudaMemcpyHostToDevice, dev->copy_stream) != cudaSuccess) return MOM_ERR_CUDA;
             if (cudaEventRecord(dev->add_ready[i], dev->copy_stream) != cudaSuccess) return MOM_ERR_CUDA;
             aptr[i] = reinterpret_cast<const float *>(cur);
-            astride[i] = d.rows * d.cols;
+            astride[i] = mom::stored_elements(d, mom::term_storage(*plan, i));
             cur += mom::align_up(bytes, mom::WS_ALIGN);
         }
         int first_rows = 0;
-        const mom::StageEvents staged{dev->slot_ready.data(), dev->add_ready.data(), dev->first_rows_done, &first_rows,
+        const mom::StageEvents staged{dev->slot_ready.data(), dev->add_ready.data(), dev->first_rows_done,
+                                      plan->result_storage == MOM_STORAGE_DENSE ? &first_rows : nullptr,
                                       dev->slot_head.data(), head_rows.data()};
         float *x = reinterpret_cast<float *>(cur);
-        const int64_t xelems = plan->result_desc.rows * plan->result_desc.cols;
+        const int64_t xelems = mom::stored_elements(plan->result_desc, plan->result_storage);
         const size_t xbytes = (size_t)xelems * sizeof(float) * batch;
         cur += mom::align_up(xbytes, mom::WS_ALIGN);
         size_t ws_bytes = 0;
@@ -750,10 +862,12 @@ mom_status_t mom_plan_host_upload_bytes(const mom_plan_t *plan, int64_t batch, s
         bool seen = false;                               // a named matrix is copied once
         if (!plan->names.empty())
             for (int j = 0; j < i && !seen; ++j) seen = plan->names[j] == plan->names[i] && plan->slot_used[j];
-        if (!seen) total += mom::upload_bytes(d, batch);
+        if (!seen) total += mom::upload_bytes(d, batch, mom::slot_storage(*plan, i));
     }
-    for (const auto &d : plan->add)
-        if (d.property != MOM_IDENTITY) total += (size_t)d.rows * d.cols * sizeof(float) * batch;
+    for (size_t i = 0; i < plan->add.size(); ++i) {
+        const auto &d = plan->add[i];
+        if (d.property != MOM_IDENTITY) total += (size_t)mom::stored_elements(d, mom::term_storage(*plan, (int)i)) * sizeof(float) * batch;
+    }
     *bytes = total;
     return MOM_OK;
 }

@@ -22,6 +22,8 @@ struct ProductArgs {
     const float *scaleA, *scaleB;
     long long scaleA_step, scaleB_step;
     int scaleA_rows, scaleB_rows;
+    // tensor-core path only: the operand (as stored) / the result is a packed triangle read / written in place
+    int packedA, packedB, packedC;
 };
 
 cudaError_t launch_product_ffma(const ProductArgs &a, int batch, cudaStream_t stream);
@@ -36,5 +38,11 @@ cudaError_t launch_scale(const ProductArgs &a, int batch, cudaStream_t stream);
 // src_mode: 0 pointer, 1 Identity, 2 X itself (in place), 3 pointer to the transposed matrix (cols x rows)
 cudaError_t launch_elementwise(const float *src, long long src_stride, int src_mode, float *X, long long x_stride,
                                int rows, int cols, int out_prop, const AddTerms &add, int batch, cudaStream_t stream);
+
+// Packed triangle -> dense n x n matrix (zeros outside the container) and back, `batch` instances.
+cudaError_t launch_unpack(const float *src, long long src_stride, float *dst, long long dst_stride, int n, bool lower, int batch,
+                          cudaStream_t stream);
+cudaError_t launch_pack(const float *src, long long src_stride, float *dst, long long dst_stride, int n, bool lower, int batch,
+                        cudaStream_t stream);
 
 }  // namespace mom

@@ -112,6 +112,11 @@ struct mom_plan {
     std::vector<char> chain_t, add_t;          // operand enters transposed: stored shape is (cols x rows) of the entry above
     std::vector<int32_t> chain_begin;          // factors of chain c are [chain_begin[c], chain_begin[c + 1])
     std::vector<int32_t> names;                // per pointer entry: equal names = the same stored matrix (empty: all distinct)
+    // storage layer (mom_equation_plan_stored): per caller pointer / Add term / for X; empty vectors: all dense
+    std::vector<int32_t> ptr_storage, add_storage;
+    int32_t result_storage = 0;
+    std::vector<char> slot_native;             // packed slot that every reader addresses in place (no dense copy needed)
+    bool result_native = false;                // packed X written in place by the product that writes X
     std::vector<int32_t> kept;                 // factor indices surviving identity simplification
     std::vector<mom::SumInfo> sums;            // nested sums first, X last
     int32_t temporaries = 0;                   // nested sums that are materialized
@@ -138,6 +143,85 @@ struct mom_plan {
 };
 
 namespace mom {
+
+// ---- storage layer (packed triangles) ----------------------------------------------------------------------
+inline bool is_lower_kind(int32_t p) { return kernel_property(p) == MOM_LOWER_TRI; }
+inline bool is_triangular_kind(int32_t p) { return kernel_property(p) == MOM_LOWER_TRI || kernel_property(p) == MOM_UPPER_TRI; }
+
+// f32 entries a matrix occupies as stored
+inline int64_t stored_elements(const mom_matrix_desc_t &d, int32_t storage) {
+    if (storage != MOM_STORAGE_PACKED) return d.rows * d.cols;
+    const int64_t n = d.rows, q = n >> 2, rest = n - 4 * q, n4 = (n + 3) & ~(int64_t)3;
+    return is_lower_kind(d.property) ? 8 * q * (q + 1) + rest * 4 * (q + 1) : n * n4 - 8 * q * (q - 1) - 4 * q * rest;
+}
+inline int32_t slot_storage(const mom_plan &p, int slot) { return p.ptr_storage.empty() ? 0 : p.ptr_storage[slot]; }
+inline int32_t term_storage(const mom_plan &p, int term) { return p.add_storage.empty() ? 0 : p.add_storage[term]; }
+
+// Shape test of the batched-chain kernel (batched_chain.cu): a right-nested chain M_S * (... (M_1 * B)) of stored,
+// untransposed factors with whole 16-row blocks of at most 64 rows, a right end of 8 or 16 columns, Add terms not
+// transposed.  (Whether a call takes that kernel also depends on its batch size.)
+constexpr int64_t BATCHED_CHAIN_MIN_BATCH = 256;
+inline bool batched_chain_shape(const mom_plan &p) {
+    const int S = (int)p.steps.size(), n_chain = (int)p.chain.size();
+    if (!p.fused_ok || p.variant == MOM_VARIANT_FFMA || p.sums.size() != 1 || S < 1 || S > 4 || p.add.size() > 8) return false;
+    for (const Summand &sm : p.sums[0].summands)
+        if (sm.kind != SUM_STEP && sm.kind != SUM_TERM) return false;
+    for (char t : p.add_t)
+        if (t) return false;
+    const int64_t n = p.steps[0].pub.n;
+    if ((n != 8 && n != 16) || !p.steps[S - 1].is_last) return false;
+    for (int s = 0; s < S; ++s) {
+        const mom_step_t &st = p.steps[s].pub;
+        if (st.kind == MOM_KIND_SCALE || st.kind == MOM_KIND_GRAM || p.steps[s].folded || p.steps[s].accumulate) return false;
+        if (st.lhs < 0 || st.lhs >= n_chain || st.lhs_transposed || p.chain_t[st.lhs] || p.factor_ptr[st.lhs] < 0) return false;
+        if (s == 0 ? (st.rhs < 0 || st.rhs >= n_chain || st.rhs_transposed || p.chain_t[st.rhs] || p.factor_ptr[st.rhs] < 0)
+                   : st.rhs != p.steps[s - 1].pub.out) return false;
+        if (st.m % 16 || st.m > 64 || st.k % 16 || st.k > 64 || st.n != n) return false;
+        const int pa = kernel_property(st.lhs_property), pb = kernel_property(st.rhs_property);
+        if (pa == MOM_DIAGONAL || pa == MOM_IDENTITY || pb == MOM_DIAGONAL || pb == MOM_IDENTITY) return false;
+    }
+    return true;
+}
+
+// A packed operand that every kernel of a call with `batch` instances reads in place (no dense copy): what the plan
+// marked (operands of tcgen05 steps), or a left factor of the batched-chain kernel when the call qualifies for it.
+inline bool storage_in_place(const mom_plan &p, int slot, int64_t batch) {
+    if (slot_storage(p, slot) != MOM_STORAGE_PACKED || !p.slot_used[slot]) return false;
+    if (p.slot_native[slot]) return true;
+    if (batch < BATCHED_CHAIN_MIN_BATCH || p.result_storage != MOM_STORAGE_DENSE || !batched_chain_shape(p)) return false;
+    for (size_t i = 0; i < p.add.size(); ++i)
+        if (term_storage(p, (int)i) != MOM_STORAGE_DENSE) return false;
+    return slot != p.factor_ptr[p.steps[0].pub.rhs];         // the right end is read dense
+}
+
+// elements between the instances of a dense copy the storage layer makes (a multiple of 4: rows stay 16-byte addressable)
+inline int64_t dense_copy_stride(const mom_matrix_desc_t &d) { return (d.rows * d.cols + 3) & ~(int64_t)3; }
+
+// Room behind the plan's own workspace for the storage layer: a dense copy of every packed operand that some kernel
+// cannot read in place, of every packed Add term, and a dense X when the packed X is not written in place.  Offsets
+// are in bytes from the start of that region (SIZE_MAX: none); returns the region's size.
+struct StorageLayout {
+    std::vector<size_t> slot_off, add_off;
+    size_t x_off = SIZE_MAX;
+    size_t bytes = 0;
+};
+inline StorageLayout storage_layout(const mom_plan &p, int64_t batch) {
+    StorageLayout l;
+    l.slot_off.assign(p.ptr_desc.size(), SIZE_MAX);
+    l.add_off.assign(p.add.size(), SIZE_MAX);
+    auto take = [&](const mom_matrix_desc_t &d) {
+        const size_t at = l.bytes;
+        l.bytes += align_up((size_t)dense_copy_stride(d) * sizeof(float) * (size_t)batch, WS_ALIGN);
+        return at;
+    };
+    for (size_t i = 0; i < p.ptr_desc.size(); ++i)
+        if (slot_storage(p, (int)i) == MOM_STORAGE_PACKED && p.slot_used[i] && !storage_in_place(p, (int)i, batch)) l.slot_off[i] = take(p.ptr_desc[i]);
+    for (size_t i = 0; i < p.add.size(); ++i)
+        if (term_storage(p, (int)i) == MOM_STORAGE_PACKED) l.add_off[i] = take(p.add[i]);
+    if (p.result_storage == MOM_STORAGE_PACKED && !p.result_native) l.x_off = take(p.result_desc);
+    return l;
+}
+
 // defined in execute.cu; releases device-side state of a plan (no-op when none exists)
 void destroy_device_state(DeviceState *);
 }  // namespace mom

@@ -786,6 +786,107 @@ mom_status_t mom_equation_plan_transposed(const mom_matrix_desc_t *stored_chain,
     return plan_flat(stored_chain, chain_transposed, nullptr, &n_chain, 1, stored_add, add_transposed, n_add, variant, out_plan);
 }
 
+mom_status_t mom_packed_elements(int64_t rows, mom_property_t property, int64_t *elements) {
+    if (!elements || rows < 1) return MOM_ERR_INVALID_ARG;
+    if (property < MOM_GENERAL || property > MOM_UNIT_UPPER) return MOM_ERR_INVALID_ARG;
+    if (!mom::is_triangular_kind(property)) return MOM_ERR_PROPERTY;
+    if (rows > mom::MAX_DIMENSION) return MOM_ERR_LIMIT;
+    const mom_matrix_desc_t d{rows, rows, (int32_t)property, MOM_F32};
+    *elements = mom::stored_elements(d, MOM_STORAGE_PACKED);
+    return MOM_OK;
+}
+
+mom_status_t mom_packed_row(int64_t rows, mom_property_t property, int64_t row, int64_t *offset, int64_t *first_col, int64_t *end_col) {
+    if (!offset || !first_col || !end_col || rows < 1 || row < 0 || row >= rows) return MOM_ERR_INVALID_ARG;
+    if (property < MOM_GENERAL || property > MOM_UNIT_UPPER) return MOM_ERR_INVALID_ARG;
+    if (!mom::is_triangular_kind(property)) return MOM_ERR_PROPERTY;
+    if (rows > mom::MAX_DIMENSION) return MOM_ERR_LIMIT;
+    // the rows before `row` are the container of a `row`-row matrix whose rows have the same lengths: for a lower
+    // triangle that is the packed `row` x `row` triangle; for an upper one the lengths depend on `rows` (n4 below)
+    const int64_t q = row >> 2, rest = row - 4 * q, n4 = (rows + 3) & ~(int64_t)3;
+    if (mom::is_lower_kind(property)) {
+        *first_col = 0;
+        *end_col = 4 * (q + 1);
+        *offset = 8 * q * (q + 1) + rest * 4 * (q + 1);
+    } else {
+        *first_col = 4 * q;
+        *end_col = n4;
+        *offset = row * n4 - 8 * q * (q - 1) - 4 * q * rest;
+    }
+    return MOM_OK;
+}
+
+mom_status_t mom_plan_result_elements(const mom_plan_t *plan, int64_t *elements) {
+    if (!plan || !elements) return MOM_ERR_INVALID_ARG;
+    *elements = mom::stored_elements(plan->result_desc, plan->result_storage);
+    return MOM_OK;
+}
+
+mom_status_t mom_equation_plan_stored(const mom_matrix_desc_t *chain, const int32_t *chain_transposed, const int32_t *chain_storage,
+                                      int32_t n_chain, const mom_matrix_desc_t *add_terms, const int32_t *add_transposed,
+                                      const int32_t *add_storage, int32_t n_add, mom_storage_t result_storage,
+                                      mom_variant_t variant, mom_plan_t **out_plan) {
+    if (result_storage != MOM_STORAGE_DENSE && result_storage != MOM_STORAGE_PACKED) return MOM_ERR_INVALID_ARG;
+    mom_plan_t *p = nullptr;
+    const mom_status_t st = mom_equation_plan_transposed(chain, chain_transposed, n_chain, add_terms, add_transposed, n_add, variant, &p);
+    if (st != MOM_OK) return st;
+    auto fail = [&](mom_status_t e) { mom_plan_destroy(p); return e; };
+    try {
+        for (int i = 0; i < n_chain; ++i) {
+            const int32_t sto = chain_storage ? chain_storage[i] : 0;
+            if (sto != MOM_STORAGE_DENSE && sto != MOM_STORAGE_PACKED) return fail(MOM_ERR_INVALID_ARG);
+            if (sto == MOM_STORAGE_PACKED && !mom::is_triangular_kind(chain[i].property)) return fail(MOM_ERR_PROPERTY);
+            p->ptr_storage.push_back(sto);
+        }
+        for (int i = 0; i < n_add; ++i) {
+            const int32_t sto = add_storage ? add_storage[i] : 0;
+            if (sto != MOM_STORAGE_DENSE && sto != MOM_STORAGE_PACKED) return fail(MOM_ERR_INVALID_ARG);
+            if (sto == MOM_STORAGE_PACKED && !mom::is_triangular_kind(add_terms[i].property)) return fail(MOM_ERR_PROPERTY);
+            p->add_storage.push_back(sto);
+        }
+        if (result_storage == MOM_STORAGE_PACKED && !mom::is_triangular_kind(p->result_desc.property)) return fail(MOM_ERR_PROPERTY);
+        p->result_storage = result_storage;
+        // which packed operands every reader addresses in place: factors read only as operands of tcgen05 steps (their
+        // operand-split pass has a packed addressing mode), as stored, not through a folded scaling, not as summands
+        const int nf = (int)p->chain.size();
+        p->slot_native.assign(p->ptr_desc.size(), 0);
+        for (size_t slot = 0; slot < p->ptr_desc.size(); ++slot) {
+            if (p->ptr_storage[slot] != MOM_STORAGE_PACKED || p->fused_ok) continue;
+            bool native = true, read = false;
+            for (int f = 0; f < nf; ++f) {
+                if (p->factor_ptr[f] != (int)slot) continue;
+                if (p->chain_t[f]) native = false;
+                for (const auto &sp : p->steps) {
+                    if (sp.pub.lhs != f && sp.pub.rhs != f) continue;
+                    read = true;
+                    if (sp.pub.uses_tensor_cores != 1 || sp.folded || sp.pub.kind == MOM_KIND_GRAM || sp.pub.kind == MOM_KIND_SCALE) native = false;
+                }
+                for (const auto &sum : p->sums)
+                    for (const auto &sm : sum.summands)
+                        if (sm.kind == mom::SUM_FACTOR && sm.index == f) native = false;
+            }
+            p->slot_native[slot] = native && read;
+        }
+        // a packed X is written in place when one tcgen05 product writes it, whole, with every summand fused
+        if (result_storage == MOM_STORAGE_PACKED) {
+            const mom::SumInfo &top = p->sums.back();
+            int roots = 0, root = -1, simple = 0;
+            for (const auto &sm : top.summands) {
+                if (sm.kind == mom::SUM_STEP) { ++roots; root = sm.index; }
+                else ++simple;
+            }
+            if (roots == 1 && simple <= mom::MAX_FUSED_ADD && !p->fused_ok) {
+                const mom::StepImpl &r = p->steps[root];
+                p->result_native = r.pub.uses_tensor_cores == 1 && r.split_k == 1 && !r.mirror && r.planes_out == 0 && !r.accumulate;
+            }
+        }
+    } catch (const std::bad_alloc &) {
+        return fail(MOM_ERR_ALLOC);
+    }
+    *out_plan = p;
+    return MOM_OK;
+}
+
 mom_status_t mom_equation_plan_sum(const mom_matrix_desc_t *factors, const int32_t *factor_transposed,
                                    const int32_t *factor_names, const int32_t *chain_lengths, int32_t n_chains,
                                    mom_variant_t variant, mom_plan_t **out_plan) {
@@ -942,17 +1043,26 @@ mom_status_t mom_plan_workspace_bytes(const mom_plan_t *plan, int64_t batch, siz
     for (const auto &s : plan->steps) any_tc |= s.pub.uses_tensor_cores == 1;
     const int64_t group = any_tc ? 1 : (batch < 65535 ? batch : 65535);
     *bytes = plan->workspace_per_instance * (size_t)group;
+    if (!plan->ptr_storage.empty() || plan->result_storage != MOM_STORAGE_DENSE) {
+        // packed storage: dense copies for the kernels that cannot address a packed matrix, behind the plan's own room
+        const size_t extra = mom::storage_layout(*plan, batch).bytes;
+        if (extra) *bytes = mom::align_up(*bytes, mom::WS_ALIGN) + extra;
+    }
     return MOM_OK;
 }
 
 mom_status_t mom_plan_host_staging_bytes(const mom_plan_t *plan, int64_t batch, size_t *bytes) {
     if (!plan || !bytes || batch < 1) return MOM_ERR_INVALID_ARG;
     size_t total = 0;
-    for (const auto &d : plan->ptr_desc)
-        if (d.property != MOM_IDENTITY) total += mom::align_up((size_t)d.rows * d.cols * sizeof(float) * batch, mom::WS_ALIGN);
-    for (const auto &d : plan->add)
-        if (d.property != MOM_IDENTITY) total += mom::align_up((size_t)d.rows * d.cols * sizeof(float) * batch, mom::WS_ALIGN);
-    total += mom::align_up((size_t)plan->result_desc.rows * plan->result_desc.cols * sizeof(float) * batch, mom::WS_ALIGN);
+    for (size_t i = 0; i < plan->ptr_desc.size(); ++i) {
+        const auto &d = plan->ptr_desc[i];
+        if (d.property != MOM_IDENTITY) total += mom::align_up((size_t)mom::stored_elements(d, mom::slot_storage(*plan, (int)i)) * sizeof(float) * batch, mom::WS_ALIGN);
+    }
+    for (size_t i = 0; i < plan->add.size(); ++i) {
+        const auto &d = plan->add[i];
+        if (d.property != MOM_IDENTITY) total += mom::align_up((size_t)mom::stored_elements(d, mom::term_storage(*plan, (int)i)) * sizeof(float) * batch, mom::WS_ALIGN);
+    }
+    total += mom::align_up((size_t)mom::stored_elements(plan->result_desc, plan->result_storage) * sizeof(float) * batch, mom::WS_ALIGN);
     size_t ws = 0;
     mom_plan_workspace_bytes(plan, batch, &ws);
     total += ws;

@@ -4,7 +4,10 @@
 // (tile_k_range), so all-zero blocks of triangular operands are never read and structurally-zero
 // output tiles are only zero-filled.
 #include "device_common.cuh"
+#include <algorithm>
+
 #include "kernels.h"
+#include "packed.cuh"
 
 namespace mom {
 
@@ -384,6 +387,74 @@ cudaError_t launch_scale(const ProductArgs &a, int batch, cudaStream_t stream) {
 cudaError_t launch_product_ffma(const ProductArgs &a, int batch, cudaStream_t stream) {
     dim3 grid((a.n + BN - 1) / BN, (a.m + BM - 1) / BM, batch);
     product_ffma_kernel<<<grid, THREADS, 0, stream>>>(a);
+    return cudaGetLastError();
+}
+
+// Packed triangle <-> dense matrix, one thread per 16-byte group of a row (see packed.cuh for the container).
+// unpack: the dense n x n matrix gets the stored entries and zeros everywhere else; pack: the container gets the
+// dense matrix's entries of every stored position (zeros beyond the last column).  Bound by HBM; grid.z = instances.
+namespace {
+__global__ void __launch_bounds__(256)
+unpack_kernel(const float *__restrict__ src, long long src_stride, float *__restrict__ dst, long long dst_stride, int n, int lower) {
+    const int groups = (n + 3) >> 2;
+    src += (long long)blockIdx.z * src_stride;
+    dst += (long long)blockIdx.z * dst_stride;
+    const bool vec = (n & 3) == 0;                               // dense rows are 16-byte aligned
+    for (long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x; e < (long long)n * groups; e += (long long)gridDim.x * blockDim.x) {
+        const int r = (int)(e / groups), c = (int)(e % groups) << 2;
+        const PackedRow row = packed_row(lower != 0, n, r);
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (c >= row.first && c < row.end) v = __ldg(reinterpret_cast<const float4 *>(src + row.offset + (c - row.first)));
+        float *d = dst + (long long)r * n + c;
+        if (vec) {
+            *reinterpret_cast<float4 *>(d) = v;
+        } else {
+            d[0] = v.x;
+            if (c + 1 < n) d[1] = v.y;
+            if (c + 2 < n) d[2] = v.z;
+            if (c + 3 < n) d[3] = v.w;
+        }
+    }
+}
+
+__global__ void __launch_bounds__(256)
+pack_kernel(const float *__restrict__ src, long long src_stride, float *__restrict__ dst, long long dst_stride, int n, int lower) {
+    const int groups = (n + 3) >> 2;
+    src += (long long)blockIdx.z * src_stride;
+    dst += (long long)blockIdx.z * dst_stride;
+    const bool vec = (n & 3) == 0;
+    for (long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x; e < (long long)n * groups; e += (long long)gridDim.x * blockDim.x) {
+        const int r = (int)(e / groups), c = (int)(e % groups) << 2;
+        const PackedRow row = packed_row(lower != 0, n, r);
+        if (c < row.first || c >= row.end) continue;
+        const float *a = src + (long long)r * n + c;
+        float4 v;
+        if (vec) {
+            v = __ldg(reinterpret_cast<const float4 *>(a));
+        } else {
+            v.x = __ldg(a);
+            v.y = c + 1 < n ? __ldg(a + 1) : 0.f;
+            v.z = c + 2 < n ? __ldg(a + 2) : 0.f;
+            v.w = c + 3 < n ? __ldg(a + 3) : 0.f;
+        }
+        *reinterpret_cast<float4 *>(dst + row.offset + (c - row.first)) = v;
+    }
+}
+}  // namespace
+
+cudaError_t launch_unpack(const float *src, long long src_stride, float *dst, long long dst_stride, int n, bool lower, int batch,
+                          cudaStream_t stream) {
+    const long long work = (long long)n * ((n + 3) >> 2);
+    const unsigned gx = (unsigned)std::min<long long>((work + 255) / 256, 148 * 16);
+    unpack_kernel<<<dim3(gx, 1, batch), 256, 0, stream>>>(src, src_stride, dst, dst_stride, n, lower ? 1 : 0);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_pack(const float *src, long long src_stride, float *dst, long long dst_stride, int n, bool lower, int batch,
+                        cudaStream_t stream) {
+    const long long work = (long long)n * ((n + 3) >> 2);
+    const unsigned gx = (unsigned)std::min<long long>((work + 255) / 256, 148 * 16);
+    pack_kernel<<<dim3(gx, 1, batch), 256, 0, stream>>>(src, src_stride, dst, dst_stride, n, lower ? 1 : 0);
     return cudaGetLastError();
 }
 

@@ -25,6 +25,7 @@
 #include <cuda.h>
 
 #include "device_info.h"
+#include "packed.cuh"
 #include "product_tc.h"
 #include "tc_probe.h"
 #include "tc_ptx.cuh"
@@ -96,6 +97,8 @@ struct TcParams {
     int pout;
     int out_mode;            // 0: f32 result through map_c; 1: hi/lo planes (map_c, map_c2); 2: transposed hi/lo planes
     int slice_rows;          // split-K: rows between the partial-sum slabs of consecutive k-slices (0: no split)
+    float *packed_c;         // not null (out_mode 0 only): the result is a packed triangle written in place with plain
+                             // 16-byte stores; entries the container does not hold are not written at all
     int mirror;              // Gram product Y * Y^T (CTA-pair kernel, out_mode 0, Symmetric Add terms only): the table holds the tiles on and
                              // below the diagonal; a tile below it is also written transposed to its mirror position
     AddTerms add;
@@ -152,6 +155,21 @@ __device__ __forceinline__ void epilogue_chunk(const TcParams &prm, const CUtens
     if (prm.pout != MOM_GENERAL) {
 #pragma unroll
         for (int j = 0; j < 32; ++j) v[j] = in_structure(prm.pout, r, col0 + j) ? v[j] : 0.0f;
+    }
+    if (prm.packed_c) {
+        // packed triangle: this thread's row holds columns [first, end); every 16-byte group of the chunk that lies in
+        // that range goes straight to its place (a lane writes whole 16-byte groups of its own row)
+        if (row_ok) {
+            const PackedRow row = packed_row(prm.pout == MOM_LOWER_TRI, prm.m, r);
+            float *dst = prm.packed_c + row.offset - row.first;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const int c = col0 + 4 * j;
+                if (c >= row.first && c < row.end)
+                    *reinterpret_cast<float4 *>(dst + c) = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+            }
+        }
+        return;
     }
     const int passes = prm.out_mode == 0 ? (mirror_this ? 2 : 1) : 2;   // f32 (and its mirror image), or hi then lo
 #pragma unroll 1
@@ -568,9 +586,11 @@ struct SplitScale {
     int by_row;
 };
 
+// `packed`: the source is a packed triangle (see packed.cuh) read in place: entry (r, c) sits at its row's offset, and
+// what the container does not hold reads as zero.  The planes are dense either way (TMA addresses them).
 template <bool TRANSPOSE>
 __device__ __forceinline__ void split_piece(const float *__restrict__ src, float *__restrict__ hi, float *__restrict__ lo, int rows,
-                                            int cols, int prop, const SplitScale &sc, int piece_x, int piece_y) {
+                                            int cols, int prop, const SplitScale &sc, int piece_x, int piece_y, int packed) {
     const int pr = piece_y * SPLIT_PIECE, pc = piece_x * SPLIT_PIECE;
     const int br = pr / SPLIT_BLOCK * SPLIT_BLOCK, bc = pc / SPLIT_BLOCK * SPLIT_BLOCK;
     if (prop == MOM_LOWER_TRI && bc > br + SPLIT_BLOCK - 1) return;     // block wholly above the diagonal
@@ -582,7 +602,14 @@ __device__ __forceinline__ void split_piece(const float *__restrict__ src, float
             const int r = pr + (e >> 4), c = pc + ((e & 15) << 2);
             if (r < rows && c < cols) {
                 const size_t off = (size_t)r * cols + c;
-                float4 a = __ldg(reinterpret_cast<const float4 *>(src + off));
+                float4 a;
+                if (packed) {
+                    const PackedRow row = packed_row(prop == MOM_LOWER_TRI, rows, r);
+                    a = c >= row.first && c < row.end ? __ldg(reinterpret_cast<const float4 *>(src + row.offset + (c - row.first)))
+                                                      : make_float4(0.f, 0.f, 0.f, 0.f);
+                } else {
+                    a = __ldg(reinterpret_cast<const float4 *>(src + off));
+                }
                 if (sc.d) {
                     if (sc.by_row) {
                         const float f = __ldg(sc.d + r * sc.step);
@@ -605,7 +632,15 @@ __device__ __forceinline__ void split_piece(const float *__restrict__ src, float
         for (int i = 0; i < 16; ++i) {
             const int e = threadIdx.x + 256 * i;                         // 64 x 64 scalars, row-contiguous reads
             const int r = e >> 6, c = e & 63;
-            float v = (pr + r < rows && pc + c < cols) ? __ldg(src + (size_t)(pr + r) * cols + pc + c) : 0.0f;
+            float v = 0.0f;
+            if (pr + r < rows && pc + c < cols) {
+                if (packed) {
+                    const PackedRow row = packed_row(prop == MOM_LOWER_TRI, rows, pr + r);
+                    if (pc + c >= row.first && pc + c < row.end) v = __ldg(src + row.offset + (pc + c - row.first));
+                } else {
+                    v = __ldg(src + (size_t)(pr + r) * cols + pc + c);
+                }
+            }
             if (sc.d && pr + r < rows && pc + c < cols) v *= __ldg(sc.d + (sc.by_row ? pr + r : pc + c) * sc.step);
             tile[r][c] = v;
         }
@@ -630,8 +665,8 @@ __device__ __forceinline__ void split_piece(const float *__restrict__ src, float
 template <bool TRANSPOSE>
 __global__ void __launch_bounds__(256)
 split_planes_kernel(const float *__restrict__ src, float *__restrict__ hi, float *__restrict__ lo, int rows, int cols, int prop,
-                    SplitScale sc) {
-    split_piece<TRANSPOSE>(src, hi, lo, rows, cols, prop, sc, blockIdx.x, blockIdx.y);
+                    SplitScale sc, int packed) {
+    split_piece<TRANSPOSE>(src, hi, lo, rows, cols, prop, sc, blockIdx.x, blockIdx.y, packed);
 }
 
 // Both operands of one product in ONE launch (a launch costs about as much as splitting a few MB): the first
@@ -641,6 +676,7 @@ struct SplitJob {
     float *hi, *lo;
     int rows, cols, prop, transpose, pieces_x;
     SplitScale sc;
+    int packed;
 };
 __global__ void __launch_bounds__(256)
 split_both_kernel(SplitJob a, SplitJob b, int pieces_a) {
@@ -648,8 +684,8 @@ split_both_kernel(SplitJob a, SplitJob b, int pieces_a) {
     const SplitJob &j = first ? a : b;
     const int piece = first ? blockIdx.x : blockIdx.x - pieces_a;
     const int px = piece % j.pieces_x, py = piece / j.pieces_x;
-    if (j.transpose) split_piece<true>(j.src, j.hi, j.lo, j.rows, j.cols, j.prop, j.sc, px, py);
-    else split_piece<false>(j.src, j.hi, j.lo, j.rows, j.cols, j.prop, j.sc, px, py);
+    if (j.transpose) split_piece<true>(j.src, j.hi, j.lo, j.rows, j.cols, j.prop, j.sc, px, py, j.packed);
+    else split_piece<false>(j.src, j.hi, j.lo, j.rows, j.cols, j.prop, j.sc, px, py, j.packed);
 }
 
 // Split-K: sum the k-slices' partial results, then the usual finish (Add terms, structure mask).
@@ -913,7 +949,7 @@ mom_status_t tc_launch_step(const mom_plan &p, TcPlanState &s, int step, const P
     const SplitScale sb{a.scaleB, a.scaleB_step, a.scaleB ? (a.scaleB_rows != 0) != (a.transB != 0) : 0};
     // as stored: rows x cols and the property of the matrix the kernel reads
     SplitJob ja{a.A, a_hi, a_lo, a.transA ? a.k : a.m, a.transA ? a.m : a.k, a.transA ? stored_prop(a.pa) : a.pa, a.transA ? 1 : 0,
-                blocks(a.transA ? a.m : a.k), sa};
+                blocks(a.transA ? a.m : a.k), sa, a.packedA};
     const bool a_by_part = part > 0 && s.steps[step].split_a_by_part;     // a general m x k matrix read as stored
     if (a_by_part) {
         const int row = s.steps[step].part_row, r0 = part == 1 ? 0 : row;
@@ -923,7 +959,7 @@ mom_status_t tc_launch_step(const mom_plan &p, TcPlanState &s, int step, const P
         ja.rows = part == 1 ? row : a.m - row;
     }
     const SplitJob jb{a.B, b_hi, b_lo, a.transB ? a.n : a.k, a.transB ? a.k : a.n, a.transB ? stored_prop(a.pb) : a.pb, a.transB ? 0 : 1,
-                      blocks(a.transB ? a.k : a.n), sb};
+                      blocks(a.transB ? a.k : a.n), sb, a.packedB};
     const bool do_a = !st.a_planes_ready && (part != 2 || a_by_part), do_b = !st.b_planes_ready && part != 2;
     auto pieces = [&](const SplitJob &j) { return j.pieces_x * blocks(j.rows); };
     if (do_a && do_b) {
@@ -931,8 +967,8 @@ mom_status_t tc_launch_step(const mom_plan &p, TcPlanState &s, int step, const P
         ++split_launches;
     } else if (do_a || do_b) {
         const SplitJob &j = do_a ? ja : jb;
-        if (j.transpose) split_planes_kernel<true><<<dim3(j.pieces_x, blocks(j.rows)), 256, 0, stream>>>(j.src, j.hi, j.lo, j.rows, j.cols, j.prop, j.sc);
-        else split_planes_kernel<false><<<dim3(j.pieces_x, blocks(j.rows)), 256, 0, stream>>>(j.src, j.hi, j.lo, j.rows, j.cols, j.prop, j.sc);
+        if (j.transpose) split_planes_kernel<true><<<dim3(j.pieces_x, blocks(j.rows)), 256, 0, stream>>>(j.src, j.hi, j.lo, j.rows, j.cols, j.prop, j.sc, j.packed);
+        else split_planes_kernel<false><<<dim3(j.pieces_x, blocks(j.rows)), 256, 0, stream>>>(j.src, j.hi, j.lo, j.rows, j.cols, j.prop, j.sc, j.packed);
         ++split_launches;
     }
     if (cudaGetLastError() != cudaSuccess) return MOM_ERR_CUDA;
@@ -971,6 +1007,12 @@ mom_status_t tc_launch_step(const mom_plan &p, TcPlanState &s, int step, const P
     prm.slice_rows = slice_rows;
     if (s.steps[step].mirror && st.planes_out != 0) return MOM_ERR_INVALID_ARG;   // the planner never asks for this
     prm.mirror = s.steps[step].mirror ? 1 : 0;
+    prm.packed_c = nullptr;
+    if (a.packedC) {
+        // only a plain f32 result of a triangular product is ever written packed (the planner checks as much)
+        if (st.planes_out != 0 || st.split_k > 1 || s.steps[step].mirror || (a.pout != MOM_LOWER_TRI && a.pout != MOM_UPPER_TRI)) return MOM_ERR_INVALID_ARG;
+        prm.packed_c = a.C;
+    }
     prm.add = a.add;
     if (st.split_k > 1) prm.add.count = 0;
     prm.status = status;
@@ -1214,8 +1256,8 @@ extern "C" mom_status_t mom_product_3xtf32_noalloc(int64_t m64, int64_t n64, int
 
     auto blocks = [](int x) { return (x + SPLIT_PIECE - 1) / SPLIT_PIECE; };
     noalloc_build_tiles_kernel<<<(unsigned)((tiles + 127) / 128), 128, 0, stream>>>(table, m, n, k, (int)pa, (int)pb);
-    split_planes_kernel<false><<<dim3(blocks(k), blocks(m)), 256, 0, stream>>>(A, a_hi, a_lo, m, k, (int)pa, SplitScale{nullptr, 0, 0});
-    split_planes_kernel<true><<<dim3(blocks(n), blocks(k)), 256, 0, stream>>>(B, b_hi, b_lo, k, n, (int)pb, SplitScale{nullptr, 0, 0});
+    split_planes_kernel<false><<<dim3(blocks(k), blocks(m)), 256, 0, stream>>>(A, a_hi, a_lo, m, k, (int)pa, SplitScale{nullptr, 0, 0}, 0);
+    split_planes_kernel<true><<<dim3(blocks(n), blocks(k)), 256, 0, stream>>>(B, b_hi, b_lo, k, n, (int)pb, SplitScale{nullptr, 0, 0}, 0);
     if (cudaGetLastError() != cudaSuccess) return MOM_ERR_CUDA;
 
     CUtensorMap ma_hi, ma_lo, mb_hi, mb_lo, mc;
@@ -1234,6 +1276,7 @@ extern "C" mom_status_t mom_product_3xtf32_noalloc(int64_t m64, int64_t n64, int
     prm.out_mode = 0;
     prm.slice_rows = 0;
     prm.mirror = 0;
+    prm.packed_c = nullptr;
     prm.add.count = 0;
     prm.status = status;
     product_tc_kernel<<<std::min(prm.num_tiles, sm_count), THREADS, SMEM_BYTES, stream>>>(ma_hi, ma_lo, mb_hi, mb_lo, mc, mc, prm);

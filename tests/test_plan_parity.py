@@ -446,3 +446,48 @@ def test_planning_from_several_threads():
     for t in threads:
         t.join()
     assert all(g == want for g in got)
+
+
+def test_packed_container_matches_the_oracle_definition():
+    # integer work: the library's closed forms against the oracle's row-by-row sums, bit for bit
+    from oracle import packed as pk
+    for n in list(range(1, 41)) + [63, 64, 65, 200, 333]:
+        for prop in (wl.LOWER_TRI, wl.UPPER_TRI, wl.STRICT_LOWER, wl.STRICT_UPPER, wl.UNIT_LOWER, wl.UNIT_UPPER):
+            oracle_prop = pk.LOWER_TRI if prop in (wl.LOWER_TRI, wl.STRICT_LOWER, wl.UNIT_LOWER) else pk.UPPER_TRI
+            assert mom.mom_packed_elements(n, prop) == pk.elements(n, oracle_prop)
+            for i in sorted({0, 1, 2, 3, 4, n // 2, n - 2, n - 1} & set(range(n))):
+                off, first, end = mom.mom_packed_row(n, prop, i)
+                assert off == pk.row_offset(n, oracle_prop, i) and (first, end) == pk.row_range(n, oracle_prop, i)
+    for prop in (wl.GENERAL, wl.IDENTITY, wl.DIAGONAL, wl.SYMMETRIC):
+        with pytest.raises(mom.MomError) as e:
+            mom.mom_packed_elements(8, prop)
+        assert e.value.status == mom.ERR_PROPERTY
+    with pytest.raises(mom.MomError) as e:
+        mom.mom_packed_row(8, wl.LOWER_TRI, 8)
+    assert e.value.status == mom.ERR_INVALID_ARG
+    # the input generator's packing agrees with the oracle's
+    rng = np.random.default_rng(1)
+    for n in (1, 5, 8, 13, 64):
+        a = rng.standard_normal((n, n)).astype(np.float32)
+        assert np.array_equal(wl.pack_triangle(np.tril(a), True), pk.pack(np.tril(a), pk.LOWER_TRI))
+        assert np.array_equal(wl.pack_triangle(np.triu(a), False), pk.pack(np.triu(a), pk.UPPER_TRI))
+
+
+def test_storage_changes_neither_the_plan_nor_its_costs():
+    P = mom.STORAGE_PACKED
+    for seed in range(60):
+        eq = wl.random_equation(seed, max_len=6, max_dim=40)
+        descs = eq.descs()
+        storage = [P if d[2] in (wl.LOWER_TRI, wl.UPPER_TRI) and seed % 2 == 0 else 0 for d in descs]
+        got = mom.mom_equation_plan_stored(descs, None, storage, eq.add_descs(), None, None, 0, mom.VARIANT_3XTF32)
+        want = op.plan(descs, eq.add_descs())
+        assert got.parenthesization() == want.paren and got.flops() == (want.mul_flops, want.add_flops)
+        rd = got.result_desc()
+        assert got.result_elements() == rd.rows * rd.cols
+    # sizes: the packed X of L*L, and the workspace the storage layer adds where no kernel reads the container in place
+    n = 200
+    dense = mom.mom_equation_plan([(n, n, wl.LOWER_TRI), (n, n, wl.LOWER_TRI)], [], mom.VARIANT_FFMA)
+    packed = mom.mom_equation_plan_stored([(n, n, wl.LOWER_TRI), (n, n, wl.LOWER_TRI)], None, [P, P], (), None, None, P, mom.VARIANT_FFMA)
+    assert packed.result_elements() == mom.mom_packed_elements(n, wl.LOWER_TRI) == n * (n + 4) // 2
+    assert packed.workspace_bytes(1) >= dense.workspace_bytes(1) + 3 * n * n * 4       # two dense copies and a dense X
+    assert packed.host_staging_bytes(1) < dense.host_staging_bytes(1) + 3 * n * n * 4

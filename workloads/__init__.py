@@ -126,6 +126,22 @@ def generate(eq: Equation):
     return chain, add
 
 
+def pack_triangle(a: np.ndarray, lower: bool) -> np.ndarray:
+    """A dense triangular matrix (or a stack of them, instance first) as a packed container: rows one after the other,
+    row i holding columns [0, 4 * (i // 4 + 1)) of a lower triangle, or [4 * (i // 4), n rounded up to a multiple of 4)
+    of an upper one; positions past the last column are zero.  Layout only: an input is re-arranged, nothing is computed."""
+    a = np.asarray(a, dtype=np.float32)
+    n = a.shape[-1]
+    n4 = 4 * ((n + 3) // 4)
+    padded = np.zeros(a.shape[:-1] + (n4,), dtype=np.float32)
+    padded[..., :n] = a
+    rows = np.arange(n)[:, None]
+    cols = np.arange(n4)[None, :]
+    group = 4 * (rows // 4)
+    keep = (cols < group + 4) if lower else (cols >= group)
+    return np.ascontiguousarray(padded[..., keep])          # boolean selection walks the matrix row by row
+
+
 # --------------------------------------------------------------------------
 # The benchmark's configurations (shapes, properties, distributions, seeds).
 # --------------------------------------------------------------------------
