@@ -306,9 +306,15 @@ def time_equation(mom, torch, eq, variant, steps, warmup, stream, timing=False, 
         eq = wl.Equation(eq.name, eq.seed, tuple(o for c in eq.chains for o in c))     # batch 1, for the code below
     elif chain_storage is not None:
         chain, add = wl.generate(eq)
-        plan = mom.mom_equation_plan_stored(eq.descs(), eq.chain_t, chain_storage, eq.add_descs(), eq.add_t, None, mom.STORAGE_DENSE, variant)
+        # triangular Add terms travel packed too, and so does X when every summand is a triangle of one orientation
         lower = (wl.LOWER_TRI, wl.STRICT_LOWER, wl.UNIT_LOWER)
+        tri = lower + (wl.UPPER_TRI, wl.STRICT_UPPER, wl.UNIT_UPPER)
+        add_storage = [mom.STORAGE_PACKED if o.prop in tri else mom.STORAGE_DENSE for o in eq.add]
+        dense_plan = mom.mom_equation_plan_transposed(eq.descs(), eq.chain_t, eq.add_descs(), eq.add_t, variant)
+        x_storage = mom.STORAGE_PACKED if dense_plan.result_desc().property in tri else mom.STORAGE_DENSE
+        plan = mom.mom_equation_plan_stored(eq.descs(), eq.chain_t, chain_storage, eq.add_descs(), eq.add_t, add_storage, x_storage, variant)
         chain = [a if s == mom.STORAGE_DENSE or a is None else wl.pack_triangle(a, o.prop in lower) for a, o, s in zip(chain, eq.chain, chain_storage)]
+        add = [a if s == mom.STORAGE_DENSE or a is None else wl.pack_triangle(a, o.prop in lower) for a, o, s in zip(add, eq.add, add_storage)]
         dchain = [None if a is None else torch.from_numpy(a).cuda() for a in chain]
     else:
         chain, add = wl.generate(eq)
@@ -326,7 +332,7 @@ def time_equation(mom, torch, eq, variant, steps, warmup, stream, timing=False, 
 
     def run():
         if eq.batch > 1:
-            plan.execute_batched(cp, cs, ap, as_, out.data_ptr(), rd.rows * rd.cols, eq.batch,
+            plan.execute_batched(cp, cs, ap, as_, out.data_ptr(), plan.result_elements(), eq.batch,
                                  ws.data_ptr() if wsb else None, wsb, stream.cuda_stream)
         else:
             plan.execute(cp, ap, out.data_ptr(), ws.data_ptr() if wsb else None, wsb, stream.cuda_stream)
@@ -366,7 +372,7 @@ def time_equation(mom, torch, eq, variant, steps, warmup, stream, timing=False, 
     if status != (0, 0):
         raise RuntimeError(f"device-side wait timed out: {status}")
     mul, addf = plan.flops()
-    stored_bytes = 4 * (sum(t.numel() for t in dchain if t is not None) + sum(t.numel() for t in dadd if t is not None) + out.numel())
+    stored_bytes = 4 * (sum(t.numel() for t in dchain if t is not None) + sum(t.numel() for t in dadd if t is not None) + plan.result_elements() * eq.batch)
     return {"ms": ms, "ms_back_to_back": ms_b2b, "plan": plan, "stored_bytes": stored_bytes, "useful_flops": (mul + addf) * eq.batch, "launches": plan.last_launch_count(),
             "step_times": step_times, "host": (chain, add), "keep": (dchain, dadd, out, ws)}
 
@@ -403,10 +409,15 @@ def run_gpu(args):
         cfgs = {c.name: c for c in (wl.config_tiny(), wl.config_five_general(), wl.config_property_heavy(),
                                     wl.config_large_square(), wl.config_batched(), wl.config_paper_chain(),
                                     wl.config_transposed(), wl.config_sum_shared(), wl.config_sum_triangular(),
-                                    wl.config_expression(), wl.config_diagonal(), wl.config_gram())}
-        cfg = cfgs[args.only]
+                                    wl.config_expression(), wl.config_diagonal(), wl.config_gram(), wl.config_square_product(1024),
+                                    wl.config_square_product(1536), wl.config_square_product(2048), wl.config_packed_triangular())}
+        packed = args.only.endswith("_packed")       # the same equation with its triangular operands handed over as packed triangles
+        cfg = cfgs[args.only[:-len("_packed")] if packed else args.only]
+        storage = None
+        if packed:
+            storage = [mom.STORAGE_PACKED if o.prop in (wl.LOWER_TRI, wl.UPPER_TRI) else mom.STORAGE_DENSE for o in cfg.chain]
         r = time_equation(mom, torch, cfg, variant, steps=args.steps, warmup=args.warmup, stream=stream,
-                          timing=getattr(cfg, "batch", 1) == 1)
+                          timing=getattr(cfg, "batch", 1) == 1 and not packed, chain_storage=storage)
         print(json.dumps({"workload": cfg.name, "variant": args.variant, "ms": r["ms"], "ms_back_to_back": r["ms_back_to_back"],
                           "useful_flops": r["useful_flops"],
                           "launches": r["launches"], "step_times_ms": r["step_times"][-1:] }))
@@ -581,7 +592,8 @@ def run_gpu(args):
         others = []
         for cfg in (wl.config_tiny(), wl.config_five_general(), wl.config_property_heavy(), wl.config_batched(),
                     wl.config_paper_chain(), wl.config_transposed(), wl.config_sum_shared(), wl.config_sum_triangular(),
-                    wl.config_expression(), wl.config_diagonal(), wl.config_gram()):
+                    wl.config_expression(), wl.config_diagonal(), wl.config_gram(), wl.config_square_product(1024),
+                    wl.config_square_product(1536), wl.config_square_product(2048)):
             batch = getattr(cfg, "batch", 1)
             r = time_equation(mom, torch, cfg, variant, steps=20, warmup=3, stream=stream, timing=batch == 1)
             ms_min, ms_med = min(r["ms"]), statistics.median(r["ms"])

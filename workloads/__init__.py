@@ -217,6 +217,18 @@ def config_diagonal(n: int = 4096, seed: int = 10) -> Equation:
         (Operand(n, n, GENERAL, "normal"),))
 
 
+def config_square_product(n: int = 1024, seed: int = 12) -> Equation:
+    """One general product A*B, both n x n, N(0, 1/n): the mid-size range between the small-product kernel and the large
+    tensor-core products (timed at 1024, 1536 and 2048)."""
+    g = Operand(n, n, GENERAL, "normal", 1.0 / np.sqrt(n))
+    return Equation(f"GG_{n}", seed, (g, g))
+
+
+def config_packed_triangular(n: int = 4096, seed: int = 13) -> Equation:
+    """X = L*L + L with both factors, the term and X meant for packed storage (the storage is chosen by the caller)."""
+    return Equation(f"LL_plus_L_{n}", seed, (Operand(n, n, LOWER_TRI), Operand(n, n, LOWER_TRI)), (Operand(n, n, LOWER_TRI),))
+
+
 def config_listing2() -> Equation:
     """Listing 2 of the paper: two 5x5 lowerTri matrices filled with the constant 1."""
     return Equation("listing2_LL_5", 0, (
