@@ -100,17 +100,22 @@ typedef enum { MOM_F32 = 0 } mom_dtype_t;
  *   MOM_VARIANT_3XTF32: tensor-core MMA (kind::tf32 / .tf32) on operands split as a = hi + lo,
  *       accumulating lo*hi + hi*lo + hi*hi in f32 (f32-level accuracy).  Large products
  *       (m*n*k >= 6 * 2^26) whose shapes TMA can address (leading dimensions that are multiples of 4
- *       elements) run on the tcgen05 kernel (operand planes, TMA, tensor memory).  Smaller products and
- *       the other shapes run on the warp-level kernel (mma.sync on the operands as stored, one launch per
- *       product): below that size the tcgen05 path's extra passes cost more than they save.
+ *       elements) run on the tcgen05 kernel that takes its operands as hi / lo planes (a pre-pass writes them;
+ *       TMA, tensor memory, persistent CTAs).  Smaller products of stored (untransposed) operands run on the
+ *       tcgen05 kernel that reads the operands as stored and splits them in shared memory: one launch per
+ *       product.  The rest (transposed operands, leading dimensions TMA cannot address, fewer than 2^21
+ *       multiplications, batches) run on the warp-level kernel (mma.sync on the operands as stored, one launch).
  *   MOM_VARIANT_FFMA: plain f32 fused multiply-add on CUDA cores.
  *   MOM_VARIANT_3XTF32_FORCE: every TMA-addressable product runs on the tcgen05 kernel, the others on
  *       the FFMA kernel; meant for testing the tcgen05 kernel on small shapes.
  *   MOM_VARIANT_3XTF32_WARP: every product runs on the warp-level kernel; meant for testing it on
  *       large shapes.
+ *   MOM_VARIANT_3XTF32_INLINE: every product the in-kernel-split tcgen05 kernel takes runs there, whatever its
+ *       size, the others on the warp-level kernel; meant for testing.
  * Whatever the variant, equations small enough for shared memory run as one fused launch, and products
  * with a Diagonal factor run on the scaling kernel. */
-typedef enum { MOM_VARIANT_3XTF32 = 0, MOM_VARIANT_FFMA = 1, MOM_VARIANT_3XTF32_FORCE = 2, MOM_VARIANT_3XTF32_WARP = 3 } mom_variant_t;
+typedef enum { MOM_VARIANT_3XTF32 = 0, MOM_VARIANT_FFMA = 1, MOM_VARIANT_3XTF32_FORCE = 2, MOM_VARIANT_3XTF32_WARP = 3,
+               MOM_VARIANT_3XTF32_INLINE = 4 } mom_variant_t;
 
 /* Kind of a binary product, by which operands are triangular. */
 typedef enum {
@@ -135,7 +140,8 @@ typedef struct {
     int32_t lhs, rhs, out;
     int32_t kind;                    /* mom_kind_t */
     int32_t lhs_property, rhs_property, out_property;
-    int32_t uses_tensor_cores;       /* 1: tcgen05 3xTF32 kernel, 2: warp-level 3xTF32 kernel, 0: FFMA kernel (MOM_KIND_SCALE: the scaling kernel) */
+    int32_t uses_tensor_cores;       /* 1: tcgen05 3xTF32 kernel on operand planes, 3: tcgen05 3xTF32 kernel splitting in shared memory,
+                                        2: warp-level 3xTF32 kernel, 0: FFMA kernel (MOM_KIND_SCALE: the scaling kernel) */
     int32_t lhs_transposed, rhs_transposed;   /* the operand is read transposed (an original chain operand used transposed; the rhs of MOM_KIND_GRAM) */
     int64_t m, n, k;                 /* out is m x n, contraction length k */
     uint64_t useful_mults;           /* scalar multiplications with both factors structurally non-zero */

@@ -15,7 +15,7 @@ from typing import List, Optional, Sequence, Tuple
 GENERAL, LOWER_TRI, UPPER_TRI, IDENTITY, DIAGONAL, SYMMETRIC = 0, 1, 2, 3, 4, 5
 STRICT_LOWER, STRICT_UPPER, UNIT_LOWER, UNIT_UPPER = 6, 7, 8, 9
 F32 = 0
-VARIANT_3XTF32, VARIANT_FFMA, VARIANT_3XTF32_FORCE, VARIANT_3XTF32_WARP = 0, 1, 2, 3
+VARIANT_3XTF32, VARIANT_FFMA, VARIANT_3XTF32_FORCE, VARIANT_3XTF32_WARP, VARIANT_3XTF32_INLINE = 0, 1, 2, 3, 4
 STORAGE_DENSE, STORAGE_PACKED = 0, 1
 KIND_GG, KIND_TG, KIND_GT, KIND_TT, KIND_TTMIX, KIND_SCALE, KIND_GRAM = 0, 1, 2, 3, 4, 5, 6
 

@@ -15,7 +15,7 @@ struct DeviceInfo {
     int max_pairs = 0;               // co-resident clusters of the CTA-pair kernel (0: not asked yet)
     bool tc_attr = false;            // dynamic shared-memory limit raised for the tensor-core kernels on this device
     bool pair_attr = false;
-    bool chain_attr = false;
+    bool inline64_attr = false, inline128_attr = false;
     int fused_max_smem[2] = {0, 0};  // largest dynamic shared-memory size set for the fused small-equation kernels
     int batched_max_smem = 0;
 };

@@ -502,9 +502,17 @@ mom_status_t execute_core(const mom_plan *p, const float *const *chain_ptrs, con
                     launches += used;
                 } else {
                     if (ev) cudaEventRecord(ev[1], stream);
-                    const cudaError_t e = stp.pub.kind == MOM_KIND_SCALE ? launch_scale(a, nb, stream)
-                                          : stp.pub.uses_tensor_cores == 2 ? launch_product_mma(a, nb, stream)
-                                                                           : launch_product_ffma(a, nb, stream);
+                    cudaError_t e = cudaErrorNotSupported;
+                    if (stp.pub.kind == MOM_KIND_SCALE) {
+                        e = launch_scale(a, nb, stream);
+                    } else if (stp.pub.uses_tensor_cores == 3 || stp.pub.uses_tensor_cores == 2) {
+                        // the one-launch tcgen05 kernel takes one instance and 16-byte aligned operands; otherwise (and for
+                        // batches) the warp-level kernel
+                        if (stp.pub.uses_tensor_cores == 3 && nb == 1) e = launch_product_tc_inline(a, p->dev->status, stream);
+                        if (e == cudaErrorNotSupported) e = launch_product_mma(a, nb, stream);
+                    } else {
+                        e = launch_product_ffma(a, nb, stream);
+                    }
                     if (e != cudaSuccess) return MOM_ERR_CUDA;
                     ++launches;
                 }

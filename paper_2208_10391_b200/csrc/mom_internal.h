@@ -26,6 +26,10 @@ constexpr int FF_BN = 128;
 
 constexpr size_t WS_ALIGN = 256;
 
+// Default variant: products with fewer multiplications than this run on the warp-level kernel (its fixed cost is the
+// smallest), larger ones up to the large-product threshold on the in-kernel-split tcgen05 kernel.
+constexpr double INLINE_MIN_WORK = 2097152.0;
+
 // Largest rows / cols a descriptor may have: every kernel indexes rows, columns and k with 32-bit integers.
 constexpr int64_t MAX_DIMENSION = 2147483647 - 1024;
 // Largest m (and n) of a product on the tcgen05 kernel: a tile-table entry keeps the tile's first row in 24 bits

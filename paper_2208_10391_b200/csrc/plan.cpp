@@ -11,6 +11,7 @@
 
 #include "fused_small.h"
 #include "mom_internal.h"
+#include "product_tc.h"
 
 namespace {
 
@@ -229,7 +230,7 @@ static mom_status_t plan_sums(const std::vector<mom_matrix_desc_t> &slots, const
                               const int32_t *slot_names, const mom_matrix_desc_t *stored_add,
                               const int32_t *add_transposed, int32_t n_add, mom_variant_t variant, mom_plan_t **out_plan) {
     if (!out_plan || sums_in.empty() || n_add < 0 || (n_add > 0 && !stored_add)) return MOM_ERR_INVALID_ARG;
-    if ((int)variant < 0 || (int)variant > 3) return MOM_ERR_INVALID_ARG;
+    if ((int)variant < 0 || (int)variant > 4) return MOM_ERR_INVALID_ARG;
     int64_t total = 0;
     int n_chains = 0;
     for (const SumIn &si : sums_in) {
@@ -558,10 +559,17 @@ static mom_status_t plan_sums(const std::vector<mom_matrix_desc_t> &slots, const
             // below this size the tcgen05 path's extra launches (operand splits, split-K reduction) cost more
             // than its faster mainloop saves; the warp-level kernel is one launch
             const bool large = (double)m * (double)n * (double)k >= 6.0 * (double)(1 << 26);
+            // in between: the tcgen05 kernel that reads the operands as stored and splits them in shared memory (one launch);
+            // it takes stored (untransposed) operands whose rows TMA can address
+            const bool inline_ok = st.pub.kind != MOM_KIND_GRAM &&
+                                   mom::product_tc_inline_takes(m, n, k, st.pub.lhs_transposed, st.pub.rhs_transposed,
+                                                                mom::kernel_property(st.pub.lhs_property), mom::kernel_property(st.pub.rhs_property));
+            const bool tiny = (double)m * (double)n * (double)k < mom::INLINE_MIN_WORK;
             if (st.pub.kind == MOM_KIND_SCALE) st.pub.uses_tensor_cores = 0;       // a Diagonal operand: one scaling pass, bound by HBM
-            else if (variant == MOM_VARIANT_3XTF32) st.pub.uses_tensor_cores = addressable && large ? 1 : 2;
+            else if (variant == MOM_VARIANT_3XTF32) st.pub.uses_tensor_cores = addressable && large ? 1 : inline_ok && !tiny ? 3 : 2;
             else if (variant == MOM_VARIANT_3XTF32_FORCE) st.pub.uses_tensor_cores = addressable ? 1 : 0;
             else if (variant == MOM_VARIANT_3XTF32_WARP) st.pub.uses_tensor_cores = 2;
+            else if (variant == MOM_VARIANT_3XTF32_INLINE) st.pub.uses_tensor_cores = inline_ok ? 3 : 2;
             else st.pub.uses_tensor_cores = 0;
             if (st.pub.uses_tensor_cores == 1) {
                 // few output tiles, long contraction: split k over otherwise idle SMs
@@ -715,7 +723,7 @@ static mom_status_t plan_sums(const std::vector<mom_matrix_desc_t> &slots, const
             p->fused_value_off.assign(values, -1);
             size_t floats = 0;
             bool ok = single_chain && ns >= 1 && ns <= mom::FUSED_MAX_STEPS && (int)p->kept.size() <= mom::FUSED_MAX_OPERANDS &&
-                      n_add <= mom::MAX_FUSED_ADD && !any_tc && variant != MOM_VARIANT_3XTF32_WARP && !any_gram;
+                      n_add <= mom::MAX_FUSED_ADD && !any_tc && variant != MOM_VARIANT_3XTF32_WARP && variant != MOM_VARIANT_3XTF32_INLINE && !any_gram;
             // every value feeds exactly one product: remember on which side
             std::vector<char> is_rhs(values, 0);
             for (const auto &st : p->steps) is_rhs[st.pub.rhs] = 1;

@@ -29,6 +29,7 @@
 #include "product_tc.h"
 #include "tc_probe.h"
 #include "tc_ptx.cuh"
+#include "tc_wait.cuh"
 
 namespace mom {
 
@@ -48,7 +49,6 @@ constexpr int NUM_BARRIERS = 2 * STAGES + 4 + 1;
 constexpr int SMEM_BYTES = 1024 + STAGES * STAGE_BYTES + EPI_BYTES + 256;
 constexpr int THREADS = 192;
 constexpr uint32_t TMEM_COLS = 512;          // two accumulators of BN columns
-constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;   // 2 s: far beyond any legitimate wait
 
 static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
 static_assert(SPLIT_BLOCK % BM == 0 && SPLIT_BLOCK % BN == 0, "split blocks must cover whole tiles");
@@ -60,31 +60,6 @@ struct Shared {
     uint32_t tmem_slot;
     volatile int *abort_flag;
 };
-
-__device__ __forceinline__ unsigned long long global_ns() {
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-    return t;
-}
-
-// Bounded wait: false when the limit was reached (records the failure) or another role gave up.
-__device__ __forceinline__ bool wait_barrier(uint32_t bar, uint32_t parity, volatile int *abort_flag, int32_t *status, int detail,
-                                             unsigned long long limit_ns = WAIT_LIMIT_NS) {
-    unsigned long long start = 0;
-    for (uint32_t i = 0;; ++i) {
-        if (ptx::mbar_try_wait(bar, parity)) return true;
-        if ((i & 63) == 63) {
-            if (*abort_flag) return false;
-            const unsigned long long now = global_ns();
-            if (start == 0) start = now;
-            else if (now - start > limit_ns) break;
-        }
-    }
-    if (atomicCAS(status, 0, (int)MOM_ERR_DEVICE_TIMEOUT) == 0) status[1] = detail;
-    *abort_flag = 1;
-    __threadfence_block();
-    return false;
-}
 
 // tile table entry: x = first row | k-slice << 24, y = first column, z..w = k-range
 constexpr int TILE_SLICE_SHIFT = 24;
@@ -731,8 +706,10 @@ EncodeTiledFn encode_fn() {
     return fn;
 }
 
+}  // namespace
+
 // 2-D f32 row-major matrix (rows x cols), box of box_rows x box_cols elements
-bool make_map(CUtensorMap *map, const void *ptr, int rows, int cols, int box_rows, int box_cols, CUtensorMapSwizzle swz) {
+bool tc_make_map(CUtensorMap *map, const void *ptr, int rows, int cols, int box_rows, int box_cols, CUtensorMapSwizzle swz) {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
     const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
@@ -742,6 +719,11 @@ bool make_map(CUtensorMap *map, const void *ptr, int rows, int cols, int box_row
     return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void *>(ptr), dims, strides, box, elem,
               CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+namespace {
+inline bool make_map(CUtensorMap *map, const void *ptr, int rows, int cols, int box_rows, int box_cols, CUtensorMapSwizzle swz) {
+    return tc_make_map(map, ptr, rows, cols, box_rows, box_cols, swz);
 }
 
 }  // namespace

@@ -1,6 +1,7 @@
 // Tensor-core (tcgen05, 3xTF32) product path: host-side interface used by the launcher.
 #pragma once
 
+#include <cuda.h>
 #include <cuda_runtime.h>
 
 #include "kernels.h"
@@ -43,6 +44,14 @@ mom_status_t tc_launch_step(const mom_plan &p, TcPlanState &s, int step, const P
                             int32_t *status, cudaStream_t stream, int *launches, cudaEvent_t before_product, int part = 0);
 
 void tc_release(TcPlanState &s);
+
+// Tensor map of a 2-D f32 row-major matrix (rows x cols) with a box of box_rows x box_cols elements.
+bool tc_make_map(CUtensorMap *map, const void *ptr, int rows, int cols, int box_rows, int box_cols, CUtensorMapSwizzle swizzle);
+
+// The small / mid-size product kernel (product_tc_inline.cu): one launch, operands read as stored and split in shared
+// memory.  Returns cudaErrorNotSupported when the product is not of a shape it takes (the caller then uses another kernel).
+cudaError_t launch_product_tc_inline(const ProductArgs &a, int32_t *status, cudaStream_t stream);
+bool product_tc_inline_takes(int64_t m, int64_t n, int64_t k, int lhs_transposed, int rhs_transposed, int pa, int pb);
 
 // One thread waits with the product kernels' bounded wait on a barrier nothing arrives on; after `limit_ns` it
 // records {MOM_ERR_DEVICE_TIMEOUT, detail} in `status` (device, 4 ints) and the kernel ends.

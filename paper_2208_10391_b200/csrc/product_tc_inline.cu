@@ -1,0 +1,360 @@
+// Small and mid-size products on the tcgen05 tensor cores in ONE launch: C = A*B (+ Add terms), 3xTF32, with the
+// operands read as stored and split into their tf32 halves in shared memory.
+//
+// The large-product kernel (product_tc.cu) takes its operands as hi / lo planes that a pre-pass writes to global
+// memory, and with few output tiles it needs a split-K reduction pass: two or three launches, which is most of the
+// time of a product below about 2000^3.  Here a product is one launch:
+//   warp 0      TMA producer: per k-block of 32 the raw f32 tile of A (128 rows x 32 k: already K-major, loaded under
+//               the 128-byte swizzle the MMA wants) and the raw tile of B (32 k-rows x BN columns, as BN / 32 swizzled
+//               boxes of 32 x 32);
+//   warps 2-5   transform: A is split where it lies (the hi half overwrites the raw tile, the lo half goes to a second
+//               tile at the same offsets); B is split AND transposed into K-major hi / lo tiles (BN rows of 32 k): a lane
+//               reads four columns of its k-row with one 16-byte load -- the eight lanes of a load phase hit eight
+//               different swizzled chunks -- and writes each value into its column's row, where the 32 lanes of a
+//               warp fill one 128-byte row: no bank conflict on either side;
+//   warp 1      MMA issuer: 4 k-steps x 3 tcgen05.mma kind::tf32 (lo*hi, hi*lo, hi*hi; M128, N = BN) per k-block into one
+//               accumulator in tensor memory; tcgen05.commit frees the stage;
+//   warps 2-5   then the epilogue: tcgen05.ld, Add terms, structure mask, 16-byte stores.
+// With few output tiles the contraction is split over the CTAs of a thread-block cluster (up to 8): each leaves its partial
+// tile in its own shared memory and CTA r finishes rows [r * 128 / s, (r + 1) * 128 / s) by adding the partial tiles through
+// distributed shared memory in k order (deterministic; no atomics, no scratch in global memory, no second launch).
+// The tile's structural k-range bounds the contraction as everywhere else.  Shared memory moves about twice the bytes per
+// flop that the plane kernel moves (the transform reads and writes every operand byte once more), so this kernel tops out
+// near half of the tensor peak; it is chosen where launches, not flops, are the cost.
+// Every wait is bounded; a CTA that gives up still meets its cluster at both cluster barriers.
+#include <algorithm>
+#include <cstring>
+
+#include <cooperative_groups.h>
+#include <cuda.h>
+
+#include "device_info.h"
+#include "product_tc.h"
+#include "tc_ptx.cuh"
+#include "tc_wait.cuh"
+
+namespace mom {
+
+namespace {
+
+namespace cg = cooperative_groups;
+
+constexpr int IBM = 128, IBK = 32, ITHREADS = 192, IMAX_SPLIT = 8;
+
+template <int BN>
+struct InlineCfg {
+    static constexpr int STAGES = BN == 64 ? 3 : 2;
+    static constexpr int A_BYTES = IBM * IBK * 4;            // 16 KB: the raw tile, then its hi half
+    static constexpr int B_RAW_BYTES = IBK * BN * 4;         // BN / 32 boxes of 32 k-rows x 32 columns
+    static constexpr int B_PLANE_BYTES = BN * IBK * 4;       // K-major: BN rows of 32 k
+    static constexpr int STAGE_BYTES = 2 * A_BYTES + B_RAW_BYTES + 2 * B_PLANE_BYTES;
+    static constexpr int LDP = BN + 4;                       // row length of the partial tile (floats)
+    static constexpr int NUM_BARRIERS = 3 * STAGES + 2;
+    static constexpr int SMEM_BYTES = 1024 + STAGES * STAGE_BYTES + 256;
+    static_assert(IBM * LDP * 4 <= STAGES * STAGE_BYTES, "the partial tile reuses the stages");
+    static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
+};
+
+struct InlineParams {
+    int m, n, k;
+    int pa, pb, pout;
+    int split, tiles_n;
+    float *C;
+    AddTerms add;
+    int32_t *status;
+};
+
+// hi = a rounded to tf32 (nearest, ties away from zero, done on the bit pattern with full-rate integer instructions),
+// lo = (a - hi) rounded the same way: the halves the operand-split pass of the large-product kernel writes
+__device__ __forceinline__ float tf32_round(float a) { return __uint_as_float((__float_as_uint(a) + 0x1000u) & 0xFFFFE000u); }
+__device__ __forceinline__ void split4(const float4 a, float4 &hi, float4 &lo) {
+    hi.x = tf32_round(a.x); hi.y = tf32_round(a.y); hi.z = tf32_round(a.z); hi.w = tf32_round(a.w);
+    lo.x = tf32_round(a.x - hi.x); lo.y = tf32_round(a.y - hi.y); lo.z = tf32_round(a.z - hi.z); lo.w = tf32_round(a.w - hi.w);
+}
+
+// K-major tile with 128-byte rows under the 128B swizzle: 8-row groups are 1024 bytes apart, a K = 8 step is 32 bytes
+__device__ __forceinline__ uint64_t kmajor_desc128(uint32_t tile, int kstep) {
+    return ptx::smem_desc(tile + kstep * 32, 16, 8 * 128, ptx::SWIZZLE_128B);
+}
+
+template <int BN>
+__global__ void __launch_bounds__(ITHREADS, 1)
+product_tc_inline_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const InlineParams prm) {
+    using Cfg = InlineCfg<BN>;
+    constexpr int S = Cfg::STAGES;
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ int abort_word;
+    const uint32_t base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t *const base_ptr = smem_raw + (base - ptx::smem_u32(smem_raw));
+    const uint32_t bars = base + S * Cfg::STAGE_BYTES;
+    auto raw_full = [&](int s) { return bars + 8 * s; };
+    auto ready = [&](int s) { return bars + 8 * (S + s); };
+    auto empty = [&](int s) { return bars + 8 * (2 * S + s); };
+    const uint32_t acc_full = bars + 8 * (3 * S), drain = bars + 8 * (3 * S + 1), tmem_slot = bars + 8 * Cfg::NUM_BARRIERS;
+    volatile int *abort_flag = &abort_word;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    cg::cluster_group cluster = cg::this_cluster();
+    const int split = prm.split;
+    const int rank = split > 1 ? (int)cluster.block_rank() : 0;          // position in the cluster = k-slice
+    const int tile = blockIdx.x / split;
+    const int r0 = (tile / prm.tiles_n) * IBM, c0 = (tile % prm.tiles_n) * BN;
+
+    int klo, khi;
+    tile_k_range(prm.pa, prm.pb, r0, min(r0 + IBM, prm.m), c0, min(c0 + BN, prm.n), prm.k, &klo, &khi);
+    klo &= ~(IBK - 1);                                                   // extra leading elements are stored zeros
+    const int blocks = klo < khi ? (khi - klo + IBK - 1) / IBK : 0;
+    const int per = (blocks + split - 1) / split;
+    const int kb0 = min(rank * per, blocks), nk = min(kb0 + per, blocks) - kb0;
+
+    if (threadIdx.x == 0) {
+        abort_word = 0;
+        for (int s = 0; s < S; ++s) { ptx::mbar_init(raw_full(s), 1); ptx::mbar_init(ready(s), 4); ptx::mbar_init(empty(s), 1); }
+        ptx::mbar_init(acc_full, 1);
+        ptx::mbar_init(drain, 1);
+        ptx::fence_barrier_init();
+    }
+    if (warp == 1) {
+        ptx::tmem_alloc(tmem_slot, BN);
+        ptx::tmem_relinquish();
+    }
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    ptx::tc_fence_after_sync();
+    uint32_t tmem_base;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(tmem_base) : "r"(tmem_slot));
+
+    bool acc_ok = nk > 0;                        // the accumulator holds this CTA's partial sums (epilogue warps)
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer
+        bool ok = true;
+        for (int i = 0; i < nk && ok; ++i) {
+            const int s = i % S;
+            if (lane == 0) ok = wait_barrier(empty(s), ((i / S) & 1) ^ 1, abort_flag, prm.status, (11 << 24) | (s << 16) | (tile & 0xFFFF));
+            ok = __shfl_sync(0xffffffffu, ok, 0);
+            if (!ok) break;
+            if (lane == 0) ptx::mbar_arrive_expect_tx(raw_full(s), Cfg::A_BYTES + Cfg::B_RAW_BYTES);
+            __syncwarp();
+            const int kb = klo + (kb0 + i) * IBK;
+            const uint32_t st = base + s * Cfg::STAGE_BYTES;
+            if (lane == 0) ptx::tma_load_2d(st, &map_a, kb, r0, raw_full(s));
+            else if (lane <= BN / 32) ptx::tma_load_2d(st + 2 * Cfg::A_BYTES + (lane - 1) * 4096, &map_b, c0 + 32 * (lane - 1), kb, raw_full(s));
+        }
+        if (*abort_flag && lane == 0) {          // failure path: loads still in flight land before the CTA's memory goes away
+            const unsigned long long t0 = global_ns();
+            while (global_ns() - t0 < 200000ull) { }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer (one thread)
+        if (lane == 0) {
+            constexpr uint32_t idesc = ptx::instr_desc_tf32(IBM, BN, 0, 0);
+            uint32_t accumulate = 0;
+            bool ok = true;
+            for (int i = 0; i < nk; ++i) {
+                const int s = i % S;
+                ok = wait_barrier(ready(s), (i / S) & 1, abort_flag, prm.status, (12 << 24) | (s << 16) | (tile & 0xFFFF));
+                if (!ok) break;
+                ptx::tc_fence_after_sync();
+                const uint32_t a_hi = base + s * Cfg::STAGE_BYTES, a_lo = a_hi + Cfg::A_BYTES;
+                const uint32_t b_hi = a_hi + 2 * Cfg::A_BYTES + Cfg::B_RAW_BYTES, b_lo = b_hi + Cfg::B_PLANE_BYTES;
+#pragma unroll
+                for (int ks = 0; ks < IBK / 8; ++ks) {
+                    const uint64_t da_hi = kmajor_desc128(a_hi, ks), da_lo = kmajor_desc128(a_lo, ks);
+                    const uint64_t db_hi = kmajor_desc128(b_hi, ks), db_lo = kmajor_desc128(b_lo, ks);
+                    ptx::mma_tf32(tmem_base, da_lo, db_hi, idesc, accumulate);       // small terms first
+                    ptx::mma_tf32(tmem_base, da_hi, db_lo, idesc, 1);
+                    ptx::mma_tf32(tmem_base, da_hi, db_hi, idesc, 1);
+                    accumulate = 1;
+                }
+                ptx::mma_commit(empty(s));                   // the stage may be refilled once these MMAs have read it
+            }
+            if (ok && nk > 0) ptx::mma_commit(acc_full);
+            if (*abort_flag) {                               // failure path: issued MMAs finish before tensor memory is freed
+                ptx::mma_commit(drain);
+                for (uint32_t i = 0; i < (1u << 20); ++i)
+                    if (ptx::mbar_try_wait(drain, 0)) break;
+            }
+        }
+        __syncwarp();
+    } else {
+        // ------------------------------------------------------------------ transform (warps 2..5), then epilogue
+        const int tid2 = threadIdx.x - 64, w2 = warp - 2;
+        bool ok = true;
+        for (int i = 0; i < nk && ok; ++i) {
+            const int s = i % S;
+            if (lane == 0) ok = wait_barrier(raw_full(s), (i / S) & 1, abort_flag, prm.status, (13 << 24) | (s << 16) | (tile & 0xFFFF));
+            ok = __shfl_sync(0xffffffffu, ok, 0);
+            if (!ok) break;
+            uint8_t *const st = base_ptr + s * Cfg::STAGE_BYTES;
+            // A: 128 rows x 8 groups of 16 bytes, split where they lie (the swizzle is a permutation of the groups: offsets stay)
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                float4 *p = reinterpret_cast<float4 *>(st) + tid2 + 128 * u;
+                float4 hi, lo;
+                split4(*p, hi, lo);
+                *p = hi;
+                *(p + Cfg::A_BYTES / 16) = lo;
+            }
+            // B: box j holds k-rows 0..31 x columns 32 j .. 32 j + 31, group c of row k at group c ^ (k & 7).  Lane = k-row.
+            uint8_t *const braw = st + 2 * Cfg::A_BYTES, *const bhi = braw + Cfg::B_RAW_BYTES, *const blo = bhi + Cfg::B_PLANE_BYTES;
+#pragma unroll
+            for (int task = w2; task < BN / 4; task += 4) {
+                const int j = task >> 3, c = task & 7;
+                const float4 v = *reinterpret_cast<const float4 *>(braw + j * 4096 + lane * 128 + ((c ^ (lane & 7)) << 4));
+                float4 hi, lo;
+                split4(v, hi, lo);
+                const int n0 = 32 * j + 4 * c;                           // column of v.x inside the tile = row of the K-major tile
+                const uint32_t in_row = (uint32_t)(lane & 3) << 2;       // k = lane: group lane / 4, word lane % 4
+                const uint32_t group = (uint32_t)lane >> 2;
+                const uint32_t o0 = (n0 + 0) * 128 + ((group ^ ((n0 + 0) & 7)) << 4) + in_row, o1 = (n0 + 1) * 128 + ((group ^ ((n0 + 1) & 7)) << 4) + in_row;
+                const uint32_t o2 = (n0 + 2) * 128 + ((group ^ ((n0 + 2) & 7)) << 4) + in_row, o3 = (n0 + 3) * 128 + ((group ^ ((n0 + 3) & 7)) << 4) + in_row;
+                *reinterpret_cast<float *>(bhi + o0) = hi.x; *reinterpret_cast<float *>(blo + o0) = lo.x;
+                *reinterpret_cast<float *>(bhi + o1) = hi.y; *reinterpret_cast<float *>(blo + o1) = lo.y;
+                *reinterpret_cast<float *>(bhi + o2) = hi.z; *reinterpret_cast<float *>(blo + o2) = lo.z;
+                *reinterpret_cast<float *>(bhi + o3) = hi.w; *reinterpret_cast<float *>(blo + o3) = lo.w;
+            }
+            ptx::fence_proxy_async_smem();                   // the MMA reads these tiles through the asynchronous proxy
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(ready(s));
+        }
+        // ---- epilogue: this warp reads TMEM lanes 32 q .. 32 q + 31 = rows of the tile
+        const int q = warp & 3, row = q * 32 + lane, r = r0 + row;
+        if (nk > 0 && ok) {
+            if (lane == 0) ok = wait_barrier(acc_full, 0, abort_flag, prm.status, (14 << 24) | (tile & 0xFFFF));
+            ok = __shfl_sync(0xffffffffu, ok, 0);
+            ptx::tc_fence_after_sync();
+        }
+        acc_ok = nk > 0 && ok;
+        const bool vec = (reinterpret_cast<uintptr_t>(prm.C) & 15) == 0 && (prm.n & 3) == 0;
+        float *const P = reinterpret_cast<float *>(base_ptr);
+#pragma unroll 1
+        for (int c = 0; c < BN / 32; ++c) {
+            const int col0 = c0 + 32 * c;
+            float v[32];
+            if (acc_ok) {
+                ptx::tmem_ld_32cols(tmem_base + c * 32 + ((uint32_t)(q * 32) << 16), v);
+            } else {
+#pragma unroll
+                for (int j = 0; j < 32; ++j) v[j] = 0.0f;
+            }
+            if (split > 1) {
+                // partial sums into this CTA's shared memory (every stage has been consumed by now)
+#pragma unroll
+                for (int j = 0; j < 8; ++j)
+                    *reinterpret_cast<float4 *>(P + row * Cfg::LDP + 32 * c + 4 * j) = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+            } else if (r < prm.m) {
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const int cc = col0 + 4 * j;
+                    if (cc >= prm.n) break;
+                    float w[4] = {v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]};
+                    finish_row4(w, prm.add, 0, r, cc, prm.n, prm.n, prm.pout, vec);
+                    float *dst = prm.C + (long long)r * prm.n + cc;
+                    if (vec && cc + 3 < prm.n) {
+                        *reinterpret_cast<float4 *>(dst) = make_float4(w[0], w[1], w[2], w[3]);
+                    } else {
+#pragma unroll
+                        for (int e = 0; e < 4; ++e)
+                            if (cc + e < prm.n) dst[e] = w[e];
+                    }
+                }
+            }
+        }
+    }
+
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    ptx::tc_fence_after_sync();
+    if (warp == 1) ptx::tmem_dealloc(tmem_base, BN);
+    if (split == 1) return;
+
+    // ---- split contraction: CTA `rank` finishes its rows of the tile, adding the cluster's partial tiles in k order
+    cluster.sync();
+    {
+        const float *const P = reinterpret_cast<const float *>(base_ptr);
+        const bool vec = (reinterpret_cast<uintptr_t>(prm.C) & 15) == 0 && (prm.n & 3) == 0;
+        const int rows_per = IBM / split;
+        for (int e = threadIdx.x; e < rows_per * (BN / 4); e += ITHREADS) {
+            const int row = rank * rows_per + e / (BN / 4), col = (e % (BN / 4)) << 2;
+            const int r = r0 + row, cc = c0 + col;
+            if (r >= prm.m || cc >= prm.n) continue;
+            float w[4] = {0.f, 0.f, 0.f, 0.f};
+            for (int peer = 0; peer < split; ++peer) {
+                const float4 x = *reinterpret_cast<const float4 *>(cluster.map_shared_rank(P, peer) + row * Cfg::LDP + col);
+                w[0] += x.x; w[1] += x.y; w[2] += x.z; w[3] += x.w;
+            }
+            finish_row4(w, prm.add, 0, r, cc, prm.n, prm.n, prm.pout, vec);
+            float *dst = prm.C + (long long)r * prm.n + cc;
+            if (vec && cc + 3 < prm.n) {
+                *reinterpret_cast<float4 *>(dst) = make_float4(w[0], w[1], w[2], w[3]);
+            } else {
+                for (int j = 0; j < 4; ++j)
+                    if (cc + j < prm.n) dst[j] = w[j];
+            }
+        }
+    }
+    cluster.sync();                                          // nobody leaves while a peer may still read its tile
+}
+
+}  // namespace
+
+bool product_tc_inline_takes(int64_t m, int64_t n, int64_t k, int lhs_transposed, int rhs_transposed, int pa, int pb) {
+    auto plain = [](int p) { return p == MOM_GENERAL || p == MOM_LOWER_TRI || p == MOM_UPPER_TRI || p == MOM_SYMMETRIC; };
+    return !lhs_transposed && !rhs_transposed && (k & 3) == 0 && (n & 3) == 0 && plain(pa) && plain(pb) && m < (1 << 30) && n < (1 << 30) &&
+           k < (1 << 30);
+}
+
+cudaError_t launch_product_tc_inline(const ProductArgs &a, int32_t *status, cudaStream_t stream) {
+    if (!product_tc_inline_takes(a.m, a.n, a.k, a.transA, a.transB, a.pa, a.pb) || !status) return cudaErrorNotSupported;
+    if ((reinterpret_cast<uintptr_t>(a.A) | reinterpret_cast<uintptr_t>(a.B)) & 15) return cudaErrorNotSupported;
+    if (a.scaleA || a.scaleB || a.packedA || a.packedB || a.packedC) return cudaErrorNotSupported;
+    const int sm_count = current_sm_count();
+    if (sm_count < 1) return cudaErrorInvalidDevice;
+    const int tiles_m = (a.m + IBM - 1) / IBM;
+    // narrow tiles while 128-column ones would leave SMs without a tile
+    const bool narrow = a.n <= 64 || (long long)tiles_m * ((a.n + 127) / 128) < sm_count;
+    const int bn = narrow ? 64 : 128;
+    const int tiles_n = (a.n + bn - 1) / bn;
+    const long long tiles = (long long)tiles_m * tiles_n;
+    if (tiles * IMAX_SPLIT > (1ll << 30)) return cudaErrorNotSupported;
+    // few tiles and a long contraction: split k over a cluster, as long as every slice keeps two k-blocks
+    int split = 1;
+    while (split < IMAX_SPLIT && tiles * split * 2 <= sm_count && a.k / (split * 2) >= 2 * IBK) split *= 2;
+
+    CUtensorMap map_a, map_b;
+    if (!tc_make_map(&map_a, a.A, a.m, a.k, IBM, IBK, CU_TENSOR_MAP_SWIZZLE_128B) ||
+        !tc_make_map(&map_b, a.B, a.k, a.n, IBK, 32, CU_TENSOR_MAP_SWIZZLE_128B))
+        return cudaErrorNotSupported;
+    InlineParams prm;
+    prm.m = a.m; prm.n = a.n; prm.k = a.k;
+    prm.pa = a.pa; prm.pb = a.pb; prm.pout = a.pout;
+    prm.split = split;
+    prm.tiles_n = tiles_n;
+    prm.C = a.C;
+    prm.add = a.add;
+    prm.status = status;
+
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(tiles * split));
+    cfg.blockDim = dim3(ITHREADS);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = (unsigned)split;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = split > 1 ? 1 : 0;
+    if (bn == 64) {
+        cudaError_t e = raise_smem_limit_once(product_tc_inline_kernel<64>, InlineCfg<64>::SMEM_BYTES, &DeviceInfo::inline64_attr);
+        if (e != cudaSuccess) return e;
+        cfg.dynamicSmemBytes = InlineCfg<64>::SMEM_BYTES;
+        return cudaLaunchKernelEx(&cfg, product_tc_inline_kernel<64>, map_a, map_b, prm);
+    }
+    cudaError_t e = raise_smem_limit_once(product_tc_inline_kernel<128>, InlineCfg<128>::SMEM_BYTES, &DeviceInfo::inline128_attr);
+    if (e != cudaSuccess) return e;
+    cfg.dynamicSmemBytes = InlineCfg<128>::SMEM_BYTES;
+    return cudaLaunchKernelEx(&cfg, product_tc_inline_kernel<128>, map_a, map_b, prm);
+}
+
+}  // namespace mom

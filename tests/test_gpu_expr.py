@@ -9,7 +9,7 @@ from gpu_util import run_expression, check_expression_against_oracle
 
 pytestmark = pytest.mark.gpu
 
-VARIANTS = [mom.VARIANT_3XTF32, mom.VARIANT_FFMA, mom.VARIANT_3XTF32_FORCE, mom.VARIANT_3XTF32_WARP]
+VARIANTS = [mom.VARIANT_3XTF32, mom.VARIANT_FFMA, mom.VARIANT_3XTF32_FORCE, mom.VARIANT_3XTF32_WARP, mom.VARIANT_3XTF32_INLINE]
 
 
 def expression(name, operands, expr, seed=21):

@@ -16,8 +16,8 @@ from gpu_util import check_against_oracle, stratified_rows, CANARY
 pytestmark = pytest.mark.gpu
 
 D, P = mom.STORAGE_DENSE, mom.STORAGE_PACKED
-VARIANTS = [mom.VARIANT_3XTF32, mom.VARIANT_FFMA, mom.VARIANT_3XTF32_FORCE, mom.VARIANT_3XTF32_WARP]
-VNAME = {mom.VARIANT_FFMA: "ffma", mom.VARIANT_3XTF32_FORCE: "tc", mom.VARIANT_3XTF32: "auto", mom.VARIANT_3XTF32_WARP: "warp"}
+VARIANTS = [mom.VARIANT_3XTF32, mom.VARIANT_FFMA, mom.VARIANT_3XTF32_FORCE, mom.VARIANT_3XTF32_WARP, mom.VARIANT_3XTF32_INLINE]
+VNAME = {mom.VARIANT_FFMA: "ffma", mom.VARIANT_3XTF32_FORCE: "tc", mom.VARIANT_3XTF32: "auto", mom.VARIANT_3XTF32_WARP: "warp", mom.VARIANT_3XTF32_INLINE: "inline"}
 LOWER_KINDS = (wl.LOWER_TRI, wl.STRICT_LOWER, wl.UNIT_LOWER)
 
 

@@ -13,8 +13,9 @@ from gpu_util import run_equation, check_against_oracle, run_expression, check_e
 
 pytestmark = pytest.mark.gpu
 
-VARIANTS = [mom.VARIANT_FFMA, mom.VARIANT_3XTF32_FORCE, mom.VARIANT_3XTF32_WARP]
-VNAME = {mom.VARIANT_FFMA: "ffma", mom.VARIANT_3XTF32_FORCE: "tc", mom.VARIANT_3XTF32: "auto", mom.VARIANT_3XTF32_WARP: "warp"}
+VARIANTS = [mom.VARIANT_FFMA, mom.VARIANT_3XTF32_FORCE, mom.VARIANT_3XTF32_WARP, mom.VARIANT_3XTF32_INLINE]
+VNAME = {mom.VARIANT_FFMA: "ffma", mom.VARIANT_3XTF32_FORCE: "tc", mom.VARIANT_3XTF32: "auto", mom.VARIANT_3XTF32_WARP: "warp",
+         mom.VARIANT_3XTF32_INLINE: "inline"}
 
 
 def both(eq, variant, **kw):
@@ -109,6 +110,29 @@ def test_config_property_heavy_small(n, variant):
 @pytest.mark.parametrize("n", [384, 776])
 def test_config_large_square_small(n, variant):
     both(wl.config_large_square(n=n), variant)
+
+
+INLINE_SHAPES = [
+    # (m, k, n, left property, right property, Add terms): the one-launch tcgen05 kernel that splits in shared memory
+    (128, 32, 64, G, G, 0), (100, 36, 100, G, G, 1), (900, 1200, 100, G, G, 0), (256, 2048, 64, G, G, 2),      # k split over a cluster
+    (64, 1024, 512, G, G, 0), (1024, 64, 512, G, G, 1), (1000, 260, 76, G, G, 0), (1, 4, 4, G, G, 0),
+    (520, 520, 520, L, G, 1), (520, 520, 136, U, G, 0), (300, 392, 392, G, L, 0), (300, 392, 392, G, U, 2),
+    (392, 392, 392, L, L, 1), (392, 392, 392, U, U, 0), (392, 392, 392, L, U, 0), (392, 392, 392, U, L, 1),
+    (1024, 1024, 1024, G, G, 0), (1536, 1152, 1280, G, G, 1),
+]
+
+
+@pytest.mark.parametrize("m,k,n,pa,pb,terms", INLINE_SHAPES)
+def test_inline_split_tensor_core_kernel(m, k, n, pa, pb, terms):
+    # every launch shape of the kernel: 64- and 128-column tiles, 1 to 8 k-slices per tile (cluster), ragged edges in
+    # m, n and k, triangular factors (structural k-ranges, masked triangular results), fused Add terms incl. Identity
+    dist = lambda p: "uniform" if p != G else "normal"
+    add = [Operand(m, n, G, "normal")] * min(terms, 1) + ([Operand(m, n, I)] if terms == 2 and m == n else
+                                                          [Operand(m, n, G, "normal")] if terms == 2 else [])
+    eq = Equation(f"inline_{m}x{k}x{n}_{pa}{pb}", 75, (Operand(m, k, pa, dist(pa), 1.0 / np.sqrt(k)), Operand(k, n, pb, dist(pb))), tuple(add))
+    x, plan, (chain, terms_h) = run_equation(eq, mom.VARIANT_3XTF32_INLINE)
+    assert plan.step(0).uses_tensor_cores == 3 and plan.last_launch_count() == 1
+    check_against_oracle(eq, x, plan, chain, terms_h)
 
 
 @pytest.mark.parametrize("case", ["LG", "GU_plus_C", "chain"])

@@ -12,7 +12,7 @@ from gpu_util import run_sum_equation, check_sum_against_oracle, stratified_rows
 
 pytestmark = pytest.mark.gpu
 
-VARIANTS = [mom.VARIANT_3XTF32, mom.VARIANT_FFMA, mom.VARIANT_3XTF32_FORCE, mom.VARIANT_3XTF32_WARP]
+VARIANTS = [mom.VARIANT_3XTF32, mom.VARIANT_FFMA, mom.VARIANT_3XTF32_FORCE, mom.VARIANT_3XTF32_WARP, mom.VARIANT_3XTF32_INLINE]
 
 
 def sum_eq(name, chains, transposed=None, names=None, seed=11):

@@ -13,8 +13,8 @@ from gpu_util import run_equation, check_against_oracle, run_sum_equation, check
 
 pytestmark = pytest.mark.gpu
 
-VARIANTS = [mom.VARIANT_3XTF32, mom.VARIANT_FFMA, mom.VARIANT_3XTF32_FORCE, mom.VARIANT_3XTF32_WARP]
-VNAME = {mom.VARIANT_FFMA: "ffma", mom.VARIANT_3XTF32_FORCE: "tc", mom.VARIANT_3XTF32: "auto", mom.VARIANT_3XTF32_WARP: "warp"}
+VARIANTS = [mom.VARIANT_3XTF32, mom.VARIANT_FFMA, mom.VARIANT_3XTF32_FORCE, mom.VARIANT_3XTF32_WARP, mom.VARIANT_3XTF32_INLINE]
+VNAME = {mom.VARIANT_FFMA: "ffma", mom.VARIANT_3XTF32_FORCE: "tc", mom.VARIANT_3XTF32: "auto", mom.VARIANT_3XTF32_WARP: "warp", mom.VARIANT_3XTF32_INLINE: "inline"}
 
 
 def both(eq, variant, **kw):

@@ -141,7 +141,7 @@ def test_more_errors():
     with pytest.raises(mom.MomError) as e:
         mom.mom_matrix_desc(3, 4, mom.LOWER_TRI)
     assert e.value.status == mom.ERR_PROPERTY
-    big = 1 << 31
+    big = (1 << 31) - 2048                                    # the largest dimensions the library takes: the count overflows
     with pytest.raises(mom.MomError) as e:
         mom.mom_equation_plan([(big, big, 0), (big, big, 0)], [])
     assert e.value.status == mom.ERR_OVERFLOW
@@ -150,7 +150,7 @@ def test_more_errors():
         mom.mom_equation_plan_sum([[(big, big, 0), (big, big, 0)]], [[False, True]], [[0, 0]])
     assert e.value.status == mom.ERR_OVERFLOW
     with pytest.raises(mom.MomError) as e:
-        mom.mom_equation_plan([(4, 4, 0)], [], 4)               # unknown variant
+        mom.mom_equation_plan([(4, 4, 0)], [], 5)               # unknown variant
     assert e.value.status == mom.ERR_INVALID_ARG
 
 
@@ -164,15 +164,16 @@ def test_workspace_covers_intermediates_and_planes():
     p = mom.mom_equation_plan(eq.descs(), (), mom.VARIANT_3XTF32)
     assert all(s.uses_tensor_cores == 1 for s in p.steps())
     assert p.workspace_bytes() >= 2 * n * n * 4 + 4 * n * n * 4
-    # shapes TMA cannot address fall back to FFMA when the tcgen05 kernel is forced; in the default variant they
-    # and all small products run on the warp-level kernel (one launch per product)
+    # shapes TMA cannot address fall back to FFMA when the tcgen05 kernel is forced; in the default variant they and tiny
+    # products run on the warp-level kernel, small and mid-size ones on the tcgen05 kernel that splits in shared memory
+    # (one launch per product either way)
     p = mom.mom_equation_plan([(5, 5, 1), (5, 5, 1)], (), mom.VARIANT_3XTF32_FORCE)
     assert p.step(0).uses_tensor_cores == 0
     p = mom.mom_equation_plan(wl.config_tiny().descs(), (), mom.VARIANT_3XTF32)
     assert all(s.uses_tensor_cores == 2 for s in p.steps())
     p = mom.mom_equation_plan(wl.config_paper_chain().descs(), (), mom.VARIANT_3XTF32)
     up = lambda b: (b + 255) // 256 * 256          # two f32 intermediates, no operand planes
-    assert all(s.uses_tensor_cores == 2 for s in p.steps()) and p.workspace_bytes() == up(900 * 100 * 4) + up(1100 * 100 * 4)
+    assert all(s.uses_tensor_cores == 3 for s in p.steps()) and p.workspace_bytes() == up(900 * 100 * 4) + up(1100 * 100 * 4)
     p = mom.mom_equation_plan([(1001, 1001, 0), (1001, 1001, 0)], (), mom.VARIANT_3XTF32)
     assert p.step(0).uses_tensor_cores == 2
     p = mom.mom_equation_plan(wl.config_property_heavy().descs(), (), mom.VARIANT_3XTF32_WARP)
@@ -417,11 +418,11 @@ def test_size_limits_of_the_library():
     with pytest.raises(mom.MomError) as e:
         mom.mom_equation_plan([D(8, big), D(big, 8)], [], mom.VARIANT_3XTF32)
     assert e.value.status == mom.ERR_LIMIT
-    # the tcgen05 kernel's tile table keeps a tile's first row in 24 bits: a taller (or wider) product goes to
-    # the warp-level kernel (default variant) or the FFMA kernel (forced variant), never to the tcgen05 kernel
+    # the plane-fed tcgen05 kernel's tile table keeps a tile's first row in 24 bits: a taller (or wider) product goes to
+    # the one-launch tcgen05 kernel, which has no table (default variant), or the FFMA kernel (forced variant)
     tall = 2 ** 24
     for m, n in ((tall, 64), (64, tall), (tall - 1024 + 4, 64)):
-        for variant, want in ((mom.VARIANT_3XTF32, 2), (mom.VARIANT_3XTF32_FORCE, 0)):
+        for variant, want in ((mom.VARIANT_3XTF32, 3), (mom.VARIANT_3XTF32_FORCE, 0)):
             plan = mom.mom_equation_plan([D(m, 64), D(64, n)], [], variant)
             assert plan.step(0).uses_tensor_cores == want
     plan = mom.mom_equation_plan([D(tall - 1024, 64), D(64, 64)], [], mom.VARIANT_3XTF32)
