@@ -26,9 +26,10 @@ constexpr int FF_BN = 128;
 
 constexpr size_t WS_ALIGN = 256;
 
-// Default variant: products with fewer multiplications than this run on the warp-level kernel (its fixed cost is the
-// smallest), larger ones up to the large-product threshold on the in-kernel-split tcgen05 kernel.
-constexpr double INLINE_MIN_WORK = 2097152.0;
+// Default variant: the window of multiplication counts in which the one-launch tcgen05 kernel (product_tc_inline.cu) is the
+// quickest of the three tensor-core kernels (measured on square products: 512^3 12.5 us against 14.9 us on the warp-level
+// kernel, 768^3 20.7 against 31.0 and 28.9 on the plane kernel, 1024^3 36.7 against 34.8 on the plane kernel).
+constexpr double INLINE_MIN_WORK = 1.0e8, INLINE_MAX_WORK = 8.0e8;
 
 // Largest rows / cols a descriptor may have: every kernel indexes rows, columns and k with 32-bit integers.
 constexpr int64_t MAX_DIMENSION = 2147483647 - 1024;

@@ -7,14 +7,15 @@
 //   warp 0      TMA producer: per k-block of 32 the raw f32 tile of A (128 rows x 32 k: already K-major, loaded under
 //               the 128-byte swizzle the MMA wants) and the raw tile of B (32 k-rows x BN columns, as BN / 32 swizzled
 //               boxes of 32 x 32);
-//   warps 2-5   transform: A is split where it lies (the hi half overwrites the raw tile, the lo half goes to a second
+//   warps 2-9   transform: A is split where it lies (the hi half overwrites the raw tile, the lo half goes to a second
 //               tile at the same offsets); B is split AND transposed into K-major hi / lo tiles (BN rows of 32 k): a lane
 //               reads four columns of its k-row with one 16-byte load -- the eight lanes of a load phase hit eight
 //               different swizzled chunks -- and writes each value into its column's row, where the 32 lanes of a
 //               warp fill one 128-byte row: no bank conflict on either side;
 //   warp 1      MMA issuer: 4 k-steps x 3 tcgen05.mma kind::tf32 (lo*hi, hi*lo, hi*hi; M128, N = BN) per k-block into one
 //               accumulator in tensor memory; tcgen05.commit frees the stage;
-//   warps 2-5   then the epilogue: tcgen05.ld, Add terms, structure mask, 16-byte stores.
+//   warps 2-9   then the epilogue: tcgen05.ld (two warps per quarter of the tile's rows, each half of the columns), Add terms,
+//               structure mask, 16-byte stores.
 // With few output tiles the contraction is split over the CTAs of a thread-block cluster (up to 8): each leaves its partial
 // tile in its own shared memory and CTA r finishes rows [r * 128 / s, (r + 1) * 128 / s) by adding the partial tiles through
 // distributed shared memory in k order (deterministic; no atomics, no scratch in global memory, no second launch).
@@ -39,7 +40,8 @@ namespace {
 
 namespace cg = cooperative_groups;
 
-constexpr int IBM = 128, IBK = 32, ITHREADS = 192, IMAX_SPLIT = 8;
+constexpr int IBM = 128, IBK = 32, ITHREADS = 320, IMAX_SPLIT = 8;    // warps: producer, MMA issuer, eight transform / epilogue warps
+constexpr int XFORM_WARPS = 8, XFORM_THREADS = 32 * XFORM_WARPS;
 
 template <int BN>
 struct InlineCfg {
@@ -64,12 +66,13 @@ struct InlineParams {
     int32_t *status;
 };
 
-// hi = a rounded to tf32 (nearest, ties away from zero, done on the bit pattern with full-rate integer instructions),
-// lo = (a - hi) rounded the same way: the halves the operand-split pass of the large-product kernel writes
+// hi = a rounded to tf32 (nearest, ties away from zero, done on the bit pattern with full-rate integer instructions);
+// lo = a - hi, exact in f32 and handed over as it is: whatever the tensor core does with the bits below tf32 changes lo
+// by at most 2^-11 of itself, i.e. 2^-22 of a, the size of the lo*lo term the scheme leaves out anyway
 __device__ __forceinline__ float tf32_round(float a) { return __uint_as_float((__float_as_uint(a) + 0x1000u) & 0xFFFFE000u); }
 __device__ __forceinline__ void split4(const float4 a, float4 &hi, float4 &lo) {
     hi.x = tf32_round(a.x); hi.y = tf32_round(a.y); hi.z = tf32_round(a.z); hi.w = tf32_round(a.w);
-    lo.x = tf32_round(a.x - hi.x); lo.y = tf32_round(a.y - hi.y); lo.z = tf32_round(a.z - hi.z); lo.w = tf32_round(a.w - hi.w);
+    lo.x = a.x - hi.x; lo.y = a.y - hi.y; lo.z = a.z - hi.z; lo.w = a.w - hi.w;
 }
 
 // K-major tile with 128-byte rows under the 128B swizzle: 8-row groups are 1024 bytes apart, a K = 8 step is 32 bytes
@@ -109,7 +112,7 @@ product_tc_inline_kernel(const __grid_constant__ CUtensorMap map_a, const __grid
 
     if (threadIdx.x == 0) {
         abort_word = 0;
-        for (int s = 0; s < S; ++s) { ptx::mbar_init(raw_full(s), 1); ptx::mbar_init(ready(s), 4); ptx::mbar_init(empty(s), 1); }
+        for (int s = 0; s < S; ++s) { ptx::mbar_init(raw_full(s), 1); ptx::mbar_init(ready(s), XFORM_WARPS); ptx::mbar_init(empty(s), 1); }
         ptx::mbar_init(acc_full, 1);
         ptx::mbar_init(drain, 1);
         ptx::fence_barrier_init();
@@ -177,8 +180,22 @@ product_tc_inline_kernel(const __grid_constant__ CUtensorMap map_a, const __grid
         }
         __syncwarp();
     } else {
-        // ------------------------------------------------------------------ transform (warps 2..5), then epilogue
+        // ------------------------------------------------------------------ transform (warps 2..9), then epilogue
         const int tid2 = threadIdx.x - 64, w2 = warp - 2;
+        // where this lane's values of B go: task t of the warp is (box j, group c) = columns 32 j + 4 c .. + 3 of k-row `lane`;
+        // value e of it lands in row n = 32 j + 4 c + e of the K-major tile, at k = lane (group lane / 4, word lane % 4)
+        constexpr int TASKS = BN / 4 / XFORM_WARPS;
+        uint32_t src_off[TASKS], dst_off[TASKS][4];
+#pragma unroll
+        for (int t = 0; t < TASKS; ++t) {
+            const int task = w2 + XFORM_WARPS * t, j = task >> 3, c = task & 7;
+            src_off[t] = j * 4096 + lane * 128 + ((c ^ (lane & 7)) << 4);
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const int n = 32 * j + 4 * c + e;
+                dst_off[t][e] = n * 128 + ((((uint32_t)lane >> 2) ^ (n & 7)) << 4) + ((lane & 3) << 2);
+            }
+        }
         bool ok = true;
         for (int i = 0; i < nk && ok; ++i) {
             const int s = i % S;
@@ -187,38 +204,37 @@ product_tc_inline_kernel(const __grid_constant__ CUtensorMap map_a, const __grid
             if (!ok) break;
             uint8_t *const st = base_ptr + s * Cfg::STAGE_BYTES;
             // A: 128 rows x 8 groups of 16 bytes, split where they lie (the swizzle is a permutation of the groups: offsets stay)
+            float4 av[1024 / XFORM_THREADS];
 #pragma unroll
-            for (int u = 0; u < 8; ++u) {
-                float4 *p = reinterpret_cast<float4 *>(st) + tid2 + 128 * u;
+            for (int u = 0; u < 1024 / XFORM_THREADS; ++u) av[u] = *(reinterpret_cast<const float4 *>(st) + tid2 + XFORM_THREADS * u);
+            // B: box j holds k-rows 0..31 x columns 32 j .. 32 j + 31, group c of row k at group c ^ (k & 7).  Lane = k-row.
+            uint8_t *const braw = st + 2 * Cfg::A_BYTES, *const bhi = braw + Cfg::B_RAW_BYTES, *const blo = bhi + Cfg::B_PLANE_BYTES;
+            float4 bv[TASKS];
+#pragma unroll
+            for (int t = 0; t < TASKS; ++t) bv[t] = *reinterpret_cast<const float4 *>(braw + src_off[t]);
+#pragma unroll
+            for (int u = 0; u < 1024 / XFORM_THREADS; ++u) {
+                float4 *p = reinterpret_cast<float4 *>(st) + tid2 + XFORM_THREADS * u;
                 float4 hi, lo;
-                split4(*p, hi, lo);
+                split4(av[u], hi, lo);
                 *p = hi;
                 *(p + Cfg::A_BYTES / 16) = lo;
             }
-            // B: box j holds k-rows 0..31 x columns 32 j .. 32 j + 31, group c of row k at group c ^ (k & 7).  Lane = k-row.
-            uint8_t *const braw = st + 2 * Cfg::A_BYTES, *const bhi = braw + Cfg::B_RAW_BYTES, *const blo = bhi + Cfg::B_PLANE_BYTES;
 #pragma unroll
-            for (int task = w2; task < BN / 4; task += 4) {
-                const int j = task >> 3, c = task & 7;
-                const float4 v = *reinterpret_cast<const float4 *>(braw + j * 4096 + lane * 128 + ((c ^ (lane & 7)) << 4));
+            for (int t = 0; t < TASKS; ++t) {
                 float4 hi, lo;
-                split4(v, hi, lo);
-                const int n0 = 32 * j + 4 * c;                           // column of v.x inside the tile = row of the K-major tile
-                const uint32_t in_row = (uint32_t)(lane & 3) << 2;       // k = lane: group lane / 4, word lane % 4
-                const uint32_t group = (uint32_t)lane >> 2;
-                const uint32_t o0 = (n0 + 0) * 128 + ((group ^ ((n0 + 0) & 7)) << 4) + in_row, o1 = (n0 + 1) * 128 + ((group ^ ((n0 + 1) & 7)) << 4) + in_row;
-                const uint32_t o2 = (n0 + 2) * 128 + ((group ^ ((n0 + 2) & 7)) << 4) + in_row, o3 = (n0 + 3) * 128 + ((group ^ ((n0 + 3) & 7)) << 4) + in_row;
-                *reinterpret_cast<float *>(bhi + o0) = hi.x; *reinterpret_cast<float *>(blo + o0) = lo.x;
-                *reinterpret_cast<float *>(bhi + o1) = hi.y; *reinterpret_cast<float *>(blo + o1) = lo.y;
-                *reinterpret_cast<float *>(bhi + o2) = hi.z; *reinterpret_cast<float *>(blo + o2) = lo.z;
-                *reinterpret_cast<float *>(bhi + o3) = hi.w; *reinterpret_cast<float *>(blo + o3) = lo.w;
+                split4(bv[t], hi, lo);
+                *reinterpret_cast<float *>(bhi + dst_off[t][0]) = hi.x; *reinterpret_cast<float *>(blo + dst_off[t][0]) = lo.x;
+                *reinterpret_cast<float *>(bhi + dst_off[t][1]) = hi.y; *reinterpret_cast<float *>(blo + dst_off[t][1]) = lo.y;
+                *reinterpret_cast<float *>(bhi + dst_off[t][2]) = hi.z; *reinterpret_cast<float *>(blo + dst_off[t][2]) = lo.z;
+                *reinterpret_cast<float *>(bhi + dst_off[t][3]) = hi.w; *reinterpret_cast<float *>(blo + dst_off[t][3]) = lo.w;
             }
             ptx::fence_proxy_async_smem();                   // the MMA reads these tiles through the asynchronous proxy
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(ready(s));
         }
-        // ---- epilogue: this warp reads TMEM lanes 32 q .. 32 q + 31 = rows of the tile
-        const int q = warp & 3, row = q * 32 + lane, r = r0 + row;
+        // ---- epilogue: this warp reads TMEM lanes 32 q .. 32 q + 31 = rows of the tile; the two warps of a quarter share the columns
+        const int q = warp & 3, row = q * 32 + lane, r = r0 + row, half = w2 >> 2;
         if (nk > 0 && ok) {
             if (lane == 0) ok = wait_barrier(acc_full, 0, abort_flag, prm.status, (14 << 24) | (tile & 0xFFFF));
             ok = __shfl_sync(0xffffffffu, ok, 0);
@@ -228,7 +244,7 @@ product_tc_inline_kernel(const __grid_constant__ CUtensorMap map_a, const __grid
         const bool vec = (reinterpret_cast<uintptr_t>(prm.C) & 15) == 0 && (prm.n & 3) == 0;
         float *const P = reinterpret_cast<float *>(base_ptr);
 #pragma unroll 1
-        for (int c = 0; c < BN / 32; ++c) {
+        for (int c = half; c < BN / 32; c += 2) {
             const int col0 = c0 + 32 * c;
             float v[32];
             if (acc_ok) {

@@ -164,16 +164,15 @@ def test_workspace_covers_intermediates_and_planes():
     p = mom.mom_equation_plan(eq.descs(), (), mom.VARIANT_3XTF32)
     assert all(s.uses_tensor_cores == 1 for s in p.steps())
     assert p.workspace_bytes() >= 2 * n * n * 4 + 4 * n * n * 4
-    # shapes TMA cannot address fall back to FFMA when the tcgen05 kernel is forced; in the default variant they and tiny
-    # products run on the warp-level kernel, small and mid-size ones on the tcgen05 kernel that splits in shared memory
-    # (one launch per product either way)
+    # shapes TMA cannot address fall back to FFMA when the tcgen05 kernel is forced; in the default variant they, small
+    # products and products with a skinny result run on the warp-level kernel (one launch per product)
     p = mom.mom_equation_plan([(5, 5, 1), (5, 5, 1)], (), mom.VARIANT_3XTF32_FORCE)
     assert p.step(0).uses_tensor_cores == 0
     p = mom.mom_equation_plan(wl.config_tiny().descs(), (), mom.VARIANT_3XTF32)
     assert all(s.uses_tensor_cores == 2 for s in p.steps())
     p = mom.mom_equation_plan(wl.config_paper_chain().descs(), (), mom.VARIANT_3XTF32)
     up = lambda b: (b + 255) // 256 * 256          # two f32 intermediates, no operand planes
-    assert all(s.uses_tensor_cores == 3 for s in p.steps()) and p.workspace_bytes() == up(900 * 100 * 4) + up(1100 * 100 * 4)
+    assert all(s.uses_tensor_cores == 2 for s in p.steps()) and p.workspace_bytes() == up(900 * 100 * 4) + up(1100 * 100 * 4)
     p = mom.mom_equation_plan([(1001, 1001, 0), (1001, 1001, 0)], (), mom.VARIANT_3XTF32)
     assert p.step(0).uses_tensor_cores == 2
     p = mom.mom_equation_plan(wl.config_property_heavy().descs(), (), mom.VARIANT_3XTF32_WARP)
@@ -419,10 +418,10 @@ def test_size_limits_of_the_library():
         mom.mom_equation_plan([D(8, big), D(big, 8)], [], mom.VARIANT_3XTF32)
     assert e.value.status == mom.ERR_LIMIT
     # the plane-fed tcgen05 kernel's tile table keeps a tile's first row in 24 bits: a taller (or wider) product goes to
-    # the one-launch tcgen05 kernel, which has no table (default variant), or the FFMA kernel (forced variant)
+    # the warp-level kernel (default variant) or the FFMA kernel (forced variant)
     tall = 2 ** 24
     for m, n in ((tall, 64), (64, tall), (tall - 1024 + 4, 64)):
-        for variant, want in ((mom.VARIANT_3XTF32, 3), (mom.VARIANT_3XTF32_FORCE, 0)):
+        for variant, want in ((mom.VARIANT_3XTF32, 2), (mom.VARIANT_3XTF32_FORCE, 0)):
             plan = mom.mom_equation_plan([D(m, 64), D(64, n)], [], variant)
             assert plan.step(0).uses_tensor_cores == want
     plan = mom.mom_equation_plan([D(tall - 1024, 64), D(64, 64)], [], mom.VARIANT_3XTF32)
@@ -492,3 +491,16 @@ def test_storage_changes_neither_the_plan_nor_its_costs():
     assert packed.result_elements() == mom.mom_packed_elements(n, wl.LOWER_TRI) == n * (n + 4) // 2
     assert packed.workspace_bytes(1) >= dense.workspace_bytes(1) + 3 * n * n * 4       # two dense copies and a dense X
     assert packed.host_staging_bytes(1) < dense.host_staging_bytes(1) + 3 * n * n * 4
+
+
+def test_kernel_choice_of_the_default_variant():
+    # three tensor-core kernels by size and shape: warp-level (2), one-launch tcgen05 with the split in shared memory (3),
+    # plane-fed tcgen05 (1)
+    G = wl.GENERAL
+    kind = lambda m, k, n, t=(False, False): mom.mom_equation_plan_transposed([(k, m, G) if t[0] else (m, k, G), (n, k, G) if t[1] else (k, n, G)], t, (), None,
+                                                                          mom.VARIANT_3XTF32).step(0).uses_tensor_cores
+    assert [kind(n, n, n) for n in (256, 384, 512, 640, 768, 896, 1024, 2048)] == [2, 2, 3, 3, 3, 3, 1, 1]
+    assert kind(900, 1200, 100) == 2                       # a skinny result: too few tiles for the one-launch kernel
+    assert kind(512, 512, 510) == 2                        # rows TMA cannot address
+    assert kind(640, 640, 640, (True, False)) == 2 and kind(640, 640, 640, (False, True)) == 2     # transposed operands
+    assert kind(1024, 1024, 1024, (True, False)) == 1      # the plane kernel reads transposed operands through its split pass
