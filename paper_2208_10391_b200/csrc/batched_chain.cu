@@ -98,8 +98,13 @@ batched_chain_kernel(const BatchedChainPlan bp) {
             for (int c = 0; c < 4; ++c)
                 if ((mask >> c) & 1u) {
                     const int col = 16 * c + 4 * t;
-                    buf[q][c][0] = col >= p0.first && col < p0.end ? load_once_f4(row0 + col) : make_float4(0.f, 0.f, 0.f, 0.f);
-                    buf[q][c][1] = col >= p1.first && col < p1.end ? load_once_f4(row1 + col) : make_float4(0.f, 0.f, 0.f, 0.f);
+                    if (c != rb) {                           // a block off the diagonal is stored in full
+                        buf[q][c][0] = load_once_f4(row0 + col);
+                        buf[q][c][1] = load_once_f4(row1 + col);
+                    } else {
+                        buf[q][c][0] = col >= p0.first && col < p0.end ? load_once_f4(row0 + col) : make_float4(0.f, 0.f, 0.f, 0.f);
+                        buf[q][c][1] = col >= p1.first && col < p1.end ? load_once_f4(row1 + col) : make_float4(0.f, 0.f, 0.f, 0.f);
+                    }
                 }
             return;
         }
