@@ -3,11 +3,48 @@
 #pragma once
 
 #include <cstdint>
+#include <utility>
 #include <cuda_runtime.h>
 
 #include "mom.h"
 
 namespace mom {
+
+// Programmatic dependent launch: a kernel that is launched with the programmatic-stream-serialization attribute may start
+// while its predecessor in the stream is still running; it must not touch global memory before grid_dependency_wait(), which
+// returns once the predecessor has completed and its writes are visible.  Such a kernel's lifetime overlaps its predecessors'
+// writes, so it must not read anything they may have produced through the non-coherent path (ld.global.nc / __ldg promises data
+// that is read-only for the kernel's whole lifetime): operands, Add terms and partial sums are read with ld.global.cg (__ldcg).  allow_dependents() lets the NEXT kernel of the stream
+// start its own prologue (it becomes resident as resources free up and waits at its grid_dependency_wait()).  Both are no-ops
+// in a kernel launched the ordinary way.
+__device__ __forceinline__ void allow_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+// Launch with the attribute that allows the overlap described above (plus, optionally, a cluster dimension).
+template <typename... KernelArgs, typename... Args>
+inline cudaError_t launch_dependent(void (*kernel)(KernelArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, unsigned cluster,
+                                    Args &&...args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[2];
+    int n = 0;
+    attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[n].val.programmaticStreamSerializationAllowed = 1;
+    ++n;
+    if (cluster > 1) {
+        attr[n].id = cudaLaunchAttributeClusterDimension;
+        attr[n].val.clusterDim.x = cluster;
+        attr[n].val.clusterDim.y = 1;
+        attr[n].val.clusterDim.z = 1;
+        ++n;
+    }
+    cfg.attrs = attr;
+    cfg.numAttrs = n;
+    return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+}
 
 constexpr int MAX_FUSED_ADD = 8;    // Add terms fused into one launch; more are added by follow-up passes
 
@@ -54,8 +91,7 @@ __device__ __forceinline__ float finish_entry(float acc, const AddTerms &add, lo
             const float *p = add.ptr[t];
             const long long at = (add.transposed >> t) & 1u ? (long long)c * add.rows + r : (long long)r * ld + c;
             if (!p) v += r == c ? 1.0f : 0.0f;
-            else if ((add.aliases_out >> t) & 1u) v += __ldcg(p + batch * add.stride[t] + at);
-            else v += __ldg(p + batch * add.stride[t] + at);
+            else v += __ldcg(p + batch * add.stride[t] + at);
         }
     }
     return in_structure(out_prop, r, c) ? v : 0.0f;
@@ -71,7 +107,7 @@ __device__ __forceinline__ float finish_entry_compact(float acc, const AddTerms 
         const float *p = add.ptr[t];
         if (!p) { v += r == c ? 1.0f : 0.0f; continue; }
         p += batch * add.stride[t] + ((add.transposed >> t) & 1u ? (long long)c * add.rows + r : (long long)r * ld + c);
-        v += (add.aliases_out >> t) & 1u ? __ldcg(p) : __ldg(p);
+        v += __ldcg(p);
     }
     return in_structure(out_prop, r, c) ? v : 0.0f;
 }
@@ -95,14 +131,14 @@ __device__ __forceinline__ void finish_row4(float (&v)[4], const AddTerms &add, 
         const bool tr = (add.transposed >> t) & 1u, alias = (add.aliases_out >> t) & 1u;
         if (!tr && vec && c + 3 < n && (reinterpret_cast<uintptr_t>(p) & 15) == 0) {
             const float4 *q = reinterpret_cast<const float4 *>(p + (long long)r * ld + c);
-            const float4 x = alias ? __ldcg(q) : __ldg(q);
+            const float4 x = __ldcg(q);
             v[0] += x.x; v[1] += x.y; v[2] += x.z; v[3] += x.w;
         } else {
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
                 if (c + j >= n) continue;
                 const long long at = tr ? (long long)(c + j) * add.rows + r : (long long)r * ld + c + j;
-                v[j] += alias ? __ldcg(p + at) : __ldg(p + at);
+                v[j] += __ldcg(p + at);
             }
         }
     }

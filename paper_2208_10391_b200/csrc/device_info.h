@@ -16,6 +16,7 @@ struct DeviceInfo {
     bool tc_attr = false;            // dynamic shared-memory limit raised for the tensor-core kernels on this device
     bool pair_attr = false;
     bool inline64_attr = false, inline128_attr = false;
+    int inline_clusters[2][4] = {};  // co-resident clusters of the one-launch tcgen05 kernel, [128-column tiles][log2 cluster size]; 0: not asked, -1: unknown
     int fused_max_smem[2] = {0, 0};  // largest dynamic shared-memory size set for the fused small-equation kernels
     int batched_max_smem = 0;
 };
@@ -35,6 +36,15 @@ cudaError_t raise_smem_limit_once(Kernel kernel, int bytes, bool DeviceInfo::*do
     if (info->*done) return cudaSuccess;
     const cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
     if (e == cudaSuccess) info->*done = true;
+    return e;
+}
+
+// The same for a caller that already holds device_info_mutex().
+template <typename Kernel>
+cudaError_t raise_smem_limit_locked(Kernel kernel, int bytes, bool *done) {
+    if (*done) return cudaSuccess;
+    const cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    if (e == cudaSuccess) *done = true;
     return e;
 }
 

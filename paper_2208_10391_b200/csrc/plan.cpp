@@ -564,12 +564,11 @@ static mom_status_t plan_sums(const std::vector<mom_matrix_desc_t> &slots, const
             const bool inline_ok = st.pub.kind != MOM_KIND_GRAM &&
                                    mom::product_tc_inline_takes(m, n, k, st.pub.lhs_transposed, st.pub.rhs_transposed,
                                                                 mom::kernel_property(st.pub.lhs_property), mom::kernel_property(st.pub.rhs_property));
-            // ... and it pays between the two: from about 500^3 on its tensor-core mainloop beats the warp-level kernel's, up to about
-            // 900^3 its single launch beats the plane kernel's two or three; with few output tiles (a skinny result) it would
-            // have to split the contraction over a cluster and the warp-level kernel is quicker (measured, see the kernel's file)
+            // ... and it pays between the two (measured, see the kernel's file): from about 450^3 on it beats the warp-level kernel, up to
+            // about 1000^3 its single launch beats the plane kernel's two or three; a result of fewer than four 128 x 128 tiles would leave
+            // each CTA a long contraction even when split over a cluster, and the warp-level kernel is quicker there
             const double work = (double)m * (double)n * (double)k;
-            const int64_t inline_tiles = ((m + 127) / 128) * ((n + 63) / 64);
-            const bool inline_pays = work >= mom::INLINE_MIN_WORK && work < mom::INLINE_MAX_WORK && inline_tiles >= 32;
+            const bool inline_pays = work >= mom::INLINE_MIN_WORK && work < mom::INLINE_MAX_WORK && (double)m * (double)n >= mom::INLINE_MIN_OUTPUT;
             if (st.pub.kind == MOM_KIND_SCALE) st.pub.uses_tensor_cores = 0;       // a Diagonal operand: one scaling pass, bound by HBM
             else if (variant == MOM_VARIANT_3XTF32) st.pub.uses_tensor_cores = inline_ok && inline_pays ? 3 : addressable && large ? 1 : 2;
             else if (variant == MOM_VARIANT_3XTF32_FORCE) st.pub.uses_tensor_cores = addressable ? 1 : 0;

@@ -109,7 +109,7 @@ __device__ __forceinline__ void epilogue_chunk(const TcParams &prm, const CUtens
             if (row_ok) {
 #pragma unroll
                 for (int j = 0; j < 32; ++j)
-                    if (col0 + j < prm.n) v[j] += __ldg(p + (long long)(col0 + j) * prm.m + r);
+                    if (col0 + j < prm.n) v[j] += __ldcg(p + (long long)(col0 + j) * prm.m + r);
             }
         } else if (p) {
             if (row_ok) {
@@ -117,7 +117,7 @@ __device__ __forceinline__ void epilogue_chunk(const TcParams &prm, const CUtens
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {
                     if (col0 + 4 * j < prm.n) {
-                        const float4 x = ((prm.add.aliases_out >> a) & 1u) ? __ldcg(src + j) : __ldg(src + j);
+                        const float4 x = __ldcg(src + j);
                         v[4 * j] += x.x; v[4 * j + 1] += x.y; v[4 * j + 2] += x.z; v[4 * j + 3] += x.w;
                     }
                 }
@@ -580,18 +580,18 @@ __device__ __forceinline__ void split_piece(const float *__restrict__ src, float
                 float4 a;
                 if (packed) {
                     const PackedRow row = packed_row(prop == MOM_LOWER_TRI, rows, r);
-                    a = c >= row.first && c < row.end ? __ldg(reinterpret_cast<const float4 *>(src + row.offset + (c - row.first)))
+                    a = c >= row.first && c < row.end ? __ldcg(reinterpret_cast<const float4 *>(src + row.offset + (c - row.first)))
                                                       : make_float4(0.f, 0.f, 0.f, 0.f);
                 } else {
-                    a = __ldg(reinterpret_cast<const float4 *>(src + off));
+                    a = __ldcg(reinterpret_cast<const float4 *>(src + off));
                 }
                 if (sc.d) {
                     if (sc.by_row) {
-                        const float f = __ldg(sc.d + r * sc.step);
+                        const float f = __ldcg(sc.d + r * sc.step);
                         a.x *= f; a.y *= f; a.z *= f; a.w *= f;
                     } else {
-                        a.x *= __ldg(sc.d + c * sc.step); a.y *= __ldg(sc.d + (c + 1) * sc.step);
-                        a.z *= __ldg(sc.d + (c + 2) * sc.step); a.w *= __ldg(sc.d + (c + 3) * sc.step);
+                        a.x *= __ldcg(sc.d + c * sc.step); a.y *= __ldcg(sc.d + (c + 1) * sc.step);
+                        a.z *= __ldcg(sc.d + (c + 2) * sc.step); a.w *= __ldcg(sc.d + (c + 3) * sc.step);
                     }
                 }
                 float4 h, l;
@@ -611,12 +611,12 @@ __device__ __forceinline__ void split_piece(const float *__restrict__ src, float
             if (pr + r < rows && pc + c < cols) {
                 if (packed) {
                     const PackedRow row = packed_row(prop == MOM_LOWER_TRI, rows, pr + r);
-                    if (pc + c >= row.first && pc + c < row.end) v = __ldg(src + row.offset + (pc + c - row.first));
+                    if (pc + c >= row.first && pc + c < row.end) v = __ldcg(src + row.offset + (pc + c - row.first));
                 } else {
-                    v = __ldg(src + (size_t)(pr + r) * cols + pc + c);
+                    v = __ldcg(src + (size_t)(pr + r) * cols + pc + c);
                 }
             }
-            if (sc.d && pr + r < rows && pc + c < cols) v *= __ldg(sc.d + (sc.by_row ? pr + r : pc + c) * sc.step);
+            if (sc.d && pr + r < rows && pc + c < cols) v *= __ldcg(sc.d + (sc.by_row ? pr + r : pc + c) * sc.step);
             tile[r][c] = v;
         }
         __syncthreads();
@@ -674,7 +674,7 @@ splitk_reduce_kernel(const float *__restrict__ partial, int slices, int slice_ro
         const int r = (int)(e / vec_per_row), c = (int)(e % vec_per_row) << 2;
         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
         for (int s = 0; s < slices; ++s) {
-            const float4 v = __ldg(reinterpret_cast<const float4 *>(partial + ((size_t)s * slice_rows + r) * n + c));
+            const float4 v = __ldcg(reinterpret_cast<const float4 *>(partial + ((size_t)s * slice_rows + r) * n + c));
             acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
         }
         float4 o;

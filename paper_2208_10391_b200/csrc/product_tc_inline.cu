@@ -87,6 +87,7 @@ product_tc_inline_kernel(const __grid_constant__ CUtensorMap map_a, const __grid
     constexpr int S = Cfg::STAGES;
     extern __shared__ uint8_t smem_raw[];
     __shared__ int abort_word;
+    allow_dependents();
     const uint32_t base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t *const base_ptr = smem_raw + (base - ptx::smem_u32(smem_raw));
     const uint32_t bars = base + S * Cfg::STAGE_BYTES;
@@ -126,6 +127,8 @@ product_tc_inline_kernel(const __grid_constant__ CUtensorMap map_a, const __grid
     ptx::tc_fence_after_sync();
     uint32_t tmem_base;
     asm volatile("ld.shared.u32 %0, [%1];" : "=r"(tmem_base) : "r"(tmem_slot));
+    grid_dependency_wait();                      // barriers and tensor memory are set up; now the previous launch's results may be read
+    asm volatile("fence.proxy.async;" ::: "memory");   // ... by TMA, i.e. through the asynchronous proxy
 
     bool acc_ok = nk > 0;                        // the accumulator holds this CTA's partial sums (epilogue warps)
     if (warp == 0) {
@@ -327,15 +330,53 @@ cudaError_t launch_product_tc_inline(const ProductArgs &a, int32_t *status, cuda
     const int sm_count = current_sm_count();
     if (sm_count < 1) return cudaErrorInvalidDevice;
     const int tiles_m = (a.m + IBM - 1) / IBM;
-    // narrow tiles while 128-column ones would leave SMs without a tile
-    const bool narrow = a.n <= 64 || (long long)tiles_m * ((a.n + 127) / 128) < sm_count;
-    const int bn = narrow ? 64 : 128;
+    const int kblocks = (a.k + IBK - 1) / IBK;
+    // Tile width and k-slices per tile: the pair with the shortest critical path, counted in k-blocks of one CTA times what a k-block
+    // costs at that width (measured: about 0.9 us at 64 columns, 1.3 us at 128), over the waves the grid needs.  A cluster of s CTAs
+    // must sit in one GPC and every CTA takes a whole SM here, so far fewer than SMs / s clusters run at once: ask the runtime.
+    int bn = 64, split = 1;
+    double best = 1e300;
+    for (int width : {64, 128}) {
+        const long long tiles = (long long)tiles_m * ((a.n + width - 1) / width);
+        if (tiles * IMAX_SPLIT > (1ll << 30)) return cudaErrorNotSupported;
+        for (int s = 1; s <= IMAX_SPLIT; s *= 2) {
+            if (s > 1 && a.k / s < 2 * IBK) break;                           // every slice keeps two k-blocks
+            int fit = sm_count / s;                                            // clusters that can run at once
+            {
+                std::lock_guard<std::mutex> lock(device_info_mutex());
+                DeviceInfo *info = current_device_info();
+                if (!info) return cudaErrorInvalidDevice;
+                int &known = info->inline_clusters[width == 128][s == 1 ? 0 : s == 2 ? 1 : s == 4 ? 2 : 3];
+                if (known == 0) {
+                    known = -1;
+                    cudaLaunchConfig_t probe = {};
+                    probe.gridDim = dim3((unsigned)(s * sm_count));
+                    probe.blockDim = dim3(ITHREADS);
+                    probe.dynamicSmemBytes = width == 128 ? InlineCfg<128>::SMEM_BYTES : InlineCfg<64>::SMEM_BYTES;
+                    cudaLaunchAttribute at[1];
+                    at[0].id = cudaLaunchAttributeClusterDimension;
+                    at[0].val.clusterDim.x = (unsigned)s; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+                    probe.attrs = at;
+                    probe.numAttrs = 1;
+                    int n = 0;
+                    cudaError_t e = width == 128 ? raise_smem_limit_locked(product_tc_inline_kernel<128>, InlineCfg<128>::SMEM_BYTES, &info->inline128_attr)
+                                                 : raise_smem_limit_locked(product_tc_inline_kernel<64>, InlineCfg<64>::SMEM_BYTES, &info->inline64_attr);
+                    if (e == cudaSuccess)
+                        e = width == 128 ? cudaOccupancyMaxActiveClusters(&n, product_tc_inline_kernel<128>, &probe)
+                                         : cudaOccupancyMaxActiveClusters(&n, product_tc_inline_kernel<64>, &probe);
+                    if (e == cudaSuccess && n > 0) known = n;
+                    else cudaGetLastError();
+                }
+                if (known > 0) fit = known;
+            }
+            if (fit < 1) continue;
+            const long long waves = (tiles + fit - 1) / fit;
+            const double cost = (double)waves * ((kblocks + s - 1) / s) * (width == 128 ? 1.3 : 0.9) + (s > 1 ? 1.5 : 0.0);
+            if (cost < best) { best = cost; bn = width; split = s; }
+        }
+    }
     const int tiles_n = (a.n + bn - 1) / bn;
     const long long tiles = (long long)tiles_m * tiles_n;
-    if (tiles * IMAX_SPLIT > (1ll << 30)) return cudaErrorNotSupported;
-    // few tiles and a long contraction: split k over a cluster, as long as every slice keeps two k-blocks
-    int split = 1;
-    while (split < IMAX_SPLIT && tiles * split * 2 <= sm_count && a.k / (split * 2) >= 2 * IBK) split *= 2;
 
     CUtensorMap map_a, map_b;
     if (!tc_make_map(&map_a, a.A, a.m, a.k, IBM, IBK, CU_TENSOR_MAP_SWIZZLE_128B) ||
@@ -350,27 +391,11 @@ cudaError_t launch_product_tc_inline(const ProductArgs &a, int32_t *status, cuda
     prm.add = a.add;
     prm.status = status;
 
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)(tiles * split));
-    cfg.blockDim = dim3(ITHREADS);
-    cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = (unsigned)split;
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = split > 1 ? 1 : 0;
-    if (bn == 64) {
-        cudaError_t e = raise_smem_limit_once(product_tc_inline_kernel<64>, InlineCfg<64>::SMEM_BYTES, &DeviceInfo::inline64_attr);
-        if (e != cudaSuccess) return e;
-        cfg.dynamicSmemBytes = InlineCfg<64>::SMEM_BYTES;
-        return cudaLaunchKernelEx(&cfg, product_tc_inline_kernel<64>, map_a, map_b, prm);
-    }
-    cudaError_t e = raise_smem_limit_once(product_tc_inline_kernel<128>, InlineCfg<128>::SMEM_BYTES, &DeviceInfo::inline128_attr);
-    if (e != cudaSuccess) return e;
-    cfg.dynamicSmemBytes = InlineCfg<128>::SMEM_BYTES;
-    return cudaLaunchKernelEx(&cfg, product_tc_inline_kernel<128>, map_a, map_b, prm);
+    if (bn == 64)
+        return launch_dependent(product_tc_inline_kernel<64>, dim3((unsigned)(tiles * split)), dim3(ITHREADS), InlineCfg<64>::SMEM_BYTES, stream,
+                                (unsigned)split, map_a, map_b, prm);
+    return launch_dependent(product_tc_inline_kernel<128>, dim3((unsigned)(tiles * split)), dim3(ITHREADS), InlineCfg<128>::SMEM_BYTES, stream,
+                            (unsigned)split, map_a, map_b, prm);
 }
 
 }  // namespace mom

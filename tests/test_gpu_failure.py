@@ -63,3 +63,34 @@ def test_only_the_first_failure_is_kept_and_a_fresh_plan_can_run_the_self_test()
         plan.probe_wait_timeout(5000.0, 1, stream)                            # limits above one second are refused
     x, plan2, (chain, add) = run_equation(eq, mom.VARIANT_3XTF32)
     check_against_oracle(eq, x, plan2, chain, add)
+
+
+@pytest.mark.parametrize("name", ["five_general", "paper_chain", "square_640", "tri_chain"])
+def test_back_to_back_executions_give_the_same_bits(name):
+    # The small-product kernels are launched so that a product's prologue overlaps the previous product's tail (programmatic
+    # dependent launch): a product must still see everything its predecessors wrote.  300 executions enqueued back to back, each
+    # into its own output: all bit-identical, and the first one within the bound of the oracle.
+    eq = {"five_general": wl.config_five_general(), "paper_chain": wl.config_paper_chain(), "square_640": wl.config_square_product(640),
+          "tri_chain": wl.Equation("tri_chain", 77, (wl.Operand(520, 520, wl.LOWER_TRI), wl.Operand(520, 520, wl.GENERAL, "normal", 0.05),
+                                                     wl.Operand(520, 520, wl.UPPER_TRI), wl.Operand(520, 136, wl.GENERAL, "normal")),
+                                   (wl.Operand(520, 136, wl.GENERAL, "normal"),))}[name]
+    chain, add = wl.generate(eq)
+    plan = mom.mom_equation_plan(eq.descs(), eq.add_descs(), mom.VARIANT_3XTF32)
+    rd = plan.result_desc()
+    dchain = [None if a is None else torch.from_numpy(a).cuda() for a in chain]
+    dadd = [None if a is None else torch.from_numpy(a).cuda() for a in add]
+    reps = 300
+    outs = torch.full((reps, rd.rows, rd.cols), float("nan"), dtype=torch.float32, device="cuda")
+    wsb = plan.workspace_bytes(1)
+    ws = torch.full((max(wsb, 256),), 255, dtype=torch.uint8, device="cuda")
+    stream = torch.cuda.current_stream().cuda_stream
+    cp = [None if t is None else t.data_ptr() for t in dchain]
+    ap = [None if t is None else t.data_ptr() for t in dadd]
+    for i in range(reps):
+        plan.execute(cp, ap, outs[i].data_ptr(), ws.data_ptr() if wsb else None, wsb, stream)
+    torch.cuda.synchronize()
+    assert plan.device_status() == (0, 0)
+    x = outs.cpu().numpy()
+    check_against_oracle(eq, x[0], plan, chain, add)
+    same = (x.view(np.uint32) == x[0].view(np.uint32)).reshape(reps, -1).all(axis=1)
+    assert same.all(), f"executions {np.nonzero(~same)[0][:10].tolist()} differ from the first"

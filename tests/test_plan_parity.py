@@ -164,15 +164,15 @@ def test_workspace_covers_intermediates_and_planes():
     p = mom.mom_equation_plan(eq.descs(), (), mom.VARIANT_3XTF32)
     assert all(s.uses_tensor_cores == 1 for s in p.steps())
     assert p.workspace_bytes() >= 2 * n * n * 4 + 4 * n * n * 4
-    # shapes TMA cannot address fall back to FFMA when the tcgen05 kernel is forced; in the default variant they, small
-    # products and products with a skinny result run on the warp-level kernel (one launch per product)
+    # shapes TMA cannot address fall back to FFMA when the tcgen05 kernel is forced; in the default variant they and small
+    # products run on the warp-level kernel, the Section-4 chain's products on the one-launch tcgen05 kernel
     p = mom.mom_equation_plan([(5, 5, 1), (5, 5, 1)], (), mom.VARIANT_3XTF32_FORCE)
     assert p.step(0).uses_tensor_cores == 0
     p = mom.mom_equation_plan(wl.config_tiny().descs(), (), mom.VARIANT_3XTF32)
     assert all(s.uses_tensor_cores == 2 for s in p.steps())
     p = mom.mom_equation_plan(wl.config_paper_chain().descs(), (), mom.VARIANT_3XTF32)
     up = lambda b: (b + 255) // 256 * 256          # two f32 intermediates, no operand planes
-    assert all(s.uses_tensor_cores == 2 for s in p.steps()) and p.workspace_bytes() == up(900 * 100 * 4) + up(1100 * 100 * 4)
+    assert all(s.uses_tensor_cores == 3 for s in p.steps()) and p.workspace_bytes() == up(900 * 100 * 4) + up(1100 * 100 * 4)
     p = mom.mom_equation_plan([(1001, 1001, 0), (1001, 1001, 0)], (), mom.VARIANT_3XTF32)
     assert p.step(0).uses_tensor_cores == 2
     p = mom.mom_equation_plan(wl.config_property_heavy().descs(), (), mom.VARIANT_3XTF32_WARP)
@@ -499,8 +499,8 @@ def test_kernel_choice_of_the_default_variant():
     G = wl.GENERAL
     kind = lambda m, k, n, t=(False, False): mom.mom_equation_plan_transposed([(k, m, G) if t[0] else (m, k, G), (n, k, G) if t[1] else (k, n, G)], t, (), None,
                                                                           mom.VARIANT_3XTF32).step(0).uses_tensor_cores
-    assert [kind(n, n, n) for n in (256, 384, 512, 640, 768, 896, 1024, 2048)] == [2, 2, 3, 3, 3, 3, 1, 1]
-    assert kind(900, 1200, 100) == 2                       # a skinny result: too few tiles for the one-launch kernel
+    assert [kind(n, n, n) for n in (256, 384, 448, 512, 768, 1024, 1280, 2048)] == [2, 2, 3, 3, 3, 3, 1, 1]
+    assert kind(900, 1200, 100) == 3 and kind(256, 2048, 64) == 2 and kind(128, 4096, 128) == 2       # small work; a result of one tile
     assert kind(512, 512, 510) == 2                        # rows TMA cannot address
     assert kind(640, 640, 640, (True, False)) == 2 and kind(640, 640, 640, (False, True)) == 2     # transposed operands
     assert kind(1024, 1024, 1024, (True, False)) == 1      # the plane kernel reads transposed operands through its split pass
