@@ -54,7 +54,6 @@ product_mma_kernel(const ProductArgs a, const int split, const int tiles_n) {
     __shared__ __align__(16) float As[STAGES * A_STAGE];
     __shared__ __align__(16) float Bs[STAGES * B_STAGE];
 
-    allow_dependents();
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
     const int wm = warp >> 1, wn = warp & 1;                 // 4 x 2 warps, 16 x 16 outputs each
     const long long inst = blockIdx.z;
@@ -121,7 +120,6 @@ product_mma_kernel(const ProductArgs a, const int split, const int tiles_n) {
 #pragma unroll
         for (int q = 0; q < 4; ++q) main_acc[j][q] = small_acc[j][q] = 0.f;
 
-    grid_dependency_wait();                                  // the operands may be the previous launch's result
     for (int s = 0; s < STAGES - 1; ++s) {
         if (s < nk) load_stage(s, klo + (kb0 + s) * BK);
         cp_async_commit();
@@ -213,12 +211,9 @@ cudaError_t launch_product_mma(const ProductArgs &a, int batch, cudaStream_t str
     int split = 1;
     const long long resident = 4LL * sm_count;
     while (split < MAX_SPLIT && tiles * batch * split * 2 <= resident && a.k / (split * 2) >= 4 * BK) split *= 2;
-    // The overlap with the previous launch (see launch_dependent) only where both operands come in through cp.async: the scalar path
-    // for transposed or unaligned operands reads through the read-only cache, which a kernel that starts early must not do.
-    const bool a_fast = !a.transA && (a.k & 3) == 0 && (reinterpret_cast<uintptr_t>(a.A) & 15) == 0 && (a.strideA & 3) == 0;
-    const bool b_fast = !a.transB && (a.n & 3) == 0 && (reinterpret_cast<uintptr_t>(a.B) & 15) == 0 && (a.strideB & 3) == 0;
-    if (a_fast && b_fast)
-        return launch_dependent(product_mma_kernel, dim3((unsigned)(tiles * split), 1, (unsigned)batch), dim3(THREADS), 0, stream, (unsigned)split, a, split, tiles_n);
+    // An ordinary launch: with the programmatic-dependent-launch attribute (the prologue overlapping the previous launch's tail) the
+    // large cluster-split products of this kernel gained 2 us, but the small ones lost more (384^3: 10.3 -> 16.2 us; the five-matrix
+    // chain 34.9 -> 37.4 us): measured, not kept.
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(tiles * split), 1, (unsigned)batch);
     cfg.blockDim = dim3(THREADS);
