@@ -388,6 +388,14 @@ mom_status_t mom_plan_device_status(const mom_plan_t *plan, int32_t *code, int32
  * ALLOC, CUDA. */
 mom_status_t mom_probe_wait_timeout(const mom_plan_t *plan, double limit_ms, int32_t detail, mom_stream_t stream);
 
+/* Steps that run side by side.  Small products leave most of the GPU idle, so where the chosen tree has a product whose two factors
+ * are themselves trees of small products (the five-matrix chain ((0*(1*2))*(3*4)): (0*(1*2)) and (3*4)), the launcher runs the right
+ * subtree, steps [*begin, *end), on a second stream the plan owns while the left one runs on the caller's stream; step *join waits
+ * for both.  (The paper's code generation is sequential; this is the launcher's.)  One such pair per plan; *join = -1: none.  Used for
+ * single equations with device operands (not by the batched and host entry points, nor while step timing is on).  The caller sees
+ * one stream: everything of an execute is ordered after what the stream held before and before what is enqueued after. */
+mom_status_t mom_plan_concurrent_steps(const mom_plan_t *plan, int32_t *begin, int32_t *end, int32_t *join);
+
 /* Number of kernels the most recent execute of this plan enqueued (0 before the first). */
 mom_status_t mom_plan_last_launch_count(const mom_plan_t *plan, int32_t *launches);
 

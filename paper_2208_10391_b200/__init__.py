@@ -100,6 +100,7 @@ _sigs = {
                                   ctypes.c_size_t, _P],
     "mom_plan_device_status": [_P, ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_int32)],
     "mom_probe_wait_timeout": [_P, ctypes.c_double, ctypes.c_int32, _P],
+    "mom_plan_concurrent_steps": [_P, ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_int32)],
     "mom_plan_last_launch_count": [_P, ctypes.POINTER(ctypes.c_int32)],
     "mom_plan_enable_step_timing": [_P, ctypes.c_int32],
     "mom_plan_step_times": [_P, ctypes.c_int32, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_float)],
@@ -299,6 +300,12 @@ class Plan:
     def probe_wait_timeout(self, limit_ms: float, detail: int, stream: int = 0) -> None:
         """Enqueue the bounded-wait self-test: a wait nothing satisfies gives up after `limit_ms`."""
         _check(_lib.mom_probe_wait_timeout(self._h, float(limit_ms), int(detail), _P(stream)), "mom_probe_wait_timeout")
+
+    def concurrent_steps(self) -> Tuple[int, int, int]:
+        """(begin, end, join): steps [begin, end) run on the plan's side stream, step `join` waits for them; join == -1: none."""
+        b, e, j = ctypes.c_int32(), ctypes.c_int32(), ctypes.c_int32()
+        _check(_lib.mom_plan_concurrent_steps(self._h, ctypes.byref(b), ctypes.byref(e), ctypes.byref(j)), "mom_plan_concurrent_steps")
+        return b.value, e.value, j.value
 
     def last_launch_count(self) -> int:
         n = ctypes.c_int32()

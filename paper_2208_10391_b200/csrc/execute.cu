@@ -24,6 +24,9 @@ struct DeviceState {
     long long timed_executes = 0;       // executes recorded since timing was enabled
     // host-staging entry point: uploads run on a stream of their own, one event per operand, so that the first
     // products start while later operands are still on their way
+    // two independent subtrees of small products run side by side: the right one on this stream (see mom_plan::side_join)
+    cudaStream_t side_stream = nullptr;
+    cudaEvent_t side_fork = nullptr, side_done = nullptr;
     cudaStream_t copy_stream = nullptr, back_stream = nullptr;
     cudaEvent_t call_start = nullptr, first_rows_done = nullptr, back_done = nullptr;
     std::vector<cudaEvent_t> slot_ready, add_ready, slot_head;
@@ -70,6 +73,9 @@ void destroy_device_state(DeviceState *d) {
     if (d->call_start) cudaEventDestroy(d->call_start);
     if (d->first_rows_done) cudaEventDestroy(d->first_rows_done);
     if (d->back_done) cudaEventDestroy(d->back_done);
+    if (d->side_fork) cudaEventDestroy(d->side_fork);
+    if (d->side_done) cudaEventDestroy(d->side_done);
+    if (d->side_stream) cudaStreamDestroy(d->side_stream);
     if (d->copy_stream) cudaStreamDestroy(d->copy_stream);
     if (d->back_stream) cudaStreamDestroy(d->back_stream);
     if (d->status) cudaFree(d->status);
@@ -395,8 +401,32 @@ mom_status_t execute_core(const mom_plan *p, const float *const *chain_ptrs, con
                 ++launches;
             }
 
-            for (int s = sum.step_begin; s < sum.step_end; ++s) {
+            // the order in which the steps are enqueued, and on which stream: normally as planned, all on the caller's stream; with two
+            // independent subtrees of small products the right one goes first, onto the plan's side stream, and the step that needs both
+            // waits for it (one instance, device operands, no per-step timing: the other cases keep the plain order)
+            const bool side_by_side = p->side_join >= sum.step_begin && p->side_join < sum.step_end && batch == 1 && !staged && !timing;
+            std::vector<int> order;
+            for (int s = sum.step_begin; s < sum.step_end; ++s)
+                if (side_by_side && s >= p->side_begin && s < p->side_end) order.push_back(s);
+            for (int s = sum.step_begin; s < sum.step_end; ++s)
+                if (!(side_by_side && s >= p->side_begin && s < p->side_end)) order.push_back(s);
+            if (side_by_side) {
+                DeviceState *dev = p->dev;
+                if (!dev->side_stream) {
+                    if (cudaStreamCreateWithFlags(&dev->side_stream, cudaStreamNonBlocking) != cudaSuccess) return MOM_ERR_CUDA;
+                    if (cudaEventCreateWithFlags(&dev->side_fork, cudaEventDisableTiming) != cudaSuccess) return MOM_ERR_CUDA;
+                    if (cudaEventCreateWithFlags(&dev->side_done, cudaEventDisableTiming) != cudaSuccess) return MOM_ERR_CUDA;
+                }
+                // the side stream starts where the caller's stream stands now (earlier work may still use the workspace)
+                if (cudaEventRecord(dev->side_fork, stream) != cudaSuccess || cudaStreamWaitEvent(dev->side_stream, dev->side_fork, 0) != cudaSuccess)
+                    return MOM_ERR_CUDA;
+            }
+            cudaStream_t const caller_stream = stream;
+            for (int s : order) {
                 const StepImpl &stp = p->steps[s];
+                const bool on_side = side_by_side && s >= p->side_begin && s < p->side_end;
+                cudaStream_t const stream = on_side ? p->dev->side_stream : caller_stream;      // shadows the caller's stream inside the step
+                if (side_by_side && s == p->side_join && cudaStreamWaitEvent(caller_stream, p->dev->side_done, 0) != cudaSuccess) return MOM_ERR_CUDA;
                 if (stp.folded) {                        // a scaling done by its reader's operand-split pass: nothing to launch
                     if (timing) {
                         cudaEvent_t *fe = &p->dev->events[((size_t)(p->dev->timed_executes % TIMING_SLOTS) * ns + s) * 3];
@@ -517,6 +547,7 @@ mom_status_t execute_core(const mom_plan *p, const float *const *chain_ptrs, con
                     ++launches;
                 }
                 if (ev) cudaEventRecord(ev[2], stream);
+                if (on_side && s + 1 == p->side_end && cudaEventRecord(p->dev->side_done, stream) != cudaSuccess) return MOM_ERR_CUDA;
             }
 
             // summands beyond the fused limit: value += T, a few at a time, in place

@@ -134,6 +134,10 @@ struct mom_plan {
     mom_matrix_desc_t product_desc{};          // chain value before the Add terms
     mom_matrix_desc_t result_desc{};
     size_t workspace_per_instance = 0;
+    // Two independent subtrees of the parenthesization, both made of small products, run side by side: steps
+    // [side_begin, side_end) -- the right subtree of step `side_join` -- go to a second stream the plan owns while the left
+    // subtree runs on the caller's stream; side_join waits for both.  side_join < 0: everything runs in order.
+    int side_begin = 0, side_end = 0, side_join = -1;
     // fused small-equation kernel: whole plan in shared memory, one instance per CTA (no workspace)
     bool fused_ok = false;
     size_t fused_smem_bytes = 0;

@@ -695,6 +695,42 @@ static mom_status_t plan_sums(const std::vector<mom_matrix_desc_t> &slots, const
                 items.push_back(Interval{mom::align_up((size_t)st.split_k * slab_rows * n * sizeof(float), mom::WS_ALIGN), s, s, &st.partial_off, 0});
             }
         }
+        // Small products leave most of the GPU idle (a launch of a few microseconds on a few dozen SMs), so two subtrees of the tree that
+        // do not depend on each other run side by side on two streams: the five-matrix chain ((0*(1*2))*(3*4)) computes (3*4) while
+        // (0*(1*2)) is under way.  One such pair per plan: the node whose smaller subtree is the largest.  Every buffer either subtree
+        // touches is kept for the whole of both (their steps no longer run one after the other).
+        if (single_chain && variant != MOM_VARIANT_FFMA) {
+            std::vector<int> first(ns, 0);                   // first step of the subtree that ends at step s (post-order: contiguous)
+            std::vector<double> work(ns, 0.0);
+            std::vector<char> small(ns, 1);
+            for (int s = 0; s < ns; ++s) {
+                const mom_step_t &st = p->steps[s].pub;
+                first[s] = s;
+                work[s] = (double)st.m * (double)st.n * (double)st.k;
+                small[s] = st.uses_tensor_cores != 1 && st.kind != MOM_KIND_SCALE && work[s] < mom::INLINE_MAX_WORK && !p->steps[s].folded;
+                for (int32_t v : {st.lhs, st.rhs})
+                    if (v >= n_chain) {
+                        const int c = v - n_chain;
+                        first[s] = std::min(first[s], first[c]);
+                        work[s] += work[c];
+                        small[s] = small[s] && small[c];
+                    }
+            }
+            double best = 0.0;
+            for (int s = 0; s < ns; ++s) {
+                const mom_step_t &st = p->steps[s].pub;
+                if (st.lhs < n_chain || st.rhs < n_chain || st.lhs == st.rhs) continue;
+                const int l = st.lhs - n_chain, r = st.rhs - n_chain;
+                if (!small[l] || !small[r] || r != s - 1 || l != first[r] - 1) continue;      // left subtree, then right subtree, then s
+                const double gain = std::min(work[l], work[r]);
+                if (gain > best) { best = gain; p->side_begin = first[r]; p->side_end = r + 1; p->side_join = s; }
+            }
+            if (p->side_join >= 0) {
+                const int lo = first[p->steps[p->side_join].pub.lhs - n_chain], hi = p->side_join;
+                for (Interval &it : items)
+                    if (!(it.last < lo || it.first > hi)) { it.first = std::min(it.first, lo); it.last = std::max(it.last, hi); }
+            }
+        }
         p->workspace_per_instance = pack(items);
         for (const Copy &c : copies) {
             if (c.owner < 0) continue;
@@ -1079,6 +1115,14 @@ mom_status_t mom_plan_host_staging_bytes(const mom_plan_t *plan, int64_t batch, 
     mom_plan_workspace_bytes(plan, batch, &ws);
     total += ws;
     *bytes = total;
+    return MOM_OK;
+}
+
+mom_status_t mom_plan_concurrent_steps(const mom_plan_t *plan, int32_t *begin, int32_t *end, int32_t *join) {
+    if (!plan || !begin || !end || !join) return MOM_ERR_INVALID_ARG;
+    *begin = plan->side_join >= 0 ? plan->side_begin : 0;
+    *end = plan->side_join >= 0 ? plan->side_end : 0;
+    *join = plan->side_join;
     return MOM_OK;
 }
 

@@ -135,6 +135,36 @@ def test_inline_split_tensor_core_kernel(m, k, n, pa, pb, terms):
     check_against_oracle(eq, x, plan, chain, terms_h)
 
 
+def test_subtrees_side_by_side_on_two_streams():
+    # chains whose chosen tree multiplies two products: the right subtree runs on the plan's side stream beside the left one.
+    # Same values as the plan computed in order (the forced variants keep the plain order), within the bound of the oracle,
+    # also when the same plan is executed again and again on the same workspace.
+    rng = np.random.default_rng(11)
+    found = 0
+    for trial in range(60):
+        n = int(rng.integers(4, 7))
+        dims = [int(rng.choice([8, 24, 64, 136, 264, 520])) for _ in range(n + 1)]
+        props = [G] * n
+        eq = Equation(f"side_{trial}", 500 + trial, tuple(Operand(dims[i], dims[i + 1], props[i], "normal", 1.0 / np.sqrt(dims[i + 1])) for i in range(n)))
+        plan = mom.mom_equation_plan(eq.descs(), (), mom.VARIANT_3XTF32)
+        if plan.concurrent_steps()[2] < 0 or plan.workspace_bytes() == 0:
+            continue
+        found += 1
+        chain, add = wl.generate(eq)
+        x, plan, _ = run_equation(eq, mom.VARIANT_3XTF32, chain, add)
+        check_against_oracle(eq, x, plan, chain, add)
+        dchain = [torch.from_numpy(a).cuda() for a in chain]
+        outs = torch.full((20,) + x.shape, float("nan"), dtype=torch.float32, device="cuda")
+        wsb = plan.workspace_bytes(1)
+        ws = torch.empty(wsb, dtype=torch.uint8, device="cuda")
+        for i in range(20):
+            plan.execute([t.data_ptr() for t in dchain], [], outs[i].data_ptr(), ws.data_ptr(), wsb, torch.cuda.current_stream().cuda_stream)
+        torch.cuda.synchronize()
+        o = outs.cpu().numpy()
+        assert all(np.array_equal(o[i], x) for i in range(20))
+    assert found >= 10
+
+
 @pytest.mark.parametrize("case", ["LG", "GU_plus_C", "chain"])
 def test_pair_kernel_ragged_shapes(case):
     # big enough for the CTA-pair tensor-core kernel (256-row tiles), with edges that are not multiples of the tile

@@ -504,3 +504,27 @@ def test_kernel_choice_of_the_default_variant():
     assert kind(512, 512, 510) == 2                        # rows TMA cannot address
     assert kind(640, 640, 640, (True, False)) == 2 and kind(640, 640, 640, (False, True)) == 2     # transposed operands
     assert kind(1024, 1024, 1024, (True, False)) == 1      # the plane kernel reads transposed operands through its split pass
+
+
+def test_independent_subtrees_of_small_products_are_marked_to_run_side_by_side():
+    G = wl.GENERAL
+    five = wl.config_five_general()
+    p = mom.mom_equation_plan(five.descs(), (), mom.VARIANT_3XTF32)
+    assert p.parenthesization() == "((0*(1*2))*(3*4))"
+    steps = p.steps()
+    assert [(s.lhs, s.rhs) for s in steps] == [(1, 2), (0, 5), (3, 4), (6, 7)]
+    assert p.concurrent_steps() == (2, 3, 3)               # (3*4) beside (0*(1*2)); the last product waits for both
+    # the buffers of both subtrees are alive together: nothing is shared between them
+    sizes = [256 * 64 * 4, 1024 * 64 * 4, 64 * 512 * 4]
+    assert p.workspace_bytes() >= sum(sizes)
+    # a right-nested chain has no such pair; large products are left in order (each fills the GPU by itself); nor does the FFMA variant pair
+    assert mom.mom_equation_plan(wl.config_paper_chain().descs(), (), mom.VARIANT_3XTF32).concurrent_steps()[2] == -1
+    big = [(512, 8192, G), (8192, 4096, G), (4096, 8192, G), (8192, 512, G)]
+    p = mom.mom_equation_plan(big, (), mom.VARIANT_3XTF32)
+    assert p.parenthesization() == "((0*1)*(2*3))" and p.concurrent_steps()[2] == -1
+    assert mom.mom_equation_plan(five.descs(), (), mom.VARIANT_FFMA).concurrent_steps()[2] == -1
+    # a pair below the root: ((0*1)*(2*3))*4
+    deep = [(200, 40, G), (40, 200, G), (200, 40, G), (40, 200, G), (200, 8, G)]
+    p = mom.mom_equation_plan(deep, (), mom.VARIANT_3XTF32)
+    if p.parenthesization() == "(((0*1)*(2*3))*4)":
+        assert p.concurrent_steps() == (1, 2, 2)
