@@ -28,9 +28,9 @@ constexpr size_t WS_ALIGN = 256;
 
 // Default variant: where the one-launch tcgen05 kernel (product_tc_inline.cu) is the quickest of the three tensor-core kernels
 // (back to back, us, warp-level / plane-fed / one-launch: 448^3 12.8 / 31.0 / 11.6, 512^3 13.1 / 26.5 / 10.0, 768^3 28.9 / 29.0 / 17.9,
-// 1024^3 63.7 / 35.2 / 32.3, 1280^3 113.5 / 50.0 / 100.4; 900 x 1200 x 100 14.8 / 27.3 / 14.2, 4096 x 256 x 64 12.8 / 22.7 / 8.0,
+// 896^3 45.7 / 33.1 / 29.1, 1024^3 65.6 / 31.2 / 32.5, 1280^3 115.3 / 48.4 / 101.5; 900 x 1200 x 100 14.8 / 27.3 / 14.2, 4096 x 256 x 64 12.8 / 22.7 / 8.0,
 // 256 x 2048 x 64 9.3 / 24.7 / 12.9, 128 x 4096 x 128 16.5 / 26.8 / 20.2).
-constexpr double INLINE_MIN_WORK = 6.0e7, INLINE_MAX_WORK = 1.2e9, INLINE_MIN_OUTPUT = 65536.0;
+constexpr double INLINE_MIN_WORK = 6.0e7, INLINE_MAX_WORK = 1.0e9, INLINE_MIN_OUTPUT = 65536.0;
 
 // Largest rows / cols a descriptor may have: every kernel indexes rows, columns and k with 32-bit integers.
 constexpr int64_t MAX_DIMENSION = 2147483647 - 1024;

@@ -565,7 +565,7 @@ static mom_status_t plan_sums(const std::vector<mom_matrix_desc_t> &slots, const
                                    mom::product_tc_inline_takes(m, n, k, st.pub.lhs_transposed, st.pub.rhs_transposed,
                                                                 mom::kernel_property(st.pub.lhs_property), mom::kernel_property(st.pub.rhs_property));
             // ... and it pays between the two (measured, see the kernel's file): from about 450^3 on it beats the warp-level kernel, up to
-            // about 1000^3 its single launch beats the plane kernel's two or three; a result of fewer than four 128 x 128 tiles would leave
+            // about 900^3 its single launch beats the plane kernel's two; a result of fewer than four 128 x 128 tiles would leave
             // each CTA a long contraction even when split over a cluster, and the warp-level kernel is quicker there
             const double work = (double)m * (double)n * (double)k;
             const bool inline_pays = work >= mom::INLINE_MIN_WORK && work < mom::INLINE_MAX_WORK && (double)m * (double)n >= mom::INLINE_MIN_OUTPUT;

@@ -51,6 +51,7 @@ constexpr int THREADS = 192;
 constexpr uint32_t TMEM_COLS = 512;          // two accumulators of BN columns
 
 static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
+static_assert(BM * (BN + 4) * 4 <= STAGES * STAGE_BYTES, "a partial tile fits where the stages were");
 static_assert(SPLIT_BLOCK % BM == 0 && SPLIT_BLOCK % BN == 0, "split blocks must cover whole tiles");
 
 struct Shared {
@@ -65,6 +66,15 @@ struct Shared {
 constexpr int TILE_SLICE_SHIFT = 24;
 constexpr int TILE_ROW_MASK = (1 << TILE_SLICE_SHIFT) - 1;
 
+// 16 bytes from the shared memory of CTA `rank` of this cluster, at this CTA's offset `addr`
+__device__ __forceinline__ float4 ld_cluster_f4(uint32_t addr, uint32_t rank) {
+    float4 v;
+    const uint32_t remote = ptx::map_to_cta(addr, rank);
+    asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(remote) : "memory");
+    return v;
+}
+constexpr int CLUSTER_LDP = TC_BN + 4;       // row length (floats) of a partial tile in shared memory: 16-byte rows, conflict-free per 8 lanes
+
 struct TcParams {
     const int4 *tiles;
     int num_tiles;
@@ -72,6 +82,9 @@ struct TcParams {
     int pout;
     int out_mode;            // 0: f32 result through map_c; 1: hi/lo planes (map_c, map_c2); 2: transposed hi/lo planes
     int slice_rows;          // split-K: rows between the partial-sum slabs of consecutive k-slices (0: no split)
+    int cluster_split;       // > 1 (1-CTA kernel): the k-slices of a tile are the CTAs of one thread-block cluster; they leave their partial
+                             // tiles in shared memory and share out the tile's rows, adding the slices through distributed shared memory
+    float *c_out;            // cluster_split: the result matrix (plain stores from the reduction)
     float *packed_c;         // not null (out_mode 0 only): the result is a packed triangle written in place with plain
                              // 16-byte stores; entries the container does not hold are not written at all
     int mirror;              // Gram product Y * Y^T (CTA-pair kernel, out_mode 0, Symmetric Add terms only): the table holds the tiles on and
@@ -341,7 +354,16 @@ product_tc_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_con
 #pragma unroll
                     for (int j = 0; j < 32; ++j) v[j] = 0.0f;
                 }
-                if (rows_left > 0) epilogue_chunk(prm, &map_c, &map_c2, v, r, store_row, col0, lane, stage_buf, store_it);
+                if (prm.cluster_split > 1) {
+                    // every stage has been consumed by now (the accumulator is complete): the partial tile takes their place
+                    const uint32_t dst = base + (uint32_t)((q * 32 + lane) * CLUSTER_LDP + c * 32) * 4u;
+#pragma unroll
+                    for (int j = 0; j < 8; ++j)
+                        asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(dst + 16 * j), "f"(v[4 * j]), "f"(v[4 * j + 1]), "f"(v[4 * j + 2]),
+                                     "f"(v[4 * j + 3]) : "memory");
+                } else if (rows_left > 0) {
+                    epilogue_chunk(prm, &map_c, &map_c2, v, r, store_row, col0, lane, stage_buf, store_it);
+                }
             }
             if (!zero_tile) {
                 ptx::tc_fence_before_sync();
@@ -357,6 +379,37 @@ product_tc_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_con
     __syncthreads();
     ptx::tc_fence_after_sync();
     if (warp == 1) ptx::tmem_dealloc(tmem_base, TMEM_COLS);
+
+    if (prm.cluster_split > 1) {
+        // ---- split contraction inside a cluster: CTA `rank` finishes rows [rank * 128 / s, (rank + 1) * 128 / s) of the tile, adding the
+        // cluster's partial tiles in k order (deterministic); Add terms and mask as in the ordinary epilogue, 16-byte stores
+        const int split = prm.cluster_split;
+        const uint32_t rank = ptx::cluster_cta_rank();
+        const int4 tile = prm.tiles[blockIdx.x];
+        const int r0 = tile.x & TILE_ROW_MASK, c0 = tile.y;
+        ptx::cluster_sync();                                  // every CTA of the cluster comes here, also one that gave up
+        const int rows_per = BM / split;
+        const bool vec = (reinterpret_cast<uintptr_t>(prm.c_out) & 15) == 0;
+        for (int e = threadIdx.x; e < rows_per * (BN / 4); e += THREADS) {
+            const int row = (int)rank * rows_per + e / (BN / 4), col = (e % (BN / 4)) << 2;
+            const int r = r0 + row, cc = c0 + col;
+            if (r >= prm.m || cc >= prm.n) continue;
+            float w[4] = {0.f, 0.f, 0.f, 0.f};
+            for (int peer = 0; peer < split; ++peer) {
+                const float4 x = ld_cluster_f4(base + (uint32_t)(row * CLUSTER_LDP + col) * 4u, (uint32_t)peer);
+                w[0] += x.x; w[1] += x.y; w[2] += x.z; w[3] += x.w;
+            }
+            finish_row4(w, prm.add, 0, r, cc, prm.n, prm.n, prm.pout, vec);
+            float *dst = prm.c_out + (long long)r * prm.n + cc;
+            if (vec && cc + 3 < prm.n) {
+                *reinterpret_cast<float4 *>(dst) = make_float4(w[0], w[1], w[2], w[3]);
+            } else {
+                for (int j = 0; j < 4; ++j)
+                    if (cc + j < prm.n) dst[j] = w[j];
+            }
+        }
+        ptx::cluster_sync();                                  // nobody leaves while a peer may still read its tile
+    }
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -863,7 +916,27 @@ mom_status_t tc_prepare(const mom_plan &p, TcPlanState &s) {
                 total += part_tables[q][i].size();
             }
         }
-        s.steps[i].units = order(tab);
+        // Split-K with up to 8 slices per tile: the slices of a tile form a thread-block cluster and add their partial tiles through
+        // distributed shared memory (no scratch, no reduction launch), provided all the clusters can run at once (a cluster sits in one
+        // GPC and every CTA here takes a whole SM).  The table then stays in tile order, slice by slice: CTA i takes entry i.
+        if (split > 1 && split <= 8 && (split & (split - 1)) == 0 && BM % split == 0 && (int)tab.size() <= sms) {
+            int fit = 0;
+            cudaLaunchConfig_t probe = {};
+            probe.gridDim = dim3((unsigned)tab.size());
+            probe.blockDim = dim3(THREADS);
+            probe.dynamicSmemBytes = SMEM_BYTES;
+            cudaLaunchAttribute at[1];
+            at[0].id = cudaLaunchAttributeClusterDimension;
+            at[0].val.clusterDim.x = (unsigned)split; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+            probe.attrs = at;
+            probe.numAttrs = 1;
+            if (raise_smem_limit_once(product_tc_kernel, SMEM_BYTES, &DeviceInfo::tc_attr) == cudaSuccess &&
+                cudaOccupancyMaxActiveClusters(&fit, product_tc_kernel, &probe) == cudaSuccess && fit * split >= (int)tab.size())
+                s.steps[i].cluster_split = split;
+            else
+                cudaGetLastError();
+        }
+        s.steps[i].units = s.steps[i].cluster_split > 1 ? (int)tab.size() : order(tab);
         total += tab.size();
     }
     if (total == 0) { s.ready = true; return MOM_OK; }
@@ -984,9 +1057,13 @@ mom_status_t tc_launch_step(const mom_plan &p, TcPlanState &s, int step, const P
     prm.num_tiles = num_tiles;
     prm.m = a.m;
     prm.n = a.n;
-    prm.pout = st.split_k > 1 ? (int)MOM_GENERAL : a.pout;      // split-K: mask and Add terms are applied by the reduction
+    const bool separate_reduction = st.split_k > 1 && !(part == 0 && s.steps[step].cluster_split > 1);
+    prm.pout = separate_reduction ? (int)MOM_GENERAL : a.pout;   // split-K with a reduction launch: it applies mask and Add terms
     prm.out_mode = st.planes_out;
     prm.slice_rows = slice_rows;
+    const int cluster_split = part == 0 ? s.steps[step].cluster_split : 0;
+    prm.cluster_split = cluster_split;
+    prm.c_out = a.C;
     if (s.steps[step].mirror && st.planes_out != 0) return MOM_ERR_INVALID_ARG;   // the planner never asks for this
     prm.mirror = s.steps[step].mirror ? 1 : 0;
     prm.packed_c = nullptr;
@@ -996,7 +1073,7 @@ mom_status_t tc_launch_step(const mom_plan &p, TcPlanState &s, int step, const P
         prm.packed_c = a.C;
     }
     prm.add = a.add;
-    if (st.split_k > 1) prm.add.count = 0;
+    if (separate_reduction) prm.add.count = 0;
     prm.status = status;
     if (s.steps[step].pair) {
         if (raise_smem_limit_once(product_tc_pair_kernel, P_SMEM_BYTES, &DeviceInfo::pair_attr) != cudaSuccess) return MOM_ERR_CUDA;
@@ -1032,11 +1109,28 @@ mom_status_t tc_launch_step(const mom_plan &p, TcPlanState &s, int step, const P
         if (cudaLaunchKernelEx(&cfg, product_tc_pair_kernel, ma_hi, ma_lo, mb_hi, mb_lo, mc, mc2, prm) != cudaSuccess) return MOM_ERR_CUDA;
     } else {
         const int grid = std::min(units, sm_count);
-        product_tc_kernel<<<grid, THREADS, SMEM_BYTES, stream>>>(ma_hi, ma_lo, mb_hi, mb_lo, mc, mc2, prm);
+        if (cluster_split > 1) {
+            if (grid != units || grid % cluster_split != 0) return MOM_ERR_CUDA;      // one table entry per CTA, whole clusters
+            cudaLaunchConfig_t cfg = {};
+            cfg.gridDim = dim3(grid);
+            cfg.blockDim = dim3(THREADS);
+            cfg.dynamicSmemBytes = SMEM_BYTES;
+            cfg.stream = stream;
+            cudaLaunchAttribute attr[1];
+            attr[0].id = cudaLaunchAttributeClusterDimension;
+            attr[0].val.clusterDim.x = (unsigned)cluster_split;
+            attr[0].val.clusterDim.y = 1;
+            attr[0].val.clusterDim.z = 1;
+            cfg.attrs = attr;
+            cfg.numAttrs = 1;
+            if (cudaLaunchKernelEx(&cfg, product_tc_kernel, ma_hi, ma_lo, mb_hi, mb_lo, mc, mc2, prm) != cudaSuccess) return MOM_ERR_CUDA;
+        } else {
+            product_tc_kernel<<<grid, THREADS, SMEM_BYTES, stream>>>(ma_hi, ma_lo, mb_hi, mb_lo, mc, mc2, prm);
+        }
     }
     if (cudaGetLastError() != cudaSuccess) return MOM_ERR_CUDA;
     *launches = 1 + split_launches;
-    if (st.split_k > 1) {
+    if (separate_reduction) {
         const long long vecs = (long long)a.m * (a.n / 4);
         const int blocks_r = (int)std::min<long long>((vecs + 255) / 256, (long long)sm_count * 8);
         splitk_reduce_kernel<<<blocks_r, 256, 0, stream>>>(partial, st.split_k, slice_rows, a.C, a.m, a.n, a.pout, a.add);
@@ -1257,6 +1351,8 @@ extern "C" mom_status_t mom_product_3xtf32_noalloc(int64_t m64, int64_t n64, int
     prm.pout = pa == MOM_GENERAL || pb == MOM_GENERAL || pa != pb ? (int)MOM_GENERAL : (int)pa;
     prm.out_mode = 0;
     prm.slice_rows = 0;
+    prm.cluster_split = 0;
+    prm.c_out = nullptr;
     prm.mirror = 0;
     prm.packed_c = nullptr;
     prm.add.count = 0;

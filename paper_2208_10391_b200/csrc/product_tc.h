@@ -24,6 +24,7 @@ struct TcStepState {
     // ranges let the host-staging entry point upload that operand in two pieces and start on the first one while the
     // second is still on its way; then each launch splits its own rows of the operand.  False: splits happen in part 1.
     bool split_a_by_part = false;
+    int cluster_split = 0;      // > 1: split-K inside thread-block clusters of this size (table in tile order, one entry per CTA)
     int units = 1;              // CTAs (or CTA pairs) the table was laid out for: unit u owns entries u, u + units, ...
 };
 
