@@ -99,11 +99,12 @@ typedef enum { MOM_F32 = 0 } mom_dtype_t;
 /* Arithmetic used by the product kernels.
  *   MOM_VARIANT_3XTF32: tensor-core MMA (kind::tf32 / .tf32) on operands split as a = hi + lo,
  *       accumulating lo*hi + hi*lo + hi*hi in f32 (f32-level accuracy).  Three kernels, chosen by size:
- *       large products (m*n*k >= 6 * 2^26, from 10^9 on when the kernel below takes the shape) whose leading
+ *       large products (m*n*k >= 6 * 2^26 that the kernel below does not take) whose leading
  *       dimensions TMA can address (multiples of 4 elements) run on the tcgen05 kernel that takes its operands as
  *       hi / lo planes (a pre-pass writes them; TMA, tensor memory, persistent CTAs); products of stored
- *       (untransposed) operands with 6 * 10^7 <= m*n*k < 10^9 and a result of at least 65536 entries run on the
- *       tcgen05 kernel that reads the operands as stored and splits them in shared memory (one launch); everything
+ *       (untransposed) operands with a result of at least 65536 entries and 6 * 10^7 <= m*n*k < 10^9, or
+ *       m*n*k < 4 * 10^9 with at most 148 result tiles of 128 x 128, run on the tcgen05 kernel that reads the
+ *       operands as stored and splits them on the way into shared and tensor memory (one launch); everything
  *       else runs on the warp-level kernel (mma.sync on the operands as stored, one launch).
  *   MOM_VARIANT_FFMA: plain f32 fused multiply-add on CUDA cores.
  *   MOM_VARIANT_3XTF32_FORCE: every TMA-addressable product runs on the tcgen05 kernel, the others on

@@ -27,10 +27,15 @@ constexpr int FF_BN = 128;
 constexpr size_t WS_ALIGN = 256;
 
 // Default variant: where the one-launch tcgen05 kernel (product_tc_inline.cu) is the quickest of the three tensor-core kernels
-// (back to back, us, warp-level / plane-fed / one-launch: 448^3 12.8 / 31.0 / 11.6, 512^3 13.1 / 26.5 / 10.0, 768^3 28.9 / 29.0 / 17.9,
-// 896^3 45.7 / 33.1 / 29.1, 1024^3 65.6 / 31.2 / 32.5, 1280^3 115.3 / 48.4 / 101.5; 900 x 1200 x 100 14.8 / 27.3 / 14.2, 4096 x 256 x 64 12.8 / 22.7 / 8.0,
-// 256 x 2048 x 64 9.3 / 24.7 / 12.9, 128 x 4096 x 128 16.5 / 26.8 / 20.2).
-constexpr double INLINE_MIN_WORK = 6.0e7, INLINE_MAX_WORK = 1.0e9, INLINE_MIN_OUTPUT = 65536.0;
+// (back to back, us, warp-level / plane-fed / one-launch: 256^3 8.6 / 24.9 / 8.2, 448^3 14.5 / 30.9 / 8.8, 512^3 14.8 / 23.8 / 9.0,
+// 768^3 31.1 / 30.0 / 14.6, 1024^3 65.2 / 31.3 / 22.0, 1280^3 115 / 48.4 / 41.0, 1536^3 - / 55.7 / 48.3, 2048^3 - / 95 / 116;
+// 900 x 1200 x 100 16.6 / 27.1 / 10.9, 4096 x 256 x 64 10.4 / 22.7 / 7.6, 256 x 2048 x 64 10.5 / 23.7 / 10.7, 128 x 4096 x 128 14.8 / 26.8 / 15.5).
+// Up to INLINE_SMALL_WORK it is taken whatever the shape; up to INLINE_MAX_WORK while its 128 x 128 tiles fit one wave of CTAs
+// (a second wave repeats the whole of the first: 1792^3 93 us against 1536^3 48 us).
+constexpr double INLINE_MIN_WORK = 6.0e7, INLINE_SMALL_WORK = 1.0e9, INLINE_MAX_WORK = 4.0e9, INLINE_MIN_OUTPUT = 65536.0;
+constexpr int64_t INLINE_WAVE_TILES = 148;
+// Products below this many multiplications count as small when independent subtrees are put side by side on two streams.
+constexpr double SIDE_BY_SIDE_MAX_WORK = 1.0e9;
 
 // Largest rows / cols a descriptor may have: every kernel indexes rows, columns and k with 32-bit integers.
 constexpr int64_t MAX_DIMENSION = 2147483647 - 1024;

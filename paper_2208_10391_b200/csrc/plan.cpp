@@ -564,11 +564,14 @@ static mom_status_t plan_sums(const std::vector<mom_matrix_desc_t> &slots, const
             const bool inline_ok = st.pub.kind != MOM_KIND_GRAM &&
                                    mom::product_tc_inline_takes(m, n, k, st.pub.lhs_transposed, st.pub.rhs_transposed,
                                                                 mom::kernel_property(st.pub.lhs_property), mom::kernel_property(st.pub.rhs_property));
-            // ... and it pays between the two (measured, see the kernel's file): from about 450^3 on it beats the warp-level kernel, up to
-            // about 900^3 its single launch beats the plane kernel's two; a result of fewer than four 128 x 128 tiles would leave
-            // each CTA a long contraction even when split over a cluster, and the warp-level kernel is quicker there
+            // ... and it pays between the two (measured, see the constants): from about 400^3 on it beats the warp-level kernel, and
+            // its single launch beats the plane kernel's two up to 1000^3 whatever the shape and up to about 1600^3 while its
+            // 128 x 128 tiles fit one wave of CTAs; a result of fewer than four 128 x 128 tiles would leave each CTA a long
+            // contraction even when split over a cluster, and the warp-level kernel is quicker there
             const double work = (double)m * (double)n * (double)k;
-            const bool inline_pays = work >= mom::INLINE_MIN_WORK && work < mom::INLINE_MAX_WORK && (double)m * (double)n >= mom::INLINE_MIN_OUTPUT;
+            const bool one_wave = ((m + 127) / 128) * ((n + 127) / 128) <= mom::INLINE_WAVE_TILES;
+            const bool inline_pays = work >= mom::INLINE_MIN_WORK && (double)m * (double)n >= mom::INLINE_MIN_OUTPUT &&
+                                     (work < mom::INLINE_SMALL_WORK || (work < mom::INLINE_MAX_WORK && one_wave));
             if (st.pub.kind == MOM_KIND_SCALE) st.pub.uses_tensor_cores = 0;       // a Diagonal operand: one scaling pass, bound by HBM
             else if (variant == MOM_VARIANT_3XTF32) st.pub.uses_tensor_cores = inline_ok && inline_pays ? 3 : addressable && large ? 1 : 2;
             else if (variant == MOM_VARIANT_3XTF32_FORCE) st.pub.uses_tensor_cores = addressable ? 1 : 0;
@@ -707,7 +710,7 @@ static mom_status_t plan_sums(const std::vector<mom_matrix_desc_t> &slots, const
                 const mom_step_t &st = p->steps[s].pub;
                 first[s] = s;
                 work[s] = (double)st.m * (double)st.n * (double)st.k;
-                small[s] = st.uses_tensor_cores != 1 && st.kind != MOM_KIND_SCALE && work[s] < mom::INLINE_MAX_WORK && !p->steps[s].folded;
+                small[s] = st.uses_tensor_cores != 1 && st.kind != MOM_KIND_SCALE && work[s] < mom::SIDE_BY_SIDE_MAX_WORK && !p->steps[s].folded;
                 for (int32_t v : {st.lhs, st.rhs})
                     if (v >= n_chain) {
                         const int c = v - n_chain;

@@ -4,23 +4,25 @@
 // The large-product kernel (product_tc.cu) takes its operands as hi / lo planes that a pre-pass writes to global
 // memory, and with few output tiles it needs a split-K reduction pass: two or three launches, which is most of the
 // time of a product below about 2000^3.  Here a product is one launch:
-//   warp 0      TMA producer: per k-block of 32 the raw f32 tile of A (128 rows x 32 k: already K-major, loaded under
-//               the 128-byte swizzle the MMA wants) and the raw tile of B (32 k-rows x BN columns, as BN / 32 swizzled
-//               boxes of 32 x 32);
-//   warps 2-9   transform: A is split where it lies (the hi half overwrites the raw tile, the lo half goes to a second
-//               tile at the same offsets); B is split AND transposed into K-major hi / lo tiles (BN rows of 32 k): a lane
-//               reads four columns of its k-row with one 16-byte load -- the eight lanes of a load phase hit eight
-//               different swizzled chunks -- and writes each value into its column's row, where the 32 lanes of a
-//               warp fill one 128-byte row: no bank conflict on either side;
-//   warp 1      MMA issuer: 4 k-steps x 3 tcgen05.mma kind::tf32 (lo*hi, hi*lo, hi*hi; M128, N = BN) per k-block into one
-//               accumulator in tensor memory; tcgen05.commit frees the stage;
+//   warp 0      TMA producer: per k-block of 32 the raw f32 tile of A (128 rows x 32 k, 128-byte swizzle) and the raw tile
+//               of B (32 k-rows x BN columns, as BN / 32 swizzled boxes of 32 x 32);
+//   warps 2-9   transform: a thread reads half of its row of A (the eight lanes of a load phase hit eight different
+//               swizzled chunks), splits it in registers and stores the hi and lo halves into TENSOR MEMORY with
+//               tcgen05.st (lane = row, one column per k): the MMA takes its A operand from there, so A is never
+//               written back to shared memory nor read from it by the tensor core.  B is split AND transposed into
+//               K-major hi / lo tiles in shared memory (BN rows of 32 k): a lane reads four columns of its k-row with
+//               one 16-byte load and writes each value into its column's row, where the 32 lanes of a warp fill one
+//               128-byte row: no bank conflict on either side;
+//   warp 1      MMA issuer: 4 k-steps x 3 tcgen05.mma kind::tf32 (lo*hi, hi*lo, hi*hi; M128, N = BN; A from tensor memory,
+//               B through a shared-memory descriptor) per k-block into one accumulator in tensor memory; tcgen05.commit
+//               frees the stage;
 //   warps 2-9   then the epilogue: tcgen05.ld (two warps per quarter of the tile's rows, each half of the columns), Add terms,
 //               structure mask, 16-byte stores.
 // With few output tiles the contraction is split over the CTAs of a thread-block cluster (up to 8): each leaves its partial
 // tile in its own shared memory and CTA r finishes rows [r * 128 / s, (r + 1) * 128 / s) by adding the partial tiles through
 // distributed shared memory in k order (deterministic; no atomics, no scratch in global memory, no second launch).
-// The tile's structural k-range bounds the contraction as everywhere else.  Shared memory moves about twice the bytes per
-// flop that the plane kernel moves (the transform reads and writes every operand byte once more), so this kernel tops out
+// The tile's structural k-range bounds the contraction as everywhere else.  Shared memory still moves more bytes per
+// flop than in the plane kernel (the transform reads every operand byte and writes B once more), so this kernel tops out
 // near half of the tensor peak; it is chosen where launches, not flops, are the cost.
 // Every wait is bounded; a CTA that gives up still meets its cluster at both cluster barriers.
 #include <algorithm>
@@ -45,11 +47,14 @@ constexpr int XFORM_WARPS = 8, XFORM_THREADS = 32 * XFORM_WARPS;
 
 template <int BN>
 struct InlineCfg {
-    static constexpr int STAGES = BN == 64 ? 3 : 2;
-    static constexpr int A_BYTES = IBM * IBK * 4;            // 16 KB: the raw tile, then its hi half
+    static constexpr int STAGES = BN == 64 ? 5 : 3;
+    static constexpr int A_BYTES = IBM * IBK * 4;            // 16 KB: the raw tile of A
     static constexpr int B_RAW_BYTES = IBK * BN * 4;         // BN / 32 boxes of 32 k-rows x 32 columns
     static constexpr int B_PLANE_BYTES = BN * IBK * 4;       // K-major: BN rows of 32 k
-    static constexpr int STAGE_BYTES = 2 * A_BYTES + B_RAW_BYTES + 2 * B_PLANE_BYTES;
+    static constexpr int STAGE_BYTES = A_BYTES + B_RAW_BYTES + 2 * B_PLANE_BYTES;
+    // tensor memory: the accumulator in columns [0, BN), then per stage 32 columns of A's hi half and 32 of its lo half
+    static constexpr int A_COLS = 2 * IBK, TMEM_COLS = 512;
+    static_assert(BN + STAGES * A_COLS <= TMEM_COLS, "tensor memory budget");
     static constexpr int LDP = BN + 4;                       // row length of the partial tile (floats)
     static constexpr int NUM_BARRIERS = 3 * STAGES + 2;
     static constexpr int SMEM_BYTES = 1024 + STAGES * STAGE_BYTES + 256;
@@ -119,7 +124,7 @@ product_tc_inline_kernel(const __grid_constant__ CUtensorMap map_a, const __grid
         ptx::fence_barrier_init();
     }
     if (warp == 1) {
-        ptx::tmem_alloc(tmem_slot, BN);
+        ptx::tmem_alloc(tmem_slot, Cfg::TMEM_COLS);
         ptx::tmem_relinquish();
     }
     ptx::tc_fence_before_sync();
@@ -144,7 +149,7 @@ product_tc_inline_kernel(const __grid_constant__ CUtensorMap map_a, const __grid
             const int kb = klo + (kb0 + i) * IBK;
             const uint32_t st = base + s * Cfg::STAGE_BYTES;
             if (lane == 0) ptx::tma_load_2d(st, &map_a, kb, r0, raw_full(s));
-            else if (lane <= BN / 32) ptx::tma_load_2d(st + 2 * Cfg::A_BYTES + (lane - 1) * 4096, &map_b, c0 + 32 * (lane - 1), kb, raw_full(s));
+            else if (lane <= BN / 32) ptx::tma_load_2d(st + Cfg::A_BYTES + (lane - 1) * 4096, &map_b, c0 + 32 * (lane - 1), kb, raw_full(s));
         }
         if (*abort_flag && lane == 0) {          // failure path: loads still in flight land before the CTA's memory goes away
             const unsigned long long t0 = global_ns();
@@ -161,15 +166,14 @@ product_tc_inline_kernel(const __grid_constant__ CUtensorMap map_a, const __grid
                 ok = wait_barrier(ready(s), (i / S) & 1, abort_flag, prm.status, (12 << 24) | (s << 16) | (tile & 0xFFFF));
                 if (!ok) break;
                 ptx::tc_fence_after_sync();
-                const uint32_t a_hi = base + s * Cfg::STAGE_BYTES, a_lo = a_hi + Cfg::A_BYTES;
-                const uint32_t b_hi = a_hi + 2 * Cfg::A_BYTES + Cfg::B_RAW_BYTES, b_lo = b_hi + Cfg::B_PLANE_BYTES;
+                const uint32_t a_hi = tmem_base + BN + s * Cfg::A_COLS, a_lo = a_hi + IBK;      // tensor-memory columns
+                const uint32_t b_hi = base + s * Cfg::STAGE_BYTES + Cfg::A_BYTES + Cfg::B_RAW_BYTES, b_lo = b_hi + Cfg::B_PLANE_BYTES;
 #pragma unroll
                 for (int ks = 0; ks < IBK / 8; ++ks) {
-                    const uint64_t da_hi = kmajor_desc128(a_hi, ks), da_lo = kmajor_desc128(a_lo, ks);
                     const uint64_t db_hi = kmajor_desc128(b_hi, ks), db_lo = kmajor_desc128(b_lo, ks);
-                    ptx::mma_tf32(tmem_base, da_lo, db_hi, idesc, accumulate);       // small terms first
-                    ptx::mma_tf32(tmem_base, da_hi, db_lo, idesc, 1);
-                    ptx::mma_tf32(tmem_base, da_hi, db_hi, idesc, 1);
+                    ptx::mma_tf32_a_tmem(tmem_base, a_lo + 8 * ks, db_hi, idesc, accumulate);   // small terms first
+                    ptx::mma_tf32_a_tmem(tmem_base, a_hi + 8 * ks, db_lo, idesc, 1);
+                    ptx::mma_tf32_a_tmem(tmem_base, a_hi + 8 * ks, db_hi, idesc, 1);
                     accumulate = 1;
                 }
                 ptx::mma_commit(empty(s));                   // the stage may be refilled once these MMAs have read it
@@ -184,7 +188,13 @@ product_tc_inline_kernel(const __grid_constant__ CUtensorMap map_a, const __grid
         __syncwarp();
     } else {
         // ------------------------------------------------------------------ transform (warps 2..9), then epilogue
-        const int tid2 = threadIdx.x - 64, w2 = warp - 2;
+        const int w2 = warp - 2;
+        // A: this thread owns row 32 q + lane of the tile (the tensor-memory lane its warp may write) and half of its 32 k
+        const int arow = (warp & 3) * 32 + lane, ahalf = w2 >> 2;
+        uint32_t a_src[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) a_src[u] = arow * 128 + (((4 * ahalf + u) ^ (arow & 7)) << 4);
+        const uint32_t a_dst = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + BN + 16 * ahalf;
         // where this lane's values of B go: task t of the warp is (box j, group c) = columns 32 j + 4 c .. + 3 of k-row `lane`;
         // value e of it lands in row n = 32 j + 4 c + e of the K-major tile, at k = lane (group lane / 4, word lane % 4)
         constexpr int TASKS = BN / 4 / XFORM_WARPS;
@@ -206,22 +216,28 @@ product_tc_inline_kernel(const __grid_constant__ CUtensorMap map_a, const __grid
             ok = __shfl_sync(0xffffffffu, ok, 0);
             if (!ok) break;
             uint8_t *const st = base_ptr + s * Cfg::STAGE_BYTES;
-            // A: 128 rows x 8 groups of 16 bytes, split where they lie (the swizzle is a permutation of the groups: offsets stay)
-            float4 av[1024 / XFORM_THREADS];
+            ptx::tc_fence_after_sync();                      // the MMAs that read this stage's columns of tensor memory are done
+            float4 av[4];
 #pragma unroll
-            for (int u = 0; u < 1024 / XFORM_THREADS; ++u) av[u] = *(reinterpret_cast<const float4 *>(st) + tid2 + XFORM_THREADS * u);
+            for (int u = 0; u < 4; ++u) av[u] = *reinterpret_cast<const float4 *>(st + a_src[u]);
             // B: box j holds k-rows 0..31 x columns 32 j .. 32 j + 31, group c of row k at group c ^ (k & 7).  Lane = k-row.
-            uint8_t *const braw = st + 2 * Cfg::A_BYTES, *const bhi = braw + Cfg::B_RAW_BYTES, *const blo = bhi + Cfg::B_PLANE_BYTES;
+            uint8_t *const braw = st + Cfg::A_BYTES, *const bhi = braw + Cfg::B_RAW_BYTES, *const blo = bhi + Cfg::B_PLANE_BYTES;
             float4 bv[TASKS];
 #pragma unroll
             for (int t = 0; t < TASKS; ++t) bv[t] = *reinterpret_cast<const float4 *>(braw + src_off[t]);
+            {
+                uint32_t hi16[16], lo16[16];
 #pragma unroll
-            for (int u = 0; u < 1024 / XFORM_THREADS; ++u) {
-                float4 *p = reinterpret_cast<float4 *>(st) + tid2 + XFORM_THREADS * u;
-                float4 hi, lo;
-                split4(av[u], hi, lo);
-                *p = hi;
-                *(p + Cfg::A_BYTES / 16) = lo;
+                for (int u = 0; u < 4; ++u) {
+                    float4 hi, lo;
+                    split4(av[u], hi, lo);
+                    hi16[4 * u] = __float_as_uint(hi.x); hi16[4 * u + 1] = __float_as_uint(hi.y);
+                    hi16[4 * u + 2] = __float_as_uint(hi.z); hi16[4 * u + 3] = __float_as_uint(hi.w);
+                    lo16[4 * u] = __float_as_uint(lo.x); lo16[4 * u + 1] = __float_as_uint(lo.y);
+                    lo16[4 * u + 2] = __float_as_uint(lo.z); lo16[4 * u + 3] = __float_as_uint(lo.w);
+                }
+                ptx::tmem_st_16cols(a_dst + s * Cfg::A_COLS, hi16);
+                ptx::tmem_st_16cols(a_dst + s * Cfg::A_COLS + IBK, lo16);
             }
 #pragma unroll
             for (int t = 0; t < TASKS; ++t) {
@@ -232,7 +248,9 @@ product_tc_inline_kernel(const __grid_constant__ CUtensorMap map_a, const __grid
                 *reinterpret_cast<float *>(bhi + dst_off[t][2]) = hi.z; *reinterpret_cast<float *>(blo + dst_off[t][2]) = lo.z;
                 *reinterpret_cast<float *>(bhi + dst_off[t][3]) = hi.w; *reinterpret_cast<float *>(blo + dst_off[t][3]) = lo.w;
             }
-            ptx::fence_proxy_async_smem();                   // the MMA reads these tiles through the asynchronous proxy
+            ptx::tmem_wait_st();
+            ptx::fence_proxy_async_smem();                   // the MMA reads B's tiles through the asynchronous proxy
+            ptx::tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(ready(s));
         }
@@ -284,7 +302,7 @@ product_tc_inline_kernel(const __grid_constant__ CUtensorMap map_a, const __grid
     ptx::tc_fence_before_sync();
     __syncthreads();
     ptx::tc_fence_after_sync();
-    if (warp == 1) ptx::tmem_dealloc(tmem_base, BN);
+    if (warp == 1) ptx::tmem_dealloc(tmem_base, Cfg::TMEM_COLS);
     if (split == 1) return;
 
     // ---- split contraction: CTA `rank` finishes its rows of the tile, adding the cluster's partial tiles in k order
@@ -331,9 +349,11 @@ cudaError_t launch_product_tc_inline(const ProductArgs &a, int32_t *status, cuda
     if (sm_count < 1) return cudaErrorInvalidDevice;
     const int tiles_m = (a.m + IBM - 1) / IBM;
     const int kblocks = (a.k + IBK - 1) / IBK;
-    // Tile width and k-slices per tile: the pair with the shortest critical path, counted in k-blocks of one CTA times what a k-block
-    // costs at that width (measured: about 0.9 us at 64 columns, 1.3 us at 128), over the waves the grid needs.  A cluster of s CTAs
-    // must sit in one GPC and every CTA takes a whole SM here, so far fewer than SMs / s clusters run at once: ask the runtime.
+    // Tile width and k-slices per tile: the pair with the shortest critical path.  A wave of CTAs costs its fixed part (set-up, epilogue:
+    // about 2 us at 64 columns, 2.5 us at 128), its k-blocks (measured: 0.66 us each at 64 columns, 0.9 us at 128) and, when the
+    // contraction is split, the cluster's reduction (1.5 us); the launch itself is the same for all.  A cluster of s CTAs must sit in
+    // one GPC and every CTA takes a whole SM here, so far fewer than SMs / s clusters run at once (148 / 74 / 33 / 15 on a B200): ask
+    // the runtime.
     int bn = 64, split = 1;
     double best = 1e300;
     for (int width : {64, 128}) {
@@ -371,7 +391,7 @@ cudaError_t launch_product_tc_inline(const ProductArgs &a, int32_t *status, cuda
             }
             if (fit < 1) continue;
             const long long waves = (tiles + fit - 1) / fit;
-            const double cost = (double)waves * ((kblocks + s - 1) / s) * (width == 128 ? 1.3 : 0.9) + (s > 1 ? 1.5 : 0.0);
+            const double cost = (double)waves * ((width == 128 ? 2.5 : 2.0) + ((kblocks + s - 1) / s) * (width == 128 ? 0.9 : 0.66) + (s > 1 ? 1.5 : 0.0));
             if (cost < best) { best = cost; bn = width; split = s; }
         }
     }
