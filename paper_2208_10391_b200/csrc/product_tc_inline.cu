@@ -47,18 +47,22 @@ constexpr int XFORM_WARPS = 8, XFORM_THREADS = 32 * XFORM_WARPS;
 
 template <int BN>
 struct InlineCfg {
-    static constexpr int STAGES = BN == 64 ? 5 : 3;
+    // Two rings.  RAW: what TMA delivers (the f32 tiles of A and B), free again as soon as the transform warps have read it, so
+    // that the loads run RAW stages ahead of the transform (a load takes about 1900 cycles, the transform of a k-block 800, its
+    // MMAs 770).  SPLIT: what the MMA reads (A's halves in tensor memory, B's in shared memory), free once its MMAs are done.
+    static constexpr int RAW = BN == 64 ? 5 : 4, SPLIT = BN == 64 ? 4 : 3;
     static constexpr int A_BYTES = IBM * IBK * 4;            // 16 KB: the raw tile of A
     static constexpr int B_RAW_BYTES = IBK * BN * 4;         // BN / 32 boxes of 32 k-rows x 32 columns
     static constexpr int B_PLANE_BYTES = BN * IBK * 4;       // K-major: BN rows of 32 k
-    static constexpr int STAGE_BYTES = A_BYTES + B_RAW_BYTES + 2 * B_PLANE_BYTES;
-    // tensor memory: the accumulator in columns [0, BN), then per stage 32 columns of A's hi half and 32 of its lo half
+    static constexpr int RAW_BYTES = A_BYTES + B_RAW_BYTES, SPLIT_BYTES = 2 * B_PLANE_BYTES;
+    static constexpr int RING_BYTES = RAW * RAW_BYTES + SPLIT * SPLIT_BYTES;
+    // tensor memory: the accumulator in columns [0, BN), then per SPLIT stage 32 columns of A's hi half and 32 of its lo half
     static constexpr int A_COLS = 2 * IBK, TMEM_COLS = 512;
-    static_assert(BN + STAGES * A_COLS <= TMEM_COLS, "tensor memory budget");
+    static_assert(BN + SPLIT * A_COLS <= TMEM_COLS, "tensor memory budget");
     static constexpr int LDP = BN + 4;                       // row length of the partial tile (floats)
-    static constexpr int NUM_BARRIERS = 3 * STAGES + 2;
-    static constexpr int SMEM_BYTES = 1024 + STAGES * STAGE_BYTES + 256;
-    static_assert(IBM * LDP * 4 <= STAGES * STAGE_BYTES, "the partial tile reuses the stages");
+    static constexpr int NUM_BARRIERS = 2 * RAW + 2 * SPLIT + 2;
+    static constexpr int SMEM_BYTES = 1024 + RING_BYTES + 256;
+    static_assert(IBM * LDP * 4 <= RING_BYTES, "the partial tile reuses the rings");
     static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
 };
 
@@ -89,17 +93,19 @@ template <int BN>
 __global__ void __launch_bounds__(ITHREADS, 1)
 product_tc_inline_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const InlineParams prm) {
     using Cfg = InlineCfg<BN>;
-    constexpr int S = Cfg::STAGES;
+    constexpr int R = Cfg::RAW, S = Cfg::SPLIT;
     extern __shared__ uint8_t smem_raw[];
     __shared__ int abort_word;
     allow_dependents();
     const uint32_t base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t *const base_ptr = smem_raw + (base - ptx::smem_u32(smem_raw));
-    const uint32_t bars = base + S * Cfg::STAGE_BYTES;
-    auto raw_full = [&](int s) { return bars + 8 * s; };
-    auto ready = [&](int s) { return bars + 8 * (S + s); };
-    auto empty = [&](int s) { return bars + 8 * (2 * S + s); };
-    const uint32_t acc_full = bars + 8 * (3 * S), drain = bars + 8 * (3 * S + 1), tmem_slot = bars + 8 * Cfg::NUM_BARRIERS;
+    const uint32_t split_base = base + R * Cfg::RAW_BYTES;
+    const uint32_t bars = base + Cfg::RING_BYTES;
+    auto raw_full = [&](int s) { return bars + 8 * s; };                    // TMA has delivered raw stage s
+    auto raw_empty = [&](int s) { return bars + 8 * (R + s); };             // the transform warps have read it
+    auto ready = [&](int s) { return bars + 8 * (2 * R + s); };             // the transform warps have filled split stage s
+    auto empty = [&](int s) { return bars + 8 * (2 * R + S + s); };         // its MMAs are done
+    const uint32_t acc_full = bars + 8 * (2 * R + 2 * S), drain = acc_full + 8, tmem_slot = bars + 8 * Cfg::NUM_BARRIERS;
     volatile int *abort_flag = &abort_word;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -118,7 +124,8 @@ product_tc_inline_kernel(const __grid_constant__ CUtensorMap map_a, const __grid
 
     if (threadIdx.x == 0) {
         abort_word = 0;
-        for (int s = 0; s < S; ++s) { ptx::mbar_init(raw_full(s), 1); ptx::mbar_init(ready(s), XFORM_WARPS); ptx::mbar_init(empty(s), 1); }
+        for (int s = 0; s < R; ++s) { ptx::mbar_init(raw_full(s), 1); ptx::mbar_init(raw_empty(s), XFORM_WARPS); }
+        for (int s = 0; s < S; ++s) { ptx::mbar_init(ready(s), XFORM_WARPS); ptx::mbar_init(empty(s), 1); }
         ptx::mbar_init(acc_full, 1);
         ptx::mbar_init(drain, 1);
         ptx::fence_barrier_init();
@@ -140,14 +147,14 @@ product_tc_inline_kernel(const __grid_constant__ CUtensorMap map_a, const __grid
         // ------------------------------------------------------------------ TMA producer
         bool ok = true;
         for (int i = 0; i < nk && ok; ++i) {
-            const int s = i % S;
-            if (lane == 0) ok = wait_barrier(empty(s), ((i / S) & 1) ^ 1, abort_flag, prm.status, (11 << 24) | (s << 16) | (tile & 0xFFFF));
+            const int s = i % R;
+            if (lane == 0) ok = wait_barrier(raw_empty(s), ((i / R) & 1) ^ 1, abort_flag, prm.status, (11 << 24) | (s << 16) | (tile & 0xFFFF));
             ok = __shfl_sync(0xffffffffu, ok, 0);
             if (!ok) break;
             if (lane == 0) ptx::mbar_arrive_expect_tx(raw_full(s), Cfg::A_BYTES + Cfg::B_RAW_BYTES);
             __syncwarp();
             const int kb = klo + (kb0 + i) * IBK;
-            const uint32_t st = base + s * Cfg::STAGE_BYTES;
+            const uint32_t st = base + s * Cfg::RAW_BYTES;
             if (lane == 0) ptx::tma_load_2d(st, &map_a, kb, r0, raw_full(s));
             else if (lane <= BN / 32) ptx::tma_load_2d(st + Cfg::A_BYTES + (lane - 1) * 4096, &map_b, c0 + 32 * (lane - 1), kb, raw_full(s));
         }
@@ -161,19 +168,24 @@ product_tc_inline_kernel(const __grid_constant__ CUtensorMap map_a, const __grid
             constexpr uint32_t idesc = ptx::instr_desc_tf32(IBM, BN, 0, 0);
             uint32_t accumulate = 0;
             bool ok = true;
-            for (int i = 0; i < nk; ++i) {
+            // The wait for the NEXT k-block's operands sits before the last MMAs of this one: while the issuer is in it the tensor
+            // pipe still has queued work, so the pipe does not run dry between k-blocks.
+            const uint64_t desc0 = kmajor_desc128(split_base, 0);            // descriptors differ only in the address field
+            if (nk > 0) ok = wait_barrier(ready(0), 0, abort_flag, prm.status, (12 << 24) | (tile & 0xFFFF));
+            for (int i = 0; i < nk && ok; ++i) {
                 const int s = i % S;
-                ok = wait_barrier(ready(s), (i / S) & 1, abort_flag, prm.status, (12 << 24) | (s << 16) | (tile & 0xFFFF));
-                if (!ok) break;
                 ptx::tc_fence_after_sync();
                 const uint32_t a_hi = tmem_base + BN + s * Cfg::A_COLS, a_lo = a_hi + IBK;      // tensor-memory columns
-                const uint32_t b_hi = base + s * Cfg::STAGE_BYTES + Cfg::A_BYTES + Cfg::B_RAW_BYTES, b_lo = b_hi + Cfg::B_PLANE_BYTES;
+                const uint64_t db_hi = desc0 + (uint64_t)((s * Cfg::SPLIT_BYTES) >> 4), db_lo = db_hi + (Cfg::B_PLANE_BYTES >> 4);
 #pragma unroll
                 for (int ks = 0; ks < IBK / 8; ++ks) {
-                    const uint64_t db_hi = kmajor_desc128(b_hi, ks), db_lo = kmajor_desc128(b_lo, ks);
-                    ptx::mma_tf32_a_tmem(tmem_base, a_lo + 8 * ks, db_hi, idesc, accumulate);   // small terms first
-                    ptx::mma_tf32_a_tmem(tmem_base, a_hi + 8 * ks, db_lo, idesc, 1);
-                    ptx::mma_tf32_a_tmem(tmem_base, a_hi + 8 * ks, db_hi, idesc, 1);
+                    if (ks == IBK / 8 - 1 && i + 1 < nk) {
+                        const int sn = (i + 1) % S;
+                        ok = wait_barrier(ready(sn), ((i + 1) / S) & 1, abort_flag, prm.status, (12 << 24) | (sn << 16) | (tile & 0xFFFF));
+                    }
+                    ptx::mma_tf32_a_tmem(tmem_base, a_lo + 8 * ks, db_hi + 2 * ks, idesc, accumulate);   // small terms first
+                    ptx::mma_tf32_a_tmem(tmem_base, a_hi + 8 * ks, db_lo + 2 * ks, idesc, 1);
+                    ptx::mma_tf32_a_tmem(tmem_base, a_hi + 8 * ks, db_hi + 2 * ks, idesc, 1);
                     accumulate = 1;
                 }
                 ptx::mma_commit(empty(s));                   // the stage may be refilled once these MMAs have read it
@@ -210,18 +222,21 @@ product_tc_inline_kernel(const __grid_constant__ CUtensorMap map_a, const __grid
             }
         }
         bool ok = true;
+        uint8_t *const split_ptr = base_ptr + R * Cfg::RAW_BYTES;
         for (int i = 0; i < nk && ok; ++i) {
-            const int s = i % S;
-            if (lane == 0) ok = wait_barrier(raw_full(s), (i / S) & 1, abort_flag, prm.status, (13 << 24) | (s << 16) | (tile & 0xFFFF));
+            const int rs = i % R, s = i % S;
+            if (lane == 0)
+                ok = wait_barrier(raw_full(rs), (i / R) & 1, abort_flag, prm.status, (13 << 24) | (rs << 16) | (tile & 0xFFFF)) &&
+                     wait_barrier(empty(s), ((i / S) & 1) ^ 1, abort_flag, prm.status, (15 << 24) | (s << 16) | (tile & 0xFFFF));
             ok = __shfl_sync(0xffffffffu, ok, 0);
             if (!ok) break;
-            uint8_t *const st = base_ptr + s * Cfg::STAGE_BYTES;
-            ptx::tc_fence_after_sync();                      // the MMAs that read this stage's columns of tensor memory are done
+            uint8_t *const st = base_ptr + rs * Cfg::RAW_BYTES;
+            ptx::tc_fence_after_sync();                      // the MMAs that read this split stage (tensor memory and B's tiles) are done
             float4 av[4];
 #pragma unroll
             for (int u = 0; u < 4; ++u) av[u] = *reinterpret_cast<const float4 *>(st + a_src[u]);
             // B: box j holds k-rows 0..31 x columns 32 j .. 32 j + 31, group c of row k at group c ^ (k & 7).  Lane = k-row.
-            uint8_t *const braw = st + Cfg::A_BYTES, *const bhi = braw + Cfg::B_RAW_BYTES, *const blo = bhi + Cfg::B_PLANE_BYTES;
+            uint8_t *const braw = st + Cfg::A_BYTES, *const bhi = split_ptr + s * Cfg::SPLIT_BYTES, *const blo = bhi + Cfg::B_PLANE_BYTES;
             float4 bv[TASKS];
 #pragma unroll
             for (int t = 0; t < TASKS; ++t) bv[t] = *reinterpret_cast<const float4 *>(braw + src_off[t]);
@@ -252,7 +267,7 @@ product_tc_inline_kernel(const __grid_constant__ CUtensorMap map_a, const __grid
             ptx::fence_proxy_async_smem();                   // the MMA reads B's tiles through the asynchronous proxy
             ptx::tc_fence_before_sync();
             __syncwarp();
-            if (lane == 0) ptx::mbar_arrive(ready(s));
+            if (lane == 0) { ptx::mbar_arrive(ready(s)); ptx::mbar_arrive(raw_empty(rs)); }
         }
         // ---- epilogue: this warp reads TMEM lanes 32 q .. 32 q + 31 = rows of the tile; the two warps of a quarter share the columns
         const int q = warp & 3, row = q * 32 + lane, r = r0 + row, half = w2 >> 2;
