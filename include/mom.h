@@ -103,9 +103,11 @@ typedef enum { MOM_F32 = 0 } mom_dtype_t;
  *       dimensions TMA can address (multiples of 4 elements) run on the tcgen05 kernel that takes its operands as
  *       hi / lo planes (a pre-pass writes them; TMA, tensor memory, persistent CTAs); products of stored
  *       (untransposed) operands with a result of at least 65536 entries and 6 * 10^7 <= m*n*k < 10^9, or
- *       m*n*k < 4 * 10^9 with at most 148 result tiles of 128 x 128, run on the tcgen05 kernel that reads the
+ *       m*n*k < 4 * 10^9 with at most 148 result tiles of 128 x 128, or (an equation of one product only)
+ *       m*n*k < 10^10 with at most 74 result tiles of 256 x 256 (CTA pairs), run on the tcgen05 kernel that reads the
  *       operands as stored and splits them on the way into shared and tensor memory (one launch); everything
- *       else runs on the warp-level kernel (mma.sync on the operands as stored, one launch).
+ *       else runs on the warp-level kernel (mma.sync on the operands as stored, one launch).  A plan with packed
+ *       operands or a packed result keeps its large products on the first kernel, which addresses the containers in place.
  *   MOM_VARIANT_FFMA: plain f32 fused multiply-add on CUDA cores.
  *   MOM_VARIANT_3XTF32_FORCE: every TMA-addressable product runs on the tcgen05 kernel, the others on
  *       the FFMA kernel; meant for testing the tcgen05 kernel on small shapes.

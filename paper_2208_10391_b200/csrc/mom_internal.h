@@ -32,8 +32,11 @@ constexpr size_t WS_ALIGN = 256;
 // 900 x 1200 x 100 16.6 / 27.1 / 10.9, 4096 x 256 x 64 10.4 / 22.7 / 7.6, 256 x 2048 x 64 10.5 / 23.7 / 10.7, 128 x 4096 x 128 14.8 / 26.8 / 15.5).
 // Up to INLINE_SMALL_WORK it is taken whatever the shape; up to INLINE_MAX_WORK while its 128 x 128 tiles fit one wave of CTAs
 // (a second wave repeats the whole of the first: 1792^3 93 us against 1536^3 48 us).
-constexpr double INLINE_MIN_WORK = 6.0e7, INLINE_SMALL_WORK = 1.0e9, INLINE_MAX_WORK = 4.0e9, INLINE_MIN_OUTPUT = 65536.0;
-constexpr int64_t INLINE_WAVE_TILES = 148;
+// Beyond that, up to INLINE_PAIR_MAX_WORK while its CTA pairs' 256 x 256 tiles fit one wave (1792^3 78.7 against the plane
+// kernel's 81.3, 2048^3 84.5 against 92.7, 2048 x 512 x 2048 31.3 against 35.9; 2560^3, 100 pairs, 204 against 187).
+constexpr double INLINE_MIN_WORK = 6.0e7, INLINE_SMALL_WORK = 1.0e9, INLINE_MAX_WORK = 4.0e9, INLINE_PAIR_MAX_WORK = 1.0e10,
+                 INLINE_MIN_OUTPUT = 65536.0;
+constexpr int64_t INLINE_WAVE_TILES = 148, INLINE_WAVE_PAIRS = 74;
 // Products below this many multiplications count as small when independent subtrees are put side by side on two streams.
 constexpr double SIDE_BY_SIDE_MAX_WORK = 1.0e9;
 

@@ -228,7 +228,8 @@ struct SumIn { std::vector<std::vector<FactorIn>> chains; };
 
 static mom_status_t plan_sums(const std::vector<mom_matrix_desc_t> &slots, const std::vector<SumIn> &sums_in,
                               const int32_t *slot_names, const mom_matrix_desc_t *stored_add,
-                              const int32_t *add_transposed, int32_t n_add, mom_variant_t variant, mom_plan_t **out_plan) {
+                              const int32_t *add_transposed, int32_t n_add, mom_variant_t variant, mom_plan_t **out_plan,
+                              bool packed_storage = false) {
     if (!out_plan || sums_in.empty() || n_add < 0 || (n_add > 0 && !stored_add)) return MOM_ERR_INVALID_ARG;
     if ((int)variant < 0 || (int)variant > 4) return MOM_ERR_INVALID_ARG;
     int64_t total = 0;
@@ -566,13 +567,20 @@ static mom_status_t plan_sums(const std::vector<mom_matrix_desc_t> &slots, const
                                                                 mom::kernel_property(st.pub.lhs_property), mom::kernel_property(st.pub.rhs_property));
             // ... and it pays between the two (measured, see the constants): from about 400^3 on it beats the warp-level kernel, and
             // its single launch beats the plane kernel's two up to 1000^3 whatever the shape and up to about 1600^3 while its
-            // 128 x 128 tiles fit one wave of CTAs; a result of fewer than four 128 x 128 tiles would leave each CTA a long
+            // 128 x 128 tiles fit one wave of CTAs, and to 2000^3 while its CTA pairs' 256 x 256 tiles do; a result of fewer than four 128 x 128 tiles would leave each CTA a long
             // contraction even when split over a cluster, and the warp-level kernel is quicker there
             const double work = (double)m * (double)n * (double)k;
             const bool one_wave = ((m + 127) / 128) * ((n + 127) / 128) <= mom::INLINE_WAVE_TILES;
+            // (only for an equation of one product: in a chain the plane kernel's steps hand each other their planes, which
+            // saves the split passes that make it the slower one here: L*A*U*B at 2048 249 us against 263 us mixed)
+            const bool one_wave_of_pairs = ns == 1 && ((m + 255) / 256) * ((n + 255) / 256) <= mom::INLINE_WAVE_PAIRS;
             const bool inline_pays = work >= mom::INLINE_MIN_WORK && (double)m * (double)n >= mom::INLINE_MIN_OUTPUT &&
-                                     (work < mom::INLINE_SMALL_WORK || (work < mom::INLINE_MAX_WORK && one_wave));
+                                     (work < mom::INLINE_SMALL_WORK || (work < mom::INLINE_MAX_WORK && one_wave) ||
+                                      (work < mom::INLINE_PAIR_MAX_WORK && one_wave_of_pairs));
             if (st.pub.kind == MOM_KIND_SCALE) st.pub.uses_tensor_cores = 0;       // a Diagonal operand: one scaling pass, bound by HBM
+            // operands or a result in packed storage: the plane kernel addresses the containers in place, the one-launch
+            // kernel would need them unpacked first
+            else if (variant == MOM_VARIANT_3XTF32 && packed_storage && addressable && large) st.pub.uses_tensor_cores = 1;
             else if (variant == MOM_VARIANT_3XTF32) st.pub.uses_tensor_cores = inline_ok && inline_pays ? 3 : addressable && large ? 1 : 2;
             else if (variant == MOM_VARIANT_3XTF32_FORCE) st.pub.uses_tensor_cores = addressable ? 1 : 0;
             else if (variant == MOM_VARIANT_3XTF32_WARP) st.pub.uses_tensor_cores = 2;
@@ -809,7 +817,8 @@ mom_status_t mom_equation_plan(const mom_matrix_desc_t *chain, int32_t n_chain,
 // one sum whose factors are the caller's array entries in order
 static mom_status_t plan_flat(const mom_matrix_desc_t *stored, const int32_t *transposed, const int32_t *names,
                               const int32_t *chain_len, int32_t n_chains, const mom_matrix_desc_t *stored_add,
-                              const int32_t *add_transposed, int32_t n_add, mom_variant_t variant, mom_plan_t **out_plan) {
+                              const int32_t *add_transposed, int32_t n_add, mom_variant_t variant, mom_plan_t **out_plan,
+                              bool packed_storage = false) {
     if (!out_plan || !stored || !chain_len || n_chains < 1) return MOM_ERR_INVALID_ARG;
     try {
         std::vector<SumIn> sums(1);
@@ -825,7 +834,7 @@ static mom_status_t plan_flat(const mom_matrix_desc_t *stored, const int32_t *tr
             sums[0].chains.push_back(std::move(chain));
         }
         std::vector<mom_matrix_desc_t> slots(stored, stored + total);
-        return plan_sums(slots, sums, names, stored_add, add_transposed, n_add, variant, out_plan);
+        return plan_sums(slots, sums, names, stored_add, add_transposed, n_add, variant, out_plan, packed_storage);
     } catch (const std::bad_alloc &) {
         return MOM_ERR_ALLOC;
     }
@@ -879,7 +888,9 @@ mom_status_t mom_equation_plan_stored(const mom_matrix_desc_t *chain, const int3
                                       mom_variant_t variant, mom_plan_t **out_plan) {
     if (result_storage != MOM_STORAGE_DENSE && result_storage != MOM_STORAGE_PACKED) return MOM_ERR_INVALID_ARG;
     mom_plan_t *p = nullptr;
-    const mom_status_t st = mom_equation_plan_transposed(chain, chain_transposed, n_chain, add_terms, add_transposed, n_add, variant, &p);
+    bool any_packed = result_storage == MOM_STORAGE_PACKED;
+    for (int i = 0; chain_storage && i < n_chain; ++i) any_packed |= chain_storage[i] == MOM_STORAGE_PACKED;
+    const mom_status_t st = plan_flat(chain, chain_transposed, nullptr, &n_chain, 1, add_terms, add_transposed, n_add, variant, &p, any_packed);
     if (st != MOM_OK) return st;
     auto fail = [&](mom_status_t e) { mom_plan_destroy(p); return e; };
     try {

@@ -348,6 +348,252 @@ product_tc_inline_kernel(const __grid_constant__ CUtensorMap map_a, const __grid
     cluster.sync();                                          // nobody leaves while a peer may still read its tile
 }
 
+
+// ---------------------------------------------------------------------------------------------
+// CTA-pair variant (cta_group::2): the two CTAs of a cluster share one 256 x (2 BNH) tile of the result.  Each CTA loads,
+// splits and keeps its own 128 rows of A (in its tensor memory) and only its own BNH columns of B (K-major hi / lo tiles in
+// its shared memory); the pair's tensor cores exchange the B halves, so per flop a CTA moves half the B bytes through its
+// shared memory and the MMAs (M 256, N = 2 BNH), not shared memory, bound the mainloop.  The leader (cluster rank 0) issues
+// every MMA; the transform warps of BOTH CTAs arrive on the leader's "ready" barrier (the peer's over the cluster, releasing
+// what they wrote), tcgen05.commit with a CTA mask frees the split stage in both CTAs and publishes the accumulator to both
+// epilogues.  No split of the contraction here: the variant is chosen when the pairs fill most of the machine.
+// ---------------------------------------------------------------------------------------------
+template <int BNH>
+struct PairCfg {
+    static constexpr int BN2 = 2 * BNH;                      // columns of the pair's tile = N of the MMA
+    static constexpr int RAW = BNH == 64 ? 5 : 4, SPLIT = BNH == 64 ? 4 : 3;
+    static constexpr int A_BYTES = IBM * IBK * 4;
+    static constexpr int B_RAW_BYTES = IBK * BNH * 4;
+    static constexpr int B_PLANE_BYTES = BNH * IBK * 4;
+    static constexpr int RAW_BYTES = A_BYTES + B_RAW_BYTES, SPLIT_BYTES = 2 * B_PLANE_BYTES;
+    static constexpr int RING_BYTES = RAW * RAW_BYTES + SPLIT * SPLIT_BYTES;
+    static constexpr int A_COLS = 2 * IBK, TMEM_COLS = 512;
+    static_assert(BN2 + SPLIT * A_COLS <= TMEM_COLS, "tensor memory budget");
+    static constexpr int NUM_BARRIERS = 2 * RAW + 2 * SPLIT + 2;
+    static constexpr int SMEM_BYTES = 1024 + RING_BYTES + 256;
+    static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
+};
+
+template <int BNH>
+__global__ void __launch_bounds__(ITHREADS, 1)
+product_tc_inline_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const InlineParams prm) {
+    using Cfg = PairCfg<BNH>;
+    constexpr int R = Cfg::RAW, S = Cfg::SPLIT, BN2 = Cfg::BN2;
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ int abort_word;
+    allow_dependents();
+    const uint32_t base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t *const base_ptr = smem_raw + (base - ptx::smem_u32(smem_raw));
+    const uint32_t split_base = base + R * Cfg::RAW_BYTES;
+    const uint32_t bars = base + Cfg::RING_BYTES;
+    auto raw_full = [&](int s) { return bars + 8 * s; };                    // own TMA has delivered raw stage s
+    auto raw_empty = [&](int s) { return bars + 8 * (R + s); };             // own transform warps have read it
+    auto ready = [&](int s) { return bars + 8 * (2 * R + s); };             // leader only: both CTAs' transform warps have filled split stage s
+    auto empty = [&](int s) { return bars + 8 * (2 * R + S + s); };         // the pair's MMAs on split stage s are done
+    const uint32_t acc_full = bars + 8 * (2 * R + 2 * S), drain = acc_full + 8, tmem_slot = bars + 8 * Cfg::NUM_BARRIERS;
+    volatile int *abort_flag = &abort_word;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = ptx::cluster_cta_rank();                           // 0 = leader
+    const int tile = blockIdx.x >> 1;
+    const int r0 = (tile / prm.tiles_n) * (2 * IBM), c0 = (tile % prm.tiles_n) * BN2;      // the pair's tile
+    const int my_r0 = r0 + (int)rank * IBM, my_c0 = c0 + (int)rank * BNH;                  // this CTA's rows of A, columns of B
+
+    int klo, khi;                                                            // the same in both CTAs
+    tile_k_range(prm.pa, prm.pb, r0, min(r0 + 2 * IBM, prm.m), c0, min(c0 + BN2, prm.n), prm.k, &klo, &khi);
+    klo &= ~(IBK - 1);
+    const int nk = klo < khi ? (khi - klo + IBK - 1) / IBK : 0;
+
+    if (threadIdx.x == 0) {
+        abort_word = 0;
+        for (int s = 0; s < R; ++s) { ptx::mbar_init(raw_full(s), 1); ptx::mbar_init(raw_empty(s), XFORM_WARPS); }
+        for (int s = 0; s < S; ++s) { ptx::mbar_init(ready(s), 2 * XFORM_WARPS); ptx::mbar_init(empty(s), 1); }
+        ptx::mbar_init(acc_full, 1);
+        ptx::mbar_init(drain, 1);
+        ptx::fence_barrier_init();
+    }
+    if (warp == 1) {
+        ptx::tmem_alloc_pair(tmem_slot, Cfg::TMEM_COLS);
+        ptx::tmem_relinquish_pair();
+    }
+    ptx::tc_fence_before_sync();
+    ptx::cluster_sync();                         // the peer's barriers exist before anything signals them
+    ptx::tc_fence_after_sync();
+    uint32_t tmem_base;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(tmem_base) : "r"(tmem_slot));
+    grid_dependency_wait();
+    asm volatile("fence.proxy.async;" ::: "memory");
+
+    bool acc_ok = nk > 0;
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer (both CTAs, own barriers)
+        bool ok = true;
+        for (int i = 0; i < nk && ok; ++i) {
+            const int s = i % R;
+            if (lane == 0) ok = wait_barrier(raw_empty(s), ((i / R) & 1) ^ 1, abort_flag, prm.status, (21 << 24) | (s << 16) | (tile & 0xFFFF));
+            ok = __shfl_sync(0xffffffffu, ok, 0);
+            if (!ok) break;
+            if (lane == 0) ptx::mbar_arrive_expect_tx(raw_full(s), Cfg::RAW_BYTES);
+            __syncwarp();
+            const int kb = klo + i * IBK;
+            const uint32_t st = base + s * Cfg::RAW_BYTES;
+            if (lane == 0) ptx::tma_load_2d(st, &map_a, kb, my_r0, raw_full(s));
+            else if (lane <= BNH / 32) ptx::tma_load_2d(st + Cfg::A_BYTES + (lane - 1) * 4096, &map_b, my_c0 + 32 * (lane - 1), kb, raw_full(s));
+        }
+        if (*abort_flag && lane == 0) {
+            const unsigned long long t0 = global_ns();
+            while (global_ns() - t0 < 200000ull) { }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer (leader CTA, one thread)
+        if (lane == 0 && rank == 0) {
+            constexpr uint32_t idesc = ptx::instr_desc_tf32(2 * IBM, BN2, 0, 0);
+            uint32_t accumulate = 0;
+            bool ok = true;
+            const uint64_t desc0 = kmajor_desc128(split_base, 0);
+            if (nk > 0) ok = wait_barrier<true>(ready(0), 0, abort_flag, prm.status, (22 << 24) | (tile & 0xFFFF));
+            for (int i = 0; i < nk && ok; ++i) {
+                const int s = i % S;
+                ptx::tc_fence_after_sync();
+                const uint32_t a_hi = tmem_base + BN2 + s * Cfg::A_COLS, a_lo = a_hi + IBK;
+                const uint64_t db_hi = desc0 + (uint64_t)((s * Cfg::SPLIT_BYTES) >> 4), db_lo = db_hi + (Cfg::B_PLANE_BYTES >> 4);
+#pragma unroll
+                for (int ks = 0; ks < IBK / 8; ++ks) {
+                    if (ks == IBK / 8 - 1 && i + 1 < nk) {
+                        const int sn = (i + 1) % S;
+                        ok = wait_barrier<true>(ready(sn), ((i + 1) / S) & 1, abort_flag, prm.status, (22 << 24) | (sn << 16) | (tile & 0xFFFF));
+                    }
+                    ptx::mma_tf32_pair_a_tmem(tmem_base, a_lo + 8 * ks, db_hi + 2 * ks, idesc, accumulate);
+                    ptx::mma_tf32_pair_a_tmem(tmem_base, a_hi + 8 * ks, db_lo + 2 * ks, idesc, 1);
+                    ptx::mma_tf32_pair_a_tmem(tmem_base, a_hi + 8 * ks, db_hi + 2 * ks, idesc, 1);
+                    accumulate = 1;
+                }
+                ptx::mma_commit_pair(empty(s), 3);           // both CTAs may refill this split stage
+            }
+            if (ok && nk > 0) ptx::mma_commit_pair(acc_full, 3);
+            if (*abort_flag) {
+                ptx::mma_commit_pair(drain, 1);
+                for (uint32_t i = 0; i < (1u << 20); ++i)
+                    if (ptx::mbar_try_wait(drain, 0)) break;
+            }
+        }
+        __syncwarp();
+    } else {
+        // ------------------------------------------------------------------ transform (warps 2..9, both CTAs), then epilogue
+        const int w2 = warp - 2;
+        const int arow = (warp & 3) * 32 + lane, ahalf = w2 >> 2;
+        uint32_t a_src[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) a_src[u] = arow * 128 + (((4 * ahalf + u) ^ (arow & 7)) << 4);
+        const uint32_t a_dst = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + BN2 + 16 * ahalf;
+        constexpr int TASKS = BNH / 4 / XFORM_WARPS;
+        uint32_t src_off[TASKS], dst_off[TASKS][4];
+#pragma unroll
+        for (int t = 0; t < TASKS; ++t) {
+            const int task = w2 + XFORM_WARPS * t, j = task >> 3, c = task & 7;
+            src_off[t] = j * 4096 + lane * 128 + ((c ^ (lane & 7)) << 4);
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const int n = 32 * j + 4 * c + e;
+                dst_off[t][e] = n * 128 + ((((uint32_t)lane >> 2) ^ (n & 7)) << 4) + ((lane & 3) << 2);
+            }
+        }
+        bool ok = true;
+        uint8_t *const split_ptr = base_ptr + R * Cfg::RAW_BYTES;
+        for (int i = 0; i < nk && ok; ++i) {
+            const int rs = i % R, s = i % S;
+            if (lane == 0)
+                ok = wait_barrier(raw_full(rs), (i / R) & 1, abort_flag, prm.status, (23 << 24) | (rs << 16) | (tile & 0xFFFF)) &&
+                     wait_barrier(empty(s), ((i / S) & 1) ^ 1, abort_flag, prm.status, (25 << 24) | (s << 16) | (tile & 0xFFFF));
+            ok = __shfl_sync(0xffffffffu, ok, 0);
+            if (!ok) break;
+            uint8_t *const st = base_ptr + rs * Cfg::RAW_BYTES;
+            ptx::tc_fence_after_sync();
+            float4 av[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) av[u] = *reinterpret_cast<const float4 *>(st + a_src[u]);
+            uint8_t *const braw = st + Cfg::A_BYTES, *const bhi = split_ptr + s * Cfg::SPLIT_BYTES, *const blo = bhi + Cfg::B_PLANE_BYTES;
+            float4 bv[TASKS];
+#pragma unroll
+            for (int t = 0; t < TASKS; ++t) bv[t] = *reinterpret_cast<const float4 *>(braw + src_off[t]);
+            {
+                uint32_t hi16[16], lo16[16];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    float4 hi, lo;
+                    split4(av[u], hi, lo);
+                    hi16[4 * u] = __float_as_uint(hi.x); hi16[4 * u + 1] = __float_as_uint(hi.y);
+                    hi16[4 * u + 2] = __float_as_uint(hi.z); hi16[4 * u + 3] = __float_as_uint(hi.w);
+                    lo16[4 * u] = __float_as_uint(lo.x); lo16[4 * u + 1] = __float_as_uint(lo.y);
+                    lo16[4 * u + 2] = __float_as_uint(lo.z); lo16[4 * u + 3] = __float_as_uint(lo.w);
+                }
+                ptx::tmem_st_16cols(a_dst + s * Cfg::A_COLS, hi16);
+                ptx::tmem_st_16cols(a_dst + s * Cfg::A_COLS + IBK, lo16);
+            }
+#pragma unroll
+            for (int t = 0; t < TASKS; ++t) {
+                float4 hi, lo;
+                split4(bv[t], hi, lo);
+                *reinterpret_cast<float *>(bhi + dst_off[t][0]) = hi.x; *reinterpret_cast<float *>(blo + dst_off[t][0]) = lo.x;
+                *reinterpret_cast<float *>(bhi + dst_off[t][1]) = hi.y; *reinterpret_cast<float *>(blo + dst_off[t][1]) = lo.y;
+                *reinterpret_cast<float *>(bhi + dst_off[t][2]) = hi.z; *reinterpret_cast<float *>(blo + dst_off[t][2]) = lo.z;
+                *reinterpret_cast<float *>(bhi + dst_off[t][3]) = hi.w; *reinterpret_cast<float *>(blo + dst_off[t][3]) = lo.w;
+            }
+            ptx::tmem_wait_st();
+            ptx::fence_proxy_async_smem();
+            ptx::tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) {
+                ptx::mbar_arrive_cluster(ptx::map_to_cta(ready(s), 0));      // the leader's barrier, from either CTA
+                ptx::mbar_arrive(raw_empty(rs));
+            }
+        }
+        // ---- epilogue: this CTA's 128 rows of the accumulator
+        const int q = warp & 3, row = q * 32 + lane, r = my_r0 + row, half = w2 >> 2;
+        if (nk > 0 && ok) {
+            if (lane == 0) ok = wait_barrier(acc_full, 0, abort_flag, prm.status, (24 << 24) | (tile & 0xFFFF));
+            ok = __shfl_sync(0xffffffffu, ok, 0);
+            ptx::tc_fence_after_sync();
+        }
+        acc_ok = nk > 0 && ok;
+        const bool vec = (reinterpret_cast<uintptr_t>(prm.C) & 15) == 0 && (prm.n & 3) == 0;
+#pragma unroll 1
+        for (int c = half; c < BN2 / 32; c += 2) {
+            const int col0 = c0 + 32 * c;
+            if (col0 >= prm.n) break;
+            float v[32];
+            if (acc_ok) {
+                ptx::tmem_ld_32cols(tmem_base + c * 32 + ((uint32_t)(q * 32) << 16), v);
+            } else {
+#pragma unroll
+                for (int j = 0; j < 32; ++j) v[j] = 0.0f;
+            }
+            if (r < prm.m) {
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const int cc = col0 + 4 * j;
+                    if (cc >= prm.n) break;
+                    float w[4] = {v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]};
+                    finish_row4(w, prm.add, 0, r, cc, prm.n, prm.n, prm.pout, vec);
+                    float *dst = prm.C + (long long)r * prm.n + cc;
+                    if (vec && cc + 3 < prm.n) {
+                        *reinterpret_cast<float4 *>(dst) = make_float4(w[0], w[1], w[2], w[3]);
+                    } else {
+#pragma unroll
+                        for (int e = 0; e < 4; ++e)
+                            if (cc + e < prm.n) dst[e] = w[e];
+                    }
+                }
+            }
+        }
+    }
+
+    ptx::tc_fence_before_sync();
+    ptx::cluster_sync();                                     // nobody leaves while the peer may still signal it or read its B tiles
+    ptx::tc_fence_after_sync();
+    if (warp == 1) ptx::tmem_dealloc_pair(tmem_base, Cfg::TMEM_COLS);
+}
+
 }  // namespace
 
 bool product_tc_inline_takes(int64_t m, int64_t n, int64_t k, int lhs_transposed, int rhs_transposed, int pa, int pb) {
@@ -410,8 +656,46 @@ cudaError_t launch_product_tc_inline(const ProductArgs &a, int32_t *status, cuda
             if (cost < best) { best = cost; bn = width; split = s; }
         }
     }
-    const int tiles_n = (a.n + bn - 1) / bn;
-    const long long tiles = (long long)tiles_m * tiles_n;
+    // CTA pairs (256 x 256 tiles, no split of the contraction): a k-block costs a pair about 1.2 us (its MMAs with A from tensor
+    // memory: 12 x 170 cycles) for four times the result a single CTA's 0.9 us pays for; it wins when the pairs fill one wave
+    // where single CTAs would need two.  (Pairs on 256 x 128 tiles were measured too: their MMAs take as long as the 256-wide
+    // ones, so they never win.)
+    int pair_bnh = 0;
+    for (int bnh : {128}) {
+        const long long pairs = (long long)((a.m + 2 * IBM - 1) / (2 * IBM)) * ((a.n + 2 * bnh - 1) / (2 * bnh));
+        if (pairs * 2 > (1ll << 30)) continue;
+        int fit = sm_count / 2;
+        {
+            std::lock_guard<std::mutex> lock(device_info_mutex());
+            DeviceInfo *info = current_device_info();
+            if (!info) return cudaErrorInvalidDevice;
+            int &known = info->inline_pair_clusters[bnh == 128];
+            if (known == 0) {
+                known = -1;
+                cudaLaunchConfig_t probe = {};
+                probe.gridDim = dim3((unsigned)(2 * sm_count));
+                probe.blockDim = dim3(ITHREADS);
+                probe.dynamicSmemBytes = PairCfg<128>::SMEM_BYTES;
+                cudaLaunchAttribute at[1];
+                at[0].id = cudaLaunchAttributeClusterDimension;
+                at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+                probe.attrs = at;
+                probe.numAttrs = 1;
+                int n = 0;
+                cudaError_t e = raise_smem_limit_locked(product_tc_inline_pair_kernel<128>, PairCfg<128>::SMEM_BYTES, &info->inline_pair_attr[1]);
+                if (e == cudaSuccess) e = cudaOccupancyMaxActiveClusters(&n, product_tc_inline_pair_kernel<128>, &probe);
+                if (e == cudaSuccess && n > 0) known = n;
+                else cudaGetLastError();
+            }
+            if (known <= 0) continue;                                          // the pair kernel cannot be launched here
+            fit = known;
+        }
+        const long long waves = (pairs + fit - 1) / fit;
+        const double cost = (double)waves * (3.0 + kblocks * 1.2);
+        if (cost < best) { best = cost; pair_bnh = bnh; }
+    }
+    const int tiles_n = pair_bnh ? (a.n + 2 * pair_bnh - 1) / (2 * pair_bnh) : (a.n + bn - 1) / bn;
+    const long long tiles = pair_bnh ? (long long)((a.m + 2 * IBM - 1) / (2 * IBM)) * tiles_n : (long long)tiles_m * tiles_n;
 
     CUtensorMap map_a, map_b;
     if (!tc_make_map(&map_a, a.A, a.m, a.k, IBM, IBK, CU_TENSOR_MAP_SWIZZLE_128B) ||
@@ -426,6 +710,9 @@ cudaError_t launch_product_tc_inline(const ProductArgs &a, int32_t *status, cuda
     prm.add = a.add;
     prm.status = status;
 
+    if (pair_bnh == 128)
+        return launch_dependent(product_tc_inline_pair_kernel<128>, dim3((unsigned)(tiles * 2)), dim3(ITHREADS), PairCfg<128>::SMEM_BYTES, stream, 2u,
+                                map_a, map_b, prm);
     if (bn == 64)
         return launch_dependent(product_tc_inline_kernel<64>, dim3((unsigned)(tiles * split)), dim3(ITHREADS), InlineCfg<64>::SMEM_BYTES, stream,
                                 (unsigned)split, map_a, map_b, prm);

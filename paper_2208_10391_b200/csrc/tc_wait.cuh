@@ -16,12 +16,14 @@ __device__ __forceinline__ unsigned long long global_ns() {
     return t;
 }
 
-// Bounded wait: false when the limit was reached (records the failure) or another role gave up.
+// Bounded wait: false when the limit was reached (records the failure) or another role gave up.  CLUSTER: the barrier's
+// arrivals come from threads of the peer CTA too, whose writes the waiter then reads (acquire at cluster scope).
+template <bool CLUSTER = false>
 __device__ __forceinline__ bool wait_barrier(uint32_t bar, uint32_t parity, volatile int *abort_flag, int32_t *status, int detail,
                                              unsigned long long limit_ns = WAIT_LIMIT_NS) {
     unsigned long long start = 0;
     for (uint32_t i = 0;; ++i) {
-        if (ptx::mbar_try_wait(bar, parity)) return true;
+        if (CLUSTER ? ptx::mbar_try_wait_cluster(bar, parity) : ptx::mbar_try_wait(bar, parity)) return true;
         if ((i & 63) == 63) {
             if (*abort_flag) return false;
             const unsigned long long now = global_ns();

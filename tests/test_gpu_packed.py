@@ -144,7 +144,7 @@ def test_large_packed_operands_and_result_on_the_tensor_core_kernel():
     # unpacking or packing pass, no extra workspace
     n = 2048
     eq = Equation("packed_LL_2048", 330, (Operand(n, n, L), Operand(n, n, L)), (Operand(n, n, L),))
-    dense = mom.mom_equation_plan(eq.descs(), eq.add_descs(), mom.VARIANT_3XTF32)
+    dense = mom.mom_equation_plan(eq.descs(), eq.add_descs(), mom.VARIANT_3XTF32_FORCE)      # the same kernel on dense storage
     x, raw, plan, (chain, add) = run_stored(eq, mom.VARIANT_3XTF32, [P, P], [D], P)
     assert plan.step(0).uses_tensor_cores == 1
     assert plan.workspace_bytes(1) == dense.workspace_bytes(1)

@@ -119,12 +119,16 @@ INLINE_SHAPES = [
     (520, 520, 520, L, G, 1), (520, 520, 136, U, G, 0), (300, 392, 392, G, L, 0), (300, 392, 392, G, U, 2),
     (392, 392, 392, L, L, 1), (392, 392, 392, U, U, 0), (392, 392, 392, L, U, 0), (392, 392, 392, U, L, 1),
     (1024, 1024, 1024, G, G, 0), (1536, 1152, 1280, G, G, 1),
+    # more than one wave of 128 x 128 tiles but at most one wave of 256 x 256 tiles: the launcher takes the CTA-pair form
+    # (A halves in both CTAs' tensor memory, each CTA half of B, the leader issues cta_group::2 MMAs)
+    (2048, 64, 2048, G, G, 1), (1800, 100, 1900, G, G, 0), (1536, 1536, 2048, L, G, 1), (1536, 2048, 2048, G, U, 0),
+    (2048, 2048, 2048, L, L, 1),
 ]
 
 
 @pytest.mark.parametrize("m,k,n,pa,pb,terms", INLINE_SHAPES)
 def test_inline_split_tensor_core_kernel(m, k, n, pa, pb, terms):
-    # every launch shape of the kernel: 64- and 128-column tiles, 1 to 8 k-slices per tile (cluster), ragged edges in
+    # every launch shape of the kernel: 64- and 128-column tiles, 1 to 8 k-slices per tile (cluster), CTA pairs, ragged edges in
     # m, n and k, triangular factors (structural k-ranges, masked triangular results), fused Add terms incl. Identity
     dist = lambda p: "uniform" if p != G else "normal"
     add = [Operand(m, n, G, "normal")] * min(terms, 1) + ([Operand(m, n, I)] if terms == 2 and m == n else
@@ -360,9 +364,9 @@ def test_host_entry_point_uploads_large_triangles_by_blocks():
 
 
 def test_host_entry_point_copies_the_first_rows_back_early():
-    # from 2048 rows on, the product that writes X runs as two launches in the host entry point (rows up to a
+    # from 2048 rows on, a plane-kernel product that writes X runs as two launches in the host entry point (rows up to a
     # multiple of 256 near 40 % first) and the first rows travel back during the second launch; same bits as one launch
-    for n, add in ((2312, ()), (2048, (Operand(2048, 2048, G, "normal"),))):
+    for n, add in ((2312, ()), (2304, (Operand(2304, 2304, G, "normal"),))):
         eq = Equation(f"host_parts_{n}", 91, (Operand(n, n, L), Operand(n, n, G, "normal", 0.02)), add)
         chain, terms = wl.generate(eq)
         xd, plan, _ = run_equation(eq, mom.VARIANT_3XTF32, chain, terms, via="device")

@@ -499,8 +499,9 @@ def test_kernel_choice_of_the_default_variant():
     G = wl.GENERAL
     kind = lambda m, k, n, t=(False, False): mom.mom_equation_plan_transposed([(k, m, G) if t[0] else (m, k, G), (n, k, G) if t[1] else (k, n, G)], t, (), None,
                                                                           mom.VARIANT_3XTF32).step(0).uses_tensor_cores
-    assert [kind(n, n, n) for n in (256, 384, 448, 512, 768, 1024, 1536, 1792, 2048)] == [2, 2, 3, 3, 3, 3, 3, 1, 1]
+    assert [kind(n, n, n) for n in (256, 384, 448, 512, 768, 1024, 1536, 1792, 2048, 2560)] == [2, 2, 3, 3, 3, 3, 3, 3, 3, 1]
     assert kind(4096, 128, 4096) == 1                        # 2 * 10^9 multiplications, but 1024 tiles: many waves
+    assert kind(2048, 512, 2048) == 3                        # 256 tiles of 128 x 128, but one wave of CTA pairs
     assert kind(900, 1200, 100) == 3 and kind(256, 2048, 64) == 2 and kind(128, 4096, 128) == 2       # small work; a result of one tile
     assert kind(512, 512, 510) == 2                        # rows TMA cannot address
     assert kind(640, 640, 640, (True, False)) == 2 and kind(640, 640, 640, (False, True)) == 2     # transposed operands
