@@ -407,10 +407,14 @@ def run_gpu(args):
     if args.only:
         # one named configuration, nothing else: the small case for profiler captures
         cfgs = {c.name: c for c in (wl.config_tiny(), wl.config_five_general(), wl.config_property_heavy(),
-                                    wl.config_large_square(), wl.config_batched(), wl.config_paper_chain(),
+                                    wl.config_large_square(), wl.config_large_square(n=2048), wl.config_batched(), wl.config_paper_chain(),
                                     wl.config_transposed(), wl.config_sum_shared(), wl.config_sum_triangular(),
                                     wl.config_expression(), wl.config_diagonal(), wl.config_gram(), wl.config_square_product(768), wl.config_square_product(1024),
-                                    wl.config_square_product(1536), wl.config_square_product(2048), wl.config_packed_triangular())}
+                                    wl.config_square_product(1536), wl.config_square_product(2048), wl.config_packed_triangular(),
+                                    # three general factors whose products have few tiles and long contractions: the plane-fed 1-CTA
+                                    # tcgen05 kernel with the contraction split inside clusters
+                                    wl.Equation("GGG_1536_2048", 14, tuple(wl.Operand(r, c, wl.GENERAL, "normal", c ** -0.5)
+                                                                         for r, c in ((1536, 2048), (2048, 1536), (1536, 2048)))))}
         packed = args.only.endswith("_packed")       # the same equation with its triangular operands handed over as packed triangles
         cfg = cfgs[args.only[:-len("_packed")] if packed else args.only]
         storage = None
