@@ -23,7 +23,7 @@ constexpr int BM = 64, BN = 32, BK = 32, THREADS = 256, STAGES = 3;
 // A[g][t] (rows 4 mod 8 words apart) and B[t][g] (rows 8 mod 16 words apart)
 constexpr int LDA = BK + 4, LDB = BN + 8, LDP = BN + 4;
 constexpr int A_STAGE = BM * LDA, B_STAGE = BK * LDB;        // floats per pipeline stage
-constexpr int MAX_SPLIT = 8;                                 // portable cluster size
+constexpr int MAX_SPLIT = 16;                                // 8 is the portable cluster size; 16 where the device takes it
 
 static_assert(BM * LDP <= STAGES * A_STAGE, "the partial tile reuses the A stages");
 
@@ -211,6 +211,29 @@ cudaError_t launch_product_mma(const ProductArgs &a, int batch, cudaStream_t str
     int split = 1;
     const long long resident = 4LL * sm_count;
     while (split < MAX_SPLIT && tiles * batch * split * 2 <= resident && a.k / (split * 2) >= 4 * BK) split *= 2;
+    if (split == 16) {
+        // a cluster of 16 needs the non-portable size allowed on this kernel, and room for all clusters at once
+        std::lock_guard<std::mutex> lock(device_info_mutex());
+        DeviceInfo *info = current_device_info();
+        if (!info) return cudaErrorInvalidDevice;
+        if (info->mma_clusters16 == 0) {
+            info->mma_clusters16 = -1;
+            if (cudaFuncSetAttribute(product_mma_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess) {
+                cudaLaunchConfig_t probe = {};
+                probe.gridDim = dim3((unsigned)(16 * sm_count));
+                probe.blockDim = dim3(THREADS);
+                cudaLaunchAttribute at[1];
+                at[0].id = cudaLaunchAttributeClusterDimension;
+                at[0].val.clusterDim.x = 16; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+                probe.attrs = at;
+                probe.numAttrs = 1;
+                int n = 0;
+                if (cudaOccupancyMaxActiveClusters(&n, product_mma_kernel, &probe) == cudaSuccess && n > 0) info->mma_clusters16 = n;
+            }
+            cudaGetLastError();
+        }
+        if (info->mma_clusters16 < tiles * batch) split = 8;
+    }
     // An ordinary launch: with the programmatic-dependent-launch attribute (the prologue overlapping the previous launch's tail) the
     // large cluster-split products of this kernel gained 2 us, but the small ones lost more (384^3: 10.3 -> 16.2 us; the five-matrix
     // chain 34.9 -> 37.4 us): measured, not kept.

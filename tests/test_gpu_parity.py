@@ -126,6 +126,17 @@ INLINE_SHAPES = [
 ]
 
 
+@pytest.mark.parametrize("m,k,n", [(256, 2048, 64), (100, 4099, 44), (64, 8192, 32), (130, 2052, 70)])
+def test_warp_level_kernel_with_sixteen_k_slices(m, k, n):
+    # very few output tiles and a contraction of 2048 or more: the warp-level kernel splits k over clusters of 16 CTAs (the
+    # non-portable cluster size) that add their partial tiles through distributed shared memory; ragged m, n and k
+    eq = Equation(f"warp16_{m}x{k}x{n}", 77, (Operand(m, k, G, "normal", 1.0 / np.sqrt(k)), Operand(k, n, G, "normal")),
+                  (Operand(m, n, G, "normal"),))
+    x, plan, (chain, terms_h) = run_equation(eq, mom.VARIANT_3XTF32_WARP)
+    assert plan.step(0).uses_tensor_cores == 2 and plan.last_launch_count() == 1
+    check_against_oracle(eq, x, plan, chain, terms_h)
+
+
 @pytest.mark.parametrize("m,k,n,pa,pb,terms", INLINE_SHAPES)
 def test_inline_split_tensor_core_kernel(m, k, n, pa, pb, terms):
     # every launch shape of the kernel: 64- and 128-column tiles, 1 to 8 k-slices per tile (cluster), CTA pairs, ragged edges in
