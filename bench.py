@@ -49,7 +49,7 @@ def whole_job_gflops(useful_flops_per_replica: int, world: int, ms_per_step: flo
 # DRAM traffic of the dominant kernel per launch on the headline workload, from one ncu capture
 # (dram__bytes_read.sum + dram__bytes_write.sum, mean over the step's three product launches).  It is only
 # reported while the kernel source is the one that was captured.
-TRAFFIC_CAPTURE = {"kernel_source_sha256_16": "3c70c3639caba115", "bytes_per_launch": 6.65e9}
+TRAFFIC_CAPTURE = {"kernel_source_sha256_16": "7c35fd35704f513b", "bytes_per_launch": 7.64e9}
 
 
 def measured_traffic():
