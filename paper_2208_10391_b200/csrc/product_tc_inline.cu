@@ -43,7 +43,7 @@ namespace {
 namespace cg = cooperative_groups;
 
 constexpr int IBM = 128, IBK = 32, ITHREADS = 320, IMAX_SPLIT = 8;    // warps: producer, MMA issuer, eight transform / epilogue warps
-constexpr int XFORM_WARPS = 8, XFORM_THREADS = 32 * XFORM_WARPS;
+constexpr int XFORM_WARPS = 8;
 
 template <int BN>
 struct InlineCfg {
@@ -87,6 +87,36 @@ __device__ __forceinline__ void split4(const float4 a, float4 &hi, float4 &lo) {
 // K-major tile with 128-byte rows under the 128B swizzle: 8-row groups are 1024 bytes apart, a K = 8 step is 32 bytes
 __device__ __forceinline__ uint64_t kmajor_desc128(uint32_t tile, int kstep) {
     return ptx::smem_desc(tile + kstep * 32, 16, 8 * 128, ptx::SWIZZLE_128B);
+}
+
+// Epilogue store of a warp's 32 x 32 chunk of the tile (lane = row, v = its 32 columns): through a 32 x 36 staging tile of the warp
+// in shared memory, so that the stores to C and the loads of the Add terms are row-contiguous (one instruction covers four rows of
+// 128 bytes instead of 32 rows of 16).  Conflict-free both ways: a store phase's eight lanes are eight rows 36 words apart, a load
+// phase's eight lanes one row's 32 words.
+constexpr int STAGE_LD = 36, STAGE_FLOATS = 32 * STAGE_LD;
+__device__ __forceinline__ void store_chunk(float *stage, const float (&v)[32], int lane, int row_base, int col0, const InlineParams &prm, bool vec) {
+#pragma unroll
+    for (int j = 0; j < 8; ++j)
+        *reinterpret_cast<float4 *>(stage + lane * STAGE_LD + 4 * j) = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+    __syncwarp();
+    const int sub = lane >> 3, cc = col0 + (lane & 7) * 4;
+#pragma unroll
+    for (int it = 0; it < 8; ++it) {
+        const int row = 4 * it + sub, r = row_base + row;
+        const float4 x = *reinterpret_cast<const float4 *>(stage + row * STAGE_LD + (lane & 7) * 4);
+        if (r >= prm.m || cc >= prm.n) continue;
+        float w[4] = {x.x, x.y, x.z, x.w};
+        finish_row4(w, prm.add, 0, r, cc, prm.n, prm.n, prm.pout, vec);
+        float *dst = prm.C + (long long)r * prm.n + cc;
+        if (vec && cc + 3 < prm.n) {
+            *reinterpret_cast<float4 *>(dst) = make_float4(w[0], w[1], w[2], w[3]);
+        } else {
+#pragma unroll
+            for (int e = 0; e < 4; ++e)
+                if (cc + e < prm.n) dst[e] = w[e];
+        }
+    }
+    __syncwarp();                                            // the staging tile is free for the warp's next chunk
 }
 
 template <int BN>
@@ -270,7 +300,7 @@ product_tc_inline_kernel(const __grid_constant__ CUtensorMap map_a, const __grid
             if (lane == 0) { ptx::mbar_arrive(ready(s)); ptx::mbar_arrive(raw_empty(rs)); }
         }
         // ---- epilogue: this warp reads TMEM lanes 32 q .. 32 q + 31 = rows of the tile; the two warps of a quarter share the columns
-        const int q = warp & 3, row = q * 32 + lane, r = r0 + row, half = w2 >> 2;
+        const int q = warp & 3, row = q * 32 + lane, half = w2 >> 2;
         if (nk > 0 && ok) {
             if (lane == 0) ok = wait_barrier(acc_full, 0, abort_flag, prm.status, (14 << 24) | (tile & 0xFFFF));
             ok = __shfl_sync(0xffffffffu, ok, 0);
@@ -294,22 +324,8 @@ product_tc_inline_kernel(const __grid_constant__ CUtensorMap map_a, const __grid
 #pragma unroll
                 for (int j = 0; j < 8; ++j)
                     *reinterpret_cast<float4 *>(P + row * Cfg::LDP + 32 * c + 4 * j) = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
-            } else if (r < prm.m) {
-#pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    const int cc = col0 + 4 * j;
-                    if (cc >= prm.n) break;
-                    float w[4] = {v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]};
-                    finish_row4(w, prm.add, 0, r, cc, prm.n, prm.n, prm.pout, vec);
-                    float *dst = prm.C + (long long)r * prm.n + cc;
-                    if (vec && cc + 3 < prm.n) {
-                        *reinterpret_cast<float4 *>(dst) = make_float4(w[0], w[1], w[2], w[3]);
-                    } else {
-#pragma unroll
-                        for (int e = 0; e < 4; ++e)
-                            if (cc + e < prm.n) dst[e] = w[e];
-                    }
-                }
+            } else {
+                store_chunk(P + w2 * STAGE_FLOATS, v, lane, r0 + q * 32, col0, prm, vec);
             }
         }
     }
@@ -549,7 +565,7 @@ product_tc_inline_pair_kernel(const __grid_constant__ CUtensorMap map_a, const _
             }
         }
         // ---- epilogue: this CTA's 128 rows of the accumulator
-        const int q = warp & 3, row = q * 32 + lane, r = my_r0 + row, half = w2 >> 2;
+        const int q = warp & 3, half = w2 >> 2;
         if (nk > 0 && ok) {
             if (lane == 0) ok = wait_barrier(acc_full, 0, abort_flag, prm.status, (24 << 24) | (tile & 0xFFFF));
             ok = __shfl_sync(0xffffffffu, ok, 0);
@@ -568,23 +584,7 @@ product_tc_inline_pair_kernel(const __grid_constant__ CUtensorMap map_a, const _
 #pragma unroll
                 for (int j = 0; j < 32; ++j) v[j] = 0.0f;
             }
-            if (r < prm.m) {
-#pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    const int cc = col0 + 4 * j;
-                    if (cc >= prm.n) break;
-                    float w[4] = {v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]};
-                    finish_row4(w, prm.add, 0, r, cc, prm.n, prm.n, prm.pout, vec);
-                    float *dst = prm.C + (long long)r * prm.n + cc;
-                    if (vec && cc + 3 < prm.n) {
-                        *reinterpret_cast<float4 *>(dst) = make_float4(w[0], w[1], w[2], w[3]);
-                    } else {
-#pragma unroll
-                        for (int e = 0; e < 4; ++e)
-                            if (cc + e < prm.n) dst[e] = w[e];
-                    }
-                }
-            }
+            store_chunk(reinterpret_cast<float *>(base_ptr) + w2 * STAGE_FLOATS, v, lane, my_r0 + q * 32, col0, prm, vec);
         }
     }
 
