@@ -16,7 +16,7 @@ struct DeviceInfo {
     bool tc_attr = false;            // dynamic shared-memory limit raised for the tensor-core kernels on this device
     bool pair_attr = false;
     bool inline64_attr = false, inline128_attr = false;
-    int inline_clusters[2][4] = {};  // co-resident clusters of the one-launch tcgen05 kernel, [128-column tiles][log2 cluster size]; 0: not asked, -1: unknown
+    int inline_clusters[2][5] = {};  // co-resident clusters of the one-launch tcgen05 kernel, [128-column tiles][log2 cluster size]; 0: not asked, -1: unknown
     bool inline_pair_attr[2] = {false, false};
     int inline_pair_clusters[2] = {0, 0};   // co-resident CTA pairs of the one-launch kernel's pair variant, [128 columns per CTA]
     int mma_clusters16 = 0;          // co-resident clusters of 16 CTAs of the warp-level kernel (0: not asked yet, -1: not available)

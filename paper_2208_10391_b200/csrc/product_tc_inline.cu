@@ -18,7 +18,7 @@
 //               frees the stage;
 //   warps 2-9   then the epilogue: tcgen05.ld (two warps per quarter of the tile's rows, each half of the columns), Add terms,
 //               structure mask, 16-byte stores.
-// With few output tiles the contraction is split over the CTAs of a thread-block cluster (up to 8): each leaves its partial
+// With few output tiles the contraction is split over the CTAs of a thread-block cluster (up to 16): each leaves its partial
 // tile in its own shared memory and CTA r finishes rows [r * 128 / s, (r + 1) * 128 / s) by adding the partial tiles through
 // distributed shared memory in k order (deterministic; no atomics, no scratch in global memory, no second launch).
 // The tile's structural k-range bounds the contraction as everywhere else.  Shared memory still moves more bytes per
@@ -42,7 +42,7 @@ namespace {
 
 namespace cg = cooperative_groups;
 
-constexpr int IBM = 128, IBK = 32, ITHREADS = 320, IMAX_SPLIT = 8;    // warps: producer, MMA issuer, eight transform / epilogue warps
+constexpr int IBM = 128, IBK = 32, ITHREADS = 320, IMAX_SPLIT = 16;    // warps: producer, MMA issuer, eight transform / epilogue warps
 constexpr int XFORM_WARPS = 8;
 
 template <int BN>
@@ -627,7 +627,7 @@ cudaError_t launch_product_tc_inline(const ProductArgs &a, int32_t *status, cuda
                 std::lock_guard<std::mutex> lock(device_info_mutex());
                 DeviceInfo *info = current_device_info();
                 if (!info) return cudaErrorInvalidDevice;
-                int &known = info->inline_clusters[width == 128][s == 1 ? 0 : s == 2 ? 1 : s == 4 ? 2 : 3];
+                int &known = info->inline_clusters[width == 128][s == 1 ? 0 : s == 2 ? 1 : s == 4 ? 2 : s == 8 ? 3 : 4];
                 if (known == 0) {
                     known = -1;
                     cudaLaunchConfig_t probe = {};
@@ -642,6 +642,9 @@ cudaError_t launch_product_tc_inline(const ProductArgs &a, int32_t *status, cuda
                     int n = 0;
                     cudaError_t e = width == 128 ? raise_smem_limit_locked(product_tc_inline_kernel<128>, InlineCfg<128>::SMEM_BYTES, &info->inline128_attr)
                                                  : raise_smem_limit_locked(product_tc_inline_kernel<64>, InlineCfg<64>::SMEM_BYTES, &info->inline64_attr);
+                    if (e == cudaSuccess && s > 8)                            // beyond the portable cluster size: allowed per kernel
+                        e = width == 128 ? cudaFuncSetAttribute(product_tc_inline_kernel<128>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1)
+                                         : cudaFuncSetAttribute(product_tc_inline_kernel<64>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
                     if (e == cudaSuccess)
                         e = width == 128 ? cudaOccupancyMaxActiveClusters(&n, product_tc_inline_kernel<128>, &probe)
                                          : cudaOccupancyMaxActiveClusters(&n, product_tc_inline_kernel<64>, &probe);
@@ -649,10 +652,11 @@ cudaError_t launch_product_tc_inline(const ProductArgs &a, int32_t *status, cuda
                     else cudaGetLastError();
                 }
                 if (known > 0) fit = known;
+                else if (s > 8) fit = 0;                                       // no cluster of 16 unless the runtime says it fits
             }
             if (fit < 1) continue;
             const long long waves = (tiles + fit - 1) / fit;
-            const double cost = (double)waves * ((width == 128 ? 2.5 : 2.0) + ((kblocks + s - 1) / s) * (width == 128 ? 0.9 : 0.66) + (s > 1 ? 1.5 : 0.0));
+            const double cost = (double)waves * ((width == 128 ? 2.5 : 2.0) + ((kblocks + s - 1) / s) * (width == 128 ? 0.9 : 0.66) + (s > 8 ? 2.0 : s > 1 ? 1.5 : 0.0));
             if (cost < best) { best = cost; bn = width; split = s; }
         }
     }

@@ -119,6 +119,7 @@ INLINE_SHAPES = [
     (520, 520, 520, L, G, 1), (520, 520, 136, U, G, 0), (300, 392, 392, G, L, 0), (300, 392, 392, G, U, 2),
     (392, 392, 392, L, L, 1), (392, 392, 392, U, U, 0), (392, 392, 392, L, U, 0), (392, 392, 392, U, L, 1),
     (1024, 1024, 1024, G, G, 0), (1536, 1152, 1280, G, G, 1),
+    (128, 4096, 128, G, G, 1), (100, 4100, 60, G, G, 0),            # one or two tiles, long contraction: clusters of 16 CTAs
     # more than one wave of 128 x 128 tiles but at most one wave of 256 x 256 tiles: the launcher takes the CTA-pair form
     # (A halves in both CTAs' tensor memory, each CTA half of B, the leader issues cta_group::2 MMAs)
     (2048, 64, 2048, G, G, 1), (1800, 100, 1900, G, G, 0), (1536, 1536, 2048, L, G, 1), (1536, 2048, 2048, G, U, 0),
