@@ -89,6 +89,69 @@ __device__ __forceinline__ uint64_t kmajor_desc128(uint32_t tile, int kstep) {
     return ptx::smem_desc(tile + kstep * 32, 16, 8 * 128, ptx::SWIZZLE_128B);
 }
 
+// The transform of one k-block, shared by the 1-CTA and the CTA-pair kernels: a warp of the eight transform warps (w2 = 0..7) splits
+// its share of the raw tiles.  NB = columns of B this CTA holds.
+//   A: the thread owns row 32 ((w2 + 2) % 4) + lane of the tile (the tensor-memory lane its warp may write) and half of its 32 k: four
+//      16-byte loads from the swizzled raw tile, two tcgen05.st of 16 columns (hi, lo).
+//   B: task t of the warp is (box j, group c) = columns 32 j + 4 c .. + 3 of k-row `lane`; value e of it lands in row
+//      n = 32 j + 4 c + e of the K-major tile, at k = lane (group lane / 4, word lane % 4).
+template <int NB>
+struct Transform {
+    static constexpr int TASKS = NB / 4 / XFORM_WARPS;
+    uint32_t a_src[4], src_off[TASKS], dst_off[TASKS][4];
+    __device__ __forceinline__ Transform(int w2, int lane) {
+        const int arow = ((w2 + 2) & 3) * 32 + lane, ahalf = w2 >> 2;     // transform warp w2 is warp w2 + 2 of the CTA: lanes 32 (warp % 4) ..
+#pragma unroll
+        for (int u = 0; u < 4; ++u) a_src[u] = arow * 128 + (((4 * ahalf + u) ^ (arow & 7)) << 4);
+#pragma unroll
+        for (int t = 0; t < TASKS; ++t) {
+            const int task = w2 + XFORM_WARPS * t, j = task >> 3, c = task & 7;
+            src_off[t] = j * 4096 + lane * 128 + ((c ^ (lane & 7)) << 4);
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const int n = 32 * j + 4 * c + e;
+                dst_off[t][e] = n * 128 + ((((uint32_t)lane >> 2) ^ (n & 7)) << 4) + ((lane & 3) << 2);
+            }
+        }
+    }
+    // araw / braw: the raw tiles of A and B; a_tmem: this thread's 16 columns of A's hi half in tensor memory (lo: + IBK);
+    // bhi / blo: B's K-major tiles.  Ends with everything the MMA will read made visible to it.
+    __device__ __forceinline__ void run(const uint8_t *araw, const uint8_t *braw, uint32_t a_tmem, uint8_t *bhi, uint8_t *blo) const {
+        float4 av[4], bv[TASKS];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) av[u] = *reinterpret_cast<const float4 *>(araw + a_src[u]);
+#pragma unroll
+        for (int t = 0; t < TASKS; ++t) bv[t] = *reinterpret_cast<const float4 *>(braw + src_off[t]);
+        {
+            uint32_t hi16[16], lo16[16];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                float4 hi, lo;
+                split4(av[u], hi, lo);
+                hi16[4 * u] = __float_as_uint(hi.x); hi16[4 * u + 1] = __float_as_uint(hi.y);
+                hi16[4 * u + 2] = __float_as_uint(hi.z); hi16[4 * u + 3] = __float_as_uint(hi.w);
+                lo16[4 * u] = __float_as_uint(lo.x); lo16[4 * u + 1] = __float_as_uint(lo.y);
+                lo16[4 * u + 2] = __float_as_uint(lo.z); lo16[4 * u + 3] = __float_as_uint(lo.w);
+            }
+            ptx::tmem_st_16cols(a_tmem, hi16);
+            ptx::tmem_st_16cols(a_tmem + IBK, lo16);
+        }
+#pragma unroll
+        for (int t = 0; t < TASKS; ++t) {
+            float4 hi, lo;
+            split4(bv[t], hi, lo);
+            *reinterpret_cast<float *>(bhi + dst_off[t][0]) = hi.x; *reinterpret_cast<float *>(blo + dst_off[t][0]) = lo.x;
+            *reinterpret_cast<float *>(bhi + dst_off[t][1]) = hi.y; *reinterpret_cast<float *>(blo + dst_off[t][1]) = lo.y;
+            *reinterpret_cast<float *>(bhi + dst_off[t][2]) = hi.z; *reinterpret_cast<float *>(blo + dst_off[t][2]) = lo.z;
+            *reinterpret_cast<float *>(bhi + dst_off[t][3]) = hi.w; *reinterpret_cast<float *>(blo + dst_off[t][3]) = lo.w;
+        }
+        ptx::tmem_wait_st();
+        ptx::fence_proxy_async_smem();                       // the MMA reads B's tiles through the asynchronous proxy
+        ptx::tc_fence_before_sync();
+        __syncwarp();
+    }
+};
+
 // Epilogue store of a warp's 32 x 32 chunk of the tile (lane = row, v = its 32 columns): through a 32 x 36 staging tile of the warp
 // in shared memory, so that the stores to C and the loads of the Add terms are row-contiguous (one instruction covers four rows of
 // 128 bytes instead of 32 rows of 16).  Conflict-free both ways: a store phase's eight lanes are eight rows 36 words apart, a load
@@ -231,26 +294,8 @@ product_tc_inline_kernel(const __grid_constant__ CUtensorMap map_a, const __grid
     } else {
         // ------------------------------------------------------------------ transform (warps 2..9), then epilogue
         const int w2 = warp - 2;
-        // A: this thread owns row 32 q + lane of the tile (the tensor-memory lane its warp may write) and half of its 32 k
-        const int arow = (warp & 3) * 32 + lane, ahalf = w2 >> 2;
-        uint32_t a_src[4];
-#pragma unroll
-        for (int u = 0; u < 4; ++u) a_src[u] = arow * 128 + (((4 * ahalf + u) ^ (arow & 7)) << 4);
-        const uint32_t a_dst = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + BN + 16 * ahalf;
-        // where this lane's values of B go: task t of the warp is (box j, group c) = columns 32 j + 4 c .. + 3 of k-row `lane`;
-        // value e of it lands in row n = 32 j + 4 c + e of the K-major tile, at k = lane (group lane / 4, word lane % 4)
-        constexpr int TASKS = BN / 4 / XFORM_WARPS;
-        uint32_t src_off[TASKS], dst_off[TASKS][4];
-#pragma unroll
-        for (int t = 0; t < TASKS; ++t) {
-            const int task = w2 + XFORM_WARPS * t, j = task >> 3, c = task & 7;
-            src_off[t] = j * 4096 + lane * 128 + ((c ^ (lane & 7)) << 4);
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                const int n = 32 * j + 4 * c + e;
-                dst_off[t][e] = n * 128 + ((((uint32_t)lane >> 2) ^ (n & 7)) << 4) + ((lane & 3) << 2);
-            }
-        }
+        const Transform<BN> xf(w2, lane);
+        const uint32_t a_dst = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + BN + 16 * (w2 >> 2);
         bool ok = true;
         uint8_t *const split_ptr = base_ptr + R * Cfg::RAW_BYTES;
         for (int i = 0; i < nk && ok; ++i) {
@@ -262,41 +307,8 @@ product_tc_inline_kernel(const __grid_constant__ CUtensorMap map_a, const __grid
             if (!ok) break;
             uint8_t *const st = base_ptr + rs * Cfg::RAW_BYTES;
             ptx::tc_fence_after_sync();                      // the MMAs that read this split stage (tensor memory and B's tiles) are done
-            float4 av[4];
-#pragma unroll
-            for (int u = 0; u < 4; ++u) av[u] = *reinterpret_cast<const float4 *>(st + a_src[u]);
-            // B: box j holds k-rows 0..31 x columns 32 j .. 32 j + 31, group c of row k at group c ^ (k & 7).  Lane = k-row.
-            uint8_t *const braw = st + Cfg::A_BYTES, *const bhi = split_ptr + s * Cfg::SPLIT_BYTES, *const blo = bhi + Cfg::B_PLANE_BYTES;
-            float4 bv[TASKS];
-#pragma unroll
-            for (int t = 0; t < TASKS; ++t) bv[t] = *reinterpret_cast<const float4 *>(braw + src_off[t]);
-            {
-                uint32_t hi16[16], lo16[16];
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    float4 hi, lo;
-                    split4(av[u], hi, lo);
-                    hi16[4 * u] = __float_as_uint(hi.x); hi16[4 * u + 1] = __float_as_uint(hi.y);
-                    hi16[4 * u + 2] = __float_as_uint(hi.z); hi16[4 * u + 3] = __float_as_uint(hi.w);
-                    lo16[4 * u] = __float_as_uint(lo.x); lo16[4 * u + 1] = __float_as_uint(lo.y);
-                    lo16[4 * u + 2] = __float_as_uint(lo.z); lo16[4 * u + 3] = __float_as_uint(lo.w);
-                }
-                ptx::tmem_st_16cols(a_dst + s * Cfg::A_COLS, hi16);
-                ptx::tmem_st_16cols(a_dst + s * Cfg::A_COLS + IBK, lo16);
-            }
-#pragma unroll
-            for (int t = 0; t < TASKS; ++t) {
-                float4 hi, lo;
-                split4(bv[t], hi, lo);
-                *reinterpret_cast<float *>(bhi + dst_off[t][0]) = hi.x; *reinterpret_cast<float *>(blo + dst_off[t][0]) = lo.x;
-                *reinterpret_cast<float *>(bhi + dst_off[t][1]) = hi.y; *reinterpret_cast<float *>(blo + dst_off[t][1]) = lo.y;
-                *reinterpret_cast<float *>(bhi + dst_off[t][2]) = hi.z; *reinterpret_cast<float *>(blo + dst_off[t][2]) = lo.z;
-                *reinterpret_cast<float *>(bhi + dst_off[t][3]) = hi.w; *reinterpret_cast<float *>(blo + dst_off[t][3]) = lo.w;
-            }
-            ptx::tmem_wait_st();
-            ptx::fence_proxy_async_smem();                   // the MMA reads B's tiles through the asynchronous proxy
-            ptx::tc_fence_before_sync();
-            __syncwarp();
+            uint8_t *const bhi = split_ptr + s * Cfg::SPLIT_BYTES;
+            xf.run(st, st + Cfg::A_BYTES, a_dst + s * Cfg::A_COLS, bhi, bhi + Cfg::B_PLANE_BYTES);
             if (lane == 0) { ptx::mbar_arrive(ready(s)); ptx::mbar_arrive(raw_empty(rs)); }
         }
         // ---- epilogue: this warp reads TMEM lanes 32 q .. 32 q + 31 = rows of the tile; the two warps of a quarter share the columns
@@ -497,23 +509,8 @@ product_tc_inline_pair_kernel(const __grid_constant__ CUtensorMap map_a, const _
     } else {
         // ------------------------------------------------------------------ transform (warps 2..9, both CTAs), then epilogue
         const int w2 = warp - 2;
-        const int arow = (warp & 3) * 32 + lane, ahalf = w2 >> 2;
-        uint32_t a_src[4];
-#pragma unroll
-        for (int u = 0; u < 4; ++u) a_src[u] = arow * 128 + (((4 * ahalf + u) ^ (arow & 7)) << 4);
-        const uint32_t a_dst = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + BN2 + 16 * ahalf;
-        constexpr int TASKS = BNH / 4 / XFORM_WARPS;
-        uint32_t src_off[TASKS], dst_off[TASKS][4];
-#pragma unroll
-        for (int t = 0; t < TASKS; ++t) {
-            const int task = w2 + XFORM_WARPS * t, j = task >> 3, c = task & 7;
-            src_off[t] = j * 4096 + lane * 128 + ((c ^ (lane & 7)) << 4);
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                const int n = 32 * j + 4 * c + e;
-                dst_off[t][e] = n * 128 + ((((uint32_t)lane >> 2) ^ (n & 7)) << 4) + ((lane & 3) << 2);
-            }
-        }
+        const Transform<BNH> xf(w2, lane);
+        const uint32_t a_dst = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + BN2 + 16 * (w2 >> 2);
         bool ok = true;
         uint8_t *const split_ptr = base_ptr + R * Cfg::RAW_BYTES;
         for (int i = 0; i < nk && ok; ++i) {
@@ -525,40 +522,8 @@ product_tc_inline_pair_kernel(const __grid_constant__ CUtensorMap map_a, const _
             if (!ok) break;
             uint8_t *const st = base_ptr + rs * Cfg::RAW_BYTES;
             ptx::tc_fence_after_sync();
-            float4 av[4];
-#pragma unroll
-            for (int u = 0; u < 4; ++u) av[u] = *reinterpret_cast<const float4 *>(st + a_src[u]);
-            uint8_t *const braw = st + Cfg::A_BYTES, *const bhi = split_ptr + s * Cfg::SPLIT_BYTES, *const blo = bhi + Cfg::B_PLANE_BYTES;
-            float4 bv[TASKS];
-#pragma unroll
-            for (int t = 0; t < TASKS; ++t) bv[t] = *reinterpret_cast<const float4 *>(braw + src_off[t]);
-            {
-                uint32_t hi16[16], lo16[16];
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    float4 hi, lo;
-                    split4(av[u], hi, lo);
-                    hi16[4 * u] = __float_as_uint(hi.x); hi16[4 * u + 1] = __float_as_uint(hi.y);
-                    hi16[4 * u + 2] = __float_as_uint(hi.z); hi16[4 * u + 3] = __float_as_uint(hi.w);
-                    lo16[4 * u] = __float_as_uint(lo.x); lo16[4 * u + 1] = __float_as_uint(lo.y);
-                    lo16[4 * u + 2] = __float_as_uint(lo.z); lo16[4 * u + 3] = __float_as_uint(lo.w);
-                }
-                ptx::tmem_st_16cols(a_dst + s * Cfg::A_COLS, hi16);
-                ptx::tmem_st_16cols(a_dst + s * Cfg::A_COLS + IBK, lo16);
-            }
-#pragma unroll
-            for (int t = 0; t < TASKS; ++t) {
-                float4 hi, lo;
-                split4(bv[t], hi, lo);
-                *reinterpret_cast<float *>(bhi + dst_off[t][0]) = hi.x; *reinterpret_cast<float *>(blo + dst_off[t][0]) = lo.x;
-                *reinterpret_cast<float *>(bhi + dst_off[t][1]) = hi.y; *reinterpret_cast<float *>(blo + dst_off[t][1]) = lo.y;
-                *reinterpret_cast<float *>(bhi + dst_off[t][2]) = hi.z; *reinterpret_cast<float *>(blo + dst_off[t][2]) = lo.z;
-                *reinterpret_cast<float *>(bhi + dst_off[t][3]) = hi.w; *reinterpret_cast<float *>(blo + dst_off[t][3]) = lo.w;
-            }
-            ptx::tmem_wait_st();
-            ptx::fence_proxy_async_smem();
-            ptx::tc_fence_before_sync();
-            __syncwarp();
+            uint8_t *const bhi = split_ptr + s * Cfg::SPLIT_BYTES;
+            xf.run(st, st + Cfg::A_BYTES, a_dst + s * Cfg::A_COLS, bhi, bhi + Cfg::B_PLANE_BYTES);
             if (lane == 0) {
                 ptx::mbar_arrive_cluster(ptx::map_to_cta(ready(s), 0));      // the leader's barrier, from either CTA
                 ptx::mbar_arrive(raw_empty(rs));
