@@ -128,7 +128,7 @@ __device__ __forceinline__ void finish_row4(float (&v)[4], const AddTerms &add, 
             continue;
         }
         p += batch * add.stride[t];
-        const bool tr = (add.transposed >> t) & 1u, alias = (add.aliases_out >> t) & 1u;
+        const bool tr = (add.transposed >> t) & 1u;          // (a term that aliases the output is read like any other: every load here is coherent)
         if (!tr && vec && c + 3 < n && (reinterpret_cast<uintptr_t>(p) & 15) == 0) {
             const float4 *q = reinterpret_cast<const float4 *>(p + (long long)r * ld + c);
             const float4 x = __ldcg(q);

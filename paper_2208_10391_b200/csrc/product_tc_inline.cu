@@ -182,6 +182,52 @@ __device__ __forceinline__ void store_chunk(float *stage, const float (&v)[32], 
     __syncwarp();                                            // the staging tile is free for the warp's next chunk
 }
 
+// Split contraction, last phase: CTA `rank` of the cluster finishes rows [rank * 128 / SPLIT, ...) of the tile, adding the cluster's
+// partial tiles (P: this CTA's, at the same address in every CTA) in k order.  A load through distributed shared memory takes
+// 500-700 cycles, so ALL the loads a thread needs (its items x SPLIT peers, at most 16 of 16 bytes) are issued before the first
+// sum.  The cluster's second barrier is split: a CTA arrives once its sums are in registers (nobody needs its peers' shared memory
+// any more on its behalf) and waits after its Add terms and stores (it may not leave while a peer still reads its tile).
+template <int BN, int SPLIT>
+__device__ __forceinline__ void reduce_partial_tiles(cg::cluster_group &cluster, const float *P, int rank, int r0, int c0, const InlineParams &prm) {
+    constexpr int LDP = BN + 4, ROWS = IBM / SPLIT, ITEMS = ROWS * (BN / 4), NI = (ITEMS + ITHREADS - 1) / ITHREADS;
+    const float *peer[SPLIT];
+#pragma unroll
+    for (int q = 0; q < SPLIT; ++q) peer[q] = cluster.map_shared_rank(P, q);
+    float4 x[NI][SPLIT];
+#pragma unroll
+    for (int i = 0; i < NI; ++i) {
+        const int e = threadIdx.x + i * ITHREADS;
+        const int off = (rank * ROWS + e / (BN / 4)) * LDP + ((e % (BN / 4)) << 2);
+#pragma unroll
+        for (int q = 0; q < SPLIT; ++q) x[i][q] = e < ITEMS ? *reinterpret_cast<const float4 *>(peer[q] + off) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+    float w[NI][4];
+#pragma unroll
+    for (int i = 0; i < NI; ++i) {
+        w[i][0] = w[i][1] = w[i][2] = w[i][3] = 0.f;
+#pragma unroll
+        for (int q = 0; q < SPLIT; ++q) { w[i][0] += x[i][q].x; w[i][1] += x[i][q].y; w[i][2] += x[i][q].z; w[i][3] += x[i][q].w; }
+    }
+    ptx::cluster_arrive();
+    const bool vec = (reinterpret_cast<uintptr_t>(prm.C) & 15) == 0 && (prm.n & 3) == 0;
+#pragma unroll
+    for (int i = 0; i < NI; ++i) {
+        const int e = threadIdx.x + i * ITHREADS;
+        const int r = r0 + rank * ROWS + e / (BN / 4), cc = c0 + ((e % (BN / 4)) << 2);
+        if (e >= ITEMS || r >= prm.m || cc >= prm.n) continue;
+        finish_row4(w[i], prm.add, 0, r, cc, prm.n, prm.n, prm.pout, vec);
+        float *dst = prm.C + (long long)r * prm.n + cc;
+        if (vec && cc + 3 < prm.n) {
+            *reinterpret_cast<float4 *>(dst) = make_float4(w[i][0], w[i][1], w[i][2], w[i][3]);
+        } else {
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                if (cc + j < prm.n) dst[j] = w[i][j];
+        }
+    }
+    ptx::cluster_wait();
+}
+
 template <int BN>
 __global__ void __launch_bounds__(ITHREADS, 1)
 product_tc_inline_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const InlineParams prm) {
@@ -345,35 +391,19 @@ product_tc_inline_kernel(const __grid_constant__ CUtensorMap map_a, const __grid
     ptx::tc_fence_before_sync();
     __syncthreads();
     ptx::tc_fence_after_sync();
+    if (split > 1) ptx::cluster_arrive();                    // this CTA's partial tile is written (the wait follows below)
     if (warp == 1) ptx::tmem_dealloc(tmem_base, Cfg::TMEM_COLS);
     if (split == 1) return;
 
     // ---- split contraction: CTA `rank` finishes its rows of the tile, adding the cluster's partial tiles in k order
-    cluster.sync();
-    {
-        const float *const P = reinterpret_cast<const float *>(base_ptr);
-        const bool vec = (reinterpret_cast<uintptr_t>(prm.C) & 15) == 0 && (prm.n & 3) == 0;
-        const int rows_per = IBM / split;
-        for (int e = threadIdx.x; e < rows_per * (BN / 4); e += ITHREADS) {
-            const int row = rank * rows_per + e / (BN / 4), col = (e % (BN / 4)) << 2;
-            const int r = r0 + row, cc = c0 + col;
-            if (r >= prm.m || cc >= prm.n) continue;
-            float w[4] = {0.f, 0.f, 0.f, 0.f};
-            for (int peer = 0; peer < split; ++peer) {
-                const float4 x = *reinterpret_cast<const float4 *>(cluster.map_shared_rank(P, peer) + row * Cfg::LDP + col);
-                w[0] += x.x; w[1] += x.y; w[2] += x.z; w[3] += x.w;
-            }
-            finish_row4(w, prm.add, 0, r, cc, prm.n, prm.n, prm.pout, vec);
-            float *dst = prm.C + (long long)r * prm.n + cc;
-            if (vec && cc + 3 < prm.n) {
-                *reinterpret_cast<float4 *>(dst) = make_float4(w[0], w[1], w[2], w[3]);
-            } else {
-                for (int j = 0; j < 4; ++j)
-                    if (cc + j < prm.n) dst[j] = w[j];
-            }
-        }
+    ptx::cluster_wait();
+    const float *const P = reinterpret_cast<const float *>(base_ptr);
+    switch (split) {
+        case 2: reduce_partial_tiles<BN, 2>(cluster, P, rank, r0, c0, prm); break;
+        case 4: reduce_partial_tiles<BN, 4>(cluster, P, rank, r0, c0, prm); break;
+        case 8: reduce_partial_tiles<BN, 8>(cluster, P, rank, r0, c0, prm); break;
+        default: reduce_partial_tiles<BN, 16>(cluster, P, rank, r0, c0, prm); break;
     }
-    cluster.sync();                                          // nobody leaves while a peer may still read its tile
 }
 
 
