@@ -369,6 +369,24 @@ def time_equation(mom, torch, eq, variant, steps, warmup, stream, timing=False, 
             run()
         b1.record(stream)
         stream.synchronize()
+        # short equations once more as a CUDA graph: one execute captured (the library's launches, its second stream and its
+        # events are capturable once the plan has run: every allocation happens in the first call) and replayed back to back
+        ms_graph = None
+        if quick:
+            try:
+                graph = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(graph, stream=stream):
+                    run()
+                graph.replay()
+                g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                g0.record(stream)
+                for _ in range(reps):
+                    graph.replay()
+                g1.record(stream)
+                stream.synchronize()
+                ms_graph = g0.elapsed_time(g1) / reps
+            except Exception:                # not capturable here: no figure
+                ms_graph = None
     ms = [e0.elapsed_time(e1) for e0, e1 in events]
     ms_b2b = b0.elapsed_time(b1) / reps
     status = plan.device_status()
@@ -376,7 +394,7 @@ def time_equation(mom, torch, eq, variant, steps, warmup, stream, timing=False, 
         raise RuntimeError(f"device-side wait timed out: {status}")
     mul, addf = plan.flops()
     stored_bytes = 4 * (sum(t.numel() for t in dchain if t is not None) + sum(t.numel() for t in dadd if t is not None) + plan.result_elements() * eq.batch)
-    return {"ms": ms, "ms_back_to_back": ms_b2b, "plan": plan, "stored_bytes": stored_bytes, "useful_flops": (mul + addf) * eq.batch, "launches": plan.last_launch_count(),
+    return {"ms": ms, "ms_back_to_back": ms_b2b, "ms_graph_replay": ms_graph, "plan": plan, "stored_bytes": stored_bytes, "useful_flops": (mul + addf) * eq.batch, "launches": plan.last_launch_count(),
             "step_times": step_times, "host": (chain, add), "keep": (dchain, dadd, out, ws)}
 
 
@@ -426,6 +444,7 @@ def run_gpu(args):
         r = time_equation(mom, torch, cfg, variant, steps=args.steps, warmup=args.warmup, stream=stream,
                           timing=getattr(cfg, "batch", 1) == 1 and not packed, chain_storage=storage)
         print(json.dumps({"workload": cfg.name, "variant": args.variant, "ms": r["ms"], "ms_back_to_back": r["ms_back_to_back"],
+                          "ms_graph_replay": r["ms_graph_replay"],
                           "useful_flops": r["useful_flops"],
                           "launches": r["launches"], "step_times_ms": r["step_times"][-1:] }))
         return
@@ -611,7 +630,7 @@ def run_gpu(args):
             ms_min, ms_med = min(r["ms"]), statistics.median(r["ms"])
             entry = {"workload": cfg.name, "parenthesization": r["plan"].parenthesization(),
                      "useful_flops": r["useful_flops"], "ms_min_of_20": ms_min, "ms_median": ms_med,
-                     "ms_back_to_back": r["ms_back_to_back"],
+                     "ms_back_to_back": r["ms_back_to_back"], "ms_graph_replay": r["ms_graph_replay"],
                      "gflops_back_to_back": r["useful_flops"] / (r["ms_back_to_back"] * 1e-3) / 1e9,
                      "gflops_at_min": r["useful_flops"] / (ms_min * 1e-3) / 1e9,
                      "gflops_at_median": r["useful_flops"] / (ms_med * 1e-3) / 1e9,

@@ -342,6 +342,10 @@ mom_status_t mom_plan_workspace_bytes(const mom_plan_t *plan, int64_t batch, siz
  *                duration of the enqueued work; may be NULL when that size is 0
  * The first execution of a plan on a device creates a small plan-owned device block (tile tables,
  * TMA descriptors, a status word) with cudaMalloc; later calls allocate nothing.
+ * CUDA graphs: after that first execution the call (and mom_equation_execute_batched) enqueues only kernel
+ * launches and, for plans that use their second stream, event records and waits; the caller may capture it on
+ * `stream` into a CUDA graph and replay the graph (same bits as the plain call).  The host-staging entry point and
+ * mom_product_3xtf32_noalloc are not covered by this statement.
  * Errors: INVALID_ARG, ALIGNMENT, WORKSPACE_TOO_SMALL, ARCH, ALLOC, CUDA. */
 mom_status_t mom_equation_execute(const mom_plan_t *plan, const float *const *chain_ptrs,
                                   const float *const *add_ptrs, float *out,
