@@ -16,6 +16,7 @@ struct DeviceInfo {
     bool tc_attr = false;            // dynamic shared-memory limit raised for the tensor-core kernels on this device
     bool pair_attr = false;
     bool inline64_attr = false, inline128_attr = false;
+    bool inline_variant_attr[2][2][2] = {}, inline_variant_np[2][2][2] = {};   // per kernel of the one-launch family: [128 columns][A transposed][B transposed]
     int inline_clusters[2][5] = {};  // co-resident clusters of the one-launch tcgen05 kernel, [128-column tiles][log2 cluster size]; 0: not asked, -1: unknown
     bool inline_pair_attr[2] = {false, false};
     int inline_pair_clusters[2] = {0, 0};   // co-resident CTA pairs of the one-launch kernel's pair variant, [128 columns per CTA]

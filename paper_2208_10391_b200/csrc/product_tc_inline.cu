@@ -95,17 +95,25 @@ __device__ __forceinline__ uint64_t kmajor_desc128(uint32_t tile, int kstep) {
 //      16-byte loads from the swizzled raw tile, two tcgen05.st of 16 columns (hi, lo).
 //   B: task t of the warp is (box j, group c) = columns 32 j + 4 c .. + 3 of k-row `lane`; value e of it lands in row
 //      n = 32 j + 4 c + e of the K-major tile, at k = lane (group lane / 4, word lane % 4).
-template <int NB>
+template <int NB, bool TA = false, bool TB = false>
 struct Transform {
     static constexpr int TASKS = NB / 4 / XFORM_WARPS;
     uint32_t a_src[4], src_off[TASKS], dst_off[TASKS][4];
+    uint32_t at_base, at_group;                              // TA: this thread's column of the raw boxes of A (stored k x m)
     __device__ __forceinline__ Transform(int w2, int lane) {
         const int arow = ((w2 + 2) & 3) * 32 + lane, ahalf = w2 >> 2;     // transform warp w2 is warp w2 + 2 of the CTA: lanes 32 (warp % 4) ..
 #pragma unroll
         for (int u = 0; u < 4; ++u) a_src[u] = arow * 128 + (((4 * ahalf + u) ^ (arow & 7)) << 4);
+        // TA: row arow of the tile is column `lane` of box (w2 + 2) % 4 (32 k-rows x 32 columns, 128-byte rows under the swizzle)
+        at_base = ((w2 + 2) & 3) * 4096 + ahalf * 16 * 128 + (lane & 3) * 4;
+        at_group = lane >> 2;
 #pragma unroll
         for (int t = 0; t < TASKS; ++t) {
             const int task = w2 + XFORM_WARPS * t, j = task >> 3, c = task & 7;
+            if (TB) {                                        // B stored n x k: the raw tile is K-major already; 16-byte groups stay where they are
+                src_off[t] = ((w2 * 32 + lane) + 32 * XFORM_WARPS * t) * 16;
+                continue;
+            }
             src_off[t] = j * 4096 + lane * 128 + ((c ^ (lane & 7)) << 4);
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
@@ -118,8 +126,16 @@ struct Transform {
     // bhi / blo: B's K-major tiles.  Ends with everything the MMA will read made visible to it.
     __device__ __forceinline__ void run(const uint8_t *araw, const uint8_t *braw, uint32_t a_tmem, uint8_t *bhi, uint8_t *blo) const {
         float4 av[4], bv[TASKS];
+        if (TA) {
+            float a16[16];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) av[u] = *reinterpret_cast<const float4 *>(araw + a_src[u]);
+            for (int u = 0; u < 16; ++u) a16[u] = *reinterpret_cast<const float *>(araw + at_base + u * 128 + ((at_group ^ (u & 7)) << 4));
+#pragma unroll
+            for (int u = 0; u < 4; ++u) av[u] = make_float4(a16[4 * u], a16[4 * u + 1], a16[4 * u + 2], a16[4 * u + 3]);
+        } else {
+#pragma unroll
+            for (int u = 0; u < 4; ++u) av[u] = *reinterpret_cast<const float4 *>(araw + a_src[u]);
+        }
 #pragma unroll
         for (int t = 0; t < TASKS; ++t) bv[t] = *reinterpret_cast<const float4 *>(braw + src_off[t]);
         {
@@ -140,6 +156,11 @@ struct Transform {
         for (int t = 0; t < TASKS; ++t) {
             float4 hi, lo;
             split4(bv[t], hi, lo);
+            if (TB) {
+                *reinterpret_cast<float4 *>(bhi + src_off[t]) = hi;
+                *reinterpret_cast<float4 *>(blo + src_off[t]) = lo;
+                continue;
+            }
             *reinterpret_cast<float *>(bhi + dst_off[t][0]) = hi.x; *reinterpret_cast<float *>(blo + dst_off[t][0]) = lo.x;
             *reinterpret_cast<float *>(bhi + dst_off[t][1]) = hi.y; *reinterpret_cast<float *>(blo + dst_off[t][1]) = lo.y;
             *reinterpret_cast<float *>(bhi + dst_off[t][2]) = hi.z; *reinterpret_cast<float *>(blo + dst_off[t][2]) = lo.z;
@@ -228,7 +249,8 @@ __device__ __forceinline__ void reduce_partial_tiles(cg::cluster_group &cluster,
     ptx::cluster_wait();
 }
 
-template <int BN>
+// TA / TB: the operand is stored transposed (A as k x m, B as n x k); the transform reads it accordingly, everything else is the same
+template <int BN, bool TA = false, bool TB = false>
 __global__ void __launch_bounds__(ITHREADS, 1)
 product_tc_inline_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const InlineParams prm) {
     using Cfg = InlineCfg<BN>;
@@ -294,8 +316,16 @@ product_tc_inline_kernel(const __grid_constant__ CUtensorMap map_a, const __grid
             __syncwarp();
             const int kb = klo + (kb0 + i) * IBK;
             const uint32_t st = base + s * Cfg::RAW_BYTES;
-            if (lane == 0) ptx::tma_load_2d(st, &map_a, kb, r0, raw_full(s));
-            else if (lane <= BN / 32) ptx::tma_load_2d(st + Cfg::A_BYTES + (lane - 1) * 4096, &map_b, c0 + 32 * (lane - 1), kb, raw_full(s));
+            // A as stored m x k: one box of 128 rows x 32 k; as k x m: four boxes of 32 k-rows x 32 columns (lanes 0..3).
+            // B as stored k x n: BN / 32 boxes of 32 k-rows x 32 columns; as n x k: one box of BN rows x 32 k (lanes 4..7).
+            if (lane < 4) {
+                if (!TA && lane == 0) ptx::tma_load_2d(st, &map_a, kb, r0, raw_full(s));
+                if (TA) ptx::tma_load_2d(st + lane * 4096, &map_a, r0 + 32 * lane, kb, raw_full(s));
+            } else if (lane < 8) {
+                const int j = lane - 4;
+                if (!TB && j < BN / 32) ptx::tma_load_2d(st + Cfg::A_BYTES + j * 4096, &map_b, c0 + 32 * j, kb, raw_full(s));
+                if (TB && j == 0) ptx::tma_load_2d(st + Cfg::A_BYTES, &map_b, kb, c0, raw_full(s));
+            }
         }
         if (*abort_flag && lane == 0) {          // failure path: loads still in flight land before the CTA's memory goes away
             const unsigned long long t0 = global_ns();
@@ -340,7 +370,7 @@ product_tc_inline_kernel(const __grid_constant__ CUtensorMap map_a, const __grid
     } else {
         // ------------------------------------------------------------------ transform (warps 2..9), then epilogue
         const int w2 = warp - 2;
-        const Transform<BN> xf(w2, lane);
+        const Transform<BN, TA, TB> xf(w2, lane);
         const uint32_t a_dst = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + BN + 16 * (w2 >> 2);
         bool ok = true;
         uint8_t *const split_ptr = base_ptr + R * Cfg::RAW_BYTES;
@@ -593,7 +623,8 @@ product_tc_inline_pair_kernel(const __grid_constant__ CUtensorMap map_a, const _
 
 bool product_tc_inline_takes(int64_t m, int64_t n, int64_t k, int lhs_transposed, int rhs_transposed, int pa, int pb) {
     auto plain = [](int p) { return p == MOM_GENERAL || p == MOM_LOWER_TRI || p == MOM_UPPER_TRI || p == MOM_SYMMETRIC; };
-    return !lhs_transposed && !rhs_transposed && (k & 3) == 0 && (n & 3) == 0 && plain(pa) && plain(pb) && m < (1 << 30) && n < (1 << 30) &&
+    // every matrix's row pitch is a multiple of 16 bytes: A is m x k, or k x m when stored transposed; B is k x n, or n x k; C is m x n
+    return (k & 3) == 0 && (n & 3) == 0 && (!lhs_transposed || (m & 3) == 0) && plain(pa) && plain(pb) && m < (1 << 30) && n < (1 << 30) &&
            k < (1 << 30);
 }
 
@@ -661,6 +692,7 @@ cudaError_t launch_product_tc_inline(const ProductArgs &a, int32_t *status, cuda
     // ones, so they never win.)
     int pair_bnh = 0;
     for (int bnh : {128}) {
+        if (a.transA || a.transB) break;                                       // the pair form reads its operands as stored only
         const long long pairs = (long long)((a.m + 2 * IBM - 1) / (2 * IBM)) * ((a.n + 2 * bnh - 1) / (2 * bnh));
         if (pairs * 2 > (1ll << 30)) continue;
         int fit = sm_count / 2;
@@ -697,8 +729,10 @@ cudaError_t launch_product_tc_inline(const ProductArgs &a, int32_t *status, cuda
     const long long tiles = pair_bnh ? (long long)((a.m + 2 * IBM - 1) / (2 * IBM)) * tiles_n : (long long)tiles_m * tiles_n;
 
     CUtensorMap map_a, map_b;
-    if (!tc_make_map(&map_a, a.A, a.m, a.k, IBM, IBK, CU_TENSOR_MAP_SWIZZLE_128B) ||
-        !tc_make_map(&map_b, a.B, a.k, a.n, IBK, 32, CU_TENSOR_MAP_SWIZZLE_128B))
+    if (!(a.transA ? tc_make_map(&map_a, a.A, a.k, a.m, IBK, 32, CU_TENSOR_MAP_SWIZZLE_128B)
+                   : tc_make_map(&map_a, a.A, a.m, a.k, IBM, IBK, CU_TENSOR_MAP_SWIZZLE_128B)) ||
+        !(a.transB ? tc_make_map(&map_b, a.B, a.n, a.k, bn, IBK, CU_TENSOR_MAP_SWIZZLE_128B)
+                   : tc_make_map(&map_b, a.B, a.k, a.n, IBK, 32, CU_TENSOR_MAP_SWIZZLE_128B)))
         return cudaErrorNotSupported;
     InlineParams prm;
     prm.m = a.m; prm.n = a.n; prm.k = a.k;
@@ -712,11 +746,28 @@ cudaError_t launch_product_tc_inline(const ProductArgs &a, int32_t *status, cuda
     if (pair_bnh == 128)
         return launch_dependent(product_tc_inline_pair_kernel<128>, dim3((unsigned)(tiles * 2)), dim3(ITHREADS), PairCfg<128>::SMEM_BYTES, stream, 2u,
                                 map_a, map_b, prm);
-    if (bn == 64)
-        return launch_dependent(product_tc_inline_kernel<64>, dim3((unsigned)(tiles * split)), dim3(ITHREADS), InlineCfg<64>::SMEM_BYTES, stream,
-                                (unsigned)split, map_a, map_b, prm);
-    return launch_dependent(product_tc_inline_kernel<128>, dim3((unsigned)(tiles * split)), dim3(ITHREADS), InlineCfg<128>::SMEM_BYTES, stream,
-                            (unsigned)split, map_a, map_b, prm);
+    // the kernel for this width and these storage orders; its shared-memory limit (and the cluster size beyond 8) is set per kernel
+    using Kernel = void (*)(CUtensorMap, CUtensorMap, InlineParams);
+    static const Kernel kernels[2][2][2] = {
+        {{product_tc_inline_kernel<64, false, false>, product_tc_inline_kernel<64, false, true>},
+         {product_tc_inline_kernel<64, true, false>, product_tc_inline_kernel<64, true, true>}},
+        {{product_tc_inline_kernel<128, false, false>, product_tc_inline_kernel<128, false, true>},
+         {product_tc_inline_kernel<128, true, false>, product_tc_inline_kernel<128, true, true>}}};
+    const int wide = bn == 128, ta = a.transA != 0, tb = a.transB != 0;
+    const Kernel kernel = kernels[wide][ta][tb];
+    const int smem = wide ? InlineCfg<128>::SMEM_BYTES : InlineCfg<64>::SMEM_BYTES;
+    {
+        std::lock_guard<std::mutex> lock(device_info_mutex());
+        DeviceInfo *info = current_device_info();
+        if (!info) return cudaErrorInvalidDevice;
+        cudaError_t e = raise_smem_limit_locked(kernel, smem, &info->inline_variant_attr[wide][ta][tb]);
+        if (e == cudaSuccess && split > 8 && !info->inline_variant_np[wide][ta][tb]) {
+            e = cudaFuncSetAttribute(kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+            if (e == cudaSuccess) info->inline_variant_np[wide][ta][tb] = true;
+        }
+        if (e != cudaSuccess) return e;
+    }
+    return launch_dependent(kernel, dim3((unsigned)(tiles * split)), dim3(ITHREADS), (size_t)smem, stream, (unsigned)split, map_a, map_b, prm);
 }
 
 }  // namespace mom

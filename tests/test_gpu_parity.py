@@ -504,3 +504,28 @@ def test_config_transposed_full_size_sampled_rows():
     x, plan, (chain, add) = run_equation(eq, mom.VARIANT_3XTF32)
     assert plan.parenthesization() == "(0^T*(1*(2^T*3)))"
     check_against_oracle(eq, x, plan, chain, add, rows=stratified_rows(4096, 6))
+
+
+INLINE_TRANSPOSED = [
+    # (m, k, n, left property as used, right property as used, A stored transposed, B stored transposed, Add terms)
+    (640, 640, 640, G, G, True, False, 0), (640, 640, 640, G, G, False, True, 1), (640, 640, 640, G, G, True, True, 0),
+    (900, 1200, 100, G, G, False, True, 0), (256, 2048, 64, G, G, True, False, 1), (520, 520, 392, U, G, True, False, 0),
+    (392, 520, 520, G, L, False, True, 1), (392, 392, 392, U, L, True, True, 0), (1024, 1024, 1024, G, G, True, True, 1),
+    (100, 36, 100, G, G, True, True, 0), (1000, 260, 76, G, G, True, False, 0),
+]
+
+
+@pytest.mark.parametrize("m,k,n,pa,pb,ta,tb,terms", INLINE_TRANSPOSED)
+def test_inline_kernel_reads_transposed_operands_as_stored(m, k, n, pa, pb, ta, tb, terms):
+    # A stored k x m and / or B stored n x k: the one-launch tcgen05 kernel loads the stored tiles and its transform warps read
+    # them the other way round (A: a thread gathers its row from a column of the raw boxes; B: the raw tile is K-major already)
+    flip = {L: U, U: L, G: G}
+    dist = lambda p: "uniform" if p != G else "normal"
+    a_op = Operand(k, m, flip[pa], dist(pa), 1.0 / np.sqrt(k)) if ta else Operand(m, k, pa, dist(pa), 1.0 / np.sqrt(k))
+    b_op = Operand(n, k, flip[pb], dist(pb)) if tb else Operand(k, n, pb, dist(pb))
+    add = (Operand(m, n, G, "normal"),) * terms
+    eq = Equation(f"inline_t_{m}x{k}x{n}_{pa}{pb}_{int(ta)}{int(tb)}", 76, (a_op, b_op), add, chain_t=(ta, tb), add_t=(False,) * terms)
+    x, plan, (chain, terms_h) = run_equation(eq, mom.VARIANT_3XTF32_INLINE)
+    assert plan.step(0).uses_tensor_cores == 3 and plan.last_launch_count() == 1
+    assert plan.step(0).lhs_property == pa and plan.step(0).rhs_property == pb
+    check_against_oracle(eq, x, plan, chain, terms_h)

@@ -504,8 +504,9 @@ def test_kernel_choice_of_the_default_variant():
     assert kind(2048, 512, 2048) == 3                        # 256 tiles of 128 x 128, but one wave of CTA pairs
     assert kind(900, 1200, 100) == 3 and kind(256, 2048, 64) == 2 and kind(128, 4096, 128) == 2       # small work; a result of one tile
     assert kind(512, 512, 510) == 2                        # rows TMA cannot address
-    assert kind(640, 640, 640, (True, False)) == 2 and kind(640, 640, 640, (False, True)) == 2     # transposed operands
-    assert kind(1024, 1024, 1024, (True, False)) == 1      # the plane kernel reads transposed operands through its split pass
+    assert kind(640, 640, 640, (True, False)) == 3 and kind(640, 640, 640, (False, True)) == 3     # transposed operands are read as stored
+    assert kind(642, 640, 640, (True, False)) == 2         # ... when their rows are 16-byte addressable (A stored 640 x 642)
+    assert kind(1024, 1024, 1024, (True, False)) == 3 and kind(2560, 2560, 2560, (True, False)) == 1   # the plane kernel reads them through its split pass
 
 
 def test_independent_subtrees_of_small_products_are_marked_to_run_side_by_side():
