@@ -101,8 +101,9 @@ typedef enum { MOM_F32 = 0 } mom_dtype_t;
  *       accumulating lo*hi + hi*lo + hi*hi in f32 (f32-level accuracy).  Three kernels, chosen by size:
  *       large products (m*n*k >= 6 * 2^26 that the kernel below does not take) whose leading
  *       dimensions TMA can address (multiples of 4 elements) run on the tcgen05 kernel that takes its operands as
- *       hi / lo planes (a pre-pass writes them; TMA, tensor memory, persistent CTAs); products of stored
- *       (untransposed) operands with a result of at least 65536 entries and 6 * 10^7 <= m*n*k < 10^9, or
+ *       hi / lo planes (a pre-pass writes them; TMA, tensor memory, persistent CTAs); products of operands
+ *       whose stored rows are 16-byte addressable (transposed ones included) with a result of at least
+ *       65536 entries and 6 * 10^7 <= m*n*k < 10^9, or
  *       m*n*k < 4 * 10^9 with at most 148 result tiles of 128 x 128, or (an equation of one product only)
  *       m*n*k < 10^10 with at most 74 result tiles of 256 x 256 (CTA pairs), run on the tcgen05 kernel that reads the
  *       operands as stored and splits them on the way into shared and tensor memory (one launch); everything

@@ -24,6 +24,8 @@
 // The tile's structural k-range bounds the contraction as everywhere else.  Shared memory still moves more bytes per
 // flop than in the plane kernel (the transform reads every operand byte and writes B once more), so this kernel tops out
 // near half of the tensor peak; it is chosen where launches, not flops, are the cost.
+// Operands stored transposed are read as stored: A as k x m arrives as four boxes of 32 k-rows x 32 columns and a transform thread
+// gathers its row from a column of them; B as n x k is K-major already and is split where it lies.
 // Every wait is bounded; a CTA that gives up still meets its cluster at both cluster barriers.
 #include <algorithm>
 #include <cstring>
