@@ -562,7 +562,8 @@ static mom_status_t plan_sums(const std::vector<mom_matrix_desc_t> &slots, const
             const bool large = (double)m * (double)n * (double)k >= 6.0 * (double)(1 << 26);
             // in between: the tcgen05 kernel that reads the operands as stored and splits them in shared memory (one launch);
             // it takes operands (transposed ones as stored) whose rows TMA can address
-            const bool inline_ok = st.pub.kind != MOM_KIND_GRAM &&
+            // (a Gram product Y * Y^T goes there only below the plane kernel's range: that one computes half of the tiles and mirrors them)
+            const bool inline_ok = (st.pub.kind != MOM_KIND_GRAM || !large) &&
                                    mom::product_tc_inline_takes(m, n, k, st.pub.lhs_transposed, st.pub.rhs_transposed,
                                                                 mom::kernel_property(st.pub.lhs_property), mom::kernel_property(st.pub.rhs_property));
             // ... and it pays between the two (measured, see the constants): from about 400^3 on it beats the warp-level kernel, and
